@@ -1,0 +1,260 @@
+/*
+ * libpask -- the online hot path of PASK (parser-aware structural KV persistence) for B200.
+ *
+ * Each token arrives with a parser-derived structural tag.  A frozen, offline-calibrated table
+ * maps (tag, layer group) to RELEASE (drop), RETAIN-LOW or RETAIN-HIGH; that decision is applied
+ * to the token's K/V at every layer, the result is compacted into a paged mixed-precision
+ * cache with a constant-size budget state per sequence, and decode attention runs over what was
+ * retained.  This header is the whole boundary: plain C, plain pointers and sizes.
+ *
+ * Conventions
+ *   - "dev" pointers are CUDA device memory, "host" pointers ordinary host memory.
+ *   - The caller owns every device buffer and the stream.  The library allocates no device
+ *     memory and owns only its small host-side handles.
+ *   - Kernels are enqueued on the given stream and calls return without waiting unless stated
+ *     otherwise.  Errors that the host can see (bad arguments, shapes, sizes) are returned at
+ *     once and enqueue nothing.  Conditions only the device can see (pool exhaustion, unknown
+ *     tags, page-table overflow, a wait that ran out) set sticky bits in a device status word
+ *     that pask_budget_state reports; an append that cannot get all its pages writes nothing
+ *     and changes no counter.
+ *   - Every dev pointer must be 16-byte aligned; the pools and meta 256-byte aligned.
+ *   - One host thread drives a cache at a time; ordering between calls is stream order.
+ *   - Supported shapes: head_dim 128, 16-token pages, n_q_heads = 4 * n_kv_heads with
+ *     n_kv_heads in {1, 2, 4, 8}.  Anything else: PASK_ERR_UNSUPPORTED_SHAPE.
+ *   - No function throws or aborts.
+ *
+ * Formats (the paper leaves them open; these are the library's documented readings)
+ *   RETAIN-HIGH keeps the token's bf16 K and V bits.  RETAIN-LOW stores, per token, per KV head
+ *   and per group of 32 consecutive head dimensions, one fp16 scale s = fp16(amax / 7) (IEEE
+ *   fp32 division, round to nearest even, saturating at 65504) and 32 four-bit codes
+ *   clamp(rint(x * (1 / s)), -7, 7) + 8; the value read back is (code - 8) * s.  s == 0 gives
+ *   codes 8.  Costs are payload bytes per token per layer: m(R) = 0,
+ *   m(L) = 2 * n_kv * (64 + 8), m(H) = 2 * n_kv * 256.
+ */
+#ifndef PASK_H_
+#define PASK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t pask_status_t;
+#define PASK_OK 0
+#define PASK_ERR_INVALID_ARG (-1)
+#define PASK_ERR_BAD_POLICY (-2)
+#define PASK_ERR_UNSUPPORTED_SHAPE (-3)
+#define PASK_ERR_POOL_EXHAUSTED (-4)
+#define PASK_ERR_BAD_SEQ (-5)
+#define PASK_ERR_CUDA (-6)
+#define PASK_ERR_TIMEOUT (-7)
+#define PASK_ERR_WORKSPACE (-8)
+
+/* Sticky bits of the device status word (pask_budget_state_t.device_status). */
+#define PASK_DEV_POOL_EXHAUSTED 0x1u  /* an append needed more pages than a pool had: nothing written */
+#define PASK_DEV_BAD_SEQ 0x2u         /* sequence id out of range or repeated within one call */
+#define PASK_DEV_SEQ_OVERFLOW 0x4u    /* a stream would exceed max_tokens_per_seq: nothing written */
+#define PASK_DEV_BAD_RAGGED 0x8u      /* cu_tokens not ascending or not ending at total_tokens */
+#define PASK_DEV_TIMEOUT 0x10u        /* a bounded wait inside a kernel ran out; results invalid */
+
+#define PASK_ACTION_RELEASE 0
+#define PASK_ACTION_RETAIN_LOW 1
+#define PASK_ACTION_RETAIN_HIGH 2
+#define PASK_TAG_PROTECTED 0xFF /* always RETAIN-HIGH, not counted as unknown */
+#define PASK_MAX_GROUPS 8
+#define PASK_MAX_SEQS_PER_CALL 1024
+
+typedef struct pask_policy pask_policy_t;
+typedef struct pask_cache pask_cache_t;
+typedef void *pask_stream_t; /* a cudaStream_t */
+typedef void *pask_event_t;  /* a cudaEvent_t */
+
+typedef struct {
+    int32_t n_layers;
+    int32_t n_q_heads;
+    int32_t n_kv_heads;
+    int32_t head_dim;           /* 128 */
+    int32_t page_tokens;        /* 16 */
+    int32_t max_seqs;           /* sequence ids are 0 .. max_seqs-1 */
+    int32_t max_tokens_per_seq; /* bound on each stream's length (sizes the page tables) */
+    int32_t max_append_tokens;  /* largest total_tokens of one pask_append_kv call */
+    uint32_t pool_high_pages;   /* capacity of the bf16 page pool, shared by all layers */
+    uint32_t pool_low_pages;    /* capacity of the int4 page pool */
+} pask_cache_desc_t;
+
+typedef struct {
+    size_t pool_high_bytes; /* pool_high_pages * high_page_bytes */
+    size_t pool_low_bytes;
+    size_t meta_bytes;      /* counters, page tables, budget states, free stacks, append scratch */
+    size_t high_page_bytes; /* n_kv * 8192: per KV head a 16x128 bf16 K tile then V tile */
+    size_t low_page_bytes;  /* n_kv * 2304: per KV head K codes, K scales, V codes, V scales */
+} pask_cache_sizes_t;
+
+/* Constant-size per-sequence budget state (Algorithm 2's R_t with the counts it is made of).
+ * Counts are token-layer events: one per token per layer call, binned by the layer's group. */
+typedef struct {
+    uint64_t n_seen[PASK_MAX_GROUPS];
+    uint64_t n_high[PASK_MAX_GROUPS];
+    uint64_t n_low[PASK_MAX_GROUPS];
+    uint64_t n_drop[PASK_MAX_GROUPS];
+    uint64_t retained_bytes;  /* sum of m(a) over everything persisted so far */
+    uint64_t full_bytes;      /* sum of m(H): what full high precision would have cost */
+    int64_t remaining_bytes;  /* floor(budget_target * full_bytes) - retained_bytes */
+    uint64_t bad_tags;        /* tags >= n_tags (kept at high precision) */
+    uint32_t pages_high;      /* pages this sequence holds in each pool */
+    uint32_t pages_low;
+    uint32_t device_status;   /* PASK_DEV_* bits, cache-wide, sticky until pask_cache_reset */
+    uint32_t reserved;
+} pask_budget_state_t;
+
+/* ---------------------------------------------------------------------------------------------
+ * pask_load_policy -- load the frozen table Lambda and the reserve Gamma.
+ * Follows: the table stores, per bucket q = (tag, layer group), the selected action, the
+ * calibrated floor and the adjacent upgrade scores (end of Section 3.3); online the action is
+ * a = max(a0, a_floor) under R < L < H (Eq. 10, Algorithm 2 steps 1-2).  Gamma is Eq. 9's
+ * per-state reserve, carried but not read by the calls below.
+ *   blob (host, len bytes), little endian:
+ *     "PASK", u32 version=1, u32 n_tags (1..255), u32 n_groups (1..8), u32 n_layers, u32 n_states,
+ *     u32 budget_target_q16, u32 recent_window (must be 0), u32 low_bits (4), u32 group_size (32),
+ *     u8 layer_group[n_layers] zero-padded to 4 bytes,
+ *     n_tags*n_groups entries, tag-major: u8 a0, u8 a_floor, u16 0, f32 rho_RL, f32 rho_LH,
+ *     u32 gamma[n_states].
+ * The blob is copied; *out is a host handle to free with pask_free_policy.  Needs no GPU.
+ * Errors: PASK_ERR_INVALID_ARG (null), PASK_ERR_BAD_POLICY (magic, version, sizes, ranges, length).
+ */
+pask_status_t pask_load_policy(const void *blob, size_t len, pask_policy_t **out);
+void pask_free_policy(pask_policy_t *policy);
+/* Effective action max(a0, a_floor) for a bucket, or -1 if out of range.  Host only. */
+int32_t pask_policy_action(const pask_policy_t *policy, int32_t tag, int32_t group);
+
+/* Bytes the caller must allocate for a cache of this shape.  Host only, needs no GPU. */
+pask_status_t pask_cache_sizes(const pask_cache_desc_t *desc, pask_cache_sizes_t *out);
+
+/* Bind caller-owned device memory (sizes from pask_cache_sizes) to a new cache and initialise
+ * it on `stream` (copies the folded table into meta, zeroes counters).  The policy's n_layers
+ * must equal desc->n_layers.  The handle is host memory; destroy frees only that. */
+pask_status_t pask_cache_create(const pask_cache_desc_t *desc, const pask_policy_t *policy, void *pool_high_dev,
+                                void *pool_low_dev, void *meta_dev, pask_stream_t stream, pask_cache_t **out);
+void pask_cache_destroy(pask_cache_t *cache);
+/* Forget every sequence, return all pages, clear the device status word. */
+pask_status_t pask_cache_reset(pask_cache_t *cache, pask_stream_t stream);
+/* Forget one sequence.  Its pages go back on the free stacks in a fixed order (layers
+ * ascending; per layer the HIGH table then the LOW table, each in table order) and are handed
+ * out again last-in first-out. */
+pask_status_t pask_seq_reset(pask_cache_t *cache, int32_t seq, pask_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * pask_append_kv -- Algorithm 2 steps 1, 2, 7 and 8 for one layer and a ragged batch of tokens:
+ * look up each token's bucket (its tag, this layer's group), take a = max(a0, a_floor), persist
+ * the token's K/V accordingly (nothing, int4 + scales, or the bf16 bits) at the end of the
+ * sequence's LOW or HIGH stream, and charge m(a) to the sequence's budget state.  The call
+ * takes no query and no attention statistics: the online path may use only the tag, the layer
+ * group and the constant-size budget state (Section 3.1, Section 3.4).
+ *   layer          0 .. n_layers-1
+ *   n_seqs         sequences in this call (1 .. PASK_MAX_SEQS_PER_CALL), each id at most once
+ *   total_tokens   sum of the per-sequence token counts (<= max_append_tokens)
+ *   seq_ids        dev int32 [n_seqs]
+ *   cu_tokens      dev int32 [n_seqs+1], ascending, cu_tokens[0] = 0, last = total_tokens
+ *                  (one token per sequence in decode, many in prefill)
+ *   k, v           dev bf16 [total_tokens][n_kv][128], post-RoPE, tokens of a sequence in order
+ *   tags           dev uint8 [total_tokens]; PASK_TAG_PROTECTED = always high; >= n_tags = high
+ *                  and counted in bad_tags
+ *   states         dev uint16 [total_tokens] parser-state ids or NULL (reserved; not read)
+ *   actions_out    dev uint8 [total_tokens] or NULL: the action taken for each token
+ * New pages are numbered in call order (sequence-major, position ascending) from each pool's
+ * free stack, else its bump counter.  If either pool cannot supply the whole call, or a stream
+ * would outgrow its page table, nothing is written and no counter changes; the condition is a
+ * sticky PASK_DEV_* bit.
+ */
+pask_status_t pask_append_kv(pask_cache_t *cache, int32_t layer, int32_t n_seqs, int32_t total_tokens,
+                             const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
+                             const uint8_t *tags, const uint16_t *states, uint8_t *actions_out,
+                             pask_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * pask_decode_attention -- attention of one new query per sequence over that sequence's
+ * retained history at `layer`, at stored precision: out = softmax(q k^T / sqrt(128)) v over
+ * the HIGH stream (bf16 values) and the LOW stream ((code - 8) * scale); released tokens take no
+ * part (Section 3.1: release removes a KV state from future attention; these are the attention
+ * outputs o of Eq. 4).  Query head h reads KV head h / 4.
+ *   seq_ids   dev int32 [n_seqs]
+ *   q         dev bf16 [n_seqs][n_q][128]
+ *   out       dev fp32 [n_seqs][n_q][128]
+ *   lse       dev fp32 [n_seqs][n_q] or NULL: natural-log sum of exp of the scaled scores
+ *   workspace dev, at least pask_workspace_bytes(cache, n_seqs) bytes, 256-byte aligned; holds
+ *             split partials between the two kernels of the call, contents undefined afterwards
+ * A sequence with nothing retained gets out = 0 and lse = -inf.
+ * Errors: PASK_ERR_INVALID_ARG, PASK_ERR_WORKSPACE (too small), PASK_ERR_CUDA (launch failed).
+ */
+pask_status_t pask_decode_attention(pask_cache_t *cache, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                    const void *q, float *out, float *lse, void *workspace,
+                                    size_t workspace_bytes, pask_stream_t stream);
+/* The full high-precision reference (the paper's "Full KV", C_KV = 1): same arguments, for a
+ * cache whose policy keeps everything at high precision; the LOW stream is not read at all
+ * (its code path is compiled out), so any LOW tokens present would be ignored. */
+pask_status_t pask_decode_attention_full(pask_cache_t *cache, int32_t layer, int32_t n_seqs,
+                                         const int32_t *seq_ids, const void *q, float *out, float *lse,
+                                         void *workspace, size_t workspace_bytes, pask_stream_t stream);
+size_t pask_workspace_bytes(const pask_cache_t *cache, int32_t n_seqs);
+
+/* One decode step of one layer from HOST buffers: copies seq_ids, the new token's k, v, tag and
+ * the query to the device (into `staging`), appends one token per sequence, runs decode
+ * attention and copies `out` back -- all enqueued on `stream`; the host buffers must stay valid
+ * (and should be pinned) until the stream has drained.
+ *   seq_ids_host int32 [n_seqs]; k_host, v_host bf16 [n_seqs][n_kv][128]; tags_host u8 [n_seqs];
+ *   q_host bf16 [n_seqs][n_q][128]; out_host fp32 [n_seqs][n_q][128];
+ *   staging dev, >= pask_step_staging_bytes(cache, n_seqs), 256-byte aligned. */
+pask_status_t pask_decode_step_host(pask_cache_t *cache, int32_t layer, int32_t n_seqs, const int32_t *seq_ids_host,
+                                    const void *k_host, const void *v_host, const uint8_t *tags_host,
+                                    const void *q_host, float *out_host, void *staging, size_t staging_bytes,
+                                    void *workspace, size_t workspace_bytes, pask_stream_t stream);
+size_t pask_step_staging_bytes(const pask_cache_t *cache, int32_t n_seqs);
+
+/* ---------------------------------------------------------------------------------------------
+ * pask_budget_state -- the constant-size budget state of one sequence (Algorithm 2 step 8:
+ * R' = R - sum_c m(a_c, c); normalised cost of Eq. 1 is retained_bytes / full_bytes) plus the
+ * cache-wide device status word.  Copies to host memory and WAITS for `stream`. */
+pask_status_t pask_budget_state(pask_cache_t *cache, int32_t seq, pask_budget_state_t *host_out,
+                                pask_stream_t stream);
+
+/* Optional timing hook: the next pask_decode_attention[_full] call records `start` just before
+ * and `stop` just after its main (page-streaming) kernel on the call's stream, then forgets
+ * them.  Pass NULLs to clear. */
+pask_status_t pask_cache_set_timing_events(pask_cache_t *cache, pask_event_t start, pask_event_t stop);
+
+/* ---------------------------------------------------------------------------------------------
+ * Debug / test access to the cache in canonical form (the physical packing inside pages is
+ * private).  All of these wait for `stream` and write HOST memory.
+ */
+pask_status_t pask_debug_stream_len(pask_cache_t *cache, int32_t layer, int32_t seq, uint32_t *n_high,
+                                    uint32_t *n_low, pask_stream_t stream);
+/* HIGH stream in arrival order: k_out, v_out bf16 bits [n_high][n_kv][128]; pages_out [ceil(n_high/16)]. */
+pask_status_t pask_debug_dump_high(pask_cache_t *cache, int32_t layer, int32_t seq, uint16_t *k_out,
+                                   uint16_t *v_out, uint32_t *pages_out, pask_stream_t stream);
+/* LOW stream in arrival order: codes u8 [n_low][n_kv][128] (values 1..15), fp16 scale bits
+ * [n_low][n_kv][4]; pages_out [ceil(n_low/16)]. */
+pask_status_t pask_debug_dump_low(pask_cache_t *cache, int32_t layer, int32_t seq, uint8_t *k_codes,
+                                  uint16_t *k_scales, uint8_t *v_codes, uint16_t *v_scales, uint32_t *pages_out,
+                                  pask_stream_t stream);
+/* out[4] = { high bump counter, high free-stack depth, low bump counter, low free-stack depth }. */
+pask_status_t pask_debug_pool_state(pask_cache_t *cache, uint32_t *out4, pask_stream_t stream);
+/* How the decode-attention kernel splits work: for a batch whose sequences hold the given page
+ * counts, and a grid of `n_ctas`, writes for each CTA b and sequence index s the half-open range
+ * of concatenated page indices (HIGH pages first, then LOW) that b processes for s, as
+ * ranges[(b * n_seqs + s) * 2 + {0,1}] (empty ranges have begin == end).  Host only, no GPU. */
+pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, const uint32_t *pages_low,
+                                   int32_t n_ctas, uint32_t *ranges);
+
+/* Override the number of CTAs the decode-attention main kernel is launched with (default: two per
+ * SM).  Any value >= 1 gives the same result up to summation order; tests use it to check that.
+ * Workspaces must be sized (pask_workspace_bytes) after the change. */
+pask_status_t pask_debug_set_attention_ctas(pask_cache_t *cache, int32_t n_ctas);
+
+const char *pask_status_string(pask_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PASK_H_ */

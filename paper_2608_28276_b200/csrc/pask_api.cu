@@ -1,0 +1,474 @@
+// Host side of libpask: policy blobs, cache set-up, budget state, canonical dumps.
+#include <cstring>
+#include <new>
+
+#include "pask_internal.h"
+
+using namespace pask;
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+uint32_t rd32(const uint8_t *p) {
+    return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24);
+}
+
+bool shape_ok(const pask_cache_desc_t *d) {
+    if (d->head_dim != kHeadDim || d->page_tokens != kPageTokens) return false;
+    const int kv = d->n_kv_heads;
+    if (!(kv == 1 || kv == 2 || kv == 4 || kv == 8)) return false;
+    return d->n_q_heads == 4 * kv;
+}
+
+MetaOffsets meta_offsets(const pask_cache_desc_t *d, int n_tags, int n_groups) {
+    MetaOffsets o{};
+    const size_t max_pages = (size_t)(d->max_tokens_per_seq + kPageTokens - 1) / kPageTokens;
+    const size_t sl = (size_t)d->max_seqs * d->n_layers;
+    size_t p = 0;
+    auto take = [&](size_t bytes) { size_t at = p; p = align_up(p + bytes, 256); return at; };
+    o.ctrl = take(kCtrlWords * 4);
+    o.free_high = take((size_t)d->pool_high_pages * 4);
+    o.free_low = take((size_t)d->pool_low_pages * 4);
+    o.zero_begin = p;
+    o.n_high = take(sl * 4);
+    o.n_low = take(sl * 4);
+    o.tbl_high = take(sl * max_pages * 4);
+    o.tbl_low = take(sl * max_pages * 4);
+    o.budget = take((size_t)d->max_seqs * sizeof(pask_budget_state_t));
+    o.seq_mark = take((size_t)d->max_seqs * 4);
+    o.zero_end = p;
+    o.plan = take((size_t)PASK_MAX_SEQS_PER_CALL * sizeof(AppendPlan));
+    o.tok_scratch = take((size_t)d->max_append_tokens * sizeof(uint2));
+    o.lut = take((size_t)n_tags * n_groups);
+    o.layer_group = take((size_t)d->n_layers);
+    o.total = p;
+    return o;
+}
+
+bool desc_ok(const pask_cache_desc_t *d) {
+    return d->n_layers > 0 && d->n_layers <= 4096 && d->max_seqs > 0 && d->max_tokens_per_seq > 0 &&
+           d->max_append_tokens > 0;
+}
+
+pask_status_t cuda_rc(cudaError_t e) { return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA; }
+
+// read n_high / n_low of (seq, layer) after draining the stream
+pask_status_t read_lens(pask_cache *c, int layer, int seq, uint32_t *nh, uint32_t *nl, cudaStream_t s) {
+    if (cudaStreamSynchronize(s) != cudaSuccess) return PASK_ERR_CUDA;
+    const size_t i = (size_t)seq * c->desc.n_layers + layer;
+    if (cudaMemcpy(nh, c->dev.n_high + i, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PASK_ERR_CUDA;
+    if (cudaMemcpy(nl, c->dev.n_low + i, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PASK_ERR_CUDA;
+    return PASK_OK;
+}
+
+bool seq_layer_ok(const pask_cache *c, int layer, int seq) {
+    return layer >= 0 && layer < c->desc.n_layers && seq >= 0 && seq < c->desc.max_seqs;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *pask_status_string(pask_status_t s) {
+    switch (s) {
+        case PASK_OK: return "ok";
+        case PASK_ERR_INVALID_ARG: return "invalid argument";
+        case PASK_ERR_BAD_POLICY: return "malformed policy blob";
+        case PASK_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case PASK_ERR_POOL_EXHAUSTED: return "page pool exhausted";
+        case PASK_ERR_BAD_SEQ: return "bad sequence id";
+        case PASK_ERR_CUDA: return "CUDA runtime error";
+        case PASK_ERR_TIMEOUT: return "device wait timed out";
+        case PASK_ERR_WORKSPACE: return "workspace too small";
+        default: return "unknown status";
+    }
+}
+
+pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **out) {
+    if (!blob_v || !out) return PASK_ERR_INVALID_ARG;
+    *out = nullptr;
+    const uint8_t *blob = static_cast<const uint8_t *>(blob_v);
+    if (len < 40 || std::memcmp(blob, "PASK", 4) != 0 || rd32(blob + 4) != 1) return PASK_ERR_BAD_POLICY;
+    pask_policy *p = new (std::nothrow) pask_policy();
+    if (!p) return PASK_ERR_INVALID_ARG;
+    p->n_tags = rd32(blob + 8);
+    p->n_groups = rd32(blob + 12);
+    p->n_layers = rd32(blob + 16);
+    p->n_states = rd32(blob + 20);
+    p->budget_q16 = rd32(blob + 24);
+    const uint32_t window = rd32(blob + 28), low_bits = rd32(blob + 32), group_size = rd32(blob + 36);
+    bool ok = p->n_tags >= 1 && p->n_tags <= 255 && p->n_groups >= 1 && p->n_groups <= PASK_MAX_GROUPS &&
+              p->n_layers >= 1 && p->n_layers <= 4096 && p->n_states <= (1u << 20) && window == 0 && low_bits == 4 &&
+              group_size == (uint32_t)kQGroup;
+    const size_t lg_pad = ok ? align_up(p->n_layers, 4) : 0;
+    const size_t n_ent = ok ? (size_t)p->n_tags * p->n_groups : 0;
+    ok = ok && len == 40 + lg_pad + n_ent * 12 + (size_t)p->n_states * 4;
+    if (ok) {
+        p->layer_group.assign(blob + 40, blob + 40 + p->n_layers);
+        for (uint8_t g : p->layer_group) ok = ok && g < p->n_groups;
+        const uint8_t *e = blob + 40 + lg_pad;
+        p->a0.resize(n_ent); p->a_floor.resize(n_ent); p->eff.resize(n_ent);
+        p->rho_rl.resize(n_ent); p->rho_lh.resize(n_ent);
+        for (size_t i = 0; i < n_ent; i++, e += 12) {
+            p->a0[i] = e[0];
+            p->a_floor[i] = e[1];
+            ok = ok && e[0] <= PASK_ACTION_RETAIN_HIGH && e[1] <= PASK_ACTION_RETAIN_HIGH && e[2] == 0 && e[3] == 0;
+            std::memcpy(&p->rho_rl[i], e + 4, 4);
+            std::memcpy(&p->rho_lh[i], e + 8, 4);
+            p->eff[i] = e[0] > e[1] ? e[0] : e[1];  // floors take priority: a = max(a0, a_floor)
+        }
+        p->gamma.resize(p->n_states);
+        for (uint32_t s = 0; s < p->n_states; s++, e += 4) p->gamma[s] = rd32(e);
+    }
+    if (!ok) { delete p; return PASK_ERR_BAD_POLICY; }
+    *out = p;
+    return PASK_OK;
+}
+
+void pask_free_policy(pask_policy_t *p) { delete p; }
+
+int32_t pask_policy_action(const pask_policy_t *p, int32_t tag, int32_t group) {
+    if (!p || tag < 0 || (uint32_t)tag >= p->n_tags || group < 0 || (uint32_t)group >= p->n_groups) return -1;
+    return p->eff[(size_t)tag * p->n_groups + group];
+}
+
+pask_status_t pask_cache_sizes(const pask_cache_desc_t *d, pask_cache_sizes_t *out) {
+    if (!d || !out) return PASK_ERR_INVALID_ARG;
+    if (!shape_ok(d)) return PASK_ERR_UNSUPPORTED_SHAPE;
+    if (!desc_ok(d)) return PASK_ERR_INVALID_ARG;
+    out->high_page_bytes = (size_t)d->n_kv_heads * kHighHeadBytes;
+    out->low_page_bytes = (size_t)d->n_kv_heads * kLowHeadBytes;
+    out->pool_high_bytes = out->high_page_bytes * d->pool_high_pages;
+    out->pool_low_bytes = out->low_page_bytes * d->pool_low_pages;
+    out->meta_bytes = meta_offsets(d, 255, PASK_MAX_GROUPS).total;  // independent of the policy loaded later
+    return PASK_OK;
+}
+
+pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t *pol, void *pool_high, void *pool_low,
+                                void *meta, pask_stream_t stream_v, pask_cache_t **out) {
+    if (!d || !pol || !meta || !out) return PASK_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!shape_ok(d)) return PASK_ERR_UNSUPPORTED_SHAPE;
+    if (!desc_ok(d) || (uint32_t)d->n_layers != pol->n_layers) return PASK_ERR_INVALID_ARG;
+    if ((d->pool_high_pages && !pool_high) || (d->pool_low_pages && !pool_low)) return PASK_ERR_INVALID_ARG;
+    if (((uintptr_t)pool_high | (uintptr_t)pool_low | (uintptr_t)meta) & 255) return PASK_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev_id = 0, sms = 0;
+    if (cudaGetDevice(&dev_id) != cudaSuccess) return PASK_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_id) != cudaSuccess) return PASK_ERR_CUDA;
+    pask_cache *c = new (std::nothrow) pask_cache();
+    if (!c) return PASK_ERR_INVALID_ARG;
+    c->desc = *d;
+    c->meta = meta;
+    c->append_serial = 0;
+    c->sm_count = sms;
+    c->ev_start = c->ev_stop = nullptr;
+    c->off = meta_offsets(d, 255, PASK_MAX_GROUPS);
+    uint8_t *m = static_cast<uint8_t *>(meta);
+    DevCache &v = c->dev;
+    v.pool_high = static_cast<uint8_t *>(pool_high);
+    v.pool_low = static_cast<uint8_t *>(pool_low);
+    v.ctrl = reinterpret_cast<uint32_t *>(m + c->off.ctrl);
+    v.free_high = reinterpret_cast<uint32_t *>(m + c->off.free_high);
+    v.free_low = reinterpret_cast<uint32_t *>(m + c->off.free_low);
+    v.n_high = reinterpret_cast<uint32_t *>(m + c->off.n_high);
+    v.n_low = reinterpret_cast<uint32_t *>(m + c->off.n_low);
+    v.tbl_high = reinterpret_cast<uint32_t *>(m + c->off.tbl_high);
+    v.tbl_low = reinterpret_cast<uint32_t *>(m + c->off.tbl_low);
+    v.budget = reinterpret_cast<pask_budget_state_t *>(m + c->off.budget);
+    v.seq_mark = reinterpret_cast<uint32_t *>(m + c->off.seq_mark);
+    v.plan = reinterpret_cast<AppendPlan *>(m + c->off.plan);
+    v.tok_scratch = reinterpret_cast<uint2 *>(m + c->off.tok_scratch);
+    v.lut = m + c->off.lut;
+    v.layer_group = m + c->off.layer_group;
+    v.n_layers = d->n_layers;
+    v.n_q = d->n_q_heads;
+    v.n_kv = d->n_kv_heads;
+    v.max_seqs = d->max_seqs;
+    v.max_pages = (d->max_tokens_per_seq + kPageTokens - 1) / kPageTokens;
+    v.max_append_tokens = d->max_append_tokens;
+    v.n_tags = (int32_t)pol->n_tags;
+    v.n_groups = (int32_t)pol->n_groups;
+    v.cap_high = d->pool_high_pages;
+    v.cap_low = d->pool_low_pages;
+    v.budget_q16 = pol->budget_q16;
+    v.high_page_bytes = (uint32_t)d->n_kv_heads * kHighHeadBytes;
+    v.low_page_bytes = (uint32_t)d->n_kv_heads * kLowHeadBytes;
+    v.bytes_h = 2u * d->n_kv_heads * kHeadDim * 2u;
+    v.bytes_l = 2u * d->n_kv_heads * (kHeadDim / 2 + kGroupsPerHead * 2);
+    c->attn_ctas = attention_grid(c);
+    // pageable host sources: the runtime stages these copies, so the vectors may die afterwards
+    cudaError_t e = cudaMemcpyAsync(v.lut, pol->eff.data(), pol->eff.size(), cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(v.layer_group, pol->layer_group.data(), pol->layer_group.size(), cudaMemcpyHostToDevice,
+                            stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) { delete c; return PASK_ERR_CUDA; }
+    pask_status_t rc = pask_cache_reset(c, stream_v);
+    if (rc != PASK_OK) { delete c; return rc; }
+    *out = c;
+    return PASK_OK;
+}
+
+void pask_cache_destroy(pask_cache_t *c) { delete c; }
+
+pask_status_t pask_cache_reset(pask_cache_t *c, pask_stream_t stream_v) {
+    if (!c) return PASK_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    uint8_t *m = static_cast<uint8_t *>(c->meta);
+    cudaError_t e = cudaMemsetAsync(m + c->off.ctrl, 0, kCtrlWords * 4, stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m + c->off.zero_begin, 0, c->off.zero_end - c->off.zero_begin, stream);
+    c->append_serial = 0;
+    return cuda_rc(e);
+}
+
+pask_status_t pask_seq_reset(pask_cache_t *c, int32_t seq, pask_stream_t stream) {
+    if (!c) return PASK_ERR_INVALID_ARG;
+    if (seq < 0 || seq >= c->desc.max_seqs) return PASK_ERR_BAD_SEQ;
+    return launch_seq_reset(c, seq, static_cast<cudaStream_t>(stream));
+}
+
+pask_status_t pask_append_kv(pask_cache_t *c, int32_t layer, int32_t n_seqs, int32_t total_tokens,
+                             const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
+                             const uint8_t *tags, const uint16_t *states, uint8_t *actions_out, pask_stream_t stream) {
+    (void)states;  // reserved for the dynamic budget adjustment (Algorithm 2 steps 3-6)
+    if (!c || !seq_ids || !cu_tokens || !tags) return PASK_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->desc.n_layers) return PASK_ERR_INVALID_ARG;
+    if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL || n_seqs > c->desc.max_seqs) return PASK_ERR_INVALID_ARG;
+    if (total_tokens < 0 || total_tokens > c->desc.max_append_tokens) return PASK_ERR_INVALID_ARG;
+    if (total_tokens > 0 && (!k || !v)) return PASK_ERR_INVALID_ARG;
+    if (((uintptr_t)k | (uintptr_t)v) & 15) return PASK_ERR_INVALID_ARG;
+    if (((uintptr_t)seq_ids | (uintptr_t)cu_tokens) & 3) return PASK_ERR_INVALID_ARG;
+    return launch_append(c, layer, n_seqs, total_tokens, seq_ids, cu_tokens, k, v, tags, actions_out,
+                         static_cast<cudaStream_t>(stream));
+}
+
+static pask_status_t attention_common(pask_cache_t *c, bool has_low, int32_t layer, int32_t n_seqs,
+                                      const int32_t *seq_ids, const void *q, float *out, float *lse, void *ws,
+                                      size_t ws_bytes, pask_stream_t stream) {
+    if (!c || !seq_ids || !q || !out || !ws) return PASK_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->desc.n_layers) return PASK_ERR_INVALID_ARG;
+    if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL) return PASK_ERR_INVALID_ARG;
+    if (((uintptr_t)q | (uintptr_t)out) & 15 || ((uintptr_t)ws & 255) || ((uintptr_t)lse & 3)) return PASK_ERR_INVALID_ARG;
+    if (ws_bytes < attention_workspace_bytes(c, n_seqs)) return PASK_ERR_WORKSPACE;
+    return launch_attention(c, has_low, layer, n_seqs, seq_ids, q, out, lse, ws, ws_bytes,
+                            static_cast<cudaStream_t>(stream));
+}
+
+pask_status_t pask_decode_attention(pask_cache_t *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                    const void *q, float *out, float *lse, void *ws, size_t ws_bytes,
+                                    pask_stream_t stream) {
+    return attention_common(c, true, layer, n_seqs, seq_ids, q, out, lse, ws, ws_bytes, stream);
+}
+
+pask_status_t pask_decode_attention_full(pask_cache_t *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                         const void *q, float *out, float *lse, void *ws, size_t ws_bytes,
+                                         pask_stream_t stream) {
+    return attention_common(c, false, layer, n_seqs, seq_ids, q, out, lse, ws, ws_bytes, stream);
+}
+
+size_t pask_workspace_bytes(const pask_cache_t *c, int32_t n_seqs) {
+    if (!c || n_seqs < 1) return 0;
+    return attention_workspace_bytes(c, n_seqs);
+}
+
+size_t pask_step_staging_bytes(const pask_cache_t *c, int32_t n_seqs) {
+    if (!c || n_seqs < 1) return 0;
+    const size_t n = (size_t)n_seqs;
+    size_t p = 0;
+    p += align_up(n * 4, 256);                                    // seq_ids
+    p += align_up((n + 1) * 4, 256);                              // cu_tokens
+    p += 2 * align_up(n * c->desc.n_kv_heads * kHeadDim * 2, 256);  // k, v
+    p += align_up(n, 256);                                        // tags
+    p += align_up(n * c->desc.n_q_heads * kHeadDim * 2, 256);     // q
+    p += align_up(n * c->desc.n_q_heads * kHeadDim * 4, 256);     // out
+    return p;
+}
+
+// fills cu_tokens = 0, 1, ..., n on the device (one token per sequence)
+__global__ void iota_kernel(int32_t *p, int n) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) p[i] = i;
+}
+
+pask_status_t pask_decode_step_host(pask_cache_t *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids_host,
+                                    const void *k_host, const void *v_host, const uint8_t *tags_host,
+                                    const void *q_host, float *out_host, void *staging, size_t staging_bytes,
+                                    void *ws, size_t ws_bytes, pask_stream_t stream_v) {
+    if (!c || !seq_ids_host || !k_host || !v_host || !tags_host || !q_host || !out_host || !staging)
+        return PASK_ERR_INVALID_ARG;
+    if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL) return PASK_ERR_INVALID_ARG;
+    if (((uintptr_t)staging & 255) || staging_bytes < pask_step_staging_bytes(c, n_seqs)) return PASK_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const size_t n = (size_t)n_seqs;
+    const size_t kv_bytes = n * c->desc.n_kv_heads * kHeadDim * 2, q_bytes = n * c->desc.n_q_heads * kHeadDim * 2;
+    uint8_t *p = static_cast<uint8_t *>(staging);
+    int32_t *d_ids = reinterpret_cast<int32_t *>(p); p += align_up(n * 4, 256);
+    int32_t *d_cu = reinterpret_cast<int32_t *>(p); p += align_up((n + 1) * 4, 256);
+    void *d_k = p; p += align_up(kv_bytes, 256);
+    void *d_v = p; p += align_up(kv_bytes, 256);
+    uint8_t *d_tags = p; p += align_up(n, 256);
+    void *d_q = p; p += align_up(q_bytes, 256);
+    float *d_out = reinterpret_cast<float *>(p);
+    cudaError_t e = cudaMemcpyAsync(d_ids, seq_ids_host, n * 4, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_k, k_host, kv_bytes, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_v, v_host, kv_bytes, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_tags, tags_host, n, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_q, q_host, q_bytes, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return PASK_ERR_CUDA;
+    iota_kernel<<<(n_seqs + 1 + 255) / 256, 256, 0, stream>>>(d_cu, n_seqs + 1);
+    pask_status_t rc = pask_append_kv(c, layer, n_seqs, n_seqs, d_ids, d_cu, d_k, d_v, d_tags, nullptr, nullptr, stream_v);
+    if (rc != PASK_OK) return rc;
+    rc = pask_decode_attention(c, layer, n_seqs, d_ids, d_q, d_out, nullptr, ws, ws_bytes, stream_v);
+    if (rc != PASK_OK) return rc;
+    e = cudaMemcpyAsync(out_host, d_out, n * c->desc.n_q_heads * kHeadDim * 4, cudaMemcpyDeviceToHost, stream);
+    return cuda_rc(e);
+}
+
+pask_status_t pask_budget_state(pask_cache_t *c, int32_t seq, pask_budget_state_t *host_out, pask_stream_t stream_v) {
+    if (!c || !host_out) return PASK_ERR_INVALID_ARG;
+    if (seq < 0 || seq >= c->desc.max_seqs) return PASK_ERR_BAD_SEQ;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    uint32_t status = 0;
+    cudaError_t e = cudaMemcpyAsync(host_out, c->dev.budget + seq, sizeof(*host_out), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&status, c->dev.ctrl + kCtrlStatus, 4, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return PASK_ERR_CUDA;
+    host_out->device_status = status;
+    host_out->reserved = 0;
+    return PASK_OK;
+}
+
+pask_status_t pask_cache_set_timing_events(pask_cache_t *c, pask_event_t start, pask_event_t stop) {
+    if (!c) return PASK_ERR_INVALID_ARG;
+    c->ev_start = static_cast<cudaEvent_t>(start);
+    c->ev_stop = static_cast<cudaEvent_t>(stop);
+    return PASK_OK;
+}
+
+pask_status_t pask_debug_stream_len(pask_cache_t *c, int32_t layer, int32_t seq, uint32_t *n_high, uint32_t *n_low,
+                                    pask_stream_t stream) {
+    if (!c || !n_high || !n_low) return PASK_ERR_INVALID_ARG;
+    if (!seq_layer_ok(c, layer, seq)) return PASK_ERR_INVALID_ARG;
+    return read_lens(c, layer, seq, n_high, n_low, static_cast<cudaStream_t>(stream));
+}
+
+pask_status_t pask_debug_pool_state(pask_cache_t *c, uint32_t *out4, pask_stream_t stream) {
+    if (!c || !out4) return PASK_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return PASK_ERR_CUDA;
+    return cuda_rc(cudaMemcpy(out4, c->dev.ctrl + kCtrlHighNext, 16, cudaMemcpyDeviceToHost));
+}
+
+pask_status_t pask_debug_dump_high(pask_cache_t *c, int32_t layer, int32_t seq, uint16_t *k_out, uint16_t *v_out,
+                                   uint32_t *pages_out, pask_stream_t stream) {
+    if (!c || !seq_layer_ok(c, layer, seq)) return PASK_ERR_INVALID_ARG;
+    uint32_t nh = 0, nl = 0;
+    pask_status_t rc = read_lens(c, layer, seq, &nh, &nl, static_cast<cudaStream_t>(stream));
+    if (rc != PASK_OK) return rc;
+    const uint32_t n_pages = (nh + kPageTokens - 1) / kPageTokens;
+    if (n_pages == 0) return PASK_OK;
+    if (!k_out || !v_out || !pages_out) return PASK_ERR_INVALID_ARG;
+    const size_t tbl = ((size_t)seq * c->desc.n_layers + layer) * c->dev.max_pages;
+    if (cudaMemcpy(pages_out, c->dev.tbl_high + tbl, (size_t)n_pages * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return PASK_ERR_CUDA;
+    const int n_kv = c->desc.n_kv_heads;
+    std::vector<uint8_t> page(c->dev.high_page_bytes);
+    for (uint32_t p = 0; p < n_pages; p++) {
+        if (pages_out[p] >= c->dev.cap_high) return PASK_ERR_CUDA;
+        if (cudaMemcpy(page.data(), c->dev.pool_high + (size_t)pages_out[p] * c->dev.high_page_bytes, page.size(),
+                       cudaMemcpyDeviceToHost) != cudaSuccess)
+            return PASK_ERR_CUDA;
+        for (uint32_t tau = 0; tau < (uint32_t)kPageTokens && p * kPageTokens + tau < nh; tau++) {
+            const size_t tok = (size_t)p * kPageTokens + tau;
+            for (int h = 0; h < n_kv; h++) {
+                const uint8_t *kt = page.data() + (size_t)h * kHighHeadBytes;
+                const uint8_t *vt = kt + kHighTileBytes;
+                uint16_t *kd = k_out + (tok * n_kv + h) * kHeadDim, *vd = v_out + (tok * n_kv + h) * kHeadDim;
+                for (int ch = 0; ch < 16; ch++) std::memcpy(kd + 8 * ch, kt + high_k_chunk_off((int)tau, ch), 16);
+                for (int q = 0; q < 4; q++)
+                    for (int g = 0; g < 8; g++)
+                        std::memcpy(vd + 32 * q + 4 * g, vt + high_v_piece_off((int)tau, q, g), 8);
+            }
+        }
+    }
+    return PASK_OK;
+}
+
+pask_status_t pask_debug_dump_low(pask_cache_t *c, int32_t layer, int32_t seq, uint8_t *k_codes, uint16_t *k_scales,
+                                  uint8_t *v_codes, uint16_t *v_scales, uint32_t *pages_out, pask_stream_t stream) {
+    if (!c || !seq_layer_ok(c, layer, seq)) return PASK_ERR_INVALID_ARG;
+    uint32_t nh = 0, nl = 0;
+    pask_status_t rc = read_lens(c, layer, seq, &nh, &nl, static_cast<cudaStream_t>(stream));
+    if (rc != PASK_OK) return rc;
+    const uint32_t n_pages = (nl + kPageTokens - 1) / kPageTokens;
+    if (n_pages == 0) return PASK_OK;
+    if (!k_codes || !k_scales || !v_codes || !v_scales || !pages_out) return PASK_ERR_INVALID_ARG;
+    const size_t tbl = ((size_t)seq * c->desc.n_layers + layer) * c->dev.max_pages;
+    if (cudaMemcpy(pages_out, c->dev.tbl_low + tbl, (size_t)n_pages * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return PASK_ERR_CUDA;
+    const int n_kv = c->desc.n_kv_heads;
+    std::vector<uint8_t> page(c->dev.low_page_bytes);
+    for (uint32_t p = 0; p < n_pages; p++) {
+        if (pages_out[p] >= c->dev.cap_low) return PASK_ERR_CUDA;
+        if (cudaMemcpy(page.data(), c->dev.pool_low + (size_t)pages_out[p] * c->dev.low_page_bytes, page.size(),
+                       cudaMemcpyDeviceToHost) != cudaSuccess)
+            return PASK_ERR_CUDA;
+        for (uint32_t tau = 0; tau < (uint32_t)kPageTokens && p * kPageTokens + tau < nl; tau++) {
+            const size_t tok = (size_t)p * kPageTokens + tau;
+            for (int h = 0; h < n_kv; h++) {
+                const uint8_t *kh = page.data() + (size_t)h * kLowHeadBytes;
+                const uint8_t *vh = kh + kLowHalfBytes;
+                uint8_t *kc = k_codes + (tok * n_kv + h) * kHeadDim, *vc = v_codes + (tok * n_kv + h) * kHeadDim;
+                uint16_t *ks = k_scales + (tok * n_kv + h) * kGroupsPerHead;
+                uint16_t *vs = v_scales + (tok * n_kv + h) * kGroupsPerHead;
+                for (int w = 0; w < 4; w++) {
+                    std::memcpy(ks + w, kh + low_scale_off((int)tau, w), 2);
+                    std::memcpy(vs + w, vh + low_scale_off((int)tau, w), 2);
+                    for (int t = 0; t < 4; t++) {
+                        uint32_t word;
+                        std::memcpy(&word, kh + low_k_word_off((int)tau, w, t), 4);
+                        for (int e = 0; e < 8; e++) kc[32 * w + 8 * t + e] = (word >> (4 * low_k_nibble(e))) & 0xF;
+                    }
+                    for (int g = 0; g < 8; g++) {
+                        uint16_t half;
+                        std::memcpy(&half, vh + low_v_half_off((int)tau, w, g), 2);
+                        for (int i = 0; i < 4; i++) vc[32 * w + 4 * g + i] = (half >> (4 * i)) & 0xF;
+                    }
+                }
+            }
+        }
+    }
+    return PASK_OK;
+}
+
+pask_status_t pask_debug_set_attention_ctas(pask_cache_t *c, int32_t n_ctas) {
+    if (!c || n_ctas < 1 || n_ctas > 65536) return PASK_ERR_INVALID_ARG;
+    c->attn_ctas = n_ctas;
+    return PASK_OK;
+}
+
+pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, const uint32_t *pages_low,
+                                   int32_t n_ctas, uint32_t *ranges) {
+    if (n_seqs < 1 || n_ctas < 1 || !pages_high || !pages_low || !ranges) return PASK_ERR_INVALID_ARG;
+    std::vector<uint64_t> prefix((size_t)n_seqs + 1, 0);
+    for (int s = 0; s < n_seqs; s++)
+        prefix[s + 1] = prefix[s] + (uint64_t)pages_high[s] * kCostHighPage + (uint64_t)pages_low[s] * kCostLowPage;
+    const uint64_t total = prefix[n_seqs];
+    for (int b = 0; b < n_ctas; b++) {
+        const uint64_t lo = total * b / n_ctas, hi = total * (b + 1) / n_ctas;
+        for (int s = 0; s < n_seqs; s++) {
+            uint32_t *r = ranges + ((size_t)b * n_seqs + s) * 2;
+            r[0] = r[1] = 0;
+            if (prefix[s + 1] <= lo || prefix[s] >= hi || prefix[s + 1] == prefix[s]) continue;
+            const uint64_t a = (lo > prefix[s] ? lo : prefix[s]) - prefix[s];
+            const uint64_t e = (hi < prefix[s + 1] ? hi : prefix[s + 1]) - prefix[s];
+            r[0] = cut_to_page((uint32_t)a, pages_high[s], pages_low[s]);
+            r[1] = (hi >= prefix[s + 1]) ? pages_high[s] + pages_low[s]
+                                        : cut_to_page((uint32_t)e, pages_high[s], pages_low[s]);
+        }
+    }
+    return PASK_OK;
+}
+
+}  // extern "C"

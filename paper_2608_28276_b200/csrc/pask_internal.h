@@ -1,0 +1,94 @@
+// Internal types shared by the host API and the kernels of libpask.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/pask.h"
+#include "pask_layout.h"
+
+namespace pask {
+
+// control words at the start of meta
+enum CtrlWord : int {
+    kCtrlStatus = 0,    // sticky PASK_DEV_* bits
+    kCtrlTicket = 1,    // arrival counter of the append plan kernel (self-resetting)
+    kCtrlHighNext = 2,  // bump counter of the HIGH pool
+    kCtrlHighFree = 3,  // depth of the HIGH free stack
+    kCtrlLowNext = 4,
+    kCtrlLowFree = 5,
+    kCtrlPlanOk = 6,    // 1 if the last append plan was committed, 0 if it was refused
+    kCtrlWords = 64
+};
+
+// one record per sequence of an append call, written by the plan kernel
+struct AppendPlan {
+    int32_t seq;
+    uint32_t old_high, old_low;    // stream lengths before the call
+    uint32_t cnt_high, cnt_low;    // tokens this call adds to each stream
+    uint32_t cnt_drop, bad_tags;
+    uint32_t new_pages_high, new_pages_low;
+    uint32_t pad[7];
+};
+static_assert(sizeof(AppendPlan) == 64, "plan record");
+
+// Device view of a cache, passed to kernels by value.
+struct DevCache {
+    uint8_t *pool_high, *pool_low;
+    uint32_t *ctrl;
+    uint32_t *free_high, *free_low;
+    uint32_t *n_high, *n_low;        // [max_seqs][n_layers] stream lengths in tokens
+    uint32_t *tbl_high, *tbl_low;    // [max_seqs][n_layers][max_pages] page ids
+    pask_budget_state_t *budget;     // [max_seqs]
+    uint32_t *seq_mark;              // [max_seqs] serial of the last append call that named the sequence
+    AppendPlan *plan;                // [PASK_MAX_SEQS_PER_CALL]
+    uint2 *tok_scratch;              // [max_append_tokens] {action | stream position << 2, index in call}
+    uint8_t *lut;                    // [n_tags][n_groups] effective action max(a0, floor)
+    uint8_t *layer_group;            // [n_layers]
+    int32_t n_layers, n_q, n_kv, max_seqs, max_pages, max_append_tokens;
+    int32_t n_tags, n_groups;
+    uint32_t cap_high, cap_low;
+    uint32_t budget_q16;
+    uint32_t high_page_bytes, low_page_bytes;
+    uint32_t bytes_h, bytes_l;       // m(H), m(L) per token per layer
+};
+
+struct MetaOffsets {
+    size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, plan, tok_scratch, lut,
+        layer_group, total;
+    size_t zero_begin, zero_end;     // the span cleared by a reset (counters, tables, budgets, marks)
+};
+
+}  // namespace pask
+
+struct pask_policy {
+    uint32_t n_tags, n_groups, n_layers, n_states, budget_q16;
+    std::vector<uint8_t> layer_group, a0, a_floor, eff;
+    std::vector<float> rho_rl, rho_lh;
+    std::vector<uint32_t> gamma;
+};
+
+struct pask_cache {
+    pask_cache_desc_t desc;
+    pask::DevCache dev;
+    pask::MetaOffsets off;
+    void *meta;
+    uint32_t append_serial;
+    int sm_count;
+    int attn_ctas;                // grid of the decode-attention main kernel
+    cudaEvent_t ev_start, ev_stop;
+};
+
+namespace pask {
+// launchers implemented next to their kernels
+pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_tokens, const int32_t *seq_ids,
+                            const int32_t *cu_tokens, const void *k, const void *v, const uint8_t *tags,
+                            uint8_t *actions_out, cudaStream_t stream);
+pask_status_t launch_seq_reset(pask_cache *c, int seq, cudaStream_t stream);
+pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seqs, const int32_t *seq_ids,
+                               const void *q, float *out, float *lse, void *workspace, size_t workspace_bytes,
+                               cudaStream_t stream);
+size_t attention_workspace_bytes(const pask_cache *c, int n_seqs);
+int attention_grid(const pask_cache *c);
+}  // namespace pask

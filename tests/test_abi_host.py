@@ -1,0 +1,106 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports what the header
+declares, parses policy blobs like the oracle does, sizes caches, and partitions decode work so
+that every page is processed exactly once."""
+import ctypes as C
+import os
+import re
+import subprocess
+
+import numpy as np
+import pytest
+
+from pask_workloads import configs as WC
+from pask_workloads import policy as WP
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def pask():
+    subprocess.run(["python", os.path.join(ROOT, "paper_2608_28276_b200", "build.py")], check=True, capture_output=True)
+    import paper_2608_28276_b200 as P
+    return P
+
+
+def test_library_exports_every_declared_symbol(pask):
+    header = open(os.path.join(ROOT, "include", "pask.h")).read()
+    declared = set(re.findall(r"\b(pask_[a-z0-9_]+)\s*\(", header))
+    declared -= {"pask_budget_state_t"}
+    assert declared == set(pask.EXPORTS), declared ^ set(pask.EXPORTS)
+    lib = C.CDLL(pask.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_struct_layouts_match_header(pask):
+    assert C.sizeof(pask.BudgetState) == 4 * 8 * 8 + 4 * 8 + 4 * 4
+    assert C.sizeof(pask.CacheDesc) == 40
+
+
+def test_policy_blob_parsing_agrees_with_oracle(pask, oracle):
+    for cfg in (WC.TINY, WC.QWEN3_4B_1LAYER):
+        w = WC.build(cfg)
+        h = pask.pask_load_policy(w.blob)
+        o = oracle.Policy(w.blob)
+        for z in range(w.policy.n_tags):
+            for c in range(w.policy.n_groups):
+                assert pask.pask_policy_action(h, z, c) == o.action(z, c) == max(w.policy.a0[z, c], w.policy.a_floor[z, c])
+        assert pask.pask_policy_action(h, w.policy.n_tags, 0) == -1
+        pask.pask_free_policy(h)
+
+
+def test_bad_blobs_and_arguments_are_refused(pask):
+    good = WC.build(WC.TINY).blob
+    bads = [good[:-1], good + b"\0", b"XASK" + good[4:], good[:4] + b"\2\0\0\0" + good[8:], b"PASK", b""]
+    broken = bytearray(good); broken[40 + 4] = 3; bads.append(bytes(broken))           # action out of range
+    broken = bytearray(good); broken[28] = 1; bads.append(bytes(broken))               # recent window != 0
+    broken = bytearray(good); broken[32] = 8; bads.append(bytes(broken))               # low_bits != 4
+    broken = bytearray(good); broken[40] = 9; bads.append(bytes(broken))               # layer group out of range
+    for b in bads:
+        with pytest.raises(pask.PaskError) as e:
+            pask.pask_load_policy(b)
+        assert e.value.status == pask.ERR_BAD_POLICY
+    d = pask.CacheDesc(1, 8, 2, 128, 16, 4, 1024, 1024, 8, 8)
+    assert pask.pask_cache_sizes(d).high_page_bytes == 2 * 8192
+    assert pask.pask_cache_sizes(d).low_page_bytes == 2 * 2304
+    for bad in (pask.CacheDesc(1, 8, 2, 64, 16, 4, 1024, 1024, 8, 8), pask.CacheDesc(1, 8, 2, 128, 32, 4, 1024, 1024, 8, 8),
+                pask.CacheDesc(1, 6, 2, 128, 16, 4, 1024, 1024, 8, 8), pask.CacheDesc(1, 12, 3, 128, 16, 4, 1024, 1024, 8, 8)):
+        with pytest.raises(pask.PaskError) as e:
+            pask.pask_cache_sizes(bad)
+        assert e.value.status == pask.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(pask.PaskError) as e:
+        pask.pask_cache_sizes(pask.CacheDesc(0, 8, 2, 128, 16, 4, 1024, 1024, 8, 8))
+    assert e.value.status == pask.ERR_INVALID_ARG
+    assert pask.pask_status_string(pask.ERR_POOL_EXHAUSTED) == "page pool exhausted"
+
+
+def test_decode_partition_covers_every_page_exactly_once(pask):
+    rng = np.random.default_rng(3)
+    cases = [([5], [0], 4), ([0], [7], 3), ([0, 0, 3], [0, 2, 0], 8), ([1], [1], 296)]
+    for _ in range(30):
+        n = int(rng.integers(1, 40))
+        cases.append((rng.integers(0, 60, n), rng.integers(0, 90, n), int(rng.choice([1, 2, 7, 64, 296]))))
+    for ph, pl, g in cases:
+        ph, pl = np.asarray(ph, np.uint32), np.asarray(pl, np.uint32)
+        r = pask.pask_debug_partition(ph, pl, g).astype(np.int64)
+        for s in range(len(ph)):
+            seen = np.zeros(int(ph[s] + pl[s]), np.int64)
+            last_end = 0
+            for b in range(g):
+                a, e = r[b, s]
+                assert a <= e
+                if e > a:
+                    assert a == last_end          # contiguous, in CTA order
+                    last_end = e
+                seen[a:e] += 1
+            assert np.all(seen == 1)
+        # balance: no CTA streams more than its share plus one page of the costliest kind
+        cost = np.zeros(g)
+        for b in range(g):
+            for s in range(len(ph)):
+                a, e = r[b, s]
+                hi_pages = max(0, min(e, int(ph[s])) - min(a, int(ph[s])))
+                cost[b] += 32 * hi_pages + 9 * ((e - a) - hi_pages)
+        total = float(32 * ph.sum() + 9 * pl.sum())
+        assert cost.sum() == total
+        assert cost.max() <= total / g + 32 + 1e-9
