@@ -1,0 +1,486 @@
+#!/usr/bin/env python
+"""Benchmark of the PASK online hot path on B200.
+
+A step is one decode step of the whole path for one batch: for every layer, pask_append_kv of
+the new token of each sequence (table lookup, drop / int4 / bf16 persist, paging, budget state)
+followed by pask_decode_attention over the mixed-precision cache. The default workload is the
+Qwen3-4B full decode step (36 layers, 4 layer groups, batch 64, sequence lengths uniform in
+[2K, 8K], KV budget 0.33); metric = decode tokens/s (batch / step time).
+
+    python bench.py --gpus 1 --steps 20 --warmup 3
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   (weak scaling: every
+        rank runs its own batch, no collective on the data path)
+    python bench.py --impl reference      times the CPU oracle on a bounded sample instead
+
+Prints one JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from pask_workloads import configs as WC                      # noqa: E402
+from pask_workloads.tensors import TENSOR_K, TENSOR_Q, TENSOR_V, normal_bf16, bf16_bits  # noqa: E402
+
+METRIC = "mixed-KV decode-attn tokens/s at KV budget 0.33"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+STEP_STREAM = 1_000_000          # decode-step inputs of step i come from generator stream (layer, STEP_STREAM + i)
+
+CONFIGS = {c.name: c for c in WC.CONFIGS}
+DEFAULT_CONFIG = WC.QWEN3_4B_STEP.name
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# workload bookkeeping (host side, inputs only)
+
+def stream_counts(w):
+    """Tokens each (sequence, layer group) keeps at high / low precision, from tags and table."""
+    pol = w.policy
+    eff = np.maximum(pol.a0, pol.a_floor)
+    B, G = w.cfg.batch, pol.n_groups
+    nh = np.zeros((B, G), np.int64)
+    nl = np.zeros((B, G), np.int64)
+    for b in range(B):
+        tags = w.tags(b, 0, w.total_len(b))
+        prot = tags == 0xFF
+        known = tags[~prot]
+        cnt = np.bincount(known[known < pol.n_tags], minlength=pol.n_tags)
+        unknown = int((known >= pol.n_tags).sum()) + int(prot.sum())
+        for g in range(G):
+            nh[b, g] = int(cnt[eff[:, g] == 2].sum()) + unknown
+            nl[b, g] = int(cnt[eff[:, g] == 1].sum())
+    return nh, nl
+
+
+def step_inputs(w, layer, step, device):
+    """K, V, Q and tags of decode step `step` at `layer` for the whole batch (row b = sequence b)."""
+    cfg = w.cfg
+    k = normal_bf16(w.seed, TENSOR_K, layer, STEP_STREAM + step, 0, cfg.batch, cfg.n_kv, device)
+    v = normal_bf16(w.seed, TENSOR_V, layer, STEP_STREAM + step, 0, cfg.batch, cfg.n_kv, device)
+    q = normal_bf16(w.seed, TENSOR_Q, layer, STEP_STREAM + step, 0, cfg.batch, cfg.n_q, device)
+    tags = np.array([w.gen_tags[b][w.gen_len(b) + step] for b in range(cfg.batch)], np.uint8)
+    return k, v, q, tags
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [r.split(", ") for r in open(self.path).read().strip().splitlines() if r.strip()]
+            os.unlink(self.path)
+            sm = [float(r[0]) for r in rows]
+            out["sm_mhz"] = statistics.median(sm) if sm else None
+            out["sm_max_mhz"] = float(rows[0][1]) if rows else None
+            out["power_w_max"] = max(float(r[2]) for r in rows) if rows else None
+            out["samples"] = len(rows)
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            for i, nme in enumerate(names):
+                if any(r[4 + i].strip().lower().startswith("active") for r in rows):
+                    out["reasons"].append(nme)
+        except Exception:
+            pass
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA arm
+
+class Job:
+    """One rank's cache, filled with the workload's history, ready to run decode steps."""
+
+    def __init__(self, P, w, device, total_steps, policy_blob=None, label="pask"):
+        self.P, self.w, self.device, self.label = P, w, device, label
+        cfg = w.cfg
+        self.cfg = cfg
+        self.B = cfg.batch
+        blob = policy_blob or w.blob
+        nh, nl = stream_counts(w)
+        if policy_blob is not None:                      # the all-high comparison cache
+            tot = np.array([w.total_len(b) for b in range(self.B)], np.int64)
+            nh = np.repeat(tot[:, None], w.policy.n_groups, axis=1)
+            nl = np.zeros_like(nh)
+        self.nh, self.nl = nh, nl
+        lg = w.policy.layer_group.astype(np.int64)
+        extra = total_steps + 1
+        pages_h = int(sum(((nh[:, lg[l]] + extra + 15) // 16).sum() for l in range(cfg.n_layers))) + 64
+        pages_l = int(sum(((nl[:, lg[l]] + extra + 15) // 16).sum() for l in range(cfg.n_layers))) + 64
+        self.lens = [w.total_len(b) for b in range(self.B)]
+        self.total_tokens = int(sum(self.lens))
+        self.cache = P.Cache(blob, cfg.n_layers, cfg.n_q, cfg.n_kv, self.B, max(self.lens) + extra + 16,
+                             self.total_tokens, pages_h, pages_l, device=device)
+        self.ids = torch.arange(self.B, dtype=torch.int32, device=device)
+        self.cu1 = torch.arange(self.B + 1, dtype=torch.int32, device=device)
+        self.ws = self.cache.workspace(self.B)
+        self.out = torch.empty((self.B, cfg.n_q, 128), dtype=torch.float32, device=device)
+        self.lse = torch.empty((self.B, cfg.n_q), dtype=torch.float32, device=device)
+        self.attn = P.pask_decode_attention_full if policy_blob is not None else P.pask_decode_attention
+
+    def fill(self):
+        """Append the whole history, one ragged bulk call per layer (generated on the device)."""
+        w, cfg, d = self.w, self.cfg, self.device
+        cu = torch.tensor(np.concatenate([[0], np.cumsum(self.lens)]), dtype=torch.int32, device=d)
+        tags = torch.from_numpy(np.concatenate([w.tags(b, 0, self.lens[b]) for b in range(self.B)])).to(d)
+        for layer in range(cfg.n_layers):
+            k = torch.cat([normal_bf16(w.seed, TENSOR_K, layer, b, 0, self.lens[b], cfg.n_kv, d) for b in range(self.B)])
+            v = torch.cat([normal_bf16(w.seed, TENSOR_V, layer, b, 0, self.lens[b], cfg.n_kv, d) for b in range(self.B)])
+            self.P.pask_append_kv(self.cache.handle, layer, self.ids, cu, k, v, tags)
+            del k, v
+        torch.cuda.synchronize()
+        st = self.P.pask_budget_state(self.cache.handle, 0)
+        if st.device_status:
+            raise RuntimeError(f"device status {st.device_status:#x} after fill")
+
+    def prepare_steps(self, n_steps):
+        w, cfg, d = self.w, self.cfg, self.device
+        self.steps = []
+        for s in range(n_steps):
+            per_layer = []
+            for layer in range(cfg.n_layers):
+                k, v, q, tags = step_inputs(w, layer, s, d)
+                per_layer.append((k, v, q, torch.from_numpy(tags).to(d)))
+            self.steps.append(per_layer)
+
+    def run_step(self, s, events=None):
+        P, h = self.P, self.cache.handle
+        for layer, (k, v, q, tags) in enumerate(self.steps[s]):
+            P.pask_append_kv(h, layer, self.ids, self.cu1, k, v, tags)
+            if events is not None:
+                P.pask_cache_set_timing_events(h, *events[layer])
+            self.attn(h, layer, self.ids, q, self.out, self.lse, self.ws)
+
+    def algorithmic_bytes_per_layer(self, steps_done=0):
+        """Bytes one decode-attention launch must move, averaged over layers: K/V payload of the
+        retained tokens (incl. scales), q, out, lse, page tables, split partials written + read."""
+        cfg = self.cfg
+        lg = self.w.policy.layer_group.astype(np.int64)
+        n_ctas = 2 * torch.cuda.get_device_properties(self.device).multi_processor_count
+        tot = 0.0
+        for l in range(cfg.n_layers):
+            nh, nl = self.nh[:, lg[l]] + steps_done, self.nl[:, lg[l]]
+            tot += float((nh * cfg.n_kv * 512).sum() + (nl * cfg.n_kv * 144).sum())
+            tot += float((((nh + 15) // 16) + ((nl + 15) // 16)).sum() * 4)
+        per_layer = tot / cfg.n_layers
+        per_layer += self.B * cfg.n_q * 128 * 2 + self.B * cfg.n_q * (128 + 1) * 4
+        per_layer += 2 * (n_ctas + self.B) * cfg.n_q * 130 * 4
+        return per_layer
+
+
+def run_cuda(args, rank, world):
+    import paper_2608_28276_b200 as P
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    torch.cuda.set_device(device)
+    cfg = CONFIGS[args.config]
+    if args.budget is not None or args.bias != "balanced":
+        cfg = WC.scaled(cfg, budget=args.budget if args.budget is not None else cfg.budget, bias=args.bias,
+                        lut="all_high" if (args.budget or 0) >= 1.0 else cfg.lut)
+    if args.layers:
+        cfg = WC.scaled(cfg, n_layers=args.layers, name=f"{cfg.name}[first {args.layers} layers]")
+    total_steps = args.warmup + args.steps
+    e2e_steps = min(args.steps, 5)
+    cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, 2 * total_steps + e2e_steps + 8))
+    w = WC.build(cfg, repeat=rank)
+    t_setup = time.time()
+    job = Job(P, w, device, 2 * total_steps + e2e_steps + 4)
+    job.fill()
+    job.prepare_steps(total_steps)
+    t_setup = time.time() - t_setup
+    ret = sum(P.pask_budget_state(job.cache.handle, b).retained_bytes for b in range(job.B))
+    full = sum(P.pask_budget_state(job.cache.handle, b).full_bytes for b in range(job.B))
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def timed(jb, first_step, n_steps, with_events):
+        evs = None
+        if with_events:
+            evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                    for _ in range(cfg.n_layers)] for _ in range(n_steps)]
+            for row in evs:
+                for a, b in row:
+                    a.record(); b.record()
+        barrier()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for i in range(n_steps):
+            jb.run_step(first_step + i, evs[i] if evs else None)
+        t1.record()
+        barrier()
+        ms = t0.elapsed_time(t1)
+        kern = [a.elapsed_time(b) for row in (evs or []) for a, b in row]
+        return ms, kern
+
+    for i in range(args.warmup):
+        job.run_step(i)
+    sampler = ClockSampler(device.index or 0)
+    if rank == 0:
+        sampler.start()
+    ms, kern_ms = timed(job, args.warmup, args.steps, True)
+    clocks = sampler.stop() if rank == 0 else {}
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms = float(t.item())
+    st = P.pask_budget_state(job.cache.handle, 0)
+    if st.device_status:
+        raise RuntimeError(f"device status {st.device_status:#x} after the timed region")
+    value = world * job.B * args.steps / (ms * 1e-3)
+
+    # ---- end to end: the same step through the host-buffer entry point, copies inside the region
+    e2e = None
+    if rank == 0 or world > 1:
+        staging = torch.empty(P.pask_step_staging_bytes(job.cache.handle, job.B), dtype=torch.uint8, device=device)
+        host = []
+        for s in range(e2e_steps):
+            rows = []
+            for layer in range(cfg.n_layers):
+                k, v, q, tags = step_inputs(w, layer, total_steps + s, "cpu")
+                rows.append((k.pin_memory(), v.pin_memory(), torch.from_numpy(tags).pin_memory(), q.pin_memory()))
+            host.append(rows)
+        ids_h = torch.arange(job.B, dtype=torch.int32).pin_memory()
+        out_h = torch.empty((job.B, cfg.n_q, 128), dtype=torch.float32).pin_memory()
+        barrier()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for rows in host:
+            for layer, (k, v, tags, q) in enumerate(rows):
+                P.pask_decode_step_host(job.cache.handle, layer, ids_h, k, v, tags, q, out_h, staging, job.ws)
+        t1.record()
+        barrier()
+        e_ms = t0.elapsed_time(t1)
+        if world > 1:
+            t = torch.tensor([e_ms], dtype=torch.float64, device=device)
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            e_ms = float(t.item())
+        h2d = cfg.n_layers * (job.B * 4 + 2 * job.B * cfg.n_kv * 256 + job.B + job.B * cfg.n_q * 256)
+        d2h = cfg.n_layers * job.B * cfg.n_q * 128 * 4
+        e2e = {"value": world * job.B * e2e_steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps}
+
+    if rank != 0:
+        return
+    peak, peak_kind = measured_peaks()
+    alg = job.algorithmic_bytes_per_layer(args.warmup + args.steps // 2)
+    k_ms = sum(kern_ms) / len(kern_ms)
+    achieved = alg / (k_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16/int4 storage, bf16 tensor-core operands with fp32 accumulation", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch_per_gpu": job.B, "layers": cfg.n_layers, "layer_groups": cfg.n_groups,
+                   "kv_budget_target": cfg.budget, "kv_budget_realised": ret / full, "table": f"greedy/{cfg.bias}",
+                   "tokens_in_cache_per_gpu": job.total_tokens, "page_tokens": 16,
+                   "l2": "inputs larger than L2: each layer streams its own ~%.0f MB of pages" % (alg / 1e6),
+                   "setup_s": round(t_setup, 1)},
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": 4 * cfg.n_layers * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "decode_attn_kernel<true>", "achieved": achieved, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "algorithmic_bytes_per_launch": alg,
+                     "avg_launch_ms": k_ms, "launches_timed": len(kern_ms), "traffic": None},
+        "attention_share_of_step": sum(kern_ms) / ms,
+    }
+    if args.full_kv and world == 1:
+        line["full_kv"] = run_full_kv(P, args, w, device, total_steps, peak)
+    if args.cpu_seconds > 0:
+        line["cpu_baseline"] = cpu_baseline(w, budget_s=args.cpu_seconds, n_seqs=args.ref_seqs)
+    print(json.dumps(line))
+
+
+def run_full_kv(P, args, w, device, total_steps, peak):
+    """The same workload with every token kept at bf16, through the library's full-KV kernel."""
+    from pask_workloads.policy import all_high_policy, write_blob
+    cfg = w.cfg
+    blob = write_blob(all_high_policy(w.policy.n_tags, cfg.n_groups, cfg.n_layers))
+    try:
+        job = Job(P, w, device, total_steps + 4, policy_blob=blob, label="full-kv")
+        job.fill()
+    except Exception as e:      # e.g. not enough memory for the dense cache next to the PASK one
+        return {"unavailable": str(e)[:200]}
+    job.prepare_steps(total_steps)
+    for i in range(args.warmup):
+        job.run_step(i)
+    evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(cfg.n_layers)]
+           for _ in range(args.steps)]
+    for row in evs:
+        for a, b in row:
+            a.record(); b.record()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(args.steps):
+        job.run_step(args.warmup + i, evs[i])
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1)
+    kern = [a.elapsed_time(b) for row in evs for a, b in row]
+    alg = job.algorithmic_bytes_per_layer(args.warmup + args.steps // 2)
+    k_ms = sum(kern) / len(kern)
+    return {"value": job.B * args.steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / args.steps,
+            "achieved_GBs": alg / (k_ms * 1e-3) / 1e9, "frac": alg / (k_ms * 1e-3) / 1e9 / peak,
+            "algorithmic_bytes_per_launch": alg, "avg_launch_ms": k_ms}
+
+
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle, timed as it stands on a bounded sample of the same workload
+
+class OracleSample:
+    """The oracle's cache holding the history of a few (layer, sequence) pairs of the workload;
+    step(i) runs decode step i on them (append one token per sequence, fp64 attention) and returns
+    the wall time. Building the history is not timed, as the GPU arm's fill is not either."""
+
+    def __init__(self, w, n_seqs, layers):
+        import oracle
+        self.oracle, self.w, self.layers = oracle, w, list(layers)
+        cfg = w.cfg
+        self.B = min(cfg.batch, n_seqs)
+        lens = [w.total_len(b) for b in range(self.B)]
+        pages = len(self.layers) * (sum(lens) // 16 + 8 * self.B) + 64
+        self.cache = oracle.Cache(oracle.Policy(w.blob), cfg.n_q, cfg.n_kv, self.B, pages, pages)
+        gen = "cuda" if torch.cuda.is_available() else "cpu"   # same generator, same bits, either device
+        cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        tags = np.concatenate([w.tags(b, 0, lens[b]) for b in range(self.B)])
+        for layer in self.layers:
+            k = torch.cat([normal_bf16(w.seed, TENSOR_K, layer, b, 0, lens[b], cfg.n_kv, gen) for b in range(self.B)]).cpu()
+            v = torch.cat([normal_bf16(w.seed, TENSOR_V, layer, b, 0, lens[b], cfg.n_kv, gen) for b in range(self.B)]).cpu()
+            rc, _ = self.cache.append(layer, list(range(self.B)), cu, bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags)
+            assert rc == 0
+            del k, v
+
+    def step(self, i):
+        B, t = self.B, 0.0
+        for layer in self.layers:
+            k, v, q, tags = step_inputs(self.w, layer, i, "cpu")
+            kb, vb, qb = bf16_bits(k[:B]).numpy(), bf16_bits(v[:B]).numpy(), bf16_bits(q[:B]).numpy()
+            t0 = time.perf_counter()
+            self.cache.append(layer, list(range(B)), np.arange(B + 1, dtype=np.int32), kb, vb, tags[:B])
+            self.cache.attention_batch(layer, list(range(B)), qb)
+            t += time.perf_counter() - t0
+        return t
+
+    def tokens_per_s(self, seconds):
+        """Decode tokens/s of the full model if every layer took as long as the sampled ones."""
+        return self.B / (seconds / len(self.layers) * self.w.cfg.n_layers)
+
+    def describe(self, n_steps, seconds):
+        cfg = self.w.cfg
+        return (f"layers {self.layers} of {cfg.n_layers} x {self.B} of {cfg.batch} sequences, {n_steps} decode steps "
+                f"(append + fp64 attention), {seconds:.1f} s wall on the host cores, scaled to {cfg.n_layers} layers")
+
+
+def cpu_baseline(w, budget_s=15.0, n_seqs=32):
+    smp = OracleSample(w, n_seqs, [0])
+    cores = smp.oracle.max_threads()
+    smp.step(0)                                    # untimed first touch
+    wall, n = 0.0, 0
+    while n < 16 and wall < budget_s / 4:
+        wall += smp.step(1 + n)
+        n += 1
+    return {"value": smp.tokens_per_s(wall / n), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": smp.describe(n, wall)}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    cfg = CONFIGS[args.config]
+    cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, args.warmup + args.steps + 8))
+    w = WC.build(cfg)
+    smp = OracleSample(w, args.ref_seqs, [0])
+    for i in range(args.warmup):
+        smp.step(i)
+    t = sum(smp.step(args.warmup + i) for i in range(args.steps))
+    value = smp.tokens_per_s(t / args.steps)
+    base = {"value": value, "unit": UNIT, "cores": smp.oracle.max_threads(), "kind": "oracle",
+            "sample": smp.describe(args.steps, t)}
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * cfg.batch / value, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "kv_budget_target": cfg.budget},
+            "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=sorted(CONFIGS))
+    ap.add_argument("--budget", type=float, default=None, help="override the KV budget of the table")
+    ap.add_argument("--bias", default="balanced", choices=["balanced", "low", "high"])
+    ap.add_argument("--no-full-kv", dest="full_kv", action="store_false")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="0 skips the CPU-oracle leg")
+    ap.add_argument("--layers", type=int, default=None, help="profiling aid: keep only the first N layers")
+    ap.add_argument("--ref-seqs", type=int, default=32, help="sequences in the oracle's timed sample")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl")
+    try:
+        run_cuda(args, rank, world)
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -170,7 +170,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
     __syncthreads();
     if (any_bad || !fits) {
         if (tid == 0) {
-            if (!fits) atomicOr(&c.ctrl[kCtrlStatus], PASK_DEV_POOL_EXHAUSTED);
+            if (!fits && !any_bad) atomicOr(&c.ctrl[kCtrlStatus], PASK_DEV_POOL_EXHAUSTED);
             c.ctrl[kCtrlPlanOk] = 0;
             c.ctrl[kCtrlTicket] = 0;
         }
