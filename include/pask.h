@@ -241,9 +241,10 @@ pask_status_t pask_debug_dump_low(pask_cache_t *cache, int32_t layer, int32_t se
 /* out[4] = { high bump counter, high free-stack depth, low bump counter, low free-stack depth }. */
 pask_status_t pask_debug_pool_state(pask_cache_t *cache, uint32_t *out4, pask_stream_t stream);
 /* How the decode-attention kernel splits work: for a batch whose sequences hold the given page
- * counts, and a grid of `n_ctas`, writes for each CTA b and sequence index s the half-open range
- * of concatenated page indices (HIGH pages first, then LOW) that b processes for s, as
- * ranges[(b * n_seqs + s) * 2 + {0,1}] (empty ranges have begin == end).  Host only, no GPU. */
+ * counts, and a grid of `n_ctas`, writes for each CTA b and sequence index s the half-open ranges
+ * of HIGH pages and of LOW pages that b processes for s, as
+ * ranges[(b * n_seqs + s) * 4 + {0,1,2,3}] = high begin, high end, low begin, low end (empty ranges
+ * have begin == end).  Host only, no GPU. */
 pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, const uint32_t *pages_low,
                                    int32_t n_ctas, uint32_t *ranges);
 

@@ -253,11 +253,12 @@ def pask_debug_pool_state(cache: int, stream=None):
 
 
 def pask_debug_partition(pages_high, pages_low, n_ctas: int):
-    """Host-only: page ranges [n_ctas][n_seqs][2] the decode-attention grid would process."""
+    """Host-only: page ranges [n_ctas][n_seqs][4] (high begin, high end, low begin, low end) the
+    decode-attention grid would process."""
     import numpy as np
     ph = np.ascontiguousarray(pages_high, dtype=np.uint32)
     pl = np.ascontiguousarray(pages_low, dtype=np.uint32)
-    out = np.zeros((n_ctas, len(ph), 2), np.uint32)
+    out = np.zeros((n_ctas, len(ph), 4), np.uint32)
     _check(_lib.pask_debug_partition(len(ph), ph.ctypes.data, pl.ctypes.data, n_ctas, out.ctypes.data),
            "pask_debug_partition")
     return out

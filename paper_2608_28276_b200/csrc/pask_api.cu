@@ -458,14 +458,16 @@ pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, c
     for (int b = 0; b < n_ctas; b++) {
         const uint64_t lo = total * b / n_ctas, hi = total * (b + 1) / n_ctas;
         for (int s = 0; s < n_seqs; s++) {
-            uint32_t *r = ranges + ((size_t)b * n_seqs + s) * 2;
-            r[0] = r[1] = 0;
+            uint32_t *r = ranges + ((size_t)b * n_seqs + s) * 4;
+            r[0] = r[1] = r[2] = r[3] = 0;
             if (prefix[s + 1] <= lo || prefix[s] >= hi || prefix[s + 1] == prefix[s]) continue;
-            const uint64_t a = (lo > prefix[s] ? lo : prefix[s]) - prefix[s];
-            const uint64_t e = (hi < prefix[s + 1] ? hi : prefix[s + 1]) - prefix[s];
-            r[0] = cut_to_page((uint32_t)a, pages_high[s], pages_low[s]);
-            r[1] = (hi >= prefix[s + 1]) ? pages_high[s] + pages_low[s]
-                                        : cut_to_page((uint32_t)e, pages_high[s], pages_low[s]);
+            const uint32_t cs = (uint32_t)(prefix[s + 1] - prefix[s]);
+            const uint32_t a = (uint32_t)((lo > prefix[s] ? lo : prefix[s]) - prefix[s]);
+            const uint32_t e = (uint32_t)((hi < prefix[s + 1] ? hi : prefix[s + 1]) - prefix[s]);
+            r[0] = cut_pages(a, cs, pages_high[s]);
+            r[1] = cut_pages(e, cs, pages_high[s]);
+            r[2] = cut_pages(a, cs, pages_low[s]);
+            r[3] = cut_pages(e, cs, pages_low[s]);
         }
     }
     return PASK_OK;

@@ -12,7 +12,8 @@
 //   * A CTA is n_kv warps; warp w handles KV head w for the CTA's page range, so the four query
 //     heads of a group share every K/V byte and no cross-warp reduction exists at all.
 //   * Sequences are laid end to end in cost space and cut into gridDim.x equal spans
-//     (pask_layout.h), so every CTA streams the same number of bytes whatever the length mix;
+//     (pask_layout.h), each cut splitting a sequence's HIGH and LOW page lists at the same
+//     fraction, so every CTA streams the same bytes and the same HIGH/LOW mix whatever the lengths;
 //     a span may cover several sequences, each yields one partial (m, l, o) and the ring is not
 //     drained in between.  A second small kernel merges the partials.
 //   * Pages are stored fragment-major (pask_layout.h): a 128-bit shared load per lane is exactly
@@ -150,9 +151,9 @@ __device__ __forceinline__ void split_pair(float x0, float x1, uint32_t &hi, uin
 // ---------------------------------------------------------------- work partition
 
 struct Segment {
-    uint32_t page_begin, page_end;  // concatenated page index: HIGH pages first, then LOW
-    uint32_t pages_high;
-    uint32_t n_high, n_low;         // tokens
+    uint32_t high_begin, high_count;  // this CTA's run of the sequence's HIGH pages
+    uint32_t low_begin, low_count;    // and of its LOW pages; jobs walk the HIGH run, then the LOW run
+    uint32_t n_high, n_low;           // tokens in the whole streams (for the ragged tail pages)
 };
 
 __device__ __forceinline__ Segment make_segment(int s, uint32_t lo, uint32_t hi, const uint32_t *s_prefix,
@@ -160,12 +161,14 @@ __device__ __forceinline__ Segment make_segment(int s, uint32_t lo, uint32_t hi,
     Segment g;
     g.n_high = s_nh[s];
     g.n_low = s_nl[s];
-    g.pages_high = (g.n_high + kPageTokens - 1) / kPageTokens;
+    const uint32_t pages_high = (g.n_high + kPageTokens - 1) / kPageTokens;
     const uint32_t pages_low = (g.n_low + kPageTokens - 1) / kPageTokens;
-    const uint32_t p0 = s_prefix[s], p1 = s_prefix[s + 1];
-    const uint32_t a = (lo > p0 ? lo : p0) - p0;
-    g.page_begin = cut_to_page(a, g.pages_high, pages_low);
-    g.page_end = hi >= p1 ? g.pages_high + pages_low : cut_to_page(hi - p0, g.pages_high, pages_low);
+    const uint32_t p0 = s_prefix[s], p1 = s_prefix[s + 1], cs = p1 - p0;
+    const uint32_t a = (lo > p0 ? lo : p0) - p0, e = (hi < p1 ? hi : p1) - p0;
+    g.high_begin = cut_pages(a, cs, pages_high);
+    g.high_count = cut_pages(e, cs, pages_high) - g.high_begin;
+    g.low_begin = cut_pages(a, cs, pages_low);
+    g.low_count = cut_pages(e, cs, pages_low) - g.low_begin;
     return g;
 }
 
@@ -174,7 +177,7 @@ __device__ __forceinline__ Segment make_segment(int s, uint32_t lo, uint32_t hi,
 struct Producer {
     int s;                    // current sequence index in the call, n_seqs when exhausted
     Segment seg;
-    uint32_t page;            // next page (concatenated index) of seg
+    uint32_t page;            // next job's page: index into the segment's HIGH run, then its LOW run
     uint32_t sub;             // 0: K tile next, 1: V tile next (HIGH pages)
     uint32_t win_base, win_id;  // 32 page ids cached across the lanes, starting at win_base
     bool win_valid;
@@ -198,11 +201,11 @@ struct Warp {
         for (; in_span(s); ++s) {
             if (s_prefix[s + 1] == s_prefix[s]) continue;
             pr.seg = make_segment(s, lo, hi, s_prefix, s_nh, s_nl);
-            if (pr.seg.page_begin < pr.seg.page_end) break;
+            if (pr.seg.high_count + pr.seg.low_count > 0) break;
         }
         if (!in_span(s)) s = p.n_seqs;
         pr.s = s;
-        pr.page = pr.seg.page_begin;
+        pr.page = 0;
         pr.sub = 0;
         pr.win_valid = false;
     }
@@ -211,7 +214,8 @@ struct Warp {
     __device__ __forceinline__ void produce() {
         if (pr.s >= p.n_seqs) return;
         const DevCache &c = p.c;
-        const bool is_high = pr.page < pr.seg.pages_high;
+        const bool is_high = pr.page < pr.seg.high_count;
+        const uint32_t n_pages = pr.seg.high_count + pr.seg.low_count;
         if (!pr.win_valid || pr.page - pr.win_base >= 32u) {
             // refill the page-id window: lane i holds the id of page win_base + i
             pr.win_base = pr.page;
@@ -219,8 +223,9 @@ struct Warp {
             const uint32_t pg = pr.page + lane;
             const size_t sl = ((size_t)p.seq_ids[pr.s] * c.n_layers + p.layer) * c.max_pages;
             uint32_t id = 0;
-            if (pg < pr.seg.page_end)
-                id = pg < pr.seg.pages_high ? c.tbl_high[sl + pg] : c.tbl_low[sl + (pg - pr.seg.pages_high)];
+            if (pg < n_pages)
+                id = pg < pr.seg.high_count ? c.tbl_high[sl + pr.seg.high_begin + pg]
+                                            : c.tbl_low[sl + pr.seg.low_begin + (pg - pr.seg.high_count)];
             pr.win_id = id;
         }
         const uint32_t id = __shfl_sync(0xffffffffu, pr.win_id, (int)(pr.page - pr.win_base));
@@ -244,7 +249,7 @@ struct Warp {
             pr.sub = 1;
         } else {
             pr.sub = 0;
-            if (++pr.page == pr.seg.page_end) producer_open(pr.s + 1);
+            if (++pr.page == n_pages) producer_open(pr.s + 1);
         }
     }
 
@@ -386,11 +391,11 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         for (int m = 0; m < 8; m++) acc[m][0] = acc[m][1] = acc[m][2] = acc[m][3] = 0.f;
         float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
 
-        for (uint32_t page = seg.page_begin; page < seg.page_end; ++page) {
-            const bool is_high = page < seg.pages_high;
+        for (uint32_t page = 0; page < seg.high_count + seg.low_count; ++page) {
+            const bool is_high = page < seg.high_count;
             uint32_t n_valid;
-            if (is_high) n_valid = min(16u, seg.n_high - page * kPageTokens);
-            else n_valid = min(16u, seg.n_low - (page - seg.pages_high) * kPageTokens);
+            if (is_high) n_valid = min(16u, seg.n_high - (seg.high_begin + page) * kPageTokens);
+            else n_valid = min(16u, seg.n_low - (seg.low_begin + page - seg.high_count) * kPageTokens);
 
             float sc[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t st = w.acquire();

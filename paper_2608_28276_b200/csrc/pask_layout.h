@@ -78,21 +78,16 @@ PASK_HD int low_v_half_off(int tau, int q, int g) {
 PASK_HD int low_scale_off(int tau, int w) { return kLowCodesBytes + tau * 8 + w * 2; }
 
 // ---- work partition of decode attention -------------------------------------------------
-// Sequences are laid end to end in "cost space" (a HIGH page costs 32, a LOW page 9); CTA b of
-// G owns [C*b/G, C*(b+1)/G).  A cut inside a sequence is moved down to a page boundary; both
-// neighbours apply the same rule, so every page is processed exactly once.
+// Sequences are laid end to end in "cost space" (a HIGH page costs kCostHighPage, a LOW page
+// kCostLowPage); CTA b of G owns [C*b/G, C*(b+1)/G).  A cut at local offset x of a sequence whose
+// cost is cs splits BOTH of its page lists at the same fraction x / cs, so every CTA gets the
+// sequence's own mix of HIGH and LOW pages (the two kinds differ in time per byte, and a CTA
+// that received only one kind would finish early or late).  Both neighbours of a cut apply the
+// same rule, so every page is processed exactly once.
 
-// page boundary (in concatenated page index: HIGH pages first) for local cost offset x
-PASK_HD uint32_t cut_to_page(uint32_t x, uint32_t pages_high, uint32_t pages_low) {
-    const uint32_t ch = pages_high * kCostHighPage;
-    if (x < ch) return x / kCostHighPage;
-    const uint32_t p = pages_high + (x - ch) / kCostLowPage;
-    const uint32_t tot = pages_high + pages_low;
-    return p < tot ? p : tot;
-}
-
-PASK_HD uint32_t span_begin(uint64_t total_cost, uint32_t b, uint32_t n_ctas) {
-    return (uint32_t)((total_cost * b) / n_ctas);
+// number of pages (of a list of n_pages) that lie before local cost offset x of a sequence of cost cs
+PASK_HD uint32_t cut_pages(uint32_t x, uint32_t cs, uint32_t n_pages) {
+    return x >= cs ? n_pages : (uint32_t)(((uint64_t)x * n_pages) / cs);
 }
 
 }  // namespace pask

@@ -83,24 +83,21 @@ def test_decode_partition_covers_every_page_exactly_once(pask):
     for ph, pl, g in cases:
         ph, pl = np.asarray(ph, np.uint32), np.asarray(pl, np.uint32)
         r = pask.pask_debug_partition(ph, pl, g).astype(np.int64)
-        for s in range(len(ph)):
-            seen = np.zeros(int(ph[s] + pl[s]), np.int64)
-            last_end = 0
-            for b in range(g):
-                a, e = r[b, s]
-                assert a <= e
-                if e > a:
-                    assert a == last_end          # contiguous, in CTA order
-                    last_end = e
-                seen[a:e] += 1
-            assert np.all(seen == 1)
-        # balance: no CTA streams more than its share plus one page of the costliest kind
         cost = np.zeros(g)
-        for b in range(g):
-            for s in range(len(ph)):
-                a, e = r[b, s]
-                hi_pages = max(0, min(e, int(ph[s])) - min(a, int(ph[s])))
-                cost[b] += 32 * hi_pages + 9 * ((e - a) - hi_pages)
+        for s in range(len(ph)):
+            for which, n_pages, w in ((0, int(ph[s]), 32), (2, int(pl[s]), 9)):
+                seen = np.zeros(n_pages, np.int64)
+                last_end = 0
+                for b in range(g):
+                    a, e = r[b, s, which], r[b, s, which + 1]
+                    assert a <= e
+                    if e > a:
+                        assert a == last_end          # contiguous, in CTA order
+                        last_end = e
+                    seen[a:e] += 1
+                    cost[b] += w * (e - a)
+                assert np.all(seen == 1)
+        # balance: no CTA streams more than its share plus one page of each kind per sequence cut
         total = float(32 * ph.sum() + 9 * pl.sum())
         assert cost.sum() == total
-        assert cost.max() <= total / g + 32 + 1e-9
+        assert cost.max() <= total / g + 2 * (32 + 9) + 1e-9
