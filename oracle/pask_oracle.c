@@ -85,6 +85,7 @@ typedef struct {
 typedef struct {
     const orc_policy *pol;
     int n_q, n_kv, max_seqs;
+    uint32_t n_layers;    /* copy of pol->n_layers, so that tearing down needs no policy */
     orc_stream *streams;  /* [max_seqs][n_layers] */
     orc_budget *budget;   /* [max_seqs] */
     orc_pool pool_high, pool_low;
@@ -233,7 +234,7 @@ orc_cache *orc_cache_create(const orc_policy *pol, int n_q, int n_kv, int max_se
                             uint32_t pool_high_pages, uint32_t pool_low_pages) {
     if (!pol || n_kv <= 0 || n_q != 4 * n_kv || max_seqs <= 0) return NULL;
     orc_cache *c = (orc_cache *)calloc(1, sizeof(*c));
-    c->pol = pol; c->n_q = n_q; c->n_kv = n_kv; c->max_seqs = max_seqs;
+    c->pol = pol; c->n_q = n_q; c->n_kv = n_kv; c->max_seqs = max_seqs; c->n_layers = pol->n_layers;
     c->streams = (orc_stream *)calloc((size_t)max_seqs * pol->n_layers, sizeof(orc_stream));
     c->budget = (orc_budget *)calloc((size_t)max_seqs, sizeof(orc_budget));
     pool_init(&c->pool_high, pool_high_pages);
@@ -249,7 +250,7 @@ static void stream_free(orc_stream *s) {
 
 void orc_cache_destroy(orc_cache *c) {
     if (!c) return;
-    for (size_t i = 0; i < (size_t)c->max_seqs * c->pol->n_layers; i++) stream_free(&c->streams[i]);
+    for (size_t i = 0; i < (size_t)c->max_seqs * c->n_layers; i++) stream_free(&c->streams[i]);
     free(c->streams); free(c->budget); free(c->pool_high.free_stack); free(c->pool_low.free_stack);
     free(c);
 }

@@ -152,7 +152,7 @@ __device__ __forceinline__ void split_pair(float x0, float x1, uint32_t &hi, uin
 
 struct Segment {
     uint32_t high_begin, high_count;  // this CTA's run of the sequence's HIGH pages
-    uint32_t low_begin, low_count;    // and of its LOW pages; jobs walk the HIGH run, then the LOW run
+    uint32_t low_begin, low_count;    // and of its LOW pages; jobs take the two runs interleaved (PageOrder)
     uint32_t n_high, n_low;           // tokens in the whole streams (for the ragged tail pages)
 };
 
@@ -172,12 +172,28 @@ __device__ __forceinline__ Segment make_segment(int s, uint32_t lo, uint32_t hi,
     return g;
 }
 
+// Order in which a segment's pages are visited: its HIGH and LOW runs are interleaved evenly
+// (page v is a HIGH page iff floor((v+1) nH / n) > floor(v nH / n), n = nH + nL).  HIGH pages are
+// bandwidth-heavy and LOW pages instruction-heavy; taking them in turn lets the bulk copies of
+// the former land while the latter are being decoded, instead of alternating between a
+// memory-bound and an issue-bound phase.
+struct PageOrder {
+    uint32_t rem, hi_idx, lo_idx;
+    __device__ __forceinline__ void reset() { rem = hi_idx = lo_idx = 0; }
+    __device__ __forceinline__ bool is_high(const Segment &g) const { return rem + g.high_count >= g.high_count + g.low_count; }
+    __device__ __forceinline__ void advance(const Segment &g) {
+        if (is_high(g)) { rem -= g.low_count; hi_idx++; }
+        else { rem += g.high_count; lo_idx++; }
+    }
+};
+
 // Producer side of a warp's pipeline: walks the CTA's pages in order and issues one bulk copy
 // per job (HIGH page: K tile, then V tile; LOW page: K and V halves together).
 struct Producer {
     int s;                    // current sequence index in the call, n_seqs when exhausted
     Segment seg;
-    uint32_t page;            // next job's page: index into the segment's HIGH run, then its LOW run
+    PageOrder ord;
+    uint32_t page;            // next job's page: position in the segment's interleaved order
     uint32_t sub;             // 0: K tile next, 1: V tile next (HIGH pages)
     uint32_t win_base, win_id;  // 32 page ids cached across the lanes, starting at win_base
     bool win_valid;
@@ -207,6 +223,7 @@ struct Warp {
         pr.s = s;
         pr.page = 0;
         pr.sub = 0;
+        pr.ord.reset();
         pr.win_valid = false;
     }
 
@@ -214,18 +231,20 @@ struct Warp {
     __device__ __forceinline__ void produce() {
         if (pr.s >= p.n_seqs) return;
         const DevCache &c = p.c;
-        const bool is_high = pr.page < pr.seg.high_count;
+        const bool is_high = pr.ord.is_high(pr.seg);
         const uint32_t n_pages = pr.seg.high_count + pr.seg.low_count;
         if (!pr.win_valid || pr.page - pr.win_base >= 32u) {
-            // refill the page-id window: lane i holds the id of page win_base + i
+            // refill the page-id window: lane i holds the id of the page at position win_base + i
             pr.win_base = pr.page;
             pr.win_valid = true;
             const uint32_t pg = pr.page + lane;
             const size_t sl = ((size_t)p.seq_ids[pr.s] * c.n_layers + p.layer) * c.max_pages;
             uint32_t id = 0;
-            if (pg < n_pages)
-                id = pg < pr.seg.high_count ? c.tbl_high[sl + pr.seg.high_begin + pg]
-                                            : c.tbl_low[sl + pr.seg.low_begin + (pg - pr.seg.high_count)];
+            if (pg < n_pages) {
+                const uint32_t h0 = (uint32_t)(((uint64_t)pg * pr.seg.high_count) / n_pages);
+                const uint32_t h1 = (uint32_t)(((uint64_t)(pg + 1) * pr.seg.high_count) / n_pages);
+                id = h1 > h0 ? c.tbl_high[sl + pr.seg.high_begin + h0] : c.tbl_low[sl + pr.seg.low_begin + (pg - h0)];
+            }
             pr.win_id = id;
         }
         const uint32_t id = __shfl_sync(0xffffffffu, pr.win_id, (int)(pr.page - pr.win_base));
@@ -249,6 +268,7 @@ struct Warp {
             pr.sub = 1;
         } else {
             pr.sub = 0;
+            pr.ord.advance(pr.seg);
             if (++pr.page == n_pages) producer_open(pr.s + 1);
         }
     }
@@ -391,11 +411,13 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         for (int m = 0; m < 8; m++) acc[m][0] = acc[m][1] = acc[m][2] = acc[m][3] = 0.f;
         float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
 
-        for (uint32_t page = 0; page < seg.high_count + seg.low_count; ++page) {
-            const bool is_high = page < seg.high_count;
+        PageOrder ord;
+        ord.reset();
+        for (uint32_t page = 0; page < seg.high_count + seg.low_count; ++page, ord.advance(seg)) {
+            const bool is_high = ord.is_high(seg);
             uint32_t n_valid;
-            if (is_high) n_valid = min(16u, seg.n_high - (seg.high_begin + page) * kPageTokens);
-            else n_valid = min(16u, seg.n_low - (seg.low_begin + page - seg.high_count) * kPageTokens);
+            if (is_high) n_valid = min(16u, seg.n_high - (seg.high_begin + ord.hi_idx) * kPageTokens);
+            else n_valid = min(16u, seg.n_low - (seg.low_begin + ord.lo_idx) * kPageTokens);
 
             float sc[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t st = w.acquire();
