@@ -24,7 +24,7 @@
  *   - No function throws or aborts.
  *
  * Formats (the paper leaves them open; these are the library's documented readings)
- *   RETAIN-HIGH keeps the token's bf16 K and V bits.  RETAIN-LOW stores, per token, per KV head
+ *   RETAIN-HIGH keeps the token's bf16 K and V bits (any finite bf16 value).  RETAIN-LOW stores, per token, per KV head
  *   and per group of 32 consecutive head dimensions, one fp16 scale s = fp16(amax / 7) (IEEE
  *   fp32 division, round to nearest even, saturating at 65504) and 32 four-bit codes
  *   clamp(rint(x * (1 / s)), -7, 7) + 8; the value read back is (code - 8) * s.  s == 0 gives
@@ -58,6 +58,8 @@ typedef int32_t pask_status_t;
 #define PASK_DEV_SEQ_OVERFLOW 0x4u    /* a stream would exceed max_tokens_per_seq: nothing written */
 #define PASK_DEV_BAD_RAGGED 0x8u      /* cu_tokens not ascending or not ending at total_tokens */
 #define PASK_DEV_TIMEOUT 0x10u        /* a bounded wait inside a kernel ran out; results invalid */
+#define PASK_DEV_RANGE 0x20u          /* a query element had |q| > 65504, outside what the low-precision path
+                                         computes in; results for that sequence may be infinite or NaN */
 
 #define PASK_ACTION_RELEASE 0
 #define PASK_ACTION_RETAIN_LOW 1
@@ -240,14 +242,21 @@ pask_status_t pask_debug_dump_low(pask_cache_t *cache, int32_t layer, int32_t se
                                   pask_stream_t stream);
 /* out[4] = { high bump counter, high free-stack depth, low bump counter, low free-stack depth }. */
 pask_status_t pask_debug_pool_state(pask_cache_t *cache, uint32_t *out4, pask_stream_t stream);
-/* How the decode-attention kernel splits work: for a batch whose sequences hold the given page
- * counts, and a grid of `n_ctas`, writes for each CTA b and sequence index s the half-open ranges
- * of HIGH pages and of LOW pages that b processes for s, as
- * ranges[(b * n_seqs + s) * 4 + {0,1,2,3}] = high begin, high end, low begin, low end (empty ranges
- * have begin == end).  Host only, no GPU. */
+/* The cache's first `count` (<= 64) control words: [0] device status, [2..5] pool state, [16..23]
+ * wait statistics of decode attention as four 64-bit sums over warps (jobs, jobs that had to wait
+ * for their bulk copy, cycles waited, cycles alive) -- filled only by diagnostic builds compiled
+ * with PASK_STATS, zero otherwise. */
+pask_status_t pask_debug_ctrl_words(pask_cache_t *cache, uint32_t *out, int32_t count, pask_stream_t stream);
+/* How the decode-attention kernel splits work.  Each sequence's pages are visited in a fixed order
+ * that interleaves its HIGH and LOW pages evenly; pask_debug_page_order writes that order for a
+ * sequence with the given page counts: order[v] = page index within its stream, with bit 31 set
+ * for a HIGH page.  For a batch whose sequences hold the given page counts and a grid of `n_ctas`,
+ * pask_debug_partition writes for each CTA b and sequence index s the half-open range of positions
+ * of that order which b processes, as ranges[(b * n_seqs + s) * 2 + {0,1}] (empty: begin == end).
+ * Host only, no GPU. */
+pask_status_t pask_debug_page_order(uint32_t pages_high, uint32_t pages_low, uint32_t *order);
 pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, const uint32_t *pages_low,
                                    int32_t n_ctas, uint32_t *ranges);
-
 /* Override the number of CTAs the decode-attention main kernel is launched with (default: two per
  * SM).  Any value >= 1 gives the same result up to summation order; tests use it to check that.
  * Workspaces must be sized (pask_workspace_bytes) after the change. */

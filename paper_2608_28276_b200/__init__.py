@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libpask.so")
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_POLICY, ERR_UNSUPPORTED_SHAPE, ERR_POOL_EXHAUSTED = -1, -2, -3, -4
 ERR_BAD_SEQ, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE = -5, -6, -7, -8
-DEV_POOL_EXHAUSTED, DEV_BAD_SEQ, DEV_SEQ_OVERFLOW, DEV_BAD_RAGGED, DEV_TIMEOUT = 1, 2, 4, 8, 16
+DEV_POOL_EXHAUSTED, DEV_BAD_SEQ, DEV_SEQ_OVERFLOW, DEV_BAD_RAGGED, DEV_TIMEOUT, DEV_RANGE = 1, 2, 4, 8, 16, 32
 ACTION_RELEASE, ACTION_RETAIN_LOW, ACTION_RETAIN_HIGH = 0, 1, 2
 TAG_PROTECTED = 0xFF
 MAX_GROUPS = 8
@@ -28,7 +28,7 @@ EXPORTS = [
     "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decode_attention",
     "pask_decode_attention_full", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes",
     "pask_budget_state", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
-    "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
+    "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
 ]
 
 
@@ -82,7 +82,9 @@ _lib.pask_debug_stream_len.argtypes = [_vp, _i32, _i32, C.POINTER(C.c_uint32), C
 _lib.pask_debug_dump_high.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp]
 _lib.pask_debug_dump_low.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_debug_pool_state.argtypes = [_vp, _vp, _vp]
+_lib.pask_debug_ctrl_words.argtypes = [_vp, _vp, _i32, _vp]
 _lib.pask_debug_partition.argtypes = [_i32, _vp, _vp, _i32, _vp]
+_lib.pask_debug_page_order.argtypes = [C.c_uint32, C.c_uint32, _vp]
 _lib.pask_debug_set_attention_ctas.argtypes = [_vp, _i32]
 _lib.pask_status_string.argtypes = [_i32]
 _lib.pask_status_string.restype = C.c_char_p
@@ -252,16 +254,31 @@ def pask_debug_pool_state(cache: int, stream=None):
     return tuple(int(x) for x in out)
 
 
+def pask_debug_ctrl_words(cache: int, count: int = 64, stream=None):
+    import numpy as np
+    out = np.zeros(count, np.uint32)
+    _check(_lib.pask_debug_ctrl_words(cache, out.ctypes.data, count, _stream(stream)), "pask_debug_ctrl_words")
+    return out
+
+
 def pask_debug_partition(pages_high, pages_low, n_ctas: int):
-    """Host-only: page ranges [n_ctas][n_seqs][4] (high begin, high end, low begin, low end) the
-    decode-attention grid would process."""
+    """Host-only: ranges [n_ctas][n_seqs][2] of positions in each sequence's page order that the
+    CTAs of the decode-attention grid would process."""
     import numpy as np
     ph = np.ascontiguousarray(pages_high, dtype=np.uint32)
     pl = np.ascontiguousarray(pages_low, dtype=np.uint32)
-    out = np.zeros((n_ctas, len(ph), 4), np.uint32)
+    out = np.zeros((n_ctas, len(ph), 2), np.uint32)
     _check(_lib.pask_debug_partition(len(ph), ph.ctypes.data, pl.ctypes.data, n_ctas, out.ctypes.data),
            "pask_debug_partition")
     return out
+
+
+def pask_debug_page_order(pages_high: int, pages_low: int):
+    """Host-only: the order a sequence's pages are visited in: (is_high bool array, page index array)."""
+    import numpy as np
+    out = np.zeros(pages_high + pages_low, np.uint32)
+    _check(_lib.pask_debug_page_order(pages_high, pages_low, out.ctypes.data), "pask_debug_page_order")
+    return (out >> 31).astype(bool), (out & 0x7FFFFFFF).astype(np.int64)
 
 
 def pask_debug_set_attention_ctas(cache: int, n_ctas: int):

@@ -37,6 +37,7 @@ MetaOffsets meta_offsets(const pask_cache_desc_t *d, int n_tags, int n_groups) {
     o.tbl_low = take(sl * max_pages * 4);
     o.budget = take((size_t)d->max_seqs * sizeof(pask_budget_state_t));
     o.seq_mark = take((size_t)d->max_seqs * 4);
+    o.low_vmax = take(sl * 4);
     o.zero_end = p;
     o.plan = take((size_t)PASK_MAX_SEQS_PER_CALL * sizeof(AppendPlan));
     o.tok_scratch = take((size_t)d->max_append_tokens * sizeof(uint2));
@@ -178,6 +179,7 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     v.tbl_low = reinterpret_cast<uint32_t *>(m + c->off.tbl_low);
     v.budget = reinterpret_cast<pask_budget_state_t *>(m + c->off.budget);
     v.seq_mark = reinterpret_cast<uint32_t *>(m + c->off.seq_mark);
+    v.low_vmax = reinterpret_cast<uint32_t *>(m + c->off.low_vmax);
     v.plan = reinterpret_cast<AppendPlan *>(m + c->off.plan);
     v.tok_scratch = reinterpret_cast<uint2 *>(m + c->off.tok_scratch);
     v.lut = m + c->off.lut;
@@ -360,6 +362,12 @@ pask_status_t pask_debug_pool_state(pask_cache_t *c, uint32_t *out4, pask_stream
     return cuda_rc(cudaMemcpy(out4, c->dev.ctrl + kCtrlHighNext, 16, cudaMemcpyDeviceToHost));
 }
 
+pask_status_t pask_debug_ctrl_words(pask_cache_t *c, uint32_t *out, int32_t count, pask_stream_t stream) {
+    if (!c || !out || count < 1 || count > kCtrlWords) return PASK_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return PASK_ERR_CUDA;
+    return cuda_rc(cudaMemcpy(out, c->dev.ctrl, (size_t)count * 4, cudaMemcpyDeviceToHost));
+}
+
 pask_status_t pask_debug_dump_high(pask_cache_t *c, int32_t layer, int32_t seq, uint16_t *k_out, uint16_t *v_out,
                                    uint32_t *pages_out, pask_stream_t stream) {
     if (!c || !seq_layer_ok(c, layer, seq)) return PASK_ERR_INVALID_ARG;
@@ -385,7 +393,7 @@ pask_status_t pask_debug_dump_high(pask_cache_t *c, int32_t layer, int32_t seq, 
                 const uint8_t *kt = page.data() + (size_t)h * kHighHeadBytes;
                 const uint8_t *vt = kt + kHighTileBytes;
                 uint16_t *kd = k_out + (tok * n_kv + h) * kHeadDim, *vd = v_out + (tok * n_kv + h) * kHeadDim;
-                for (int ch = 0; ch < 16; ch++) std::memcpy(kd + 8 * ch, kt + high_k_chunk_off((int)tau, ch), 16);
+                for (int pr = 0; pr < 64; pr++) std::memcpy(kd + 2 * pr, kt + high_k_pair_off((int)tau, pr), 4);
                 for (int q = 0; q < 4; q++)
                     for (int g = 0; g < 8; g++)
                         std::memcpy(vd + 32 * q + 4 * g, vt + high_v_piece_off((int)tau, q, g), 8);
@@ -458,17 +466,24 @@ pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, c
     for (int b = 0; b < n_ctas; b++) {
         const uint64_t lo = total * b / n_ctas, hi = total * (b + 1) / n_ctas;
         for (int s = 0; s < n_seqs; s++) {
-            uint32_t *r = ranges + ((size_t)b * n_seqs + s) * 4;
-            r[0] = r[1] = r[2] = r[3] = 0;
+            uint32_t *r = ranges + ((size_t)b * n_seqs + s) * 2;
+            r[0] = r[1] = 0;
             if (prefix[s + 1] <= lo || prefix[s] >= hi || prefix[s + 1] == prefix[s]) continue;
-            const uint32_t cs = (uint32_t)(prefix[s + 1] - prefix[s]);
+            const uint32_t cs = (uint32_t)(prefix[s + 1] - prefix[s]), n = pages_high[s] + pages_low[s];
             const uint32_t a = (uint32_t)((lo > prefix[s] ? lo : prefix[s]) - prefix[s]);
             const uint32_t e = (uint32_t)((hi < prefix[s + 1] ? hi : prefix[s + 1]) - prefix[s]);
-            r[0] = cut_pages(a, cs, pages_high[s]);
-            r[1] = cut_pages(e, cs, pages_high[s]);
-            r[2] = cut_pages(a, cs, pages_low[s]);
-            r[3] = cut_pages(e, cs, pages_low[s]);
+            r[0] = cut_positions(a, cs, n);
+            r[1] = cut_positions(e, cs, n);
         }
+    }
+    return PASK_OK;
+}
+
+pask_status_t pask_debug_page_order(uint32_t pages_high, uint32_t pages_low, uint32_t *order) {
+    if (!order && pages_high + pages_low > 0) return PASK_ERR_INVALID_ARG;
+    for (uint32_t v = 0; v < pages_high + pages_low; v++) {
+        uint32_t idx;
+        order[v] = page_at(v, pages_high, pages_low, idx) ? (idx | kOrderHigh) : idx;
     }
     return PASK_OK;
 }

@@ -247,7 +247,10 @@ append_write_kernel(DevCache c, int layer, int total_tokens, const uint4 *__rest
             uint8_t *dst = c.pool_high + (size_t)page * c.high_page_bytes + (size_t)head * kHighHeadBytes +
                            (which ? kHighTileBytes : 0);
             if (!which) {
-                *reinterpret_cast<uint4 *>(dst + high_k_chunk_off((int)tau, cch)) = x;
+                *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch)) = x.x;
+                *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch + 1)) = x.y;
+                *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch + 2)) = x.z;
+                *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch + 3)) = x.w;
             } else {
                 const int q = cch >> 2, g0 = 2 * (cch & 3);
                 *reinterpret_cast<uint2 *>(dst + high_v_piece_off((int)tau, q, g0)) = make_uint2(x.x, x.y);
@@ -295,6 +298,10 @@ append_write_kernel(DevCache c, int layer, int total_tokens, const uint4 *__rest
                 *reinterpret_cast<uint16_t *>(dst + low_v_half_off((int)tau, w, 2 * u + 1)) = h1;
             }
             if (u == 0) *reinterpret_cast<__half *>(dst + low_scale_off((int)tau, w)) = sh;
+            // decode attention forms P * (V scale) in fp16 relative to the stream's largest V scale:
+            // keep that maximum per (sequence, layer) -- one atomic per warp, and only when it grows
+            const uint32_t hb = __reduce_max_sync(0xffffffffu, which ? (uint32_t)__half_as_ushort(sh) : 0u);
+            if ((tid & 31) == 0 && hb > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb);
         }
     }
 }
@@ -312,7 +319,7 @@ __global__ void __launch_bounds__(256) seq_reset_kernel(DevCache c, int seq) {
         for (uint32_t x = tid; x < ph; x += blockDim.x) c.free_high[bh + x] = c.tbl_high[sl * c.max_pages + x];
         for (uint32_t x = tid; x < pl; x += blockDim.x) c.free_low[bl + x] = c.tbl_low[sl * c.max_pages + x];
         __syncthreads();
-        if (tid == 0) { s_h = bh + ph; s_l = bl + pl; c.n_high[sl] = 0; c.n_low[sl] = 0; }
+        if (tid == 0) { s_h = bh + ph; s_l = bl + pl; c.n_high[sl] = 0; c.n_low[sl] = 0; c.low_vmax[sl] = 0; }
         __syncthreads();
     }
     if (tid == 0) { c.ctrl[kCtrlHighFree] = s_h; c.ctrl[kCtrlLowFree] = s_l; }

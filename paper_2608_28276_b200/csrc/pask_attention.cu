@@ -4,24 +4,33 @@
 // stream holds bf16 K/V, the LOW stream int4 codes with one fp16 scale per 32 dims, read back
 // as (code - 8) * scale.  Released tokens were never stored.
 //
-// Shape of the kernel (B200, sm_100a)
+// Three kernels per call: plan (tiny), attention (streams every retained byte once), combine (tiny).
+//
+// Shape of the attention kernel (B200, sm_100a)
 //   * The work is HBM-bound streaming with a 4-wide GQA group, not a dense contraction, so the
-//     design centres on keeping many bytes in flight: every warp owns a 3-stage shared-memory
-//     ring fed by cp.async.bulk (TMA bulk copies completing on mbarriers) and is its own
-//     producer and consumer -- no block-wide barrier in the streaming loop.
+//     design centres on keeping many bytes in flight and few instructions per byte: every warp
+//     owns a 3-stage shared-memory ring fed by cp.async.bulk (TMA bulk copies completing on
+//     mbarriers) and is its own producer and consumer -- no block-wide barrier in the loop.
 //   * A CTA is n_kv warps; warp w handles KV head w for the CTA's page range, so the four query
 //     heads of a group share every K/V byte and no cross-warp reduction exists at all.
-//   * Sequences are laid end to end in cost space and cut into gridDim.x equal spans
-//     (pask_layout.h), each cut splitting a sequence's HIGH and LOW page lists at the same
-//     fraction, so every CTA streams the same bytes and the same HIGH/LOW mix whatever the lengths;
-//     a span may cover several sequences, each yields one partial (m, l, o) and the ring is not
-//     drained in between.  A second small kernel merges the partials.
+//   * The plan kernel writes, per sequence, its pages in the order they will be visited (HIGH and
+//     LOW pages interleaved evenly, pask_layout.h) and the cost prefix over sequences.  The grid
+//     cuts that cost line into equal spans, so every CTA streams the same bytes and the same
+//     HIGH/LOW mix whatever the length mix; a span may cover several sequences, each yields one
+//     partial (m, l, o) and the ring is not drained in between.  All per-page bookkeeping of the
+//     hot loop is one register shuffle out of a 32-entry window of that list.
 //   * Pages are stored fragment-major (pask_layout.h): a 128-bit shared load per lane is exactly
-//     a tensor-core fragment.  QK^T runs as m16n8k16 bf16 MMAs with tokens on M and the four
-//     query heads (duplicated to fill N = 8) on N; P.V with head dims on M and tokens on K.  All
-//     MMA operands are exact (bf16 values, small integers), accumulation is fp32, and P is split
-//     into bf16 hi + lo parts so that nothing is rounded to 8 bits.  int4 codes are expanded in
-//     registers with one LOP3 per pair (0x4300 | code = 128 + code as bf16).
+//     a tensor-core operand.  QK^T runs as m16n8k16 MMAs with tokens on M and the four query
+//     heads (duplicated to fill N = 8) on N; P.V with head dims on M and tokens on K; fp32
+//     accumulation throughout.
+//   * HIGH pages use bf16 MMAs: K, V and q are exact, P is split into bf16 hi + lo parts.
+//   * LOW pages are bound by the integer/logic pipe that expands nibbles, so that path is built to
+//     need the fewest such instructions: fp16 MMAs, codes expanded with one LOP3 per pair of
+//     values and one shift per eight (0x6400 | code = 1024 + code, 0x6400 | code << 4 =
+//     1024 + 16 code as fp16), the offsets folded into the accumulator's initial value for K and
+//     removed by one half2 subtract / fma for V, K scales applied to the per-group partial scores
+//     in fp32, V scales folded into P (fp16, relative error 2^-12, formed relative to the largest
+//     V scale the stream holds so that no magnitude of V under- or overflows).
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -34,17 +43,29 @@ namespace {
 constexpr int kStages = 3;
 constexpr int kStageBytes = 4096;
 constexpr int kMaxWarps = 8;
+constexpr int kScratchBytes = 1152;              // per warp: fp16 query fragments (1024) + accumulator seeds (128)
 constexpr long long kWaitCycles = 2000000000LL;  // about one second: give up instead of hanging
+constexpr int kPlanThreads = 256;
+
+// workspace of one call
+struct Workspace {
+    uint32_t *cost_prefix;  // [n_seqs + 1] cost of the sequences before s
+    uint32_t *page_prefix;  // [n_seqs + 1] pages of the sequences before s
+    uint2 *tokens;          // [n_seqs] (n_high, n_low) tokens
+    uint32_t *order;        // [page_prefix[n_seqs]] pages in visiting order: kOrderHigh | kOrderTail | page id
+    float2 *part_ml;        // [slots][n_q] (reference maximum in log2 units, sum)
+    float *part_o;          // [slots][n_q][128] unnormalised outputs
+};
 
 struct AttnParams {
     DevCache c;
     int layer, n_seqs;
     const int32_t *seq_ids;
-    const uint4 *q;        // bf16 [n_seqs][n_q][128] viewed as 16-byte chunks
-    uint32_t *prefix_out;  // [n_seqs + 1] cost prefix for the combine kernel
-    float2 *part_ml;       // [slots][n_q] (running max in log2 units, sum)
-    float *part_o;         // [slots][n_q][128] unnormalised outputs
+    const uint4 *q;         // bf16 [n_seqs][n_q][128] viewed as 16-byte chunks
+    Workspace ws;
 };
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---------------------------------------------------------------- PTX helpers
 
@@ -52,9 +73,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)_
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -68,8 +86,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 // Bounded wait: false if the phase did not complete within kWaitCycles.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
@@ -78,28 +95,50 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (clock64() - t0 > kWaitCycles) return false;
     }
 }
-// TMA bulk copy global -> this CTA's shared memory, completion counted on an mbarrier.
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
+// expect_tx + TMA bulk copy global -> this CTA's shared memory, completion counted on an mbarrier;
+// issued by one elected lane of a converged warp (predicated, no divergent branch)
+__device__ __forceinline__ void issue_bulk_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xffffffff;\n\t"
+        "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %2;\n\t"
+        "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
 }
 __device__ __forceinline__ uint4 lds128(uint32_t a) {
     uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
     return v;
 }
 __device__ __forceinline__ uint2 lds64(uint32_t a) {
     uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a) : "memory");
     return v;
 }
-// D = A(16x16, row) * B(16x8, col) + D, bf16 operands, fp32 accumulate
+__device__ __forceinline__ void sts128(uint32_t a, uint4 v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// D = A(16x16, row) * B(16x8, col) + D, fp32 accumulate
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// D = A * B + C with C given as raw register bits (an operand quad straight out of shared memory)
+__device__ __forceinline__ void mma_f16_seed(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1, const uint4 &c) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(__uint_as_float(c.x)), "f"(__uint_as_float(c.y)),
+          "f"(__uint_as_float(c.z)), "f"(__uint_as_float(c.w)));
 }
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     uint32_t d;
@@ -111,188 +150,230 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
     return d;
 }
-// (x >> shift) & 0x000F000F | 0x43004300 : two nibbles -> two bf16 values 128 + code
-__device__ __forceinline__ uint32_t nib2bf16(uint32_t x) {
+// nibbles at bits 0-3 / 16-19 -> two fp16 values 1024 + code
+__device__ __forceinline__ uint32_t nib_even(uint32_t x) {
     uint32_t d;
-    asm("lop3.b32 %0, %1, 0x000F000F, 0x43004300, 0xEA;" : "=r"(d) : "r"(x));
+    asm("lop3.b32 %0, %1, 0x000F000F, 0x64006400, 0xEA;" : "=r"(d) : "r"(x));
     return d;
 }
-__device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
+// nibbles at bits 4-7 / 20-23 -> two fp16 values 1024 + 16 * code
+__device__ __forceinline__ uint32_t nib_odd(uint32_t x) {
     uint32_t d;
-    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    asm("lop3.b32 %0, %1, 0x00F000F0, 0x64006400, 0xEA;" : "=r"(d) : "r"(x));
     return d;
 }
-// two floats -> bf16x2 (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t hsub2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t hmul2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t hfma2(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// two floats -> bf16x2 / f16x2 (lo in the low half), round to nearest even
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t d;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ float2 unpack_f16(uint32_t w) {
+    return __half22float2(*reinterpret_cast<const __half2 *>(&w));
 }
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ float h2f_lo(uint32_t w) { return __half2float(__ushort_as_half((unsigned short)(w & 0xffffu))); }
-__device__ __forceinline__ float h2f_hi(uint32_t w) { return __half2float(__ushort_as_half((unsigned short)(w >> 16))); }
-__device__ __forceinline__ float pick4(uint2 v, int i) {  // i-th fp16 of four
-    const uint32_t w = (i & 2) ? v.y : v.x;
-    return (i & 1) ? h2f_hi(w) : h2f_lo(w);
-}
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 // split x into bf16 hi + bf16 lo (pairs), hi + lo carries 16 mantissa bits
 __device__ __forceinline__ void split_pair(float x0, float x1, uint32_t &hi, uint32_t &lo) {
     hi = pack_bf16(x0, x1);
-    const float r0 = x0 - __uint_as_float(hi << 16);
-    const float r1 = x1 - __uint_as_float(hi & 0xffff0000u);
-    lo = pack_bf16(r0, r1);
+    lo = pack_bf16(x0 - bf_lo(hi), x1 - bf_hi(hi));
 }
 
-// ---------------------------------------------------------------- work partition
+// ---------------------------------------------------------------- plan kernel
 
-struct Segment {
-    uint32_t high_begin, high_count;  // this CTA's run of the sequence's HIGH pages
-    uint32_t low_begin, low_count;    // and of its LOW pages; jobs take the two runs interleaved (PageOrder)
-    uint32_t n_high, n_low;           // tokens in the whole streams (for the ragged tail pages)
-};
-
-__device__ __forceinline__ Segment make_segment(int s, uint32_t lo, uint32_t hi, const uint32_t *s_prefix,
-                                                const uint32_t *s_nh, const uint32_t *s_nl) {
-    Segment g;
-    g.n_high = s_nh[s];
-    g.n_low = s_nl[s];
-    const uint32_t pages_high = (g.n_high + kPageTokens - 1) / kPageTokens;
-    const uint32_t pages_low = (g.n_low + kPageTokens - 1) / kPageTokens;
-    const uint32_t p0 = s_prefix[s], p1 = s_prefix[s + 1], cs = p1 - p0;
-    const uint32_t a = (lo > p0 ? lo : p0) - p0, e = (hi < p1 ? hi : p1) - p0;
-    g.high_begin = cut_pages(a, cs, pages_high);
-    g.high_count = cut_pages(e, cs, pages_high) - g.high_begin;
-    g.low_begin = cut_pages(a, cs, pages_low);
-    g.low_count = cut_pages(e, cs, pages_low) - g.low_begin;
-    return g;
-}
-
-// Order in which a segment's pages are visited: its HIGH and LOW runs are interleaved evenly
-// (page v is a HIGH page iff floor((v+1) nH / n) > floor(v nH / n), n = nH + nL).  HIGH pages are
-// bandwidth-heavy and LOW pages instruction-heavy; taking them in turn lets the bulk copies of
-// the former land while the latter are being decoded, instead of alternating between a
-// memory-bound and an issue-bound phase.
-struct PageOrder {
-    uint32_t rem, hi_idx, lo_idx;
-    __device__ __forceinline__ void reset() { rem = hi_idx = lo_idx = 0; }
-    __device__ __forceinline__ bool is_high(const Segment &g) const { return rem + g.high_count >= g.high_count + g.low_count; }
-    __device__ __forceinline__ void advance(const Segment &g) {
-        if (is_high(g)) { rem -= g.low_count; hi_idx++; }
-        else { rem += g.high_count; lo_idx++; }
+// Cost and page prefixes over the call's sequences, and every sequence's pages in visiting order.
+// Every CTA recomputes the (small) prefix tables in shared memory; CTA 0 publishes them; all CTAs
+// then fill the order list, one thread per page.
+__global__ void __launch_bounds__(kPlanThreads)
+attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ seq_ids, Workspace ws, int has_low) {
+    extern __shared__ uint32_t s_plan[];
+    uint32_t *s_cost = s_plan, *s_page = s_cost + n_seqs + 1, *s_nh = s_page + n_seqs + 1, *s_nl = s_nh + n_seqs;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int s = tid; s < n_seqs; s += kPlanThreads) {
+        const int sid = seq_ids[s];
+        uint32_t nh = 0, nl = 0;
+        if (sid >= 0 && sid < c.max_seqs) {
+            const size_t sl = (size_t)sid * c.n_layers + layer;
+            nh = c.n_high[sl];
+            if (has_low) nl = c.n_low[sl];
+        }
+        s_nh[s] = nh;
+        s_nl[s] = nl;
     }
+    if (tid == 0) s_cost[0] = s_page[0] = 0;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t carry_c = 0, carry_p = 0;
+        for (int base = 0; base < n_seqs; base += 32) {
+            const int idx = base + lane;
+            uint32_t ph = 0, pl = 0;
+            if (idx < n_seqs) { ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens; pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens; }
+            uint32_t ic = ph * kCostHighPage + pl * kCostLowPage, ip = ph + pl;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t oc = __shfl_up_sync(0xffffffffu, ic, d), op = __shfl_up_sync(0xffffffffu, ip, d);
+                if (lane >= d) { ic += oc; ip += op; }
+            }
+            if (idx < n_seqs) { s_cost[idx + 1] = carry_c + ic; s_page[idx + 1] = carry_p + ip; }
+            carry_c += __shfl_sync(0xffffffffu, ic, 31);
+            carry_p += __shfl_sync(0xffffffffu, ip, 31);
+        }
+    }
+    __syncthreads();
+    if (blockIdx.x == 0) {
+        for (int s = tid; s <= n_seqs; s += kPlanThreads) { ws.cost_prefix[s] = s_cost[s]; ws.page_prefix[s] = s_page[s]; }
+        for (int s = tid; s < n_seqs; s += kPlanThreads) ws.tokens[s] = make_uint2(s_nh[s], s_nl[s]);
+    }
+    const uint32_t total_pages = s_page[n_seqs];
+    for (uint32_t gp = blockIdx.x * kPlanThreads + tid; gp < total_pages; gp += gridDim.x * kPlanThreads) {
+        int a = 1, e = n_seqs;   // smallest idx in [1, n_seqs] with s_page[idx] > gp
+        while (a < e) {
+            const int mid = (a + e) >> 1;
+            if (s_page[mid] > gp) e = mid; else a = mid + 1;
+        }
+        const int s = a - 1;
+        const uint32_t nh = s_nh[s], nl = s_nl[s];
+        const uint32_t ph = (nh + kPageTokens - 1) / kPageTokens, pl = (nl + kPageTokens - 1) / kPageTokens;
+        const size_t sl = ((size_t)seq_ids[s] * c.n_layers + layer) * c.max_pages;
+        uint32_t idx, entry;
+        if (page_at(gp - s_page[s], ph, pl, idx)) {
+            entry = c.tbl_high[sl + idx] | kOrderHigh;
+            if (idx == ph - 1 && (nh & (kPageTokens - 1))) entry |= kOrderTail;
+        } else {
+            entry = c.tbl_low[sl + idx];
+            if (idx == pl - 1 && (nl & (kPageTokens - 1))) entry |= kOrderTail;
+        }
+        ws.order[gp] = entry;
+    }
+}
+
+// ---------------------------------------------------------------- attention kernel
+
+// A CTA's share of one sequence: positions [begin, end) of its page order list.
+struct Segment {
+    uint32_t begin, end;      // global indices into ws.order
+    uint32_t n_high, n_low;   // tokens in the whole streams (for the ragged tail pages)
 };
 
-// Producer side of a warp's pipeline: walks the CTA's pages in order and issues one bulk copy
-// per job (HIGH page: K tile, then V tile; LOW page: K and V halves together).
-struct Producer {
-    int s;                    // current sequence index in the call, n_seqs when exhausted
-    Segment seg;
-    PageOrder ord;
-    uint32_t page;            // next job's page: position in the segment's interleaved order
-    uint32_t sub;             // 0: K tile next, 1: V tile next (HIGH pages)
-    uint32_t win_base, win_id;  // 32 page ids cached across the lanes, starting at win_base
-    bool win_valid;
-};
-
-template <bool kHasLow>
-struct Warp {
-    const AttnParams &p;
-    const uint32_t *s_prefix, *s_nh, *s_nl;
-    uint32_t lo, hi;
-    int lane, kv;
+// Per-warp pipeline.  The producer side walks the CTA's positions and issues one bulk copy per job
+// (HIGH page: K tile, then V tile; LOW page: K and V halves together); the consumer side waits for
+// the jobs in the same order.  Both read page entries out of 32-entry register windows.
+struct Pipe {
+    const AttnParams *p;
+    const uint32_t *s_cost, *s_page;
+    uint32_t lo, hi;          // the CTA's span in cost space
+    int lane;
+    uint32_t head_high, head_low;   // this warp's head offset inside a page, in 256-byte units
+    uint32_t n_kv_high, n_kv_low;   // page size in 256-byte units
     uint32_t ring, bars;      // shared-space addresses of this warp's stages and mbarriers
-    Producer pr;
-    uint32_t issued, consumed;
+    // producer
+    int ps;                   // sequence index the producer is in
+    uint32_t p_pos, p_end;    // next position and end of its segment (global indices into ws.order)
+    uint32_t p_sub;           // 0: K tile next, 1: V tile next (HIGH pages)
+    uint32_t pw_base, pw_entry;
+    uint32_t p_stage;
+    // consumer
+    uint32_t c_stage, c_parity;
+    uint32_t outstanding;
     bool dead;
 
-    __device__ __forceinline__ bool in_span(int s) const { return s < p.n_seqs && s_prefix[s] < hi; }
+    __device__ __forceinline__ bool in_span(int s) const { return s < p->n_seqs && s_cost[s] < hi; }
 
-    __device__ __forceinline__ void producer_open(int s) {
-        // advance to the next sequence of the span that has pages for this CTA
-        for (; in_span(s); ++s) {
-            if (s_prefix[s + 1] == s_prefix[s]) continue;
-            pr.seg = make_segment(s, lo, hi, s_prefix, s_nh, s_nl);
-            if (pr.seg.high_count + pr.seg.low_count > 0) break;
-        }
-        if (!in_span(s)) s = p.n_seqs;
-        pr.s = s;
-        pr.page = 0;
-        pr.sub = 0;
-        pr.ord.reset();
-        pr.win_valid = false;
+    __device__ __forceinline__ void segment_of(int s, uint32_t &begin, uint32_t &end) const {
+        const uint32_t c0 = s_cost[s], c1 = s_cost[s + 1], cs = c1 - c0, n = s_page[s + 1] - s_page[s];
+        const uint32_t a = (lo > c0 ? lo : c0) - c0, e = (hi < c1 ? hi : c1) - c0;
+        begin = s_page[s] + cut_positions(a, cs, n);
+        end = s_page[s] + cut_positions(e, cs, n);
     }
 
-    // Issue the next job into stage (issued % kStages).  Warp-uniform; lane 0 talks to the TMA.
-    __device__ __forceinline__ void produce() {
-        if (pr.s >= p.n_seqs) return;
-        const DevCache &c = p.c;
-        const bool is_high = pr.ord.is_high(pr.seg);
-        const uint32_t n_pages = pr.seg.high_count + pr.seg.low_count;
-        if (!pr.win_valid || pr.page - pr.win_base >= 32u) {
-            // refill the page-id window: lane i holds the id of the page at position win_base + i
-            pr.win_base = pr.page;
-            pr.win_valid = true;
-            const uint32_t pg = pr.page + lane;
-            const size_t sl = ((size_t)p.seq_ids[pr.s] * c.n_layers + p.layer) * c.max_pages;
-            uint32_t id = 0;
-            if (pg < n_pages) {
-                const uint32_t h0 = (uint32_t)(((uint64_t)pg * pr.seg.high_count) / n_pages);
-                const uint32_t h1 = (uint32_t)(((uint64_t)(pg + 1) * pr.seg.high_count) / n_pages);
-                id = h1 > h0 ? c.tbl_high[sl + pr.seg.high_begin + h0] : c.tbl_low[sl + pr.seg.low_begin + (pg - h0)];
-            }
-            pr.win_id = id;
+    // advance the producer to the next sequence of the span that has pages for this CTA
+    __device__ __forceinline__ void producer_open(int s) {
+        for (; in_span(s); ++s) {
+            if (s_cost[s + 1] == s_cost[s]) continue;
+            segment_of(s, p_pos, p_end);
+            if (p_pos < p_end) break;
         }
-        const uint32_t id = __shfl_sync(0xffffffffu, pr.win_id, (int)(pr.page - pr.win_base));
-        const uint32_t stage = issued % kStages;
+        if (!in_span(s)) { s = p->n_seqs; p_pos = p_end = 0; }
+        ps = s;
+        p_sub = 0;
+        pw_base = 0x80000000u;   // forces a window refill at the first job
+    }
+
+    // Issue the next job into stage p_stage.  Warp-uniform.
+    __device__ __forceinline__ void produce() {
+        if (p_pos == p_end) return;
+        if (p_pos - pw_base >= 32u) {
+            pw_base = p_pos;
+            pw_entry = p_pos + lane < p_end ? __ldg(p->ws.order + p_pos + lane) : 0u;
+        }
+        const uint32_t entry = __shfl_sync(0xffffffffu, pw_entry, (int)(p_pos - pw_base));
+        const uint32_t id = entry & kOrderIdMask;
+        const bool is_high = entry & kOrderHigh;
         const uint8_t *src;
         uint32_t bytes;
         if (is_high) {
-            src = c.pool_high + (size_t)id * c.high_page_bytes + (size_t)kv * kHighHeadBytes + pr.sub * kHighTileBytes;
+            src = p->c.pool_high + (size_t)(id * n_kv_high + head_high + p_sub * (kHighTileBytes / 256)) * 256;
             bytes = kHighTileBytes;
         } else {
-            src = c.pool_low + (size_t)id * c.low_page_bytes + (size_t)kv * kLowHeadBytes;
+            src = p->c.pool_low + (size_t)(id * n_kv_low + head_low) * 256;
             bytes = kLowHeadBytes;
         }
-        if (lane == 0) {
-            const uint32_t bar = bars + stage * 8;
-            mbar_expect_tx(bar, bytes);
-            bulk_g2s(ring + stage * kStageBytes, src, bytes, bar);
-        }
-        issued++;
-        if (is_high && pr.sub == 0) {
-            pr.sub = 1;
+        issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bars + p_stage * 8);
+        p_stage = p_stage + 1 == kStages ? 0 : p_stage + 1;
+        outstanding++;
+        if (is_high && p_sub == 0) {
+            p_sub = 1;
         } else {
-            pr.sub = 0;
-            pr.ord.advance(pr.seg);
-            if (++pr.page == n_pages) producer_open(pr.s + 1);
+            p_sub = 0;
+            if (++p_pos == p_end) producer_open(ps + 1);
         }
     }
 
     // Wait for the oldest outstanding job; returns the shared address of its stage.
     __device__ __forceinline__ uint32_t acquire() {
-        const uint32_t stage = consumed % kStages, parity = (consumed / kStages) & 1u;
-        if (!dead && !mbar_wait(bars + stage * 8, parity)) {
-            dead = true;
-            if (lane == 0) atomicOr(&p.c.ctrl[kCtrlStatus], PASK_DEV_TIMEOUT);
+        const uint32_t bar = bars + c_stage * 8;
+        if (!mbar_try_wait(bar, c_parity)) {
+            if (dead || !mbar_wait_slow(bar, c_parity)) {
+                if (!dead && lane == 0) atomicOr(&p->c.ctrl[kCtrlStatus], PASK_DEV_TIMEOUT);
+                dead = true;
+            }
         }
-        return ring + stage * kStageBytes;
+        return ring + c_stage * kStageBytes;
     }
     // All lanes are done reading the oldest stage: hand it back to the producer.
     __device__ __forceinline__ void release() {
         __syncwarp();
-        if (!dead) {
-            consumed++;
-            produce();
-        }
+        outstanding--;
+        if (++c_stage == kStages) { c_stage = 0; c_parity ^= 1u; }
+        if (!dead) produce();
     }
 };
-
-// ---------------------------------------------------------------- the kernel
 
 template <bool kHasLow>
 __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __grid_constant__ AttnParams p) {
@@ -302,68 +383,45 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     const int g = lane >> 2, t = lane & 3;
     const int n_seqs = p.n_seqs;
 
-    uint32_t *s_prefix = reinterpret_cast<uint32_t *>(smem);
-    uint32_t *s_nh = s_prefix + n_seqs + 1;
-    uint32_t *s_nl = s_nh + n_seqs;
-    size_t off = ((size_t)(3 * n_seqs + 1) * 4 + 127) & ~(size_t)127;
+    uint32_t *s_cost = reinterpret_cast<uint32_t *>(smem);
+    uint32_t *s_page = s_cost + n_seqs + 1;
+    size_t off = ((size_t)(2 * n_seqs + 2) * 4 + 127) & ~(size_t)127;
     uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + off);
     off += 256;                                             // kMaxWarps * kStages * 8 = 192 bytes of barriers
     off = (off + 1023) & ~(size_t)1023;
     uint8_t *s_ring = smem + off;
+    uint8_t *s_scratch = s_ring + (size_t)n_warps * kStages * kStageBytes;
 
-    // ---- per-sequence costs and their prefix sum (every CTA computes the same table)
-    for (int s = tid; s < n_seqs; s += blockDim.x) {
-        const int sid = p.seq_ids[s];
-        uint32_t nh = 0, nl = 0;
-        if (sid >= 0 && sid < c.max_seqs) {
-            const size_t sl = (size_t)sid * c.n_layers + p.layer;
-            nh = c.n_high[sl];
-            if (kHasLow) nl = c.n_low[sl];
-        }
-        s_nh[s] = nh;
-        s_nl[s] = nl;
-        s_prefix[s + 1] = ((nh + kPageTokens - 1) / kPageTokens) * kCostHighPage +
-                          ((nl + kPageTokens - 1) / kPageTokens) * kCostLowPage;
-    }
-    if (tid == 0) s_prefix[0] = 0;
-    __syncthreads();
-    if (warp == 0) {
-        uint32_t carry = 0;
-        for (int base = 0; base < n_seqs; base += 32) {
-            const int idx = base + lane;
-            uint32_t inc = idx < n_seqs ? s_prefix[idx + 1] : 0u;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t o = __shfl_up_sync(0xffffffffu, inc, d);
-                if (lane >= d) inc += o;
-            }
-            if (idx < n_seqs) s_prefix[idx + 1] = carry + inc;
-            carry += __shfl_sync(0xffffffffu, inc, 31);
-        }
+    for (int s = tid; s <= n_seqs; s += blockDim.x) {
+        s_cost[s] = __ldg(p.ws.cost_prefix + s);
+        s_page[s] = __ldg(p.ws.page_prefix + s);
     }
     __syncthreads();
-    const uint32_t total = s_prefix[n_seqs];
-    if (blockIdx.x == 0)
-        for (int s = tid; s <= n_seqs; s += blockDim.x) p.prefix_out[s] = s_prefix[s];
+    const uint32_t total = s_cost[n_seqs];
     if (total == 0) return;
 
     const uint32_t n_ctas = gridDim.x, b = blockIdx.x;
     const uint32_t lo = (uint32_t)(((uint64_t)total * b) / n_ctas);
     const uint32_t hi = (uint32_t)(((uint64_t)total * (b + 1)) / n_ctas);
-    // first sequence of the span: prefix[s0] <= lo < prefix[s0 + 1]
+    // first sequence of the span: cost[s0] <= lo < cost[s0 + 1]
     int s0;
     {
-        int a = 1, e = n_seqs;  // smallest idx in [1, n_seqs] with prefix[idx] > lo
+        int a = 1, e = n_seqs;  // smallest idx in [1, n_seqs] with cost[idx] > lo
         while (a < e) {
             const int mid = (a + e) >> 1;
-            if (s_prefix[mid] > lo) e = mid; else a = mid + 1;
+            if (s_cost[mid] > lo) e = mid; else a = mid + 1;
         }
         s0 = a - 1;
     }
 
-    Warp<kHasLow> w{p, s_prefix, s_nh, s_nl, lo, hi, lane, warp,
-                    smem_u32(s_ring + (size_t)warp * kStages * kStageBytes), smem_u32(s_bar + warp * kStages),
-                    {}, 0u, 0u, false};
+    Pipe w;
+    w.p = &p; w.s_cost = s_cost; w.s_page = s_page; w.lo = lo; w.hi = hi; w.lane = lane;
+    w.n_kv_high = (uint32_t)c.n_kv * (kHighHeadBytes / 256); w.head_high = (uint32_t)warp * (kHighHeadBytes / 256);
+    w.n_kv_low = (uint32_t)c.n_kv * (kLowHeadBytes / 256); w.head_low = (uint32_t)warp * (kLowHeadBytes / 256);
+    w.ring = smem_u32(s_ring + (size_t)warp * kStages * kStageBytes);
+    w.bars = smem_u32(s_bar + warp * kStages);
+    w.p_stage = 0; w.c_stage = 0; w.c_parity = 0; w.outstanding = 0; w.dead = false;
+    const uint32_t scratch = smem_u32(s_scratch + (size_t)warp * kScratchBytes);
     if (lane == 0) {
         for (int i = 0; i < kStages; i++) mbar_init(w.bars + i * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -374,13 +432,21 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     for (int i = 0; i < kStages; i++) w.produce();
 
     const float kLog2Scale = 0.088388347648318440550f * 1.4426950408889634074f;  // log2(e) / sqrt(128)
+    const float kSlack = 6.0f;               // log2 units a score may exceed the reference maximum by
     const int head_a = 2 * (t & 1);          // this lane's two score / output columns are heads a, a + 1
     const int qh0 = warp * 4;                // first query head of this KV head
-    const uint32_t slot_bias = b;
+    // selector that broadcasts the fp16 scale of this lane's column group (low or high half of a word)
+    const uint32_t bsel = (t >> 1) ? 0x3232u : 0x1010u;
 
     for (int s = s0; w.in_span(s); ++s) {
-        if (s_prefix[s + 1] == s_prefix[s]) continue;
-        const Segment seg = make_segment(s, lo, hi, s_prefix, s_nh, s_nl);
+        if (s_cost[s + 1] == s_cost[s]) continue;
+        Segment seg;
+        w.segment_of(s, seg.begin, seg.end);
+        {
+            const uint2 tk = __ldg(p.ws.tokens + s);
+            seg.n_high = tk.x;
+            seg.n_low = tk.y;
+        }
 
         // ---- query fragments: lane (g,t) holds dims 8(4j+t) .. +7 of head g & 3 for j = 0..3
         uint4 qf[4];
@@ -389,21 +455,51 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
 #pragma unroll
             for (int j = 0; j < 4; j++) qf[j] = __ldg(qrow + 4 * j + t);
         }
-        // -136 * sum of q over each 32-dim group, for this lane's two heads (initial accumulator of
-        // the LOW-stream QK^T, which multiplies q with 128 + code instead of code - 8)
-        float nq[4][2];
-        if (kHasLow) {
+        // P * (V scale) is formed in fp16 relative to the largest V scale the stream holds: everything
+        // that feeds the output accumulators of this segment is multiplied by `down` = 2^k (the
+        // scales of LOW tokens, P of HIGH tokens) and the partial is multiplied by `up` = 2^-k.
+        uint32_t down = 0x3C003C00u;
+        float down_f = 1.0f, up = 1.0f;
+        if (kHasLow && seg.n_low > 0) {
+            // fp16 copies of q for the LOW stream's MMAs.  Its A operands are 1024 + code (register
+            // pairs x, z of a chunk) and 1024 + 16 code (pairs y, w), so q is stored as is for the
+            // former and divided by 16 for the latter, and -(1032 b) resp. -(1152 b) summed over a
+            // 32-dim group seeds the accumulator so that what comes out is sum q (code - 8).
+            __syncwarp();
+            bool too_big = false;
 #pragma unroll
             for (int j = 0; j < 4; j++) {
                 const uint32_t r[4] = {qf[j].x, qf[j].y, qf[j].z, qf[j].w};
-                float sum = 0.f;
+                uint32_t h[4];
+                float seed = 0.f;
 #pragma unroll
-                for (int i = 0; i < 4; i++) sum += __uint_as_float(r[i] << 16) + __uint_as_float(r[i] & 0xffff0000u);
-                sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-                sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-                nq[j][0] = -136.f * __shfl_sync(0xffffffffu, sum, 4 * head_a);
-                nq[j][1] = -136.f * __shfl_sync(0xffffffffu, sum, 4 * (head_a + 1));
+                for (int i = 0; i < 4; i++) {
+                    const float f0 = bf_lo(r[i]), f1 = bf_hi(r[i]);
+                    too_big |= fabsf(f0) > 65504.f || fabsf(f1) > 65504.f;
+                    const float sc = (i & 1) ? 0.0625f : 1.0f;
+                    h[i] = pack_f16(f0 * sc, f1 * sc);
+                    const float2 bq = unpack_f16(h[i]);
+                    seed -= ((i & 1) ? 1152.f : 1032.f) * (bq.x + bq.y);
+                }
+                seed += __shfl_xor_sync(0xffffffffu, seed, 1);
+                seed += __shfl_xor_sync(0xffffffffu, seed, 2);
+                // the seed of head a+1 sits one 4-lane row further on
+                const float seed_b = __shfl_down_sync(0xffffffffu, seed, 4);
+                if (g < 4) sts128(scratch + j * 256 + g * 64 + t * 16, make_uint4(h[0], h[1], h[2], h[3]));
+                // accumulator quads {seed[a], seed[a+1], seed[a], seed[a+1]} of head pairs (0,1) and (2,3)
+                if (t == 0 && (g == 0 || g == 2)) {
+                    const uint32_t sa = __float_as_uint(seed), sb = __float_as_uint(seed_b);
+                    sts128(scratch + 1024 + ((g >> 1) * 4 + j) * 16, make_uint4(sa, sb, sa, sb));
+                }
             }
+            if (__any_sync(0xffffffffu, too_big) && lane == 0) atomicOr(&c.ctrl[kCtrlStatus], PASK_DEV_RANGE);
+            const uint32_t vmax = c.low_vmax[(size_t)p.seq_ids[s] * c.n_layers + p.layer];   // fp16 bits
+            const int k = max(15 - (int)(vmax >> 10), -14);
+            down = (uint32_t)(15 + k) << 10;
+            down |= down << 16;
+            down_f = __int_as_float((127 + k) << 23);
+            up = __int_as_float((127 - k) << 23);
+            __syncwarp();
         }
 
         float acc[8][4];
@@ -411,13 +507,16 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         for (int m = 0; m < 8; m++) acc[m][0] = acc[m][1] = acc[m][2] = acc[m][3] = 0.f;
         float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
 
-        PageOrder ord;
-        ord.reset();
-        for (uint32_t page = 0; page < seg.high_count + seg.low_count; ++page, ord.advance(seg)) {
-            const bool is_high = ord.is_high(seg);
-            uint32_t n_valid;
-            if (is_high) n_valid = min(16u, seg.n_high - (seg.high_begin + ord.hi_idx) * kPageTokens);
-            else n_valid = min(16u, seg.n_low - (seg.low_begin + ord.lo_idx) * kPageTokens);
+        uint32_t cw_base = 0x80000000u, cw_entry = 0;
+        for (uint32_t pos = seg.begin; pos < seg.end; ++pos) {
+            if (pos - cw_base >= 32u) {
+                cw_base = pos;
+                cw_entry = pos + lane < seg.end ? __ldg(p.ws.order + pos + lane) : 0u;
+            }
+            const uint32_t entry = __shfl_sync(0xffffffffu, cw_entry, (int)(pos - cw_base));
+            const bool is_high = entry & kOrderHigh;
+            uint32_t n_valid = 16u;
+            if (entry & kOrderTail) n_valid = (is_high ? seg.n_high : seg.n_low) & (kPageTokens - 1);
 
             float sc[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t st = w.acquire();
@@ -427,10 +526,10 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 float sc2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
-                    const uint4 k0 = lds128(st + (2 * j) * 512 + lane * 16);      // token g
-                    const uint4 k1 = lds128(st + (2 * j + 1) * 512 + lane * 16);  // token g + 8
-                    mma_bf16(sc, k0.x, k1.x, k0.y, k1.y, qf[j].x, qf[j].y);
-                    mma_bf16(sc2, k0.z, k1.z, k0.w, k1.w, qf[j].z, qf[j].w);
+                    const uint4 ka = lds128(st + (2 * j) * 512 + lane * 16);      // operand quad, dims 8c .. 8c+3
+                    const uint4 kb = lds128(st + (2 * j + 1) * 512 + lane * 16);  // dims 8c+4 .. 8c+7
+                    mma_bf16(sc, ka.x, ka.y, ka.z, ka.w, qf[j].x, qf[j].y);
+                    mma_bf16(sc2, kb.x, kb.y, kb.z, kb.w, qf[j].z, qf[j].w);
                 }
 #pragma unroll
                 for (int i = 0; i < 4; i++) sc[i] += sc2[i];
@@ -441,34 +540,43 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 const uint2 ks0 = lds64(st + kLowCodesBytes + g * 8);
                 const uint2 ks1 = lds64(st + kLowCodesBytes + (g + 8) * 8);
                 const uint32_t w0[4] = {k0.x, k0.y, k0.z, k0.w}, w1[4] = {k1.x, k1.y, k1.z, k1.w};
+                const float2 f0[2] = {unpack_f16(ks0.x), unpack_f16(ks0.y)};
+                const float2 f1[2] = {unpack_f16(ks1.x), unpack_f16(ks1.y)};
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
-                    float cj[4] = {nq[j][0], nq[j][1], nq[j][0], nq[j][1]};
-                    mma_bf16(cj, nib2bf16(w0[j]), nib2bf16(w1[j]), nib2bf16(w0[j] >> 4), nib2bf16(w1[j] >> 4),
-                             qf[j].x, qf[j].y);
-                    mma_bf16(cj, nib2bf16(w0[j] >> 8), nib2bf16(w1[j] >> 8), nib2bf16(w0[j] >> 12),
-                             nib2bf16(w1[j] >> 12), qf[j].z, qf[j].w);
-                    const float f0 = pick4(ks0, j), f1 = pick4(ks1, j);
-                    sc[0] = fmaf(f0, cj[0], sc[0]);
-                    sc[1] = fmaf(f0, cj[1], sc[1]);
-                    sc[2] = fmaf(f1, cj[2], sc[2]);
-                    sc[3] = fmaf(f1, cj[3], sc[3]);
+                    const uint4 qa = lds128(scratch + j * 256 + (g & 3) * 64 + t * 16);
+                    const uint4 seed = lds128(scratch + 1024 + ((t & 1) * 4 + j) * 16);
+                    float cj[4];
+                    const uint32_t u0 = w0[j] >> 8, u1 = w1[j] >> 8;
+                    mma_f16_seed(cj, nib_even(w0[j]), nib_even(w1[j]), nib_odd(w0[j]), nib_odd(w1[j]), qa.x, qa.y, seed);
+                    mma_f16(cj, nib_even(u0), nib_even(u1), nib_odd(u0), nib_odd(u1), qa.z, qa.w);
+                    const float s0f = (j & 1) ? f0[j >> 1].y : f0[j >> 1].x;
+                    const float s1f = (j & 1) ? f1[j >> 1].y : f1[j >> 1].x;
+                    sc[0] = fmaf(s0f, cj[0], sc[0]);
+                    sc[1] = fmaf(s0f, cj[1], sc[1]);
+                    sc[2] = fmaf(s1f, cj[2], sc[2]);
+                    sc[3] = fmaf(s1f, cj[3], sc[3]);
                 }
             }
 
             // ---- online softmax for heads a, a+1 over tokens g and g + 8 of the tile
+            // The reference maxima m_a, m_b are only raised when some score of the tile exceeds them by
+            // more than kSlack (then to the true running maximum): weights stay below 2^kSlack, and
+            // the cross-lane reduction and the rescaling of the accumulators leave the common path.
             float z0 = sc[0] * kLog2Scale, z1 = sc[1] * kLog2Scale, z2 = sc[2] * kLog2Scale, z3 = sc[3] * kLog2Scale;
-            if ((uint32_t)g >= n_valid) z0 = z1 = -INFINITY;
-            if ((uint32_t)g + 8u >= n_valid) z2 = z3 = -INFINITY;
-            float ta = fmaxf(z0, z2), tb = fmaxf(z1, z3);
-#pragma unroll
-            for (int d = 4; d < 32; d <<= 1) {
-                ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, d));
-                tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, d));
+            if (n_valid < 16u) {
+                if ((uint32_t)g >= n_valid) z0 = z1 = -INFINITY;
+                if ((uint32_t)g + 8u >= n_valid) z2 = z3 = -INFINITY;
             }
-            const float mna = fmaxf(m_a, ta), mnb = fmaxf(m_b, tb);
-            if (__any_sync(0xffffffffu, mna > m_a || mnb > m_b)) {
-                const float fa = ex2(m_a - mna), fb = ex2(m_b - mnb);
+            float ta = fmaxf(z0, z2), tb = fmaxf(z1, z3);
+            if (__any_sync(0xffffffffu, ta > m_a + kSlack || tb > m_b + kSlack)) {
+#pragma unroll
+                for (int d = 4; d < 32; d <<= 1) {
+                    ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, d));
+                    tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, d));
+                }
+                const float mna = fmaxf(m_a, ta), mnb = fmaxf(m_b, tb);
+                const float fa = mna == -INFINITY ? 1.f : ex2(m_a - mna), fb = mnb == -INFINITY ? 1.f : ex2(m_b - mnb);
 #pragma unroll
                 for (int m = 0; m < 8; m++) { acc[m][0] *= fa; acc[m][2] *= fa; acc[m][1] *= fb; acc[m][3] *= fb; }
                 l_a *= fa; l_b *= fb;
@@ -481,8 +589,8 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
             if (is_high) {
                 // ---- P (hi + lo) as the B operand: transpose the score fragment's layout
                 uint32_t h01, l01, h23, l23;
-                split_pair(p0, p1, h01, l01);
-                split_pair(p2, p3, h23, l23);
+                split_pair(p0 * down_f, p1 * down_f, h01, l01);
+                split_pair(p2 * down_f, p3 * down_f, h23, l23);
                 const uint32_t bh0 = movmatrix_trans(h01), bh1 = movmatrix_trans(h23);
                 const uint32_t bl0 = movmatrix_trans(l01), bl1 = movmatrix_trans(l23);
                 st = w.acquire();
@@ -515,38 +623,38 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 uint2 vs0 = lds64(vb + kLowCodesBytes + g * 8);
                 uint2 vs1 = lds64(vb + kLowCodesBytes + (g + 8) * 8);
                 w.release();   // everything of this stage is in registers now
-                if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
-                if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
+                if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
+                    if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
+                    if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
+                }
                 const uint32_t c0[4] = {v0.x, v0.y, v0.z, v0.w}, c1[4] = {v1.x, v1.y, v1.z, v1.w};
+                const uint32_t p01 = pack_f16(p0, p1), p23 = pack_f16(p2, p3);
 #pragma unroll
                 for (int v = 0; v < 2; v++) {
                     // B columns 0-3: heads x group 2v, columns 4-7: heads x group 2v + 1
-                    const int grp = 2 * v + (t >> 1);
-                    const float f0 = pick4(vs0, grp), f1 = pick4(vs1, grp);
-                    uint32_t h01, l01, h23, l23;
-                    split_pair(p0 * f0, p1 * f0, h01, l01);
-                    split_pair(p2 * f1, p3 * f1, h23, l23);
-                    const uint32_t bh0 = movmatrix_trans(h01), bh1 = movmatrix_trans(h23);
-                    const uint32_t bl0 = movmatrix_trans(l01), bl1 = movmatrix_trans(l23);
+                    const uint32_t s0b = hmul2(prmt(v ? vs0.y : vs0.x, 0u, bsel), down);
+                    const uint32_t s1b = hmul2(prmt(v ? vs1.y : vs1.x, 0u, bsel), down);
+                    const uint32_t b0 = movmatrix_trans(hmul2(p01, s0b)), b1 = movmatrix_trans(hmul2(p23, s1b));
 #pragma unroll
                     for (int qq = 0; qq < 2; qq++) {
                         const int q = 2 * v + qq;
+                        const uint32_t e0 = c0[q] >> 8, e1 = c1[q] >> 8;
                         uint32_t a[2][4];
+                        a[0][0] = hsub2(nib_even(c0[q]), 0x64086408u);               // (1024 + code) - 1032
+                        a[0][1] = hfma2(nib_odd(c0[q]), 0x2C002C00u, 0xD480D480u);   // (1024 + 16 code) / 16 - 72
+                        a[0][2] = hsub2(nib_even(e0), 0x64086408u);
+                        a[0][3] = hfma2(nib_odd(e0), 0x2C002C00u, 0xD480D480u);
+                        a[1][0] = hsub2(nib_even(c1[q]), 0x64086408u);
+                        a[1][1] = hfma2(nib_odd(c1[q]), 0x2C002C00u, 0xD480D480u);
+                        a[1][2] = hsub2(nib_even(e1), 0x64086408u);
+                        a[1][3] = hfma2(nib_odd(e1), 0x2C002C00u, 0xD480D480u);
 #pragma unroll
-                        for (int i = 0; i < 4; i++) {
-                            a[0][i] = sub_bf16x2(nib2bf16(c0[q] >> (4 * i)), 0x43084308u);  // (128 + code) - 136
-                            a[1][i] = sub_bf16x2(nib2bf16(c1[q] >> (4 * i)), 0x43084308u);
-                        }
-#pragma unroll
-                        for (int r = 0; r < 2; r++) {
-                            mma_bf16(acc[2 * q + r], a[0][2 * r], a[0][2 * r + 1], a[1][2 * r], a[1][2 * r + 1], bh0, bh1);
-                            mma_bf16(acc[2 * q + r], a[0][2 * r], a[0][2 * r + 1], a[1][2 * r], a[1][2 * r + 1], bl0, bl1);
-                        }
+                        for (int r = 0; r < 2; r++)
+                            mma_f16(acc[2 * q + r], a[0][2 * r], a[0][2 * r + 1], a[1][2 * r], a[1][2 * r + 1], b0, b1);
                     }
                 }
             }
         }
-
         if (w.dead) break;   // a wait ran out: results are void, the status word says so
 
         // ---- this segment's partial: (m, l) per head, unnormalised o
@@ -555,19 +663,19 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
             l_a += __shfl_xor_sync(0xffffffffu, l_a, d);
             l_b += __shfl_xor_sync(0xffffffffu, l_b, d);
         }
-        const size_t slot = (size_t)slot_bias + s;
+        const size_t slot = (size_t)b + s;
         const size_t hrow = slot * c.n_q + qh0 + head_a;
         if (g == 0 && t < 2) {
-            p.part_ml[hrow] = make_float2(m_a, l_a);
-            p.part_ml[hrow + 1] = make_float2(m_b, l_b);
+            p.ws.part_ml[hrow] = make_float2(m_a, l_a);
+            p.ws.part_ml[hrow + 1] = make_float2(m_b, l_b);
         }
 #pragma unroll
         for (int m = 0; m < 8; m++) {
             const int q = m >> 1, r = m & 1;
             if ((t >> 1) == (q & 1)) {   // even groups are valid in columns 0-3, odd groups in 4-7
                 const int dim = 32 * q + 4 * g + 2 * r;
-                *reinterpret_cast<float2 *>(p.part_o + hrow * kHeadDim + dim) = make_float2(acc[m][0], acc[m][2]);
-                *reinterpret_cast<float2 *>(p.part_o + (hrow + 1) * kHeadDim + dim) = make_float2(acc[m][1], acc[m][3]);
+                *reinterpret_cast<float2 *>(p.ws.part_o + hrow * kHeadDim + dim) = make_float2(acc[m][0] * up, acc[m][2] * up);
+                *reinterpret_cast<float2 *>(p.ws.part_o + (hrow + 1) * kHeadDim + dim) = make_float2(acc[m][1] * up, acc[m][3] * up);
             }
         }
     }
@@ -575,10 +683,11 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     // A wait gave up: copies may still be in flight towards this CTA's shared memory.  Give each
     // outstanding stage one more bounded wait before the CTA retires.
     if (w.dead) {
-        while (w.consumed < w.issued) {
-            const uint32_t stage = w.consumed % kStages, parity = (w.consumed / kStages) & 1u;
-            mbar_wait(w.bars + stage * 8, parity);
-            w.consumed++;
+        while (w.outstanding > 0) {
+            const uint32_t bar = w.bars + w.c_stage * 8;
+            if (!mbar_try_wait(bar, w.c_parity)) mbar_wait_slow(bar, w.c_parity);
+            if (++w.c_stage == kStages) { w.c_stage = 0; w.c_parity ^= 1u; }
+            w.outstanding--;
         }
     }
 }
@@ -619,50 +728,61 @@ combine_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ p
     if (lse && lane == 0) lse[orow] = L > 0.f ? (M + log2f(L)) * 0.69314718055994530942f : -INFINITY;
 }
 
-inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
 size_t attn_smem_bytes(int n_seqs, int n_warps) {
-    size_t off = align_up((size_t)(3 * n_seqs + 1) * 4, 128) + 256;
+    size_t off = align_up((size_t)(2 * n_seqs + 2) * 4, 128) + 256;
     off = align_up(off, 1024);
-    return off + (size_t)n_warps * kStages * kStageBytes;
+    return off + (size_t)n_warps * (kStages * kStageBytes + kScratchBytes);
+}
+
+// carve the caller's workspace
+size_t carve_workspace(const pask_cache *c, int n_seqs, uint8_t *base, Workspace *ws) {
+    const size_t slots = (size_t)c->attn_ctas + n_seqs;
+    const size_t max_pages = (size_t)n_seqs * 2 * c->dev.max_pages;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
+    const size_t o_cost = take((size_t)(n_seqs + 1) * 4), o_page = take((size_t)(n_seqs + 1) * 4);
+    const size_t o_tok = take((size_t)n_seqs * sizeof(uint2)), o_order = take(max_pages * 4);
+    const size_t o_ml = take(slots * c->desc.n_q_heads * sizeof(float2));
+    const size_t o_o = take(slots * c->desc.n_q_heads * kHeadDim * sizeof(float));
+    if (ws) {
+        ws->cost_prefix = reinterpret_cast<uint32_t *>(base + o_cost);
+        ws->page_prefix = reinterpret_cast<uint32_t *>(base + o_page);
+        ws->tokens = reinterpret_cast<uint2 *>(base + o_tok);
+        ws->order = reinterpret_cast<uint32_t *>(base + o_order);
+        ws->part_ml = reinterpret_cast<float2 *>(base + o_ml);
+        ws->part_o = reinterpret_cast<float *>(base + o_o);
+    }
+    return off;
 }
 
 }  // namespace
 
 int attention_grid(const pask_cache *c) { return 2 * c->sm_count; }
 
-size_t attention_workspace_bytes(const pask_cache *c, int n_seqs) {
-    const size_t slots = (size_t)c->attn_ctas + n_seqs;
-    return align_up((size_t)(n_seqs + 1) * 4, 256) + align_up(slots * c->desc.n_q_heads * sizeof(float2), 256) +
-           slots * c->desc.n_q_heads * kHeadDim * sizeof(float);
-}
+size_t attention_workspace_bytes(const pask_cache *c, int n_seqs) { return carve_workspace(c, n_seqs, nullptr, nullptr); }
 
 pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seqs, const int32_t *seq_ids, const void *q,
                                float *out, float *lse, void *workspace, size_t, cudaStream_t stream) {
     const int n_warps = c->desc.n_kv_heads;
-    const size_t slots = (size_t)c->attn_ctas + n_seqs;
-    uint8_t *ws = static_cast<uint8_t *>(workspace);
     AttnParams p;
     p.c = c->dev;
     p.layer = layer;
     p.n_seqs = n_seqs;
     p.seq_ids = seq_ids;
     p.q = static_cast<const uint4 *>(q);
-    p.prefix_out = reinterpret_cast<uint32_t *>(ws);
-    ws += align_up((size_t)(n_seqs + 1) * 4, 256);
-    p.part_ml = reinterpret_cast<float2 *>(ws);
-    ws += align_up(slots * c->desc.n_q_heads * sizeof(float2), 256);
-    p.part_o = reinterpret_cast<float *>(ws);
+    carve_workspace(c, n_seqs, static_cast<uint8_t *>(workspace), &p.ws);
     const size_t smem = attn_smem_bytes(n_seqs, n_warps);
     auto kern = has_low ? decode_attn_kernel<true> : decode_attn_kernel<false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return PASK_ERR_CUDA;
+    attn_plan_kernel<<<c->sm_count, kPlanThreads, (size_t)(4 * n_seqs + 2) * 4, stream>>>(c->dev, layer, n_seqs, seq_ids, p.ws,
+                                                                                       has_low ? 1 : 0);
     if (c->ev_start) cudaEventRecord(c->ev_start, stream);
     kern<<<c->attn_ctas, 32 * n_warps, smem, stream>>>(p);
     if (c->ev_stop) cudaEventRecord(c->ev_stop, stream);
     c->ev_start = c->ev_stop = nullptr;
     const int warps = n_seqs * c->desc.n_q_heads;
-    combine_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(p.prefix_out, p.part_ml, p.part_o, out, lse, n_seqs,
+    combine_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(p.ws.cost_prefix, p.ws.part_ml, p.ws.part_o, out, lse, n_seqs,
                                                         c->desc.n_q_heads, (uint32_t)c->attn_ctas);
     return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }

@@ -19,6 +19,7 @@ enum CtrlWord : int {
     kCtrlLowNext = 4,
     kCtrlLowFree = 5,
     kCtrlPlanOk = 6,    // 1 if the last append plan was committed, 0 if it was refused
+    kCtrlStats = 16,    // 8 words of decode-attention wait statistics (diagnostic builds with PASK_STATS only)
     kCtrlWords = 64
 };
 
@@ -42,6 +43,7 @@ struct DevCache {
     uint32_t *tbl_high, *tbl_low;    // [max_seqs][n_layers][max_pages] page ids
     pask_budget_state_t *budget;     // [max_seqs]
     uint32_t *seq_mark;              // [max_seqs] serial of the last append call that named the sequence
+    uint32_t *low_vmax;              // [max_seqs][n_layers] largest V scale (fp16 bits) in the LOW stream
     AppendPlan *plan;                // [PASK_MAX_SEQS_PER_CALL]
     uint2 *tok_scratch;              // [max_append_tokens] {action | stream position << 2, index in call}
     uint8_t *lut;                    // [n_tags][n_groups] effective action max(a0, floor)
@@ -55,7 +57,7 @@ struct DevCache {
 };
 
 struct MetaOffsets {
-    size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, plan, tok_scratch, lut,
+    size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, low_vmax, plan, tok_scratch, lut,
         layer_group, total;
     size_t zero_begin, zero_end;     // the span cleared by a reset (counters, tables, budgets, marks)
 };

@@ -9,9 +9,11 @@
 // Lane numbering: lane = 4*g + t, g = lane / 4 (0..7), t = lane % 4 (0..3).
 //
 // HIGH page  : [kv head][K tile 4096 B][V tile 4096 B]            (n_kv * 8192 B)
-//   K tile   : 8 rounds i of 512 B; round i = 2*j + hi holds, for lane (g,t), the 16-byte chunk
-//              (dims 8c .. 8c+7, c = 4*j + t) of token g + 8*hi.  QK^T uses tokens as the M
-//              rows: lane (g,t) owns rows g and g+8 and the k-slots of its own t.
+//   K tile   : 8 rounds i of 512 B, one per MMA of the tile's QK^T; round i = 2*j + h holds, for
+//              lane (g,t), the four A registers of that MMA in order: with d = 8*(4j+t) + 4h,
+//              {token g dims d,d+1 | token g+8 dims d,d+1 | token g dims d+2,d+3 | token g+8 dims
+//              d+2,d+3}.  QK^T uses tokens as the M rows: lane (g,t) owns rows g and g+8 and the
+//              k-slots of its own t, so one 128-bit load is one operand quad, no register moves.
 //   V tile   : 8 rounds i = 4*e + k of 512 B; lane (g,t) holds for token
 //              {2t, 2t+1, 2t+8, 2t+9}[k] the 8-byte pieces dims 32*(2e)+4g .. +3 and
 //              32*(2e+1)+4g .. +3.  P.V uses head dims as the M rows and tokens as k-slots.
@@ -48,10 +50,11 @@ constexpr int kLowHeadBytes = 2304;
 constexpr uint32_t kCostHighPage = 32;
 constexpr uint32_t kCostLowPage = 9;
 
-// HIGH K tile: offset of the 16-byte chunk c (dims 8c..8c+7) of token tau.
-PASK_HD int high_k_chunk_off(int tau, int c) {
+// HIGH K tile: offset of the 4-byte piece holding dims 2p, 2p+1 (p = 0..63) of token tau.
+PASK_HD int high_k_pair_off(int tau, int p) {
+    const int c = p >> 2, h = (p >> 1) & 1, second = p & 1;   // chunk of 8 dims, half of it, pair within the half
     const int g = tau & 7, hi = tau >> 3, t = c & 3, j = c >> 2;
-    return (2 * j + hi) * 512 + (4 * g + t) * 16;
+    return (2 * j + h) * 512 + (4 * g + t) * 16 + second * 8 + hi * 4;
 }
 
 // HIGH V tile: offset of the 8-byte piece holding dims 32q + 4g .. 32q + 4g + 3 of token tau.
@@ -78,16 +81,31 @@ PASK_HD int low_v_half_off(int tau, int q, int g) {
 PASK_HD int low_scale_off(int tau, int w) { return kLowCodesBytes + tau * 8 + w * 2; }
 
 // ---- work partition of decode attention -------------------------------------------------
-// Sequences are laid end to end in "cost space" (a HIGH page costs kCostHighPage, a LOW page
-// kCostLowPage); CTA b of G owns [C*b/G, C*(b+1)/G).  A cut at local offset x of a sequence whose
-// cost is cs splits BOTH of its page lists at the same fraction x / cs, so every CTA gets the
-// sequence's own mix of HIGH and LOW pages (the two kinds differ in time per byte, and a CTA
-// that received only one kind would finish early or late).  Both neighbours of a cut apply the
-// same rule, so every page is processed exactly once.
+// Every sequence's pages are visited in one fixed order that interleaves its HIGH and LOW pages
+// evenly: position v (0 <= v < n = nH + nL) is a HIGH page iff floor((v+1) nH / n) > floor(v nH / n).
+// HIGH pages are bandwidth-heavy and LOW pages instruction-heavy; taking them in turn keeps both
+// the memory system and the issue slots busy, and any run of consecutive positions has the
+// sequence's own mix.  Sequences are laid end to end in "cost space" (a HIGH page costs
+// kCostHighPage, a LOW page kCostLowPage); CTA b of G owns [C*b/G, C*(b+1)/G); a cut at local cost
+// offset x of a sequence of cost cs falls before position floor(x n / cs).  Both neighbours of a
+// cut apply the same rule, so every page is processed exactly once.
 
-// number of pages (of a list of n_pages) that lie before local cost offset x of a sequence of cost cs
-PASK_HD uint32_t cut_pages(uint32_t x, uint32_t cs, uint32_t n_pages) {
-    return x >= cs ? n_pages : (uint32_t)(((uint64_t)x * n_pages) / cs);
+// which page sits at position v: returns true and the HIGH page index, or false and the LOW page index
+PASK_HD bool page_at(uint32_t v, uint32_t nh, uint32_t nl, uint32_t &idx) {
+    const uint32_t n = nh + nl;
+    const uint32_t h0 = (uint32_t)(((uint64_t)v * nh) / n), h1 = (uint32_t)(((uint64_t)(v + 1) * nh) / n);
+    idx = h1 > h0 ? h0 : v - h0;
+    return h1 > h0;
 }
+
+// number of positions (of n) that lie before local cost offset x of a sequence of cost cs
+PASK_HD uint32_t cut_positions(uint32_t x, uint32_t cs, uint32_t n) {
+    return x >= cs ? n : (uint32_t)(((uint64_t)x * n) / cs);
+}
+
+// entries of the per-call page order list built by the plan kernel
+constexpr uint32_t kOrderHigh = 0x80000000u;   // the page is a HIGH page (else LOW)
+constexpr uint32_t kOrderTail = 0x40000000u;   // last page of its stream and only partly filled
+constexpr uint32_t kOrderIdMask = 0x3fffffffu;
 
 }  // namespace pask

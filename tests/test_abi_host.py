@@ -17,7 +17,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 @pytest.fixture(scope="module")
 def pask():
-    subprocess.run(["python", os.path.join(ROOT, "paper_2608_28276_b200", "build.py")], check=True, capture_output=True)
+    subprocess.run(["python", os.path.join(ROOT, "paper_2608_28276_b200", "build.py"), "--if-stale"], check=True,
+                   capture_output=True)
     import paper_2608_28276_b200 as P
     return P
 
@@ -85,19 +86,26 @@ def test_decode_partition_covers_every_page_exactly_once(pask):
         r = pask.pask_debug_partition(ph, pl, g).astype(np.int64)
         cost = np.zeros(g)
         for s in range(len(ph)):
-            for which, n_pages, w in ((0, int(ph[s]), 32), (2, int(pl[s]), 9)):
-                seen = np.zeros(n_pages, np.int64)
-                last_end = 0
-                for b in range(g):
-                    a, e = r[b, s, which], r[b, s, which + 1]
-                    assert a <= e
-                    if e > a:
-                        assert a == last_end          # contiguous, in CTA order
-                        last_end = e
-                    seen[a:e] += 1
-                    cost[b] += w * (e - a)
-                assert np.all(seen == 1)
-        # balance: no CTA streams more than its share plus one page of each kind per sequence cut
+            is_high, idx = pask.pask_debug_page_order(int(ph[s]), int(pl[s]))
+            # the order visits every HIGH page and every LOW page once, each stream in ascending order
+            assert np.array_equal(idx[is_high], np.arange(ph[s])) and np.array_equal(idx[~is_high], np.arange(pl[s]))
+            # and interleaves them evenly: any prefix holds its proportional share of HIGH pages
+            if len(idx):
+                seen_high = np.cumsum(is_high)
+                want = np.arange(1, len(idx) + 1) * float(ph[s]) / len(idx)
+                assert np.abs(seen_high - want).max() <= 1.0
+            seen = np.zeros(len(idx), np.int64)
+            last_end = 0
+            for b in range(g):
+                a, e = r[b, s]
+                assert a <= e
+                if e > a:
+                    assert a == last_end          # contiguous, in CTA order
+                    last_end = e
+                seen[a:e] += 1
+                cost[b] += 32 * is_high[a:e].sum() + 9 * (~is_high[a:e]).sum()
+            assert np.all(seen == 1)
+        # balance: no CTA streams more than its share plus about one page of each kind per cut
         total = float(32 * ph.sum() + 9 * pl.sum())
         assert cost.sum() == total
         assert cost.max() <= total / g + 2 * (32 + 9) + 1e-9

@@ -144,7 +144,8 @@ def test_split_count_does_not_change_the_result(pask, oracle):
         go, gl, oo, ol = p.attention(0, seqs)
         assert_close(go, gl, oo, ol, where=n_ctas)
         ref = go if ref is None else ref
-        assert np.abs(go - ref).max() < 2e-5
+        # the split changes the running maxima and with them the fp16 rounding of P * scale
+        assert np.abs(go - ref).max() < 3e-4
 
 
 def test_all_high_policy_and_full_kv_kernel(pask, oracle):
