@@ -61,6 +61,8 @@ typedef int32_t pask_status_t;
 #define PASK_DEV_RANGE 0x20u          /* a query element had |q| > 65504, outside what the low-precision path
                                          computes in; results for that sequence may be infinite or NaN */
 
+#define PASK_DEV_INTERNAL 0x40u       /* an internal bounds check refused an access (a page id out of range) */
+
 #define PASK_ACTION_RELEASE 0
 #define PASK_ACTION_RETAIN_LOW 1
 #define PASK_ACTION_RETAIN_HIGH 2

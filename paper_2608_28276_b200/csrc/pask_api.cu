@@ -200,6 +200,8 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     v.bytes_h = 2u * d->n_kv_heads * kHeadDim * 2u;
     v.bytes_l = 2u * d->n_kv_heads * (kHeadDim / 2 + kGroupsPerHead * 2);
     c->attn_ctas = attention_grid(c);
+    c->lut = pol->eff;
+    c->layer_group = pol->layer_group;
     // pageable host sources: the runtime stages these copies, so the vectors may die afterwards
     cudaError_t e = cudaMemcpyAsync(v.lut, pol->eff.data(), pol->eff.size(), cudaMemcpyHostToDevice, stream);
     if (e == cudaSuccess)

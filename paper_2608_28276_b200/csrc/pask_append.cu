@@ -223,8 +223,77 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-// One CTA (32 * n_kv threads) per token at a time; thread = one 16-byte chunk (8 head dims) of
-// K (first half of the block) or V (second half).
+// Persist one 16-byte chunk (8 head dims; chunk cch of KV head `head`, K if !which else V) of a token
+// that takes action a (RETAIN-HIGH or RETAIN-LOW) at position `at` of its stream, which lives in
+// pool page `page`.  The four lanes that hold the chunks of one 32-dim group must call together
+// (RETAIN-LOW reduces the group's amax across them); the whole warp must be converged.
+__device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uint32_t at, uint32_t page, size_t sl, int head,
+                                              int cch, int which, const uint4 x) {
+    const uint32_t tau = at & 15u;
+    if (page >= (a == PASK_ACTION_RETAIN_HIGH ? c.cap_high : c.cap_low)) {   // never expected: refuse, do not write
+        atomicOr(&c.ctrl[kCtrlStatus], PASK_DEV_INTERNAL);
+        return;
+    }
+    if (a == PASK_ACTION_RETAIN_HIGH) {
+        uint8_t *dst = c.pool_high + (size_t)page * c.high_page_bytes + (size_t)head * kHighHeadBytes +
+                       (which ? kHighTileBytes : 0);
+        if (!which) {
+            *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch)) = x.x;
+            *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch + 1)) = x.y;
+            *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch + 2)) = x.z;
+            *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch + 3)) = x.w;
+        } else {
+            const int q = cch >> 2, g0 = 2 * (cch & 3);
+            *reinterpret_cast<uint2 *>(dst + high_v_piece_off((int)tau, q, g0)) = make_uint2(x.x, x.y);
+            *reinterpret_cast<uint2 *>(dst + high_v_piece_off((int)tau, q, g0 + 1)) = make_uint2(x.z, x.w);
+        }
+        return;
+    }
+    uint8_t *dst = c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLowHeadBytes + (which ? kLowHalfBytes : 0);
+    float f[8] = {bf16_lo(x.x), bf16_hi(x.x), bf16_lo(x.y), bf16_hi(x.y), bf16_lo(x.z), bf16_hi(x.z), bf16_lo(x.w), bf16_hi(x.w)};
+    float amax = 0.0f;
+#pragma unroll
+    for (int e = 0; e < 8; e++) amax = fmaxf(amax, fabsf(f[e]));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));   // the 4 chunks of a 32-dim group
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));   // sit in 4 adjacent lanes
+    const float s32 = __fdiv_rn(amax, 7.0f);
+    __half sh = __float2half_rn(s32);
+    if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);  // saturate, never infinite
+    const float s = __half2float(sh);
+    uint32_t code[8];
+    if (s == 0.0f) {
+#pragma unroll
+        for (int e = 0; e < 8; e++) code[e] = 8u;
+    } else {
+        const float inv = __fdiv_rn(1.0f, s);
+#pragma unroll
+        for (int e = 0; e < 8; e++) {
+            float r = rintf(__fmul_rn(f[e], inv));
+            r = fminf(fmaxf(r, -7.0f), 7.0f);
+            code[e] = (uint32_t)((int)r + 8);
+        }
+    }
+    const int w = cch >> 2, u = cch & 3;
+    if (!which) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int e = 0; e < 8; e++) word |= code[e] << (4 * low_k_nibble(e));
+        *reinterpret_cast<uint32_t *>(dst + low_k_word_off((int)tau, w, u)) = word;
+    } else {
+        const uint16_t h0 = (uint16_t)(code[0] | (code[1] << 4) | (code[2] << 8) | (code[3] << 12));
+        const uint16_t h1 = (uint16_t)(code[4] | (code[5] << 4) | (code[6] << 8) | (code[7] << 12));
+        *reinterpret_cast<uint16_t *>(dst + low_v_half_off((int)tau, w, 2 * u)) = h0;
+        *reinterpret_cast<uint16_t *>(dst + low_v_half_off((int)tau, w, 2 * u + 1)) = h1;
+    }
+    if (u == 0) *reinterpret_cast<__half *>(dst + low_scale_off((int)tau, w)) = sh;
+    // decode attention forms P * (V scale) in fp16 relative to the stream's largest V scale:
+    // keep that maximum per (sequence, layer) -- one atomic per warp, and only when it grows
+    const uint32_t hb = __reduce_max_sync(0xffffffffu, which ? (uint32_t)__half_as_ushort(sh) : 0u);
+    if ((threadIdx.x & 31) == 0 && hb > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb);
+}
+
+// General path, second kernel.  One CTA (32 * n_kv threads) per token at a time; thread = one
+// 16-byte chunk (8 head dims) of K (first half of the block) or V (second half).
 __global__ void __launch_bounds__(256)
 append_write_kernel(DevCache c, int layer, int total_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v) {
     if (c.ctrl[kCtrlPlanOk] == 0) return;
@@ -241,69 +310,197 @@ append_write_kernel(DevCache c, int layer, int total_tokens, const uint4 *__rest
         const AppendPlan &p = c.plan[sc.y];
         const size_t sl = (size_t)p.seq * c.n_layers + layer;
         const uint4 x = src[(size_t)t * chunks + cg];
-        if (a == PASK_ACTION_RETAIN_HIGH) {
-            const uint32_t at = p.old_high + pos, tau = at & 15u;
-            const uint32_t page = c.tbl_high[sl * c.max_pages + (at >> 4)];
-            uint8_t *dst = c.pool_high + (size_t)page * c.high_page_bytes + (size_t)head * kHighHeadBytes +
-                           (which ? kHighTileBytes : 0);
-            if (!which) {
-                *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch)) = x.x;
-                *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch + 1)) = x.y;
-                *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch + 2)) = x.z;
-                *reinterpret_cast<uint32_t *>(dst + high_k_pair_off((int)tau, 4 * cch + 3)) = x.w;
-            } else {
-                const int q = cch >> 2, g0 = 2 * (cch & 3);
-                *reinterpret_cast<uint2 *>(dst + high_v_piece_off((int)tau, q, g0)) = make_uint2(x.x, x.y);
-                *reinterpret_cast<uint2 *>(dst + high_v_piece_off((int)tau, q, g0 + 1)) = make_uint2(x.z, x.w);
-            }
-        } else {
-            const uint32_t at = p.old_low + pos, tau = at & 15u;
-            const uint32_t page = c.tbl_low[sl * c.max_pages + (at >> 4)];
-            uint8_t *dst = c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLowHeadBytes +
-                           (which ? kLowHalfBytes : 0);
-            float f[8] = {bf16_lo(x.x), bf16_hi(x.x), bf16_lo(x.y), bf16_hi(x.y),
-                          bf16_lo(x.z), bf16_hi(x.z), bf16_lo(x.w), bf16_hi(x.w)};
-            float amax = 0.0f;
-#pragma unroll
-            for (int e = 0; e < 8; e++) amax = fmaxf(amax, fabsf(f[e]));
-            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));   // the 4 chunks of a 32-dim group
-            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));   // sit in 4 adjacent lanes
-            const float s32 = __fdiv_rn(amax, 7.0f);
-            __half sh = __float2half_rn(s32);
-            if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);  // saturate, never infinite
-            const float s = __half2float(sh);
-            uint32_t code[8];
-            if (s == 0.0f) {
-#pragma unroll
-                for (int e = 0; e < 8; e++) code[e] = 8u;
-            } else {
-                const float inv = __fdiv_rn(1.0f, s);
-#pragma unroll
-                for (int e = 0; e < 8; e++) {
-                    float r = rintf(__fmul_rn(f[e], inv));
-                    r = fminf(fmaxf(r, -7.0f), 7.0f);
-                    code[e] = (uint32_t)((int)r + 8);
-                }
-            }
-            const int w = cch >> 2, u = cch & 3;
-            if (!which) {
-                uint32_t word = 0;
-#pragma unroll
-                for (int e = 0; e < 8; e++) word |= code[e] << (4 * low_k_nibble(e));
-                *reinterpret_cast<uint32_t *>(dst + low_k_word_off((int)tau, w, u)) = word;
-            } else {
-                const uint16_t h0 = (uint16_t)(code[0] | (code[1] << 4) | (code[2] << 8) | (code[3] << 12));
-                const uint16_t h1 = (uint16_t)(code[4] | (code[5] << 4) | (code[6] << 8) | (code[7] << 12));
-                *reinterpret_cast<uint16_t *>(dst + low_v_half_off((int)tau, w, 2 * u)) = h0;
-                *reinterpret_cast<uint16_t *>(dst + low_v_half_off((int)tau, w, 2 * u + 1)) = h1;
-            }
-            if (u == 0) *reinterpret_cast<__half *>(dst + low_scale_off((int)tau, w)) = sh;
-            // decode attention forms P * (V scale) in fp16 relative to the stream's largest V scale:
-            // keep that maximum per (sequence, layer) -- one atomic per warp, and only when it grows
-            const uint32_t hb = __reduce_max_sync(0xffffffffu, which ? (uint32_t)__half_as_ushort(sh) : 0u);
-            if ((tid & 31) == 0 && hb > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb);
+        const uint32_t at = (a == PASK_ACTION_RETAIN_HIGH ? p.old_high : p.old_low) + pos;
+        const uint32_t *tbl = a == PASK_ACTION_RETAIN_HIGH ? c.tbl_high : c.tbl_low;
+        persist_chunk(c, a, at, tbl[sl * c.max_pages + (at >> 4)], sl, head, cch, which, x);
+    }
+}
+
+// Small calls (decode: a token or a few per sequence): the whole of pask_append_kv in one launch
+// of one CTA per token, built so that the chain of dependent global round trips is as short as it
+// can be.  The table column and the layer's group arrive as kernel arguments; every CTA fetches
+// every per-sequence word in one round and works out the identical plan for the whole call in
+// shared memory (decisions, ranks, page allocation by a scan); then it writes its own token.  All
+// CTAs only read the cache state while planning; the CTA that finishes planning last (arrival
+// counter, nobody waits) commits the counters, tables and budget states for everybody.
+constexpr int kSmallMax = 128;       // at most this many sequences and tokens
+constexpr int kSmallThreads = 256;
+struct SmallLut { uint8_t action[256]; };
+
+__global__ void __launch_bounds__(kSmallThreads)
+append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, const int32_t *__restrict__ seq_ids,
+                    const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
+                    const uint8_t *__restrict__ tags, uint8_t *__restrict__ actions_out, const SmallLut lut) {
+    __shared__ int s_seq[kSmallMax], s_cu[kSmallMax + 1];
+    __shared__ uint32_t s_old_h[kSmallMax], s_old_l[kSmallMax], s_cnt_h[kSmallMax], s_cnt_l[kSmallMax], s_cnt_bad[kSmallMax];
+    __shared__ uint32_t s_new_h[kSmallMax], s_new_l[kSmallMax], s_base_h[kSmallMax], s_base_l[kSmallMax];
+    __shared__ uint8_t s_act[kSmallMax], s_tok_seq[kSmallMax], s_tok_bad[kSmallMax];
+    __shared__ uint32_t s_pos[kSmallMax], s_ctrl[4], s_err;
+    __shared__ int s_last;
+    const int tid = threadIdx.x;
+    // this CTA's token and this thread's chunk of it: fetch the data first, it depends on nothing
+    const int my_tok = blockIdx.x;
+    const int chunks = 16 * c.n_kv;
+    const bool writer = tid < 2 * chunks;
+    const int which = tid >= chunks, cg = which ? tid - chunks : tid;
+    uint4 x = make_uint4(0, 0, 0, 0);
+    if (writer) x = (which ? v : k)[(size_t)my_tok * chunks + cg];
+    if (tid == 0) s_err = 0;
+    if (tid < 4) s_ctrl[tid] = c.ctrl[kCtrlHighNext + tid];     // high next, high free, low next, low free
+    if (tid <= n_seqs) s_cu[tid] = cu_tokens[tid];
+    if (tid < n_seqs) {
+        const int seq = seq_ids[tid];
+        s_seq[tid] = seq;
+        uint32_t oh = 0, ol = 0;
+        if (seq >= 0 && seq < c.max_seqs) {
+            const size_t sl = (size_t)seq * c.n_layers + layer;
+            oh = c.n_high[sl];
+            ol = c.n_low[sl];
+        }
+        s_old_h[tid] = oh;
+        s_old_l[tid] = ol;
+    }
+    int my_tag = 0;
+    if (tid < total) my_tag = tags[tid];
+    __syncthreads();
+
+    // ---- validate the call; decide every token
+    uint32_t err = 0;
+    if (tid < n_seqs) {
+        const int seq = s_seq[tid];
+        if (seq < 0 || seq >= c.max_seqs) err |= PASK_DEV_BAD_SEQ;
+        for (int j = 0; j < tid; j++) if (s_seq[j] == seq) err |= PASK_DEV_BAD_SEQ;       // named twice
+        if (s_cu[tid] < 0 || s_cu[tid + 1] < s_cu[tid] || (tid == 0 && s_cu[0] != 0) ||
+            (tid == n_seqs - 1 && s_cu[n_seqs] != total)) err |= PASK_DEV_BAD_RAGGED;
+    }
+    if (err) atomicOr(&s_err, err);
+    __syncthreads();
+    if (s_err) {   // every CTA sees the same; the last one to get here resets the arrival counter
+        if (tid == 0) {
+            atomicOr(&c.ctrl[kCtrlStatus], s_err);
+            if (atomicAdd(&c.ctrl[kCtrlTicket], 1u) == gridDim.x - 1) { c.ctrl[kCtrlPlanOk] = 0; c.ctrl[kCtrlTicket] = 0; }
+        }
+        return;
+    }
+    if (tid < total) {
+        int i = 0;                                   // the sequence this token belongs to
+        while (s_cu[i + 1] <= tid) i++;
+        const int a = lut.action[my_tag];
+        s_tok_seq[tid] = (uint8_t)i;
+        s_act[tid] = (uint8_t)a;
+        s_tok_bad[tid] = my_tag != PASK_TAG_PROTECTED && my_tag >= c.n_tags;
+        if (actions_out && blockIdx.x == 0) actions_out[tid] = (uint8_t)a;
+    }
+    __syncthreads();
+
+    // ---- per token: rank inside its stream; per sequence: counts and new pages
+    if (tid < total) {
+        const int i = s_tok_seq[tid], a = s_act[tid];
+        uint32_t pos = 0;
+        for (int t = s_cu[i]; t < tid; t++) pos += s_act[t] == a;
+        s_pos[tid] = pos;
+    }
+    if (tid < n_seqs) {
+        uint32_t ch = 0, cl = 0, cb = 0;
+        for (int t = s_cu[tid]; t < s_cu[tid + 1]; t++) {
+            ch += s_act[t] == PASK_ACTION_RETAIN_HIGH;
+            cl += s_act[t] == PASK_ACTION_RETAIN_LOW;
+            cb += s_tok_bad[t];
+        }
+        s_cnt_h[tid] = ch; s_cnt_l[tid] = cl; s_cnt_bad[tid] = cb;
+        const uint32_t oh = s_old_h[tid], ol = s_old_l[tid];
+        const uint32_t ph1 = (oh + ch + kPageTokens - 1) / kPageTokens, pl1 = (ol + cl + kPageTokens - 1) / kPageTokens;
+        s_new_h[tid] = ph1 - (oh + kPageTokens - 1) / kPageTokens;
+        s_new_l[tid] = pl1 - (ol + kPageTokens - 1) / kPageTokens;
+        if (ph1 > (uint32_t)c.max_pages || pl1 > (uint32_t)c.max_pages) atomicOr(&s_err, PASK_DEV_SEQ_OVERFLOW);
+    }
+    __syncthreads();
+
+    // ---- allocate for the whole call (sequence-major, like the general path) or refuse it
+    uint32_t need_h = 0, need_l = 0;
+    if (tid < n_seqs) {
+        uint32_t bh = 0, bl = 0;
+        for (int j = 0; j < n_seqs; j++) {
+            if (j == tid) { bh = need_h; bl = need_l; }
+            need_h += s_new_h[j]; need_l += s_new_l[j];
+        }
+        s_base_h[tid] = bh; s_base_l[tid] = bl;
+        const bool fits = need_h <= s_ctrl[1] + (c.cap_high - s_ctrl[0]) && need_l <= s_ctrl[3] + (c.cap_low - s_ctrl[2]);
+        if (tid == 0 && !fits && !s_err) atomicOr(&s_err, PASK_DEV_POOL_EXHAUSTED);
+    }
+    __syncthreads();
+    // old page of this CTA's token, if it continues one (page tables are only appended to by the commit)
+    uint32_t my_page = 0, my_at = 0;
+    const uint32_t my_a = s_act[my_tok];
+    const int my_i = s_tok_seq[my_tok];
+    const size_t my_sl = (size_t)s_seq[my_i] * c.n_layers + layer;
+    if (my_a != PASK_ACTION_RELEASE) {
+        const bool high = my_a == PASK_ACTION_RETAIN_HIGH;
+        const uint32_t old = high ? s_old_h[my_i] : s_old_l[my_i];
+        my_at = old + s_pos[my_tok];
+        const uint32_t old_pages = (old + kPageTokens - 1) / kPageTokens, pg = my_at >> 4;
+        if (pg < old_pages) {
+            my_page = (high ? c.tbl_high : c.tbl_low)[my_sl * c.max_pages + pg];
+        } else {   // one of the pages this call allocates: same formula as the commit below
+            const uint32_t kk = (high ? s_base_h[my_i] : s_base_l[my_i]) + (pg - old_pages);
+            const uint32_t fr = high ? s_ctrl[1] : s_ctrl[3], nx = high ? s_ctrl[0] : s_ctrl[2];
+            my_page = kk < fr ? (high ? c.free_high : c.free_low)[fr - 1 - kk] : nx + (kk - fr);
         }
     }
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(&c.ctrl[kCtrlTicket], 1u) == gridDim.x - 1;   // every read of the old state is done
+    __syncthreads();
+    if (s_err) {
+        if (tid == 0) {
+            atomicOr(&c.ctrl[kCtrlStatus], s_err);
+            if (s_last) { c.ctrl[kCtrlPlanOk] = 0; c.ctrl[kCtrlTicket] = 0; }
+        }
+        return;
+    }
+
+    // ---- commit (last CTA to arrive only): page tables, stream lengths, budget states, pool state
+    if (s_last && tid < n_seqs) {
+        const int seq = s_seq[tid];
+        const size_t sl = (size_t)seq * c.n_layers + layer;
+        const uint32_t oh = s_old_h[tid], ol = s_old_l[tid], ch = s_cnt_h[tid], cl = s_cnt_l[tid];
+        const uint32_t n_tok = (uint32_t)(s_cu[tid + 1] - s_cu[tid]);
+        const uint32_t ph0 = (oh + kPageTokens - 1) / kPageTokens, pl0 = (ol + kPageTokens - 1) / kPageTokens;
+        for (uint32_t x = 0; x < s_new_h[tid]; x++) {
+            const uint32_t kk = s_base_h[tid] + x;
+            c.tbl_high[sl * c.max_pages + ph0 + x] = kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]);
+        }
+        for (uint32_t x = 0; x < s_new_l[tid]; x++) {
+            const uint32_t kk = s_base_l[tid] + x;
+            c.tbl_low[sl * c.max_pages + pl0 + x] = kk < s_ctrl[3] ? c.free_low[s_ctrl[3] - 1 - kk] : s_ctrl[2] + (kk - s_ctrl[3]);
+        }
+        c.n_high[sl] = oh + ch;
+        c.n_low[sl] = ol + cl;
+        pask_budget_state_t &b = c.budget[seq];
+        b.n_seen[group] += n_tok;
+        b.n_high[group] += ch;
+        b.n_low[group] += cl;
+        b.n_drop[group] += n_tok - ch - cl;
+        const uint64_t retained = b.retained_bytes + (uint64_t)ch * c.bytes_h + (uint64_t)cl * c.bytes_l;
+        const uint64_t full = b.full_bytes + (uint64_t)n_tok * c.bytes_h;
+        b.retained_bytes = retained;
+        b.full_bytes = full;
+        b.remaining_bytes = (int64_t)(((uint64_t)c.budget_q16 * full) >> 16) - (int64_t)retained;
+        b.bad_tags += s_cnt_bad[tid];
+        b.pages_high += s_new_h[tid];
+        b.pages_low += s_new_l[tid];
+        if (tid == 0) {
+            const uint32_t pop_h = need_h < s_ctrl[1] ? need_h : s_ctrl[1], pop_l = need_l < s_ctrl[3] ? need_l : s_ctrl[3];
+            c.ctrl[kCtrlHighFree] = s_ctrl[1] - pop_h;
+            c.ctrl[kCtrlHighNext] = s_ctrl[0] + (need_h - pop_h);
+            c.ctrl[kCtrlLowFree] = s_ctrl[3] - pop_l;
+            c.ctrl[kCtrlLowNext] = s_ctrl[2] + (need_l - pop_l);
+            c.ctrl[kCtrlPlanOk] = 1;
+            c.ctrl[kCtrlTicket] = 0;
+        }
+    }
+
+    // ---- persist this CTA's token: one thread per 16-byte chunk of K and of V
+    if (writer && my_a != PASK_ACTION_RELEASE) persist_chunk(c, my_a, my_at, my_page, my_sl, cg >> 4, cg & 15, which, x);
 }
 
 // Return every page of one sequence to the free stacks and clear its counters.
@@ -332,6 +529,17 @@ __global__ void __launch_bounds__(256) seq_reset_kernel(DevCache c, int seq) {
 pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_tokens, const int32_t *seq_ids,
                             const int32_t *cu_tokens, const void *k, const void *v, const uint8_t *tags,
                             uint8_t *actions_out, cudaStream_t stream) {
+    if (n_seqs <= kSmallMax && total_tokens <= kSmallMax) {
+        SmallLut lut;
+        const int group = c->layer_group[layer];
+        for (int z = 0; z < 256; z++)
+            lut.action[z] = z < c->dev.n_tags ? c->lut[(size_t)z * c->dev.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
+        if (total_tokens == 0) return PASK_OK;
+        append_small_kernel<<<total_tokens, kSmallThreads, 0, stream>>>(c->dev, layer, group, n_seqs, total_tokens, seq_ids, cu_tokens,
+                                                            static_cast<const uint4 *>(k), static_cast<const uint4 *>(v), tags,
+                                                            actions_out, lut);
+        return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
+    }
     if (++c->append_serial == 0) c->append_serial = 1;
     append_plan_kernel<<<n_seqs, kPlanThreads, 0, stream>>>(c->dev, layer, n_seqs, total_tokens, seq_ids, cu_tokens, tags,
                                                            actions_out, c->append_serial);

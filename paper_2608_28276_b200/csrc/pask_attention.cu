@@ -706,16 +706,26 @@ combine_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ p
     if (p1 > p0) {
         const uint32_t b_first = (uint32_t)((((uint64_t)p0 + 1) * n_ctas - 1) / total);
         const uint32_t b_last = (uint32_t)(((uint64_t)p1 * n_ctas - 1) / total);
-        for (uint32_t b = b_first; b <= b_last; b++) M = fmaxf(M, part_ml[((size_t)b + s) * n_q + h].x);
-        if (M > -INFINITY) {
-            for (uint32_t b = b_first; b <= b_last; b++) {
-                const size_t row = ((size_t)b + s) * n_q + h;
-                const float2 ml = part_ml[row];
-                if (ml.x == -INFINITY) continue;      // a CTA whose share of this sequence was empty
-                const float wgt = exp2f(ml.x - M);
-                const float4 v = *reinterpret_cast<const float4 *>(part_o + row * kHeadDim + lane * 4);
-                o.x = fmaf(wgt, v.x, o.x); o.y = fmaf(wgt, v.y, o.y); o.z = fmaf(wgt, v.z, o.z); o.w = fmaf(wgt, v.w, o.w);
-                L = fmaf(wgt, ml.y, L);
+        // online merge, four partials per round trip
+        for (uint32_t b = b_first; b <= b_last; b += 4) {
+            float2 ml[4];
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; u++) {
+                const bool have = b + u <= b_last;
+                const size_t row = ((size_t)b + u + s) * n_q + h;
+                ml[u] = have ? part_ml[row] : make_float2(-INFINITY, 0.f);
+                v[u] = have ? *reinterpret_cast<const float4 *>(part_o + row * kHeadDim + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; u++) {
+                if (ml[u].x == -INFINITY) continue;      // a CTA whose share of this sequence was empty
+                const float Mn = fmaxf(M, ml[u].x);
+                const float fo = exp2f(M - Mn), fn = exp2f(ml[u].x - Mn);   // exp2f(-inf) = 0 on the first one
+                o.x = fmaf(fn, v[u].x, o.x * fo); o.y = fmaf(fn, v[u].y, o.y * fo);
+                o.z = fmaf(fn, v[u].z, o.z * fo); o.w = fmaf(fn, v[u].w, o.w * fo);
+                L = fmaf(fn, ml[u].y, L * fo);
+                M = Mn;
             }
         }
     }

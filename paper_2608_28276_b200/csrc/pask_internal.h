@@ -77,6 +77,7 @@ struct pask_cache {
     pask::MetaOffsets off;
     void *meta;
     uint32_t append_serial;
+    std::vector<uint8_t> lut, layer_group;   // host copies of the folded table [n_tags][n_groups] and the layer map
     int sm_count;
     int attn_ctas;                // grid of the decode-attention main kernel
     cudaEvent_t ev_start, ev_stop;

@@ -93,7 +93,14 @@ PASK_HD int low_scale_off(int tau, int w) { return kLowCodesBytes + tau * 8 + w 
 // which page sits at position v: returns true and the HIGH page index, or false and the LOW page index
 PASK_HD bool page_at(uint32_t v, uint32_t nh, uint32_t nl, uint32_t &idx) {
     const uint32_t n = nh + nl;
-    const uint32_t h0 = (uint32_t)(((uint64_t)v * nh) / n), h1 = (uint32_t)(((uint64_t)(v + 1) * nh) / n);
+    uint32_t h0, h1;
+    if (n < 65536u) {   // products fit 32 bits (streams below a million tokens): cheap division
+        h0 = (v * nh) / n;
+        h1 = ((v + 1) * nh) / n;
+    } else {
+        h0 = (uint32_t)(((uint64_t)v * nh) / n);
+        h1 = (uint32_t)(((uint64_t)(v + 1) * nh) / n);
+    }
     idx = h1 > h0 ? h0 : v - h0;
     return h1 > h0;
 }
