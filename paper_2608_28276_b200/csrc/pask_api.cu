@@ -339,6 +339,8 @@ pask_status_t pask_budget_state(pask_cache_t *c, int32_t seq, pask_budget_state_
     if (e == cudaSuccess) e = cudaMemcpyAsync(&status, c->dev.ctrl + kCtrlStatus, 4, cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return PASK_ERR_CUDA;
+    host_out->remaining_bytes =
+        (int64_t)(((uint64_t)c->dev.budget_q16 * host_out->full_bytes) >> 16) - (int64_t)host_out->retained_bytes;
     host_out->device_status = status;
     host_out->reserved = 0;
     return PASK_OK;

@@ -22,6 +22,10 @@ __device__ __forceinline__ AppendPlan load_plan_cg(const AppendPlan *p) {
     return u.plan;
 }
 
+__device__ __forceinline__ void budget_add(uint64_t *p, uint64_t v) {
+    if (v) atomicAdd(reinterpret_cast<unsigned long long *>(p), (unsigned long long)v);
+}
+
 __device__ __forceinline__ uint32_t lanemask_lt() {
     uint32_t m;
     asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
@@ -204,7 +208,6 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         b.n_drop[grp] += p.cnt_drop;
         b.retained_bytes += (uint64_t)p.cnt_high * c.bytes_h + (uint64_t)p.cnt_low * c.bytes_l;
         b.full_bytes += n_tok * c.bytes_h;
-        b.remaining_bytes = (int64_t)(((uint64_t)c.budget_q16 * b.full_bytes) >> 16) - (int64_t)b.retained_bytes;
         b.bad_tags += p.bad_tags;
         b.pages_high += nh[r];
         b.pages_low += nl[r];
@@ -338,6 +341,8 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     __shared__ uint32_t s_pos[kSmallMax], s_ctrl[4], s_err;
     __shared__ int s_last;
     const int tid = threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     // this CTA's token and this thread's chunk of it: fetch the data first, it depends on nothing
     const int my_tok = blockIdx.x;
     const int chunks = 16 * c.n_kv;
@@ -475,19 +480,18 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         }
         c.n_high[sl] = oh + ch;
         c.n_low[sl] = ol + cl;
+        // budget state: additions only (no read-modify-write round trip); remaining_bytes is derived
+        // from retained_bytes and full_bytes when the state is read
         pask_budget_state_t &b = c.budget[seq];
-        b.n_seen[group] += n_tok;
-        b.n_high[group] += ch;
-        b.n_low[group] += cl;
-        b.n_drop[group] += n_tok - ch - cl;
-        const uint64_t retained = b.retained_bytes + (uint64_t)ch * c.bytes_h + (uint64_t)cl * c.bytes_l;
-        const uint64_t full = b.full_bytes + (uint64_t)n_tok * c.bytes_h;
-        b.retained_bytes = retained;
-        b.full_bytes = full;
-        b.remaining_bytes = (int64_t)(((uint64_t)c.budget_q16 * full) >> 16) - (int64_t)retained;
-        b.bad_tags += s_cnt_bad[tid];
-        b.pages_high += s_new_h[tid];
-        b.pages_low += s_new_l[tid];
+        budget_add(&b.n_seen[group], n_tok);
+        budget_add(&b.n_high[group], ch);
+        budget_add(&b.n_low[group], cl);
+        budget_add(&b.n_drop[group], n_tok - ch - cl);
+        budget_add(&b.retained_bytes, (uint64_t)ch * c.bytes_h + (uint64_t)cl * c.bytes_l);
+        budget_add(&b.full_bytes, (uint64_t)n_tok * c.bytes_h);
+        budget_add(&b.bad_tags, s_cnt_bad[tid]);
+        if (s_new_h[tid]) atomicAdd(&b.pages_high, s_new_h[tid]);
+        if (s_new_l[tid]) atomicAdd(&b.pages_low, s_new_l[tid]);
         if (tid == 0) {
             const uint32_t pop_h = need_h < s_ctrl[1] ? need_h : s_ctrl[1], pop_l = need_l < s_ctrl[3] ? need_l : s_ctrl[3];
             c.ctrl[kCtrlHighFree] = s_ctrl[1] - pop_h;
@@ -535,10 +539,10 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
         for (int z = 0; z < 256; z++)
             lut.action[z] = z < c->dev.n_tags ? c->lut[(size_t)z * c->dev.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
         if (total_tokens == 0) return PASK_OK;
-        append_small_kernel<<<total_tokens, kSmallThreads, 0, stream>>>(c->dev, layer, group, n_seqs, total_tokens, seq_ids, cu_tokens,
-                                                            static_cast<const uint4 *>(k), static_cast<const uint4 *>(v), tags,
-                                                            actions_out, lut);
-        return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
+        const cudaError_t e = launch_pdl(append_small_kernel, dim3(total_tokens), dim3(kSmallThreads), 0, stream, c->dev, layer,
+                                         group, n_seqs, total_tokens, seq_ids, cu_tokens, static_cast<const uint4 *>(k),
+                                         static_cast<const uint4 *>(v), tags, actions_out, lut);
+        return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
     }
     if (++c->append_serial == 0) c->append_serial = 1;
     append_plan_kernel<<<n_seqs, kPlanThreads, 0, stream>>>(c->dev, layer, n_seqs, total_tokens, seq_ids, cu_tokens, tags,

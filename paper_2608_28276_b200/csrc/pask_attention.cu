@@ -213,6 +213,8 @@ __device__ __forceinline__ void split_pair(float x0, float x1, uint32_t &hi, uin
 __global__ void __launch_bounds__(kPlanThreads)
 attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ seq_ids, Workspace ws, int has_low) {
     extern __shared__ uint32_t s_plan[];
+    pdl_launch_dependents();
+    pdl_wait();
     uint32_t *s_cost = s_plan, *s_page = s_cost + n_seqs + 1, *s_nh = s_page + n_seqs + 1, *s_nl = s_nh + n_seqs;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int s = tid; s < n_seqs; s += kPlanThreads) {
@@ -392,6 +394,8 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     uint8_t *s_ring = smem + off;
     uint8_t *s_scratch = s_ring + (size_t)n_warps * kStages * kStageBytes;
 
+    pdl_launch_dependents();
+    pdl_wait();
     for (int s = tid; s <= n_seqs; s += blockDim.x) {
         s_cost[s] = __ldg(p.ws.cost_prefix + s);
         s_page[s] = __ldg(p.ws.page_prefix + s);
@@ -697,6 +701,8 @@ __global__ void __launch_bounds__(256)
 combine_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ part_ml, const float *__restrict__ part_o,
                float *__restrict__ out, float *__restrict__ lse, int n_seqs, int n_q, uint32_t n_ctas) {
     const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    pdl_wait();
     if (wid >= n_seqs * n_q) return;
     const int s = wid / n_q, h = wid % n_q;
     const uint32_t p0 = prefix[s], p1 = prefix[s + 1];
@@ -785,16 +791,18 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
     auto kern = has_low ? decode_attn_kernel<true> : decode_attn_kernel<false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return PASK_ERR_CUDA;
-    attn_plan_kernel<<<c->sm_count, kPlanThreads, (size_t)(4 * n_seqs + 2) * 4, stream>>>(c->dev, layer, n_seqs, seq_ids, p.ws,
-                                                                                       has_low ? 1 : 0);
+    cudaError_t e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(4 * n_seqs + 2) * 4, stream,
+                               c->dev, layer, n_seqs, seq_ids, p.ws, has_low ? 1 : 0);
     if (c->ev_start) cudaEventRecord(c->ev_start, stream);
-    kern<<<c->attn_ctas, 32 * n_warps, smem, stream>>>(p);
+    if (e == cudaSuccess) e = launch_pdl(kern, dim3(c->attn_ctas), dim3(32 * n_warps), smem, stream, p);
     if (c->ev_stop) cudaEventRecord(c->ev_stop, stream);
     c->ev_start = c->ev_stop = nullptr;
     const int warps = n_seqs * c->desc.n_q_heads;
-    combine_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(p.ws.cost_prefix, p.ws.part_ml, p.ws.part_o, out, lse, n_seqs,
-                                                        c->desc.n_q_heads, (uint32_t)c->attn_ctas);
-    return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
+    if (e == cudaSuccess)
+        e = launch_pdl(combine_kernel, dim3((warps + 7) / 8), dim3(256), 0, stream, (const uint32_t *)p.ws.cost_prefix,
+                       (const float2 *)p.ws.part_ml, (const float *)p.ws.part_o, out, lse, n_seqs, (int)c->desc.n_q_heads,
+                       (uint32_t)c->attn_ctas);
+    return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }
 
 }  // namespace pask
