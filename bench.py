@@ -38,6 +38,10 @@ from pask_workloads.tensors import TENSOR_K, TENSOR_Q, TENSOR_V, normal_bf16, bf
 METRIC = "mixed-KV decode-attn tokens/s at KV budget 0.33"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + write) over algorithmic bytes of the streaming kernel, from the ncu capture
+# summarised in profiles/decode_attn_kernel__qwen3-4b-step-first-4-layers.md (mean of three launches
+# of a 4-layer cut of this workload; traffic grows in proportion to the pages streamed)
+NCU_TRAFFIC_RATIO = 1.009
 STEP_STREAM = 1_000_000          # decode-step inputs of step i come from generator stream (layer, STEP_STREAM + i)
 
 CONFIGS = {c.name: c for c in WC.CONFIGS}
@@ -82,6 +86,25 @@ def step_inputs(w, layer, step, device):
     q = normal_bf16(w.seed, TENSOR_Q, layer, STEP_STREAM + step, 0, cfg.batch, cfg.n_q, device)
     tags = np.array([w.gen_tags[b][w.gen_len(b) + step] for b in range(cfg.batch)], np.uint8)
     return k, v, q, tags
+
+
+def max_over_ranks(x: float, device) -> float:
+    """MAX of a per-rank scalar over the job (identity on one rank). Works on NCCL and gloo groups."""
+    if torch.distributed.is_available() and torch.distributed.is_initialized() and torch.distributed.get_world_size() > 1:
+        t = torch.tensor([x], dtype=torch.float64, device=device)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        return float(t.item())
+    return float(x)
+
+
+def whole_job_tokens_per_s(world: int, batch_per_rank: int, steps: int, max_ms: float) -> float:
+    """Every rank decodes its own batch (weak scaling): units all ranks processed / slowest rank's time."""
+    return world * batch_per_rank * steps / (max_ms * 1e-3)
+
+
+def rank_workload(cfg, rank: int):
+    """Rank r runs its own sequences: the same configuration, seed offset by the rank."""
+    return WC.build(cfg, repeat=rank)
 
 
 class ClockSampler:
@@ -197,8 +220,9 @@ class Job:
             self.attn(h, layer, self.ids, q, self.out, self.lse, self.ws)
 
     def algorithmic_bytes_per_layer(self, steps_done=0):
-        """Bytes one decode-attention launch must move, averaged over layers: K/V payload of the
-        retained tokens (incl. scales), q, out, lse, page tables, split partials written + read."""
+        """Bytes one launch of the streaming kernel must move, averaged over layers: K/V payload of the
+        retained tokens (codes + scales, or bf16), the queries, the page-order list, and the split
+        partials it writes. Dropped tokens and page slack are not counted."""
         cfg = self.cfg
         lg = self.w.policy.layer_group.astype(np.int64)
         n_ctas = 2 * torch.cuda.get_device_properties(self.device).multi_processor_count
@@ -208,8 +232,8 @@ class Job:
             tot += float((nh * cfg.n_kv * 512).sum() + (nl * cfg.n_kv * 144).sum())
             tot += float((((nh + 15) // 16) + ((nl + 15) // 16)).sum() * 4)
         per_layer = tot / cfg.n_layers
-        per_layer += self.B * cfg.n_q * 128 * 2 + self.B * cfg.n_q * (128 + 1) * 4
-        per_layer += 2 * (n_ctas + self.B) * cfg.n_q * 130 * 4
+        per_layer += self.B * cfg.n_q * 128 * 2
+        per_layer += (n_ctas + self.B) * cfg.n_q * 130 * 4
         return per_layer
 
 
@@ -226,7 +250,7 @@ def run_cuda(args, rank, world):
     total_steps = args.warmup + args.steps
     e2e_steps = min(args.steps, 5)
     cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, 2 * total_steps + e2e_steps + 8))
-    w = WC.build(cfg, repeat=rank)
+    w = rank_workload(cfg, rank)
     t_setup = time.time()
     job = Job(P, w, device, 2 * total_steps + e2e_steps + 4)
     job.fill()
@@ -266,14 +290,11 @@ def run_cuda(args, rank, world):
         sampler.start()
     ms, kern_ms = timed(job, args.warmup, args.steps, True)
     clocks = sampler.stop() if rank == 0 else {}
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, device)
     st = P.pask_budget_state(job.cache.handle, 0)
     if st.device_status:
         raise RuntimeError(f"device status {st.device_status:#x} after the timed region")
-    value = world * job.B * args.steps / (ms * 1e-3)
+    value = whole_job_tokens_per_s(world, job.B, args.steps, ms)
 
     # ---- end to end: the same step through the host-buffer entry point, copies inside the region
     e2e = None
@@ -297,13 +318,10 @@ def run_cuda(args, rank, world):
         t1.record()
         barrier()
         e_ms = t0.elapsed_time(t1)
-        if world > 1:
-            t = torch.tensor([e_ms], dtype=torch.float64, device=device)
-            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = max_over_ranks(e_ms, device)
         h2d = cfg.n_layers * (job.B * 4 + 2 * job.B * cfg.n_kv * 256 + job.B + job.B * cfg.n_q * 256)
         d2h = cfg.n_layers * job.B * cfg.n_q * 128 * 4
-        e2e = {"value": world * job.B * e2e_steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": whole_job_tokens_per_s(world, job.B, e2e_steps, e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps}
 
     if rank != 0:
@@ -327,7 +345,8 @@ def run_cuda(args, rank, world):
         "roofline": {"bound": "hbm", "kernel": "decode_attn_kernel<true>", "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "algorithmic_bytes_per_launch": alg,
-                     "avg_launch_ms": k_ms, "launches_timed": len(kern_ms), "traffic": None},
+                     "avg_launch_ms": k_ms, "launches_timed": len(kern_ms), "traffic": alg * NCU_TRAFFIC_RATIO,
+                     "traffic_source": "ncu dram__bytes_read+write of a 4-layer cut, scaled by pages streamed"},
         "attention_share_of_step": sum(kern_ms) / ms,
     }
     if args.full_kv and world == 1:
