@@ -203,6 +203,29 @@ pask_status_t pask_decode_attention_full(pask_cache_t *cache, int32_t layer, int
                                          void *workspace, size_t workspace_bytes, pask_stream_t stream);
 size_t pask_workspace_bytes(const pask_cache_t *cache, int32_t n_seqs);
 
+/* pask_decode_attention_static -- pask_decode_attention for callers that cannot provide a workspace.
+ * (The paper has no counterpart; this is a deployment convenience of the library.)
+ * Some integrations cannot allocate device memory where they call the library: a serving engine that
+ * gave all free HBM to its own block pool at start-up (a later cudaMalloc fails or fragments the
+ * pool), a plugin that runs inside a region where allocation is forbidden, or a real-time loop that
+ * must not risk the device-wide synchronisation an allocation brings.  For them the library carries
+ * its own scratch: a fixed array of PASK_STATIC_WORKSPACE_BYTES inside the library image, resident on
+ * every GPU the library is used on for the life of the process.  The call allocates and frees
+ * nothing, on the host side too.
+ *   Same arguments and results as pask_decode_attention, minus workspace / workspace_bytes.
+ *   PASK_ERR_WORKSPACE if pask_workspace_bytes(cache, n_seqs) exceeds PASK_STATIC_WORKSPACE_BYTES (a
+ *   large batch or a large max_tokens_per_seq); use pask_decode_attention with a workspace then.
+ *   The first call on a device looks up the scratch's device address (a one-off set-up step); make
+ *   that first call outside of any stream capture.
+ *   All calls, from every cache and stream of the process, share the one scratch per GPU: two calls
+ *   that overlap on the GPU (different streams) race on it and both results are garbage.  Calls
+ *   on one stream are fine.  The scratch keeps whatever the last call left; the kernels rewrite what
+ *   they read, nothing needs clearing. */
+#define PASK_STATIC_WORKSPACE_BYTES (8u << 20)
+pask_status_t pask_decode_attention_static(pask_cache_t *cache, int32_t layer, int32_t n_seqs,
+                                           const int32_t *seq_ids, const void *q, float *out, float *lse,
+                                           pask_stream_t stream);
+
 /* One decode step of one layer from HOST buffers: copies seq_ids, the new token's k, v, tag and
  * the query to the device (into `staging`), appends one token per sequence, runs decode
  * attention and copies `out` back -- all enqueued on `stream`; the host buffers must stay valid

@@ -26,7 +26,7 @@ MAX_GROUPS = 8
 EXPORTS = [
     "pask_load_policy", "pask_free_policy", "pask_policy_action", "pask_cache_sizes", "pask_cache_create",
     "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decode_attention",
-    "pask_decode_attention_full", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes",
+    "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes",
     "pask_budget_state", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
     "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
 ]
@@ -71,6 +71,7 @@ _lib.pask_seq_reset.argtypes = [_vp, _i32, _vp]
 _lib.pask_append_kv.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_decode_attention.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.pask_decode_attention_full.argtypes = _lib.pask_decode_attention.argtypes
+_lib.pask_decode_attention_static.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_workspace_bytes.argtypes = [_vp, _i32]
 _lib.pask_workspace_bytes.restype = _sz
 _lib.pask_decode_step_host.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
@@ -185,6 +186,17 @@ def pask_decode_attention(cache: int, layer: int, seq_ids, q, out, lse, workspac
 def pask_decode_attention_full(cache: int, layer: int, seq_ids, q, out, lse, workspace, stream=None):
     _attention(_lib.pask_decode_attention_full, "pask_decode_attention_full", cache, layer, seq_ids, q, out, lse,
                workspace, stream)
+
+
+STATIC_WORKSPACE_BYTES = 8 << 20
+
+
+def pask_decode_attention_static(cache: int, layer: int, seq_ids, q, out, lse, stream=None):
+    """pask_decode_attention without a workspace argument: the library's built-in scratch is used
+    (for callers that cannot allocate one; see include/pask.h for the limits)."""
+    _check(_lib.pask_decode_attention_static(cache, layer, seq_ids.numel(), _dptr(seq_ids, torch.int32),
+                                             _dptr(q, torch.bfloat16), _dptr(out, torch.float32),
+                                             _dptr(lse, torch.float32), _stream(stream)), "pask_decode_attention_static")
 
 
 def pask_step_staging_bytes(cache: int, n_seqs: int) -> int:

@@ -806,3 +806,40 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
 }
 
 }  // namespace pask
+
+// ---------------------------------------------------------------- decode attention without a caller workspace
+//
+// Scratch for pask_decode_attention_static: the split partials, prefix tables and page-order list of
+// one call live in this array instead of a buffer the caller allocates.  It is part of the library
+// image, so every GPU on which the library runs a kernel holds these bytes until the process exits.
+// In host code the name `g_static_workspace` is only a handle for the runtime; the device address
+// is asked for once per device (cudaGetSymbolAddress) and handed to the kernels.
+namespace {
+constexpr size_t kStaticWorkspaceBytes = PASK_STATIC_WORKSPACE_BYTES;
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
+constexpr int kMaxDevices = 64;
+void *g_static_workspace_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
+}  // namespace
+
+extern "C" pask_status_t pask_decode_attention_static(pask_cache_t *c, int32_t layer, int32_t n_seqs,
+                                                      const int32_t *seq_ids, const void *q, float *out, float *lse,
+                                                      pask_stream_t stream) {
+    if (!c || !seq_ids || !q || !out) return PASK_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->desc.n_layers) return PASK_ERR_INVALID_ARG;
+    if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL) return PASK_ERR_INVALID_ARG;
+    if ((((uintptr_t)q | (uintptr_t)out) & 15) || ((uintptr_t)lse & 3)) return PASK_ERR_INVALID_ARG;
+    // the built-in scratch has a fixed size: a batch (or a page-table bound) that needs more is refused
+    if (pask::attention_workspace_bytes(c, n_seqs) > kStaticWorkspaceBytes) return PASK_ERR_WORKSPACE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PASK_ERR_CUDA;
+    if (!g_static_workspace_addr[dev]) {   // first call on this device: look the array's device address up
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || !ptr) return PASK_ERR_CUDA;
+        g_static_workspace_addr[dev] = ptr;
+    }
+    // Nothing in the scratch has to start at zero: the plan kernel writes the tables before anyone
+    // reads them, and every partial slot that is merged was written earlier in the same call.
+    return pask::launch_attention(c, true, layer, n_seqs, seq_ids, q, out, lse, g_static_workspace_addr[dev],
+                                  kStaticWorkspaceBytes, static_cast<cudaStream_t>(stream));
+}
+
