@@ -96,15 +96,23 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
     }
 }
 // expect_tx + TMA bulk copy global -> this CTA's shared memory, completion counted on an mbarrier;
-// issued by one elected lane of a converged warp (predicated, no divergent branch)
-__device__ __forceinline__ void issue_bulk_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+// issued by one elected lane of a converged warp
+// (predicated, no divergent branch); the same lane leaves `word` at shared address `note`
+__device__ __forceinline__ void issue_bulk_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint32_t note,
+                                                   uint32_t word) {
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
         "elect.sync _|P, 0xffffffff;\n\t"
+        "@P st.shared.u32 [%4], %5;\n\t"
         "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %2;\n\t"
         "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "r"(note), "r"(word)
         : "memory");
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+    return v;
 }
 __device__ __forceinline__ uint4 lds128(uint32_t a) {
     uint4 v;
@@ -277,95 +285,59 @@ attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ 
 
 // ---------------------------------------------------------------- attention kernel
 
-// A CTA's share of one sequence: positions [begin, end) of its page order list.
-struct Segment {
-    uint32_t begin, end;      // global indices into ws.order
-    uint32_t n_high, n_low;   // tokens in the whole streams (for the ragged tail pages)
-};
-
-// Per-warp pipeline.  The producer side walks the CTA's positions and issues one bulk copy per job
-// (HIGH page: K tile, then V tile; LOW page: K and V halves together); the consumer side waits for
-// the jobs in the same order.  Both read page entries out of 32-entry register windows.
+// Per-warp pipeline.  The CTA's share of the work is one contiguous range of the page-order list
+// (sequences follow one another in it).  The producer side walks that range and issues one bulk
+// copy per job (HIGH page: K tile, then V tile; LOW page: K and V halves together), leaving the
+// page's list entry next to the stage's mbarrier; the consumer side waits for the jobs in the same
+// order and reads the entry back, so it needs no bookkeeping of its own.
 struct Pipe {
-    const AttnParams *p;
-    const uint32_t *s_cost, *s_page;
-    uint32_t lo, hi;          // the CTA's span in cost space
+    const uint32_t *order;    // the page-order list
+    const uint8_t *base_high, *base_low;   // pool + this warp's head offset
+    uint32_t stride_high, stride_low;      // page size in bytes
+    uint32_t *status;         // the cache's device status word
     int lane;
-    uint32_t head_high, head_low;   // this warp's head offset inside a page, in 256-byte units
-    uint32_t n_kv_high, n_kv_low;   // page size in 256-byte units
-    uint32_t ring, bars;      // shared-space addresses of this warp's stages and mbarriers
+    uint32_t ring, bars, meta;   // shared-space addresses of this warp's stages, mbarriers and entry words
     // producer
-    int ps;                   // sequence index the producer is in
-    uint32_t p_pos, p_end;    // next position and end of its segment (global indices into ws.order)
+    uint32_t p_pos, p_end;    // next position and end of the CTA's range
     uint32_t p_sub;           // 0: K tile next, 1: V tile next (HIGH pages)
-    uint32_t pw_base, pw_entry;
+    uint32_t pw_base, pw_entry;   // window: lane i holds the entry of position pw_base + i
     uint32_t p_stage;
     // consumer
     uint32_t c_stage, c_parity;
     uint32_t outstanding;
     bool dead;
 
-    __device__ __forceinline__ bool in_span(int s) const { return s < p->n_seqs && s_cost[s] < hi; }
-
-    __device__ __forceinline__ void segment_of(int s, uint32_t &begin, uint32_t &end) const {
-        const uint32_t c0 = s_cost[s], c1 = s_cost[s + 1], cs = c1 - c0, n = s_page[s + 1] - s_page[s];
-        const uint32_t a = (lo > c0 ? lo : c0) - c0, e = (hi < c1 ? hi : c1) - c0;
-        begin = s_page[s] + cut_positions(a, cs, n);
-        end = s_page[s] + cut_positions(e, cs, n);
-    }
-
-    // advance the producer to the next sequence of the span that has pages for this CTA
-    __device__ __forceinline__ void producer_open(int s) {
-        for (; in_span(s); ++s) {
-            if (s_cost[s + 1] == s_cost[s]) continue;
-            segment_of(s, p_pos, p_end);
-            if (p_pos < p_end) break;
-        }
-        if (!in_span(s)) { s = p->n_seqs; p_pos = p_end = 0; }
-        ps = s;
-        p_sub = 0;
-        pw_base = 0x80000000u;   // forces a window refill at the first job
-    }
-
     // Issue the next job into stage p_stage.  Warp-uniform.
     __device__ __forceinline__ void produce() {
         if (p_pos == p_end) return;
         if (p_pos - pw_base >= 32u) {
             pw_base = p_pos;
-            pw_entry = p_pos + lane < p_end ? __ldg(p->ws.order + p_pos + lane) : 0u;
+            pw_entry = p_pos + lane < p_end ? __ldg(order + p_pos + lane) : 0u;
         }
         const uint32_t entry = __shfl_sync(0xffffffffu, pw_entry, (int)(p_pos - pw_base));
         const uint32_t id = entry & kOrderIdMask;
         const bool is_high = entry & kOrderHigh;
-        const uint8_t *src;
-        uint32_t bytes;
-        if (is_high) {
-            src = p->c.pool_high + (size_t)(id * n_kv_high + head_high + p_sub * (kHighTileBytes / 256)) * 256;
-            bytes = kHighTileBytes;
-        } else {
-            src = p->c.pool_low + (size_t)(id * n_kv_low + head_low) * 256;
-            bytes = kLowHeadBytes;
-        }
-        issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bars + p_stage * 8);
+        const uint8_t *src = is_high ? base_high + (size_t)id * stride_high + p_sub * kHighTileBytes
+                                     : base_low + (size_t)id * stride_low;
+        const uint32_t bytes = is_high ? kHighTileBytes : kLowHeadBytes;
+        issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bars + p_stage * 8, meta + p_stage * 4, entry);
         p_stage = p_stage + 1 == kStages ? 0 : p_stage + 1;
         outstanding++;
-        if (is_high && p_sub == 0) {
-            p_sub = 1;
-        } else {
-            p_sub = 0;
-            if (++p_pos == p_end) producer_open(ps + 1);
-        }
+        const uint32_t page_done = is_high ? p_sub : 1u;   // a HIGH page is two jobs
+        p_sub = is_high ? p_sub ^ 1u : 0u;
+        p_pos += page_done;
     }
 
-    // Wait for the oldest outstanding job; returns the shared address of its stage.
-    __device__ __forceinline__ uint32_t acquire() {
+    // Wait for the oldest outstanding job; returns the shared address of its stage and the page's entry.
+    __device__ __forceinline__ uint32_t acquire(uint32_t &entry) {
         const uint32_t bar = bars + c_stage * 8;
         if (!mbar_try_wait(bar, c_parity)) {
             if (dead || !mbar_wait_slow(bar, c_parity)) {
-                if (!dead && lane == 0) atomicOr(&p->c.ctrl[kCtrlStatus], PASK_DEV_TIMEOUT);
+                if (!dead && lane == 0) atomicOr(status, PASK_DEV_TIMEOUT);
                 dead = true;
             }
         }
+        entry = lds32(meta + c_stage * 4);
         return ring + c_stage * kStageBytes;
     }
     // All lanes are done reading the oldest stage: hand it back to the producer.
@@ -389,7 +361,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     uint32_t *s_page = s_cost + n_seqs + 1;
     size_t off = ((size_t)(2 * n_seqs + 2) * 4 + 127) & ~(size_t)127;
     uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + off);
-    off += 256;                                             // kMaxWarps * kStages * 8 = 192 bytes of barriers
+    off += 384;                                             // 192 bytes of barriers + 96 bytes of entry words
     off = (off + 1023) & ~(size_t)1023;
     uint8_t *s_ring = smem + off;
     uint8_t *s_scratch = s_ring + (size_t)n_warps * kStages * kStageBytes;
@@ -418,12 +390,31 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         s0 = a - 1;
     }
 
+    // the CTA's range of the page-order list, and this warp's pipeline over it
+    auto position_of = [&](uint32_t x) -> uint32_t {   // first position at or after cost offset x
+        if (x >= total) return s_page[n_seqs];
+        int a = 1, e = n_seqs;                          // smallest idx in [1, n_seqs] with cost[idx] > x
+        while (a < e) {
+            const int mid = (a + e) >> 1;
+            if (s_cost[mid] > x) e = mid; else a = mid + 1;
+        }
+        const int s = a - 1;
+        return s_page[s] + cut_positions(x - s_cost[s], s_cost[s + 1] - s_cost[s], s_page[s + 1] - s_page[s]);
+    };
     Pipe w;
-    w.p = &p; w.s_cost = s_cost; w.s_page = s_page; w.lo = lo; w.hi = hi; w.lane = lane;
-    w.n_kv_high = (uint32_t)c.n_kv * (kHighHeadBytes / 256); w.head_high = (uint32_t)warp * (kHighHeadBytes / 256);
-    w.n_kv_low = (uint32_t)c.n_kv * (kLowHeadBytes / 256); w.head_low = (uint32_t)warp * (kLowHeadBytes / 256);
+    w.order = p.ws.order;
+    w.base_high = c.pool_high + (size_t)warp * kHighHeadBytes;
+    w.base_low = c.pool_low + (size_t)warp * kLowHeadBytes;
+    w.stride_high = c.high_page_bytes;
+    w.stride_low = c.low_page_bytes;
+    w.status = c.ctrl + kCtrlStatus;
+    w.lane = lane;
     w.ring = smem_u32(s_ring + (size_t)warp * kStages * kStageBytes);
     w.bars = smem_u32(s_bar + warp * kStages);
+    w.meta = smem_u32(s_bar) + kMaxWarps * kStages * 8 + warp * kStages * 4;   // after the 192 bytes of barriers
+    w.p_pos = position_of(lo);
+    w.p_end = position_of(hi);
+    w.p_sub = 0; w.pw_base = 0x80000000u; w.pw_entry = 0;
     w.p_stage = 0; w.c_stage = 0; w.c_parity = 0; w.outstanding = 0; w.dead = false;
     const uint32_t scratch = smem_u32(s_scratch + (size_t)warp * kScratchBytes);
     if (lane == 0) {
@@ -432,7 +423,6 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncwarp();
-    w.producer_open(s0);
     for (int i = 0; i < kStages; i++) w.produce();
 
     const float kLog2Scale = 0.088388347648318440550f * 1.4426950408889634074f;  // log2(e) / sqrt(128)
@@ -442,15 +432,14 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     // selector that broadcasts the fp16 scale of this lane's column group (low or high half of a word)
     const uint32_t bsel = (t >> 1) ? 0x3232u : 0x1010u;
 
-    for (int s = s0; w.in_span(s); ++s) {
+    for (int s = s0; s < n_seqs && s_cost[s] < hi; ++s) {
         if (s_cost[s + 1] == s_cost[s]) continue;
-        Segment seg;
-        w.segment_of(s, seg.begin, seg.end);
-        {
-            const uint2 tk = __ldg(p.ws.tokens + s);
-            seg.n_high = tk.x;
-            seg.n_low = tk.y;
-        }
+        const uint32_t c0 = s_cost[s], c1 = s_cost[s + 1], n_pos = s_page[s + 1] - s_page[s];
+        // number of this sequence's pages that fall to this CTA (same cuts as position_of)
+        const uint32_t n_pages = cut_positions((hi < c1 ? hi : c1) - c0, c1 - c0, n_pos) -
+                                 cut_positions((lo > c0 ? lo : c0) - c0, c1 - c0, n_pos);
+        const uint2 tk = __ldg(p.ws.tokens + s);
+        const uint32_t seq_n_high = tk.x, seq_n_low = tk.y;
 
         // ---- query fragments: lane (g,t) holds dims 8(4j+t) .. +7 of head g & 3 for j = 0..3
         uint4 qf[4];
@@ -464,7 +453,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         // scales of LOW tokens, P of HIGH tokens) and the partial is multiplied by `up` = 2^-k.
         uint32_t down = 0x3C003C00u;
         float down_f = 1.0f, up = 1.0f;
-        if (kHasLow && seg.n_low > 0) {
+        if (kHasLow && seq_n_low > 0) {
             // fp16 copies of q for the LOW stream's MMAs.  Its A operands are 1024 + code (register
             // pairs x, z of a chunk) and 1024 + 16 code (pairs y, w), so q is stored as is for the
             // former and divided by 16 for the latter, and -(1032 b) resp. -(1152 b) summed over a
@@ -511,20 +500,15 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         for (int m = 0; m < 8; m++) acc[m][0] = acc[m][1] = acc[m][2] = acc[m][3] = 0.f;
         float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
 
-        uint32_t cw_base = 0x80000000u, cw_entry = 0;
-        for (uint32_t pos = seg.begin; pos < seg.end; ++pos) {
-            if (pos - cw_base >= 32u) {
-                cw_base = pos;
-                cw_entry = pos + lane < seg.end ? __ldg(p.ws.order + pos + lane) : 0u;
-            }
-            const uint32_t entry = __shfl_sync(0xffffffffu, cw_entry, (int)(pos - cw_base));
+        for (uint32_t page = 0; page < n_pages; ++page) {
+            uint32_t entry;
+            uint32_t st = w.acquire(entry);
+            if (w.dead) break;
             const bool is_high = entry & kOrderHigh;
             uint32_t n_valid = 16u;
-            if (entry & kOrderTail) n_valid = (is_high ? seg.n_high : seg.n_low) & (kPageTokens - 1);
+            if (entry & kOrderTail) n_valid = (is_high ? seq_n_high : seq_n_low) & (kPageTokens - 1);
 
             float sc[4] = {0.f, 0.f, 0.f, 0.f};
-            uint32_t st = w.acquire();
-            if (w.dead) break;
             if (is_high) {
                 // ---- QK^T over a bf16 K tile: 8 MMAs, two independent accumulators
                 float sc2[4] = {0.f, 0.f, 0.f, 0.f};
@@ -597,7 +581,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 split_pair(p2 * down_f, p3 * down_f, h23, l23);
                 const uint32_t bh0 = movmatrix_trans(h01), bh1 = movmatrix_trans(h23);
                 const uint32_t bl0 = movmatrix_trans(l01), bl1 = movmatrix_trans(l23);
-                st = w.acquire();
+                st = w.acquire(entry);
                 if (w.dead) break;
 #pragma unroll
                 for (int e = 0; e < 2; e++) {
@@ -745,7 +729,7 @@ combine_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ p
 }
 
 size_t attn_smem_bytes(int n_seqs, int n_warps) {
-    size_t off = align_up((size_t)(2 * n_seqs + 2) * 4, 128) + 256;
+    size_t off = align_up((size_t)(2 * n_seqs + 2) * 4, 128) + 384;
     off = align_up(off, 1024);
     return off + (size_t)n_warps * (kStages * kStageBytes + kScratchBytes);
 }
