@@ -265,6 +265,9 @@ pask_status_t pask_debug_dump_high(pask_cache_t *cache, int32_t layer, int32_t s
 pask_status_t pask_debug_dump_low(pask_cache_t *cache, int32_t layer, int32_t seq, uint8_t *k_codes,
                                   uint16_t *k_scales, uint8_t *v_codes, uint16_t *v_scales, uint32_t *pages_out,
                                   pask_stream_t stream);
+/* Page ids only (no page contents): high_out [ceil(n_high/16)], low_out [ceil(n_low/16)]; either may be NULL. */
+pask_status_t pask_debug_page_ids(pask_cache_t *cache, int32_t layer, int32_t seq, uint32_t *high_out, uint32_t *low_out,
+                                  pask_stream_t stream);
 /* out[4] = { high bump counter, high free-stack depth, low bump counter, low free-stack depth }. */
 pask_status_t pask_debug_pool_state(pask_cache_t *cache, uint32_t *out4, pask_stream_t stream);
 /* The cache's first `count` (<= 64) control words: [0] device status, [2..5] pool state, [16..23]

@@ -28,7 +28,7 @@ EXPORTS = [
     "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decode_attention",
     "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes",
     "pask_budget_state", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
-    "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
+    "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
 ]
 
 
@@ -83,6 +83,7 @@ _lib.pask_debug_stream_len.argtypes = [_vp, _i32, _i32, C.POINTER(C.c_uint32), C
 _lib.pask_debug_dump_high.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp]
 _lib.pask_debug_dump_low.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_debug_pool_state.argtypes = [_vp, _vp, _vp]
+_lib.pask_debug_page_ids.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp]
 _lib.pask_debug_ctrl_words.argtypes = [_vp, _vp, _i32, _vp]
 _lib.pask_debug_partition.argtypes = [_i32, _vp, _vp, _i32, _vp]
 _lib.pask_debug_page_order.argtypes = [C.c_uint32, C.c_uint32, _vp]
@@ -257,6 +258,14 @@ def pask_debug_dump_low(cache: int, layer: int, seq: int, n_kv: int, stream=None
     _check(_lib.pask_debug_dump_low(cache, layer, seq, kc.ctypes.data, ks.ctypes.data, vc.ctypes.data, vs.ctypes.data,
                                     pages.ctypes.data, _stream(stream)), "pask_debug_dump_low")
     return kc, ks, vc, vs, pages
+
+
+def pask_debug_page_ids(cache: int, layer: int, seq: int, stream=None):
+    import numpy as np
+    nh, nl = pask_debug_stream_len(cache, layer, seq, stream)
+    hi, lo = np.zeros((nh + 15) // 16, np.uint32), np.zeros((nl + 15) // 16, np.uint32)
+    _check(_lib.pask_debug_page_ids(cache, layer, seq, hi.ctypes.data, lo.ctypes.data, _stream(stream)), "pask_debug_page_ids")
+    return hi, lo
 
 
 def pask_debug_pool_state(cache: int, stream=None):

@@ -372,6 +372,21 @@ pask_status_t pask_debug_ctrl_words(pask_cache_t *c, uint32_t *out, int32_t coun
     return cuda_rc(cudaMemcpy(out, c->dev.ctrl, (size_t)count * 4, cudaMemcpyDeviceToHost));
 }
 
+pask_status_t pask_debug_page_ids(pask_cache_t *c, int32_t layer, int32_t seq, uint32_t *high_out, uint32_t *low_out,
+                                  pask_stream_t stream) {
+    if (!c || !seq_layer_ok(c, layer, seq)) return PASK_ERR_INVALID_ARG;
+    uint32_t nh = 0, nl = 0;
+    pask_status_t rc = read_lens(c, layer, seq, &nh, &nl, static_cast<cudaStream_t>(stream));
+    if (rc != PASK_OK) return rc;
+    const size_t tbl = ((size_t)seq * c->desc.n_layers + layer) * c->dev.max_pages;
+    const uint32_t ph = (nh + kPageTokens - 1) / kPageTokens, pl = (nl + kPageTokens - 1) / kPageTokens;
+    if (high_out && ph && cudaMemcpy(high_out, c->dev.tbl_high + tbl, (size_t)ph * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return PASK_ERR_CUDA;
+    if (low_out && pl && cudaMemcpy(low_out, c->dev.tbl_low + tbl, (size_t)pl * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return PASK_ERR_CUDA;
+    return PASK_OK;
+}
+
 pask_status_t pask_debug_dump_high(pask_cache_t *c, int32_t layer, int32_t seq, uint16_t *k_out, uint16_t *v_out,
                                    uint32_t *pages_out, pask_stream_t stream) {
     if (!c || !seq_layer_ok(c, layer, seq)) return PASK_ERR_INVALID_ARG;
