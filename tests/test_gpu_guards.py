@@ -1,0 +1,112 @@
+"""Memory-safety and determinism checks on the GPU: caller-owned buffers are wrapped in canary
+regions that must survive every kernel, the same calls on two caches must leave byte-identical
+pools, page tables and outputs, and a stream may be filled exactly to its bound."""
+import numpy as np
+import pytest
+import torch
+
+from pask_workloads import configs as WC
+
+pytestmark = pytest.mark.gpu
+
+GUARD = 4096          # bytes of canary before and after each buffer
+PATTERN = 0xA5
+
+
+def _guarded(nbytes, device):
+    """A zero-filled buffer of nbytes (256-byte aligned) inside a larger allocation painted with a canary."""
+    total = GUARD + nbytes + GUARD
+    raw = torch.full((total + 256,), PATTERN, dtype=torch.uint8, device=device)
+    off = (-raw.data_ptr()) % 256
+    whole = raw[off:off + total]
+    whole[GUARD:GUARD + nbytes] = 0
+    return raw, whole, whole[GUARD:GUARD + nbytes]
+
+
+def _canaries_intact(whole, nbytes):
+    return bool((whole[:GUARD] == PATTERN).all()) and bool((whole[GUARD + nbytes:] == PATTERN).all())
+
+
+def _run(P, w, device):
+    """Bulk append + three decode steps + attention on caller-created, canary-guarded buffers."""
+    cfg = w.cfg
+    lens = [w.total_len(b) for b in range(cfg.batch)]
+    pages = cfg.n_layers * (sum(lens) // 16 + 4 * cfg.batch)
+    desc = P.CacheDesc(cfg.n_layers, cfg.n_q, cfg.n_kv, 128, 16, cfg.batch, max(lens) + 16, sum(lens), pages, pages)
+    sizes = P.pask_cache_sizes(desc)
+    bufs = [_guarded(n, device) for n in (sizes.pool_high_bytes, sizes.pool_low_bytes, sizes.meta_bytes)]
+    policy = P.pask_load_policy(w.blob)
+    h = P.pask_cache_create(desc, policy, bufs[0][2], bufs[1][2], bufs[2][2])
+    ws_raw, ws_whole, ws = _guarded(P.pask_workspace_bytes(h, cfg.batch), device)
+    ids = torch.arange(cfg.batch, dtype=torch.int32, device=device)
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device=device)
+    tags = torch.from_numpy(np.concatenate([w.tags(b, 0, lens[b]) for b in range(cfg.batch)])).to(device)
+    outs = []
+    for layer in range(cfg.n_layers):
+        k = torch.cat([w.kv(layer, b, 0, lens[b])[0] for b in range(cfg.batch)]).to(device)
+        v = torch.cat([w.kv(layer, b, 0, lens[b])[1] for b in range(cfg.batch)]).to(device)
+        P.pask_append_kv(h, layer, ids, cu, k, v, tags)
+    cu1 = torch.arange(cfg.batch + 1, dtype=torch.int32, device=device)
+    for step in range(3):
+        for layer in range(cfg.n_layers):
+            k = torch.stack([w.kv(layer, b, lens[b] + step, 1)[0][0] for b in range(cfg.batch)]).to(device)
+            v = torch.stack([w.kv(layer, b, lens[b] + step, 1)[1][0] for b in range(cfg.batch)]).to(device)
+            t = torch.from_numpy(np.array([w.tags(b, lens[b] + step, 1)[0] for b in range(cfg.batch)], np.uint8)).to(device)
+            q = torch.stack([w.q(layer, b, lens[b] + step + 1) for b in range(cfg.batch)]).to(device)
+            out = torch.empty((cfg.batch, cfg.n_q, 128), dtype=torch.float32, device=device)
+            lse = torch.empty((cfg.batch, cfg.n_q), dtype=torch.float32, device=device)
+            P.pask_append_kv(h, layer, ids, cu1, k, v, t)
+            P.pask_decode_attention(h, layer, ids, q, out, lse, ws)
+            outs.append(out)
+    torch.cuda.synchronize()
+    assert P.pask_budget_state(h, 0).device_status == 0
+    sizes_list = (sizes.pool_high_bytes, sizes.pool_low_bytes, sizes.meta_bytes)
+    for (raw, whole, inner), n in zip(bufs, sizes_list):
+        assert _canaries_intact(whole, n)
+    assert _canaries_intact(ws_whole, ws.numel())
+    # snapshot: pools, and the meta without the status/ticket control words' volatile parts
+    snap = [bufs[0][2].clone(), bufs[1][2].clone(), bufs[2][2].clone(), torch.stack(outs).clone()]
+    P.pask_cache_destroy(h)
+    P.pask_free_policy(policy)
+    return snap
+
+
+def test_canaries_survive_and_runs_are_deterministic():
+    import paper_2608_28276_b200 as P
+    dev = torch.device("cuda", 0)
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=5, n_layers=2, n_groups=2, prompt_len=450, gen_len=390)
+    w = WC.build(cfg)
+    a = _run(P, w, dev)
+    b = _run(P, w, dev)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)          # pools, meta (tables, counters, budgets) and outputs: byte for byte
+
+
+def test_stream_filled_exactly_to_its_bound():
+    import paper_2608_28276_b200 as P
+    d = "cuda"
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=1, n_layers=1, n_groups=1, lut="all_high")
+    w = WC.build(cfg)
+    cache = P.Cache(w.blob, 1, cfg.n_q, cfg.n_kv, 1, 64, 64, 4, 4)      # streams of at most 64 tokens = 4 pages
+    ids = torch.zeros(1, dtype=torch.int32, device=d)
+    k, v = w.kv(0, 0, 0, 64)
+    tags = torch.zeros(64, dtype=torch.uint8, device=d)
+    P.pask_append_kv(cache.handle, 0, ids, torch.tensor([0, 63], dtype=torch.int32, device=d), k[:63].to(d), v[:63].to(d), tags[:63].contiguous())
+    P.pask_append_kv(cache.handle, 0, ids, torch.tensor([0, 1], dtype=torch.int32, device=d), k[63:].to(d), v[63:].to(d), tags[:1].contiguous())
+    assert P.pask_debug_stream_len(cache.handle, 0, 0) == (64, 0)
+    assert P.pask_budget_state(cache.handle, 0).device_status == 0
+    assert P.pask_debug_pool_state(cache.handle) == (4, 0, 0, 0)
+    # full attention over exactly four full pages equals the library routine
+    q = w.q(0, 0, 64)
+    out = torch.empty((1, cfg.n_q, 128), dtype=torch.float32, device=d)
+    P.pask_decode_attention(cache.handle, 0, ids, q.unsqueeze(0).to(d), out, None, cache.workspace(1))
+    kk = k.double().repeat_interleave(4, dim=1).permute(1, 0, 2)
+    vv = v.double().repeat_interleave(4, dim=1).permute(1, 0, 2)
+    sc = torch.einsum("hd,hnd->hn", q.double(), kk) / 128 ** 0.5
+    ref = torch.einsum("hn,hnd->hd", torch.softmax(sc, -1), vv)
+    assert float((out[0].cpu().double() - ref).abs().max()) < 2e-3
+    # one more token does not fit: refused, flagged, nothing changes
+    P.pask_append_kv(cache.handle, 0, ids, torch.tensor([0, 1], dtype=torch.int32, device=d), k[:1].to(d), v[:1].to(d), tags[:1].contiguous())
+    assert P.pask_budget_state(cache.handle, 0).device_status == P.DEV_SEQ_OVERFLOW
+    assert P.pask_debug_stream_len(cache.handle, 0, 0) == (64, 0)
+    cache.close()
