@@ -98,8 +98,20 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
 // expect_tx + TMA bulk copy global -> this CTA's shared memory, completion counted on an mbarrier;
 // issued by one elected lane of a converged warp
 // (predicated, no divergent branch); the same lane leaves `word` at shared address `note`
+// The copy carries an L2 evict-first hint: every page is read exactly once per call.
 __device__ __forceinline__ void issue_bulk_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint32_t note,
-                                                   uint32_t word) {
+                                                   uint32_t word, uint64_t policy) {
+#ifndef PASK_NO_EVICT_FIRST
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xffffffff;\n\t"
+        "@P st.shared.u32 [%4], %5;\n\t"
+        "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %2;\n\t"
+        "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %6;\n\t}"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "r"(note), "r"(word), "l"(policy)
+        : "memory");
+#else
+    (void)policy;
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
         "elect.sync _|P, 0xffffffff;\n\t"
@@ -108,6 +120,12 @@ __device__ __forceinline__ void issue_bulk_elected(uint32_t dst, const void *src
         "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "r"(note), "r"(word)
         : "memory");
+#endif
+}
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
 }
 __device__ __forceinline__ uint32_t lds32(uint32_t a) {
     uint32_t v;
@@ -295,6 +313,7 @@ struct Pipe {
     const uint8_t *base_high, *base_low;   // pool + this warp's head offset
     uint32_t stride_high, stride_low;      // page size in bytes
     uint32_t *status;         // the cache's device status word
+    uint64_t policy;          // L2 cache policy of the bulk copies
     int lane;
     uint32_t ring, bars, meta;   // shared-space addresses of this warp's stages, mbarriers and entry words
     // producer
@@ -320,7 +339,7 @@ struct Pipe {
         const uint8_t *src = is_high ? base_high + (size_t)id * stride_high + p_sub * kHighTileBytes
                                      : base_low + (size_t)id * stride_low;
         const uint32_t bytes = is_high ? kHighTileBytes : kLowHeadBytes;
-        issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bars + p_stage * 8, meta + p_stage * 4, entry);
+        issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bars + p_stage * 8, meta + p_stage * 4, entry, policy);
         p_stage = p_stage + 1 == kStages ? 0 : p_stage + 1;
         outstanding++;
         const uint32_t page_done = is_high ? p_sub : 1u;   // a HIGH page is two jobs
@@ -408,6 +427,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     w.stride_high = c.high_page_bytes;
     w.stride_low = c.low_page_bytes;
     w.status = c.ctrl + kCtrlStatus;
+    w.policy = l2_evict_first_policy();
     w.lane = lane;
     w.ring = smem_u32(s_ring + (size_t)warp * kStages * kStageBytes);
     w.bars = smem_u32(s_bar + warp * kStages);
