@@ -21,7 +21,9 @@ class Budget(C.Structure):
                 ("n_low", C.c_uint64 * MAX_GROUPS), ("n_drop", C.c_uint64 * MAX_GROUPS),
                 ("retained_bytes", C.c_uint64), ("full_bytes", C.c_uint64),
                 ("remaining_bytes", C.c_int64), ("bad_tags", C.c_uint64),
-                ("pages_high", C.c_uint32), ("pages_low", C.c_uint32)]
+                ("pages_high", C.c_uint32), ("pages_low", C.c_uint32),
+                ("decided_full_bytes", C.c_uint64), ("decided_retained_bytes", C.c_uint64),
+                ("n_demoted", C.c_uint64), ("n_promoted", C.c_uint64), ("n_floor_conflicts", C.c_uint64)]
 
 
 _lib = None
@@ -50,6 +52,8 @@ def lib():
         L.orc_cache_destroy.restype = None
         L.orc_seq_reset.argtypes = [vp, i32]
         L.orc_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.orc_append_decided.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.orc_decide.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.orc_stream_len.argtypes = [vp, i32, i32, C.POINTER(u32), C.POINTER(u32)]
         L.orc_dump_high.argtypes = [vp, i32, i32, vp, vp, vp]
         L.orc_dump_low.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
@@ -123,8 +127,25 @@ class Cache:
             lib().orc_cache_destroy(self.h)
             self.h = None
 
-    def append(self, layer, seq_ids, cu_tokens, k_bits, v_bits, tags):
-        """k_bits / v_bits: int16/uint16 [total][n_kv][128]; returns (status, actions u8 [total])."""
+    def decide(self, seq_ids, cu_tokens, tags, states=None, n_groups=None):
+        """Algorithm 2 steps 1-6 and 8; returns (status, actions u8 [total][n_groups])."""
+        seq_ids = np.ascontiguousarray(seq_ids, dtype=np.int32)
+        cu = np.ascontiguousarray(cu_tokens, dtype=np.int32)
+        tags = np.ascontiguousarray(tags, dtype=np.uint8)
+        total = int(cu[-1])
+        assert tags.size == total
+        st = None
+        if states is not None:
+            st = np.ascontiguousarray(states, dtype=np.uint16)
+            assert st.size == total
+        actions = np.full((total, n_groups), 0xEE, dtype=np.uint8)
+        rc = lib().orc_decide(self.h, len(seq_ids), _ptr(seq_ids), _ptr(cu), _ptr(tags),
+                              _ptr(st) if st is not None else None, _ptr(actions))
+        return rc, actions
+
+    def append(self, layer, seq_ids, cu_tokens, k_bits, v_bits, tags, decided=None):
+        """k_bits / v_bits: int16/uint16 [total][n_kv][128]; returns (status, actions u8 [total]).
+        decided: u8 [total][n_groups] from decide(), persisted instead of the table's actions."""
         seq_ids = np.ascontiguousarray(seq_ids, dtype=np.int32)
         cu = np.ascontiguousarray(cu_tokens, dtype=np.int32)
         k = np.ascontiguousarray(k_bits).view(np.uint16)
@@ -133,8 +154,12 @@ class Cache:
         total = int(cu[-1])
         assert k.size == total * self.n_kv * 128 and v.size == k.size and tags.size == total
         actions = np.full(total, 0xEE, dtype=np.uint8)
-        rc = lib().orc_append(self.h, layer, len(seq_ids), _ptr(seq_ids), _ptr(cu), _ptr(k), _ptr(v), _ptr(tags),
-                              _ptr(actions))
+        dec = None
+        if decided is not None:
+            dec = np.ascontiguousarray(decided, dtype=np.uint8)
+            assert dec.ndim == 2 and dec.shape[0] == total
+        rc = lib().orc_append_decided(self.h, layer, len(seq_ids), _ptr(seq_ids), _ptr(cu), _ptr(k), _ptr(v),
+                                      _ptr(tags), _ptr(dec) if dec is not None else None, _ptr(actions))
         return rc, actions
 
     def stream_len(self, layer, seq):

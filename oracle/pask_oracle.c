@@ -13,6 +13,10 @@
  *   - the frozen table stores selected action, floor and upgrade scores per bucket (end of
  *     Section 3.3); online, a = max(a0, a_floor) (Eq. 10, Algorithm 2 steps 1-2);
  *   - Persist(a) (Algorithm 2 step 7) and the budget recurrence R' = R - sum m(a) (step 8);
+ *   - the dynamic adjustment between them (Algorithm 2 steps 3-6, Eq. 10 and the paragraph after
+ *     it): B = [R - Gamma(s)]+, demotions above the floors in ascending upgrade score while the
+ *     token's cost exceeds B, promotions in descending score in critical states while they fit,
+ *     floors first when budget and protection conflict (orc_decide);
  *   - normalised cost C_KV = sum m(a) / sum m(H) (Eq. 1);
  *   - the reference policy is full high precision (Section 3.1), whose attention outputs are the
  *     ones Eq. 4 compares against: plain softmax(q k^T / sqrt(d)) v over the retained history.
@@ -24,7 +28,10 @@
  * are handed out in call order from a per-pool free stack, else a bump counter; costs are
  * payload bytes.  Parity unpinned by the paper for: the low-bit format itself, the absence of a
  * recent window, the initial budget, and the treatment of prompt tags -- those are pinned only
- * by this library's own documentation.
+ * by this library's own documentation.  The paper gives Demote, Promote and Crit in one sentence
+ * each and R's starting value not at all: the reading written out above decide_token (budget
+ * accrued per token seen, one step at a time, ties to the first group, "eligible" = fits in B)
+ * is this library's, pinned by hand-worked cases and invariants, not by values the paper prints.
  *
  * Arithmetic: decisions, codes, scales, page ids and counters are integer / IEEE fp32 with no
  * contraction (build with -ffp-contract=off); attention is fp64 over the dequantised values.
@@ -56,7 +63,9 @@ typedef struct {
     uint8_t *a0, *a_floor;  /* [n_tags * n_groups] */
     uint8_t *eff;           /* max(a0, a_floor) */
     float *rho_rl, *rho_lh;
-    uint32_t *gamma;
+    uint32_t *gamma;        /* [n_states] reserve, in units of 2^gamma_shift bytes */
+    uint8_t *crit;          /* [n_states] 1 = critical or lookahead-critical state */
+    uint32_t gamma_shift;
 } orc_policy;
 
 typedef struct {
@@ -65,6 +74,9 @@ typedef struct {
     int64_t remaining_bytes;
     uint64_t bad_tags;
     uint32_t pages_high, pages_low;
+    /* Algorithm 2's own running budget, advanced by orc_decide (one step per token, all groups) */
+    uint64_t decided_full_bytes, decided_retained_bytes;
+    uint64_t n_demoted, n_promoted, n_floor_conflicts;
 } orc_budget;
 
 typedef struct {          /* one (sequence, layer) pair: two compacted streams */
@@ -178,13 +190,15 @@ static uint32_t rd32(const uint8_t *p) {
 void orc_policy_free(orc_policy *p) {
     if (!p) return;
     free(p->layer_group); free(p->a0); free(p->a_floor); free(p->eff);
-    free(p->rho_rl); free(p->rho_lh); free(p->gamma);
+    free(p->rho_rl); free(p->rho_lh); free(p->gamma); free(p->crit);
     free(p);
 }
 
 orc_policy *orc_policy_load(const uint8_t *blob, size_t len, int *err) {
     *err = ORC_ERR_POLICY;
-    if (!blob || len < 40 || memcmp(blob, "PASK", 4) != 0 || rd32(blob + 4) != 1) return NULL;
+    if (!blob || len < 40 || memcmp(blob, "PASK", 4) != 0) return NULL;
+    const uint32_t version = rd32(blob + 4);
+    if (version != 1 && version != 2) return NULL;
     orc_policy *p = (orc_policy *)calloc(1, sizeof(*p));
     p->n_tags = rd32(blob + 8); p->n_groups = rd32(blob + 12); p->n_layers = rd32(blob + 16);
     p->n_states = rd32(blob + 20); p->budget_q16 = rd32(blob + 24); p->recent_window = rd32(blob + 28);
@@ -195,12 +209,14 @@ orc_policy *orc_policy_load(const uint8_t *blob, size_t len, int *err) {
     size_t lg_pad = (p->n_layers + 3u) & ~(size_t)3u;
     size_t n_ent = (size_t)p->n_tags * p->n_groups;
     size_t need = 40 + lg_pad + n_ent * 12 + (size_t)p->n_states * 4;
+    if (version == 2) need += 4 + (((size_t)p->n_states + 3u) & ~(size_t)3u);
     if (len != need) { free(p); return NULL; }
     p->layer_group = (uint8_t *)malloc(p->n_layers);
     memcpy(p->layer_group, blob + 40, p->n_layers);
     p->a0 = (uint8_t *)malloc(n_ent); p->a_floor = (uint8_t *)malloc(n_ent); p->eff = (uint8_t *)malloc(n_ent);
     p->rho_rl = (float *)malloc(n_ent * 4); p->rho_lh = (float *)malloc(n_ent * 4);
     p->gamma = (uint32_t *)malloc((size_t)p->n_states * 4 + 4);
+    p->crit = (uint8_t *)calloc((size_t)p->n_states + 4, 1);
     int bad = 0;
     for (uint32_t l = 0; l < p->n_layers; l++) if (p->layer_group[l] >= p->n_groups) bad = 1;
     const uint8_t *e = blob + 40 + lg_pad;
@@ -208,9 +224,15 @@ orc_policy *orc_policy_load(const uint8_t *blob, size_t len, int *err) {
         p->a0[i] = e[0]; p->a_floor[i] = e[1];
         if (e[0] > ACT_H || e[1] > ACT_H || e[2] || e[3]) bad = 1;
         memcpy(&p->rho_rl[i], e + 4, 4); memcpy(&p->rho_lh[i], e + 8, 4);
+        if (isnan(p->rho_rl[i]) || isnan(p->rho_lh[i])) bad = 1;   /* scores must be comparable */
         p->eff[i] = (uint8_t)orc_lut_fold(e[0], e[1]);
     }
     for (uint32_t s = 0; s < p->n_states; s++, e += 4) p->gamma[s] = rd32(e);
+    if (version == 2) {
+        p->gamma_shift = rd32(e); e += 4;
+        if (p->gamma_shift > 16) bad = 1;
+        for (uint32_t s = 0; s < p->n_states; s++) { p->crit[s] = e[s]; if (e[s] > 1) bad = 1; }
+    }
     if (bad) { orc_policy_free(p); return NULL; }
     *err = ORC_OK;
     return p;
@@ -283,13 +305,26 @@ static int decide(const orc_policy *p, int group, uint8_t tag, int *bad) {
          while (nc < (need)) nc *= 2;                                          \
          (ptr) = realloc((ptr), (size_t)nc * (elem)); (cap) = nc; } } while (0)
 
+/* The action of token t at layer group `group`: the table's (Algorithm 2 steps 1-2), or, when
+ * `decided` is given, the one orc_decide chose for it (steps 3-6), row t of [total][n_groups]. */
+static int action_of(const orc_policy *p, int group, const uint8_t *tags, const uint8_t *decided, int t, int *bad) {
+    int a = decide(p, group, tags[t], bad);
+    if (decided) a = decided[(size_t)t * p->n_groups + group];
+    return a;
+}
+
 /* Algorithm 2 steps 1, 2, 7, 8 for one layer call.  Sequences in call order, tokens in order.
- * If the call needs more pages than a pool can supply nothing changes at all. */
-int orc_append(orc_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,
-               const uint16_t *k_bits, const uint16_t *v_bits, const uint8_t *tags, uint8_t *actions_out) {
+ * If the call needs more pages than a pool can supply nothing changes at all.
+ * With `decided` (may be NULL) step 7 persists the actions chosen by orc_decide instead. */
+int orc_append_decided(orc_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,
+                       const uint16_t *k_bits, const uint16_t *v_bits, const uint8_t *tags, const uint8_t *decided,
+                       uint8_t *actions_out) {
     const orc_policy *p = c->pol;
     if (layer < 0 || (uint32_t)layer >= p->n_layers || n_seqs < 0) return ORC_ERR_ARG;
     int group = p->layer_group[layer];
+    if (decided)
+        for (int t = 0; t < cu_tokens[n_seqs]; t++)
+            if (decided[(size_t)t * p->n_groups + group] > ACT_H) return ORC_ERR_ARG;
     /* pass 1: how many new pages does the whole call need? */
     uint64_t need_high = 0, need_low = 0;
     for (int i = 0; i < n_seqs; i++) {
@@ -299,7 +334,7 @@ int orc_append(orc_cache *c, int layer, int n_seqs, const int32_t *seq_ids, cons
         orc_stream *s = stream_of(c, seq, layer);
         uint32_t nh = s->n_high, nl = s->n_low;
         for (int t = cu_tokens[i]; t < cu_tokens[i + 1]; t++) {
-            int bad, a = decide(p, group, tags[t], &bad);
+            int bad, a = action_of(p, group, tags, decided, t, &bad);
             if (a == ACT_H) { if (nh % PAGE_TOKENS == 0) need_high++; nh++; }
             else if (a == ACT_L) { if (nl % PAGE_TOKENS == 0) need_low++; nl++; }
         }
@@ -312,7 +347,7 @@ int orc_append(orc_cache *c, int layer, int n_seqs, const int32_t *seq_ids, cons
         orc_stream *s = stream_of(c, seq, layer);
         orc_budget *b = &c->budget[seq];
         for (int t = cu_tokens[i]; t < cu_tokens[i + 1]; t++) {
-            int bad, a = decide(p, group, tags[t], &bad);
+            int bad, a = action_of(p, group, tags, decided, t, &bad);
             if (actions_out) actions_out[t] = (uint8_t)a;
             b->bad_tags += (uint64_t)bad;
             b->n_seen[group]++;
@@ -363,6 +398,126 @@ int orc_append(orc_cache *c, int layer, int n_seqs, const int32_t *seq_ids, cons
         /* floor(B * full) - retained with B in Q16; full_bytes < 2^47 here so the product fits */
         b->remaining_bytes = (int64_t)(((uint64_t)p->budget_q16 * b->full_bytes) >> 16) - (int64_t)b->retained_bytes;
     }
+    return ORC_OK;
+}
+
+int orc_append(orc_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,
+               const uint16_t *k_bits, const uint16_t *v_bits, const uint8_t *tags, uint8_t *actions_out) {
+    return orc_append_decided(c, layer, n_seqs, seq_ids, cu_tokens, k_bits, v_bits, tags, NULL, actions_out);
+}
+
+/* ------------------------------------------------------------------ dynamic budget adjustment */
+
+/* m(a, c): what action a costs for one token over all the layers of group c (Section 3.1's
+ * m(R) = 0 < m(L) < m(H), summed over the group's layers). */
+static uint64_t group_cost(const orc_cache *c, int a, uint32_t layers_in_group) {
+    if (a == ACT_H) return layers_in_group * bytes_high(c);
+    if (a == ACT_L) return layers_in_group * bytes_low(c);
+    return 0;
+}
+
+/* The adjacent upgrade score of bucket (tag, group) for the step (a-1 -> a). */
+static float rho_of(const orc_policy *p, int tag, int group, int a) {
+    size_t i = (size_t)tag * p->n_groups + group;
+    return a == ACT_H ? p->rho_lh[i] : p->rho_rl[i];
+}
+
+/* Algorithm 2 for one token, all layer groups at once (steps 1-6 and 8; step 7, Persist, is
+ * orc_append_decided, layer by layer).  a_out [n_groups].
+ *   R_t   = floor(target * (full cost of every token seen so far, this one included))
+ *           - (cost of everything decided so far)          -- the remaining target budget
+ *   B_t   = max(0, R_t - Gamma(s_t))                                           (Eq. 10)
+ *   Demote: while the token's cost exceeds B_t and some group sits above its floor, lower by
+ *           one step the group whose step (a-1 -> a) has the smallest upgrade score: that is
+ *           the smallest distortion loss per saved cost (first such group on ties).  Floors are
+ *           never crossed, even if the cost still exceeds B_t.
+ *   Promote (critical states only): while some group below H can take one step up and the
+ *           token's cost stays within B_t, raise the one with the largest upgrade score (first
+ *           such group on ties).
+ * Groups that own no layer cost nothing and are left alone.  Protected and unknown tags are
+ * high precision with a high-precision floor.  A state id outside the reserve table has
+ * Gamma = 0 and is not critical. */
+static void decide_token(const orc_cache *c, orc_budget *b, const uint32_t *layers_in_group, uint8_t tag,
+                         int has_state, uint32_t state, uint8_t *a_out) {
+    const orc_policy *p = c->pol;
+    const int G = (int)p->n_groups;
+    int a[MAX_GROUPS], fl[MAX_GROUPS];
+    const int table_tag = tag != TAG_PROTECTED && tag < p->n_tags;
+    uint64_t token_full = 0;
+    for (int g = 0; g < G; g++) {                                      /* steps 1-2 */
+        if (table_tag) {
+            fl[g] = p->a_floor[(size_t)tag * G + g];
+            a[g] = orc_lut_fold(p->a0[(size_t)tag * G + g], fl[g]);
+        } else {
+            fl[g] = a[g] = ACT_H;
+        }
+        token_full += group_cost(c, ACT_H, layers_in_group[g]);
+    }
+    uint64_t gamma = 0;
+    int crit = 0;
+    if (has_state && state < p->n_states) {
+        gamma = (uint64_t)p->gamma[state] << p->gamma_shift;
+        crit = p->crit[state];
+    }
+    const uint64_t full_now = b->decided_full_bytes + token_full;
+    const int64_t R = (int64_t)(((uint64_t)p->budget_q16 * full_now) >> 16) - (int64_t)b->decided_retained_bytes;
+    const int64_t B = R - (int64_t)gamma > 0 ? R - (int64_t)gamma : 0;   /* step 3 */
+
+    uint64_t cost = 0;
+    for (int g = 0; g < G; g++) cost += group_cost(c, a[g], layers_in_group[g]);
+
+    while ((int64_t)cost > B) {                                        /* step 4: Demote */
+        int pick = -1;
+        for (int g = 0; g < G; g++) {
+            if (a[g] <= fl[g] || layers_in_group[g] == 0) continue;
+            if (pick < 0 || rho_of(p, tag, g, a[g]) < rho_of(p, tag, pick, a[pick])) pick = g;
+        }
+        if (pick < 0) break;                                           /* only floors left */
+        cost -= group_cost(c, a[pick], layers_in_group[pick]) - group_cost(c, a[pick] - 1, layers_in_group[pick]);
+        a[pick]--;
+        b->n_demoted++;
+    }
+    if ((int64_t)cost > B) b->n_floor_conflicts++;
+
+    if (crit) {                                                        /* steps 5-6: Promote */
+        for (;;) {
+            int pick = -1;
+            for (int g = 0; g < G; g++) {
+                if (a[g] >= ACT_H || layers_in_group[g] == 0) continue;
+                uint64_t up = group_cost(c, a[g] + 1, layers_in_group[g]) - group_cost(c, a[g], layers_in_group[g]);
+                if ((int64_t)(cost + up) > B) continue;                /* not eligible: does not fit */
+                if (pick < 0 || rho_of(p, tag, g, a[g] + 1) > rho_of(p, tag, pick, a[pick] + 1)) pick = g;
+            }
+            if (pick < 0) break;
+            cost += group_cost(c, a[pick] + 1, layers_in_group[pick]) - group_cost(c, a[pick], layers_in_group[pick]);
+            a[pick]++;
+            b->n_promoted++;
+        }
+    }
+    b->decided_full_bytes = full_now;                                  /* step 8 */
+    b->decided_retained_bytes += cost;
+    for (int g = 0; g < G; g++) a_out[g] = (uint8_t)a[g];
+}
+
+/* Algorithm 2 steps 1-6 and 8 for a ragged batch: each sequence's tokens in order, one budget
+ * state per sequence.  states may be NULL (no reserve, nothing critical).
+ * actions_out [total_tokens][n_groups].  A bad sequence id or a sequence named twice refuses the
+ * whole call and changes nothing. */
+int orc_decide(orc_cache *c, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens, const uint8_t *tags,
+               const uint16_t *states, uint8_t *actions_out) {
+    const orc_policy *p = c->pol;
+    if (n_seqs < 0) return ORC_ERR_ARG;
+    for (int i = 0; i < n_seqs; i++) {
+        if (seq_ids[i] < 0 || seq_ids[i] >= c->max_seqs) return ORC_ERR_SEQ;
+        for (int j = 0; j < i; j++) if (seq_ids[j] == seq_ids[i]) return ORC_ERR_SEQ;
+        if (cu_tokens[i + 1] < cu_tokens[i]) return ORC_ERR_ARG;
+    }
+    uint32_t layers_in_group[MAX_GROUPS] = {0};
+    for (uint32_t l = 0; l < p->n_layers; l++) layers_in_group[p->layer_group[l]]++;
+    for (int i = 0; i < n_seqs; i++)
+        for (int t = cu_tokens[i]; t < cu_tokens[i + 1]; t++)
+            decide_token(c, &c->budget[seq_ids[i]], layers_in_group, tags[t], states != NULL,
+                         states ? states[t] : 0u, actions_out + (size_t)t * p->n_groups);
     return ORC_OK;
 }
 

@@ -14,6 +14,9 @@ Little-endian layout written by `write_blob`:
     40 u8  layer_group[n_layers], zero padded to a multiple of 4 bytes
     then n_tags*n_groups entries, tag-major: u8 a0, u8 a_floor, u16 0, f32 rho_RL, f32 rho_LH
     then u32 gamma[n_states]
+Version 2 (written when the policy carries critical-state flags) appends
+    u32 gamma_shift (0..16: the reserve of state s is gamma[s] << gamma_shift bytes)
+    u8  crit[n_states] (0 or 1), zero padded to a multiple of 4 bytes
 Actions: 0 = release (drop), 1 = retain-low, 2 = retain-high.
 """
 from __future__ import annotations
@@ -44,6 +47,8 @@ class Policy:
     recent_window: int = 0
     low_bits: int = 4
     group_size: int = 32
+    crit: np.ndarray | None = None     # u8 [n_states] critical-state flags (None: version-1 blob)
+    gamma_shift: int = 0
 
     @property
     def n_layers(self) -> int:
@@ -54,7 +59,8 @@ def write_blob(p: Policy) -> bytes:
     q16 = int(round(p.budget_target * 65536.0))
     out = bytearray()
     out += b"PASK"
-    out += struct.pack("<9I", 1, p.n_tags, p.n_groups, p.n_layers, int(p.gamma.shape[0]), q16,
+    version = 1 if p.crit is None else 2
+    out += struct.pack("<9I", version, p.n_tags, p.n_groups, p.n_layers, int(p.gamma.shape[0]), q16,
                        p.recent_window, p.low_bits, p.group_size)
     lg = bytes(np.asarray(p.layer_group, dtype=np.uint8).tolist())
     out += lg + b"\0" * ((-len(lg)) % 4)
@@ -63,6 +69,11 @@ def write_blob(p: Policy) -> bytes:
             out += struct.pack("<BBHff", int(p.a0[z, c]), int(p.a_floor[z, c]), 0,
                                float(p.rho_rl[z, c]), float(p.rho_lh[z, c]))
     out += np.asarray(p.gamma, dtype="<u4").tobytes()
+    if version == 2:
+        assert p.crit.shape[0] == p.gamma.shape[0]
+        out += struct.pack("<I", p.gamma_shift)
+        cr = bytes(np.asarray(p.crit, dtype=np.uint8).tolist())
+        out += cr + b"\0" * ((-len(cr)) % 4)
     return bytes(out)
 
 
