@@ -62,6 +62,7 @@ typedef int32_t pask_status_t;
                                          computes in; results for that sequence may be infinite or NaN */
 
 #define PASK_DEV_INTERNAL 0x40u       /* an internal bounds check refused an access (a page id out of range) */
+#define PASK_DEV_BAD_ACTION 0x80u     /* pask_append_kv_decided was given an action outside R, L, H; call refused */
 
 #define PASK_ACTION_RELEASE 0
 #define PASK_ACTION_RETAIN_LOW 1
@@ -111,6 +112,15 @@ typedef struct {
     uint32_t pages_low;
     uint32_t device_status;   /* PASK_DEV_* bits, cache-wide, sticky until pask_cache_reset */
     uint32_t reserved;
+    /* Algorithm 2's own running budget, advanced by pask_decide once per token for all groups:
+     * R_t = floor(budget_target * decided_full_bytes, this token included) - decided_retained_bytes.
+     * Once every layer of the decided tokens has been appended with pask_append_kv_decided these
+     * two equal full_bytes and retained_bytes. */
+    uint64_t decided_full_bytes;
+    uint64_t decided_retained_bytes;
+    uint64_t n_demoted;         /* single steps H->L or L->R taken by Demote */
+    uint64_t n_promoted;        /* single steps R->L or L->H taken by Promote */
+    uint64_t n_floor_conflicts; /* tokens whose floors alone exceeded B_t (floors were kept) */
 } pask_budget_state_t;
 
 /* ---------------------------------------------------------------------------------------------
@@ -118,13 +128,19 @@ typedef struct {
  * Follows: the table stores, per bucket q = (tag, layer group), the selected action, the
  * calibrated floor and the adjacent upgrade scores (end of Section 3.3); online the action is
  * a = max(a0, a_floor) under R < L < H (Eq. 10, Algorithm 2 steps 1-2).  Gamma is Eq. 9's
- * per-state reserve, carried but not read by the calls below.
+ * per-state reserve; the upgrade scores, Gamma and the critical-state flags are read by
+ * pask_decide only.
  *   blob (host, len bytes), little endian:
- *     "PASK", u32 version=1, u32 n_tags (1..255), u32 n_groups (1..8), u32 n_layers, u32 n_states,
- *     u32 budget_target_q16, u32 recent_window (must be 0), u32 low_bits (4), u32 group_size (32),
+ *     "PASK", u32 version (1 or 2), u32 n_tags (1..255), u32 n_groups (1..8), u32 n_layers,
+ *     u32 n_states, u32 budget_target_q16, u32 recent_window (must be 0), u32 low_bits (4),
+ *     u32 group_size (32),
  *     u8 layer_group[n_layers] zero-padded to 4 bytes,
- *     n_tags*n_groups entries, tag-major: u8 a0, u8 a_floor, u16 0, f32 rho_RL, f32 rho_LH,
- *     u32 gamma[n_states].
+ *     n_tags*n_groups entries, tag-major: u8 a0, u8 a_floor, u16 0, f32 rho_RL, f32 rho_LH
+ *       (scores of the adjacent upgrades R->L and L->H; any value but NaN),
+ *     u32 gamma[n_states],
+ *     version 2 only: u32 gamma_shift (0..16; the reserve of state s is gamma[s] << gamma_shift
+ *       bytes), u8 crit[n_states] (1 = critical or lookahead-critical) zero-padded to 4 bytes.
+ *       Version 1 means gamma_shift = 0 and no critical state.
  * The blob is copied; *out is a host handle to free with pask_free_policy.  Needs no GPU.
  * Errors: PASK_ERR_INVALID_ARG (null), PASK_ERR_BAD_POLICY (magic, version, sizes, ranges, length).
  */
@@ -165,7 +181,8 @@ pask_status_t pask_seq_reset(pask_cache_t *cache, int32_t seq, pask_stream_t str
  *   k, v           dev bf16 [total_tokens][n_kv][128], post-RoPE, tokens of a sequence in order
  *   tags           dev uint8 [total_tokens]; PASK_TAG_PROTECTED = always high; >= n_tags = high
  *                  and counted in bad_tags
- *   states         dev uint16 [total_tokens] parser-state ids or NULL (reserved; not read)
+ *   states         dev uint16 [total_tokens] or NULL; not read: this call applies the frozen table
+ *                  as it stands, the budget-dependent adjustment is pask_decide
  *   actions_out    dev uint8 [total_tokens] or NULL: the action taken for each token
  * New pages are numbered in call order (sequence-major, position ascending) from each pool's
  * free stack, else its bump counter.  If either pool cannot supply the whole call, or a stream
@@ -176,6 +193,42 @@ pask_status_t pask_append_kv(pask_cache_t *cache, int32_t layer, int32_t n_seqs,
                              const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
                              const uint8_t *tags, const uint16_t *states, uint8_t *actions_out,
                              pask_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * pask_decide -- Algorithm 2 steps 1-6 and 8 for a ragged batch of tokens, all layer groups at
+ * once: the budget-dependent adjustment of the table's actions (Eq. 10 and the paragraph after
+ * it).  For each token, in sequence order, with the sequence's own running budget:
+ *   a_c  = max(a0, a_floor) per group c (protected and unknown tags: H with floor H);
+ *   R_t  = floor(budget_target * decided_full_bytes, this token's full cost included)
+ *          - decided_retained_bytes;         B_t = max(0, R_t - Gamma(s_t));
+ *   cost = sum over groups of (layers in the group) * m(a_c);
+ *   Demote: while cost > B_t and some group is above its floor, lower by one step (H->L or L->R)
+ *     the group whose step has the smallest upgrade score rho (the least distortion lost per
+ *     byte saved; the first such group on ties).  Floors are never crossed: if they alone exceed
+ *     B_t they stay and n_floor_conflicts counts the token;
+ *   Promote, only if crit[s_t]: while some group below H can go up one step with cost still
+ *     <= B_t, raise the one with the largest rho (first group on ties);
+ *   decided_full_bytes += the token's full cost; decided_retained_bytes += cost.
+ * Groups that own no layer are left alone.  A state id >= n_states (or states == NULL) has no
+ * reserve and is not critical.
+ *   seq_ids, cu_tokens, tags, states (may be NULL)   as for pask_append_kv, device memory
+ *   actions_out    dev uint8 [total_tokens][n_groups]: feed it to pask_append_kv_decided for
+ *                  every layer (in any order) before the next pask_decide of these sequences
+ * The call takes no query and no statistics of K or V: constant work and constant state per token
+ * (Section 3.4).  A bad sequence id, a sequence named twice or a malformed cu_tokens refuses the
+ * whole call (sticky PASK_DEV_* bit): no budget state changes and actions_out is undefined.
+ */
+pask_status_t pask_decide(pask_cache_t *cache, int32_t n_seqs, int32_t total_tokens, const int32_t *seq_ids,
+                          const int32_t *cu_tokens, const uint8_t *tags, const uint16_t *states,
+                          uint8_t *actions_out, pask_stream_t stream);
+/* pask_append_kv with Algorithm 2 step 7 applied to decided actions: token t takes
+ * actions[t * n_groups + group of `layer`] instead of the table's entry (tags still count
+ * bad_tags).  An action > 2 refuses the call with PASK_DEV_BAD_ACTION.  Everything else --
+ * arguments, page numbering, all-or-nothing refusal, accounting -- is pask_append_kv's. */
+pask_status_t pask_append_kv_decided(pask_cache_t *cache, int32_t layer, int32_t n_seqs, int32_t total_tokens,
+                                     const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
+                                     const uint8_t *tags, const uint8_t *actions, uint8_t *actions_out,
+                                     pask_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------------
  * pask_decode_attention -- attention of one new query per sequence over that sequence's

@@ -19,13 +19,15 @@ OK = 0
 ERR_INVALID_ARG, ERR_BAD_POLICY, ERR_UNSUPPORTED_SHAPE, ERR_POOL_EXHAUSTED = -1, -2, -3, -4
 ERR_BAD_SEQ, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE = -5, -6, -7, -8
 DEV_POOL_EXHAUSTED, DEV_BAD_SEQ, DEV_SEQ_OVERFLOW, DEV_BAD_RAGGED, DEV_TIMEOUT, DEV_RANGE, DEV_INTERNAL = 1, 2, 4, 8, 16, 32, 64
+DEV_BAD_ACTION = 128
 ACTION_RELEASE, ACTION_RETAIN_LOW, ACTION_RETAIN_HIGH = 0, 1, 2
 TAG_PROTECTED = 0xFF
 MAX_GROUPS = 8
 
 EXPORTS = [
     "pask_load_policy", "pask_free_policy", "pask_policy_action", "pask_cache_sizes", "pask_cache_create",
-    "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decode_attention",
+    "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decide",
+    "pask_append_kv_decided", "pask_decode_attention",
     "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes",
     "pask_budget_state", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
     "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
@@ -49,7 +51,9 @@ class BudgetState(C.Structure):
                 ("n_low", C.c_uint64 * MAX_GROUPS), ("n_drop", C.c_uint64 * MAX_GROUPS),
                 ("retained_bytes", C.c_uint64), ("full_bytes", C.c_uint64), ("remaining_bytes", C.c_int64),
                 ("bad_tags", C.c_uint64), ("pages_high", C.c_uint32), ("pages_low", C.c_uint32),
-                ("device_status", C.c_uint32), ("reserved", C.c_uint32)]
+                ("device_status", C.c_uint32), ("reserved", C.c_uint32),
+                ("decided_full_bytes", C.c_uint64), ("decided_retained_bytes", C.c_uint64),
+                ("n_demoted", C.c_uint64), ("n_promoted", C.c_uint64), ("n_floor_conflicts", C.c_uint64)]
 
 
 if not os.path.exists(LIB_PATH):
@@ -69,6 +73,8 @@ _lib.pask_cache_destroy.restype = None
 _lib.pask_cache_reset.argtypes = [_vp, _vp]
 _lib.pask_seq_reset.argtypes = [_vp, _i32, _vp]
 _lib.pask_append_kv.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.pask_decide.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.pask_append_kv_decided.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_decode_attention.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.pask_decode_attention_full.argtypes = _lib.pask_decode_attention.argtypes
 _lib.pask_decode_attention_static.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
@@ -168,6 +174,25 @@ def pask_append_kv(cache: int, layer: int, seq_ids, cu_tokens, k, v, tags, state
     _check(_lib.pask_append_kv(cache, layer, n_seqs, total, _dptr(seq_ids, torch.int32), _dptr(cu_tokens, torch.int32),
                                _dptr(k, torch.bfloat16), _dptr(v, torch.bfloat16), _dptr(tags, torch.uint8),
                                _dptr(states), _dptr(actions_out, torch.uint8), _stream(stream)), "pask_append_kv")
+
+
+def pask_decide(cache: int, seq_ids, cu_tokens, tags, states, actions_out, stream=None):
+    """Algorithm 2 steps 1-6 and 8: tags u8 [total], states u16/i16 [total] or None,
+    actions_out u8 [total][n_groups]."""
+    _check(_lib.pask_decide(cache, seq_ids.numel(), tags.numel(), _dptr(seq_ids, torch.int32),
+                            _dptr(cu_tokens, torch.int32), _dptr(tags, torch.uint8), _dptr(states),
+                            _dptr(actions_out, torch.uint8), _stream(stream)), "pask_decide")
+
+
+def pask_append_kv_decided(cache: int, layer: int, seq_ids, cu_tokens, k, v, tags, actions, actions_out=None,
+                           stream=None, total_tokens=None):
+    n_seqs = seq_ids.numel()
+    total = k.shape[0] if total_tokens is None else total_tokens
+    _check(_lib.pask_append_kv_decided(cache, layer, n_seqs, total, _dptr(seq_ids, torch.int32),
+                                       _dptr(cu_tokens, torch.int32), _dptr(k, torch.bfloat16),
+                                       _dptr(v, torch.bfloat16), _dptr(tags, torch.uint8),
+                                       _dptr(actions, torch.uint8), _dptr(actions_out, torch.uint8),
+                                       _stream(stream)), "pask_append_kv_decided")
 
 
 def pask_workspace_bytes(cache: int, n_seqs: int) -> int:

@@ -43,6 +43,10 @@ MetaOffsets meta_offsets(const pask_cache_desc_t *d, int n_tags, int n_groups) {
     o.tok_scratch = take((size_t)d->max_append_tokens * sizeof(uint2));
     o.lut = take((size_t)n_tags * n_groups);
     o.layer_group = take((size_t)d->n_layers);
+    o.dec_row = take(256 * sizeof(uint2));
+    o.dec_rho = take((size_t)n_tags * n_groups * sizeof(float2));
+    o.gamma = take((size_t)kMaxStatesDev * 4);
+    o.crit = take((size_t)kMaxStatesDev);
     o.total = p;
     return o;
 }
@@ -90,7 +94,9 @@ pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **o
     if (!blob_v || !out) return PASK_ERR_INVALID_ARG;
     *out = nullptr;
     const uint8_t *blob = static_cast<const uint8_t *>(blob_v);
-    if (len < 40 || std::memcmp(blob, "PASK", 4) != 0 || rd32(blob + 4) != 1) return PASK_ERR_BAD_POLICY;
+    if (len < 40 || std::memcmp(blob, "PASK", 4) != 0) return PASK_ERR_BAD_POLICY;
+    const uint32_t version = rd32(blob + 4);
+    if (version != 1 && version != 2) return PASK_ERR_BAD_POLICY;
     pask_policy *p = new (std::nothrow) pask_policy();
     if (!p) return PASK_ERR_INVALID_ARG;
     p->n_tags = rd32(blob + 8);
@@ -104,7 +110,9 @@ pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **o
               group_size == (uint32_t)kQGroup;
     const size_t lg_pad = ok ? align_up(p->n_layers, 4) : 0;
     const size_t n_ent = ok ? (size_t)p->n_tags * p->n_groups : 0;
-    ok = ok && len == 40 + lg_pad + n_ent * 12 + (size_t)p->n_states * 4;
+    const size_t tail = ok && version == 2 ? 4 + align_up(p->n_states, 4) : 0;
+    ok = ok && len == 40 + lg_pad + n_ent * 12 + (size_t)p->n_states * 4 + tail;
+    p->gamma_shift = 0;
     if (ok) {
         p->layer_group.assign(blob + 40, blob + 40 + p->n_layers);
         for (uint8_t g : p->layer_group) ok = ok && g < p->n_groups;
@@ -117,10 +125,18 @@ pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **o
             ok = ok && e[0] <= PASK_ACTION_RETAIN_HIGH && e[1] <= PASK_ACTION_RETAIN_HIGH && e[2] == 0 && e[3] == 0;
             std::memcpy(&p->rho_rl[i], e + 4, 4);
             std::memcpy(&p->rho_lh[i], e + 8, 4);
+            ok = ok && p->rho_rl[i] == p->rho_rl[i] && p->rho_lh[i] == p->rho_lh[i];   // scores are compared: no NaN
             p->eff[i] = e[0] > e[1] ? e[0] : e[1];  // floors take priority: a = max(a0, a_floor)
         }
         p->gamma.resize(p->n_states);
         for (uint32_t s = 0; s < p->n_states; s++, e += 4) p->gamma[s] = rd32(e);
+        p->crit.assign(p->n_states, 0);
+        if (version == 2) {
+            p->gamma_shift = rd32(e);
+            e += 4;
+            ok = ok && p->gamma_shift <= 16;
+            for (uint32_t s = 0; s < p->n_states; s++) { p->crit[s] = e[s]; ok = ok && e[s] <= 1; }
+        }
     }
     if (!ok) { delete p; return PASK_ERR_BAD_POLICY; }
     *out = p;
@@ -184,6 +200,14 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     v.tok_scratch = reinterpret_cast<uint2 *>(m + c->off.tok_scratch);
     v.lut = m + c->off.lut;
     v.layer_group = m + c->off.layer_group;
+    v.dec_row = reinterpret_cast<uint2 *>(m + c->off.dec_row);
+    v.dec_rho = reinterpret_cast<float2 *>(m + c->off.dec_rho);
+    v.gamma = reinterpret_cast<uint32_t *>(m + c->off.gamma);
+    v.crit = m + c->off.crit;
+    v.n_states_dev = pol->n_states < kMaxStatesDev ? pol->n_states : kMaxStatesDev;
+    v.gamma_shift = pol->gamma_shift;
+    for (int g = 0; g < PASK_MAX_GROUPS; g++) v.group_layers[g] = 0;
+    for (uint8_t g : pol->layer_group) v.group_layers[g]++;
     v.n_layers = d->n_layers;
     v.n_q = d->n_q_heads;
     v.n_kv = d->n_kv_heads;
@@ -202,11 +226,36 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     c->attn_ctas = attention_grid(c);
     c->lut = pol->eff;
     c->layer_group = pol->layer_group;
+    // per tag byte: the table's actions and floors packed two bits per group, and what the actions cost
+    std::vector<uint2> dec_row(256);
+    std::vector<float2> dec_rho((size_t)pol->n_tags * pol->n_groups);
+    for (uint32_t z = 0; z < 256; z++) {
+        uint32_t acts = 0, floors = 0, cost = 0;
+        for (uint32_t g = 0; g < pol->n_groups; g++) {
+            uint32_t a = PASK_ACTION_RETAIN_HIGH, f = PASK_ACTION_RETAIN_HIGH;   // protected and unknown tags
+            if (z < pol->n_tags) {
+                a = pol->eff[(size_t)z * pol->n_groups + g];
+                f = pol->a_floor[(size_t)z * pol->n_groups + g];
+                dec_rho[(size_t)z * pol->n_groups + g] = make_float2(pol->rho_rl[(size_t)z * pol->n_groups + g],
+                                                                     pol->rho_lh[(size_t)z * pol->n_groups + g]);
+            }
+            acts |= a << (2 * g);
+            floors |= f << (2 * g);
+            cost += v.group_layers[g] * (a == PASK_ACTION_RETAIN_HIGH ? v.bytes_h : a == PASK_ACTION_RETAIN_LOW ? v.bytes_l : 0u);
+        }
+        dec_row[z] = make_uint2(acts | (floors << 16), cost);
+    }
     // pageable host sources: the runtime stages these copies, so the vectors may die afterwards
     cudaError_t e = cudaMemcpyAsync(v.lut, pol->eff.data(), pol->eff.size(), cudaMemcpyHostToDevice, stream);
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(v.layer_group, pol->layer_group.data(), pol->layer_group.size(), cudaMemcpyHostToDevice,
                             stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(v.dec_row, dec_row.data(), dec_row.size() * sizeof(uint2), cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(v.dec_rho, dec_rho.data(), dec_rho.size() * sizeof(float2), cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess && v.n_states_dev)
+        e = cudaMemcpyAsync(v.gamma, pol->gamma.data(), (size_t)v.n_states_dev * 4, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess && v.n_states_dev)
+        e = cudaMemcpyAsync(v.crit, pol->crit.data(), (size_t)v.n_states_dev, cudaMemcpyHostToDevice, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) { delete c; return PASK_ERR_CUDA; }
     pask_status_t rc = pask_cache_reset(c, stream_v);
@@ -233,10 +282,10 @@ pask_status_t pask_seq_reset(pask_cache_t *c, int32_t seq, pask_stream_t stream)
     return launch_seq_reset(c, seq, static_cast<cudaStream_t>(stream));
 }
 
-pask_status_t pask_append_kv(pask_cache_t *c, int32_t layer, int32_t n_seqs, int32_t total_tokens,
-                             const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
-                             const uint8_t *tags, const uint16_t *states, uint8_t *actions_out, pask_stream_t stream) {
-    (void)states;  // reserved for the dynamic budget adjustment (Algorithm 2 steps 3-6)
+static pask_status_t append_common(pask_cache_t *c, int32_t layer, int32_t n_seqs, int32_t total_tokens,
+                                   const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
+                                   const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out,
+                                   pask_stream_t stream) {
     if (!c || !seq_ids || !cu_tokens || !tags) return PASK_ERR_INVALID_ARG;
     if (layer < 0 || layer >= c->desc.n_layers) return PASK_ERR_INVALID_ARG;
     if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL || n_seqs > c->desc.max_seqs) return PASK_ERR_INVALID_ARG;
@@ -244,7 +293,33 @@ pask_status_t pask_append_kv(pask_cache_t *c, int32_t layer, int32_t n_seqs, int
     if (total_tokens > 0 && (!k || !v)) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)k | (uintptr_t)v) & 15) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)seq_ids | (uintptr_t)cu_tokens) & 3) return PASK_ERR_INVALID_ARG;
-    return launch_append(c, layer, n_seqs, total_tokens, seq_ids, cu_tokens, k, v, tags, actions_out,
+    return launch_append(c, layer, n_seqs, total_tokens, seq_ids, cu_tokens, k, v, tags, decided, actions_out,
+                         static_cast<cudaStream_t>(stream));
+}
+
+pask_status_t pask_append_kv(pask_cache_t *c, int32_t layer, int32_t n_seqs, int32_t total_tokens,
+                             const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
+                             const uint8_t *tags, const uint16_t *states, uint8_t *actions_out, pask_stream_t stream) {
+    (void)states;  // the frozen table as it stands; the budget-dependent adjustment is pask_decide
+    return append_common(c, layer, n_seqs, total_tokens, seq_ids, cu_tokens, k, v, tags, nullptr, actions_out, stream);
+}
+
+pask_status_t pask_append_kv_decided(pask_cache_t *c, int32_t layer, int32_t n_seqs, int32_t total_tokens,
+                                     const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
+                                     const uint8_t *tags, const uint8_t *actions, uint8_t *actions_out,
+                                     pask_stream_t stream) {
+    if (!actions) return PASK_ERR_INVALID_ARG;
+    return append_common(c, layer, n_seqs, total_tokens, seq_ids, cu_tokens, k, v, tags, actions, actions_out, stream);
+}
+
+pask_status_t pask_decide(pask_cache_t *c, int32_t n_seqs, int32_t total_tokens, const int32_t *seq_ids,
+                          const int32_t *cu_tokens, const uint8_t *tags, const uint16_t *states, uint8_t *actions_out,
+                          pask_stream_t stream) {
+    if (!c || !seq_ids || !cu_tokens || !tags || !actions_out) return PASK_ERR_INVALID_ARG;
+    if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL || n_seqs > c->desc.max_seqs) return PASK_ERR_INVALID_ARG;
+    if (total_tokens < 0) return PASK_ERR_INVALID_ARG;
+    if (((uintptr_t)seq_ids | (uintptr_t)cu_tokens) & 3 || ((uintptr_t)states & 1)) return PASK_ERR_INVALID_ARG;
+    return launch_decide(c, n_seqs, total_tokens, seq_ids, cu_tokens, tags, states, actions_out,
                          static_cast<cudaStream_t>(stream));
 }
 

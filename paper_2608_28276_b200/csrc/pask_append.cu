@@ -62,7 +62,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *s_warp
 __global__ void __launch_bounds__(kPlanThreads)
 append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const int32_t *__restrict__ seq_ids,
                    const int32_t *__restrict__ cu_tokens, const uint8_t *__restrict__ tags,
-                   uint8_t *__restrict__ actions_out, uint32_t serial) {
+                   const uint8_t *__restrict__ decided, uint8_t *__restrict__ actions_out, uint32_t serial) {
     __shared__ uint8_t s_lut[256];
     __shared__ uint32_t s_wh[kPlanThreads / 32], s_wl[kPlanThreads / 32], s_wb[kPlanThreads / 32];
     __shared__ uint32_t s_scan[kPlanThreads / 32];
@@ -85,6 +85,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
     __syncthreads();
     if (s_flag) err |= PASK_DEV_BAD_SEQ;
 
+    int bad_action = 0;
     if (!err) {
         for (int base = t0; base < t1; base += kPlanThreads) {
             const int t = base + tid;
@@ -95,6 +96,10 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
                 const int tag = tags[t];
                 a = s_lut[tag];
                 bad = tag != PASK_TAG_PROTECTED && tag >= c.n_tags;
+                if (decided) {   // Algorithm 2 step 7 on the actions pask_decide chose
+                    a = decided[(size_t)t * c.n_groups + group];
+                    if (a > PASK_ACTION_RETAIN_HIGH) { bad_action = 1; a = PASK_ACTION_RELEASE; }
+                }
             }
             const uint32_t mh = __ballot_sync(0xffffffffu, a == PASK_ACTION_RETAIN_HIGH);
             const uint32_t ml = __ballot_sync(0xffffffffu, a == PASK_ACTION_RETAIN_LOW);
@@ -120,6 +125,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         }
     }
 
+    if (__syncthreads_or(bad_action)) err |= PASK_DEV_BAD_ACTION;
     if (tid == 0) {
         AppendPlan p{};
         p.seq = err ? -1 : seq;
@@ -333,7 +339,8 @@ struct SmallLut { uint8_t action[256]; };
 __global__ void __launch_bounds__(kSmallThreads)
 append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, const int32_t *__restrict__ seq_ids,
                     const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
-                    const uint8_t *__restrict__ tags, uint8_t *__restrict__ actions_out, const SmallLut lut) {
+                    const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided,
+                    uint8_t *__restrict__ actions_out, const SmallLut lut) {
     __shared__ int s_seq[kSmallMax], s_cu[kSmallMax + 1];
     __shared__ uint32_t s_old_h[kSmallMax], s_old_l[kSmallMax], s_cnt_h[kSmallMax], s_cnt_l[kSmallMax], s_cnt_bad[kSmallMax];
     __shared__ uint32_t s_new_h[kSmallMax], s_new_l[kSmallMax], s_base_h[kSmallMax], s_base_l[kSmallMax];
@@ -365,8 +372,11 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         s_old_h[tid] = oh;
         s_old_l[tid] = ol;
     }
-    int my_tag = 0;
-    if (tid < total) my_tag = tags[tid];
+    int my_tag = 0, my_decided = 0;
+    if (tid < total) {
+        my_tag = tags[tid];
+        if (decided) my_decided = decided[(size_t)tid * c.n_groups + group];
+    }
     __syncthreads();
 
     // ---- validate the call; decide every token
@@ -390,7 +400,11 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     if (tid < total) {
         int i = 0;                                   // the sequence this token belongs to
         while (s_cu[i + 1] <= tid) i++;
-        const int a = lut.action[my_tag];
+        int a = lut.action[my_tag];
+        if (decided) {   // Algorithm 2 step 7 on the actions pask_decide chose
+            a = my_decided;
+            if (a > PASK_ACTION_RETAIN_HIGH) { atomicOr(&s_err, PASK_DEV_BAD_ACTION); a = PASK_ACTION_RELEASE; }
+        }
         s_tok_seq[tid] = (uint8_t)i;
         s_act[tid] = (uint8_t)a;
         s_tok_bad[tid] = my_tag != PASK_TAG_PROTECTED && my_tag >= c.n_tags;
@@ -532,7 +546,7 @@ __global__ void __launch_bounds__(256) seq_reset_kernel(DevCache c, int seq) {
 
 pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_tokens, const int32_t *seq_ids,
                             const int32_t *cu_tokens, const void *k, const void *v, const uint8_t *tags,
-                            uint8_t *actions_out, cudaStream_t stream) {
+                            const uint8_t *decided, uint8_t *actions_out, cudaStream_t stream) {
     if (n_seqs <= kSmallMax && total_tokens <= kSmallMax) {
         SmallLut lut;
         const int group = c->layer_group[layer];
@@ -541,12 +555,12 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
         if (total_tokens == 0) return PASK_OK;
         const cudaError_t e = launch_pdl(append_small_kernel, dim3(total_tokens), dim3(kSmallThreads), 0, stream, c->dev, layer,
                                          group, n_seqs, total_tokens, seq_ids, cu_tokens, static_cast<const uint4 *>(k),
-                                         static_cast<const uint4 *>(v), tags, actions_out, lut);
+                                         static_cast<const uint4 *>(v), tags, decided, actions_out, lut);
         return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
     }
     if (++c->append_serial == 0) c->append_serial = 1;
     append_plan_kernel<<<n_seqs, kPlanThreads, 0, stream>>>(c->dev, layer, n_seqs, total_tokens, seq_ids, cu_tokens, tags,
-                                                           actions_out, c->append_serial);
+                                                           decided, actions_out, c->append_serial);
     if (total_tokens > 0) {
         const int ctas = total_tokens < c->sm_count * 8 ? total_tokens : c->sm_count * 8;
         append_write_kernel<<<ctas, 32 * c->desc.n_kv_heads, 0, stream>>>(c->dev, layer, total_tokens,

@@ -34,6 +34,18 @@ struct AppendPlan {
 };
 static_assert(sizeof(AppendPlan) == 64, "plan record");
 
+// pask_decide reuses the plan records (calls on one cache are ordered by their stream): what one
+// sequence's tokens add to its running budget, committed by the CTA that arrives last
+struct DecidePlan {
+    int32_t seq;                   // -1: this entry of the call is invalid
+    uint32_t pad0;
+    uint64_t full, retained;       // bytes added to decided_full_bytes / decided_retained_bytes
+    uint64_t demoted, promoted, conflicts;
+    uint64_t pad1[2];
+};
+static_assert(sizeof(DecidePlan) == sizeof(AppendPlan), "plan record");
+constexpr uint32_t kMaxStatesDev = 65536;   // state ids are 16-bit
+
 // Device view of a cache, passed to kernels by value.
 struct DevCache {
     uint8_t *pool_high, *pool_low;
@@ -48,6 +60,13 @@ struct DevCache {
     uint2 *tok_scratch;              // [max_append_tokens] {action | stream position << 2, index in call}
     uint8_t *lut;                    // [n_tags][n_groups] effective action max(a0, floor)
     uint8_t *layer_group;            // [n_layers]
+    // tables of the budget-dependent adjustment (pask_decide)
+    uint2 *dec_row;                  // [256] per tag byte: x = actions (2 bits per group) | floors << 16, y = cost of the actions
+    float2 *dec_rho;                 // [n_tags][n_groups] upgrade scores {R->L, L->H}
+    uint32_t *gamma;                 // [n_states_dev] reserve in units of 2^gamma_shift bytes
+    uint8_t *crit;                   // [n_states_dev] critical-state flags
+    uint32_t n_states_dev, gamma_shift;
+    uint32_t group_layers[PASK_MAX_GROUPS];   // layers per group
     int32_t n_layers, n_q, n_kv, max_seqs, max_pages, max_append_tokens;
     int32_t n_tags, n_groups;
     uint32_t cap_high, cap_low;
@@ -58,7 +77,7 @@ struct DevCache {
 
 struct MetaOffsets {
     size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, low_vmax, plan, tok_scratch, lut,
-        layer_group, total;
+        layer_group, dec_row, dec_rho, gamma, crit, total;
     size_t zero_begin, zero_end;     // the span cleared by a reset (counters, tables, budgets, marks)
 };
 
@@ -69,6 +88,8 @@ struct pask_policy {
     std::vector<uint8_t> layer_group, a0, a_floor, eff;
     std::vector<float> rho_rl, rho_lh;
     std::vector<uint32_t> gamma;
+    std::vector<uint8_t> crit;
+    uint32_t gamma_shift;
 };
 
 struct pask_cache {
@@ -113,7 +134,9 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // launchers implemented next to their kernels
 pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_tokens, const int32_t *seq_ids,
                             const int32_t *cu_tokens, const void *k, const void *v, const uint8_t *tags,
-                            uint8_t *actions_out, cudaStream_t stream);
+                            const uint8_t *decided, uint8_t *actions_out, cudaStream_t stream);
+pask_status_t launch_decide(pask_cache *c, int n_seqs, int total_tokens, const int32_t *seq_ids, const int32_t *cu_tokens,
+                            const uint8_t *tags, const uint16_t *states, uint8_t *actions_out, cudaStream_t stream);
 pask_status_t launch_seq_reset(pask_cache *c, int seq, cudaStream_t stream);
 pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seqs, const int32_t *seq_ids,
                                const void *q, float *out, float *lse, void *workspace, size_t workspace_bytes,

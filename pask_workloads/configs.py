@@ -15,7 +15,8 @@ import numpy as np
 import torch
 
 from . import tags as T
-from .policy import Policy, greedy_policy, random_policy, all_high_policy, write_blob, expected_cost
+from .policy import (Policy, greedy_policy, random_policy, all_high_policy, write_blob, expected_cost,
+                     with_dynamic_budget)
 from .rng import BASE_SEED, CounterRng
 from .tensors import TENSOR_K, TENSOR_Q, TENSOR_V, normal_bf16
 
@@ -88,6 +89,19 @@ class Workload:
         """Tags of tokens t0 .. t0+n-1 of sequence b (prompt first, then generated)."""
         full = np.concatenate([self.prompt_tags[b], self.gen_tags[b]])
         return full[t0:t0 + n]
+
+    def states(self, b: int, t0: int, n: int) -> np.ndarray:
+        """Synthetic parser-state ids of the same tokens."""
+        full = np.concatenate([self.prompt_tags[b], self.gen_tags[b]])
+        return T.parser_states(full)[t0:t0 + n]
+
+    def dynamic_blob(self, reserve_tokens: int = 32, budget: Optional[float] = None) -> bytes:
+        """The table with critical-state flags, reserves and floors attached (version-2 blob)."""
+        full = self.cfg.n_layers * 2 * self.cfg.n_kv * 128 * 2
+        pol = with_dynamic_budget(self.policy, self.seed, full, reserve_tokens)
+        if budget is not None:
+            pol = replace(pol, budget_target=budget)
+        return write_blob(pol)
 
     def kv(self, layer: int, b: int, t0: int, n: int, device="cpu"):
         k = normal_bf16(self.seed, TENSOR_K, layer, b, t0, n, self.cfg.n_kv, device)

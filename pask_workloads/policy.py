@@ -180,3 +180,20 @@ def expected_cost(p: Policy, tag_counts: np.ndarray) -> float:
     per = np.where(eff == H, 1.0, np.where(eff == L, COST_L_OVER_H, 0.0))
     f = tag_counts.astype(np.float64) / max(1.0, float(tag_counts.sum()))
     return float((f[:, None] * w[None, :] * per).sum())
+
+
+def with_dynamic_budget(p: Policy, seed: int, token_full_bytes: int, reserve_tokens: int = 32,
+                        gamma_shift: int = 8) -> Policy:
+    """A copy of `p` that carries what the budget-dependent adjustment reads: critical-state flags
+    for the synthetic parser states and a reserve per state of up to `reserve_tokens` tokens' full
+    cost (Eq. 9's quantile needs calibration traces; here it is a seeded random amount), plus
+    floors on the required-key and enum-value rows so that protection and budget can conflict."""
+    from dataclasses import replace
+    rng = CounterRng(seed, 808)
+    gamma = np.asarray([(rng.below(reserve_tokens + 1) * token_full_bytes) >> gamma_shift
+                        for _ in range(T.N_STATES)], dtype=np.uint32)
+    fl = p.a_floor.copy()
+    for z in (T.REQUIRED_KEY, T.ENUM_VALUE):
+        if z < p.n_tags:
+            fl[z, :] = np.maximum(fl[z, :], L)
+    return replace(p, a_floor=fl, gamma=gamma, gamma_shift=gamma_shift, crit=T.critical_states())

@@ -227,3 +227,37 @@ def mix_decode_tags(seed: int, seq: int, n_tokens: int) -> np.ndarray:
 def mix_prompt_tags(seed: int, seq: int, n_tokens: int) -> np.ndarray:
     ids = [P_SCHEMA_SCAFFOLD, P_PARAMETER_KEY, P_CONSTRAINT, P_FUNCTION_NAME, P_PROTECTED]
     return mix_tags(seed, seq, n_tokens, ids, [0.55, 0.15, 0.15, 0.05, 0.10], stream=404)
+
+
+# ---- synthetic parser states -------------------------------------------------------------
+# The online lookup also sees the parser state s_t (it selects the reserve and says whether the
+# position is critical).  The toy grammar above has no automaton to take states from, so a state
+# id is derived from the tag stream itself: which structural class the token belongs to and how
+# far into a run of that class it sits (0, 1, 2, 3+).  Ids: tag * 4 + min(run position, 3) for
+# the eleven table tags, 44 for protected tokens, 47 for anything else.
+N_STATES = 48
+STATE_PROTECTED = 44
+STATE_OTHER = 47
+
+
+def parser_states(tags: np.ndarray) -> np.ndarray:
+    out = np.zeros(tags.shape[0], dtype=np.uint16)
+    run = 0
+    for i, z in enumerate(tags.tolist()):
+        run = run + 1 if i and tags[i - 1] == z else 0
+        if z < N_ALL_TAGS:
+            out[i] = z * 4 + min(run, 3)
+        else:
+            out[i] = STATE_PROTECTED if z == TAG_PROTECTED else STATE_OTHER
+    return out
+
+
+def critical_states() -> np.ndarray:
+    """Flags of the states treated as critical or lookahead-critical: everything inside a required
+    key or an enum value, and the first token of an argument value or of a boundary."""
+    crit = np.zeros(N_STATES, dtype=np.uint8)
+    for z in (REQUIRED_KEY, ENUM_VALUE):
+        crit[z * 4:z * 4 + 4] = 1
+    crit[ARGUMENT_VALUE * 4] = 1
+    crit[BOUNDARY * 4] = 1
+    return crit

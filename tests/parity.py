@@ -57,6 +57,49 @@ class Pair:
             assert np.array_equal(act_g.cpu().numpy()[:len(tags)], act_o), "actions differ"
         return rc, act_o
 
+    # ------------------------------------------------------------------ dynamic budget adjustment
+    def gather(self, seq_ids, counts, starts, layer=None):
+        """tags, states (and k, v of `layer`) of tokens starts[i] .. +counts[i]-1, call order."""
+        w = self.w
+        ts = [w.tags(int(s), int(t0), int(n)) for s, n, t0 in zip(seq_ids, counts, starts)]
+        ss = [w.states(int(s), int(t0), int(n)) for s, n, t0 in zip(seq_ids, counts, starts)]
+        tags = np.concatenate(ts) if ts else np.zeros(0, np.uint8)
+        states = np.concatenate(ss) if ss else np.zeros(0, np.uint16)
+        if layer is None:
+            return tags, states
+        kv = [w.kv(layer, int(s), int(t0), int(n)) for s, n, t0 in zip(seq_ids, counts, starts)]
+        return tags, states, torch.cat([a for a, _ in kv]), torch.cat([b for _, b in kv])
+
+    def decide(self, seq_ids, counts, tags, states, expect_ok=True):
+        """pask_decide on both sides; returns (oracle status, oracle actions, gpu actions tensor)."""
+        d = "cuda"
+        cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+        G = self.cfg.n_groups
+        rc, act_o = self.orc.decide(seq_ids, cu, tags, states=states, n_groups=G)
+        act_g = torch.full((max(1, len(tags)), G), 0xEE, dtype=torch.uint8, device=d)
+        st = None if states is None else torch.from_numpy(states.astype(np.int16)).to(d)
+        self.pask.pask_decide(self.gpu.handle, torch.tensor(seq_ids, dtype=torch.int32, device=d),
+                              torch.from_numpy(cu).to(d), torch.from_numpy(tags).to(d), st, act_g)
+        torch.cuda.synchronize()
+        if expect_ok:
+            assert rc == 0
+            assert np.array_equal(act_g.cpu().numpy()[:len(tags)], act_o), "decided actions differ"
+        return rc, act_o, act_g
+
+    def append_decided(self, layer, seq_ids, counts, k, v, tags, act_o, act_g, expect_ok=True):
+        d = "cuda"
+        cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+        rc, used_o = self.orc.append(layer, seq_ids, cu, bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags, decided=act_o)
+        used_g = torch.full((max(1, len(tags)),), 0xEE, dtype=torch.uint8, device=d)
+        self.pask.pask_append_kv_decided(self.gpu.handle, layer, torch.tensor(seq_ids, dtype=torch.int32, device=d),
+                                         torch.from_numpy(cu).to(d), k.to(d), v.to(d), torch.from_numpy(tags).to(d),
+                                         act_g, actions_out=used_g, total_tokens=len(tags))
+        torch.cuda.synchronize()
+        if expect_ok:
+            assert rc == 0
+            assert np.array_equal(used_g.cpu().numpy()[:len(tags)], used_o), "persisted actions differ"
+        return rc
+
     # ------------------------------------------------------------------ state
     def compare_state(self, layers=None, seqs=None):
         P, h = self.pask, self.gpu.handle
@@ -84,7 +127,8 @@ class Pair:
         g, o = self.pask.pask_budget_state(self.gpu.handle, s), self.orc.budget(s)
         for f in ("n_seen", "n_high", "n_low", "n_drop"):
             assert list(getattr(g, f)) == list(getattr(o, f)), (f, s)
-        for f in ("retained_bytes", "full_bytes", "remaining_bytes", "bad_tags", "pages_high", "pages_low"):
+        for f in ("retained_bytes", "full_bytes", "remaining_bytes", "bad_tags", "pages_high", "pages_low",
+                  "decided_full_bytes", "decided_retained_bytes", "n_demoted", "n_promoted", "n_floor_conflicts"):
             assert getattr(g, f) == getattr(o, f), (f, s, getattr(g, f), getattr(o, f))
         assert g.device_status == expect_status, g.device_status
         return g

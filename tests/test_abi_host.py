@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol(pask):
 
 
 def test_struct_layouts_match_header(pask):
-    assert C.sizeof(pask.BudgetState) == 4 * 8 * 8 + 4 * 8 + 4 * 4
+    assert C.sizeof(pask.BudgetState) == 4 * 8 * 8 + 4 * 8 + 4 * 4 + 5 * 8
     assert C.sizeof(pask.CacheDesc) == 40
 
 
@@ -48,6 +48,27 @@ def test_policy_blob_parsing_agrees_with_oracle(pask, oracle):
                 assert pask.pask_policy_action(h, z, c) == o.action(z, c) == max(w.policy.a0[z, c], w.policy.a_floor[z, c])
         assert pask.pask_policy_action(h, w.policy.n_tags, 0) == -1
         pask.pask_free_policy(h)
+
+
+def test_version_2_blobs(pask, oracle):
+    # critical-state flags and the reserve shift ride behind gamma; both loaders take and refuse the same blobs
+    w = WC.build(WC.scaled(WC.QWEN3_4B_1LAYER, batch=1, prompt_len=32, gen_len=32))
+    good = w.dynamic_blob()
+    assert good[4] == 2
+    pask.pask_free_policy(pask.pask_load_policy(good))
+    oracle.Policy(good)
+    n_states = int.from_bytes(good[20:24], "little")
+    crit_at = len(good) - ((n_states + 3) // 4) * 4
+    bads = [good[:-4], good + b"\0\0\0\0"]
+    b = bytearray(good); b[crit_at] = 2; bads.append(bytes(b))                 # a flag that is not 0 or 1
+    b = bytearray(good); b[crit_at - 4] = 17; bads.append(bytes(b))            # gamma_shift > 16
+    b = bytearray(good); b[40 + 4 + 4:40 + 4 + 8] = b"\x00\x00\xc0\x7f"; bads.append(bytes(b))   # a NaN score
+    for blob in bads:
+        with pytest.raises(pask.PaskError) as e:
+            pask.pask_load_policy(blob)
+        assert e.value.status == pask.ERR_BAD_POLICY
+        with pytest.raises(ValueError):
+            oracle.Policy(blob)
 
 
 def test_bad_blobs_and_arguments_are_refused(pask):
