@@ -173,8 +173,9 @@ class ClockSampler:
 class Job:
     """One rank's cache, filled with the workload's history, ready to run decode steps."""
 
-    def __init__(self, P, w, device, total_steps, policy_blob=None, label="pask"):
+    def __init__(self, P, w, device, total_steps, policy_blob=None, label="pask", dynamic=False):
         self.P, self.w, self.device, self.label = P, w, device, label
+        self.dynamic = dynamic
         cfg = w.cfg
         self.cfg = cfg
         self.B = cfg.batch
@@ -184,6 +185,13 @@ class Job:
             tot = np.array([w.total_len(b) for b in range(self.B)], np.int64)
             nh = np.repeat(tot[:, None], w.policy.n_groups, axis=1)
             nl = np.zeros_like(nh)
+        if dynamic:
+            # actions depend on the running budget: size both pools for the worst case (the
+            # realised counts are read back from the budget states after the fill)
+            blob = w.dynamic_blob()
+            tot = np.array([w.total_len(b) for b in range(self.B)], np.int64)
+            nh = np.repeat(tot[:, None], w.policy.n_groups, axis=1)
+            nl = nh.copy()
         self.nh, self.nl = nh, nl
         lg = w.policy.layer_group.astype(np.int64)
         extra = total_steps + 1
@@ -205,15 +213,35 @@ class Job:
         w, cfg, d = self.w, self.cfg, self.device
         cu = torch.tensor(np.concatenate([[0], np.cumsum(self.lens)]), dtype=torch.int32, device=d)
         tags = torch.from_numpy(np.concatenate([w.tags(b, 0, self.lens[b]) for b in range(self.B)])).to(d)
+        decided = None
+        if self.dynamic:
+            states = torch.from_numpy(np.concatenate([w.states(b, 0, self.lens[b]) for b in range(self.B)]).astype(np.int16)).to(d)
+            decided = torch.empty((self.total_tokens, cfg.n_groups), dtype=torch.uint8, device=d)
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            self.P.pask_decide(self.cache.handle, self.ids, cu, tags, states, decided)
+            b_.record()
+            torch.cuda.synchronize()
+            self.prefill_decide_ms = a.elapsed_time(b_)
         for layer in range(cfg.n_layers):
             k = torch.cat([normal_bf16(w.seed, TENSOR_K, layer, b, 0, self.lens[b], cfg.n_kv, d) for b in range(self.B)])
             v = torch.cat([normal_bf16(w.seed, TENSOR_V, layer, b, 0, self.lens[b], cfg.n_kv, d) for b in range(self.B)])
-            self.P.pask_append_kv(self.cache.handle, layer, self.ids, cu, k, v, tags)
+            if decided is None:
+                self.P.pask_append_kv(self.cache.handle, layer, self.ids, cu, k, v, tags)
+            else:
+                self.P.pask_append_kv_decided(self.cache.handle, layer, self.ids, cu, k, v, tags, decided)
             del k, v
         torch.cuda.synchronize()
         st = self.P.pask_budget_state(self.cache.handle, 0)
         if st.device_status:
             raise RuntimeError(f"device status {st.device_status:#x} after fill")
+        if self.dynamic:       # what was actually kept, per (sequence, group), in tokens per layer
+            lig = np.bincount(w.policy.layer_group, minlength=cfg.n_groups)
+            for b in range(self.B):
+                st = self.P.pask_budget_state(self.cache.handle, b)
+                for g in range(cfg.n_groups):
+                    self.nh[b, g] = st.n_high[g] // max(1, lig[g])
+                    self.nl[b, g] = st.n_low[g] // max(1, lig[g])
 
     def prepare_steps(self, n_steps):
         w, cfg, d = self.w, self.cfg, self.device
@@ -224,12 +252,21 @@ class Job:
                 k, v, q, tags = step_inputs(w, layer, s, d)
                 per_layer.append((k, v, q, torch.from_numpy(tags).to(d)))
             self.steps.append(per_layer)
+        if self.dynamic:
+            self.step_states = [torch.from_numpy(np.array([w.states(b, w.total_len(b) + s, 1)[0] for b in range(self.B)],
+                                                          np.int16)).to(d) for s in range(n_steps)]
+            self.decided = torch.empty((self.B, cfg.n_groups), dtype=torch.uint8, device=d)
 
     def run_step(self, s, events=None):
         """events: {layer: (start, stop)} for the launches of this step whose streaming kernel is timed."""
         P, h = self.P, self.cache.handle
+        if self.dynamic:       # Algorithm 2 steps 1-6 once per token, then step 7 layer by layer
+            P.pask_decide(h, self.ids, self.cu1, self.steps[s][0][3], self.step_states[s], self.decided)
         for layer, (k, v, q, tags) in enumerate(self.steps[s]):
-            P.pask_append_kv(h, layer, self.ids, self.cu1, k, v, tags)
+            if self.dynamic:
+                P.pask_append_kv_decided(h, layer, self.ids, self.cu1, k, v, tags, self.decided)
+            else:
+                P.pask_append_kv(h, layer, self.ids, self.cu1, k, v, tags)
             if events is not None and layer in events:
                 P.pask_cache_set_timing_events(h, *events[layer])
             self.attn(h, layer, self.ids, q, self.out, self.lse, self.ws)
@@ -267,7 +304,7 @@ def run_cuda(args, rank, world):
     cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, 2 * total_steps + e2e_steps + 8))
     w = rank_workload(cfg, rank)
     t_setup = time.time()
-    job = Job(P, w, device, 2 * total_steps + e2e_steps + 4)
+    job = Job(P, w, device, 2 * total_steps + e2e_steps + 4, dynamic=args.dynamic)
     job.fill()
     job.prepare_steps(total_steps)
     t_setup = time.time() - t_setup
@@ -309,7 +346,7 @@ def run_cuda(args, rank, world):
 
     # ---- end to end: the same step through the host-buffer entry point, copies inside the region
     e2e = None
-    if rank == 0 or world > 1:
+    if (rank == 0 or world > 1) and not args.dynamic:   # the host-buffer entry point applies the frozen table
         staging = torch.empty(P.pask_step_staging_bytes(job.cache.handle, job.B), dtype=torch.uint8, device=device)
         host = []
         for s in range(e2e_steps):
@@ -352,7 +389,7 @@ def run_cuda(args, rank, world):
                    "setup_s": round(t_setup, 1)},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": 4 * cfg.n_layers * args.steps,
+        "gpu_launches": (4 * cfg.n_layers + (1 if args.dynamic else 0)) * args.steps,
         "roofline": {"bound": "hbm", "kernel": "decode_attn_kernel<true>", "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "algorithmic_bytes_per_launch": alg,
@@ -361,6 +398,12 @@ def run_cuda(args, rank, world):
         "attention_share_of_step": k_ms * cfg.n_layers * args.steps / ms,
         "attention_only_tokens_per_s": world * job.B / (k_ms * 1e-3 * cfg.n_layers),
     }
+    if args.dynamic:
+        sts = [P.pask_budget_state(job.cache.handle, b) for b in range(job.B)]
+        line["dynamic_budget"] = {"prefill_decide_ms": job.prefill_decide_ms, "prefill_tokens": job.total_tokens,
+                                  "demoted": sum(s.n_demoted for s in sts), "promoted": sum(s.n_promoted for s in sts),
+                                  "floor_conflicts": sum(s.n_floor_conflicts for s in sts)}
+        line["config"]["table"] += " + budget-dependent adjustment (pask_decide)"
     if args.full_kv and world == 1:
         line["full_kv"] = run_full_kv(P, args, w, device, total_steps, peak)
     if args.cpu_seconds > 0:
@@ -491,6 +534,8 @@ def main():
     ap.add_argument("--no-full-kv", dest="full_kv", action="store_false")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="0 skips the CPU-oracle leg")
     ap.add_argument("--event-stride", type=int, default=4, help="time the streaming kernel of every n-th launch")
+    ap.add_argument("--dynamic", action="store_true",
+                    help="decide every token against the running budget (pask_decide) instead of the frozen table alone")
     ap.add_argument("--layers", type=int, default=None, help="profiling aid: keep only the first N layers")
     ap.add_argument("--ref-seqs", type=int, default=32, help="sequences in the oracle's timed sample")
     args = ap.parse_args()

@@ -29,11 +29,13 @@ decide_kernel(DevCache c, int n_seqs, int total_tokens, const int32_t *__restric
               const int32_t *__restrict__ cu_tokens, const uint8_t *__restrict__ tags,
               const uint16_t *__restrict__ states, uint8_t *__restrict__ actions_out, uint32_t serial) {
     __shared__ uint2 s_row[256];
+    __shared__ float2 s_rho[255 * PASK_MAX_GROUPS];   // upgrade scores: read inside the Demote / Promote loops
     __shared__ uint32_t s_layers[PASK_MAX_GROUPS];
     __shared__ int s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = c.n_groups;
     s_row[tid] = c.dec_row[tid];
+    for (int x = tid; x < c.n_tags * G; x += kDecideThreads) s_rho[x] = c.dec_rho[x];
     if (tid < PASK_MAX_GROUPS) s_layers[tid] = c.group_layers[tid];
     __syncthreads();
     uint32_t token_full = 0;                       // full cost of one token over all layers
@@ -91,7 +93,7 @@ decide_kernel(DevCache c, int n_seqs, int total_tokens, const int32_t *__restric
                             for (int g = 0; g < G; g++) {
                                 const uint32_t ag = act_of(a, g);
                                 if (ag <= act_of(fl, g) || s_layers[g] == 0) continue;
-                                const float2 rho = c.dec_rho[tag * G + g];
+                                const float2 rho = s_rho[tag * G + g];
                                 const float score = ag == PASK_ACTION_RETAIN_HIGH ? rho.y : rho.x;
                                 if (pick < 0 || score < best) { pick = g; best = score; }
                             }
@@ -112,7 +114,7 @@ decide_kernel(DevCache c, int n_seqs, int total_tokens, const int32_t *__restric
                                 if (ag >= PASK_ACTION_RETAIN_HIGH || s_layers[g] == 0) continue;
                                 const uint64_t up = (uint64_t)s_layers[g] * (ag == PASK_ACTION_RETAIN_LOW ? step_hl : step_lr);
                                 if ((int64_t)(cost + up) > B) continue;
-                                const float2 rho = c.dec_rho[tag * G + g];
+                                const float2 rho = s_rho[tag * G + g];
                                 const float score = ag == PASK_ACTION_RETAIN_LOW ? rho.y : rho.x;
                                 if (pick < 0 || score > best) { pick = g; best = score; }
                             }

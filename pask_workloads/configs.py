@@ -92,8 +92,10 @@ class Workload:
 
     def states(self, b: int, t0: int, n: int) -> np.ndarray:
         """Synthetic parser-state ids of the same tokens."""
-        full = np.concatenate([self.prompt_tags[b], self.gen_tags[b]])
-        return T.parser_states(full)[t0:t0 + n]
+        cache = self.__dict__.setdefault("_states", {})
+        if b not in cache:
+            cache[b] = T.parser_states(np.concatenate([self.prompt_tags[b], self.gen_tags[b]]))
+        return cache[b][t0:t0 + n]
 
     def dynamic_blob(self, reserve_tokens: int = 32, budget: Optional[float] = None) -> bytes:
         """The table with critical-state flags, reserves and floors attached (version-2 blob)."""
