@@ -40,7 +40,8 @@ MetaOffsets meta_offsets(const pask_cache_desc_t *d, int n_tags, int n_groups) {
     o.low_vmax = take(sl * 4);
     o.zero_end = p;
     o.plan = take((size_t)PASK_MAX_SEQS_PER_CALL * sizeof(AppendPlan));
-    o.tok_scratch = take((size_t)d->max_append_tokens * sizeof(uint2));
+    o.tok_list = take((size_t)d->max_append_tokens * 4);
+    o.item_base = take((size_t)(PASK_MAX_SEQS_PER_CALL + 1) * 4);
     o.lut = take((size_t)n_tags * n_groups);
     o.layer_group = take((size_t)d->n_layers);
     o.dec_row = take(256 * sizeof(uint2));
@@ -197,7 +198,8 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     v.seq_mark = reinterpret_cast<uint32_t *>(m + c->off.seq_mark);
     v.low_vmax = reinterpret_cast<uint32_t *>(m + c->off.low_vmax);
     v.plan = reinterpret_cast<AppendPlan *>(m + c->off.plan);
-    v.tok_scratch = reinterpret_cast<uint2 *>(m + c->off.tok_scratch);
+    v.tok_list = reinterpret_cast<uint32_t *>(m + c->off.tok_list);
+    v.item_base = reinterpret_cast<uint32_t *>(m + c->off.item_base);
     v.lut = m + c->off.lut;
     v.layer_group = m + c->off.layer_group;
     v.dec_row = reinterpret_cast<uint2 *>(m + c->off.dec_row);

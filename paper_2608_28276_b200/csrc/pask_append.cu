@@ -32,6 +32,12 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
     return m;
 }
 
+// pages of a stream that an append of cnt tokens at length old writes into (the first may be a page
+// the stream already holds)
+__device__ __forceinline__ uint32_t pages_touched(uint32_t old, uint32_t cnt) {
+    return cnt ? ((old + cnt - 1) >> 4) - (old >> 4) + 1 : 0u;
+}
+
 // exclusive scan of one value per thread over a 256-thread block; returns the block total too
 __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *s_warp, uint32_t *total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -116,7 +122,10 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
                 uint32_t pos = 0;
                 if (a == PASK_ACTION_RETAIN_HIGH) pos = off_h + __popc(mh & lanemask_lt());
                 else if (a == PASK_ACTION_RETAIN_LOW) pos = off_l + __popc(ml & lanemask_lt());
-                c.tok_scratch[t] = make_uint2((uint32_t)a | (pos << 2), (uint32_t)i);
+                // stream-ordered token lists for the write kernel: HIGH from the front of the
+                // sequence's token range, LOW from its back
+                if (a == PASK_ACTION_RETAIN_HIGH) c.tok_list[t0 + pos] = (uint32_t)t;
+                else if (a == PASK_ACTION_RETAIN_LOW) c.tok_list[t1 - 1 - pos] = (uint32_t)t;
                 if (actions_out) actions_out[t] = (uint8_t)a;
             }
             __syncthreads();
@@ -141,6 +150,8 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
             const uint32_t pl0 = (p.old_low + kPageTokens - 1) / kPageTokens, pl1 = (p.old_low + p.cnt_low + kPageTokens - 1) / kPageTokens;
             p.new_pages_high = ph1 - ph0;
             p.new_pages_low = pl1 - pl0;
+            p.tok0 = t0;
+            p.tok1 = t1;
             if (ph1 > (uint32_t)c.max_pages || pl1 > (uint32_t)c.max_pages) { err |= PASK_DEV_SEQ_OVERFLOW; p.seq = -1; }
         }
         if (err) atomicOr(&c.ctrl[kCtrlStatus], err);
@@ -154,25 +165,28 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
     // ---- last CTA: allocate for the whole call and commit, or refuse
     __threadfence();
     constexpr int kPer = PASK_MAX_SEQS_PER_CALL / kPlanThreads;  // sequences per thread, blocked
-    uint32_t nh[kPer], nl[kPer];
-    uint32_t sum_h = 0, sum_l = 0;
+    uint32_t nh[kPer], nl[kPer], ni[kPer];
+    uint32_t sum_h = 0, sum_l = 0, sum_i = 0;
     int any_bad = 0;
 #pragma unroll
     for (int r = 0; r < kPer; r++) {
         const int j = tid * kPer + r;
-        nh[r] = nl[r] = 0;
+        nh[r] = nl[r] = ni[r] = 0;
         if (j < n_seqs) {
             const AppendPlan p = load_plan_cg(&c.plan[j]);
             if (p.seq < 0) any_bad = 1;
             nh[r] = p.new_pages_high;
             nl[r] = p.new_pages_low;
+            ni[r] = pages_touched(p.old_high, p.cnt_high) + pages_touched(p.old_low, p.cnt_low);
         }
         sum_h += nh[r];
         sum_l += nl[r];
+        sum_i += ni[r];
     }
-    uint32_t need_h, need_l;
+    uint32_t need_h, need_l, n_items;
     uint32_t base_h = block_excl_scan(sum_h, s_scan, &need_h);
     uint32_t base_l = block_excl_scan(sum_l, s_scan, &need_l);
+    uint32_t base_i = block_excl_scan(sum_i, s_scan, &n_items);
     any_bad = __syncthreads_or(any_bad);
     const uint32_t free_h = c.ctrl[kCtrlHighFree], next_h = c.ctrl[kCtrlHighNext];
     const uint32_t free_l = c.ctrl[kCtrlLowFree], next_l = c.ctrl[kCtrlLowNext];
@@ -204,6 +218,8 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         }
         base_h += nh[r];
         base_l += nl[r];
+        c.item_base[j] = base_i;
+        base_i += ni[r];
         c.n_high[sl] = p.old_high + p.cnt_high;
         c.n_low[sl] = p.old_low + p.cnt_low;
         pask_budget_state_t &b = c.budget[p.seq];
@@ -224,6 +240,8 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         c.ctrl[kCtrlHighNext] = next_h + (need_h - pop_h);
         c.ctrl[kCtrlLowFree] = free_l - pop_l;
         c.ctrl[kCtrlLowNext] = next_l + (need_l - pop_l);
+        c.ctrl[kCtrlItems] = n_items;
+        c.item_base[n_seqs] = n_items;
         c.ctrl[kCtrlPlanOk] = 1;
         c.ctrl[kCtrlTicket] = 0;
     }
@@ -301,27 +319,172 @@ __device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uin
     if ((threadIdx.x & 31) == 0 && hb > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb);
 }
 
-// General path, second kernel.  One CTA (32 * n_kv threads) per token at a time; thread = one
-// 16-byte chunk (8 head dims) of K (first half of the block) or V (second half).
-__global__ void __launch_bounds__(256)
-append_write_kernel(DevCache c, int layer, int total_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v) {
+// General path, second kernel: page-centric.  The plan kernel left, per sequence, its retained
+// tokens in stream order (tok_list) and a prefix over sequences of the stream pages the call
+// writes into (item_base).  A work item is one such page; CTA b takes the items
+// [T b / G, T (b+1) / G).  A page whose 16 tokens all come from this call -- nearly every page of
+// a prefill -- is assembled head by head in shared memory from the 16 source rows and leaves as
+// one run of 128-bit stores in the packed layout; a partly filled page (the first and last page of
+// a stream's range at most) is written token by token with persist_chunk.
+constexpr int kWriteThreads = 256;
+constexpr int kRowBytes = 2 * kHeadDim + 16;      // one token's K (or V) row of a head in shared memory, padded
+
+__global__ void __launch_bounds__(kWriteThreads, 4)
+append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__ k, const uint4 *__restrict__ v) {
+    __shared__ uint32_t s_base[PASK_MAX_SEQS_PER_CALL + 1];
+    __shared__ __align__(16) uint8_t s_in[2][kPageTokens][kRowBytes];   // [K|V][token][dims of one head]
+    __shared__ __align__(16) uint8_t s_low[kLowHeadBytes];              // one head of a LOW page, packed
+    __shared__ uint32_t s_tok[kPageTokens];
     if (c.ctrl[kCtrlPlanOk] == 0) return;
     const int tid = threadIdx.x;
-    const int chunks = 16 * c.n_kv;            // 16-byte chunks per token per tensor
-    const int which = tid >= chunks;           // 0 = K, 1 = V
-    const int cg = which ? tid - chunks : tid;
-    const int head = cg >> 4, cch = cg & 15;
-    const uint4 *src = which ? v : k;
-    for (int t = blockIdx.x; t < total_tokens; t += gridDim.x) {
-        const uint2 sc = c.tok_scratch[t];
-        const uint32_t a = sc.x & 3u, pos = sc.x >> 2;
-        if (a == PASK_ACTION_RELEASE) continue;
-        const AppendPlan &p = c.plan[sc.y];
+    const uint32_t n_items = c.ctrl[kCtrlItems];
+    const uint32_t item0 = (uint32_t)(((uint64_t)n_items * blockIdx.x) / gridDim.x);
+    const uint32_t item1 = (uint32_t)(((uint64_t)n_items * (blockIdx.x + 1)) / gridDim.x);
+    if (item0 >= item1) return;
+    for (int x = tid; x <= n_seqs; x += kWriteThreads) s_base[x] = c.item_base[x];
+    __syncthreads();
+    int j = 0;                                     // the sequence item0 belongs to: s_base[j] <= item0 < s_base[j + 1]
+    {
+        int lo = 0, hi = n_seqs - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (s_base[mid] <= item0) lo = mid; else hi = mid - 1;
+        }
+        j = lo;
+    }
+    const int chunks = 16 * c.n_kv;                // 16-byte chunks per token per tensor
+    AppendPlan p = c.plan[j];
+    for (uint32_t item = item0; item < item1; item++) {
+        bool moved = false;
+        while (item >= s_base[j + 1]) { j++; moved = true; }
+        if (moved) p = c.plan[j];
+        const uint32_t in_seq = item - s_base[j];
+        const uint32_t items_h = pages_touched(p.old_high, p.cnt_high);
+        const bool high = in_seq < items_h;
+        const uint32_t old = high ? p.old_high : p.old_low, cnt = high ? p.cnt_high : p.cnt_low;
+        const uint32_t pg = (old >> 4) + (high ? in_seq : in_seq - items_h);
+        const uint32_t at0 = old > 16u * pg ? old : 16u * pg;
+        const uint32_t at1 = old + cnt < 16u * pg + 16u ? old + cnt : 16u * pg + 16u;
         const size_t sl = (size_t)p.seq * c.n_layers + layer;
-        const uint4 x = src[(size_t)t * chunks + cg];
-        const uint32_t at = (a == PASK_ACTION_RETAIN_HIGH ? p.old_high : p.old_low) + pos;
-        const uint32_t *tbl = a == PASK_ACTION_RETAIN_HIGH ? c.tbl_high : c.tbl_low;
-        persist_chunk(c, a, at, tbl[sl * c.max_pages + (at >> 4)], sl, head, cch, which, x);
+        const uint32_t page = (high ? c.tbl_high : c.tbl_low)[sl * c.max_pages + pg];
+        const uint32_t action = high ? PASK_ACTION_RETAIN_HIGH : PASK_ACTION_RETAIN_LOW;
+        __syncthreads();                           // the previous item is done with s_tok
+        if ((uint32_t)tid < at1 - at0) {
+            const uint32_t r = at0 + tid - old;     // rank among the sequence's tokens of this stream
+            s_tok[tid] = c.tok_list[high ? p.tok0 + r : p.tok1 - 1 - r];
+        }
+        __syncthreads();
+        if (at1 - at0 < (uint32_t)kPageTokens || page >= (high ? c.cap_high : c.cap_low)) {
+            // partly filled page (or a page id the bounds check refuses): token by token
+            if (tid < 2 * chunks) {
+                const int which = tid >= chunks, cg = which ? tid - chunks : tid;
+                for (uint32_t at = at0; at < at1; at++) {
+                    const uint4 x = (which ? v : k)[(size_t)s_tok[at - at0] * chunks + cg];
+                    persist_chunk(c, action, at, page, sl, cg >> 4, cg & 15, which, x);
+                }
+            }
+            continue;
+        }
+        // ---- a full page: per head, 16 rows of K and of V in, one packed block out
+        uint4 nx[2];
+#pragma unroll
+        for (int r = 0; r < 2; r++) {              // rows of head 0: chunk idx = which * 256 + token * 16 + chunk
+            const int idx = tid + r * kWriteThreads, which = idx >> 8, tau = (idx >> 4) & 15, ch = idx & 15;
+            nx[r] = (which ? v : k)[(size_t)s_tok[tau] * chunks + ch];
+        }
+        uint32_t vmax_bits = 0;
+        for (int head = 0; head < c.n_kv; head++) {
+            __syncthreads();                       // readers of the previous head's rows (and of s_low) are done
+#pragma unroll
+            for (int r = 0; r < 2; r++) {
+                const int idx = tid + r * kWriteThreads, which = idx >> 8, tau = (idx >> 4) & 15, ch = idx & 15;
+                *reinterpret_cast<uint4 *>(&s_in[which][tau][ch * 16]) = nx[r];
+            }
+            if (head + 1 < c.n_kv) {
+#pragma unroll
+                for (int r = 0; r < 2; r++) {
+                    const int idx = tid + r * kWriteThreads, which = idx >> 8, tau = (idx >> 4) & 15, ch = idx & 15;
+                    nx[r] = (which ? v : k)[(size_t)s_tok[tau] * chunks + (head + 1) * 16 + ch];
+                }
+            }
+            __syncthreads();
+            if (high) {
+                uint4 *dst = reinterpret_cast<uint4 *>(c.pool_high + (size_t)page * c.high_page_bytes + (size_t)head * kHighHeadBytes);
+                const int lane = tid & 31, g = lane >> 2, t = lane & 3, i = tid >> 5;
+                {   // K tile, round i = 2 jj + hh: the operand quad of lane (g, t), see pask_layout.h
+                    const int jj = i >> 1, hh = i & 1, off = 2 * (8 * (4 * jj + t) + 4 * hh);
+                    uint4 q;
+                    q.x = *reinterpret_cast<const uint32_t *>(&s_in[0][g][off]);
+                    q.y = *reinterpret_cast<const uint32_t *>(&s_in[0][g + 8][off]);
+                    q.z = *reinterpret_cast<const uint32_t *>(&s_in[0][g][off + 4]);
+                    q.w = *reinterpret_cast<const uint32_t *>(&s_in[0][g + 8][off + 4]);
+                    dst[tid] = q;
+                }
+                {   // V tile, round i = 4 e + kk: token {2t, 2t+1, 2t+8, 2t+9}[kk], dims 64e + 4g.. and 64e + 32 + 4g..
+                    const int e = i >> 2, kk = i & 3, tau = 2 * t + (kk & 1) + 8 * (kk >> 1);
+                    const uint2 a = *reinterpret_cast<const uint2 *>(&s_in[1][tau][128 * e + 8 * g]);
+                    const uint2 b = *reinterpret_cast<const uint2 *>(&s_in[1][tau][128 * e + 64 + 8 * g]);
+                    dst[256 + tid] = make_uint4(a.x, a.y, b.x, b.y);
+                }
+            } else {
+                // thread = (K|V, token, 32-dim group, half of it): 16 values
+                const int half = tid & 1, w = (tid >> 1) & 3, tau = (tid >> 3) & 15, which = tid >> 7;
+                const uint4 x0 = *reinterpret_cast<const uint4 *>(&s_in[which][tau][64 * w + 32 * half]);
+                const uint4 x1 = *reinterpret_cast<const uint4 *>(&s_in[which][tau][64 * w + 32 * half + 16]);
+                const uint32_t xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                float f[16];
+                float amax = 0.0f;
+#pragma unroll
+                for (int e = 0; e < 8; e++) {
+                    f[2 * e] = bf16_lo(xs[e]);
+                    f[2 * e + 1] = bf16_hi(xs[e]);
+                    amax = fmaxf(amax, fmaxf(fabsf(f[2 * e]), fabsf(f[2 * e + 1])));
+                }
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                const float s32 = __fdiv_rn(amax, 7.0f);
+                __half sh = __float2half_rn(s32);
+                if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);   // saturate, never infinite
+                const float sc = __half2float(sh);
+                uint32_t code[16];
+                if (sc == 0.0f) {
+#pragma unroll
+                    for (int e = 0; e < 16; e++) code[e] = 8u;
+                } else {
+                    const float inv = __fdiv_rn(1.0f, sc);
+#pragma unroll
+                    for (int e = 0; e < 16; e++) {
+                        float r = rintf(__fmul_rn(f[e], inv));
+                        r = fminf(fmaxf(r, -7.0f), 7.0f);
+                        code[e] = (uint32_t)((int)r + 8);
+                    }
+                }
+                uint8_t *img = s_low + (which ? kLowHalfBytes : 0);
+                if (!which) {
+#pragma unroll
+                    for (int u = 0; u < 2; u++) {  // the words of dims 32w + 8t .. +7, t = 2 half + u
+                        uint32_t word = 0;
+#pragma unroll
+                        for (int e = 0; e < 8; e++) word |= code[8 * u + e] << (4 * low_k_nibble(e));
+                        *reinterpret_cast<uint32_t *>(img + low_k_word_off(tau, w, 2 * half + u)) = word;
+                    }
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 4; u++) {  // the half-words of dims 32w + 4g .. +3, g = 4 half + u
+                        const uint16_t hw = (uint16_t)(code[4 * u] | (code[4 * u + 1] << 4) | (code[4 * u + 2] << 8) | (code[4 * u + 3] << 12));
+                        *reinterpret_cast<uint16_t *>(img + low_v_half_off(tau, w, 4 * half + u)) = hw;
+                    }
+                    vmax_bits = max(vmax_bits, (uint32_t)__half_as_ushort(sh));
+                }
+                if (half == 0) *reinterpret_cast<__half *>(img + low_scale_off(tau, w)) = sh;
+                __syncthreads();
+                uint4 *dst = reinterpret_cast<uint4 *>(c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLowHeadBytes);
+                if (tid < kLowHeadBytes / 16) dst[tid] = reinterpret_cast<const uint4 *>(s_low)[tid];
+            }
+        }
+        if (!high) {   // largest V scale of the stream (decode attention forms P * scale relative to it)
+            const uint32_t hb = __reduce_max_sync(0xffffffffu, vmax_bits);
+            if ((tid & 31) == 0 && hb > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb);
+        }
     }
 }
 
@@ -562,10 +725,11 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
     append_plan_kernel<<<n_seqs, kPlanThreads, 0, stream>>>(c->dev, layer, n_seqs, total_tokens, seq_ids, cu_tokens, tags,
                                                            decided, actions_out, c->append_serial);
     if (total_tokens > 0) {
-        const int ctas = total_tokens < c->sm_count * 8 ? total_tokens : c->sm_count * 8;
-        append_write_kernel<<<ctas, 32 * c->desc.n_kv_heads, 0, stream>>>(c->dev, layer, total_tokens,
-                                                                         static_cast<const uint4 *>(k),
-                                                                         static_cast<const uint4 *>(v));
+        // at most one item per 16 tokens plus two partly filled pages per stream
+        const long long bound = (long long)total_tokens / 16 + 4LL * n_seqs;
+        const int ctas = bound < (long long)c->sm_count * 4 ? (int)bound : c->sm_count * 4;
+        append_write_kernel<<<ctas, kWriteThreads, 0, stream>>>(c->dev, layer, n_seqs, static_cast<const uint4 *>(k),
+                                                               static_cast<const uint4 *>(v));
     }
     return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }

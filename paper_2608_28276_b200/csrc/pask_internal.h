@@ -19,6 +19,7 @@ enum CtrlWord : int {
     kCtrlLowNext = 4,
     kCtrlLowFree = 5,
     kCtrlPlanOk = 6,    // 1 if the last append plan was committed, 0 if it was refused
+    kCtrlItems = 7,     // work items (stream pages touched) of the last committed bulk append
     kCtrlStats = 16,    // 8 words of decode-attention wait statistics (diagnostic builds with PASK_STATS only)
     kCtrlWords = 64
 };
@@ -30,7 +31,8 @@ struct AppendPlan {
     uint32_t cnt_high, cnt_low;    // tokens this call adds to each stream
     uint32_t cnt_drop, bad_tags;
     uint32_t new_pages_high, new_pages_low;
-    uint32_t pad[7];
+    int32_t tok0, tok1;            // the sequence's token range in the call
+    uint32_t pad[5];
 };
 static_assert(sizeof(AppendPlan) == 64, "plan record");
 
@@ -57,7 +59,9 @@ struct DevCache {
     uint32_t *seq_mark;              // [max_seqs] serial of the last append call that named the sequence
     uint32_t *low_vmax;              // [max_seqs][n_layers] largest V scale (fp16 bits) in the LOW stream
     AppendPlan *plan;                // [PASK_MAX_SEQS_PER_CALL]
-    uint2 *tok_scratch;              // [max_append_tokens] {action | stream position << 2, index in call}
+    uint32_t *tok_list;              // [max_append_tokens] bulk appends: each sequence's retained tokens in stream order
+                                     // (HIGH from the front of its token range, LOW from the back)
+    uint32_t *item_base;             // [PASK_MAX_SEQS_PER_CALL + 1] prefix over sequences of the pages a bulk append touches
     uint8_t *lut;                    // [n_tags][n_groups] effective action max(a0, floor)
     uint8_t *layer_group;            // [n_layers]
     // tables of the budget-dependent adjustment (pask_decide)
@@ -76,7 +80,7 @@ struct DevCache {
 };
 
 struct MetaOffsets {
-    size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, low_vmax, plan, tok_scratch, lut,
+    size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, low_vmax, plan, tok_list, item_base, lut,
         layer_group, dec_row, dec_rho, gamma, crit, total;
     size_t zero_begin, zero_end;     // the span cleared by a reset (counters, tables, budgets, marks)
 };
