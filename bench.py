@@ -407,14 +407,18 @@ def run_cuda(args, rank, world):
     }
     if len(job.fill_ms) > 1:
         f_ms = sum(job.fill_ms[1:]) / (len(job.fill_ms) - 1)
-        in_b = job.total_tokens * 2 * cfg.n_kv * 256                   # K and V read once, bf16
+        lg = w.policy.layer_group.astype(np.int64)
+        kept = sum(float((job.nh[:, lg[l]] + job.nl[:, lg[l]]).sum()) for l in range(cfg.n_layers)) / cfg.n_layers
+        in_b = kept * 2 * cfg.n_kv * 256 + job.total_tokens * 5        # K, V rows of retained tokens (bf16), tag + list word
         out_b = ret / cfg.n_layers                                     # payload written, per layer
         line["bulk_append"] = {"tokens_per_call": job.total_tokens, "ms_per_layer_call": f_ms,
                                "token_layers_per_s": job.total_tokens / (f_ms * 1e-3),
                                "achieved_gbs": (in_b + out_b) / (f_ms * 1e-3) / 1e9,
                                "frac_of_peak": (in_b + out_b) / (f_ms * 1e-3) / 1e9 / peak,
                                "algorithmic_bytes_per_call": in_b + out_b,
-                               "note": "one ragged pask_append_kv call per layer over the whole history (plan + write kernels)"}
+                               "retained_tokens_per_layer": kept,
+                               "note": "one ragged pask_append_kv call per layer over the whole history (plan + write "
+                                       "kernels); rows of dropped tokens are never read"}
     if args.dynamic:
         sts = [P.pask_budget_state(job.cache.handle, b) for b in range(job.B)]
         line["dynamic_budget"] = {"prefill_decide_ms": job.prefill_decide_ms, "prefill_tokens": job.total_tokens,

@@ -3,6 +3,7 @@
 //
 // Algorithm 2 of the paper, steps 1-2 (lookup, a = max(a0, floor)), 7 (persist) and 8 (budget
 // recurrence), applied to a ragged batch of tokens for one layer.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "pask_internal.h"
@@ -70,9 +71,9 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
                    const int32_t *__restrict__ cu_tokens, const uint8_t *__restrict__ tags,
                    const uint8_t *__restrict__ decided, uint8_t *__restrict__ actions_out, uint32_t serial) {
     __shared__ uint8_t s_lut[256];
-    __shared__ uint32_t s_wh[kPlanThreads / 32], s_wl[kPlanThreads / 32], s_wb[kPlanThreads / 32];
+    __shared__ uint32_t s_wh[2 * (kPlanThreads / 32)], s_wb[2 * (kPlanThreads / 32)];
     __shared__ uint32_t s_scan[kPlanThreads / 32];
-    __shared__ uint32_t s_run_h, s_run_l, s_run_b;
+    __shared__ uint32_t s_first_h[PASK_MAX_SEQS_PER_CALL], s_first_l[PASK_MAX_SEQS_PER_CALL];
     __shared__ int s_flag;
     const int i = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int group = c.layer_group[layer];
@@ -84,53 +85,71 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         err |= PASK_DEV_BAD_RAGGED;
     if (seq < 0 || seq >= c.max_seqs) err |= PASK_DEV_BAD_SEQ;
     if (tid == 0) {
-        s_run_h = s_run_l = s_run_b = 0;
         if (!(err & PASK_DEV_BAD_SEQ) && atomicExch(&c.seq_mark[seq], serial) == serial) s_flag = 1;  // named twice
         else s_flag = 0;
     }
     __syncthreads();
     if (s_flag) err |= PASK_DEV_BAD_SEQ;
 
+    // Four consecutive tokens per thread and round; counts of a round travel packed (HIGH in the low
+    // half-word, LOW in the high one; at most 1024 each), running totals stay in registers (every
+    // thread adds the same round totals), and the per-warp slots alternate between rounds, so a
+    // round costs one barrier.
     int bad_action = 0;
+    uint32_t run_h = 0, run_l = 0, run_b = 0;
     if (!err) {
-        for (int base = t0; base < t1; base += kPlanThreads) {
-            const int t = base + tid;
-            const bool valid = t < t1;
-            int a = 3;
-            bool bad = false;
-            if (valid) {
-                const int tag = tags[t];
-                a = s_lut[tag];
-                bad = tag != PASK_TAG_PROTECTED && tag >= c.n_tags;
-                if (decided) {   // Algorithm 2 step 7 on the actions pask_decide chose
-                    a = decided[(size_t)t * c.n_groups + group];
-                    if (a > PASK_ACTION_RETAIN_HIGH) { bad_action = 1; a = PASK_ACTION_RELEASE; }
+        int buf = 0;
+        for (int base = t0; base < t1; base += 4 * kPlanThreads, buf ^= 1) {
+            const int tb = base + 4 * tid;
+            int a[4];
+            uint32_t cnt = 0, nbad = 0;
+#pragma unroll
+            for (int e = 0; e < 4; e++) {
+                const int t = tb + e;
+                a[e] = 3;
+                if (t < t1) {
+                    const int tag = tags[t];
+                    a[e] = s_lut[tag];
+                    nbad += tag != PASK_TAG_PROTECTED && tag >= c.n_tags;
+                    if (decided) {   // Algorithm 2 step 7 on the actions pask_decide chose
+                        a[e] = decided[(size_t)t * c.n_groups + group];
+                        if (a[e] > PASK_ACTION_RETAIN_HIGH) { bad_action = 1; a[e] = PASK_ACTION_RELEASE; }
+                    }
                 }
+                cnt += (a[e] == PASK_ACTION_RETAIN_HIGH ? 1u : 0u) + (a[e] == PASK_ACTION_RETAIN_LOW ? 0x10000u : 0u);
             }
-            const uint32_t mh = __ballot_sync(0xffffffffu, a == PASK_ACTION_RETAIN_HIGH);
-            const uint32_t ml = __ballot_sync(0xffffffffu, a == PASK_ACTION_RETAIN_LOW);
-            const uint32_t mb = __ballot_sync(0xffffffffu, bad);
-            if (lane == 0) { s_wh[warp] = __popc(mh); s_wl[warp] = __popc(ml); s_wb[warp] = __popc(mb); }
+            uint32_t inc = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t o = __shfl_up_sync(0xffffffffu, inc, d);
+                if (lane >= d) inc += o;
+            }
+            nbad = __reduce_add_sync(0xffffffffu, nbad);
+            if (lane == 31) { s_wh[buf * (kPlanThreads / 32) + warp] = inc; s_wb[buf * (kPlanThreads / 32) + warp] = nbad; }
             __syncthreads();
-            uint32_t off_h = s_run_h, off_l = s_run_l, tot_h = 0, tot_l = 0, tot_b = 0;
+            uint32_t before = 0, tot = 0, tot_b = 0;
 #pragma unroll
             for (int w = 0; w < kPlanThreads / 32; w++) {
-                if (w < warp) { off_h += s_wh[w]; off_l += s_wl[w]; }
-                tot_h += s_wh[w]; tot_l += s_wl[w]; tot_b += s_wb[w];
+                const uint32_t x = s_wh[buf * (kPlanThreads / 32) + w];
+                if (w < warp) before += x;
+                tot += x;
+                tot_b += s_wb[buf * (kPlanThreads / 32) + w];
             }
-            if (valid) {
-                uint32_t pos = 0;
-                if (a == PASK_ACTION_RETAIN_HIGH) pos = off_h + __popc(mh & lanemask_lt());
-                else if (a == PASK_ACTION_RETAIN_LOW) pos = off_l + __popc(ml & lanemask_lt());
+            const uint32_t excl = before + inc - cnt;
+            uint32_t pos_h = run_h + (excl & 0xffffu), pos_l = run_l + (excl >> 16);
+#pragma unroll
+            for (int e = 0; e < 4; e++) {
+                const int t = tb + e;
+                if (t >= t1) break;
                 // stream-ordered token lists for the write kernel: HIGH from the front of the
                 // sequence's token range, LOW from its back
-                if (a == PASK_ACTION_RETAIN_HIGH) c.tok_list[t0 + pos] = (uint32_t)t;
-                else if (a == PASK_ACTION_RETAIN_LOW) c.tok_list[t1 - 1 - pos] = (uint32_t)t;
-                if (actions_out) actions_out[t] = (uint8_t)a;
+                if (a[e] == PASK_ACTION_RETAIN_HIGH) c.tok_list[t0 + pos_h++] = (uint32_t)t;
+                else if (a[e] == PASK_ACTION_RETAIN_LOW) c.tok_list[t1 - 1 - pos_l++] = (uint32_t)t;
+                if (actions_out) actions_out[t] = (uint8_t)a[e];
             }
-            __syncthreads();
-            if (tid == 0) { s_run_h += tot_h; s_run_l += tot_l; s_run_b += tot_b; }
-            __syncthreads();
+            run_h += tot & 0xffffu;
+            run_l += tot >> 16;
+            run_b += tot_b;
         }
     }
 
@@ -142,10 +161,10 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
             const size_t sl = (size_t)seq * c.n_layers + layer;
             p.old_high = c.n_high[sl];
             p.old_low = c.n_low[sl];
-            p.cnt_high = s_run_h;
-            p.cnt_low = s_run_l;
-            p.cnt_drop = (uint32_t)(t1 - t0) - s_run_h - s_run_l;
-            p.bad_tags = s_run_b;
+            p.cnt_high = run_h;
+            p.cnt_low = run_l;
+            p.cnt_drop = (uint32_t)(t1 - t0) - run_h - run_l;
+            p.bad_tags = run_b;
             const uint32_t ph0 = (p.old_high + kPageTokens - 1) / kPageTokens, ph1 = (p.old_high + p.cnt_high + kPageTokens - 1) / kPageTokens;
             const uint32_t pl0 = (p.old_low + kPageTokens - 1) / kPageTokens, pl1 = (p.old_low + p.cnt_low + kPageTokens - 1) / kPageTokens;
             p.new_pages_high = ph1 - ph0;
@@ -207,15 +226,8 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         if (j >= n_seqs) break;
         const AppendPlan p = load_plan_cg(&c.plan[j]);
         const size_t sl = (size_t)p.seq * c.n_layers + layer;
-        const uint32_t ph0 = (p.old_high + kPageTokens - 1) / kPageTokens, pl0 = (p.old_low + kPageTokens - 1) / kPageTokens;
-        for (uint32_t x = 0; x < nh[r]; x++) {
-            const uint32_t kk = base_h + x;
-            c.tbl_high[sl * c.max_pages + ph0 + x] = kk < free_h ? c.free_high[free_h - 1 - kk] : next_h + (kk - free_h);
-        }
-        for (uint32_t x = 0; x < nl[r]; x++) {
-            const uint32_t kk = base_l + x;
-            c.tbl_low[sl * c.max_pages + pl0 + x] = kk < free_l ? c.free_low[free_l - 1 - kk] : next_l + (kk - free_l);
-        }
+        s_first_h[j] = base_h;                     // where this sequence's new pages start in the call's numbering
+        s_first_l[j] = base_l;
         base_h += nh[r];
         base_l += nl[r];
         c.item_base[j] = base_i;
@@ -234,6 +246,22 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         b.pages_high += nh[r];
         b.pages_low += nl[r];
     }
+    // page tables: a warp per sequence, its lanes over the sequence's new pages (a prefill hands
+    // out hundreds of pages per sequence)
+    __syncthreads();
+    for (int j = warp; j < n_seqs; j += kPlanThreads / 32) {
+        const AppendPlan p = load_plan_cg(&c.plan[j]);
+        const size_t sl = (size_t)p.seq * c.n_layers + layer;
+        const uint32_t ph0 = (p.old_high + kPageTokens - 1) / kPageTokens, pl0 = (p.old_low + kPageTokens - 1) / kPageTokens;
+        for (uint32_t x = lane; x < p.new_pages_high; x += 32) {
+            const uint32_t kk = s_first_h[j] + x;
+            c.tbl_high[sl * c.max_pages + ph0 + x] = kk < free_h ? c.free_high[free_h - 1 - kk] : next_h + (kk - free_h);
+        }
+        for (uint32_t x = lane; x < p.new_pages_low; x += 32) {
+            const uint32_t kk = s_first_l[j] + x;
+            c.tbl_low[sl * c.max_pages + pl0 + x] = kk < free_l ? c.free_low[free_l - 1 - kk] : next_l + (kk - free_l);
+        }
+    }
     if (tid == 0) {
         const uint32_t pop_h = need_h < free_h ? need_h : free_h, pop_l = need_l < free_l ? need_l : free_l;
         c.ctrl[kCtrlHighFree] = free_h - pop_h;
@@ -245,6 +273,11 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         c.ctrl[kCtrlPlanOk] = 1;
         c.ctrl[kCtrlTicket] = 0;
     }
+}
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
 }
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -329,36 +362,47 @@ __device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uin
 constexpr int kWriteThreads = 256;
 constexpr int kRowBytes = 2 * kHeadDim + 16;      // one token's K (or V) row of a head in shared memory, padded
 
-__global__ void __launch_bounds__(kWriteThreads, 4)
+__global__ void __launch_bounds__(kWriteThreads, 3)
 append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__ k, const uint4 *__restrict__ v) {
-    __shared__ uint32_t s_base[PASK_MAX_SEQS_PER_CALL + 1];
-    __shared__ __align__(16) uint8_t s_in[2][kPageTokens][kRowBytes];   // [K|V][token][dims of one head]
-    __shared__ __align__(16) uint8_t s_low[kLowHeadBytes];              // one head of a LOW page, packed
+    extern __shared__ __align__(16) uint8_t s_dyn[];                    // the page's source rows, see in_row()
+    __shared__ __align__(16) uint8_t s_low[2][kLowHeadBytes];           // one head of a LOW page, packed (two in turn)
     __shared__ uint32_t s_tok[kPageTokens];
+    // source rows of the page being written: [head][K|V][token][kRowBytes]
+    auto in_row = [&](int head, int which, int tau) -> uint8_t * {
+        return s_dyn + (size_t)((head * 2 + which) * kPageTokens + tau) * kRowBytes;
+    };
     if (c.ctrl[kCtrlPlanOk] == 0) return;
     const int tid = threadIdx.x;
     const uint32_t n_items = c.ctrl[kCtrlItems];
     const uint32_t item0 = (uint32_t)(((uint64_t)n_items * blockIdx.x) / gridDim.x);
     const uint32_t item1 = (uint32_t)(((uint64_t)n_items * (blockIdx.x + 1)) / gridDim.x);
     if (item0 >= item1) return;
-    for (int x = tid; x <= n_seqs; x += kWriteThreads) s_base[x] = c.item_base[x];
-    __syncthreads();
-    int j = 0;                                     // the sequence item0 belongs to: s_base[j] <= item0 < s_base[j + 1]
+    // find the sequence item0 belongs to (base[j] <= item0 < base[j + 1]) with the prefix table staged
+    // in the row buffer, which is free until the first page is fetched
+    int j = 0;
+    uint32_t base_j, base_next;
     {
+        uint32_t *s_base = reinterpret_cast<uint32_t *>(s_dyn);
+        for (int x = tid; x <= n_seqs; x += kWriteThreads) s_base[x] = c.item_base[x];
+        __syncthreads();
         int lo = 0, hi = n_seqs - 1;
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
             if (s_base[mid] <= item0) lo = mid; else hi = mid - 1;
         }
         j = lo;
+        base_j = s_base[j];
+        base_next = s_base[j + 1];
+        __syncthreads();
     }
-    const int chunks = 16 * c.n_kv;                // 16-byte chunks per token per tensor
+    const int chunks = 16 * c.n_kv;                // 16-byte chunks per token per tensor (a power of two)
+    const int chunks_shift = 31 - __clz(chunks);
     AppendPlan p = c.plan[j];
     for (uint32_t item = item0; item < item1; item++) {
         bool moved = false;
-        while (item >= s_base[j + 1]) { j++; moved = true; }
+        while (item >= base_next) { j++; base_j = base_next; base_next = c.item_base[j + 1]; moved = true; }
         if (moved) p = c.plan[j];
-        const uint32_t in_seq = item - s_base[j];
+        const uint32_t in_seq = item - base_j;
         const uint32_t items_h = pages_touched(p.old_high, p.cnt_high);
         const bool high = in_seq < items_h;
         const uint32_t old = high ? p.old_high : p.old_low, cnt = high ? p.cnt_high : p.cnt_low;
@@ -385,80 +429,69 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
             }
             continue;
         }
-        // ---- a full page: per head, 16 rows of K and of V in, one packed block out
-        uint4 nx[2];
-#pragma unroll
-        for (int r = 0; r < 2; r++) {              // rows of head 0: chunk idx = which * 256 + token * 16 + chunk
-            const int idx = tid + r * kWriteThreads, which = idx >> 8, tau = (idx >> 4) & 15, ch = idx & 15;
-            nx[r] = (which ? v : k)[(size_t)s_tok[tau] * chunks + ch];
+        // ---- a full page: all 16 tokens' rows (every head, K and V) go to shared memory with
+        // asynchronous 16-byte copies, all in flight at once; then each head leaves as one packed block
+        {
+            const int per_tensor = kPageTokens * chunks;        // 16-byte chunks of K (or of V) in the page
+            for (int idx = tid; idx < 2 * per_tensor; idx += kWriteThreads) {
+                const int which = idx >= per_tensor, rem = which ? idx - per_tensor : idx;
+                const int tau = rem >> chunks_shift, cc = rem & (chunks - 1);      // consecutive threads: consecutive bytes of a row
+                cp_async16(in_row(cc >> 4, which, tau) + (cc & 15) * 16, (which ? v : k) + (size_t)s_tok[tau] * chunks + cc);
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
+        __syncthreads();
         uint32_t vmax_bits = 0;
         for (int head = 0; head < c.n_kv; head++) {
-            __syncthreads();                       // readers of the previous head's rows (and of s_low) are done
-#pragma unroll
-            for (int r = 0; r < 2; r++) {
-                const int idx = tid + r * kWriteThreads, which = idx >> 8, tau = (idx >> 4) & 15, ch = idx & 15;
-                *reinterpret_cast<uint4 *>(&s_in[which][tau][ch * 16]) = nx[r];
-            }
-            if (head + 1 < c.n_kv) {
-#pragma unroll
-                for (int r = 0; r < 2; r++) {
-                    const int idx = tid + r * kWriteThreads, which = idx >> 8, tau = (idx >> 4) & 15, ch = idx & 15;
-                    nx[r] = (which ? v : k)[(size_t)s_tok[tau] * chunks + (head + 1) * 16 + ch];
-                }
-            }
-            __syncthreads();
             if (high) {
                 uint4 *dst = reinterpret_cast<uint4 *>(c.pool_high + (size_t)page * c.high_page_bytes + (size_t)head * kHighHeadBytes);
                 const int lane = tid & 31, g = lane >> 2, t = lane & 3, i = tid >> 5;
                 {   // K tile, round i = 2 jj + hh: the operand quad of lane (g, t), see pask_layout.h
                     const int jj = i >> 1, hh = i & 1, off = 2 * (8 * (4 * jj + t) + 4 * hh);
                     uint4 q;
-                    q.x = *reinterpret_cast<const uint32_t *>(&s_in[0][g][off]);
-                    q.y = *reinterpret_cast<const uint32_t *>(&s_in[0][g + 8][off]);
-                    q.z = *reinterpret_cast<const uint32_t *>(&s_in[0][g][off + 4]);
-                    q.w = *reinterpret_cast<const uint32_t *>(&s_in[0][g + 8][off + 4]);
+                    q.x = *reinterpret_cast<const uint32_t *>(in_row(head, 0, g) + off);
+                    q.y = *reinterpret_cast<const uint32_t *>(in_row(head, 0, g + 8) + off);
+                    q.z = *reinterpret_cast<const uint32_t *>(in_row(head, 0, g) + off + 4);
+                    q.w = *reinterpret_cast<const uint32_t *>(in_row(head, 0, g + 8) + off + 4);
                     dst[tid] = q;
                 }
                 {   // V tile, round i = 4 e + kk: token {2t, 2t+1, 2t+8, 2t+9}[kk], dims 64e + 4g.. and 64e + 32 + 4g..
                     const int e = i >> 2, kk = i & 3, tau = 2 * t + (kk & 1) + 8 * (kk >> 1);
-                    const uint2 a = *reinterpret_cast<const uint2 *>(&s_in[1][tau][128 * e + 8 * g]);
-                    const uint2 b = *reinterpret_cast<const uint2 *>(&s_in[1][tau][128 * e + 64 + 8 * g]);
+                    const uint2 a = *reinterpret_cast<const uint2 *>(in_row(head, 1, tau) + 128 * e + 8 * g);
+                    const uint2 b = *reinterpret_cast<const uint2 *>(in_row(head, 1, tau) + 128 * e + 64 + 8 * g);
                     dst[256 + tid] = make_uint4(a.x, a.y, b.x, b.y);
                 }
             } else {
                 // thread = (K|V, token, 32-dim group, half of it): 16 values
                 const int half = tid & 1, w = (tid >> 1) & 3, tau = (tid >> 3) & 15, which = tid >> 7;
-                const uint4 x0 = *reinterpret_cast<const uint4 *>(&s_in[which][tau][64 * w + 32 * half]);
-                const uint4 x1 = *reinterpret_cast<const uint4 *>(&s_in[which][tau][64 * w + 32 * half + 16]);
+                const uint4 x0 = *reinterpret_cast<const uint4 *>(in_row(head, which, tau) + 64 * w + 32 * half);
+                const uint4 x1 = *reinterpret_cast<const uint4 *>(in_row(head, which, tau) + 64 * w + 32 * half + 16);
                 const uint32_t xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-                float f[16];
-                float amax = 0.0f;
+                // amax on the packed bf16 pairs (abs and max are exact in any format)
+                __nv_bfloat162 m2 = __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&xs[0]));
 #pragma unroll
-                for (int e = 0; e < 8; e++) {
-                    f[2 * e] = bf16_lo(xs[e]);
-                    f[2 * e + 1] = bf16_hi(xs[e]);
-                    amax = fmaxf(amax, fmaxf(fabsf(f[2 * e]), fabsf(f[2 * e + 1])));
-                }
+                for (int e = 1; e < 8; e++) m2 = __hmax2(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&xs[e])));
+                const uint32_t m2b = *reinterpret_cast<const uint32_t *>(&m2);
+                float amax = fmaxf(bf16_lo(m2b), bf16_hi(m2b));
                 amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
                 const float s32 = __fdiv_rn(amax, 7.0f);
                 __half sh = __float2half_rn(s32);
                 if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);   // saturate, never infinite
                 const float sc = __half2float(sh);
+                // code = clamp(rint(x * (1/s)), -7, 7) + 8.  Clamping first gives the same integer
+                // (the bounds are integers), and adding 1.5 * 2^23 + 8 to a value in [-7, 7] rounds it
+                // to the nearest integer, ties to even, leaving code in the low 4 bits of the sum.
+                // s == 0 means every value is zero: 1/s is replaced by 0 and all codes come out 8.
+                const float inv = sc == 0.0f ? 0.0f : __fdiv_rn(1.0f, sc);
                 uint32_t code[16];
-                if (sc == 0.0f) {
 #pragma unroll
-                    for (int e = 0; e < 16; e++) code[e] = 8u;
-                } else {
-                    const float inv = __fdiv_rn(1.0f, sc);
-#pragma unroll
-                    for (int e = 0; e < 16; e++) {
-                        float r = rintf(__fmul_rn(f[e], inv));
-                        r = fminf(fmaxf(r, -7.0f), 7.0f);
-                        code[e] = (uint32_t)((int)r + 8);
-                    }
+                for (int e = 0; e < 16; e++) {
+                    const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
+                    const float cl = fminf(fmaxf(__fmul_rn(f, inv), -7.0f), 7.0f);
+                    code[e] = __float_as_uint(__fadd_rn(cl, 12582920.0f)) & 15u;
                 }
-                uint8_t *img = s_low + (which ? kLowHalfBytes : 0);
+                uint8_t *img = s_low[head & 1] + (which ? kLowHalfBytes : 0);
                 if (!which) {
 #pragma unroll
                     for (int u = 0; u < 2; u++) {  // the words of dims 32w + 8t .. +7, t = 2 half + u
@@ -478,7 +511,7 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
                 if (half == 0) *reinterpret_cast<__half *>(img + low_scale_off(tau, w)) = sh;
                 __syncthreads();
                 uint4 *dst = reinterpret_cast<uint4 *>(c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLowHeadBytes);
-                if (tid < kLowHeadBytes / 16) dst[tid] = reinterpret_cast<const uint4 *>(s_low)[tid];
+                if (tid < kLowHeadBytes / 16) dst[tid] = reinterpret_cast<const uint4 *>(s_low[head & 1])[tid];
             }
         }
         if (!high) {   // largest V scale of the stream (decode attention forms P * scale relative to it)
@@ -727,9 +760,12 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
     if (total_tokens > 0) {
         // at most one item per 16 tokens plus two partly filled pages per stream
         const long long bound = (long long)total_tokens / 16 + 4LL * n_seqs;
-        const int ctas = bound < (long long)c->sm_count * 4 ? (int)bound : c->sm_count * 4;
-        append_write_kernel<<<ctas, kWriteThreads, 0, stream>>>(c->dev, layer, n_seqs, static_cast<const uint4 *>(k),
-                                                               static_cast<const uint4 *>(v));
+        const int ctas = bound < (long long)c->sm_count * 3 ? (int)bound : c->sm_count * 3;
+        const size_t smem = (size_t)c->desc.n_kv_heads * 2 * kPageTokens * kRowBytes;
+        if (cudaFuncSetAttribute(append_write_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return PASK_ERR_CUDA;
+        append_write_kernel<<<ctas, kWriteThreads, smem, stream>>>(c->dev, layer, n_seqs, static_cast<const uint4 *>(k),
+                                                                  static_cast<const uint4 *>(v));
     }
     return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }
