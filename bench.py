@@ -264,6 +264,21 @@ class Job:
                                                           np.int16)).to(d) for s in range(n_steps)]
             self.decided = torch.empty((self.B, cfg.n_groups), dtype=torch.uint8, device=d)
 
+    def capture_steps(self, first, n_steps):
+        """One CUDA graph per step (its inputs are fixed buffers): the step's launches are then
+        issued by a single graph launch."""
+        self.graphs = {}
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for s in range(first, first + n_steps):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    self.run_step(s)
+                self.graphs[s] = g
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+
     def run_step(self, s, events=None):
         """events: {layer: (start, stop)} for the launches of this step whose streaming kernel is timed."""
         P, h = self.P, self.cache.handle
@@ -331,7 +346,10 @@ def run_cuda(args, rank, world):
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0.record()
         for i in range(n_steps):
-            jb.run_step(first_step + i, evs[i] if evs else None)
+            if args.graph and jb is job:
+                jb.graphs[first_step + i].replay()
+            else:
+                jb.run_step(first_step + i, evs[i] if evs else None)
         t1.record()
         barrier()
         ms = t0.elapsed_time(t1)
@@ -340,10 +358,12 @@ def run_cuda(args, rank, world):
 
     for i in range(args.warmup):
         job.run_step(i)
+    if args.graph:
+        job.capture_steps(args.warmup, args.steps)
     sampler = ClockSampler(device.index or 0)
     if rank == 0:
         sampler.start()
-    ms, kern_ms = timed(job, args.warmup, args.steps, True)
+    ms, kern_ms = timed(job, args.warmup, args.steps, not args.graph)
     clocks = sampler.stop() if rank == 0 else {}
     ms = max_over_ranks(ms, device)
     st = P.pask_budget_state(job.cache.handle, 0)
@@ -383,6 +403,8 @@ def run_cuda(args, rank, world):
         return
     peak, peak_kind = measured_peaks()
     alg = job.algorithmic_bytes_per_layer(args.warmup + args.steps // 2)
+    if not kern_ms:      # graph replay carries no per-kernel events: the kernel figures come from a plain run
+        kern_ms = [float("inf")]
     k_ms = sum(kern_ms) / len(kern_ms)
     achieved = alg / (k_ms * 1e-3) / 1e9
     line = {
@@ -405,6 +427,10 @@ def run_cuda(args, rank, world):
         "attention_share_of_step": k_ms * cfg.n_layers * args.steps / ms,
         "attention_only_tokens_per_s": world * job.B / (k_ms * 1e-3 * cfg.n_layers),
     }
+    if args.graph:
+        line["config"]["launch"] = "one CUDA graph per step"
+        line["roofline"] = None
+        line["attention_share_of_step"] = line["attention_only_tokens_per_s"] = None
     if len(job.fill_ms) > 1:
         f_ms = sum(job.fill_ms[1:]) / (len(job.fill_ms) - 1)
         lg = w.policy.layer_group.astype(np.int64)
@@ -445,6 +471,8 @@ def run_full_kv(P, args, w, device, total_steps, peak):
     job.prepare_steps(total_steps)
     for i in range(args.warmup):
         job.run_step(i)
+    if args.graph:
+        job.capture_steps(args.warmup, args.steps)
     evs = kernel_events(cfg.n_layers, args.steps, args.event_stride)
     torch.cuda.synchronize()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -555,6 +583,7 @@ def main():
     ap.add_argument("--no-full-kv", dest="full_kv", action="store_false")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="0 skips the CPU-oracle leg")
     ap.add_argument("--event-stride", type=int, default=4, help="time the streaming kernel of every n-th launch")
+    ap.add_argument("--graph", action="store_true", help="replay each timed step as one CUDA graph (launch-bound shapes)")
     ap.add_argument("--dynamic", action="store_true",
                     help="decide every token against the running budget (pask_decide) instead of the frozen table alone")
     ap.add_argument("--layers", type=int, default=None, help="profiling aid: keep only the first N layers")

@@ -53,9 +53,16 @@ QWEN3_8B_LONG = Config("qwen3-8b-36layer-b128-16k-mix", 3, n_layers=36, n_groups
 QWEN3_4B_SWEEP = Config("qwen3-4b-36layer-b64-8k-sweep", 4, n_layers=36, n_groups=4, n_q=32, n_kv=8,
                         batch=64, prompt_len=4096, gen_len=4096)
 SWEEP_BUDGETS = (0.2, 0.33, 0.5, 0.75, 1.0)
+# The shapes of the paper's latency table (Table 3): concurrency 8, 8K or 32K input tokens and
+# 256 / 1024 / 2048 generated ones (here: the state after 1024 generated tokens).  Small batch, long
+# context: few bytes per launch at 8K, deep splits at 32K.
+TABLE3_8K = Config("qwen3-4b-36layer-c8-8k-in-1k-out", 5, n_layers=36, n_groups=4, n_q=32, n_kv=8, batch=8,
+                   prompt_len=8192, gen_len=1024)
+TABLE3_32K = Config("qwen3-4b-36layer-c8-32k-in-1k-out", 6, n_layers=36, n_groups=4, n_q=32, n_kv=8, batch=8,
+                    prompt_len=32768, gen_len=1024)
 
 # The one-layer configuration is run once per layer-group column: four layers, one per group.
-CONFIGS = [TINY, QWEN3_4B_1LAYER, QWEN3_4B_STEP, QWEN3_8B_LONG, QWEN3_4B_SWEEP]
+CONFIGS = [TINY, QWEN3_4B_1LAYER, QWEN3_4B_STEP, QWEN3_8B_LONG, QWEN3_4B_SWEEP, TABLE3_8K, TABLE3_32K]
 
 
 def scaled(cfg: Config, **kw) -> Config:
