@@ -17,6 +17,8 @@
  *     it): B = [R - Gamma(s)]+, demotions above the floors in ascending upgrade score while the
  *     token's cost exceeds B, promotions in descending score in critical states while they fit,
  *     floors first when budget and protection conflict (orc_decide);
+ *   - the protected recent window (Section 3.1): release and the low format take effect on a state
+ *     only after it has left the window, so the last W tokens are attended at full precision;
  *   - normalised cost C_KV = sum m(a) / sum m(H) (Eq. 1);
  *   - the reference policy is full high precision (Section 3.1), whose attention outputs are the
  *     ones Eq. 4 compares against: plain softmax(q k^T / sqrt(d)) v over the retained history.
@@ -26,8 +28,10 @@
  * per group of 32 consecutive head dimensions with one fp16 scale (amax/7, round to nearest
  * even, codes stored offset by 8); RETAIN-HIGH keeps the bf16 bits; pages hold 16 tokens and
  * are handed out in call order from a per-pool free stack, else a bump counter; costs are
- * payload bytes.  Parity unpinned by the paper for: the low-bit format itself, the absence of a
- * recent window, the initial budget, and the treatment of prompt tags -- those are pinned only
+ * payload bytes.  Parity unpinned by the paper for: the low-bit format itself, the size of the
+ * recent window (a policy parameter here, 0 by default; the paper gives no number) and that a
+ * token is charged m(a) when it arrives rather than when it leaves the window, the initial
+ * budget, and the treatment of prompt tags -- those are pinned only
  * by this library's own documentation.  The paper gives Demote, Promote and Crit in one sentence
  * each and R's starting value not at all: the reading written out above decide_token (budget
  * accrued per token seen, one step at a time, ties to the first group, "eligible" = fits in B)
@@ -52,6 +56,7 @@
 #define QGROUP 32
 #define GROUPS_PER_HEAD (HEAD_DIM / QGROUP)
 #define MAX_GROUPS 8
+#define MAX_WINDOW 256
 #define TAG_PROTECTED 0xFF
 
 enum { ACT_R = 0, ACT_L = 1, ACT_H = 2 };
@@ -87,6 +92,11 @@ typedef struct {          /* one (sequence, layer) pair: two compacted streams *
     uint16_t *lks, *lvs;  /* [n_low][n_kv][4] fp16 scale bit patterns */
     uint32_t *pg_high, *pg_low; /* page ids, one per started 16-token page */
     uint32_t npg_high, npg_low, cap_pg_high, cap_pg_low;
+    /* protected recent window (W = policy recent_window > 0): the last W tokens of this
+     * (sequence, layer), whatever their action, as bf16 bits; token t sits in slot t mod W */
+    uint32_t n_tok;       /* tokens appended so far, released ones included */
+    uint16_t *wk, *wv;    /* [W][n_kv][128] */
+    uint8_t *wact;        /* [W] the action each of them took */
 } orc_stream;
 
 typedef struct {
@@ -204,7 +214,7 @@ orc_policy *orc_policy_load(const uint8_t *blob, size_t len, int *err) {
     p->n_states = rd32(blob + 20); p->budget_q16 = rd32(blob + 24); p->recent_window = rd32(blob + 28);
     p->low_bits = rd32(blob + 32); p->group_size = rd32(blob + 36);
     if (p->n_tags == 0 || p->n_tags > 255 || p->n_groups == 0 || p->n_groups > MAX_GROUPS ||
-        p->n_layers == 0 || p->n_layers > 4096 || p->n_states > (1u << 20) || p->recent_window != 0 ||
+        p->n_layers == 0 || p->n_layers > 4096 || p->n_states > (1u << 20) || p->recent_window % PAGE_TOKENS != 0 || p->recent_window > MAX_WINDOW ||
         p->low_bits != 4 || p->group_size != QGROUP) { free(p); return NULL; }
     size_t lg_pad = (p->n_layers + 3u) & ~(size_t)3u;
     size_t n_ent = (size_t)p->n_tags * p->n_groups;
@@ -266,7 +276,7 @@ orc_cache *orc_cache_create(const orc_policy *pol, int n_q, int n_kv, int max_se
 
 static void stream_free(orc_stream *s) {
     free(s->hk); free(s->hv); free(s->lk); free(s->lv); free(s->lks); free(s->lvs);
-    free(s->pg_high); free(s->pg_low);
+    free(s->pg_high); free(s->pg_low); free(s->wk); free(s->wv); free(s->wact);
     memset(s, 0, sizeof(*s));
 }
 
@@ -352,6 +362,17 @@ int orc_append_decided(orc_cache *c, int layer, int n_seqs, const int32_t *seq_i
             b->bad_tags += (uint64_t)bad;
             b->n_seen[group]++;
             b->full_bytes += bytes_high(c);
+            if (p->recent_window) {   /* every token, released ones too, enters the recent window */
+                const uint32_t W = p->recent_window, slot = s->n_tok % W;
+                if (!s->wk) {
+                    s->wk = (uint16_t *)malloc((size_t)W * row * 2); s->wv = (uint16_t *)malloc((size_t)W * row * 2);
+                    s->wact = (uint8_t *)malloc(W);
+                }
+                memcpy(s->wk + (size_t)slot * row, k_bits + (size_t)t * row, row * 2);
+                memcpy(s->wv + (size_t)slot * row, v_bits + (size_t)t * row, row * 2);
+                s->wact[slot] = (uint8_t)a;
+            }
+            s->n_tok++;
             if (a == ACT_R) { b->n_drop[group]++; continue; }
             if (a == ACT_H) {
                 uint32_t pos = s->n_high;
@@ -565,12 +586,22 @@ void orc_pool_state(orc_cache *c, uint32_t *high_next, uint32_t *high_free, uint
 
 /* One query head: softmax(q k^T / sqrt(d)) v over every retained token of (seq, layer), fp64.
  * q_bits [128] bf16 bit patterns of head h; out [128]; *lse natural log of the softmax denominator
- * (times e^max).  Nothing retained: out = 0, lse = -inf. */
+ * (times e^max).  Nothing retained: out = 0, lse = -inf.
+ * With a protected recent window W > 0 (Section 3.1: release and the low format apply to a state
+ * only once it has left the window) the last min(W, tokens seen) tokens are attended with their
+ * original bf16 values whatever their action; only older tokens are attended as stored.  Both
+ * streams are in arrival order, so the window's high- and low-precision members are exactly the
+ * last entries of the HIGH and of the LOW stream: those are skipped there. */
 static void attention_head(orc_cache *c, int layer, int seq, int h, const uint16_t *q_bits, double *out, double *lse) {
     orc_stream *s = stream_of(c, seq, layer);
     const int kv = h / (c->n_q / c->n_kv);
     const size_t row = (size_t)c->n_kv * HEAD_DIM, srow = (size_t)c->n_kv * GROUPS_PER_HEAD;
-    const size_t n = (size_t)s->n_high + s->n_low;
+    const uint32_t W = c->pol->recent_window;
+    const size_t nw = W ? (s->n_tok < W ? s->n_tok : W) : 0;          /* tokens in the window */
+    size_t win_h = 0, win_l = 0;
+    for (size_t i = 0; i < nw; i++) { win_h += s->wact[i] == ACT_H; win_l += s->wact[i] == ACT_L; }
+    const size_t nh = s->n_high - win_h, nl = s->n_low - win_l;        /* older than the window */
+    const size_t n = nh + nl + nw;
     const double inv_sqrt_d = 1.0 / sqrt((double)HEAD_DIM);
     double *score = (double *)malloc((n ? n : 1) * sizeof(double));
     double q[HEAD_DIM];
@@ -578,11 +609,14 @@ static void attention_head(orc_cache *c, int layer, int seq, int h, const uint16
     double m = -INFINITY;
     for (size_t j = 0; j < n; j++) {
         double dot = 0.0;
-        if (j < s->n_high) {
+        if (j < nh) {
             const uint16_t *k = s->hk + j * row + (size_t)kv * HEAD_DIM;
             for (int i = 0; i < HEAD_DIM; i++) dot += q[i] * (double)bf16_to_f32(k[i]);
+        } else if (j >= nh + nl) {
+            const uint16_t *k = s->wk + (j - nh - nl) * row + (size_t)kv * HEAD_DIM;
+            for (int i = 0; i < HEAD_DIM; i++) dot += q[i] * (double)bf16_to_f32(k[i]);
         } else {
-            size_t jl = j - s->n_high;
+            size_t jl = j - nh;
             const uint8_t *kc = s->lk + jl * row + (size_t)kv * HEAD_DIM;
             const uint16_t *ks = s->lks + jl * srow + (size_t)kv * GROUPS_PER_HEAD;
             for (int i = 0; i < HEAD_DIM; i++)
@@ -597,11 +631,14 @@ static void attention_head(orc_cache *c, int layer, int seq, int h, const uint16
     for (size_t j = 0; j < n; j++) {
         double pj = exp(score[j] - m);
         denom += pj;
-        if (j < s->n_high) {
+        if (j < nh) {
             const uint16_t *v = s->hv + j * row + (size_t)kv * HEAD_DIM;
             for (int i = 0; i < HEAD_DIM; i++) acc[i] += pj * (double)bf16_to_f32(v[i]);
+        } else if (j >= nh + nl) {
+            const uint16_t *v = s->wv + (j - nh - nl) * row + (size_t)kv * HEAD_DIM;
+            for (int i = 0; i < HEAD_DIM; i++) acc[i] += pj * (double)bf16_to_f32(v[i]);
         } else {
-            size_t jl = j - s->n_high;
+            size_t jl = j - nh;
             const uint8_t *vc = s->lv + jl * row + (size_t)kv * HEAD_DIM;
             const uint16_t *vs = s->lvs + jl * srow + (size_t)kv * GROUPS_PER_HEAD;
             for (int i = 0; i < HEAD_DIM; i++)
