@@ -70,6 +70,7 @@ typedef int32_t pask_status_t;
 #define PASK_TAG_PROTECTED 0xFF /* always RETAIN-HIGH, not counted as unknown */
 #define PASK_MAX_GROUPS 8
 #define PASK_MAX_SEQS_PER_CALL 1024
+#define PASK_MAX_WINDOW 256
 
 typedef struct pask_policy pask_policy_t;
 typedef struct pask_cache pask_cache_t;
@@ -87,10 +88,12 @@ typedef struct {
     int32_t max_append_tokens;  /* largest total_tokens of one pask_append_kv call */
     uint32_t pool_high_pages;   /* capacity of the bf16 page pool, shared by all layers */
     uint32_t pool_low_pages;    /* capacity of the int4 page pool */
+    int32_t recent_window;      /* the policy's protected recent window W (0, or a multiple of 16 up to
+                                   PASK_MAX_WINDOW); sizes W/16 bf16 pages per (sequence, layer) behind the bf16 pool */
 } pask_cache_desc_t;
 
 typedef struct {
-    size_t pool_high_bytes; /* pool_high_pages * high_page_bytes */
+    size_t pool_high_bytes; /* (pool_high_pages + max_seqs * n_layers * recent_window / 16) * high_page_bytes */
     size_t pool_low_bytes;
     size_t meta_bytes;      /* counters, page tables, budget states, free stacks, append scratch */
     size_t high_page_bytes; /* n_kv * 8192: per KV head a 16x128 bf16 K tile then V tile */
@@ -132,7 +135,8 @@ typedef struct {
  * pask_decide only.
  *   blob (host, len bytes), little endian:
  *     "PASK", u32 version (1 or 2), u32 n_tags (1..255), u32 n_groups (1..8), u32 n_layers,
- *     u32 n_states, u32 budget_target_q16, u32 recent_window (must be 0), u32 low_bits (4),
+ *     u32 n_states, u32 budget_target_q16, u32 recent_window (0, or a multiple of 16 up to
+ *     PASK_MAX_WINDOW: the protected recent window in tokens, see pask_decode_attention), u32 low_bits (4),
  *     u32 group_size (32),
  *     u8 layer_group[n_layers] zero-padded to 4 bytes,
  *     n_tags*n_groups entries, tag-major: u8 a0, u8 a_floor, u16 0, f32 rho_RL, f32 rho_LH
@@ -154,7 +158,7 @@ pask_status_t pask_cache_sizes(const pask_cache_desc_t *desc, pask_cache_sizes_t
 
 /* Bind caller-owned device memory (sizes from pask_cache_sizes) to a new cache and initialise
  * it on `stream` (copies the folded table into meta, zeroes counters).  The policy's n_layers
- * must equal desc->n_layers.  The handle is host memory; destroy frees only that. */
+ * and recent_window must equal desc's.  The handle is host memory; destroy frees only that. */
 pask_status_t pask_cache_create(const pask_cache_desc_t *desc, const pask_policy_t *policy, void *pool_high_dev,
                                 void *pool_low_dev, void *meta_dev, pask_stream_t stream, pask_cache_t **out);
 void pask_cache_destroy(pask_cache_t *cache);
@@ -236,6 +240,12 @@ pask_status_t pask_append_kv_decided(pask_cache_t *cache, int32_t layer, int32_t
  * the HIGH stream (bf16 values) and the LOW stream ((code - 8) * scale); released tokens take no
  * part (Section 3.1: release removes a KV state from future attention; these are the attention
  * outputs o of Eq. 4).  Query head h reads KV head h / 4.
+ * Protected recent window (Section 3.1: release and the low format apply to a state only after it
+ * has left the window): with recent_window = W > 0 the last min(W, tokens appended) tokens of the
+ * sequence at this layer are attended with their original bf16 K/V whatever their action; only
+ * older tokens are attended as stored.  Appends then also keep a bf16 copy of every token,
+ * released ones included, in a ring of W slots per (sequence, layer); streams, page ids and the
+ * budget state are the same as with W = 0 (a token is charged m(a) when it arrives).
  *   seq_ids   dev int32 [n_seqs]
  *   q         dev bf16 [n_seqs][n_q][128]
  *   out       dev fp32 [n_seqs][n_q][128]

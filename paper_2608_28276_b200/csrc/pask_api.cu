@@ -38,7 +38,9 @@ MetaOffsets meta_offsets(const pask_cache_desc_t *d, int n_tags, int n_groups) {
     o.budget = take((size_t)d->max_seqs * sizeof(pask_budget_state_t));
     o.seq_mark = take((size_t)d->max_seqs * 4);
     o.low_vmax = take(sl * 4);
+    o.n_tok = take(sl * 4);
     o.zero_end = p;
+    o.win_act = take(sl * (size_t)d->recent_window);
     o.plan = take((size_t)PASK_MAX_SEQS_PER_CALL * sizeof(AppendPlan));
     o.tok_list = take((size_t)d->max_append_tokens * 4);
     o.item_base = take((size_t)(PASK_MAX_SEQS_PER_CALL + 1) * 4);
@@ -52,9 +54,15 @@ MetaOffsets meta_offsets(const pask_cache_desc_t *d, int n_tags, int n_groups) {
     return o;
 }
 
+// pages of the recent-window rings, which sit behind the HIGH pool's own pages
+size_t window_pages(const pask_cache_desc_t *d) {
+    return (size_t)d->max_seqs * d->n_layers * (size_t)(d->recent_window / kPageTokens);
+}
+
 bool desc_ok(const pask_cache_desc_t *d) {
     return d->n_layers > 0 && d->n_layers <= 4096 && d->max_seqs > 0 && d->max_tokens_per_seq > 0 &&
-           d->max_append_tokens > 0;
+           d->max_append_tokens > 0 && d->recent_window >= 0 && d->recent_window <= PASK_MAX_WINDOW &&
+           d->recent_window % kPageTokens == 0;
 }
 
 pask_status_t cuda_rc(cudaError_t e) { return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA; }
@@ -105,9 +113,10 @@ pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **o
     p->n_layers = rd32(blob + 16);
     p->n_states = rd32(blob + 20);
     p->budget_q16 = rd32(blob + 24);
-    const uint32_t window = rd32(blob + 28), low_bits = rd32(blob + 32), group_size = rd32(blob + 36);
+    p->window = rd32(blob + 28);
+    const uint32_t window = p->window, low_bits = rd32(blob + 32), group_size = rd32(blob + 36);
     bool ok = p->n_tags >= 1 && p->n_tags <= 255 && p->n_groups >= 1 && p->n_groups <= PASK_MAX_GROUPS &&
-              p->n_layers >= 1 && p->n_layers <= 4096 && p->n_states <= (1u << 20) && window == 0 && low_bits == 4 &&
+              p->n_layers >= 1 && p->n_layers <= 4096 && p->n_states <= (1u << 20) && window <= PASK_MAX_WINDOW && window % kPageTokens == 0 && low_bits == 4 &&
               group_size == (uint32_t)kQGroup;
     const size_t lg_pad = ok ? align_up(p->n_layers, 4) : 0;
     const size_t n_ent = ok ? (size_t)p->n_tags * p->n_groups : 0;
@@ -157,7 +166,7 @@ pask_status_t pask_cache_sizes(const pask_cache_desc_t *d, pask_cache_sizes_t *o
     if (!desc_ok(d)) return PASK_ERR_INVALID_ARG;
     out->high_page_bytes = (size_t)d->n_kv_heads * kHighHeadBytes;
     out->low_page_bytes = (size_t)d->n_kv_heads * kLowHeadBytes;
-    out->pool_high_bytes = out->high_page_bytes * d->pool_high_pages;
+    out->pool_high_bytes = out->high_page_bytes * ((size_t)d->pool_high_pages + window_pages(d));
     out->pool_low_bytes = out->low_page_bytes * d->pool_low_pages;
     out->meta_bytes = meta_offsets(d, 255, PASK_MAX_GROUPS).total;  // independent of the policy loaded later
     return PASK_OK;
@@ -168,9 +177,12 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     if (!d || !pol || !meta || !out) return PASK_ERR_INVALID_ARG;
     *out = nullptr;
     if (!shape_ok(d)) return PASK_ERR_UNSUPPORTED_SHAPE;
-    if (!desc_ok(d) || (uint32_t)d->n_layers != pol->n_layers) return PASK_ERR_INVALID_ARG;
-    if ((d->pool_high_pages && !pool_high) || (d->pool_low_pages && !pool_low)) return PASK_ERR_INVALID_ARG;
+    if (!desc_ok(d) || (uint32_t)d->n_layers != pol->n_layers || (uint32_t)d->recent_window != pol->window)
+        return PASK_ERR_INVALID_ARG;
+    if (((d->pool_high_pages || d->recent_window) && !pool_high) || (d->pool_low_pages && !pool_low)) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)pool_high | (uintptr_t)pool_low | (uintptr_t)meta) & 255) return PASK_ERR_INVALID_ARG;
+    if ((size_t)d->pool_high_pages + window_pages(d) > kOrderIdMask || d->pool_low_pages > kOrderIdMask)
+        return PASK_ERR_INVALID_ARG;   // page ids travel in the low bits of the page-order entries
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     int dev_id = 0, sms = 0;
     if (cudaGetDevice(&dev_id) != cudaSuccess) return PASK_ERR_CUDA;
@@ -197,6 +209,9 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     v.budget = reinterpret_cast<pask_budget_state_t *>(m + c->off.budget);
     v.seq_mark = reinterpret_cast<uint32_t *>(m + c->off.seq_mark);
     v.low_vmax = reinterpret_cast<uint32_t *>(m + c->off.low_vmax);
+    v.n_tok = reinterpret_cast<uint32_t *>(m + c->off.n_tok);
+    v.win_act = m + c->off.win_act;
+    v.window = (uint32_t)d->recent_window;
     v.plan = reinterpret_cast<AppendPlan *>(m + c->off.plan);
     v.tok_list = reinterpret_cast<uint32_t *>(m + c->off.tok_list);
     v.item_base = reinterpret_cast<uint32_t *>(m + c->off.item_base);
@@ -220,6 +235,7 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     v.n_groups = (int32_t)pol->n_groups;
     v.cap_high = d->pool_high_pages;
     v.cap_low = d->pool_low_pages;
+    v.high_limit = d->pool_high_pages + (uint32_t)window_pages(d);
     v.budget_q16 = pol->budget_q16;
     v.high_page_bytes = (uint32_t)d->n_kv_heads * kHighHeadBytes;
     v.low_page_bytes = (uint32_t)d->n_kv_heads * kLowHeadBytes;

@@ -27,12 +27,6 @@ __device__ __forceinline__ void budget_add(uint64_t *p, uint64_t v) {
     if (v) atomicAdd(reinterpret_cast<unsigned long long *>(p), (unsigned long long)v);
 }
 
-__device__ __forceinline__ uint32_t lanemask_lt() {
-    uint32_t m;
-    asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
-    return m;
-}
-
 // pages of a stream that an append of cnt tokens at length old writes into (the first may be a page
 // the stream already holds)
 __device__ __forceinline__ uint32_t pages_touched(uint32_t old, uint32_t cnt) {
@@ -161,6 +155,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
             const size_t sl = (size_t)seq * c.n_layers + layer;
             p.old_high = c.n_high[sl];
             p.old_low = c.n_low[sl];
+            p.old_tok = c.n_tok[sl];
             p.cnt_high = run_h;
             p.cnt_low = run_l;
             p.cnt_drop = (uint32_t)(t1 - t0) - run_h - run_l;
@@ -236,6 +231,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         c.n_low[sl] = p.old_low + p.cnt_low;
         pask_budget_state_t &b = c.budget[p.seq];
         const uint64_t n_tok = (uint64_t)p.cnt_high + p.cnt_low + p.cnt_drop;
+        if (c.window) c.n_tok[sl] = p.old_tok + (uint32_t)n_tok;
         b.n_seen[grp] += n_tok;
         b.n_high[grp] += p.cnt_high;
         b.n_low[grp] += p.cnt_low;
@@ -290,7 +286,7 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 __device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uint32_t at, uint32_t page, size_t sl, int head,
                                               int cch, int which, const uint4 x) {
     const uint32_t tau = at & 15u;
-    if (page >= (a == PASK_ACTION_RETAIN_HIGH ? c.cap_high : c.cap_low)) {   // never expected: refuse, do not write
+    if (page >= (a == PASK_ACTION_RETAIN_HIGH ? c.high_limit : c.cap_low)) {   // never expected: refuse, do not write
         atomicOr(&c.ctrl[kCtrlStatus], PASK_DEV_INTERNAL);
         return;
     }
@@ -538,6 +534,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
                     const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided,
                     uint8_t *__restrict__ actions_out, const SmallLut lut) {
     __shared__ int s_seq[kSmallMax], s_cu[kSmallMax + 1];
+    __shared__ uint32_t s_old_n[kSmallMax];
     __shared__ uint32_t s_old_h[kSmallMax], s_old_l[kSmallMax], s_cnt_h[kSmallMax], s_cnt_l[kSmallMax], s_cnt_bad[kSmallMax];
     __shared__ uint32_t s_new_h[kSmallMax], s_new_l[kSmallMax], s_base_h[kSmallMax], s_base_l[kSmallMax];
     __shared__ uint8_t s_act[kSmallMax], s_tok_seq[kSmallMax], s_tok_bad[kSmallMax];
@@ -559,14 +556,16 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     if (tid < n_seqs) {
         const int seq = seq_ids[tid];
         s_seq[tid] = seq;
-        uint32_t oh = 0, ol = 0;
+        uint32_t oh = 0, ol = 0, on = 0;
         if (seq >= 0 && seq < c.max_seqs) {
             const size_t sl = (size_t)seq * c.n_layers + layer;
             oh = c.n_high[sl];
             ol = c.n_low[sl];
+            if (c.window) on = c.n_tok[sl];
         }
         s_old_h[tid] = oh;
         s_old_l[tid] = ol;
+        s_old_n[tid] = on;
     }
     int my_tag = 0, my_decided = 0;
     if (tid < total) {
@@ -690,6 +689,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         }
         c.n_high[sl] = oh + ch;
         c.n_low[sl] = ol + cl;
+        if (c.window) c.n_tok[sl] = s_old_n[tid] + n_tok;
         // budget state: additions only (no read-modify-write round trip); remaining_bytes is derived
         // from retained_bytes and full_bytes when the state is read
         pask_budget_state_t &b = c.budget[seq];
@@ -715,6 +715,47 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
 
     // ---- persist this CTA's token: one thread per 16-byte chunk of K and of V
     if (writer && my_a != PASK_ACTION_RELEASE) persist_chunk(c, my_a, my_at, my_page, my_sl, cg >> 4, cg & 15, which, x);
+
+    // ---- protected recent window: every token, released ones too, also goes to slot (index mod W)
+    // of its (sequence, layer) ring as bf16; of a sequence's tokens in this call only the last W can
+    // still be in the window afterwards (and they have distinct slots)
+    if (c.window) {
+        const int W = (int)c.window, r = my_tok - s_cu[my_i], n_i = s_cu[my_i + 1] - s_cu[my_i];
+        if (r >= n_i - W) {
+            const uint32_t slot = (s_old_n[my_i] + (uint32_t)r) % (uint32_t)W;
+            const uint32_t ring_page = c.cap_high + (uint32_t)my_sl * (uint32_t)(W >> 4) + (slot >> 4);
+            if (writer) persist_chunk(c, PASK_ACTION_RETAIN_HIGH, slot, ring_page, my_sl, cg >> 4, cg & 15, which, x);
+            if (tid == 0) c.win_act[my_sl * (size_t)W + slot] = (uint8_t)my_a;
+        }
+    }
+}
+
+// General path, recent window: one CTA per sequence copies the last W of the sequence's tokens in
+// this call (released ones too) into its ring as bf16 and records their actions.
+__global__ void __launch_bounds__(256)
+append_window_kernel(DevCache c, int layer, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
+                     const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided) {
+    if (c.ctrl[kCtrlPlanOk] == 0) return;
+    const AppendPlan p = c.plan[blockIdx.x];
+    const int tid = threadIdx.x, chunks = 16 * c.n_kv, W = (int)c.window;
+    const int n = p.tok1 - p.tok0, group = c.layer_group[layer];
+    const size_t sl = (size_t)p.seq * c.n_layers + layer;
+    const int which = tid >= chunks, cg = which ? tid - chunks : tid;
+    for (int r = n > W ? n - W : 0; r < n; r++) {
+        const int t = p.tok0 + r;
+        const uint32_t slot = (p.old_tok + (uint32_t)r) % (uint32_t)W;
+        const uint32_t ring_page = c.cap_high + (uint32_t)sl * (uint32_t)(W >> 4) + (slot >> 4);
+        if (tid < 2 * chunks) {
+            const uint4 x = (which ? v : k)[(size_t)t * chunks + cg];
+            persist_chunk(c, PASK_ACTION_RETAIN_HIGH, slot, ring_page, sl, cg >> 4, cg & 15, which, x);
+        }
+        if (tid == 0) {
+            const int tag = tags[t];
+            int a = tag < c.n_tags ? c.lut[tag * c.n_groups + group] : PASK_ACTION_RETAIN_HIGH;   // protected, unknown: high
+            if (decided) a = decided[(size_t)t * c.n_groups + group];
+            c.win_act[sl * (size_t)W + slot] = (uint8_t)a;
+        }
+    }
 }
 
 // Return every page of one sequence to the free stacks and clear its counters.
@@ -730,7 +771,7 @@ __global__ void __launch_bounds__(256) seq_reset_kernel(DevCache c, int seq) {
         for (uint32_t x = tid; x < ph; x += blockDim.x) c.free_high[bh + x] = c.tbl_high[sl * c.max_pages + x];
         for (uint32_t x = tid; x < pl; x += blockDim.x) c.free_low[bl + x] = c.tbl_low[sl * c.max_pages + x];
         __syncthreads();
-        if (tid == 0) { s_h = bh + ph; s_l = bl + pl; c.n_high[sl] = 0; c.n_low[sl] = 0; c.low_vmax[sl] = 0; }
+        if (tid == 0) { s_h = bh + ph; s_l = bl + pl; c.n_high[sl] = 0; c.n_low[sl] = 0; c.low_vmax[sl] = 0; c.n_tok[sl] = 0; }
         __syncthreads();
     }
     if (tid == 0) { c.ctrl[kCtrlHighFree] = s_h; c.ctrl[kCtrlLowFree] = s_l; }
@@ -767,6 +808,9 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
         append_write_kernel<<<ctas, kWriteThreads, smem, stream>>>(c->dev, layer, n_seqs, static_cast<const uint4 *>(k),
                                                                   static_cast<const uint4 *>(v));
     }
+    if (c->dev.window && total_tokens > 0)
+        append_window_kernel<<<n_seqs, 256, 0, stream>>>(c->dev, layer, static_cast<const uint4 *>(k),
+                                                        static_cast<const uint4 *>(v), tags, decided);
     return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }
 

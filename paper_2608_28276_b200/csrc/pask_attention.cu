@@ -52,7 +52,7 @@ struct Workspace {
     uint32_t *cost_prefix;  // [n_seqs + 1] cost of the sequences before s
     uint32_t *page_prefix;  // [n_seqs + 1] pages of the sequences before s
     uint2 *tokens;          // [n_seqs] (n_high, n_low) tokens
-    uint32_t *order;        // [page_prefix[n_seqs]] pages in visiting order: kOrderHigh | kOrderTail | page id
+    uint32_t *order;        // [page_prefix[n_seqs]] pages in visiting order: kOrderHigh | tokens to attend << 27 | page id
     float2 *part_ml;        // [slots][n_q] (reference maximum in log2 units, sum)
     float *part_o;          // [slots][n_q][128] unnormalised outputs
 };
@@ -242,17 +242,39 @@ attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ 
     pdl_launch_dependents();
     pdl_wait();
     uint32_t *s_cost = s_plan, *s_page = s_cost + n_seqs + 1, *s_nh = s_page + n_seqs + 1, *s_nl = s_nh + n_seqs;
+    uint32_t *s_nw = s_nl + n_seqs;           // tokens in the protected recent window
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int s = tid; s < n_seqs; s += kPlanThreads) {
         const int sid = seq_ids[s];
-        uint32_t nh = 0, nl = 0;
+        uint32_t nh = 0, nl = 0, nw = 0;
         if (sid >= 0 && sid < c.max_seqs) {
             const size_t sl = (size_t)sid * c.n_layers + layer;
             nh = c.n_high[sl];
             if (has_low) nl = c.n_low[sl];
+            if (c.window) {
+                // The last min(W, tokens seen) tokens are attended from the bf16 ring whatever their
+                // action.  Streams are in arrival order, so the window's HIGH and LOW members are the
+                // last entries of the two streams: shorten those by as many.
+                const uint32_t seen = c.n_tok[sl];
+                nw = seen < c.window ? seen : c.window;
+                const uint4 *act = reinterpret_cast<const uint4 *>(c.win_act + sl * c.window);
+                uint32_t wh = 0, wl = 0;
+                for (uint32_t i = 0; i < nw; i += 16) {
+                    const uint4 a4 = act[i >> 4];
+                    const uint32_t w4[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int b = 0; b < 16; b++) {
+                        const uint32_t a = (w4[b >> 2] >> (8 * (b & 3))) & 0xffu;
+                        if (i + b < nw) { wh += a == PASK_ACTION_RETAIN_HIGH; wl += a == PASK_ACTION_RETAIN_LOW; }
+                    }
+                }
+                nh -= wh;
+                if (has_low) nl -= wl;
+            }
         }
         s_nh[s] = nh;
         s_nl[s] = nl;
+        s_nw[s] = nw;
     }
     if (tid == 0) s_cost[0] = s_page[0] = 0;
     __syncthreads();
@@ -261,7 +283,10 @@ attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ 
         for (int base = 0; base < n_seqs; base += 32) {
             const int idx = base + lane;
             uint32_t ph = 0, pl = 0;
-            if (idx < n_seqs) { ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens; pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens; }
+            if (idx < n_seqs) {   // the ring's pages have the HIGH format and count as HIGH pages
+                ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens + (s_nw[idx] + kPageTokens - 1) / kPageTokens;
+                pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens;
+            }
             uint32_t ic = ph * kCostHighPage + pl * kCostLowPage, ip = ph + pl;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
@@ -286,16 +311,22 @@ attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ 
             if (s_page[mid] > gp) e = mid; else a = mid + 1;
         }
         const int s = a - 1;
-        const uint32_t nh = s_nh[s], nl = s_nl[s];
+        const uint32_t nh = s_nh[s], nl = s_nl[s], nw = s_nw[s];
         const uint32_t ph = (nh + kPageTokens - 1) / kPageTokens, pl = (nl + kPageTokens - 1) / kPageTokens;
-        const size_t sl = ((size_t)seq_ids[s] * c.n_layers + layer) * c.max_pages;
+        const uint32_t pw = (nw + kPageTokens - 1) / kPageTokens;
+        const size_t slw = (size_t)seq_ids[s] * c.n_layers + layer, sl = slw * c.max_pages;
         uint32_t idx, entry;
-        if (page_at(gp - s_page[s], ph, pl, idx)) {
-            entry = c.tbl_high[sl + idx] | kOrderHigh;
-            if (idx == ph - 1 && (nh & (kPageTokens - 1))) entry |= kOrderTail;
+        if (page_at(gp - s_page[s], ph + pw, pl, idx)) {
+            if (idx < ph) {
+                entry = c.tbl_high[sl + idx] | kOrderHigh;
+                if (idx == ph - 1) entry |= (nh & (kPageTokens - 1)) << kOrderValidShift;
+            } else {            // a page of the recent-window ring
+                entry = (c.cap_high + (uint32_t)slw * (c.window / kPageTokens) + (idx - ph)) | kOrderHigh;
+                if (idx - ph == pw - 1) entry |= (nw & (kPageTokens - 1)) << kOrderValidShift;
+            }
         } else {
             entry = c.tbl_low[sl + idx];
-            if (idx == pl - 1 && (nl & (kPageTokens - 1))) entry |= kOrderTail;
+            if (idx == pl - 1) entry |= (nl & (kPageTokens - 1)) << kOrderValidShift;
         }
         ws.order[gp] = entry;
     }
@@ -459,7 +490,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         const uint32_t n_pages = cut_positions((hi < c1 ? hi : c1) - c0, c1 - c0, n_pos) -
                                  cut_positions((lo > c0 ? lo : c0) - c0, c1 - c0, n_pos);
         const uint2 tk = __ldg(p.ws.tokens + s);
-        const uint32_t seq_n_high = tk.x, seq_n_low = tk.y;
+        const uint32_t seq_n_low = tk.y;
 
         // ---- query fragments: lane (g,t) holds dims 8(4j+t) .. +7 of head g & 3 for j = 0..3
         uint4 qf[4];
@@ -525,8 +556,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
             uint32_t st = w.acquire(entry);
             if (w.dead) break;
             const bool is_high = entry & kOrderHigh;
-            uint32_t n_valid = 16u;
-            if (entry & kOrderTail) n_valid = (is_high ? seq_n_high : seq_n_low) & (kPageTokens - 1);
+            const uint32_t n_valid = (((entry >> kOrderValidShift) - 1u) & 15u) + 1u;   // 0 in the entry means all 16
 
             float sc[4] = {0.f, 0.f, 0.f, 0.f};
             if (is_high) {
@@ -757,7 +787,7 @@ size_t attn_smem_bytes(int n_seqs, int n_warps) {
 // carve the caller's workspace
 size_t carve_workspace(const pask_cache *c, int n_seqs, uint8_t *base, Workspace *ws) {
     const size_t slots = (size_t)c->attn_ctas + n_seqs;
-    const size_t max_pages = (size_t)n_seqs * 2 * c->dev.max_pages;
+    const size_t max_pages = (size_t)n_seqs * (2 * c->dev.max_pages + c->dev.window / kPageTokens);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
     const size_t o_cost = take((size_t)(n_seqs + 1) * 4), o_page = take((size_t)(n_seqs + 1) * 4);
@@ -795,7 +825,7 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
     auto kern = has_low ? decode_attn_kernel<true> : decode_attn_kernel<false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return PASK_ERR_CUDA;
-    cudaError_t e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(4 * n_seqs + 2) * 4, stream,
+    cudaError_t e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(5 * n_seqs + 2) * 4, stream,
                                c->dev, layer, n_seqs, seq_ids, p.ws, has_low ? 1 : 0);
     if (c->ev_start) cudaEventRecord(c->ev_start, stream);
     if (e == cudaSuccess) e = launch_pdl(kern, dim3(c->attn_ctas), dim3(32 * n_warps), smem, stream, p);

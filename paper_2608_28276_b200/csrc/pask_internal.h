@@ -32,7 +32,8 @@ struct AppendPlan {
     uint32_t cnt_drop, bad_tags;
     uint32_t new_pages_high, new_pages_low;
     int32_t tok0, tok1;            // the sequence's token range in the call
-    uint32_t pad[5];
+    uint32_t old_tok;              // tokens the (sequence, layer) had seen before the call
+    uint32_t pad[4];
 };
 static_assert(sizeof(AppendPlan) == 64, "plan record");
 
@@ -58,6 +59,10 @@ struct DevCache {
     pask_budget_state_t *budget;     // [max_seqs]
     uint32_t *seq_mark;              // [max_seqs] serial of the last append call that named the sequence
     uint32_t *low_vmax;              // [max_seqs][n_layers] largest V scale (fp16 bits) in the LOW stream
+    uint32_t *n_tok;                 // [max_seqs][n_layers] tokens appended so far, released ones included
+    uint8_t *win_act;                // [max_seqs][n_layers][window] action of the token in each slot of the recent window
+    uint32_t window;                 // protected recent window W in tokens (0: none); its W/16 bf16 pages per (sequence,
+                                     // layer) are pages cap_high + (seq * n_layers + layer) * W/16 .. of the HIGH pool
     AppendPlan *plan;                // [PASK_MAX_SEQS_PER_CALL]
     uint32_t *tok_list;              // [max_append_tokens] bulk appends: each sequence's retained tokens in stream order
                                      // (HIGH from the front of its token range, LOW from the back)
@@ -74,13 +79,14 @@ struct DevCache {
     int32_t n_layers, n_q, n_kv, max_seqs, max_pages, max_append_tokens;
     int32_t n_tags, n_groups;
     uint32_t cap_high, cap_low;
+    uint32_t high_limit;             // cap_high plus the pages of the recent-window rings
     uint32_t budget_q16;
     uint32_t high_page_bytes, low_page_bytes;
     uint32_t bytes_h, bytes_l;       // m(H), m(L) per token per layer
 };
 
 struct MetaOffsets {
-    size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, low_vmax, plan, tok_list, item_base, lut,
+    size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, low_vmax, n_tok, win_act, plan, tok_list, item_base, lut,
         layer_group, dec_row, dec_rho, gamma, crit, total;
     size_t zero_begin, zero_end;     // the span cleared by a reset (counters, tables, budgets, marks)
 };
@@ -88,7 +94,7 @@ struct MetaOffsets {
 }  // namespace pask
 
 struct pask_policy {
-    uint32_t n_tags, n_groups, n_layers, n_states, budget_q16;
+    uint32_t n_tags, n_groups, n_layers, n_states, budget_q16, window;
     std::vector<uint8_t> layer_group, a0, a_floor, eff;
     std::vector<float> rho_rl, rho_lh;
     std::vector<uint32_t> gamma;

@@ -111,8 +111,8 @@ PASK_HD uint32_t cut_positions(uint32_t x, uint32_t cs, uint32_t n) {
 }
 
 // entries of the per-call page order list built by the plan kernel
-constexpr uint32_t kOrderHigh = 0x80000000u;   // the page is a HIGH page (else LOW)
-constexpr uint32_t kOrderTail = 0x40000000u;   // last page of its stream and only partly filled
-constexpr uint32_t kOrderIdMask = 0x3fffffffu;
+constexpr uint32_t kOrderHigh = 0x80000000u;   // the page has the HIGH (bf16) format (else LOW)
+constexpr int kOrderValidShift = 27;           // bits 27..30: tokens of the page to attend, 0 meaning all 16
+constexpr uint32_t kOrderIdMask = 0x07ffffffu;
 
 }  // namespace pask

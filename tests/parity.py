@@ -28,8 +28,9 @@ class Pair:
         self.hp = pool_high_pages if pool_high_pages is not None else pages
         self.lp = pool_low_pages if pool_low_pages is not None else pages
         blob = blob or workload.blob
+        window = int.from_bytes(blob[28:32], "little")                  # the policy's protected recent window
         self.gpu = pask.Cache(blob, cfg.n_layers, cfg.n_q, cfg.n_kv, self.max_seqs, self.max_tokens,
-                              max_append_tokens or total, self.hp, self.lp)
+                              max_append_tokens or total, self.hp, self.lp, recent_window=window)
         self.orc = oracle.Cache(oracle.Policy(blob), cfg.n_q, cfg.n_kv, self.max_seqs, self.hp, self.lp)
 
     # ------------------------------------------------------------------ append
