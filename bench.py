@@ -199,8 +199,9 @@ class Job:
         pages_l = int(sum(((nl[:, lg[l]] + extra + 15) // 16).sum() for l in range(cfg.n_layers))) + 64
         self.lens = [w.total_len(b) for b in range(self.B)]
         self.total_tokens = int(sum(self.lens))
+        self.window = int.from_bytes(blob[28:32], "little")
         self.cache = P.Cache(blob, cfg.n_layers, cfg.n_q, cfg.n_kv, self.B, max(self.lens) + extra + 16,
-                             self.total_tokens, pages_h, pages_l, device=device)
+                             self.total_tokens, pages_h, pages_l, device=device, recent_window=self.window)
         self.ids = torch.arange(self.B, dtype=torch.int32, device=device)
         self.cu1 = torch.arange(self.B + 1, dtype=torch.int32, device=device)
         self.ws = self.cache.workspace(self.B)
@@ -301,8 +302,16 @@ class Job:
         lg = self.w.policy.layer_group.astype(np.int64)
         n_ctas = 2 * torch.cuda.get_device_properties(self.device).multi_processor_count
         tot = 0.0
+        win_h = win_l = np.zeros((self.B, self.w.policy.n_groups), np.int64)
+        if self.window:     # window members are read from the bf16 ring instead of from their streams
+            eff = np.maximum(self.w.policy.a0, self.w.policy.a_floor)
+            win_h, win_l = win_h.copy(), win_l.copy()
+            for b in range(self.B):
+                tags = self.w.tags(b, self.lens[b] + steps_done - self.window, self.window)
+                acts = np.where(tags[:, None] < self.w.policy.n_tags, eff[np.minimum(tags, self.w.policy.n_tags - 1)], 2)
+                win_h[b], win_l[b] = (acts == 2).sum(0), (acts == 1).sum(0)
         for l in range(cfg.n_layers):
-            nh, nl = self.nh[:, lg[l]] + steps_done, self.nl[:, lg[l]]
+            nh, nl = self.nh[:, lg[l]] + steps_done - win_h[:, lg[l]] + self.window, self.nl[:, lg[l]] - win_l[:, lg[l]]
             tot += float((nh * cfg.n_kv * 512).sum() + (nl * cfg.n_kv * 144).sum())
             tot += float((((nh + 15) // 16) + ((nl + 15) // 16)).sum() * 4)
         per_layer = tot / cfg.n_layers
@@ -325,6 +334,9 @@ def run_cuda(args, rank, world):
     e2e_steps = min(args.steps, 5)
     cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, 2 * total_steps + e2e_steps + 8))
     w = rank_workload(cfg, rank)
+    if args.window:
+        from dataclasses import replace as _replace
+        w.policy = _replace(w.policy, recent_window=args.window)
     t_setup = time.time()
     job = Job(P, w, device, 2 * total_steps + e2e_steps + 4, dynamic=args.dynamic)
     job.fill()
@@ -413,6 +425,7 @@ def run_cuda(args, rank, world):
         "dtype": "bf16/int4 storage, bf16 tensor-core operands with fp32 accumulation", "data": "synthetic",
         "config": {"workload": cfg.name, "batch_per_gpu": job.B, "layers": cfg.n_layers, "layer_groups": cfg.n_groups,
                    "kv_budget_target": cfg.budget, "kv_budget_realised": ret / full, "table": f"greedy/{cfg.bias}",
+                   "recent_window": args.window,
                    "tokens_in_cache_per_gpu": job.total_tokens, "page_tokens": 16,
                    "l2": "inputs larger than L2: each layer streams its own ~%.0f MB of pages" % (alg / 1e6),
                    "setup_s": round(t_setup, 1)},
@@ -583,6 +596,7 @@ def main():
     ap.add_argument("--no-full-kv", dest="full_kv", action="store_false")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="0 skips the CPU-oracle leg")
     ap.add_argument("--event-stride", type=int, default=4, help="time the streaming kernel of every n-th launch")
+    ap.add_argument("--window", type=int, default=0, help="protected recent window in tokens (multiple of 16, <= 256)")
     ap.add_argument("--graph", action="store_true", help="replay each timed step as one CUDA graph (launch-bound shapes)")
     ap.add_argument("--dynamic", action="store_true",
                     help="decide every token against the running budget (pask_decide) instead of the frozen table alone")

@@ -730,8 +730,9 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     }
 }
 
-// General path, recent window: one CTA per sequence copies the last W of the sequence's tokens in
-// this call (released ones too) into its ring as bf16 and records their actions.
+// General path, recent window: CTA (j, y) copies the y-th newest of sequence j's tokens in this call
+// (released ones too) into the sequence's ring as bf16 and records its action; only the last W
+// tokens of a sequence can still be in the window afterwards, and they have distinct slots.
 __global__ void __launch_bounds__(256)
 append_window_kernel(DevCache c, int layer, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
                      const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided) {
@@ -739,22 +740,21 @@ append_window_kernel(DevCache c, int layer, const uint4 *__restrict__ k, const u
     const AppendPlan p = c.plan[blockIdx.x];
     const int tid = threadIdx.x, chunks = 16 * c.n_kv, W = (int)c.window;
     const int n = p.tok1 - p.tok0, group = c.layer_group[layer];
+    if ((int)blockIdx.y >= n) return;
+    const int r = n - 1 - (int)blockIdx.y, t = p.tok0 + r;
     const size_t sl = (size_t)p.seq * c.n_layers + layer;
     const int which = tid >= chunks, cg = which ? tid - chunks : tid;
-    for (int r = n > W ? n - W : 0; r < n; r++) {
-        const int t = p.tok0 + r;
-        const uint32_t slot = (p.old_tok + (uint32_t)r) % (uint32_t)W;
-        const uint32_t ring_page = c.cap_high + (uint32_t)sl * (uint32_t)(W >> 4) + (slot >> 4);
-        if (tid < 2 * chunks) {
-            const uint4 x = (which ? v : k)[(size_t)t * chunks + cg];
-            persist_chunk(c, PASK_ACTION_RETAIN_HIGH, slot, ring_page, sl, cg >> 4, cg & 15, which, x);
-        }
-        if (tid == 0) {
-            const int tag = tags[t];
-            int a = tag < c.n_tags ? c.lut[tag * c.n_groups + group] : PASK_ACTION_RETAIN_HIGH;   // protected, unknown: high
-            if (decided) a = decided[(size_t)t * c.n_groups + group];
-            c.win_act[sl * (size_t)W + slot] = (uint8_t)a;
-        }
+    const uint32_t slot = (p.old_tok + (uint32_t)r) % (uint32_t)W;
+    const uint32_t ring_page = c.cap_high + (uint32_t)sl * (uint32_t)(W >> 4) + (slot >> 4);
+    if (tid < 2 * chunks) {
+        const uint4 x = (which ? v : k)[(size_t)t * chunks + cg];
+        persist_chunk(c, PASK_ACTION_RETAIN_HIGH, slot, ring_page, sl, cg >> 4, cg & 15, which, x);
+    }
+    if (tid == 0) {
+        const int tag = tags[t];
+        int a = tag < c.n_tags ? c.lut[tag * c.n_groups + group] : PASK_ACTION_RETAIN_HIGH;   // protected, unknown: high
+        if (decided) a = decided[(size_t)t * c.n_groups + group];
+        c.win_act[sl * (size_t)W + slot] = (uint8_t)a;
     }
 }
 
@@ -809,7 +809,7 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
                                                                   static_cast<const uint4 *>(v));
     }
     if (c->dev.window && total_tokens > 0)
-        append_window_kernel<<<n_seqs, 256, 0, stream>>>(c->dev, layer, static_cast<const uint4 *>(k),
+        append_window_kernel<<<dim3(n_seqs, c->dev.window), 256, 0, stream>>>(c->dev, layer, static_cast<const uint4 *>(k),
                                                         static_cast<const uint4 *>(v), tags, decided);
     return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }

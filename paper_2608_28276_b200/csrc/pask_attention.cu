@@ -251,30 +251,34 @@ attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ 
             const size_t sl = (size_t)sid * c.n_layers + layer;
             nh = c.n_high[sl];
             if (has_low) nl = c.n_low[sl];
-            if (c.window) {
-                // The last min(W, tokens seen) tokens are attended from the bf16 ring whatever their
-                // action.  Streams are in arrival order, so the window's HIGH and LOW members are the
-                // last entries of the two streams: shorten those by as many.
-                const uint32_t seen = c.n_tok[sl];
-                nw = seen < c.window ? seen : c.window;
-                const uint4 *act = reinterpret_cast<const uint4 *>(c.win_act + sl * c.window);
-                uint32_t wh = 0, wl = 0;
-                for (uint32_t i = 0; i < nw; i += 16) {
-                    const uint4 a4 = act[i >> 4];
-                    const uint32_t w4[4] = {a4.x, a4.y, a4.z, a4.w};
-#pragma unroll
-                    for (int b = 0; b < 16; b++) {
-                        const uint32_t a = (w4[b >> 2] >> (8 * (b & 3))) & 0xffu;
-                        if (i + b < nw) { wh += a == PASK_ACTION_RETAIN_HIGH; wl += a == PASK_ACTION_RETAIN_LOW; }
-                    }
-                }
-                nh -= wh;
-                if (has_low) nl -= wl;
-            }
+            if (c.window) { const uint32_t seen = c.n_tok[sl]; nw = seen < c.window ? seen : c.window; }
         }
         s_nh[s] = nh;
         s_nl[s] = nl;
         s_nw[s] = nw;
+    }
+    if (c.window) {
+        // The last min(W, tokens seen) tokens are attended from the bf16 ring whatever their action.
+        // Streams are in arrival order, so the window's HIGH and LOW members are the last entries
+        // of the two streams: shorten those by as many.  One thread per 16 slots, all loads at once.
+        __syncthreads();
+        const int per = (int)c.window / kPageTokens;
+        for (int idx = tid; idx < n_seqs * per; idx += kPlanThreads) {
+            const int s = idx / per, i = idx - s * per;
+            const uint32_t nw = s_nw[s];
+            if ((uint32_t)i * 16u >= nw) continue;
+            const size_t sl = (size_t)seq_ids[s] * c.n_layers + layer;
+            const uint4 a4 = reinterpret_cast<const uint4 *>(c.win_act + sl * c.window)[i];
+            const uint32_t w4[4] = {a4.x, a4.y, a4.z, a4.w};
+            uint32_t wh = 0, wl = 0;
+#pragma unroll
+            for (int b = 0; b < 16; b++) {
+                const uint32_t a = (w4[b >> 2] >> (8 * (b & 3))) & 0xffu;
+                if ((uint32_t)i * 16u + b < nw) { wh += a == PASK_ACTION_RETAIN_HIGH; wl += a == PASK_ACTION_RETAIN_LOW; }
+            }
+            if (wh) atomicSub(&s_nh[s], wh);
+            if (wl && has_low) atomicSub(&s_nl[s], wl);
+        }
     }
     if (tid == 0) s_cost[0] = s_page[0] = 0;
     __syncthreads();
