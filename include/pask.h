@@ -303,6 +303,21 @@ pask_status_t pask_decode_step_host(pask_cache_t *cache, int32_t layer, int32_t 
 size_t pask_step_staging_bytes(const pask_cache_t *cache, int32_t n_seqs);
 
 /* ---------------------------------------------------------------------------------------------
+ * pask_distortion -- the inner term of the attention-output distortion (Eq. 4): for each row r
+ * (one decode position of one sequence at one layer) max over query heads h of
+ * || o_ref[r][h][:] - o_test[r][h][:] ||_2^2, where o_ref is the output of pask_decode_attention_full
+ * on the full high-precision cache and o_test the output under the policy being probed.  Summing it
+ * over the layers of a group and averaging over positions, as Eq. 4 does, is left to the caller:
+ * sum_inout accumulates over calls.
+ *   o_ref, o_test  dev fp32 [n_rows][n_q_heads][128], 16-byte aligned; n_q_heads <= 32
+ *   per_row_out    dev fp32 [n_rows] or NULL
+ *   sum_inout      dev fp64 or NULL: the sum over rows is ADDED to it (clear it before the first call;
+ *                  the order of the additions, hence the last bits, is not fixed)
+ */
+pask_status_t pask_distortion(int32_t n_rows, int32_t n_q_heads, const float *o_ref, const float *o_test,
+                              float *per_row_out, double *sum_inout, pask_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
  * pask_budget_state -- the constant-size budget state of one sequence (Algorithm 2 step 8:
  * R' = R - sum_c m(a_c, c); normalised cost of Eq. 1 is retained_bytes / full_bytes) plus the
  * cache-wide device status word.  Copies to host memory and WAITS for `stream`. */

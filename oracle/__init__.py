@@ -62,6 +62,8 @@ def lib():
         L.orc_pool_state.restype = None
         L.orc_attention.argtypes = [vp, i32, i32, vp, vp, vp]
         L.orc_attention_batch.argtypes = [vp, i32, i32, vp, vp, vp, vp]
+        L.orc_distortion.restype = C.c_double
+        L.orc_distortion.argtypes = [i32, i32, vp, vp, vp]
         assert L.orc_sizeof_budget() == C.sizeof(Budget)
         _lib = L
     return _lib
@@ -220,6 +222,16 @@ class Cache:
         rc = lib().orc_attention_batch(self.h, layer, n, _ptr(seq_ids), _ptr(q), _ptr(out), _ptr(lse))
         assert rc == 0
         return out, lse
+
+
+def distortion(o_ref: np.ndarray, o_test: np.ndarray):
+    """Eq. 4's inner term: (per-row max over heads of the squared distance, their sum). fp32 [rows][n_q][128] in."""
+    a = np.ascontiguousarray(o_ref, dtype=np.float32)
+    b = np.ascontiguousarray(o_test, dtype=np.float32)
+    assert a.shape == b.shape and a.ndim == 3 and a.shape[2] == 128
+    per = np.zeros(a.shape[0], np.float64)
+    total = lib().orc_distortion(a.shape[0], a.shape[1], _ptr(a), _ptr(b), _ptr(per))
+    return per, float(total)
 
 
 def max_threads() -> int:

@@ -674,6 +674,27 @@ int orc_attention_batch(orc_cache *c, int layer, int n_seqs, const int32_t *seq_
     return ORC_OK;
 }
 
+/* Eq. 4's inner term for each row: max over heads of the squared Euclidean distance between two
+ * attention outputs.  o_ref, o_test fp32 [n_rows][n_q][128]; per_row fp64 [n_rows]; returns their sum. */
+double orc_distortion(int n_rows, int n_q, const float *o_ref, const float *o_test, double *per_row) {
+    double total = 0.0;
+    for (int r = 0; r < n_rows; r++) {
+        double worst = 0.0;
+        for (int h = 0; h < n_q; h++) {
+            double d2 = 0.0;
+            for (int i = 0; i < HEAD_DIM; i++) {
+                size_t at = ((size_t)r * n_q + h) * HEAD_DIM + i;
+                double d = (double)o_ref[at] - (double)o_test[at];
+                d2 += d * d;
+            }
+            if (d2 > worst) worst = d2;
+        }
+        if (per_row) per_row[r] = worst;
+        total += worst;
+    }
+    return total;
+}
+
 int orc_max_threads(void) {
 #ifdef _OPENMP
     extern int omp_get_max_threads(void);

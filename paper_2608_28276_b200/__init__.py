@@ -30,7 +30,7 @@ EXPORTS = [
     "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decide",
     "pask_append_kv_decided", "pask_decode_attention",
     "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes",
-    "pask_budget_state", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
+    "pask_budget_state", "pask_distortion", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
     "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
 ]
 
@@ -84,6 +84,7 @@ _lib.pask_workspace_bytes.restype = _sz
 _lib.pask_decode_step_host.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
 _lib.pask_step_staging_bytes.argtypes = [_vp, _i32]
 _lib.pask_step_staging_bytes.restype = _sz
+_lib.pask_distortion.argtypes = [_i32, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_budget_state.argtypes = [_vp, _i32, C.POINTER(BudgetState), _vp]
 _lib.pask_cache_set_timing_events.argtypes = [_vp, _vp, _vp]
 _lib.pask_debug_stream_len.argtypes = [_vp, _i32, _i32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), _vp]
@@ -240,6 +241,15 @@ def pask_decode_step_host(cache: int, layer: int, seq_ids_host, k_host, v_host, 
                                       _dptr(staging), staging.numel() * staging.element_size(), _dptr(workspace),
                                       workspace.numel() * workspace.element_size(), _stream(stream)),
            "pask_decode_step_host")
+
+
+def pask_distortion(o_ref, o_test, per_row_out=None, sum_inout=None, stream=None):
+    """Eq. 4's inner term: per row max over heads of the squared distance of two attention outputs
+    [rows][n_q][128] fp32; per_row_out fp32 [rows] and / or sum_inout fp64 [1] (added to)."""
+    assert o_ref.shape == o_test.shape and o_ref.shape[-1] == 128
+    _check(_lib.pask_distortion(o_ref.shape[0], o_ref.shape[1], _dptr(o_ref, torch.float32), _dptr(o_test, torch.float32),
+                                _dptr(per_row_out, torch.float32), _dptr(sum_inout, torch.float64), _stream(stream)),
+           "pask_distortion")
 
 
 def pask_budget_state(cache: int, seq: int, stream=None) -> BudgetState:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libpask.so")
-SOURCES = ["pask_api.cu", "pask_append.cu", "pask_decide.cu", "pask_attention.cu"]
+SOURCES = ["pask_api.cu", "pask_append.cu", "pask_decide.cu", "pask_attention.cu", "pask_probe.cu"]
 HEADERS = ["pask_internal.h", "pask_layout.h", os.path.join("..", "..", "include", "pask.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "--ftz=false", "--prec-div=true", "--prec-sqrt=true", "--fmad=true"]
