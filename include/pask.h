@@ -258,6 +258,19 @@ pask_status_t pask_append_kv_decided(pask_cache_t *cache, int32_t layer, int32_t
 pask_status_t pask_decode_attention(pask_cache_t *cache, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                     const void *q, float *out, float *lse, void *workspace,
                                     size_t workspace_bytes, pask_stream_t stream);
+/* pask_append_attend -- one layer of a decode step in one call: pask_append_kv (or, with `actions`
+ * != NULL, pask_append_kv_decided) for a ragged batch, then pask_decode_attention with one query
+ * per sequence of the same batch.  Results are those of the two calls made one after the other.
+ * For small batches (<= 128 sequences and tokens, no recent window) the append's single launch also
+ * writes the attention's work plan, which saves a launch per layer; otherwise the two calls are
+ * simply issued in turn.  If the append is refused (sticky PASK_DEV_* bit) out and lse are
+ * undefined.  Arguments as for the two calls. */
+pask_status_t pask_append_attend(pask_cache_t *cache, int32_t layer, int32_t n_seqs, int32_t total_tokens,
+                                 const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
+                                 const uint8_t *tags, const uint8_t *actions, uint8_t *actions_out, const void *q,
+                                 float *out, float *lse, void *workspace, size_t workspace_bytes,
+                                 pask_stream_t stream);
+
 /* The full high-precision reference (the paper's "Full KV", C_KV = 1): same arguments, for a
  * cache whose policy keeps everything at high precision; the LOW stream is not read at all
  * (its code path is compiled out), so any LOW tokens present would be ignored. */

@@ -28,7 +28,7 @@ MAX_WINDOW = 256
 EXPORTS = [
     "pask_load_policy", "pask_free_policy", "pask_policy_action", "pask_cache_sizes", "pask_cache_create",
     "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decide",
-    "pask_append_kv_decided", "pask_decode_attention",
+    "pask_append_kv_decided", "pask_append_attend", "pask_decode_attention",
     "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes",
     "pask_budget_state", "pask_distortion", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
     "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
@@ -76,6 +76,7 @@ _lib.pask_seq_reset.argtypes = [_vp, _i32, _vp]
 _lib.pask_append_kv.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_decide.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_append_kv_decided.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.pask_append_attend.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.pask_decode_attention.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.pask_decode_attention_full.argtypes = _lib.pask_decode_attention.argtypes
 _lib.pask_decode_attention_static.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
@@ -195,6 +196,18 @@ def pask_append_kv_decided(cache: int, layer: int, seq_ids, cu_tokens, k, v, tag
                                        _dptr(v, torch.bfloat16), _dptr(tags, torch.uint8),
                                        _dptr(actions, torch.uint8), _dptr(actions_out, torch.uint8),
                                        _stream(stream)), "pask_append_kv_decided")
+
+
+def pask_append_attend(cache: int, layer: int, seq_ids, cu_tokens, k, v, tags, q, out, lse, workspace, actions=None,
+                       actions_out=None, stream=None, total_tokens=None):
+    """One layer of a decode step: append (table actions, or `actions` from pask_decide) then attention."""
+    total = k.shape[0] if total_tokens is None else total_tokens
+    _check(_lib.pask_append_attend(cache, layer, seq_ids.numel(), total, _dptr(seq_ids, torch.int32),
+                                   _dptr(cu_tokens, torch.int32), _dptr(k, torch.bfloat16), _dptr(v, torch.bfloat16),
+                                   _dptr(tags, torch.uint8), _dptr(actions, torch.uint8), _dptr(actions_out, torch.uint8),
+                                   _dptr(q, torch.bfloat16), _dptr(out, torch.float32), _dptr(lse, torch.float32),
+                                   _dptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "pask_append_attend")
 
 
 def pask_workspace_bytes(cache: int, n_seqs: int) -> int:

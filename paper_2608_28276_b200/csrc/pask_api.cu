@@ -303,7 +303,7 @@ pask_status_t pask_seq_reset(pask_cache_t *c, int32_t seq, pask_stream_t stream)
 static pask_status_t append_common(pask_cache_t *c, int32_t layer, int32_t n_seqs, int32_t total_tokens,
                                    const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
                                    const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out,
-                                   pask_stream_t stream) {
+                                   pask_stream_t stream, const Workspace *fuse_ws = nullptr, bool *fused = nullptr) {
     if (!c || !seq_ids || !cu_tokens || !tags) return PASK_ERR_INVALID_ARG;
     if (layer < 0 || layer >= c->desc.n_layers) return PASK_ERR_INVALID_ARG;
     if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL || n_seqs > c->desc.max_seqs) return PASK_ERR_INVALID_ARG;
@@ -312,7 +312,7 @@ static pask_status_t append_common(pask_cache_t *c, int32_t layer, int32_t n_seq
     if (((uintptr_t)k | (uintptr_t)v) & 15) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)seq_ids | (uintptr_t)cu_tokens) & 3) return PASK_ERR_INVALID_ARG;
     return launch_append(c, layer, n_seqs, total_tokens, seq_ids, cu_tokens, k, v, tags, decided, actions_out,
-                         static_cast<cudaStream_t>(stream));
+                         static_cast<cudaStream_t>(stream), fuse_ws, fused);
 }
 
 pask_status_t pask_append_kv(pask_cache_t *c, int32_t layer, int32_t n_seqs, int32_t total_tokens,
@@ -343,14 +343,31 @@ pask_status_t pask_decide(pask_cache_t *c, int32_t n_seqs, int32_t total_tokens,
 
 static pask_status_t attention_common(pask_cache_t *c, bool has_low, int32_t layer, int32_t n_seqs,
                                       const int32_t *seq_ids, const void *q, float *out, float *lse, void *ws,
-                                      size_t ws_bytes, pask_stream_t stream) {
+                                      size_t ws_bytes, pask_stream_t stream, bool plan_done = false, bool check_only = false) {
     if (!c || !seq_ids || !q || !out || !ws) return PASK_ERR_INVALID_ARG;
     if (layer < 0 || layer >= c->desc.n_layers) return PASK_ERR_INVALID_ARG;
     if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)q | (uintptr_t)out) & 15 || ((uintptr_t)ws & 255) || ((uintptr_t)lse & 3)) return PASK_ERR_INVALID_ARG;
     if (ws_bytes < attention_workspace_bytes(c, n_seqs)) return PASK_ERR_WORKSPACE;
+    if (check_only) return PASK_OK;
     return launch_attention(c, has_low, layer, n_seqs, seq_ids, q, out, lse, ws, ws_bytes,
-                            static_cast<cudaStream_t>(stream));
+                            static_cast<cudaStream_t>(stream), plan_done);
+}
+
+pask_status_t pask_append_attend(pask_cache_t *c, int32_t layer, int32_t n_seqs, int32_t total_tokens,
+                                 const int32_t *seq_ids, const int32_t *cu_tokens, const void *k, const void *v,
+                                 const uint8_t *tags, const uint8_t *actions, uint8_t *actions_out, const void *q,
+                                 float *out, float *lse, void *ws, size_t ws_bytes, pask_stream_t stream) {
+    // every argument of the second call is checked before the first one is issued
+    pask_status_t rc = attention_common(c, true, layer, n_seqs, seq_ids, q, out, lse, ws, ws_bytes, stream, false, true);
+    if (rc != PASK_OK) return rc;
+    Workspace plan;
+    carve_workspace(c, n_seqs, static_cast<uint8_t *>(ws), &plan);
+    bool fused = false;
+    rc = append_common(c, layer, n_seqs, total_tokens, seq_ids, cu_tokens, k, v, tags, actions, actions_out, stream, &plan,
+                       &fused);
+    if (rc != PASK_OK) return rc;
+    return attention_common(c, true, layer, n_seqs, seq_ids, q, out, lse, ws, ws_bytes, stream, fused);
 }
 
 pask_status_t pask_decode_attention(pask_cache_t *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
@@ -415,9 +432,8 @@ pask_status_t pask_decode_step_host(pask_cache_t *c, int32_t layer, int32_t n_se
     if (e == cudaSuccess) e = cudaMemcpyAsync(d_q, q_host, q_bytes, cudaMemcpyHostToDevice, stream);
     if (e != cudaSuccess) return PASK_ERR_CUDA;
     iota_kernel<<<(n_seqs + 1 + 255) / 256, 256, 0, stream>>>(d_cu, n_seqs + 1);
-    pask_status_t rc = pask_append_kv(c, layer, n_seqs, n_seqs, d_ids, d_cu, d_k, d_v, d_tags, nullptr, nullptr, stream_v);
-    if (rc != PASK_OK) return rc;
-    rc = pask_decode_attention(c, layer, n_seqs, d_ids, d_q, d_out, nullptr, ws, ws_bytes, stream_v);
+    pask_status_t rc = pask_append_attend(c, layer, n_seqs, n_seqs, d_ids, d_cu, d_k, d_v, d_tags, nullptr, nullptr, d_q, d_out,
+                                          nullptr, ws, ws_bytes, stream_v);
     if (rc != PASK_OK) return rc;
     e = cudaMemcpyAsync(out_host, d_out, n * c->desc.n_q_heads * kHeadDim * 4, cudaMemcpyDeviceToHost, stream);
     return cuda_rc(e);

@@ -532,8 +532,9 @@ __global__ void __launch_bounds__(kSmallThreads)
 append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, const int32_t *__restrict__ seq_ids,
                     const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
                     const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided,
-                    uint8_t *__restrict__ actions_out, const SmallLut lut) {
+                    uint8_t *__restrict__ actions_out, const SmallLut lut, const int fuse_plan, const Workspace ws) {
     __shared__ int s_seq[kSmallMax], s_cu[kSmallMax + 1];
+    __shared__ uint32_t s_cost[kSmallMax + 1], s_page[kSmallMax + 1], s_nh[kSmallMax], s_nl[kSmallMax];   // fused attention plan
     __shared__ uint32_t s_old_n[kSmallMax];
     __shared__ uint32_t s_old_h[kSmallMax], s_old_l[kSmallMax], s_cnt_h[kSmallMax], s_cnt_l[kSmallMax], s_cnt_bad[kSmallMax];
     __shared__ uint32_t s_new_h[kSmallMax], s_new_l[kSmallMax], s_base_h[kSmallMax], s_base_l[kSmallMax];
@@ -590,6 +591,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             atomicOr(&c.ctrl[kCtrlStatus], s_err);
             if (atomicAdd(&c.ctrl[kCtrlTicket], 1u) == gridDim.x - 1) { c.ctrl[kCtrlPlanOk] = 0; c.ctrl[kCtrlTicket] = 0; }
         }
+        if (fuse_plan && blockIdx.x == 0 && tid <= n_seqs) ws.cost_prefix[tid] = ws.page_prefix[tid] = 0;   // nothing to attend
         return;
     }
     if (tid < total) {
@@ -669,6 +671,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             atomicOr(&c.ctrl[kCtrlStatus], s_err);
             if (s_last) { c.ctrl[kCtrlPlanOk] = 0; c.ctrl[kCtrlTicket] = 0; }
         }
+        if (fuse_plan && blockIdx.x == 0 && tid <= n_seqs) ws.cost_prefix[tid] = ws.page_prefix[tid] = 0;   // nothing to attend
         return;
     }
 
@@ -728,6 +731,70 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             if (tid == 0) c.win_act[my_sl * (size_t)W + slot] = (uint8_t)my_a;
         }
     }
+
+    // ---- fused decode-attention plan for the same sequences (what attn_plan_kernel would compute after
+    // this append): every CTA knows every sequence's lengths after the call and the ids of the pages the
+    // call allocates, so the plan needs nothing that the commit writes.  Only without a recent window.
+    if (!fuse_plan) return;
+    if (tid < n_seqs) { s_nh[tid] = s_old_h[tid] + s_cnt_h[tid]; s_nl[tid] = s_old_l[tid] + s_cnt_l[tid]; }
+    if (tid == 0) s_cost[0] = s_page[0] = 0;
+    __syncthreads();
+    if (tid < 32) {
+        uint32_t carry_c = 0, carry_p = 0;
+        for (int base = 0; base < n_seqs; base += 32) {
+            const int idx = base + tid;
+            uint32_t ph = 0, pl = 0;
+            if (idx < n_seqs) { ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens; pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens; }
+            uint32_t ic = ph * kCostHighPage + pl * kCostLowPage, ip = ph + pl;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t oc = __shfl_up_sync(0xffffffffu, ic, d), op = __shfl_up_sync(0xffffffffu, ip, d);
+                if (tid >= d) { ic += oc; ip += op; }
+            }
+            if (idx < n_seqs) { s_cost[idx + 1] = carry_c + ic; s_page[idx + 1] = carry_p + ip; }
+            carry_c += __shfl_sync(0xffffffffu, ic, 31);
+            carry_p += __shfl_sync(0xffffffffu, ip, 31);
+        }
+    }
+    __syncthreads();
+    if (blockIdx.x == 0) {
+        if (tid <= n_seqs) { ws.cost_prefix[tid] = s_cost[tid]; ws.page_prefix[tid] = s_page[tid]; }
+        if (tid < n_seqs) ws.tokens[tid] = make_uint2(s_nh[tid], s_nl[tid]);
+    }
+    const uint32_t total_pages = s_page[n_seqs];
+    for (uint32_t gp = blockIdx.x * kSmallThreads + tid; gp < total_pages; gp += gridDim.x * kSmallThreads) {
+        int a = 1, e = n_seqs;   // smallest idx in [1, n_seqs] with s_page[idx] > gp
+        while (a < e) {
+            const int mid = (a + e) >> 1;
+            if (s_page[mid] > gp) e = mid; else a = mid + 1;
+        }
+        const int s = a - 1;
+        const uint32_t nh = s_nh[s], nl = s_nl[s];
+        const uint32_t ph = (nh + kPageTokens - 1) / kPageTokens, pl = (nl + kPageTokens - 1) / kPageTokens;
+        const size_t sl = ((size_t)s_seq[s] * c.n_layers + layer) * c.max_pages;
+        uint32_t idx, entry;
+        if (page_at(gp - s_page[s], ph, pl, idx)) {
+            const uint32_t old_pages = (s_old_h[s] + kPageTokens - 1) / kPageTokens;
+            if (idx < old_pages) {
+                entry = c.tbl_high[sl + idx];
+            } else {             // a page this call allocates: the commit's formula
+                const uint32_t kk = s_base_h[s] + (idx - old_pages);
+                entry = kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]);
+            }
+            entry |= kOrderHigh;
+            if (idx == ph - 1) entry |= (nh & (kPageTokens - 1)) << kOrderValidShift;
+        } else {
+            const uint32_t old_pages = (s_old_l[s] + kPageTokens - 1) / kPageTokens;
+            if (idx < old_pages) {
+                entry = c.tbl_low[sl + idx];
+            } else {
+                const uint32_t kk = s_base_l[s] + (idx - old_pages);
+                entry = kk < s_ctrl[3] ? c.free_low[s_ctrl[3] - 1 - kk] : s_ctrl[2] + (kk - s_ctrl[3]);
+            }
+            if (idx == pl - 1) entry |= (nl & (kPageTokens - 1)) << kOrderValidShift;
+        }
+        ws.order[gp] = entry;
+    }
 }
 
 // General path, recent window: CTA (j, y) copies the y-th newest of sequence j's tokens in this call
@@ -783,16 +850,21 @@ __global__ void __launch_bounds__(256) seq_reset_kernel(DevCache c, int seq) {
 
 pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_tokens, const int32_t *seq_ids,
                             const int32_t *cu_tokens, const void *k, const void *v, const uint8_t *tags,
-                            const uint8_t *decided, uint8_t *actions_out, cudaStream_t stream) {
+                            const uint8_t *decided, uint8_t *actions_out, cudaStream_t stream, const Workspace *fuse_ws,
+                            bool *fused) {
+    if (fused) *fused = false;
     if (n_seqs <= kSmallMax && total_tokens <= kSmallMax) {
         SmallLut lut;
         const int group = c->layer_group[layer];
         for (int z = 0; z < 256; z++)
             lut.action[z] = z < c->dev.n_tags ? c->lut[(size_t)z * c->dev.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
         if (total_tokens == 0) return PASK_OK;
+        const int fuse = fuse_ws != nullptr && c->dev.window == 0;
+        if (fused) *fused = fuse != 0;
         const cudaError_t e = launch_pdl(append_small_kernel, dim3(total_tokens), dim3(kSmallThreads), 0, stream, c->dev, layer,
                                          group, n_seqs, total_tokens, seq_ids, cu_tokens, static_cast<const uint4 *>(k),
-                                         static_cast<const uint4 *>(v), tags, decided, actions_out, lut);
+                                         static_cast<const uint4 *>(v), tags, decided, actions_out, lut, fuse,
+                                         fuse ? *fuse_ws : Workspace{});
         return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
     }
     if (++c->append_serial == 0) c->append_serial = 1;

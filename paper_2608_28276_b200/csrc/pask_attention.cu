@@ -47,16 +47,6 @@ constexpr int kScratchBytes = 1152;              // per warp: fp16 query fragmen
 constexpr long long kWaitCycles = 2000000000LL;  // about one second: give up instead of hanging
 constexpr int kPlanThreads = 256;
 
-// workspace of one call
-struct Workspace {
-    uint32_t *cost_prefix;  // [n_seqs + 1] cost of the sequences before s
-    uint32_t *page_prefix;  // [n_seqs + 1] pages of the sequences before s
-    uint2 *tokens;          // [n_seqs] (n_high, n_low) tokens
-    uint32_t *order;        // [page_prefix[n_seqs]] pages in visiting order: kOrderHigh | tokens to attend << 27 | page id
-    float2 *part_ml;        // [slots][n_q] (reference maximum in log2 units, sum)
-    float *part_o;          // [slots][n_q][128] unnormalised outputs
-};
-
 struct AttnParams {
     DevCache c;
     int layer, n_seqs;
@@ -788,6 +778,8 @@ size_t attn_smem_bytes(int n_seqs, int n_warps) {
     return off + (size_t)n_warps * (kStages * kStageBytes + kScratchBytes);
 }
 
+}  // namespace
+
 // carve the caller's workspace
 size_t carve_workspace(const pask_cache *c, int n_seqs, uint8_t *base, Workspace *ws) {
     const size_t slots = (size_t)c->attn_ctas + n_seqs;
@@ -809,14 +801,13 @@ size_t carve_workspace(const pask_cache *c, int n_seqs, uint8_t *base, Workspace
     return off;
 }
 
-}  // namespace
 
 int attention_grid(const pask_cache *c) { return 2 * c->sm_count; }
 
 size_t attention_workspace_bytes(const pask_cache *c, int n_seqs) { return carve_workspace(c, n_seqs, nullptr, nullptr); }
 
 pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seqs, const int32_t *seq_ids, const void *q,
-                               float *out, float *lse, void *workspace, size_t, cudaStream_t stream) {
+                               float *out, float *lse, void *workspace, size_t, cudaStream_t stream, bool plan_done) {
     const int n_warps = c->desc.n_kv_heads;
     AttnParams p;
     p.c = c->dev;
@@ -829,8 +820,10 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
     auto kern = has_low ? decode_attn_kernel<true> : decode_attn_kernel<false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return PASK_ERR_CUDA;
-    cudaError_t e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(5 * n_seqs + 2) * 4, stream,
-                               c->dev, layer, n_seqs, seq_ids, p.ws, has_low ? 1 : 0);
+    cudaError_t e = cudaSuccess;
+    if (!plan_done)   // (a fused append has already left the plan in the workspace)
+        e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(5 * n_seqs + 2) * 4, stream, c->dev,
+                       layer, n_seqs, seq_ids, p.ws, has_low ? 1 : 0);
     if (c->ev_start) cudaEventRecord(c->ev_start, stream);
     if (e == cudaSuccess) e = launch_pdl(kern, dim3(c->attn_ctas), dim3(32 * n_warps), smem, stream, p);
     if (c->ev_stop) cudaEventRecord(c->ev_stop, stream);

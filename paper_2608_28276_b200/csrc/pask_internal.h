@@ -85,6 +85,16 @@ struct DevCache {
     uint32_t bytes_h, bytes_l;       // m(H), m(L) per token per layer
 };
 
+// workspace of one decode-attention call
+struct Workspace {
+    uint32_t *cost_prefix;  // [n_seqs + 1] cost of the sequences before s
+    uint32_t *page_prefix;  // [n_seqs + 1] pages of the sequences before s
+    uint2 *tokens;          // [n_seqs] (n_high, n_low) tokens attended from the two streams
+    uint32_t *order;        // [page_prefix[n_seqs]] pages in visiting order: kOrderHigh | tokens to attend << 27 | page id
+    float2 *part_ml;        // [slots][n_q] (reference maximum in log2 units, sum)
+    float *part_o;          // [slots][n_q][128] unnormalised outputs
+};
+
 struct MetaOffsets {
     size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, low_vmax, n_tok, win_act, plan, tok_list, item_base, lut,
         layer_group, dec_row, dec_rho, gamma, crit, total;
@@ -142,15 +152,19 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 #endif
 
 // launchers implemented next to their kernels
+// fuse_ws != nullptr: if the call goes down the one-launch path, that launch also writes the decode-attention plan for
+// the same sequences into *fuse_ws and *fused is set
 pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_tokens, const int32_t *seq_ids,
                             const int32_t *cu_tokens, const void *k, const void *v, const uint8_t *tags,
-                            const uint8_t *decided, uint8_t *actions_out, cudaStream_t stream);
+                            const uint8_t *decided, uint8_t *actions_out, cudaStream_t stream,
+                            const Workspace *fuse_ws = nullptr, bool *fused = nullptr);
 pask_status_t launch_decide(pask_cache *c, int n_seqs, int total_tokens, const int32_t *seq_ids, const int32_t *cu_tokens,
                             const uint8_t *tags, const uint16_t *states, uint8_t *actions_out, cudaStream_t stream);
 pask_status_t launch_seq_reset(pask_cache *c, int seq, cudaStream_t stream);
 pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seqs, const int32_t *seq_ids,
                                const void *q, float *out, float *lse, void *workspace, size_t workspace_bytes,
-                               cudaStream_t stream);
+                               cudaStream_t stream, bool plan_done = false);
+size_t carve_workspace(const pask_cache *c, int n_seqs, uint8_t *base, Workspace *ws);
 size_t attention_workspace_bytes(const pask_cache *c, int n_seqs);
 int attention_grid(const pask_cache *c);
 }  // namespace pask

@@ -1,0 +1,124 @@
+"""pask_append_attend (append + attention of one layer in one call; for small batches the append's
+launch also writes the attention plan) against the oracle and against the two separate calls."""
+import numpy as np
+import pytest
+import torch
+
+from pask_workloads import configs as WC
+from pask_workloads import policy as WP
+from pask_workloads.tensors import bf16_bits
+
+from parity import Pair, assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pask():
+    import paper_2608_28276_b200 as P      # fails loudly if libpask.so is missing
+    assert torch.cuda.is_available()
+    return P
+
+
+def _step(p, layer, seqs, counts, starts, acts=None):
+    """One fused call on the GPU side, the two steps on the oracle side; returns both outputs.
+    acts: (oracle actions, gpu actions) from Pair.decide for these tokens, or None (table actions)."""
+    d = "cuda"
+    tags, states, k, v = p.gather(seqs, counts, starts, layer)
+    cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    act_o, act_g = acts if acts else (None, None)
+    rc, used_o = p.orc.append(layer, seqs, cu, bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags, decided=act_o)
+    assert rc == 0
+    q = torch.stack([p.w.q(layer, int(s), int(t0 + n)) for s, n, t0 in zip(seqs, counts, starts)])
+    n = len(seqs)
+    out = torch.full((n, p.cfg.n_q, 128), float("nan"), dtype=torch.float32, device=d)
+    lse = torch.full((n, p.cfg.n_q), float("nan"), dtype=torch.float32, device=d)
+    used_g = torch.full((max(1, len(tags)),), 0xEE, dtype=torch.uint8, device=d)
+    ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+    p.pask.pask_append_attend(p.gpu.handle, layer, ids, torch.from_numpy(cu).to(d), k.to(d), v.to(d),
+                              torch.from_numpy(tags).to(d), q.to(d), out, lse, p.gpu.workspace(n), actions=act_g,
+                              actions_out=used_g, total_tokens=len(tags))
+    torch.cuda.synchronize()
+    assert np.array_equal(used_g.cpu().numpy()[:len(tags)], used_o)
+    oo, ol = p.orc.attention_batch(layer, seqs, bf16_bits(q).numpy())
+    go, gl = out.cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+    assert_close(go, gl, oo, ol, where=(layer, seqs))
+    return out, lse, (ids, torch.from_numpy(cu).to(d), k.to(d), v.to(d), torch.from_numpy(tags).to(d), q.to(d), act_g)
+
+
+def _pair(pask, oracle, batch, prompt, gen, window=0, dynamic=False, **kw):
+    from dataclasses import replace
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=batch, prompt_len=prompt, gen_len=gen, extra_gen=64)
+    w = WC.build(cfg)
+    blob = w.dynamic_blob(reserve_tokens=4, budget=0.3) if dynamic else WP.write_blob(replace(w.policy, recent_window=window))
+    if dynamic and window:
+        blob = blob[:28] + int(window).to_bytes(4, "little") + blob[32:]
+    return Pair(pask, oracle, w, blob=blob, **kw), w
+
+
+@pytest.mark.parametrize("batch,window,dynamic", [(5, 0, False), (64, 0, False), (7, 0, True), (5, 32, False), (130, 0, False)])
+def test_decode_steps(pask, oracle, batch, window, dynamic):
+    prompt, gen = (40, 24) if batch > 8 else (150, 70)
+    p, w = _pair(pask, oracle, batch, prompt, gen, window=window, dynamic=dynamic)
+    seqs = list(range(batch))
+    lens = [w.total_len(s) - (3 * s) % 17 for s in seqs]
+    if dynamic:
+        tags, states = p.gather(seqs, lens, [0] * batch)
+        _, act_o, act_g = p.decide(seqs, lens, tags, states)
+        for layer in range(w.cfg.n_layers):
+            _, _, k, v = p.gather(seqs, lens, [0] * batch, layer)
+            p.append_decided(layer, seqs, lens, k, v, tags, act_o, act_g)
+    else:
+        for layer in range(w.cfg.n_layers):
+            p.append(layer, seqs, lens, [0] * batch)
+    pos = list(lens)
+    ones = [1] * batch
+    for step in range(20):                                              # pages fill up and new ones are allocated on the way
+        order = seqs if step % 2 == 0 else seqs[::-1]
+        starts = [pos[s] for s in order]
+        acts = None
+        if dynamic:                                                     # Algorithm 2 steps 1-6 once per token, then every layer
+            tags, states = p.gather(order, ones, starts)
+            _, act_o, act_g = p.decide(order, ones, tags, states)
+            acts = (act_o, act_g)
+        for layer in range(w.cfg.n_layers):
+            _step(p, layer, order, ones, starts, acts)
+        pos = [x + 1 for x in pos]
+    p.compare_state()
+
+
+def test_ragged_small_batches_and_identity_with_separate_calls(pask, oracle):
+    p, w = _pair(pask, oracle, 4, 100, 60)
+    q2, _ = _pair(pask, oracle, 4, 100, 60)                             # second cache: the two separate calls
+    seqs = [3, 1, 0, 2]
+    pos = {s: 0 for s in seqs}
+    for counts in ([1, 1, 1, 1], [16, 3, 0, 31], [40, 40, 40, 8], [1, 0, 0, 2], [33, 17, 16, 15]):
+        starts = [pos[s] for s in seqs]
+        for layer in range(w.cfg.n_layers):
+            out, lse, (ids, cu, k, v, tags, q, _) = _step(p, layer, seqs, counts, starts)
+            pask.pask_append_kv(q2.gpu.handle, layer, ids, cu, k, v, tags, total_tokens=int(cu[-1]))
+            out2, lse2 = torch.empty_like(out), torch.empty_like(lse)
+            pask.pask_decode_attention(q2.gpu.handle, layer, ids, q, out2, lse2, q2.gpu.workspace(4))
+            torch.cuda.synchronize()
+            assert torch.equal(out, out2) and torch.equal(lse, lse2)    # same plan, same kernels: same bits
+        pos = {s: pos[s] + n for s, n in zip(seqs, counts)}
+    p.compare_state()
+
+
+def test_refused_append_inside_the_fused_call(pask, oracle):
+    p, w = _pair(pask, oracle, 2, 40, 20, pool_high_pages=1, pool_low_pages=1)
+    d = "cuda"
+    ids = torch.tensor([0, 1], dtype=torch.int32, device=d)
+    n = 100                                                             # needs more pages than either pool has
+    tags, states, k, v = p.gather([0, 1], [n, 20], [0, 0], 0)
+    cu = torch.tensor([0, n, n + 20], dtype=torch.int32, device=d)
+    q = torch.stack([w.q(0, s, 0) for s in (0, 1)]).to(d)
+    out = torch.zeros((2, w.cfg.n_q, 128), device=d)
+    lse = torch.zeros((2, w.cfg.n_q), device=d)
+    pask.pask_append_attend(p.gpu.handle, 0, ids, cu, k.to(d), v.to(d), torch.from_numpy(tags).to(d), q, out, lse,
+                            p.gpu.workspace(2), total_tokens=n + 20)
+    torch.cuda.synchronize()
+    st = pask.pask_budget_state(p.gpu.handle, 0)
+    assert st.device_status & pask.DEV_POOL_EXHAUSTED and st.full_bytes == 0
+    assert pask.pask_debug_stream_len(p.gpu.handle, 0, 0) == (0, 0)
+    assert pask.pask_debug_pool_state(p.gpu.handle) == (0, 0, 0, 0)
