@@ -208,6 +208,7 @@ class Job:
         self.out = torch.empty((self.B, cfg.n_q, 128), dtype=torch.float32, device=device)
         self.lse = torch.empty((self.B, cfg.n_q), dtype=torch.float32, device=device)
         self.attn = P.pask_decode_attention_full if policy_blob is not None else P.pask_decode_attention
+        self.fused = False
 
     def fill(self):
         """Append the whole history, one ragged bulk call per layer (generated on the device)."""
@@ -286,12 +287,16 @@ class Job:
         if self.dynamic:       # Algorithm 2 steps 1-6 once per token, then step 7 layer by layer
             P.pask_decide(h, self.ids, self.cu1, self.steps[s][0][3], self.step_states[s], self.decided)
         for layer, (k, v, q, tags) in enumerate(self.steps[s]):
+            if events is not None and layer in events:
+                P.pask_cache_set_timing_events(h, *events[layer])
+            if self.fused:     # the library's one-call form of append + attention for a layer
+                P.pask_append_attend(h, layer, self.ids, self.cu1, k, v, tags, q, self.out, self.lse, self.ws,
+                                     actions=self.decided if self.dynamic else None)
+                continue
             if self.dynamic:
                 P.pask_append_kv_decided(h, layer, self.ids, self.cu1, k, v, tags, self.decided)
             else:
                 P.pask_append_kv(h, layer, self.ids, self.cu1, k, v, tags)
-            if events is not None and layer in events:
-                P.pask_cache_set_timing_events(h, *events[layer])
             self.attn(h, layer, self.ids, q, self.out, self.lse, self.ws)
 
     def algorithmic_bytes_per_layer(self, steps_done=0):
@@ -339,6 +344,9 @@ def run_cuda(args, rank, world):
         w.policy = _replace(w.policy, recent_window=args.window)
     t_setup = time.time()
     job = Job(P, w, device, 2 * total_steps + e2e_steps + 4, dynamic=args.dynamic)
+    job.fused = not args.unfused
+    # launches per layer: append (+ plan), streaming kernel, combine
+    per_layer_launches = 3 if (job.fused and job.B <= 128 and not args.window) else 4
     job.fill()
     job.prepare_steps(total_steps)
     t_setup = time.time() - t_setup
@@ -387,29 +395,36 @@ def run_cuda(args, rank, world):
     e2e = None
     if (rank == 0 or world > 1) and not args.dynamic:   # the host-buffer entry point applies the frozen table
         staging = torch.empty(P.pask_step_staging_bytes(job.cache.handle, job.B), dtype=torch.uint8, device=device)
+        off, in_bytes = P.pask_step_packed_layout(job.cache.handle, job.B)
         host = []
-        for s in range(e2e_steps):
+        for s in range(e2e_steps):          # a layer's inputs sit in one pinned block, as an engine would stage them
             rows = []
             for layer in range(cfg.n_layers):
                 k, v, q, tags = step_inputs(w, layer, total_steps + s, "cpu")
-                rows.append((k.pin_memory(), v.pin_memory(), torch.from_numpy(tags).pin_memory(), q.pin_memory()))
+                block = torch.zeros(in_bytes, dtype=torch.uint8).pin_memory()
+                parts = [torch.arange(job.B, dtype=torch.int32), torch.arange(job.B + 1, dtype=torch.int32), k, v,
+                         torch.from_numpy(tags), q]
+                for o, t in zip(off, parts):
+                    raw = t.contiguous().view(torch.uint8).reshape(-1)
+                    block[o:o + raw.numel()] = raw
+                rows.append(block)
             host.append(rows)
-        ids_h = torch.arange(job.B, dtype=torch.int32).pin_memory()
         out_h = torch.empty((job.B, cfg.n_q, 128), dtype=torch.float32).pin_memory()
         barrier()
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0.record()
         for rows in host:
-            for layer, (k, v, tags, q) in enumerate(rows):
-                P.pask_decode_step_host(job.cache.handle, layer, ids_h, k, v, tags, q, out_h, staging, job.ws)
+            for layer, block in enumerate(rows):
+                P.pask_decode_step_packed(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
         t1.record()
         barrier()
         e_ms = t0.elapsed_time(t1)
         e_ms = max_over_ranks(e_ms, device)
-        h2d = cfg.n_layers * (job.B * 4 + 2 * job.B * cfg.n_kv * 256 + job.B + job.B * cfg.n_q * 256)
+        h2d = cfg.n_layers * in_bytes
         d2h = cfg.n_layers * job.B * cfg.n_q * 128 * 4
         e2e = {"value": whole_job_tokens_per_s(world, job.B, e2e_steps, e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps}
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps,
+               "api": "pask_decode_step_packed: one pinned host block in, attention output out, per layer"}
 
     if rank != 0:
         return
@@ -431,7 +446,7 @@ def run_cuda(args, rank, world):
                    "setup_s": round(t_setup, 1)},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": (4 * cfg.n_layers + (1 if args.dynamic else 0)) * args.steps,
+        "gpu_launches": (per_layer_launches * cfg.n_layers + (1 if args.dynamic else 0)) * args.steps,
         "roofline": {"bound": "hbm", "kernel": "decode_attn_kernel<true>", "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "algorithmic_bytes_per_launch": alg,
@@ -596,6 +611,8 @@ def main():
     ap.add_argument("--no-full-kv", dest="full_kv", action="store_false")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="0 skips the CPU-oracle leg")
     ap.add_argument("--event-stride", type=int, default=4, help="time the streaming kernel of every n-th launch")
+    ap.add_argument("--unfused", action="store_true",
+                    help="issue pask_append_kv and pask_decode_attention separately instead of pask_append_attend")
     ap.add_argument("--window", type=int, default=0, help="protected recent window in tokens (multiple of 16, <= 256)")
     ap.add_argument("--graph", action="store_true", help="replay each timed step as one CUDA graph (launch-bound shapes)")
     ap.add_argument("--dynamic", action="store_true",

@@ -314,6 +314,15 @@ pask_status_t pask_decode_step_host(pask_cache_t *cache, int32_t layer, int32_t 
                                     const void *q_host, float *out_host, void *staging, size_t staging_bytes,
                                     void *workspace, size_t workspace_bytes, pask_stream_t stream);
 size_t pask_step_staging_bytes(const pask_cache_t *cache, int32_t n_seqs);
+/* The same step from ONE host block (one host-to-device copy instead of five): the caller lays the
+ * step's inputs out in a pinned block at the byte offsets pask_step_packed_layout returns --
+ * offsets[0..5] = seq_ids (int32 [n]), cu_tokens (int32 [n+1] = 0, 1, ..., n), k, v (bf16
+ * [n][n_kv][128]), tags (u8 [n]), q (bf16 [n][n_q][128]); *in_bytes is the size of the block.
+ * staging and workspace as for pask_decode_step_host. */
+pask_status_t pask_step_packed_layout(const pask_cache_t *cache, int32_t n_seqs, size_t offsets[6], size_t *in_bytes);
+pask_status_t pask_decode_step_packed(pask_cache_t *cache, int32_t layer, int32_t n_seqs, const void *packed_host,
+                                      float *out_host, void *staging, size_t staging_bytes, void *workspace,
+                                      size_t workspace_bytes, pask_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------------
  * pask_distortion -- the inner term of the attention-output distortion (Eq. 4): for each row r

@@ -29,7 +29,7 @@ EXPORTS = [
     "pask_load_policy", "pask_free_policy", "pask_policy_action", "pask_cache_sizes", "pask_cache_create",
     "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decide",
     "pask_append_kv_decided", "pask_append_attend", "pask_decode_attention",
-    "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes",
+    "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes", "pask_step_packed_layout", "pask_decode_step_packed",
     "pask_budget_state", "pask_distortion", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
     "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
 ]
@@ -83,6 +83,8 @@ _lib.pask_decode_attention_static.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _v
 _lib.pask_workspace_bytes.argtypes = [_vp, _i32]
 _lib.pask_workspace_bytes.restype = _sz
 _lib.pask_decode_step_host.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
+_lib.pask_step_packed_layout.argtypes = [_vp, _i32, C.POINTER(_sz * 6), C.POINTER(_sz)]
+_lib.pask_decode_step_packed.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
 _lib.pask_step_staging_bytes.argtypes = [_vp, _i32]
 _lib.pask_step_staging_bytes.restype = _sz
 _lib.pask_distortion.argtypes = [_i32, _i32, _vp, _vp, _vp, _vp, _vp]
@@ -263,6 +265,22 @@ def pask_distortion(o_ref, o_test, per_row_out=None, sum_inout=None, stream=None
     _check(_lib.pask_distortion(o_ref.shape[0], o_ref.shape[1], _dptr(o_ref, torch.float32), _dptr(o_test, torch.float32),
                                 _dptr(per_row_out, torch.float32), _dptr(sum_inout, torch.float64), _stream(stream)),
            "pask_distortion")
+
+
+def pask_step_packed_layout(cache: int, n_seqs: int):
+    """(offsets of seq_ids, cu_tokens, k, v, tags, q in the packed host block; its size in bytes)."""
+    off, n = (_sz * 6)(), _sz(0)
+    _check(_lib.pask_step_packed_layout(cache, n_seqs, C.byref(off), C.byref(n)), "pask_step_packed_layout")
+    return [int(x) for x in off], int(n.value)
+
+
+def pask_decode_step_packed(cache: int, layer: int, n_seqs: int, packed_host, out_host, staging, workspace, stream=None):
+    """packed_host: CPU uint8 tensor (pinned) laid out per pask_step_packed_layout; out_host CPU fp32."""
+    assert not packed_host.is_cuda and packed_host.is_contiguous() and not out_host.is_cuda and out_host.is_contiguous()
+    _check(_lib.pask_decode_step_packed(cache, layer, n_seqs, packed_host.data_ptr(), out_host.data_ptr(), _dptr(staging),
+                                        staging.numel() * staging.element_size(), _dptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream)),
+           "pask_decode_step_packed")
 
 
 def pask_budget_state(cache: int, seq: int, stream=None) -> BudgetState:

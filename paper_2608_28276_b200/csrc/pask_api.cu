@@ -439,6 +439,41 @@ pask_status_t pask_decode_step_host(pask_cache_t *c, int32_t layer, int32_t n_se
     return cuda_rc(e);
 }
 
+pask_status_t pask_step_packed_layout(const pask_cache_t *c, int32_t n_seqs, size_t offsets[6], size_t *in_bytes) {
+    if (!c || n_seqs < 1 || !offsets || !in_bytes) return PASK_ERR_INVALID_ARG;
+    const size_t n = (size_t)n_seqs;
+    const size_t kv_bytes = n * c->desc.n_kv_heads * kHeadDim * 2, q_bytes = n * c->desc.n_q_heads * kHeadDim * 2;
+    size_t p = 0;
+    offsets[0] = p; p += align_up(n * 4, 256);          // seq_ids
+    offsets[1] = p; p += align_up((n + 1) * 4, 256);    // cu_tokens
+    offsets[2] = p; p += align_up(kv_bytes, 256);       // k
+    offsets[3] = p; p += align_up(kv_bytes, 256);       // v
+    offsets[4] = p; p += align_up(n, 256);              // tags
+    offsets[5] = p; p += align_up(q_bytes, 256);        // q
+    *in_bytes = p;
+    return PASK_OK;
+}
+
+pask_status_t pask_decode_step_packed(pask_cache_t *c, int32_t layer, int32_t n_seqs, const void *packed_host,
+                                      float *out_host, void *staging, size_t staging_bytes, void *ws, size_t ws_bytes,
+                                      pask_stream_t stream_v) {
+    if (!c || !packed_host || !out_host || !staging) return PASK_ERR_INVALID_ARG;
+    if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL) return PASK_ERR_INVALID_ARG;
+    if (((uintptr_t)staging & 255) || staging_bytes < pask_step_staging_bytes(c, n_seqs)) return PASK_ERR_WORKSPACE;
+    size_t off[6], in_bytes = 0;
+    pask_step_packed_layout(c, n_seqs, off, &in_bytes);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    uint8_t *p = static_cast<uint8_t *>(staging);
+    if (cudaMemcpyAsync(p, packed_host, in_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return PASK_ERR_CUDA;
+    float *d_out = reinterpret_cast<float *>(p + in_bytes);
+    pask_status_t rc = pask_append_attend(c, layer, n_seqs, n_seqs, reinterpret_cast<const int32_t *>(p + off[0]),
+                                          reinterpret_cast<const int32_t *>(p + off[1]), p + off[2], p + off[3], p + off[4],
+                                          nullptr, nullptr, p + off[5], d_out, nullptr, ws, ws_bytes, stream_v);
+    if (rc != PASK_OK) return rc;
+    return cuda_rc(cudaMemcpyAsync(out_host, d_out, (size_t)n_seqs * c->desc.n_q_heads * kHeadDim * 4, cudaMemcpyDeviceToHost,
+                                   stream));
+}
+
 pask_status_t pask_budget_state(pask_cache_t *c, int32_t seq, pask_budget_state_t *host_out, pask_stream_t stream_v) {
     if (!c || !host_out) return PASK_ERR_INVALID_ARG;
     if (seq < 0 || seq >= c->desc.max_seqs) return PASK_ERR_BAD_SEQ;

@@ -304,3 +304,33 @@ def test_decode_step_from_host_buffers(pask, oracle):
     go = out.numpy().astype(np.float64)
     assert_close(go, ol.copy(), oo, ol)
     p.compare_state()
+
+
+def test_decode_step_from_one_packed_host_block(pask, oracle):
+    # the same step with all inputs in one pinned block (one host-to-device copy)
+    from pask_workloads.tensors import bf16_bits
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=4, n_layers=1, n_groups=1, prompt_len=200, gen_len=100)
+    w = WC.build(cfg)
+    p = Pair(pask, oracle, w)
+    seqs = [2, 0, 3, 1]
+    p.append(0, seqs, [300] * 4, [0] * 4)
+    P, h = pask, p.gpu.handle
+    k = torch.stack([w.kv(0, b, 300, 1)[0][0] for b in seqs])
+    v = torch.stack([w.kv(0, b, 300, 1)[1][0] for b in seqs])
+    tags = torch.from_numpy(np.array([w.tags(b, 300, 1)[0] for b in seqs], np.uint8))
+    q = torch.stack([w.q(0, b, 301) for b in seqs])
+    off, n_in = P.pask_step_packed_layout(h, 4)
+    block = torch.zeros(n_in, dtype=torch.uint8).pin_memory()
+    parts = [torch.tensor(seqs, dtype=torch.int32), torch.arange(5, dtype=torch.int32), k, v, tags, q]
+    for o, t in zip(off, parts):
+        raw = t.contiguous().view(torch.uint8).reshape(-1)
+        block[o:o + raw.numel()] = raw
+    out = torch.empty((4, 32, 128), dtype=torch.float32).pin_memory()
+    staging = torch.empty(P.pask_step_staging_bytes(h, 4), dtype=torch.uint8, device="cuda")
+    P.pask_decode_step_packed(h, 0, 4, block, out, staging, p.gpu.workspace(4))
+    torch.cuda.synchronize()
+    rc, _ = p.orc.append(0, seqs, [0, 1, 2, 3, 4], bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags.numpy())
+    assert rc == 0
+    oo, ol = p.orc.attention_batch(0, seqs, bf16_bits(q).numpy())
+    assert_close(out.numpy().astype(np.float64), ol.copy(), oo, ol)
+    p.compare_state()
