@@ -48,3 +48,20 @@ def test_shape(pask, oracle, n_kv, window):
         p.append(layer, seqs, [14, 14, 14], [pos[s] for s in seqs], expect_ok=True)
     p.compare_state()
     p.check_attention(1, [0, 1, 2], pos=pos[0] + 14)
+
+
+def test_largest_call_1024_sequences(pask, oracle):
+    # PASK_MAX_SEQS_PER_CALL sequences in one append and one attention call, some of them empty
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, n_kv=2, n_q=8, n_layers=1, n_groups=1, batch=1024, prompt_len=20, gen_len=20,
+                    extra_gen=8)
+    w = WC.build(cfg)
+    p = Pair(pask, oracle, w)
+    seqs = list(range(1023, -1, -1))
+    counts = [0 if s % 97 == 0 else 17 + s % 23 for s in seqs]
+    p.append(0, seqs, counts, [0] * 1024)
+    for step in range(3):
+        p.append(0, seqs, [1] * 1024, [c + step for c in counts])
+    p.compare_state(seqs=[0, 1, 96, 97, 500, 1023])
+    assert pask.pask_debug_pool_state(p.gpu.handle) == p.orc.pool_state()
+    p.check_attention(0, list(range(1024)), pos=40)
+    p.check_attention(0, seqs[:300], pos=40)
