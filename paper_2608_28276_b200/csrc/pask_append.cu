@@ -524,7 +524,7 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
 // shared memory (decisions, ranks, page allocation by a scan); then it writes its own token.  All
 // CTAs only read the cache state while planning; the CTA that finishes planning last (arrival
 // counter, nobody waits) commits the counters, tables and budget states for everybody.
-constexpr int kSmallMax = 128;       // at most this many sequences and tokens
+constexpr int kSmallMax = 255;       // at most this many sequences and tokens (one thread each, index n_seqs included)
 constexpr int kSmallThreads = 256;
 struct SmallLut { uint8_t action[256]; };
 

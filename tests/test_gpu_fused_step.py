@@ -56,7 +56,7 @@ def _pair(pask, oracle, batch, prompt, gen, window=0, dynamic=False, **kw):
     return Pair(pask, oracle, w, blob=blob, **kw), w
 
 
-@pytest.mark.parametrize("batch,window,dynamic", [(5, 0, False), (64, 0, False), (7, 0, True), (5, 32, False), (130, 0, False)])
+@pytest.mark.parametrize("batch,window,dynamic", [(5, 0, False), (64, 0, False), (7, 0, True), (5, 32, False), (130, 0, False), (255, 0, False), (256, 0, False)])
 def test_decode_steps(pask, oracle, batch, window, dynamic):
     prompt, gen = (40, 24) if batch > 8 else (150, 70)
     p, w = _pair(pask, oracle, batch, prompt, gen, window=window, dynamic=dynamic)
