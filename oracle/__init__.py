@@ -40,6 +40,8 @@ def lib():
         L.orc_f16_to_f32.argtypes = [C.c_uint16]
         L.orc_quantize_group.argtypes = [vp, vp, vp]
         L.orc_quantize_group.restype = None
+        L.orc_quantize_group_bits.argtypes = [vp, vp, vp, i32]
+        L.orc_quantize_group_bits.restype = None
         L.orc_lut_fold.argtypes = [i32, i32]
         L.orc_policy_load.restype = vp
         L.orc_policy_load.argtypes = [C.c_char_p, C.c_size_t, C.POINTER(C.c_int)]
@@ -82,13 +84,13 @@ def f16_bits_to_f32(h: int) -> float:
     return float(lib().orc_f16_to_f32(C.c_uint16(h)))
 
 
-def quantize_group(x_bits: np.ndarray):
-    """32 bf16 bit patterns -> (fp16 scale bit pattern, 32 codes)."""
+def quantize_group(x_bits: np.ndarray, bits: int = 4):
+    """32 bf16 bit patterns -> (fp16 scale bit pattern, 32 codes); bits = 4 or 8."""
     x = np.ascontiguousarray(x_bits, dtype=np.uint16)
     assert x.shape == (32,)
     s = np.zeros(1, np.uint16)
     c = np.zeros(32, np.uint8)
-    lib().orc_quantize_group(_ptr(x), _ptr(s), _ptr(c))
+    lib().orc_quantize_group_bits(_ptr(x), _ptr(s), _ptr(c), bits)
     return int(s[0]), c
 
 

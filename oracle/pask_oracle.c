@@ -26,7 +26,8 @@
  * Readings where the paper is silent (the low-precision format, paging, budget units, unknown
  * tags) are the library's documented ones: RETAIN-LOW is symmetric int4 per token, per KV head,
  * per group of 32 consecutive head dimensions with one fp16 scale (amax/7, round to nearest
- * even, codes stored offset by 8); RETAIN-HIGH keeps the bf16 bits; pages hold 16 tokens and
+ * even, codes stored offset by 8) -- or, policy low_bits = 8, symmetric int8 in the same grouping
+ * (amax/127, codes offset by 128); RETAIN-HIGH keeps the bf16 bits; pages hold 16 tokens and
  * are handed out in call order from a per-pool free stack, else a bump counter; costs are
  * payload bytes.  Parity unpinned by the paper for: the low-bit format itself, the size of the
  * recent window (a policy parameter here, 0 by default; the paper gives no number) and that a
@@ -165,28 +166,36 @@ float orc_f16_to_f32(uint16_t h) {
     return mag;
 }
 
-/* RETAIN-LOW of one group of 32 values (bf16 bit patterns in): one fp16 scale, 32 codes. */
-void orc_quantize_group(const uint16_t *x_bits, uint16_t *scale_bits, uint8_t *codes) {
+/* RETAIN-LOW of one group of 32 values (bf16 bit patterns in): one fp16 scale, 32 codes.
+ * bits = 4: codes clamp(rint(x / s), -7, 7) + 8 with s = fp16(amax / 7);
+ * bits = 8: codes clamp(rint(x / s), -127, 127) + 128 with s = fp16(amax / 127). */
+void orc_quantize_group_bits(const uint16_t *x_bits, uint16_t *scale_bits, uint8_t *codes, int bits) {
+    const float qmax = bits == 8 ? 127.0f : 7.0f;
+    const int zero = bits == 8 ? 128 : 8;
     float amax = 0.0f;
     for (int i = 0; i < QGROUP; i++) {
         float a = fabsf(bf16_to_f32(x_bits[i]));
         if (a > amax) amax = a;
     }
-    float s32 = amax / 7.0f;
+    float s32 = amax / qmax;
     uint16_t sh = orc_f32_to_f16_rne(s32);
     float s = orc_f16_to_f32(sh);
     *scale_bits = sh;
     if (s == 0.0f) {
-        for (int i = 0; i < QGROUP; i++) codes[i] = 8;
+        for (int i = 0; i < QGROUP; i++) codes[i] = (uint8_t)zero;
         return;
     }
     float inv = 1.0f / s;
     for (int i = 0; i < QGROUP; i++) {
         float r = rintf(bf16_to_f32(x_bits[i]) * inv); /* ties to even in the default mode */
-        if (r > 7.0f) r = 7.0f;
-        if (r < -7.0f) r = -7.0f;
-        codes[i] = (uint8_t)((int)r + 8);
+        if (r > qmax) r = qmax;
+        if (r < -qmax) r = -qmax;
+        codes[i] = (uint8_t)((int)r + zero);
     }
+}
+
+void orc_quantize_group(const uint16_t *x_bits, uint16_t *scale_bits, uint8_t *codes) {
+    orc_quantize_group_bits(x_bits, scale_bits, codes, 4);
 }
 
 /* ------------------------------------------------------------------ policy */
@@ -215,7 +224,7 @@ orc_policy *orc_policy_load(const uint8_t *blob, size_t len, int *err) {
     p->low_bits = rd32(blob + 32); p->group_size = rd32(blob + 36);
     if (p->n_tags == 0 || p->n_tags > 255 || p->n_groups == 0 || p->n_groups > MAX_GROUPS ||
         p->n_layers == 0 || p->n_layers > 4096 || p->n_states > (1u << 20) || p->recent_window % PAGE_TOKENS != 0 || p->recent_window > MAX_WINDOW ||
-        p->low_bits != 4 || p->group_size != QGROUP) { free(p); return NULL; }
+        (p->low_bits != 4 && p->low_bits != 8) || p->group_size != QGROUP) { free(p); return NULL; }
     size_t lg_pad = (p->n_layers + 3u) & ~(size_t)3u;
     size_t n_ent = (size_t)p->n_tags * p->n_groups;
     size_t need = 40 + lg_pad + n_ent * 12 + (size_t)p->n_states * 4;
@@ -253,7 +262,9 @@ int orc_policy_action(const orc_policy *p, int tag, int group) { return p->eff[(
 /* ------------------------------------------------------------------ cache */
 
 static uint64_t bytes_high(const orc_cache *c) { return 2ull * c->n_kv * HEAD_DIM * 2; }
-static uint64_t bytes_low(const orc_cache *c) { return 2ull * c->n_kv * (HEAD_DIM / 2 + GROUPS_PER_HEAD * 2); }
+static uint64_t bytes_low(const orc_cache *c) {   /* codes at low_bits each, one fp16 scale per group */
+    return 2ull * c->n_kv * (HEAD_DIM * c->pol->low_bits / 8 + GROUPS_PER_HEAD * 2);
+}
 
 static void pool_init(orc_pool *p, uint32_t cap) {
     p->cap = cap; p->next = 0; p->n_free = 0;
@@ -406,10 +417,10 @@ int orc_append_decided(orc_cache *c, int layer, int n_seqs, const int32_t *seq_i
                     GROW(s->lvs, s->cap_low, pos + 1, srow * 2);
                 }
                 for (size_t g = 0; g < srow; g++) {
-                    orc_quantize_group(k_bits + (size_t)t * row + g * QGROUP, s->lks + (size_t)pos * srow + g,
-                                       s->lk + (size_t)pos * row + g * QGROUP);
-                    orc_quantize_group(v_bits + (size_t)t * row + g * QGROUP, s->lvs + (size_t)pos * srow + g,
-                                       s->lv + (size_t)pos * row + g * QGROUP);
+                    orc_quantize_group_bits(k_bits + (size_t)t * row + g * QGROUP, s->lks + (size_t)pos * srow + g,
+                                            s->lk + (size_t)pos * row + g * QGROUP, (int)p->low_bits);
+                    orc_quantize_group_bits(v_bits + (size_t)t * row + g * QGROUP, s->lvs + (size_t)pos * srow + g,
+                                            s->lv + (size_t)pos * row + g * QGROUP, (int)p->low_bits);
                 }
                 s->n_low++;
                 b->n_low[group]++;
@@ -596,6 +607,7 @@ static void attention_head(orc_cache *c, int layer, int seq, int h, const uint16
     orc_stream *s = stream_of(c, seq, layer);
     const int kv = h / (c->n_q / c->n_kv);
     const size_t row = (size_t)c->n_kv * HEAD_DIM, srow = (size_t)c->n_kv * GROUPS_PER_HEAD;
+    const int zero = c->pol->low_bits == 8 ? 128 : 8;                 /* the code that stands for 0 */
     const uint32_t W = c->pol->recent_window;
     const size_t nw = W ? (s->n_tok < W ? s->n_tok : W) : 0;          /* tokens in the window */
     size_t win_h = 0, win_l = 0;
@@ -620,7 +632,7 @@ static void attention_head(orc_cache *c, int layer, int seq, int h, const uint16
             const uint8_t *kc = s->lk + jl * row + (size_t)kv * HEAD_DIM;
             const uint16_t *ks = s->lks + jl * srow + (size_t)kv * GROUPS_PER_HEAD;
             for (int i = 0; i < HEAD_DIM; i++)
-                dot += q[i] * ((double)((int)kc[i] - 8) * (double)orc_f16_to_f32(ks[i / QGROUP]));
+                dot += q[i] * ((double)((int)kc[i] - zero) * (double)orc_f16_to_f32(ks[i / QGROUP]));
         }
         score[j] = dot * inv_sqrt_d;
         if (score[j] > m) m = score[j];
@@ -642,7 +654,7 @@ static void attention_head(orc_cache *c, int layer, int seq, int h, const uint16
             const uint8_t *vc = s->lv + jl * row + (size_t)kv * HEAD_DIM;
             const uint16_t *vs = s->lvs + jl * srow + (size_t)kv * GROUPS_PER_HEAD;
             for (int i = 0; i < HEAD_DIM; i++)
-                acc[i] += pj * ((double)((int)vc[i] - 8) * (double)orc_f16_to_f32(vs[i / QGROUP]));
+                acc[i] += pj * ((double)((int)vc[i] - zero) * (double)orc_f16_to_f32(vs[i / QGROUP]));
         }
     }
     for (int i = 0; i < HEAD_DIM; i++) out[i] = n ? acc[i] / denom : 0.0;

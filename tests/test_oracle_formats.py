@@ -146,3 +146,54 @@ def test_action_cost_table_matches_formats():
         assert h == 2 * n_kv * 128 * 2                      # K and V, bf16
         assert l == 2 * n_kv * (128 // 2 + (128 // 32) * 2)  # nibbles + one fp16 scale per 32 values
         assert 0 < l < h and abs(l / h - 0.28125) < 1e-12
+
+
+# ---- the 8-bit variant of RETAIN-LOW (policy low_bits = 8): same recipe with 127 in place of 7
+
+def test_quantizer8_invariants_and_exact_nearest(oracle):
+    for scale in (1.0, 1e-3, 1e3):
+        for xb in _groups(21, 1500, scale):
+            x = _bf16_val(xb).astype(np.float64)
+            sb, codes = oracle.quantize_group(xb, bits=8)
+            s = float(np.array([sb], np.uint16).view(np.float16)[0])
+            assert codes.min() >= 1 and codes.max() <= 255
+            assert sb == int(np.float16(np.float32(np.abs(x).max()) / np.float32(127.0)).view(np.uint16))
+            xh = (codes.astype(np.int64) - 128) * s
+            assert np.all(np.abs(x - xh) <= 0.5 * s * (1 + 2.0 ** -9) + 1e-30)
+    for xb in _groups(22, 300):
+        sb, codes = oracle.quantize_group(xb, bits=8)
+        s = Fraction(float(np.array([sb], np.uint16).view(np.float16)[0]))
+        for xi, c in zip(_bf16_val(xb), codes):
+            r = max(Fraction(-127), min(Fraction(127), Fraction(float(xi)) / s))
+            assert abs(r - (int(c) - 128)) <= Fraction(1, 2) + Fraction(1, 1 << 16)
+
+
+def test_quantizer8_degenerate_groups_and_symmetry(oracle):
+    sb, codes = oracle.quantize_group(np.zeros(32, np.uint16), bits=8)
+    assert sb == 0 and np.all(codes == 128)
+    xb = _bf16_bits(np.full(32, 1e-9, np.float32))                  # scale underflows to zero
+    sb, codes = oracle.quantize_group(xb, bits=8)
+    assert sb == 0 and np.all(codes == 128)
+    xb = _bf16_bits(np.array([1e7, -1e7] * 16, np.float32))         # scale saturates, codes clamp
+    sb, codes = oracle.quantize_group(xb, bits=8)
+    assert sb == 0x7BFF and set(codes.tolist()) == {1, 255}
+    xb = _bf16_bits(np.full(32, 127.0, np.float32))                 # scale exactly 1: codes are the values
+    sb, codes = oracle.quantize_group(xb, bits=8)
+    assert sb == 0x3C00 and np.all(codes == 255)
+    xb = _bf16_bits(np.arange(-16, 16, dtype=np.float32) * 8 - 1)   # amax 129 -> not a clean scale; still symmetric
+    for xb in _groups(23, 300):
+        sb, codes = oracle.quantize_group(xb, bits=8)
+        sb2, codes2 = oracle.quantize_group(xb ^ np.uint16(0x8000), bits=8)
+        assert sb == sb2 and np.array_equal(codes2.astype(np.int64) - 128, -(codes.astype(np.int64) - 128))
+
+
+def test_eight_bit_is_finer_than_four_bit(oracle):
+    # the same group at both widths: the 8-bit reconstruction error is never larger than half a 4-bit step
+    for xb in _groups(24, 300):
+        x = _bf16_val(xb).astype(np.float64)
+        s4, c4 = oracle.quantize_group(xb, bits=4)
+        s8, c8 = oracle.quantize_group(xb, bits=8)
+        f = lambda b: float(np.array([b], np.uint16).view(np.float16)[0])
+        e4 = np.abs(x - (c4.astype(np.int64) - 8) * f(s4)).max()
+        e8 = np.abs(x - (c8.astype(np.int64) - 128) * f(s8)).max()
+        assert e8 <= e4 + 1e-12 and e8 <= 0.5 * f(s8) * (1 + 2.0 ** -9)
