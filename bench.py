@@ -200,8 +200,10 @@ class Job:
         self.lens = [w.total_len(b) for b in range(self.B)]
         self.total_tokens = int(sum(self.lens))
         self.window = int.from_bytes(blob[28:32], "little")
+        self.low_bits = int.from_bytes(blob[32:36], "little")
         self.cache = P.Cache(blob, cfg.n_layers, cfg.n_q, cfg.n_kv, self.B, max(self.lens) + extra + 16,
-                             self.total_tokens, pages_h, pages_l, device=device, recent_window=self.window)
+                             self.total_tokens, pages_h, pages_l, device=device, recent_window=self.window,
+                             low_bits=self.low_bits)
         self.ids = torch.arange(self.B, dtype=torch.int32, device=device)
         self.cu1 = torch.arange(self.B + 1, dtype=torch.int32, device=device)
         self.ws = self.cache.workspace(self.B)
@@ -317,7 +319,7 @@ class Job:
                 win_h[b], win_l[b] = (acts == 2).sum(0), (acts == 1).sum(0)
         for l in range(cfg.n_layers):
             nh, nl = self.nh[:, lg[l]] + steps_done - win_h[:, lg[l]] + self.window, self.nl[:, lg[l]] - win_l[:, lg[l]]
-            tot += float((nh * cfg.n_kv * 512).sum() + (nl * cfg.n_kv * 144).sum())
+            tot += float((nh * cfg.n_kv * 512).sum() + (nl * cfg.n_kv * (272 if self.low_bits == 8 else 144)).sum())
             tot += float((((nh + 15) // 16) + ((nl + 15) // 16)).sum() * 4)
         per_layer = tot / cfg.n_layers
         per_layer += self.B * cfg.n_q * 128 * 2
@@ -333,6 +335,8 @@ def run_cuda(args, rank, world):
     if args.budget is not None or args.bias != "balanced":
         cfg = WC.scaled(cfg, budget=args.budget if args.budget is not None else cfg.budget, bias=args.bias,
                         lut="all_high" if (args.budget or 0) >= 1.0 else cfg.lut)
+    if args.low_bits != 4:
+        cfg = WC.scaled(cfg, low_bits=args.low_bits, name=f"{cfg.name}[{args.low_bits}-bit low]")
     if args.layers:
         cfg = WC.scaled(cfg, n_layers=args.layers, name=f"{cfg.name}[first {args.layers} layers]")
     total_steps = args.warmup + args.steps
@@ -447,7 +451,7 @@ def run_cuda(args, rank, world):
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": (per_layer_launches * cfg.n_layers + (1 if args.dynamic else 0)) * args.steps,
-        "roofline": {"bound": "hbm", "kernel": "decode_attn_kernel<true>", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": f"decode_attn_kernel<{job.low_bits}>", "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "algorithmic_bytes_per_launch": alg,
                      "avg_launch_ms": k_ms, "launches_timed": len(kern_ms), "traffic": alg * NCU_TRAFFIC_RATIO,
@@ -611,6 +615,7 @@ def main():
     ap.add_argument("--no-full-kv", dest="full_kv", action="store_false")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="0 skips the CPU-oracle leg")
     ap.add_argument("--event-stride", type=int, default=4, help="time the streaming kernel of every n-th launch")
+    ap.add_argument("--low-bits", type=int, default=4, choices=[4, 8], help="width of the RETAIN-LOW codes")
     ap.add_argument("--unfused", action="store_true",
                     help="issue pask_append_kv and pask_decode_attention separately instead of pask_append_attend")
     ap.add_argument("--window", type=int, default=0, help="protected recent window in tokens (multiple of 16, <= 256)")

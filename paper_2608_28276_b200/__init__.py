@@ -39,7 +39,8 @@ class CacheDesc(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("page_tokens", C.c_int32), ("max_seqs", C.c_int32),
                 ("max_tokens_per_seq", C.c_int32), ("max_append_tokens", C.c_int32),
-                ("pool_high_pages", C.c_uint32), ("pool_low_pages", C.c_uint32), ("recent_window", C.c_int32)]
+                ("pool_high_pages", C.c_uint32), ("pool_low_pages", C.c_uint32), ("recent_window", C.c_int32),
+                ("low_bits", C.c_int32)]
 
 
 class CacheSizes(C.Structure):
@@ -377,10 +378,10 @@ class Cache:
     """Convenience owner of the device buffers a cache needs (torch allocations) plus its handle."""
 
     def __init__(self, blob: bytes, n_layers, n_q, n_kv, max_seqs, max_tokens_per_seq, max_append_tokens,
-                 pool_high_pages, pool_low_pages, device="cuda", recent_window=0):
+                 pool_high_pages, pool_low_pages, device="cuda", recent_window=0, low_bits=4):
         self.policy = pask_load_policy(blob)
         self.desc = CacheDesc(n_layers, n_q, n_kv, 128, 16, max_seqs, max_tokens_per_seq, max_append_tokens,
-                              pool_high_pages, pool_low_pages, recent_window)
+                              pool_high_pages, pool_low_pages, recent_window, low_bits)
         self.sizes = pask_cache_sizes(self.desc)
         self.n_q, self.n_kv, self.n_layers = n_q, n_kv, n_layers
         self.pool_high = torch.empty(max(256, self.sizes.pool_high_bytes), dtype=torch.uint8, device=device)

@@ -62,7 +62,7 @@ size_t window_pages(const pask_cache_desc_t *d) {
 bool desc_ok(const pask_cache_desc_t *d) {
     return d->n_layers > 0 && d->n_layers <= 4096 && d->max_seqs > 0 && d->max_tokens_per_seq > 0 &&
            d->max_append_tokens > 0 && d->recent_window >= 0 && d->recent_window <= PASK_MAX_WINDOW &&
-           d->recent_window % kPageTokens == 0;
+           d->recent_window % kPageTokens == 0 && (d->low_bits == 0 || d->low_bits == 4 || d->low_bits == 8);
 }
 
 pask_status_t cuda_rc(cudaError_t e) { return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA; }
@@ -114,9 +114,10 @@ pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **o
     p->n_states = rd32(blob + 20);
     p->budget_q16 = rd32(blob + 24);
     p->window = rd32(blob + 28);
+    p->low_bits = rd32(blob + 32);
     const uint32_t window = p->window, low_bits = rd32(blob + 32), group_size = rd32(blob + 36);
     bool ok = p->n_tags >= 1 && p->n_tags <= 255 && p->n_groups >= 1 && p->n_groups <= PASK_MAX_GROUPS &&
-              p->n_layers >= 1 && p->n_layers <= 4096 && p->n_states <= (1u << 20) && window <= PASK_MAX_WINDOW && window % kPageTokens == 0 && low_bits == 4 &&
+              p->n_layers >= 1 && p->n_layers <= 4096 && p->n_states <= (1u << 20) && window <= PASK_MAX_WINDOW && window % kPageTokens == 0 && (low_bits == 4 || low_bits == 8) &&
               group_size == (uint32_t)kQGroup;
     const size_t lg_pad = ok ? align_up(p->n_layers, 4) : 0;
     const size_t n_ent = ok ? (size_t)p->n_tags * p->n_groups : 0;
@@ -165,7 +166,7 @@ pask_status_t pask_cache_sizes(const pask_cache_desc_t *d, pask_cache_sizes_t *o
     if (!shape_ok(d)) return PASK_ERR_UNSUPPORTED_SHAPE;
     if (!desc_ok(d)) return PASK_ERR_INVALID_ARG;
     out->high_page_bytes = (size_t)d->n_kv_heads * kHighHeadBytes;
-    out->low_page_bytes = (size_t)d->n_kv_heads * kLowHeadBytes;
+    out->low_page_bytes = (size_t)d->n_kv_heads * (d->low_bits == 8 ? kLow8HeadBytes : kLowHeadBytes);
     out->pool_high_bytes = out->high_page_bytes * ((size_t)d->pool_high_pages + window_pages(d));
     out->pool_low_bytes = out->low_page_bytes * d->pool_low_pages;
     out->meta_bytes = meta_offsets(d, 255, PASK_MAX_GROUPS).total;  // independent of the policy loaded later
@@ -177,7 +178,8 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     if (!d || !pol || !meta || !out) return PASK_ERR_INVALID_ARG;
     *out = nullptr;
     if (!shape_ok(d)) return PASK_ERR_UNSUPPORTED_SHAPE;
-    if (!desc_ok(d) || (uint32_t)d->n_layers != pol->n_layers || (uint32_t)d->recent_window != pol->window)
+    if (!desc_ok(d) || (uint32_t)d->n_layers != pol->n_layers || (uint32_t)d->recent_window != pol->window ||
+        (uint32_t)(d->low_bits ? d->low_bits : 4) != pol->low_bits)
         return PASK_ERR_INVALID_ARG;
     if (((d->pool_high_pages || d->recent_window) && !pool_high) || (d->pool_low_pages && !pool_low)) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)pool_high | (uintptr_t)pool_low | (uintptr_t)meta) & 255) return PASK_ERR_INVALID_ARG;
@@ -238,9 +240,12 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     v.high_limit = d->pool_high_pages + (uint32_t)window_pages(d);
     v.budget_q16 = pol->budget_q16;
     v.high_page_bytes = (uint32_t)d->n_kv_heads * kHighHeadBytes;
-    v.low_page_bytes = (uint32_t)d->n_kv_heads * kLowHeadBytes;
+    v.low_bits = pol->low_bits;
+    v.low_head_bytes = pol->low_bits == 8 ? kLow8HeadBytes : kLowHeadBytes;
+    v.cost_low_page = pol->low_bits == 8 ? kCostLow8Page : kCostLowPage;
+    v.low_page_bytes = (uint32_t)d->n_kv_heads * v.low_head_bytes;
     v.bytes_h = 2u * d->n_kv_heads * kHeadDim * 2u;
-    v.bytes_l = 2u * d->n_kv_heads * (kHeadDim / 2 + kGroupsPerHead * 2);
+    v.bytes_l = 2u * d->n_kv_heads * (kHeadDim * pol->low_bits / 8 + kGroupsPerHead * 2);
     c->attn_ctas = attention_grid(c);
     c->lut = pol->eff;
     c->layer_group = pol->layer_group;
@@ -588,11 +593,23 @@ pask_status_t pask_debug_dump_low(pask_cache_t *c, int32_t layer, int32_t seq, u
         for (uint32_t tau = 0; tau < (uint32_t)kPageTokens && p * kPageTokens + tau < nl; tau++) {
             const size_t tok = (size_t)p * kPageTokens + tau;
             for (int h = 0; h < n_kv; h++) {
-                const uint8_t *kh = page.data() + (size_t)h * kLowHeadBytes;
-                const uint8_t *vh = kh + kLowHalfBytes;
+                const uint8_t *kh = page.data() + (size_t)h * c->dev.low_head_bytes;
                 uint8_t *kc = k_codes + (tok * n_kv + h) * kHeadDim, *vc = v_codes + (tok * n_kv + h) * kHeadDim;
                 uint16_t *ks = k_scales + (tok * n_kv + h) * kGroupsPerHead;
                 uint16_t *vs = v_scales + (tok * n_kv + h) * kGroupsPerHead;
+                if (c->dev.low_bits == 8) {
+                    const uint8_t *v8 = kh + kLow8HalfBytes;
+                    for (int w = 0; w < 4; w++) {
+                        std::memcpy(ks + w, kh + low8_scale_off((int)tau, w), 2);
+                        std::memcpy(vs + w, v8 + low8_scale_off((int)tau, w), 2);
+                    }
+                    for (int dd = 0; dd < kHeadDim; dd++) {
+                        kc[dd] = kh[low8_k_off((int)tau, dd)];
+                        vc[dd] = v8[low8_v_off((int)tau, dd)];
+                    }
+                    continue;
+                }
+                const uint8_t *vh = kh + kLowHalfBytes;
                 for (int w = 0; w < 4; w++) {
                     std::memcpy(ks + w, kh + low_scale_off((int)tau, w), 2);
                     std::memcpy(vs + w, vh + low_scale_off((int)tau, w), 2);

@@ -305,13 +305,38 @@ __device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uin
         }
         return;
     }
-    uint8_t *dst = c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLowHeadBytes + (which ? kLowHalfBytes : 0);
     float f[8] = {bf16_lo(x.x), bf16_hi(x.x), bf16_lo(x.y), bf16_hi(x.y), bf16_lo(x.z), bf16_hi(x.z), bf16_lo(x.w), bf16_hi(x.w)};
     float amax = 0.0f;
 #pragma unroll
     for (int e = 0; e < 8; e++) amax = fmaxf(amax, fabsf(f[e]));
     amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));   // the 4 chunks of a 32-dim group
     amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));   // sit in 4 adjacent lanes
+    if (c.low_bits == 8) {   // eight-bit codes: the same recipe with 127 in place of 7, codes offset by 128
+        uint8_t *dst8 = c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLow8HeadBytes + (which ? kLow8HalfBytes : 0);
+        __half sh8 = __float2half_rn(__fdiv_rn(amax, 127.0f));
+        if (__hisinf(sh8)) sh8 = __ushort_as_half((unsigned short)0x7BFF);
+        const float s8 = __half2float(sh8);
+        const float inv8 = s8 == 0.0f ? 0.0f : __fdiv_rn(1.0f, s8);
+        uint32_t code8[8];
+#pragma unroll
+        for (int e = 0; e < 8; e++) {   // clamp, then 1.5 * 2^23 + 128 leaves the rounded code in the low byte
+            const float cl = fminf(fmaxf(__fmul_rn(f[e], inv8), -127.0f), 127.0f);
+            code8[e] = __float_as_uint(__fadd_rn(cl, 12583040.0f)) & 255u;
+        }
+        if (!which) {
+#pragma unroll
+            for (int e = 0; e < 8; e += 2)
+                *reinterpret_cast<uint16_t *>(dst8 + low8_k_off((int)tau, 8 * cch + e)) = (uint16_t)(code8[e] | (code8[e + 1] << 8));
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; e++) dst8[low8_v_off((int)tau, 8 * cch + e)] = (uint8_t)code8[e];
+        }
+        if ((cch & 3) == 0) *reinterpret_cast<__half *>(dst8 + low8_scale_off((int)tau, cch >> 2)) = sh8;
+        const uint32_t hb8 = __reduce_max_sync(0xffffffffu, which ? (uint32_t)__half_as_ushort(sh8) : 0u);
+        if ((threadIdx.x & 31) == 0 && hb8 > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb8);
+        return;
+    }
+    uint8_t *dst = c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLowHeadBytes + (which ? kLowHalfBytes : 0);
     const float s32 = __fdiv_rn(amax, 7.0f);
     __half sh = __float2half_rn(s32);
     if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);  // saturate, never infinite
@@ -471,6 +496,38 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
                 const uint32_t m2b = *reinterpret_cast<const uint32_t *>(&m2);
                 float amax = fmaxf(bf16_lo(m2b), bf16_hi(m2b));
                 amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                if (c.low_bits == 8) {
+                    // eight-bit codes: this thread's 16 values are the k-chunk 2w + half of its token.
+                    // One image buffer (both halves of s_low): wait until the previous head has left.
+                    __half sh8 = __float2half_rn(__fdiv_rn(amax, 127.0f));
+                    if (__hisinf(sh8)) sh8 = __ushort_as_half((unsigned short)0x7BFF);
+                    const float s8 = __half2float(sh8);
+                    const float inv8 = s8 == 0.0f ? 0.0f : __fdiv_rn(1.0f, s8);
+                    uint32_t c8[16];
+#pragma unroll
+                    for (int e = 0; e < 16; e++) {
+                        const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
+                        const float cl = fminf(fmaxf(__fmul_rn(f, inv8), -127.0f), 127.0f);
+                        c8[e] = __float_as_uint(__fadd_rn(cl, 12583040.0f)) & 255u;
+                    }
+                    __syncthreads();
+                    uint8_t *img8 = &s_low[0][0] + (which ? kLow8HalfBytes : 0);
+                    const int d0 = 32 * w + 16 * half;
+                    if (!which) {
+#pragma unroll
+                        for (int e = 0; e < 16; e += 2)
+                            *reinterpret_cast<uint16_t *>(img8 + low8_k_off(tau, d0 + e)) = (uint16_t)(c8[e] | (c8[e + 1] << 8));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 16; e++) img8[low8_v_off(tau, d0 + e)] = (uint8_t)c8[e];
+                        vmax_bits = max(vmax_bits, (uint32_t)__half_as_ushort(sh8));
+                    }
+                    if (half == 0) *reinterpret_cast<__half *>(img8 + low8_scale_off(tau, w)) = sh8;
+                    __syncthreads();
+                    uint4 *dst8 = reinterpret_cast<uint4 *>(c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLow8HeadBytes);
+                    for (int x = tid; x < kLow8HeadBytes / 16; x += kWriteThreads) dst8[x] = reinterpret_cast<const uint4 *>(&s_low[0][0])[x];
+                    continue;
+                }
                 const float s32 = __fdiv_rn(amax, 7.0f);
                 __half sh = __float2half_rn(s32);
                 if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);   // saturate, never infinite
@@ -745,7 +802,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             const int idx = base + tid;
             uint32_t ph = 0, pl = 0;
             if (idx < n_seqs) { ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens; pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens; }
-            uint32_t ic = ph * kCostHighPage + pl * kCostLowPage, ip = ph + pl;
+            uint32_t ic = ph * kCostHighPage + pl * c.cost_low_page, ip = ph + pl;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
                 const uint32_t oc = __shfl_up_sync(0xffffffffu, ic, d), op = __shfl_up_sync(0xffffffffu, ip, d);

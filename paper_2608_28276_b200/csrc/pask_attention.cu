@@ -132,6 +132,9 @@ __device__ __forceinline__ uint2 lds64(uint32_t a) {
     asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a) : "memory");
     return v;
 }
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
 __device__ __forceinline__ void sts128(uint32_t a, uint4 v) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
@@ -281,7 +284,7 @@ attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ 
                 ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens + (s_nw[idx] + kPageTokens - 1) / kPageTokens;
                 pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens;
             }
-            uint32_t ic = ph * kCostHighPage + pl * kCostLowPage, ip = ph + pl;
+            uint32_t ic = ph * kCostHighPage + pl * c.cost_low_page, ip = ph + pl;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
                 const uint32_t oc = __shfl_up_sync(0xffffffffu, ic, d), op = __shfl_up_sync(0xffffffffu, ip, d);
@@ -337,6 +340,7 @@ struct Pipe {
     const uint32_t *order;    // the page-order list
     const uint8_t *base_high, *base_low;   // pool + this warp's head offset
     uint32_t stride_high, stride_low;      // page size in bytes
+    uint32_t low_two, low_job_bytes;       // 8-bit LOW pages come as two jobs (K half, V half) of low_job_bytes each
     uint32_t *status;         // the cache's device status word
     uint64_t policy;          // L2 cache policy of the bulk copies
     int lane;
@@ -362,13 +366,14 @@ struct Pipe {
         const uint32_t id = entry & kOrderIdMask;
         const bool is_high = entry & kOrderHigh;
         const uint8_t *src = is_high ? base_high + (size_t)id * stride_high + p_sub * kHighTileBytes
-                                     : base_low + (size_t)id * stride_low;
-        const uint32_t bytes = is_high ? kHighTileBytes : kLowHeadBytes;
+                                     : base_low + (size_t)id * stride_low + p_sub * low_job_bytes;
+        const uint32_t bytes = is_high ? kHighTileBytes : low_job_bytes;
         issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bars + p_stage * 8, meta + p_stage * 4, entry, policy);
         p_stage = p_stage + 1 == kStages ? 0 : p_stage + 1;
         outstanding++;
-        const uint32_t page_done = is_high ? p_sub : 1u;   // a HIGH page is two jobs
-        p_sub = is_high ? p_sub ^ 1u : 0u;
+        const bool two = is_high || low_two;               // a HIGH page is two jobs, an 8-bit LOW page too
+        const uint32_t page_done = two ? p_sub : 1u;
+        p_sub = two ? p_sub ^ 1u : 0u;
         p_pos += page_done;
     }
 
@@ -393,8 +398,10 @@ struct Pipe {
     }
 };
 
-template <bool kHasLow>
+// kLow: 0 = the LOW stream is compiled out (full high-precision cache), 4 / 8 = width of its codes
+template <int kLow>
 __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __grid_constant__ AttnParams p) {
+    constexpr bool kHasLow = kLow != 0;
     extern __shared__ __align__(1024) uint8_t smem[];
     const DevCache &c = p.c;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
@@ -448,9 +455,11 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     Pipe w;
     w.order = p.ws.order;
     w.base_high = c.pool_high + (size_t)warp * kHighHeadBytes;
-    w.base_low = c.pool_low + (size_t)warp * kLowHeadBytes;
+    w.base_low = c.pool_low + (size_t)warp * (kLow == 8 ? kLow8HeadBytes : kLowHeadBytes);
     w.stride_high = c.high_page_bytes;
     w.stride_low = c.low_page_bytes;
+    w.low_two = kLow == 8;
+    w.low_job_bytes = kLow == 8 ? kLow8HalfBytes : kLowHeadBytes;
     w.status = c.ctrl + kCtrlStatus;
     w.policy = l2_evict_first_policy();
     w.lane = lane;
@@ -514,16 +523,26 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 for (int i = 0; i < 4; i++) {
                     const float f0 = bf_lo(r[i]), f1 = bf_hi(r[i]);
                     too_big |= fabsf(f0) > 65504.f || fabsf(f1) > 65504.f;
-                    const float sc = (i & 1) ? 0.0625f : 1.0f;
+                    // (8-bit codes: every A operand is 1024 + code, so q is stored as is and the offset is 1152)
+                    const float sc = (kLow == 4 && (i & 1)) ? 0.0625f : 1.0f;
                     h[i] = pack_f16(f0 * sc, f1 * sc);
                     const float2 bq = unpack_f16(h[i]);
-                    seed -= ((i & 1) ? 1152.f : 1032.f) * (bq.x + bq.y);
+                    seed -= ((kLow == 8 || (i & 1)) ? 1152.f : 1032.f) * (bq.x + bq.y);
                 }
                 seed += __shfl_xor_sync(0xffffffffu, seed, 1);
                 seed += __shfl_xor_sync(0xffffffffu, seed, 2);
                 // the seed of head a+1 sits one 4-lane row further on
                 const float seed_b = __shfl_down_sync(0xffffffffu, seed, 4);
-                if (g < 4) sts128(scratch + j * 256 + g * 64 + t * 16, make_uint4(h[0], h[1], h[2], h[3]));
+                if (kLow == 8) {
+                    // B operands of the k-chunks of 16 dims: chunk c, head, lane t -> {dims 16c+2t,+1 | dims 16c+2t+8,+9};
+                    // this lane holds dims 32j + 8t + 2i, +1, i.e. chunk 2j + t/2, slot i, half t & 1
+                    if (g < 4) {
+#pragma unroll
+                        for (int i = 0; i < 4; i++) sts32(scratch + (2 * j + (t >> 1)) * 128 + g * 32 + i * 8 + (t & 1) * 4, h[i]);
+                    }
+                } else if (g < 4) {
+                    sts128(scratch + j * 256 + g * 64 + t * 16, make_uint4(h[0], h[1], h[2], h[3]));
+                }
                 // accumulator quads {seed[a], seed[a+1], seed[a], seed[a+1]} of head pairs (0,1) and (2,3)
                 if (t == 0 && (g == 0 || g == 2)) {
                     const uint32_t sa = __float_as_uint(seed), sb = __float_as_uint(seed_b);
@@ -566,6 +585,33 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
 #pragma unroll
                 for (int i = 0; i < 4; i++) sc[i] += sc2[i];
                 w.release();
+            } else if (kLow == 8) {
+                // ---- QK^T over 8-bit K codes: per 32-dim group two k-chunks, A = 1024 + code by byte permutes
+                const uint2 ks0 = lds64(st + kLow8CodesBytes + g * 8);
+                const uint2 ks1 = lds64(st + kLow8CodesBytes + (g + 8) * 8);
+                const float2 f0[2] = {unpack_f16(ks0.x), unpack_f16(ks0.y)};
+                const float2 f1[2] = {unpack_f16(ks1.x), unpack_f16(ks1.y)};
+                uint4 kw[4];
+#pragma unroll
+                for (int j = 0; j < 4; j++) kw[j] = lds128(st + j * 512 + lane * 16);
+                w.release();
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint2 qa = lds64(scratch + (2 * j) * 128 + (g & 3) * 32 + t * 8);
+                    const uint2 qb = lds64(scratch + (2 * j + 1) * 128 + (g & 3) * 32 + t * 8);
+                    const uint4 seed = lds128(scratch + 1024 + ((t & 1) * 4 + j) * 16);
+                    float cj[4];
+                    mma_f16_seed(cj, prmt(kw[j].x, 0x64646464u, 0x4140), prmt(kw[j].x, 0x64646464u, 0x4342),
+                                 prmt(kw[j].y, 0x64646464u, 0x4140), prmt(kw[j].y, 0x64646464u, 0x4342), qa.x, qa.y, seed);
+                    mma_f16(cj, prmt(kw[j].z, 0x64646464u, 0x4140), prmt(kw[j].z, 0x64646464u, 0x4342),
+                            prmt(kw[j].w, 0x64646464u, 0x4140), prmt(kw[j].w, 0x64646464u, 0x4342), qb.x, qb.y);
+                    const float s0f = (j & 1) ? f0[j >> 1].y : f0[j >> 1].x;
+                    const float s1f = (j & 1) ? f1[j >> 1].y : f1[j >> 1].x;
+                    sc[0] = fmaf(s0f, cj[0], sc[0]);
+                    sc[1] = fmaf(s0f, cj[1], sc[1]);
+                    sc[2] = fmaf(s1f, cj[2], sc[2]);
+                    sc[3] = fmaf(s1f, cj[3], sc[3]);
+                }
             } else if (kHasLow) {
                 const uint4 k0 = lds128(st + lane * 16);
                 const uint4 k1 = lds128(st + 512 + lane * 16);
@@ -648,6 +694,40 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                     }
                 }
                 w.release();
+            } else if (kLow == 8) {
+                // ---- P.V over 8-bit V codes: the V half is a job of its own
+                const uint32_t p01 = pack_f16(p0, p1), p23 = pack_f16(p2, p3);
+                st = w.acquire(entry);
+                if (w.dead) break;
+                uint4 vw[4];
+#pragma unroll
+                for (int q = 0; q < 4; q++) vw[q] = lds128(st + q * 512 + lane * 16);   // group q: tiles r = 0 (x, y) and 1 (z, w)
+                uint2 vs0 = lds64(st + kLow8CodesBytes + g * 8);
+                uint2 vs1 = lds64(st + kLow8CodesBytes + (g + 8) * 8);
+                w.release();
+                if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
+                    if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
+                    if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
+                }
+#pragma unroll
+                for (int v = 0; v < 2; v++) {
+                    const uint32_t s0b = hmul2(prmt(v ? vs0.y : vs0.x, 0u, bsel), down);
+                    const uint32_t s1b = hmul2(prmt(v ? vs1.y : vs1.x, 0u, bsel), down);
+                    const uint32_t b0 = movmatrix_trans(hmul2(p01, s0b)), b1 = movmatrix_trans(hmul2(p23, s1b));
+#pragma unroll
+                    for (int qq = 0; qq < 2; qq++) {
+                        const int q = 2 * v + qq;
+#pragma unroll
+                        for (int r = 0; r < 2; r++) {
+                            const uint32_t w0 = r ? vw[q].z : vw[q].x, w1 = r ? vw[q].w : vw[q].y;
+                            // (1024 + code) - 1152 = code - 128, exact in fp16
+                            mma_f16(acc[2 * q + r], hsub2(prmt(w0, 0x64646464u, 0x4140), 0x64806480u),
+                                    hsub2(prmt(w0, 0x64646464u, 0x4342), 0x64806480u),
+                                    hsub2(prmt(w1, 0x64646464u, 0x4140), 0x64806480u),
+                                    hsub2(prmt(w1, 0x64646464u, 0x4342), 0x64806480u), b0, b1);
+                        }
+                    }
+                }
             } else if (kHasLow) {
                 const uint32_t vb = st + kLowHalfBytes;
                 const uint4 v0 = lds128(vb + lane * 16);        // tokens 2t, 2t+1
@@ -817,7 +897,7 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
     p.q = static_cast<const uint4 *>(q);
     carve_workspace(c, n_seqs, static_cast<uint8_t *>(workspace), &p.ws);
     const size_t smem = attn_smem_bytes(n_seqs, n_warps);
-    auto kern = has_low ? decode_attn_kernel<true> : decode_attn_kernel<false>;
+    auto kern = !has_low ? decode_attn_kernel<0> : c->dev.low_bits == 8 ? decode_attn_kernel<8> : decode_attn_kernel<4>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return PASK_ERR_CUDA;
     cudaError_t e = cudaSuccess;

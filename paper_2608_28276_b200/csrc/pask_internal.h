@@ -83,6 +83,9 @@ struct DevCache {
     uint32_t budget_q16;
     uint32_t high_page_bytes, low_page_bytes;
     uint32_t bytes_h, bytes_l;       // m(H), m(L) per token per layer
+    uint32_t low_bits;               // 4 or 8: width of the RETAIN-LOW codes
+    uint32_t low_head_bytes;         // one KV head of a LOW page (2304 or 4352)
+    uint32_t cost_low_page;          // cost of a LOW page in units of n_kv * 256 bytes (9 or 17)
 };
 
 // workspace of one decode-attention call
@@ -104,7 +107,7 @@ struct MetaOffsets {
 }  // namespace pask
 
 struct pask_policy {
-    uint32_t n_tags, n_groups, n_layers, n_states, budget_q16, window;
+    uint32_t n_tags, n_groups, n_layers, n_states, budget_q16, window, low_bits;
     std::vector<uint8_t> layer_group, a0, a_floor, eff;
     std::vector<float> rho_rl, rho_lh;
     std::vector<uint32_t> gamma;

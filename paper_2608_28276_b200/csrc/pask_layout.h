@@ -25,6 +25,16 @@
 //              32q + 4g + i (i = 0..3), token 2t + 8*ps in nibble i and token 2t + 1 + 8*ps in
 //              nibble i + 4, so the same mask yields (even token, odd token) pairs per dim.
 //   scales   : [token 16][group 4] fp16.
+// LOW page, 8-bit codes (policy low_bits = 8):
+//              [kv head][K codes 2048][K scales 128][V codes 2048][V scales 128]   (n_kv * 4352 B)
+//   K codes  : 4 rounds of 512 B; round rr holds, for lane (g,t), the 16 dims of k-chunks 2rr and
+//              2rr+1 as two 8-byte pieces; the piece of chunk c is {token g dims 16c+2t,+1 | token g+8
+//              same dims | token g dims 16c+2t+8,+9 | token g+8 same dims}, one byte per code: two PRMTs
+//              per 32-bit word turn it into the fp16 pairs 1024 + code of an m16n8k16 A operand.
+//   V codes  : 4 rounds of 512 B, one per 32-dim group q; lane (g,t) holds for r = 0,1 the piece
+//              {dim D tokens 2t,2t+1 | dim D+1 tokens 2t,2t+1 | dim D tokens 2t+8,+9 | dim D+1 tokens
+//              2t+8,+9} with D = 32q + 4g + 2r: the A operand of the P.V tile whose rows g, g+8 are
+//              dims D, D+1 (the row order the bf16 and 4-bit paths use too).
 #pragma once
 #include <stdint.h>
 
@@ -46,9 +56,13 @@ constexpr int kLowCodesBytes = 1024;
 constexpr int kLowScalesBytes = 128;
 constexpr int kLowHalfBytes = 1152;  // codes + scales of K (or of V)
 constexpr int kLowHeadBytes = 2304;
+constexpr int kLow8CodesBytes = 2048;
+constexpr int kLow8HalfBytes = 2176;  // codes + scales of K (or of V), 8-bit codes
+constexpr int kLow8HeadBytes = 4352;
 // cost of streaming one page (all heads), in units of n_kv * 256 bytes
 constexpr uint32_t kCostHighPage = 32;
 constexpr uint32_t kCostLowPage = 9;
+constexpr uint32_t kCostLow8Page = 17;
 
 // HIGH K tile: offset of the 4-byte piece holding dims 2p, 2p+1 (p = 0..63) of token tau.
 PASK_HD int high_k_pair_off(int tau, int p) {
@@ -79,6 +93,18 @@ PASK_HD int low_v_half_off(int tau, int q, int g) {
 
 // scales (relative to the K or V half): fp16 of (token tau, group w)
 PASK_HD int low_scale_off(int tau, int w) { return kLowCodesBytes + tau * 8 + w * 2; }
+
+// 8-bit LOW K codes: byte offset of the code of (token tau, dim d) within the K codes
+PASK_HD int low8_k_off(int tau, int d) {
+    const int c = d >> 4, within = d & 15, t = (within & 7) >> 1, upper = within >> 3;
+    return (c >> 1) * 512 + (4 * (tau & 7) + t) * 16 + (c & 1) * 8 + upper * 4 + (tau >> 3) * 2 + (within & 1);
+}
+// 8-bit LOW V codes (relative to the V half)
+PASK_HD int low8_v_off(int tau, int d) {
+    const int q = d >> 5, g = (d & 31) >> 2, i = d & 3, t = (tau & 7) >> 1;
+    return q * 512 + (4 * g + t) * 16 + (i >> 1) * 8 + (tau >> 3) * 4 + (i & 1) * 2 + (tau & 1);
+}
+PASK_HD int low8_scale_off(int tau, int w) { return kLow8CodesBytes + tau * 8 + w * 2; }
 
 // ---- work partition of decode attention -------------------------------------------------
 // Every sequence's pages are visited in one fixed order that interleaves its HIGH and LOW pages

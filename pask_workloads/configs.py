@@ -38,6 +38,7 @@ class Config:
     mode: str = "grammar"            # "grammar" | "mix"
     lut: str = "greedy"              # "greedy" | "random" | "all_high"
     bias: str = "balanced"           # greedy table flavour: "balanced" | "low" | "high"
+    low_bits: int = 4                # width of the RETAIN-LOW codes: 4 or 8
     protected_prompt: bool = False   # prompt tokens carry TAG_PROTECTED (tiny)
     extra_gen: int = 64              # generated tokens beyond gen_len kept ready for decode steps
 
@@ -158,5 +159,5 @@ def build(cfg: Config, seed: Optional[int] = None, repeat: int = 0) -> Workload:
     elif cfg.lut == "all_high":
         pol = all_high_policy(n_tags, cfg.n_groups, cfg.n_layers)
     else:
-        pol = greedy_policy(seed, counts, cfg.n_groups, cfg.n_layers, cfg.budget, cfg.bias)
+        pol = greedy_policy(seed, counts, cfg.n_groups, cfg.n_layers, cfg.budget, cfg.bias, cfg.low_bits)
     return Workload(cfg, seed, prompt_tags, gen_tags, pol, counts)

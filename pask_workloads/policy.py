@@ -33,6 +33,11 @@ R, L, H = 0, 1, 2
 COST_L_OVER_H = 1152.0 / 4096.0      # int4 codes + fp16 scale per 32 values, against bf16
 
 
+def cost_l_over_h(low_bits: int) -> float:
+    """m(L) / m(H): codes of low_bits each plus one fp16 scale per 32 values, against bf16."""
+    return (128 * low_bits / 8 + 8) / 256.0
+
+
 @dataclass
 class Policy:
     n_tags: int
@@ -110,7 +115,7 @@ _PRIOR = {
 
 
 def greedy_policy(seed: int, tag_counts: np.ndarray, n_groups: int, n_layers: int, budget: float,
-                  bias: str = "balanced") -> Policy:
+                  bias: str = "balanced", low_bits: int = 4) -> Policy:
     """Greedy adjacent-upgrade table that reaches (without exceeding) a target normalised cost.
 
     tag_counts[z] is how many tokens of the workload carry tag z (all sequences, prompt and
@@ -130,6 +135,7 @@ def greedy_policy(seed: int, tag_counts: np.ndarray, n_groups: int, n_layers: in
     rl = np.zeros((n_tags, n_groups), np.float32)
     lh = np.zeros((n_tags, n_groups), np.float32)
     lh_penalty = {"balanced": 0.5, "low": 5.0, "high": -5.0}[bias]
+    cost_l = cost_l_over_h(low_bits)
     ups = []
     for z in range(n_tags):
         for c in range(n_groups):
@@ -150,8 +156,8 @@ def greedy_policy(seed: int, tag_counts: np.ndarray, n_groups: int, n_layers: in
                 if a[z, c] >= tgt:
                     continue
                 # an H upgrade may arrive before its L (bias="high"): take both steps at once
-                step = (COST_L_OVER_H if a[z, c] == R else 0.0) if tgt == L else \
-                       (1.0 - (COST_L_OVER_H if a[z, c] == L else 0.0))
+                step = (cost_l if a[z, c] == R else 0.0) if tgt == L else \
+                       (1.0 - (cost_l if a[z, c] == L else 0.0))
                 dc = f[z] * w[c] * step
                 if cost + dc <= budget + 1e-12:
                     a[z, c] = tgt
@@ -161,7 +167,7 @@ def greedy_policy(seed: int, tag_counts: np.ndarray, n_groups: int, n_layers: in
             pending = rest
     fl = np.zeros((n_tags, n_groups), np.uint8)
     gamma = np.asarray([rng.below(1 << 20) for _ in range(16)], dtype=np.uint32)
-    return Policy(n_tags, n_groups, lg, a, fl, rl, lh, gamma, budget_target=budget)
+    return Policy(n_tags, n_groups, lg, a, fl, rl, lh, gamma, budget_target=budget, low_bits=low_bits)
 
 
 def all_high_policy(n_tags: int, n_groups: int, n_layers: int) -> Policy:
@@ -177,7 +183,7 @@ def expected_cost(p: Policy, tag_counts: np.ndarray) -> float:
     which are not in tag_counts, are not included)."""
     eff = np.maximum(p.a0, p.a_floor).astype(np.int64)
     w = np.bincount(p.layer_group, minlength=p.n_groups).astype(np.float64) / p.n_layers
-    per = np.where(eff == H, 1.0, np.where(eff == L, COST_L_OVER_H, 0.0))
+    per = np.where(eff == H, 1.0, np.where(eff == L, cost_l_over_h(p.low_bits), 0.0))
     f = tag_counts.astype(np.float64) / max(1.0, float(tag_counts.sum()))
     return float((f[:, None] * w[None, :] * per).sum())
 

@@ -30,7 +30,8 @@ class Pair:
         blob = blob or workload.blob
         window = int.from_bytes(blob[28:32], "little")                  # the policy's protected recent window
         self.gpu = pask.Cache(blob, cfg.n_layers, cfg.n_q, cfg.n_kv, self.max_seqs, self.max_tokens,
-                              max_append_tokens or total, self.hp, self.lp, recent_window=window)
+                              max_append_tokens or total, self.hp, self.lp, recent_window=window,
+                              low_bits=int.from_bytes(blob[32:36], "little"))
         self.orc = oracle.Cache(oracle.Policy(blob), cfg.n_q, cfg.n_kv, self.max_seqs, self.hp, self.lp)
 
     # ------------------------------------------------------------------ append

@@ -35,7 +35,7 @@ def test_library_exports_every_declared_symbol(pask):
 
 def test_struct_layouts_match_header(pask):
     assert C.sizeof(pask.BudgetState) == 4 * 8 * 8 + 4 * 8 + 4 * 4 + 5 * 8
-    assert C.sizeof(pask.CacheDesc) == 44
+    assert C.sizeof(pask.CacheDesc) == 48
 
 
 def test_policy_blob_parsing_agrees_with_oracle(pask, oracle):
@@ -77,7 +77,7 @@ def test_bad_blobs_and_arguments_are_refused(pask):
     broken = bytearray(good); broken[40 + 4] = 3; bads.append(bytes(broken))           # action out of range
     broken = bytearray(good); broken[28] = 1; bads.append(bytes(broken))               # recent window not a multiple of 16
     broken = bytearray(good); broken[29] = 2; bads.append(bytes(broken))               # recent window too large (512)
-    broken = bytearray(good); broken[32] = 8; bads.append(bytes(broken))               # low_bits != 4
+    broken = bytearray(good); broken[32] = 6; bads.append(bytes(broken))               # low_bits neither 4 nor 8
     broken = bytearray(good); broken[40] = 9; bads.append(bytes(broken))               # layer group out of range
     for b in bads:
         with pytest.raises(pask.PaskError) as e:
