@@ -23,8 +23,9 @@ def pask():
     return P
 
 
-@pytest.mark.parametrize("seed,n_kv,window", [(1, 2, 0), (2, 8, 0), (3, 4, 16), (4, 1, 48), (5, 8, 0), (6, 2, 0)])
-def test_random_call_sequences(pask, oracle, seed, n_kv, window):
+@pytest.mark.parametrize("seed,n_kv,window,low_bits", [(1, 2, 0, 4), (2, 8, 0, 4), (3, 4, 16, 4), (4, 1, 48, 4), (5, 8, 0, 4),
+                                                       (6, 2, 0, 4), (7, 8, 0, 8), (8, 2, 32, 8), (9, 1, 0, 8)])
+def test_random_call_sequences(pask, oracle, seed, n_kv, window, low_bits):
     from dataclasses import replace
     rng = CounterRng(seed, 4242)
     n_layers, G, B = 2, 2, 4
@@ -33,7 +34,7 @@ def test_random_call_sequences(pask, oracle, seed, n_kv, window):
     w = WC.build(cfg)
     tight = seed % 2 == 0                                               # every other case runs out of pages now and then
     pages = 16 if tight else 400
-    p = Pair(pask, oracle, w, blob=WP.write_blob(replace(w.policy, recent_window=window)), pool_high_pages=pages,
+    p = Pair(pask, oracle, w, blob=WP.write_blob(replace(w.policy, recent_window=window, low_bits=low_bits)), pool_high_pages=pages,
              pool_low_pages=pages, max_tokens_per_seq=4096, max_append_tokens=2048)
     d = "cuda"
     serial = 0
