@@ -702,6 +702,71 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         if (tid == 0 && !fits && !s_err) atomicOr(&s_err, PASK_DEV_POOL_EXHAUSTED);
     }
     __syncthreads();
+    // ---- fused decode-attention plan for the same sequences (what attn_plan_kernel would compute after
+    // this append): every CTA knows every sequence's lengths after the call and the ids of the pages the
+    // call allocates, so the plan needs nothing that the commit writes.  Only without a recent window.
+    if (fuse_plan && !s_err) {
+        if (tid < n_seqs) { s_nh[tid] = s_old_h[tid] + s_cnt_h[tid]; s_nl[tid] = s_old_l[tid] + s_cnt_l[tid]; }
+        if (tid == 0) s_cost[0] = s_page[0] = 0;
+        __syncthreads();
+        if (tid < 32) {
+            uint32_t carry_c = 0, carry_p = 0;
+            for (int base = 0; base < n_seqs; base += 32) {
+                const int idx = base + tid;
+                uint32_t ph = 0, pl = 0;
+                if (idx < n_seqs) { ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens; pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens; }
+                uint32_t ic = ph * kCostHighPage + pl * c.cost_low_page, ip = ph + pl;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const uint32_t oc = __shfl_up_sync(0xffffffffu, ic, d), op = __shfl_up_sync(0xffffffffu, ip, d);
+                    if (tid >= d) { ic += oc; ip += op; }
+                }
+                if (idx < n_seqs) { s_cost[idx + 1] = carry_c + ic; s_page[idx + 1] = carry_p + ip; }
+                carry_c += __shfl_sync(0xffffffffu, ic, 31);
+                carry_p += __shfl_sync(0xffffffffu, ip, 31);
+            }
+        }
+        __syncthreads();
+        if (blockIdx.x == 0) {
+            if (tid <= n_seqs) { ws.cost_prefix[tid] = s_cost[tid]; ws.page_prefix[tid] = s_page[tid]; }
+            if (tid < n_seqs) ws.tokens[tid] = make_uint2(s_nh[tid], s_nl[tid]);
+        }
+        const uint32_t total_pages = s_page[n_seqs];
+        for (uint32_t gp = blockIdx.x * kSmallThreads + tid; gp < total_pages; gp += gridDim.x * kSmallThreads) {
+            int a = 1, e = n_seqs;   // smallest idx in [1, n_seqs] with s_page[idx] > gp
+            while (a < e) {
+                const int mid = (a + e) >> 1;
+                if (s_page[mid] > gp) e = mid; else a = mid + 1;
+            }
+            const int s = a - 1;
+            const uint32_t nh = s_nh[s], nl = s_nl[s];
+            const uint32_t ph = (nh + kPageTokens - 1) / kPageTokens, pl = (nl + kPageTokens - 1) / kPageTokens;
+            const size_t sl = ((size_t)s_seq[s] * c.n_layers + layer) * c.max_pages;
+            uint32_t idx, entry;
+            if (page_at(gp - s_page[s], ph, pl, idx)) {
+                const uint32_t old_pages = (s_old_h[s] + kPageTokens - 1) / kPageTokens;
+                if (idx < old_pages) {
+                    entry = c.tbl_high[sl + idx];
+                } else {             // a page this call allocates: the commit's formula
+                    const uint32_t kk = s_base_h[s] + (idx - old_pages);
+                    entry = kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]);
+                }
+                entry |= kOrderHigh;
+                if (idx == ph - 1) entry |= (nh & (kPageTokens - 1)) << kOrderValidShift;
+            } else {
+                const uint32_t old_pages = (s_old_l[s] + kPageTokens - 1) / kPageTokens;
+                if (idx < old_pages) {
+                    entry = c.tbl_low[sl + idx];
+                } else {
+                    const uint32_t kk = s_base_l[s] + (idx - old_pages);
+                    entry = kk < s_ctrl[3] ? c.free_low[s_ctrl[3] - 1 - kk] : s_ctrl[2] + (kk - s_ctrl[3]);
+                }
+                if (idx == pl - 1) entry |= (nl & (kPageTokens - 1)) << kOrderValidShift;
+            }
+            ws.order[gp] = entry;
+        }
+    
+    }
     // old page of this CTA's token, if it continues one (page tables are only appended to by the commit)
     uint32_t my_page = 0, my_at = 0;
     const uint32_t my_a = s_act[my_tok];
@@ -789,69 +854,6 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         }
     }
 
-    // ---- fused decode-attention plan for the same sequences (what attn_plan_kernel would compute after
-    // this append): every CTA knows every sequence's lengths after the call and the ids of the pages the
-    // call allocates, so the plan needs nothing that the commit writes.  Only without a recent window.
-    if (!fuse_plan) return;
-    if (tid < n_seqs) { s_nh[tid] = s_old_h[tid] + s_cnt_h[tid]; s_nl[tid] = s_old_l[tid] + s_cnt_l[tid]; }
-    if (tid == 0) s_cost[0] = s_page[0] = 0;
-    __syncthreads();
-    if (tid < 32) {
-        uint32_t carry_c = 0, carry_p = 0;
-        for (int base = 0; base < n_seqs; base += 32) {
-            const int idx = base + tid;
-            uint32_t ph = 0, pl = 0;
-            if (idx < n_seqs) { ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens; pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens; }
-            uint32_t ic = ph * kCostHighPage + pl * c.cost_low_page, ip = ph + pl;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t oc = __shfl_up_sync(0xffffffffu, ic, d), op = __shfl_up_sync(0xffffffffu, ip, d);
-                if (tid >= d) { ic += oc; ip += op; }
-            }
-            if (idx < n_seqs) { s_cost[idx + 1] = carry_c + ic; s_page[idx + 1] = carry_p + ip; }
-            carry_c += __shfl_sync(0xffffffffu, ic, 31);
-            carry_p += __shfl_sync(0xffffffffu, ip, 31);
-        }
-    }
-    __syncthreads();
-    if (blockIdx.x == 0) {
-        if (tid <= n_seqs) { ws.cost_prefix[tid] = s_cost[tid]; ws.page_prefix[tid] = s_page[tid]; }
-        if (tid < n_seqs) ws.tokens[tid] = make_uint2(s_nh[tid], s_nl[tid]);
-    }
-    const uint32_t total_pages = s_page[n_seqs];
-    for (uint32_t gp = blockIdx.x * kSmallThreads + tid; gp < total_pages; gp += gridDim.x * kSmallThreads) {
-        int a = 1, e = n_seqs;   // smallest idx in [1, n_seqs] with s_page[idx] > gp
-        while (a < e) {
-            const int mid = (a + e) >> 1;
-            if (s_page[mid] > gp) e = mid; else a = mid + 1;
-        }
-        const int s = a - 1;
-        const uint32_t nh = s_nh[s], nl = s_nl[s];
-        const uint32_t ph = (nh + kPageTokens - 1) / kPageTokens, pl = (nl + kPageTokens - 1) / kPageTokens;
-        const size_t sl = ((size_t)s_seq[s] * c.n_layers + layer) * c.max_pages;
-        uint32_t idx, entry;
-        if (page_at(gp - s_page[s], ph, pl, idx)) {
-            const uint32_t old_pages = (s_old_h[s] + kPageTokens - 1) / kPageTokens;
-            if (idx < old_pages) {
-                entry = c.tbl_high[sl + idx];
-            } else {             // a page this call allocates: the commit's formula
-                const uint32_t kk = s_base_h[s] + (idx - old_pages);
-                entry = kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]);
-            }
-            entry |= kOrderHigh;
-            if (idx == ph - 1) entry |= (nh & (kPageTokens - 1)) << kOrderValidShift;
-        } else {
-            const uint32_t old_pages = (s_old_l[s] + kPageTokens - 1) / kPageTokens;
-            if (idx < old_pages) {
-                entry = c.tbl_low[sl + idx];
-            } else {
-                const uint32_t kk = s_base_l[s] + (idx - old_pages);
-                entry = kk < s_ctrl[3] ? c.free_low[s_ctrl[3] - 1 - kk] : s_ctrl[2] + (kk - s_ctrl[3]);
-            }
-            if (idx == pl - 1) entry |= (nl & (kPageTokens - 1)) << kOrderValidShift;
-        }
-        ws.order[gp] = entry;
-    }
 }
 
 // General path, recent window: CTA (j, y) copies the y-th newest of sequence j's tokens in this call
