@@ -327,6 +327,21 @@ pask_status_t pask_decode_step_packed(pask_cache_t *cache, int32_t layer, int32_
                                       float *out_host, void *staging, size_t staging_bytes, void *workspace,
                                       size_t workspace_bytes, pask_stream_t stream);
 
+/* Pipelined form of pask_decode_step_packed for a caller that issues layer after layer from host
+ * blocks: the host-to-device copy of a call runs on a copy stream of its own and so overlaps the
+ * kernels of the call before, and the device-to-host copy of the output runs on a second copy
+ * stream and overlaps the call after.  The two streams and six events are created for the cache at
+ * the first call (host-side handles; no device memory) and destroyed with it; kernels still run
+ * on `stream`, in call order.
+ *   staging        dev, >= 2 * pask_step_staging_bytes(cache, n_seqs): two slots used in turn
+ *   packed_host    must stay valid, and out_host is not valid, until pask_decode_step_drain returns
+ *                  (synchronising `stream` alone is not enough: the output copy is not on it)
+ * pask_decode_step_drain blocks the host until every pipelined call issued so far has finished. */
+pask_status_t pask_decode_step_pipelined(pask_cache_t *cache, int32_t layer, int32_t n_seqs, const void *packed_host,
+                                         float *out_host, void *staging, size_t staging_bytes, void *workspace,
+                                         size_t workspace_bytes, pask_stream_t stream);
+pask_status_t pask_decode_step_drain(pask_cache_t *cache);
+
 /* ---------------------------------------------------------------------------------------------
  * pask_distortion -- the inner term of the attention-output distortion (Eq. 4): for each row r
  * (one decode position of one sequence at one layer) max over query heads h of

@@ -287,7 +287,21 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     return PASK_OK;
 }
 
-void pask_cache_destroy(pask_cache_t *c) { delete c; }
+void pask_cache_destroy(pask_cache_t *c) {
+    if (!c) return;
+    if (c->pipe.ready) {
+        cudaStreamSynchronize(c->pipe.in);
+        cudaStreamSynchronize(c->pipe.out);
+        for (int i = 0; i < 2; i++) {
+            cudaEventDestroy(c->pipe.ev_in[i]);
+            cudaEventDestroy(c->pipe.ev_done[i]);
+            cudaEventDestroy(c->pipe.ev_out[i]);
+        }
+        cudaStreamDestroy(c->pipe.in);
+        cudaStreamDestroy(c->pipe.out);
+    }
+    delete c;
+}
 
 pask_status_t pask_cache_reset(pask_cache_t *c, pask_stream_t stream_v) {
     if (!c) return PASK_ERR_INVALID_ARG;
@@ -477,6 +491,60 @@ pask_status_t pask_decode_step_packed(pask_cache_t *c, int32_t layer, int32_t n_
     if (rc != PASK_OK) return rc;
     return cuda_rc(cudaMemcpyAsync(out_host, d_out, (size_t)n_seqs * c->desc.n_q_heads * kHeadDim * 4, cudaMemcpyDeviceToHost,
                                    stream));
+}
+
+pask_status_t pask_decode_step_pipelined(pask_cache_t *c, int32_t layer, int32_t n_seqs, const void *packed_host,
+                                         float *out_host, void *staging, size_t staging_bytes, void *ws, size_t ws_bytes,
+                                         pask_stream_t stream_v) {
+    if (!c || !packed_host || !out_host || !staging) return PASK_ERR_INVALID_ARG;
+    if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL) return PASK_ERR_INVALID_ARG;
+    const size_t slot_bytes = pask_step_staging_bytes(c, n_seqs);
+    if (((uintptr_t)staging & 255) || staging_bytes < 2 * slot_bytes) return PASK_ERR_WORKSPACE;
+    auto &pp = c->pipe;
+    if (!pp.ready) {   // host-side handles only; no device memory
+        bool ok = cudaStreamCreateWithFlags(&pp.in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&pp.out, cudaStreamNonBlocking) == cudaSuccess;
+        for (int i = 0; i < 2 && ok; i++)
+            ok = cudaEventCreateWithFlags(&pp.ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&pp.ev_done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&pp.ev_out[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return PASK_ERR_CUDA;
+        pp.ready = true;
+        pp.calls = 0;
+    }
+    size_t off[6], in_bytes = 0;
+    pask_step_packed_layout(c, n_seqs, off, &in_bytes);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int slot = (int)(pp.calls & 1);
+    uint8_t *p = static_cast<uint8_t *>(staging) + (size_t)slot * slot_bytes;
+    float *d_out = reinterpret_cast<float *>(p + in_bytes);
+    cudaError_t e = cudaSuccess;
+    // this slot's inputs were last read by the kernels of two calls ago, its output by that call's copy-out
+    if (pp.calls >= 2) e = cudaStreamWaitEvent(pp.in, pp.ev_done[slot], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(p, packed_host, in_bytes, cudaMemcpyHostToDevice, pp.in);
+    if (e == cudaSuccess) e = cudaEventRecord(pp.ev_in[slot], pp.in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, pp.ev_in[slot], 0);
+    if (e == cudaSuccess && pp.calls >= 2) e = cudaStreamWaitEvent(stream, pp.ev_out[slot], 0);
+    if (e != cudaSuccess) return PASK_ERR_CUDA;
+    pask_status_t rc = pask_append_attend(c, layer, n_seqs, n_seqs, reinterpret_cast<const int32_t *>(p + off[0]),
+                                          reinterpret_cast<const int32_t *>(p + off[1]), p + off[2], p + off[3], p + off[4],
+                                          nullptr, nullptr, p + off[5], d_out, nullptr, ws, ws_bytes, stream_v);
+    if (rc != PASK_OK) return rc;
+    e = cudaEventRecord(pp.ev_done[slot], stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(pp.out, pp.ev_done[slot], 0);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(out_host, d_out, (size_t)n_seqs * c->desc.n_q_heads * kHeadDim * 4, cudaMemcpyDeviceToHost, pp.out);
+    if (e == cudaSuccess) e = cudaEventRecord(pp.ev_out[slot], pp.out);
+    pp.calls++;
+    return cuda_rc(e);
+}
+
+pask_status_t pask_decode_step_drain(pask_cache_t *c) {
+    if (!c) return PASK_ERR_INVALID_ARG;
+    if (!c->pipe.ready) return PASK_OK;
+    cudaError_t e = cudaStreamSynchronize(c->pipe.in);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->pipe.out);
+    return cuda_rc(e);
 }
 
 pask_status_t pask_budget_state(pask_cache_t *c, int32_t seq, pask_budget_state_t *host_out, pask_stream_t stream_v) {

@@ -125,6 +125,13 @@ struct pask_cache {
     int sm_count;
     int attn_ctas;                // grid of the decode-attention main kernel
     cudaEvent_t ev_start, ev_stop;
+    // pask_decode_step_pipelined: two copy streams and the events that order them against the caller's stream
+    struct StepPipe {
+        bool ready = false;
+        cudaStream_t in = nullptr, out = nullptr;
+        cudaEvent_t ev_in[2] = {}, ev_done[2] = {}, ev_out[2] = {};
+        uint64_t calls = 0;
+    } pipe;
 };
 
 namespace pask {

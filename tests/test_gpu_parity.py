@@ -334,3 +334,40 @@ def test_decode_step_from_one_packed_host_block(pask, oracle):
     oo, ol = p.orc.attention_batch(0, seqs, bf16_bits(q).numpy())
     assert_close(out.numpy().astype(np.float64), ol.copy(), oo, ol)
     p.compare_state()
+
+
+def test_pipelined_host_steps(pask, oracle):
+    # layer after layer from host blocks with the copies on the cache's own streams: every output is
+    # that of the oracle, whatever overlapped with whatever
+    from pask_workloads.tensors import bf16_bits
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=5, n_layers=3, n_groups=3, prompt_len=150, gen_len=60, extra_gen=32)
+    w = WC.build(cfg)
+    p = Pair(pask, oracle, w)
+    seqs = [3, 0, 4, 1, 2]
+    for layer in range(3):
+        p.append(layer, seqs, [210] * 5, [0] * 5)
+    P, h = pask, p.gpu.handle
+    off, n_in = P.pask_step_packed_layout(h, 5)
+    staging = torch.empty(2 * P.pask_step_staging_bytes(h, 5), dtype=torch.uint8, device="cuda")
+    calls = []
+    for step in range(6):
+        for layer in range(3):
+            k = torch.stack([w.kv(layer, b, 210 + step, 1)[0][0] for b in seqs])
+            v = torch.stack([w.kv(layer, b, 210 + step, 1)[1][0] for b in seqs])
+            tags = torch.from_numpy(np.array([w.tags(b, 210 + step, 1)[0] for b in seqs], np.uint8))
+            q = torch.stack([w.q(layer, b, 211 + step) for b in seqs])
+            block = torch.zeros(n_in, dtype=torch.uint8).pin_memory()
+            for o, t in zip(off, [torch.tensor(seqs, dtype=torch.int32), torch.arange(6, dtype=torch.int32), k, v, tags, q]):
+                raw = t.contiguous().view(torch.uint8).reshape(-1)
+                block[o:o + raw.numel()] = raw
+            out = torch.full((5, 32, 128), float("nan"), dtype=torch.float32).pin_memory()
+            P.pask_decode_step_pipelined(h, layer, 5, block, out, staging, p.gpu.workspace(5))
+            rc, _ = p.orc.append(layer, seqs, list(range(6)), bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags.numpy())
+            assert rc == 0
+            oo, ol = p.orc.attention_batch(layer, seqs, bf16_bits(q).numpy())
+            calls.append((block, out, oo, ol))
+    P.pask_decode_step_drain(h)
+    torch.cuda.synchronize()
+    for block, out, oo, ol in calls:
+        assert_close(out.numpy().astype(np.float64), ol.copy(), oo, ol)
+    p.compare_state()
