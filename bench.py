@@ -616,7 +616,7 @@ def main():
     ap.add_argument("--bias", default="balanced", choices=["balanced", "low", "high"])
     ap.add_argument("--no-full-kv", dest="full_kv", action="store_false")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="0 skips the CPU-oracle leg")
-    ap.add_argument("--event-stride", type=int, default=4, help="time the streaming kernel of every n-th launch")
+    ap.add_argument("--event-stride", type=int, default=9, help="time the streaming kernel of every n-th launch")
     ap.add_argument("--low-bits", type=int, default=4, choices=[4, 8], help="width of the RETAIN-LOW codes")
     ap.add_argument("--unfused", action="store_true",
                     help="issue pask_append_kv and pask_decode_attention separately instead of pask_append_attend")
