@@ -340,14 +340,15 @@ def run_cuda(args, rank, world):
     if args.layers:
         cfg = WC.scaled(cfg, n_layers=args.layers, name=f"{cfg.name}[first {args.layers} layers]")
     total_steps = args.warmup + args.steps
-    e2e_steps = min(args.steps, 5)
-    cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, 2 * total_steps + e2e_steps + 8))
+    e2e_steps = min(args.steps, 10)
+    e2e_warm = 2                       # untimed end-to-end steps (the first call creates the library's copy streams)
+    cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, 2 * total_steps + e2e_steps + e2e_warm + 8))
     w = rank_workload(cfg, rank)
     if args.window:
         from dataclasses import replace as _replace
         w.policy = _replace(w.policy, recent_window=args.window)
     t_setup = time.time()
-    job = Job(P, w, device, 2 * total_steps + e2e_steps + 4, dynamic=args.dynamic)
+    job = Job(P, w, device, 2 * total_steps + e2e_steps + e2e_warm + 4, dynamic=args.dynamic)
     job.fused = not args.unfused
     # launches per layer: append (+ plan), streaming kernel, combine
     per_layer_launches = 3 if (job.fused and job.B <= 255 and not args.window) else 4
@@ -401,7 +402,7 @@ def run_cuda(args, rank, world):
         staging = torch.empty(2 * P.pask_step_staging_bytes(job.cache.handle, job.B), dtype=torch.uint8, device=device)
         off, in_bytes = P.pask_step_packed_layout(job.cache.handle, job.B)
         host = []
-        for s in range(e2e_steps):          # a layer's inputs sit in one pinned block, as an engine would stage them
+        for s in range(e2e_warm + e2e_steps):   # a layer's inputs sit in one pinned block, as an engine would stage them
             rows = []
             for layer in range(cfg.n_layers):
                 k, v, q, tags = step_inputs(w, layer, total_steps + s, "cpu")
@@ -414,10 +415,14 @@ def run_cuda(args, rank, world):
                 rows.append(block)
             host.append(rows)
         out_h = torch.empty((job.B, cfg.n_q, 128), dtype=torch.float32).pin_memory()
+        for rows in host[:e2e_warm]:
+            for layer, block in enumerate(rows):
+                P.pask_decode_step_pipelined(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
+        P.pask_decode_step_drain(job.cache.handle)
         barrier()
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0.record()
-        for rows in host:
+        for rows in host[e2e_warm:]:
             for layer, block in enumerate(rows):
                 P.pask_decode_step_pipelined(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
         P.pask_decode_step_drain(job.cache.handle)      # the host holds every output before the clock stops
