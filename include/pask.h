@@ -19,6 +19,11 @@
  *     and changes no counter.
  *   - Every dev pointer must be 16-byte aligned; the pools and meta 256-byte aligned.
  *   - One host thread drives a cache at a time; ordering between calls is stream order.
+ *   - Calls that only enqueue work (append, decide, attention, pask_append_attend) may be recorded by
+ *     a stream capture and replayed as a CUDA graph: nothing that changes from call to call is passed
+ *     by value, a replay works on whatever the recorded device buffers hold then.  Not for capture:
+ *     calls that wait for the stream (pask_budget_state, pask_debug_*), the host-buffer steps, and the
+ *     first pask_decode_attention_static call on a device.
  *   - Supported shapes: head_dim 128, 16-token pages, n_q_heads = 4 * n_kv_heads with
  *     n_kv_heads in {1, 2, 4, 8}.  Anything else: PASK_ERR_UNSUPPORTED_SHAPE.
  *   - No function throws or aborts.

@@ -193,7 +193,6 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     if (!c) return PASK_ERR_INVALID_ARG;
     c->desc = *d;
     c->meta = meta;
-    c->append_serial = 0;
     c->sm_count = sms;
     c->ev_start = c->ev_stop = nullptr;
     c->off = meta_offsets(d, 255, PASK_MAX_GROUPS);
@@ -309,7 +308,6 @@ pask_status_t pask_cache_reset(pask_cache_t *c, pask_stream_t stream_v) {
     uint8_t *m = static_cast<uint8_t *>(c->meta);
     cudaError_t e = cudaMemsetAsync(m + c->off.ctrl, 0, kCtrlWords * 4, stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m + c->off.zero_begin, 0, c->off.zero_end - c->off.zero_begin, stream);
-    c->append_serial = 0;
     return cuda_rc(e);
 }
 

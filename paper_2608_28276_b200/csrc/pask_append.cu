@@ -63,7 +63,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *s_warp
 __global__ void __launch_bounds__(kPlanThreads)
 append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const int32_t *__restrict__ seq_ids,
                    const int32_t *__restrict__ cu_tokens, const uint8_t *__restrict__ tags,
-                   const uint8_t *__restrict__ decided, uint8_t *__restrict__ actions_out, uint32_t serial) {
+                   const uint8_t *__restrict__ decided, uint8_t *__restrict__ actions_out) {
     __shared__ uint8_t s_lut[256];
     __shared__ uint32_t s_wh[2 * (kPlanThreads / 32)], s_wb[2 * (kPlanThreads / 32)];
     __shared__ uint32_t s_scan[kPlanThreads / 32];
@@ -72,6 +72,9 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
     const int i = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int group = c.layer_group[layer];
     s_lut[tid] = tid < c.n_tags ? c.lut[tid * c.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
+    // this launch's serial: every CTA reads it before its arrival ticket, the CTA arriving last stores it back
+    uint32_t serial = c.ctrl[kCtrlSerial] + 1u;
+    if (serial == 0) serial = 1;
     const int seq = seq_ids[i];
     const int t0 = cu_tokens[i], t1 = cu_tokens[i + 1];
     uint32_t err = 0;
@@ -210,6 +213,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         if (tid == 0) {
             if (!fits && !any_bad) atomicOr(&c.ctrl[kCtrlStatus], PASK_DEV_POOL_EXHAUSTED);
             c.ctrl[kCtrlPlanOk] = 0;
+            c.ctrl[kCtrlSerial] = serial;
             c.ctrl[kCtrlTicket] = 0;
         }
         return;
@@ -267,6 +271,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
         c.ctrl[kCtrlItems] = n_items;
         c.item_base[n_seqs] = n_items;
         c.ctrl[kCtrlPlanOk] = 1;
+        c.ctrl[kCtrlSerial] = serial;
         c.ctrl[kCtrlTicket] = 0;
     }
 }
@@ -926,9 +931,8 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
                                          fuse ? *fuse_ws : Workspace{});
         return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
     }
-    if (++c->append_serial == 0) c->append_serial = 1;
     append_plan_kernel<<<n_seqs, kPlanThreads, 0, stream>>>(c->dev, layer, n_seqs, total_tokens, seq_ids, cu_tokens, tags,
-                                                           decided, actions_out, c->append_serial);
+                                                           decided, actions_out);
     if (total_tokens > 0) {
         // at most one item per 16 tokens plus two partly filled pages per stream
         const long long bound = (long long)total_tokens / 16 + 4LL * n_seqs;

@@ -27,13 +27,17 @@ __device__ __forceinline__ uint32_t act_of(uint32_t packed, int g) { return (pac
 __global__ void __launch_bounds__(kDecideThreads)
 decide_kernel(DevCache c, int n_seqs, int total_tokens, const int32_t *__restrict__ seq_ids,
               const int32_t *__restrict__ cu_tokens, const uint8_t *__restrict__ tags,
-              const uint16_t *__restrict__ states, uint8_t *__restrict__ actions_out, uint32_t serial) {
+              const uint16_t *__restrict__ states, uint8_t *__restrict__ actions_out) {
     __shared__ uint2 s_row[256];
     __shared__ float2 s_rho[255 * PASK_MAX_GROUPS];   // upgrade scores: read inside the Demote / Promote loops
     __shared__ uint32_t s_layers[PASK_MAX_GROUPS];
     __shared__ int s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = c.n_groups;
+    // this launch's serial (for spotting a sequence named twice): read by every CTA before its arrival
+    // ticket, stored back by the CTA that arrives last
+    uint32_t serial = c.ctrl[kCtrlSerial] + 1u;
+    if (serial == 0) serial = 1;
     s_row[tid] = c.dec_row[tid];
     for (int x = tid; x < c.n_tags * G; x += kDecideThreads) s_rho[x] = c.dec_rho[x];
     if (tid < PASK_MAX_GROUPS) s_layers[tid] = c.group_layers[tid];
@@ -170,17 +174,16 @@ decide_kernel(DevCache c, int n_seqs, int total_tokens, const int32_t *__restric
             b.n_floor_conflicts += u.p.conflicts;
         }
     }
-    if (tid == 0) c.ctrl[kCtrlTicket] = 0;
+    if (tid == 0) { c.ctrl[kCtrlSerial] = serial; c.ctrl[kCtrlTicket] = 0; }
 }
 
 }  // namespace
 
 pask_status_t launch_decide(pask_cache *c, int n_seqs, int total_tokens, const int32_t *seq_ids, const int32_t *cu_tokens,
                             const uint8_t *tags, const uint16_t *states, uint8_t *actions_out, cudaStream_t stream) {
-    if (++c->append_serial == 0) c->append_serial = 1;
     const int ctas = (n_seqs + kDecideWarps - 1) / kDecideWarps;
     decide_kernel<<<ctas, kDecideThreads, 0, stream>>>(c->dev, n_seqs, total_tokens, seq_ids, cu_tokens, tags, states,
-                                                      actions_out, c->append_serial);
+                                                      actions_out);
     return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }
 

@@ -20,6 +20,8 @@ enum CtrlWord : int {
     kCtrlLowFree = 5,
     kCtrlPlanOk = 6,    // 1 if the last append plan was committed, 0 if it was refused
     kCtrlItems = 7,     // work items (stream pages touched) of the last committed bulk append
+    kCtrlSerial = 8,    // serial of the last launch that marks sequences (duplicate detection); kept on the device so
+                        // that a launch recorded in a CUDA graph gets a fresh one at every replay
     kCtrlStats = 16,    // 8 words of decode-attention wait statistics (diagnostic builds with PASK_STATS only)
     kCtrlWords = 64
 };
@@ -120,7 +122,6 @@ struct pask_cache {
     pask::DevCache dev;
     pask::MetaOffsets off;
     void *meta;
-    uint32_t append_serial;
     std::vector<uint8_t> lut, layer_group;   // host copies of the folded table [n_tags][n_groups] and the layer map
     int sm_count;
     int attn_ctas;                // grid of the decode-attention main kernel

@@ -122,3 +122,68 @@ def test_refused_append_inside_the_fused_call(pask, oracle):
     assert st.device_status & pask.DEV_POOL_EXHAUSTED and st.full_bytes == 0
     assert pask.pask_debug_stream_len(p.gpu.handle, 0, 0) == (0, 0)
     assert pask.pask_debug_pool_state(p.gpu.handle) == (0, 0, 0, 0)
+
+
+def test_a_step_replayed_as_a_cuda_graph(pask, oracle):
+    # the calls of a step only enqueue work, so a stream capture can record them; replaying the
+    # graph must leave the same state and outputs as issuing the calls
+    from pask_workloads.tensors import bf16_bits
+    p, w = _pair(pask, oracle, 6, 120, 60, dynamic=True)
+    seqs = list(range(6))
+    lens = [w.total_len(s) for s in seqs]
+    tags, states = p.gather(seqs, lens, [0] * 6)
+    _, act_o, act_g = p.decide(seqs, lens, tags, states)
+    for layer in range(w.cfg.n_layers):
+        _, _, k, v = p.gather(seqs, lens, [0] * 6, layer)
+        p.append_decided(layer, seqs, lens, k, v, tags, act_o, act_g)
+    d = "cuda"
+    ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+    cu = torch.arange(7, dtype=torch.int32, device=d)
+    G, L = w.cfg.n_groups, w.cfg.n_layers
+    # static buffers the graph reads from and writes to
+    tg = torch.zeros(6, dtype=torch.uint8, device=d)
+    st = torch.zeros(6, dtype=torch.int16, device=d)
+    act = torch.zeros((6, G), dtype=torch.uint8, device=d)
+    ks = [torch.zeros((6, w.cfg.n_kv, 128), dtype=torch.bfloat16, device=d) for _ in range(L)]
+    vs = [torch.zeros_like(ks[0]) for _ in range(L)]
+    qs = [torch.zeros((6, w.cfg.n_q, 128), dtype=torch.bfloat16, device=d) for _ in range(L)]
+    outs = [torch.zeros((6, w.cfg.n_q, 128), dtype=torch.float32, device=d) for _ in range(L)]
+    lse = torch.zeros((6, w.cfg.n_q), dtype=torch.float32, device=d)
+    ws = p.gpu.workspace(6)
+    # warm the kernels up outside the capture on a throw-away cache (captures must not see first-use set-up)
+    warm, _ = _pair(pask, oracle, 6, 120, 60, dynamic=True)
+    pask.pask_decide(warm.gpu.handle, ids, cu, tg, st, act)
+    pask.pask_append_attend(warm.gpu.handle, 0, ids, cu, ks[0], vs[0], tg, qs[0], outs[0], lse, warm.gpu.workspace(6), actions=act)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            pask.pask_decide(p.gpu.handle, ids, cu, tg, st, act)
+            for layer in range(L):
+                pask.pask_append_attend(p.gpu.handle, layer, ids, cu, ks[layer], vs[layer], tg, qs[layer], outs[layer], lse, ws,
+                                        actions=act)
+    torch.cuda.current_stream().wait_stream(side)
+    pos = list(lens)
+    for step in range(5):                                               # the same graph, new inputs each time
+        tags, states = p.gather(seqs, [1] * 6, pos)
+        tg.copy_(torch.from_numpy(tags)); st.copy_(torch.from_numpy(states.astype(np.int16)))
+        rc, a_o = p.orc.decide(seqs, list(range(7)), tags, states=states, n_groups=G)
+        assert rc == 0
+        want = []
+        for layer in range(L):
+            _, _, k, v = p.gather(seqs, [1] * 6, pos, layer)
+            q = torch.stack([w.q(layer, s, pos[s] + 1) for s in seqs])
+            ks[layer].copy_(k); vs[layer].copy_(v); qs[layer].copy_(q)
+            rc, _ = p.orc.append(layer, seqs, list(range(7)), bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags, decided=a_o)
+            assert rc == 0
+            want.append(p.orc.attention_batch(layer, seqs, bf16_bits(q).numpy()))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(act.cpu().numpy(), a_o)
+        for layer in range(L):
+            go = outs[layer].cpu().numpy().astype(np.float64)
+            assert_close(go, want[layer][1].copy(), want[layer][0], want[layer][1], where=(step, layer))
+        pos = [x + 1 for x in pos]
+    p.compare_state()
