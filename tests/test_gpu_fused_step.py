@@ -187,3 +187,42 @@ def test_a_step_replayed_as_a_cuda_graph(pask, oracle):
             assert_close(go, want[layer][1].copy(), want[layer][0], want[layer][1], where=(step, layer))
         pos = [x + 1 for x in pos]
     p.compare_state()
+
+
+def test_bulk_append_replayed_as_a_cuda_graph(pask, oracle):
+    # the two-kernel bulk path recorded once and replayed on new data: the duplicate check and the
+    # page numbering must behave as if the call had been issued each time
+    from pask_workloads.tensors import bf16_bits
+    p, w = _pair(pask, oracle, 3, 700, 100)
+    d = "cuda"
+    seqs = [2, 0, 1]
+    counts = [200, 170, 150]
+    total = sum(counts)
+    ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(counts)]), dtype=torch.int32, device=d)
+    k = torch.zeros((total, w.cfg.n_kv, 128), dtype=torch.bfloat16, device=d)
+    v = torch.zeros_like(k)
+    tg = torch.zeros(total, dtype=torch.uint8, device=d)
+    used = torch.zeros(total, dtype=torch.uint8, device=d)
+    warm, _ = _pair(pask, oracle, 3, 700, 100)
+    pask.pask_append_kv(warm.gpu.handle, 0, ids, cu, k, v, tg, actions_out=used, total_tokens=total)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            pask.pask_append_kv(p.gpu.handle, 0, ids, cu, k, v, tg, actions_out=used, total_tokens=total)
+    torch.cuda.current_stream().wait_stream(side)
+    start = {s: 0 for s in seqs}
+    for rep in range(3):
+        tags, _, kk, vv = p.gather(seqs, counts, [start[s] for s in seqs], 0)
+        k.copy_(kk); v.copy_(vv); tg.copy_(torch.from_numpy(tags))
+        rc, act_o = p.orc.append(0, seqs, cu.cpu().numpy(), bf16_bits(kk).numpy(), bf16_bits(vv).numpy(), tags)
+        assert rc == 0
+        graph.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(used.cpu().numpy(), act_o)
+        start = {s: start[s] + n for s, n in zip(seqs, counts)}
+        p.compare_state(layers=[0])
+    p.check_attention(0, [0, 1, 2], pos=600)
