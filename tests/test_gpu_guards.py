@@ -110,3 +110,38 @@ def test_stream_filled_exactly_to_its_bound():
     assert P.pask_budget_state(cache.handle, 0).device_status == P.DEV_SEQ_OVERFLOW
     assert P.pask_debug_stream_len(cache.handle, 0, 0) == (64, 0)
     cache.close()
+
+
+def test_everything_on_a_side_stream_and_after_a_cache_reset(oracle):
+    import paper_2608_28276_b200 as pask
+    # every call on a non-default stream (nothing may lean on the legacy default stream), with busy
+    # work queued in front so that a missing dependency would show; then the cache is reset, used
+    # again with decided actions and a window, and still agrees with a fresh oracle
+    from dataclasses import replace
+    from pask_workloads import policy as WP
+    from parity import Pair
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=3, n_layers=2, n_groups=2, prompt_len=200, gen_len=100, extra_gen=32)
+    w = WC.build(cfg)
+    blob = WP.write_blob(replace(w.policy, recent_window=16))
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        p = Pair(pask, oracle, w, blob=blob)
+        busy = torch.randn((4096, 4096), device="cuda")
+        for rnd in range(2):
+            for _ in range(6):
+                busy = busy @ busy * 1e-4                               # keeps the stream occupied ahead of the library's work
+            seqs = [1, 2, 0]
+            for layer in range(2):
+                p.append(layer, seqs, [250, 260, 270], [0, 0, 0])
+            for step in range(3):
+                for layer in range(2):
+                    p.append(layer, seqs, [1, 1, 1], [250 + step, 260 + step, 270 + step])
+            p.compare_state()
+            for layer in range(2):
+                p.check_attention(layer, [0, 1, 2], pos=273)
+            if rnd == 0:                                                # wipe both sides and go again
+                pask.pask_cache_reset(p.gpu.handle)
+                p.orc = oracle.Cache(oracle.Policy(blob), cfg.n_q, cfg.n_kv, p.max_seqs, p.hp, p.lp)
+                assert pask.pask_debug_pool_state(p.gpu.handle) == (0, 0, 0, 0)
+                assert pask.pask_budget_state(p.gpu.handle, 1).full_bytes == 0
+    torch.cuda.synchronize()
