@@ -226,3 +226,19 @@ def test_bulk_append_replayed_as_a_cuda_graph(pask, oracle):
         start = {s: start[s] + n for s, n in zip(seqs, counts)}
         p.compare_state(layers=[0])
     p.check_attention(0, [0, 1, 2], pos=600)
+
+
+def test_fused_step_with_nothing_retained(pask, oracle):
+    # every token released: the plan is empty, outputs are zero and lse is -inf, through the one-call form too
+    a = np.zeros((11, 4), np.uint8)
+    z = np.zeros((11, 4), np.float32)
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=3, prompt_len=40, gen_len=20, extra_gen=16)
+    w = WC.build(cfg)
+    pol = WP.Policy(11, 4, WP.equal_layer_groups(4, 4), a, a.copy(), z, z.copy(), np.zeros(1, np.uint32), budget_target=0.0)
+    p = Pair(pask, oracle, w, blob=WP.write_blob(pol))
+    for step in range(3):
+        for layer in range(4):
+            out, lse, _ = _step(p, layer, [2, 0, 1], [1, 1, 1], [step] * 3)
+            assert torch.all(out == 0) and torch.all(torch.isinf(lse) & (lse < 0))
+    assert pask.pask_debug_pool_state(p.gpu.handle) == (0, 0, 0, 0)
+    p.compare_state()
