@@ -85,7 +85,7 @@ def f16_bits_to_f32(h: int) -> float:
 
 
 def quantize_group(x_bits: np.ndarray, bits: int = 4):
-    """32 bf16 bit patterns -> (fp16 scale bit pattern, 32 codes); bits = 4 or 8."""
+    """32 bf16 bit patterns -> (fp16 scale bit pattern, 32 codes); bits = 2, 4 or 8."""
     x = np.ascontiguousarray(x_bits, dtype=np.uint16)
     assert x.shape == (32,)
     s = np.zeros(1, np.uint16)

@@ -27,7 +27,8 @@
  * tags) are the library's documented ones: RETAIN-LOW is symmetric int4 per token, per KV head,
  * per group of 32 consecutive head dimensions with one fp16 scale (amax/7, round to nearest
  * even, codes stored offset by 8) -- or, policy low_bits = 8, symmetric int8 in the same grouping
- * (amax/127, codes offset by 128); RETAIN-HIGH keeps the bf16 bits; pages hold 16 tokens and
+ * (amax/127, codes offset by 128), or, low_bits = 2, the three levels -s, 0, +s with s = amax
+ * (codes offset by 2); RETAIN-HIGH keeps the bf16 bits; pages hold 16 tokens and
  * are handed out in call order from a per-pool free stack, else a bump counter; costs are
  * payload bytes.  Parity unpinned by the paper for: the low-bit format itself, the size of the
  * recent window (a policy parameter here, 0 by default; the paper gives no number) and that a
@@ -168,10 +169,12 @@ float orc_f16_to_f32(uint16_t h) {
 
 /* RETAIN-LOW of one group of 32 values (bf16 bit patterns in): one fp16 scale, 32 codes.
  * bits = 4: codes clamp(rint(x / s), -7, 7) + 8 with s = fp16(amax / 7);
- * bits = 8: codes clamp(rint(x / s), -127, 127) + 128 with s = fp16(amax / 127). */
+ * bits = 8: codes clamp(rint(x / s), -127, 127) + 128 with s = fp16(amax / 127);
+ * bits = 2: codes clamp(rint(x / s), -1, 1) + 2 with s = fp16(amax) (three levels: -s, 0, +s).
+ * In general the largest level is 2^(bits-1) - 1 and the code of zero 2^(bits-1). */
 void orc_quantize_group_bits(const uint16_t *x_bits, uint16_t *scale_bits, uint8_t *codes, int bits) {
-    const float qmax = bits == 8 ? 127.0f : 7.0f;
-    const int zero = bits == 8 ? 128 : 8;
+    const float qmax = (float)((1 << (bits - 1)) - 1);
+    const int zero = 1 << (bits - 1);
     float amax = 0.0f;
     for (int i = 0; i < QGROUP; i++) {
         float a = fabsf(bf16_to_f32(x_bits[i]));
@@ -224,7 +227,7 @@ orc_policy *orc_policy_load(const uint8_t *blob, size_t len, int *err) {
     p->low_bits = rd32(blob + 32); p->group_size = rd32(blob + 36);
     if (p->n_tags == 0 || p->n_tags > 255 || p->n_groups == 0 || p->n_groups > MAX_GROUPS ||
         p->n_layers == 0 || p->n_layers > 4096 || p->n_states > (1u << 20) || p->recent_window % PAGE_TOKENS != 0 || p->recent_window > MAX_WINDOW ||
-        (p->low_bits != 4 && p->low_bits != 8) || p->group_size != QGROUP) { free(p); return NULL; }
+        (p->low_bits != 4 && p->low_bits != 8 && p->low_bits != 2) || p->group_size != QGROUP) { free(p); return NULL; }
     size_t lg_pad = (p->n_layers + 3u) & ~(size_t)3u;
     size_t n_ent = (size_t)p->n_tags * p->n_groups;
     size_t need = 40 + lg_pad + n_ent * 12 + (size_t)p->n_states * 4;
@@ -607,7 +610,7 @@ static void attention_head(orc_cache *c, int layer, int seq, int h, const uint16
     orc_stream *s = stream_of(c, seq, layer);
     const int kv = h / (c->n_q / c->n_kv);
     const size_t row = (size_t)c->n_kv * HEAD_DIM, srow = (size_t)c->n_kv * GROUPS_PER_HEAD;
-    const int zero = c->pol->low_bits == 8 ? 128 : 8;                 /* the code that stands for 0 */
+    const int zero = 1 << (c->pol->low_bits - 1);                     /* the code that stands for 0 */
     const uint32_t W = c->pol->recent_window;
     const size_t nw = W ? (s->n_tok < W ? s->n_tok : W) : 0;          /* tokens in the window */
     size_t win_h = 0, win_l = 0;

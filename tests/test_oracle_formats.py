@@ -187,6 +187,44 @@ def test_quantizer8_degenerate_groups_and_symmetry(oracle):
         assert sb == sb2 and np.array_equal(codes2.astype(np.int64) - 128, -(codes.astype(np.int64) - 128))
 
 
+# ---- the 2-bit variant (policy low_bits = 2): three levels -s, 0, +s with s = fp16(amax)
+
+def test_quantizer2_is_the_nearest_of_three_levels(oracle):
+    for scale in (1.0, 1e-3, 1e3):
+        for xb in _groups(31, 600, scale):
+            x = _bf16_val(xb).astype(np.float64)
+            sb, codes = oracle.quantize_group(xb, bits=2)
+            assert sb == int(np.float16(np.float32(np.abs(x).max())).view(np.uint16))      # amax / 1
+            s = Fraction(float(np.array([sb], np.uint16).view(np.float16)[0]))
+            assert set(codes.tolist()) <= {1, 2, 3}
+            for xi, c in zip(x, codes):
+                # brute force over the three levels in exact arithmetic; a value half-way goes to the even level 0
+                d = [abs(Fraction(float(xi)) - lv * s) for lv in (-1, 0, 1)]
+                best = min(d)
+                picks = [lv for lv, di in zip((-1, 0, 1), d) if di - best <= s * Fraction(1, 1 << 16)]
+                assert (int(c) - 2) in picks
+                if len(picks) > 1 and abs(abs(Fraction(float(xi))) - s / 2) == 0:
+                    assert int(c) == 2
+
+
+def test_quantizer2_degenerate_groups_and_symmetry(oracle):
+    sb, codes = oracle.quantize_group(np.zeros(32, np.uint16), bits=2)
+    assert sb == 0 and np.all(codes == 2)
+    xb = _bf16_bits(np.full(32, 1e-9, np.float32))                  # scale underflows to zero
+    sb, codes = oracle.quantize_group(xb, bits=2)
+    assert sb == 0 and np.all(codes == 2)
+    xb = _bf16_bits(np.array([1e7, -1e7] * 16, np.float32))         # scale saturates, codes clamp
+    sb, codes = oracle.quantize_group(xb, bits=2)
+    assert sb == 0x7BFF and set(codes.tolist()) == {1, 3}
+    xb = _bf16_bits(np.array([1.0, 0.5, 0.25, -0.5, -0.75, -1.0, 0.0, 0.51] * 4, np.float32))
+    sb, codes = oracle.quantize_group(xb, bits=2)                   # ties at half the scale go to the even level 0
+    assert sb == 0x3C00 and codes[:8].tolist() == [3, 2, 2, 2, 1, 1, 2, 3]
+    for xb in _groups(32, 300):
+        sb, codes = oracle.quantize_group(xb, bits=2)
+        sb2, codes2 = oracle.quantize_group(xb ^ np.uint16(0x8000), bits=2)
+        assert sb == sb2 and np.array_equal(codes2.astype(np.int64) - 2, -(codes.astype(np.int64) - 2))
+
+
 def test_eight_bit_is_finer_than_four_bit(oracle):
     # the same group at both widths: the 8-bit reconstruction error is never larger than half a 4-bit step
     for xb in _groups(24, 300):

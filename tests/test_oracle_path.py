@@ -366,3 +366,32 @@ def test_eight_bit_low_stream_against_library_attention(oracle):
     b = c.budget(0)
     n_l, n_h = int((act == 1).sum()), int((act == 2).sum())
     assert b.retained_bytes == n_h * H_BYTES[2] + n_l * 2 * 2 * (128 + 8)   # codes at one byte each + scales
+
+
+def test_two_bit_low_stream_against_library_attention(oracle):
+    # policy low_bits = 2: the LOW stream holds the codes 1, 2, 3 and is attended as (code - 2) * scale
+    from dataclasses import replace
+    n = 200
+    pol = replace(_policy([[1], [2], [0], [1]]), low_bits=2)
+    c = _mk(oracle, pol)
+    k, v = _rand_kv(9, n, 2)
+    tags = (np.arange(n) % 4).astype(np.uint8)
+    act = _append(c, 0, 0, k, v, tags)
+    kc, ks, vc, vs, _ = c.dump_low(0, 0)
+    assert set(np.unique(kc).tolist()) == {1, 2, 3} and set(np.unique(vc).tolist()) == {1, 2, 3}
+    hk, hv, _ = c.dump_high(0, 0)
+    s = lambda b: b.view(np.float16).astype(np.float64)
+    dq = lambda codes, sc: (codes.astype(np.float64) - 2.0) * np.repeat(s(sc), 32, axis=-1)
+    from_bits = lambda b: torch.from_numpy(b.astype(np.int32) << 16).view(torch.float32).double()
+    K = torch.cat([from_bits(hk), torch.from_numpy(dq(kc, ks))])
+    V = torch.cat([from_bits(hv), torch.from_numpy(dq(vc, vs))])
+    q = normal_bf16(8, 0, 0, 0, n, 1, 8)[0]
+    out, lse = c.attention(0, 0, bf16_bits(q).numpy())
+    ro, rl = _ref_attention(q, K, V)
+    assert np.abs(out - ro.numpy()).max() < 1e-12 and np.abs(lse - rl.numpy()).max() < 1e-12
+    # every value is within half a step of its level, the step being the group's amax
+    kl = k[act == 1].double().numpy()
+    assert np.abs(dq(kc, ks) - kl).max() <= 0.5 * s(ks).max() * 1.01
+    b = c.budget(0)
+    n_l, n_h = int((act == 1).sum()), int((act == 2).sum())
+    assert b.retained_bytes == n_h * H_BYTES[2] + n_l * 2 * 2 * (32 + 8)     # four codes per byte + scales
