@@ -319,7 +319,7 @@ class Job:
                 win_h[b], win_l[b] = (acts == 2).sum(0), (acts == 1).sum(0)
         for l in range(cfg.n_layers):
             nh, nl = self.nh[:, lg[l]] + steps_done - win_h[:, lg[l]] + self.window, self.nl[:, lg[l]] - win_l[:, lg[l]]
-            tot += float((nh * cfg.n_kv * 512).sum() + (nl * cfg.n_kv * (272 if self.low_bits == 8 else 144)).sum())
+            tot += float((nh * cfg.n_kv * 512).sum() + (nl * cfg.n_kv * {8: 272, 4: 144, 2: 80}[self.low_bits]).sum())
             tot += float((((nh + 15) // 16) + ((nl + 15) // 16)).sum() * 4)
         per_layer = tot / cfg.n_layers
         per_layer += self.B * cfg.n_q * 128 * 2
@@ -622,7 +622,7 @@ def main():
     ap.add_argument("--no-full-kv", dest="full_kv", action="store_false")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="0 skips the CPU-oracle leg")
     ap.add_argument("--event-stride", type=int, default=9, help="time the streaming kernel of every n-th launch")
-    ap.add_argument("--low-bits", type=int, default=4, choices=[4, 8], help="width of the RETAIN-LOW codes")
+    ap.add_argument("--low-bits", type=int, default=4, choices=[2, 4, 8], help="width of the RETAIN-LOW codes")
     ap.add_argument("--unfused", action="store_true",
                     help="issue pask_append_kv and pask_decode_attention separately instead of pask_append_attend")
     ap.add_argument("--window", type=int, default=0, help="protected recent window in tokens (multiple of 16, <= 256)")

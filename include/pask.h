@@ -37,6 +37,8 @@
  *   m(L) = 2 * n_kv * (64 + 8), m(H) = 2 * n_kv * 256.
  *   A policy with low_bits = 8 keeps RETAIN-LOW at eight bits instead: s = fp16(amax / 127), codes
  *   clamp(rint(x * (1 / s)), -127, 127) + 128, value (code - 128) * s, m(L) = 2 * n_kv * (128 + 8).
+ *   A policy with low_bits = 2 keeps three levels: s = fp16(amax), codes clamp(rint(x * (1 / s)), -1, 1) + 2,
+ *   value (code - 2) * s, m(L) = 2 * n_kv * (32 + 8).
  */
 #ifndef PASK_H_
 #define PASK_H_
@@ -97,7 +99,7 @@ typedef struct {
     uint32_t pool_low_pages;    /* capacity of the int4 page pool */
     int32_t recent_window;      /* the policy's protected recent window W (0, or a multiple of 16 up to
                                    PASK_MAX_WINDOW); sizes W/16 bf16 pages per (sequence, layer) behind the bf16 pool */
-    int32_t low_bits;           /* the policy's low_bits: 4 (0 means 4) or 8; sizes the pages of the low pool */
+    int32_t low_bits;           /* the policy's low_bits: 4 (0 means 4), 8 or 2; sizes the pages of the low pool */
 } pask_cache_desc_t;
 
 typedef struct {
@@ -105,7 +107,7 @@ typedef struct {
     size_t pool_low_bytes;
     size_t meta_bytes;      /* counters, page tables, budget states, free stacks, append scratch */
     size_t high_page_bytes; /* n_kv * 8192: per KV head a 16x128 bf16 K tile then V tile */
-    size_t low_page_bytes;  /* n_kv * 2304 (4-bit codes) or n_kv * 4352 (8-bit): per KV head K codes, K scales, V codes, V scales */
+    size_t low_page_bytes;  /* n_kv * 2304 (4-bit codes), n_kv * 4352 (8-bit) or n_kv * 1280 (2-bit): per KV head K codes, K scales, V codes, V scales */
 } pask_cache_sizes_t;
 
 /* Constant-size per-sequence budget state (Algorithm 2's R_t with the counts it is made of).
@@ -144,7 +146,7 @@ typedef struct {
  *   blob (host, len bytes), little endian:
  *     "PASK", u32 version (1 or 2), u32 n_tags (1..255), u32 n_groups (1..8), u32 n_layers,
  *     u32 n_states, u32 budget_target_q16, u32 recent_window (0, or a multiple of 16 up to
- *     PASK_MAX_WINDOW: the protected recent window in tokens, see pask_decode_attention), u32 low_bits (4 or 8),
+ *     PASK_MAX_WINDOW: the protected recent window in tokens, see pask_decode_attention), u32 low_bits (4, 8 or 2),
  *     u32 group_size (32),
  *     u8 layer_group[n_layers] zero-padded to 4 bytes,
  *     n_tags*n_groups entries, tag-major: u8 a0, u8 a_floor, u16 0, f32 rho_RL, f32 rho_LH

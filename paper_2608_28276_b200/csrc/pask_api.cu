@@ -62,7 +62,7 @@ size_t window_pages(const pask_cache_desc_t *d) {
 bool desc_ok(const pask_cache_desc_t *d) {
     return d->n_layers > 0 && d->n_layers <= 4096 && d->max_seqs > 0 && d->max_tokens_per_seq > 0 &&
            d->max_append_tokens > 0 && d->recent_window >= 0 && d->recent_window <= PASK_MAX_WINDOW &&
-           d->recent_window % kPageTokens == 0 && (d->low_bits == 0 || d->low_bits == 4 || d->low_bits == 8);
+           d->recent_window % kPageTokens == 0 && (d->low_bits == 0 || d->low_bits == 4 || d->low_bits == 8 || d->low_bits == 2);
 }
 
 pask_status_t cuda_rc(cudaError_t e) { return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA; }
@@ -117,7 +117,7 @@ pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **o
     p->low_bits = rd32(blob + 32);
     const uint32_t window = p->window, low_bits = rd32(blob + 32), group_size = rd32(blob + 36);
     bool ok = p->n_tags >= 1 && p->n_tags <= 255 && p->n_groups >= 1 && p->n_groups <= PASK_MAX_GROUPS &&
-              p->n_layers >= 1 && p->n_layers <= 4096 && p->n_states <= (1u << 20) && window <= PASK_MAX_WINDOW && window % kPageTokens == 0 && (low_bits == 4 || low_bits == 8) &&
+              p->n_layers >= 1 && p->n_layers <= 4096 && p->n_states <= (1u << 20) && window <= PASK_MAX_WINDOW && window % kPageTokens == 0 && (low_bits == 4 || low_bits == 8 || low_bits == 2) &&
               group_size == (uint32_t)kQGroup;
     const size_t lg_pad = ok ? align_up(p->n_layers, 4) : 0;
     const size_t n_ent = ok ? (size_t)p->n_tags * p->n_groups : 0;
@@ -166,7 +166,7 @@ pask_status_t pask_cache_sizes(const pask_cache_desc_t *d, pask_cache_sizes_t *o
     if (!shape_ok(d)) return PASK_ERR_UNSUPPORTED_SHAPE;
     if (!desc_ok(d)) return PASK_ERR_INVALID_ARG;
     out->high_page_bytes = (size_t)d->n_kv_heads * kHighHeadBytes;
-    out->low_page_bytes = (size_t)d->n_kv_heads * (d->low_bits == 8 ? kLow8HeadBytes : kLowHeadBytes);
+    out->low_page_bytes = (size_t)d->n_kv_heads * (d->low_bits == 8 ? kLow8HeadBytes : d->low_bits == 2 ? kLow2HeadBytes : kLowHeadBytes);
     out->pool_high_bytes = out->high_page_bytes * ((size_t)d->pool_high_pages + window_pages(d));
     out->pool_low_bytes = out->low_page_bytes * d->pool_low_pages;
     out->meta_bytes = meta_offsets(d, 255, PASK_MAX_GROUPS).total;  // independent of the policy loaded later
@@ -240,8 +240,8 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     v.budget_q16 = pol->budget_q16;
     v.high_page_bytes = (uint32_t)d->n_kv_heads * kHighHeadBytes;
     v.low_bits = pol->low_bits;
-    v.low_head_bytes = pol->low_bits == 8 ? kLow8HeadBytes : kLowHeadBytes;
-    v.cost_low_page = pol->low_bits == 8 ? kCostLow8Page : kCostLowPage;
+    v.low_head_bytes = pol->low_bits == 8 ? kLow8HeadBytes : pol->low_bits == 2 ? kLow2HeadBytes : kLowHeadBytes;
+    v.cost_low_page = pol->low_bits == 8 ? kCostLow8Page : pol->low_bits == 2 ? kCostLow2Page : kCostLowPage;
     v.low_page_bytes = (uint32_t)d->n_kv_heads * v.low_head_bytes;
     v.bytes_h = 2u * d->n_kv_heads * kHeadDim * 2u;
     v.bytes_l = 2u * d->n_kv_heads * (kHeadDim * pol->low_bits / 8 + kGroupsPerHead * 2);
@@ -672,6 +672,18 @@ pask_status_t pask_debug_dump_low(pask_cache_t *c, int32_t layer, int32_t seq, u
                     for (int dd = 0; dd < kHeadDim; dd++) {
                         kc[dd] = kh[low8_k_off((int)tau, dd)];
                         vc[dd] = v8[low8_v_off((int)tau, dd)];
+                    }
+                    continue;
+                }
+                if (c->dev.low_bits == 2) {
+                    const uint8_t *v2 = kh + kLow2HalfBytes;
+                    for (int w = 0; w < 4; w++) {
+                        std::memcpy(ks + w, kh + low2_scale_off((int)tau, w), 2);
+                        std::memcpy(vs + w, v2 + low2_scale_off((int)tau, w), 2);
+                    }
+                    for (int dd = 0; dd < kHeadDim; dd++) {
+                        kc[dd] = (kh[low2_k_byte_off((int)tau, dd >> 3, dd & 1)] >> (2 * ((dd >> 1) & 3))) & 3;
+                        vc[dd] = (v2[low2_v_byte_off((int)tau, dd >> 2)] >> (2 * (dd & 3))) & 3;
                     }
                     continue;
                 }

@@ -341,6 +341,30 @@ __device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uin
         if ((threadIdx.x & 31) == 0 && hb8 > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb8);
         return;
     }
+    if (c.low_bits == 2) {   // two-bit codes: the levels -s, 0, +s with s = fp16(amax), codes offset by 2
+        uint8_t *dst2 = c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLow2HeadBytes + (which ? kLow2HalfBytes : 0);
+        __half sh2 = __float2half_rn(amax);
+        if (__hisinf(sh2)) sh2 = __ushort_as_half((unsigned short)0x7BFF);
+        const float s2 = __half2float(sh2);
+        const float inv2 = s2 == 0.0f ? 0.0f : __fdiv_rn(1.0f, s2);
+        uint32_t code2[8];
+#pragma unroll
+        for (int e = 0; e < 8; e++) {   // clamp, then 1.5 * 2^23 + 2 leaves the rounded code in the low two bits
+            const float cl = fminf(fmaxf(__fmul_rn(f[e], inv2), -1.0f), 1.0f);
+            code2[e] = __float_as_uint(__fadd_rn(cl, 12582914.0f)) & 3u;
+        }
+        if (!which) {   // even dims in one byte, odd dims in the other
+            dst2[low2_k_byte_off((int)tau, cch, 0)] = (uint8_t)(code2[0] | (code2[2] << 2) | (code2[4] << 4) | (code2[6] << 6));
+            dst2[low2_k_byte_off((int)tau, cch, 1)] = (uint8_t)(code2[1] | (code2[3] << 2) | (code2[5] << 4) | (code2[7] << 6));
+        } else {        // four consecutive dims per byte
+            dst2[low2_v_byte_off((int)tau, 2 * cch)] = (uint8_t)(code2[0] | (code2[1] << 2) | (code2[2] << 4) | (code2[3] << 6));
+            dst2[low2_v_byte_off((int)tau, 2 * cch + 1)] = (uint8_t)(code2[4] | (code2[5] << 2) | (code2[6] << 4) | (code2[7] << 6));
+        }
+        if ((cch & 3) == 0) *reinterpret_cast<__half *>(dst2 + low2_scale_off((int)tau, cch >> 2)) = sh2;
+        const uint32_t hb2 = __reduce_max_sync(0xffffffffu, which ? (uint32_t)__half_as_ushort(sh2) : 0u);
+        if ((threadIdx.x & 31) == 0 && hb2 > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb2);
+        return;
+    }
     uint8_t *dst = c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLowHeadBytes + (which ? kLowHalfBytes : 0);
     const float s32 = __fdiv_rn(amax, 7.0f);
     __half sh = __float2half_rn(s32);
@@ -531,6 +555,40 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
                     __syncthreads();
                     uint4 *dst8 = reinterpret_cast<uint4 *>(c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLow8HeadBytes);
                     for (int x = tid; x < kLow8HeadBytes / 16; x += kWriteThreads) dst8[x] = reinterpret_cast<const uint4 *>(&s_low[0][0])[x];
+                    continue;
+                }
+                if (c.low_bits == 2) {
+                    // two-bit codes: this thread's 16 values are the chunks 4w + 2 half, +1 of its token's row
+                    __half sh2 = __float2half_rn(amax);
+                    if (__hisinf(sh2)) sh2 = __ushort_as_half((unsigned short)0x7BFF);
+                    const float s2 = __half2float(sh2);
+                    const float inv2 = s2 == 0.0f ? 0.0f : __fdiv_rn(1.0f, s2);
+                    uint32_t c2[16];
+#pragma unroll
+                    for (int e = 0; e < 16; e++) {
+                        const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
+                        const float cl = fminf(fmaxf(__fmul_rn(f, inv2), -1.0f), 1.0f);
+                        c2[e] = __float_as_uint(__fadd_rn(cl, 12582914.0f)) & 3u;
+                    }
+                    uint8_t *img2 = s_low[head & 1] + (which ? kLow2HalfBytes : 0);
+                    if (!which) {
+#pragma unroll
+                        for (int cc = 0; cc < 2; cc++)
+#pragma unroll
+                            for (int e = 0; e < 2; e++)
+                                img2[low2_k_byte_off(tau, 4 * w + 2 * half + cc, e)] =
+                                    (uint8_t)(c2[8 * cc + e] | (c2[8 * cc + 2 + e] << 2) | (c2[8 * cc + 4 + e] << 4) | (c2[8 * cc + 6 + e] << 6));
+                    } else {
+#pragma unroll
+                        for (int uu = 0; uu < 4; uu++)
+                            img2[low2_v_byte_off(tau, 8 * w + 4 * half + uu)] =
+                                (uint8_t)(c2[4 * uu] | (c2[4 * uu + 1] << 2) | (c2[4 * uu + 2] << 4) | (c2[4 * uu + 3] << 6));
+                        vmax_bits = max(vmax_bits, (uint32_t)__half_as_ushort(sh2));
+                    }
+                    if (half == 0) *reinterpret_cast<__half *>(img2 + low2_scale_off(tau, w)) = sh2;
+                    __syncthreads();
+                    uint4 *dst2 = reinterpret_cast<uint4 *>(c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLow2HeadBytes);
+                    if (tid < kLow2HeadBytes / 16) dst2[tid] = reinterpret_cast<const uint4 *>(s_low[head & 1])[tid];
                     continue;
                 }
                 const float s32 = __fdiv_rn(amax, 7.0f);

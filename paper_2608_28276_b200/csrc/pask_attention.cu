@@ -181,6 +181,8 @@ __device__ __forceinline__ uint32_t nib_odd(uint32_t x) {
     asm("lop3.b32 %0, %1, 0x00F000F0, 0x64006400, 0xEA;" : "=r"(d) : "r"(x));
     return d;
 }
+// field i (bits 2i, 2i+1 of byte 0) of both half-words as the fp16 pair 1024 + 4^i code
+__device__ __forceinline__ uint32_t two_bit(uint32_t x, int i) { return (x & (0x00030003u << (2 * i))) | 0x64006400u; }
 __device__ __forceinline__ uint32_t hsub2(uint32_t a, uint32_t b) {
     uint32_t d;
     asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
@@ -398,7 +400,7 @@ struct Pipe {
     }
 };
 
-// kLow: 0 = the LOW stream is compiled out (full high-precision cache), 4 / 8 = width of its codes
+// kLow: 0 = the LOW stream is compiled out (full high-precision cache), 2 / 4 / 8 = width of its codes
 template <int kLow>
 __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __grid_constant__ AttnParams p) {
     constexpr bool kHasLow = kLow != 0;
@@ -455,11 +457,11 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     Pipe w;
     w.order = p.ws.order;
     w.base_high = c.pool_high + (size_t)warp * kHighHeadBytes;
-    w.base_low = c.pool_low + (size_t)warp * (kLow == 8 ? kLow8HeadBytes : kLowHeadBytes);
+    w.base_low = c.pool_low + (size_t)warp * (kLow == 8 ? kLow8HeadBytes : kLow == 2 ? kLow2HeadBytes : kLowHeadBytes);
     w.stride_high = c.high_page_bytes;
     w.stride_low = c.low_page_bytes;
     w.low_two = kLow == 8;
-    w.low_job_bytes = kLow == 8 ? kLow8HalfBytes : kLowHeadBytes;
+    w.low_job_bytes = kLow == 8 ? kLow8HalfBytes : kLow == 2 ? kLow2HeadBytes : kLowHeadBytes;
     w.status = c.ctrl + kCtrlStatus;
     w.policy = l2_evict_first_policy();
     w.lane = lane;
@@ -523,11 +525,16 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 for (int i = 0; i < 4; i++) {
                     const float f0 = bf_lo(r[i]), f1 = bf_hi(r[i]);
                     too_big |= fabsf(f0) > 65504.f || fabsf(f1) > 65504.f;
-                    // (8-bit codes: every A operand is 1024 + code, so q is stored as is and the offset is 1152)
-                    const float sc = (kLow == 4 && (i & 1)) ? 0.0625f : 1.0f;
+                    // (8-bit codes: every A operand is 1024 + code, so q is stored as is and the offset is 1152;
+                    // 2-bit codes: pair i of a chunk comes out as 1024 + 4^i code, so q is divided by 4^i and the
+                    // offset is 1024 + 2 * 4^i)
+                    const float sc = kLow == 4 ? ((i & 1) ? 0.0625f : 1.0f)
+                                   : kLow == 2 ? (i == 0 ? 1.0f : i == 1 ? 0.25f : i == 2 ? 0.0625f : 0.015625f) : 1.0f;
+                    const float offs = kLow == 8 ? 1152.f : kLow == 4 ? ((i & 1) ? 1152.f : 1032.f)
+                                     : (i == 0 ? 1026.f : i == 1 ? 1032.f : i == 2 ? 1056.f : 1152.f);
                     h[i] = pack_f16(f0 * sc, f1 * sc);
                     const float2 bq = unpack_f16(h[i]);
-                    seed -= ((kLow == 8 || (i & 1)) ? 1152.f : 1032.f) * (bq.x + bq.y);
+                    seed -= offs * (bq.x + bq.y);
                 }
                 seed += __shfl_xor_sync(0xffffffffu, seed, 1);
                 seed += __shfl_xor_sync(0xffffffffu, seed, 2);
@@ -605,6 +612,29 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                                  prmt(kw[j].y, 0x64646464u, 0x4140), prmt(kw[j].y, 0x64646464u, 0x4342), qa.x, qa.y, seed);
                     mma_f16(cj, prmt(kw[j].z, 0x64646464u, 0x4140), prmt(kw[j].z, 0x64646464u, 0x4342),
                             prmt(kw[j].w, 0x64646464u, 0x4140), prmt(kw[j].w, 0x64646464u, 0x4342), qb.x, qb.y);
+                    const float s0f = (j & 1) ? f0[j >> 1].y : f0[j >> 1].x;
+                    const float s1f = (j & 1) ? f1[j >> 1].y : f1[j >> 1].x;
+                    sc[0] = fmaf(s0f, cj[0], sc[0]);
+                    sc[1] = fmaf(s0f, cj[1], sc[1]);
+                    sc[2] = fmaf(s1f, cj[2], sc[2]);
+                    sc[3] = fmaf(s1f, cj[3], sc[3]);
+                }
+            } else if (kLow == 2) {
+                // ---- QK^T over 2-bit K codes: one word per 32-dim group holds both token rows of this lane
+                const uint4 kq = lds128(st + lane * 16);
+                const uint2 ks0 = lds64(st + kLow2CodesBytes + g * 8);
+                const uint2 ks1 = lds64(st + kLow2CodesBytes + (g + 8) * 8);
+                const uint32_t kwd[4] = {kq.x, kq.y, kq.z, kq.w};
+                const float2 f0[2] = {unpack_f16(ks0.x), unpack_f16(ks0.y)};
+                const float2 f1[2] = {unpack_f16(ks1.x), unpack_f16(ks1.y)};
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint4 qa = lds128(scratch + j * 256 + (g & 3) * 64 + t * 16);
+                    const uint4 seed = lds128(scratch + 1024 + ((t & 1) * 4 + j) * 16);
+                    float cj[4];
+                    const uint32_t x = kwd[j], y = x >> 8;      // byte 0: token g, byte 1: token g + 8
+                    mma_f16_seed(cj, two_bit(x, 0), two_bit(y, 0), two_bit(x, 1), two_bit(y, 1), qa.x, qa.y, seed);
+                    mma_f16(cj, two_bit(x, 2), two_bit(y, 2), two_bit(x, 3), two_bit(y, 3), qa.z, qa.w);
                     const float s0f = (j & 1) ? f0[j >> 1].y : f0[j >> 1].x;
                     const float s1f = (j & 1) ? f1[j >> 1].y : f1[j >> 1].x;
                     sc[0] = fmaf(s0f, cj[0], sc[0]);
@@ -726,6 +756,35 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                                     hsub2(prmt(w1, 0x64646464u, 0x4140), 0x64806480u),
                                     hsub2(prmt(w1, 0x64646464u, 0x4342), 0x64806480u), b0, b1);
                         }
+                    }
+                }
+            } else if (kLow == 2) {
+                // ---- P.V over 2-bit V codes: fields 0, 1 of a byte are rows g, g+8 of tile 2q, fields 2, 3 of tile 2q+1
+                const uint32_t vb2 = st + kLow2HalfBytes;
+                const uint4 vq = lds128(vb2 + lane * 16);        // byte 0: tokens 2t, 2t+1; byte 1: tokens 2t+8, 2t+9
+                uint2 vs0 = lds64(vb2 + kLow2CodesBytes + g * 8);
+                uint2 vs1 = lds64(vb2 + kLow2CodesBytes + (g + 8) * 8);
+                w.release();   // everything of this stage is in registers now
+                if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
+                    if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
+                    if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
+                }
+                const uint32_t cw[4] = {vq.x, vq.y, vq.z, vq.w};
+                const uint32_t p01 = pack_f16(p0, p1), p23 = pack_f16(p2, p3);
+#pragma unroll
+                for (int v = 0; v < 2; v++) {
+                    const uint32_t s0b = hmul2(prmt(v ? vs0.y : vs0.x, 0u, bsel), down);
+                    const uint32_t s1b = hmul2(prmt(v ? vs1.y : vs1.x, 0u, bsel), down);
+                    const uint32_t b0 = movmatrix_trans(hmul2(p01, s0b)), b1 = movmatrix_trans(hmul2(p23, s1b));
+#pragma unroll
+                    for (int qq = 0; qq < 2; qq++) {
+                        const int q = 2 * v + qq;
+                        const uint32_t x = cw[q], y = x >> 8;
+                        // (1024 + 4^i code) / 4^i - (1024 / 4^i + 2) = code - 2, exact in fp16
+                        mma_f16(acc[2 * q], hsub2(two_bit(x, 0), 0x64026402u), hfma2(two_bit(x, 1), 0x34003400u, 0xDC08DC08u),
+                                hsub2(two_bit(y, 0), 0x64026402u), hfma2(two_bit(y, 1), 0x34003400u, 0xDC08DC08u), b0, b1);
+                        mma_f16(acc[2 * q + 1], hfma2(two_bit(x, 2), 0x2C002C00u, 0xD420D420u), hfma2(two_bit(x, 3), 0x24002400u, 0xCC80CC80u),
+                                hfma2(two_bit(y, 2), 0x2C002C00u, 0xD420D420u), hfma2(two_bit(y, 3), 0x24002400u, 0xCC80CC80u), b0, b1);
                     }
                 }
             } else if (kHasLow) {
@@ -897,7 +956,8 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
     p.q = static_cast<const uint4 *>(q);
     carve_workspace(c, n_seqs, static_cast<uint8_t *>(workspace), &p.ws);
     const size_t smem = attn_smem_bytes(n_seqs, n_warps);
-    auto kern = !has_low ? decode_attn_kernel<0> : c->dev.low_bits == 8 ? decode_attn_kernel<8> : decode_attn_kernel<4>;
+    auto kern = !has_low ? decode_attn_kernel<0> : c->dev.low_bits == 8 ? decode_attn_kernel<8>
+              : c->dev.low_bits == 2 ? decode_attn_kernel<2> : decode_attn_kernel<4>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return PASK_ERR_CUDA;
     cudaError_t e = cudaSuccess;

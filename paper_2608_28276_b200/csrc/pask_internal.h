@@ -85,7 +85,7 @@ struct DevCache {
     uint32_t budget_q16;
     uint32_t high_page_bytes, low_page_bytes;
     uint32_t bytes_h, bytes_l;       // m(H), m(L) per token per layer
-    uint32_t low_bits;               // 4 or 8: width of the RETAIN-LOW codes
+    uint32_t low_bits;               // 2, 4 or 8: width of the RETAIN-LOW codes
     uint32_t low_head_bytes;         // one KV head of a LOW page (2304 or 4352)
     uint32_t cost_low_page;          // cost of a LOW page in units of n_kv * 256 bytes (9 or 17)
 };

@@ -35,6 +35,17 @@
 //              {dim D tokens 2t,2t+1 | dim D+1 tokens 2t,2t+1 | dim D tokens 2t+8,+9 | dim D+1 tokens
 //              2t+8,+9} with D = 32q + 4g + 2r: the A operand of the P.V tile whose rows g, g+8 are
 //              dims D, D+1 (the row order the bf16 and 4-bit paths use too).
+// LOW page, 2-bit codes (policy low_bits = 2):
+//              [kv head][K codes 512][K scales 128][V codes 512][V scales 128]     (n_kv * 1280 B)
+//   K codes  : one round of 512 B; lane (g,t) holds 4 words j (one per 32-dim group); in word j the
+//              low half-word holds even dims and the high one odd dims, byte 0 of either token g and
+//              byte 1 token g+8, and the field at bits 2i of a byte dims 32j + 8t + 2i (+1): so
+//              ((word >> 8 hi) & (0x00030003 << 2i)) | 0x64006400 is the fp16 pair 1024 + 4^i code of an
+//              A register, and the eight dims of a token's 16-byte chunk fill two whole bytes.
+//   V codes  : one round of 512 B; lane (g,t) holds 4 words q; low half-word token 2t (+8 in byte 1),
+//              high half-word token 2t+1 (+8 in byte 1); the field at bits 2i of a byte is dim
+//              32q + 4g + i: fields 0, 1 are rows g, g+8 of P.V tile 2q, fields 2, 3 of tile 2q+1
+//              (the row order of the other formats).
 #pragma once
 #include <stdint.h>
 
@@ -59,10 +70,14 @@ constexpr int kLowHeadBytes = 2304;
 constexpr int kLow8CodesBytes = 2048;
 constexpr int kLow8HalfBytes = 2176;  // codes + scales of K (or of V), 8-bit codes
 constexpr int kLow8HeadBytes = 4352;
+constexpr int kLow2CodesBytes = 512;
+constexpr int kLow2HalfBytes = 640;   // codes + scales of K (or of V), 2-bit codes
+constexpr int kLow2HeadBytes = 1280;
 // cost of streaming one page (all heads), in units of n_kv * 256 bytes
 constexpr uint32_t kCostHighPage = 32;
 constexpr uint32_t kCostLowPage = 9;
 constexpr uint32_t kCostLow8Page = 17;
+constexpr uint32_t kCostLow2Page = 5;
 
 // HIGH K tile: offset of the 4-byte piece holding dims 2p, 2p+1 (p = 0..63) of token tau.
 PASK_HD int high_k_pair_off(int tau, int p) {
@@ -105,6 +120,17 @@ PASK_HD int low8_v_off(int tau, int d) {
     return q * 512 + (4 * g + t) * 16 + (i >> 1) * 8 + (tau >> 3) * 4 + (i & 1) * 2 + (tau & 1);
 }
 PASK_HD int low8_scale_off(int tau, int w) { return kLow8CodesBytes + tau * 8 + w * 2; }
+
+// 2-bit LOW K codes: byte offset of the byte holding dims {8c + 2i + e, i = 0..3} (c = 0..15 the
+// 16-byte chunk of the token's row, e = 0 even / 1 odd dims) of token tau; dim 8c + 2i + e sits at bits 2i
+PASK_HD int low2_k_byte_off(int tau, int c, int e) {
+    return (4 * (tau & 7) + (c & 3)) * 16 + (c >> 2) * 4 + e * 2 + (tau >> 3);
+}
+// 2-bit LOW V codes (relative to the V half): byte holding dims 4u .. 4u+3 (u = 0..31) of token tau; dim 4u + i at bits 2i
+PASK_HD int low2_v_byte_off(int tau, int u) {
+    return (4 * (u & 7) + ((tau & 7) >> 1)) * 16 + (u >> 3) * 4 + (tau & 1) * 2 + (tau >> 3);
+}
+PASK_HD int low2_scale_off(int tau, int w) { return kLow2CodesBytes + tau * 8 + w * 2; }
 
 // ---- work partition of decode attention -------------------------------------------------
 // Every sequence's pages are visited in one fixed order that interleaves its HIGH and LOW pages

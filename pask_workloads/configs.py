@@ -38,7 +38,7 @@ class Config:
     mode: str = "grammar"            # "grammar" | "mix"
     lut: str = "greedy"              # "greedy" | "random" | "all_high"
     bias: str = "balanced"           # greedy table flavour: "balanced" | "low" | "high"
-    low_bits: int = 4                # width of the RETAIN-LOW codes: 4 or 8
+    low_bits: int = 4                # width of the RETAIN-LOW codes: 2, 4 or 8
     protected_prompt: bool = False   # prompt tokens carry TAG_PROTECTED (tiny)
     extra_gen: int = 64              # generated tokens beyond gen_len kept ready for decode steps
 

@@ -77,7 +77,7 @@ def test_bad_blobs_and_arguments_are_refused(pask):
     broken = bytearray(good); broken[40 + 4] = 3; bads.append(bytes(broken))           # action out of range
     broken = bytearray(good); broken[28] = 1; bads.append(bytes(broken))               # recent window not a multiple of 16
     broken = bytearray(good); broken[29] = 2; bads.append(bytes(broken))               # recent window too large (512)
-    broken = bytearray(good); broken[32] = 6; bads.append(bytes(broken))               # low_bits neither 4 nor 8
+    broken = bytearray(good); broken[32] = 6; bads.append(bytes(broken))               # low_bits none of 2, 4, 8
     broken = bytearray(good); broken[40] = 9; bads.append(bytes(broken))               # layer group out of range
     for b in bads:
         with pytest.raises(pask.PaskError) as e:

@@ -24,7 +24,8 @@ def pask():
 
 
 @pytest.mark.parametrize("seed,n_kv,window,low_bits", [(1, 2, 0, 4), (2, 8, 0, 4), (3, 4, 16, 4), (4, 1, 48, 4), (5, 8, 0, 4),
-                                                       (6, 2, 0, 4), (7, 8, 0, 8), (8, 2, 32, 8), (9, 1, 0, 8)])
+                                                       (6, 2, 0, 4), (7, 8, 0, 8), (8, 2, 32, 8), (9, 1, 0, 8), (10, 8, 0, 2),
+                                                       (11, 2, 16, 2), (12, 4, 0, 2)])
 def test_random_call_sequences(pask, oracle, seed, n_kv, window, low_bits):
     from dataclasses import replace
     rng = CounterRng(seed, 4242)
