@@ -448,7 +448,7 @@ def run_cuda(args, rank, world):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16/int4 storage, bf16 tensor-core operands with fp32 accumulation", "data": "synthetic",
+        "dtype": f"bf16/int{job.low_bits} storage, bf16 / fp16 tensor-core operands with fp32 accumulation", "data": "synthetic",
         "config": {"workload": cfg.name, "batch_per_gpu": job.B, "layers": cfg.n_layers, "layer_groups": cfg.n_groups,
                    "kv_budget_target": cfg.budget, "kv_budget_realised": ret / full, "table": f"greedy/{cfg.bias}",
                    "recent_window": args.window,
