@@ -60,6 +60,7 @@ typedef int32_t pask_status_t;
 #define PASK_ERR_CUDA (-6)
 #define PASK_ERR_TIMEOUT (-7)
 #define PASK_ERR_WORKSPACE (-8)
+#define PASK_ERR_NO_MEMORY (-9)   /* host memory for a handle or a staging copy could not be had */
 
 /* Sticky bits of the device status word (pask_budget_state_t.device_status). */
 #define PASK_DEV_POOL_EXHAUSTED 0x1u  /* an append needed more pages than a pool had: nothing written */

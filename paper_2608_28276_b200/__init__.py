@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libpask.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_POLICY, ERR_UNSUPPORTED_SHAPE, ERR_POOL_EXHAUSTED = -1, -2, -3, -4
-ERR_BAD_SEQ, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE = -5, -6, -7, -8
+ERR_BAD_SEQ, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE, ERR_NO_MEMORY = -5, -6, -7, -8, -9
 DEV_POOL_EXHAUSTED, DEV_BAD_SEQ, DEV_SEQ_OVERFLOW, DEV_BAD_RAGGED, DEV_TIMEOUT, DEV_RANGE, DEV_INTERNAL = 1, 2, 4, 8, 16, 32, 64
 DEV_BAD_ACTION = 128
 ACTION_RELEASE, ACTION_RETAIN_LOW, ACTION_RETAIN_HIGH = 0, 1, 2

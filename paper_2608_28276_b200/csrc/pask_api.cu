@@ -1,5 +1,6 @@
 // Host side of libpask: policy blobs, cache set-up, budget state, canonical dumps.
 #include <cstring>
+#include <memory>
 #include <new>
 
 #include "pask_internal.h"
@@ -95,19 +96,20 @@ const char *pask_status_string(pask_status_t s) {
         case PASK_ERR_CUDA: return "CUDA runtime error";
         case PASK_ERR_TIMEOUT: return "device wait timed out";
         case PASK_ERR_WORKSPACE: return "workspace too small";
+        case PASK_ERR_NO_MEMORY: return "out of host memory";
         default: return "unknown status";
     }
 }
 
-pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **out) {
+pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **out) try {
     if (!blob_v || !out) return PASK_ERR_INVALID_ARG;
     *out = nullptr;
     const uint8_t *blob = static_cast<const uint8_t *>(blob_v);
     if (len < 40 || std::memcmp(blob, "PASK", 4) != 0) return PASK_ERR_BAD_POLICY;
     const uint32_t version = rd32(blob + 4);
     if (version != 1 && version != 2) return PASK_ERR_BAD_POLICY;
-    pask_policy *p = new (std::nothrow) pask_policy();
-    if (!p) return PASK_ERR_INVALID_ARG;
+    std::unique_ptr<pask_policy> p(new (std::nothrow) pask_policy());
+    if (!p) return PASK_ERR_NO_MEMORY;
     p->n_tags = rd32(blob + 8);
     p->n_groups = rd32(blob + 12);
     p->n_layers = rd32(blob + 16);
@@ -149,9 +151,11 @@ pask_status_t pask_load_policy(const void *blob_v, size_t len, pask_policy_t **o
             for (uint32_t s = 0; s < p->n_states; s++) { p->crit[s] = e[s]; ok = ok && e[s] <= 1; }
         }
     }
-    if (!ok) { delete p; return PASK_ERR_BAD_POLICY; }
-    *out = p;
+    if (!ok) return PASK_ERR_BAD_POLICY;
+    *out = p.release();
     return PASK_OK;
+} catch (...) {   // the tables could not be allocated
+    return PASK_ERR_NO_MEMORY;
 }
 
 void pask_free_policy(pask_policy_t *p) { delete p; }
@@ -174,7 +178,7 @@ pask_status_t pask_cache_sizes(const pask_cache_desc_t *d, pask_cache_sizes_t *o
 }
 
 pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t *pol, void *pool_high, void *pool_low,
-                                void *meta, pask_stream_t stream_v, pask_cache_t **out) {
+                                void *meta, pask_stream_t stream_v, pask_cache_t **out) try {
     if (!d || !pol || !meta || !out) return PASK_ERR_INVALID_ARG;
     *out = nullptr;
     if (!shape_ok(d)) return PASK_ERR_UNSUPPORTED_SHAPE;
@@ -189,8 +193,9 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     int dev_id = 0, sms = 0;
     if (cudaGetDevice(&dev_id) != cudaSuccess) return PASK_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_id) != cudaSuccess) return PASK_ERR_CUDA;
-    pask_cache *c = new (std::nothrow) pask_cache();
-    if (!c) return PASK_ERR_INVALID_ARG;
+    std::unique_ptr<pask_cache> holder(new (std::nothrow) pask_cache());
+    if (!holder) return PASK_ERR_NO_MEMORY;
+    pask_cache *c = holder.get();
     c->desc = *d;
     c->meta = meta;
     c->sm_count = sms;
@@ -279,11 +284,13 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     if (e == cudaSuccess && v.n_states_dev)
         e = cudaMemcpyAsync(v.crit, pol->crit.data(), (size_t)v.n_states_dev, cudaMemcpyHostToDevice, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
-    if (e != cudaSuccess) { delete c; return PASK_ERR_CUDA; }
+    if (e != cudaSuccess) return PASK_ERR_CUDA;
     pask_status_t rc = pask_cache_reset(c, stream_v);
-    if (rc != PASK_OK) { delete c; return rc; }
-    *out = c;
+    if (rc != PASK_OK) return rc;
+    *out = holder.release();
     return PASK_OK;
+} catch (...) {   // a host-side table could not be allocated
+    return PASK_ERR_NO_MEMORY;
 }
 
 void pask_cache_destroy(pask_cache_t *c) {
@@ -449,6 +456,7 @@ pask_status_t pask_decode_step_host(pask_cache_t *c, int32_t layer, int32_t n_se
     if (e == cudaSuccess) e = cudaMemcpyAsync(d_q, q_host, q_bytes, cudaMemcpyHostToDevice, stream);
     if (e != cudaSuccess) return PASK_ERR_CUDA;
     iota_kernel<<<(n_seqs + 1 + 255) / 256, 256, 0, stream>>>(d_cu, n_seqs + 1);
+    if (cudaPeekAtLastError() != cudaSuccess) return PASK_ERR_CUDA;
     pask_status_t rc = pask_append_attend(c, layer, n_seqs, n_seqs, d_ids, d_cu, d_k, d_v, d_tags, nullptr, nullptr, d_q, d_out,
                                           nullptr, ws, ws_bytes, stream_v);
     if (rc != PASK_OK) return rc;
@@ -603,7 +611,7 @@ pask_status_t pask_debug_page_ids(pask_cache_t *c, int32_t layer, int32_t seq, u
 }
 
 pask_status_t pask_debug_dump_high(pask_cache_t *c, int32_t layer, int32_t seq, uint16_t *k_out, uint16_t *v_out,
-                                   uint32_t *pages_out, pask_stream_t stream) {
+                                   uint32_t *pages_out, pask_stream_t stream) try {
     if (!c || !seq_layer_ok(c, layer, seq)) return PASK_ERR_INVALID_ARG;
     uint32_t nh = 0, nl = 0;
     pask_status_t rc = read_lens(c, layer, seq, &nh, &nl, static_cast<cudaStream_t>(stream));
@@ -635,10 +643,12 @@ pask_status_t pask_debug_dump_high(pask_cache_t *c, int32_t layer, int32_t seq, 
         }
     }
     return PASK_OK;
+} catch (...) {   // the staging copy could not be allocated
+    return PASK_ERR_NO_MEMORY;
 }
 
 pask_status_t pask_debug_dump_low(pask_cache_t *c, int32_t layer, int32_t seq, uint8_t *k_codes, uint16_t *k_scales,
-                                  uint8_t *v_codes, uint16_t *v_scales, uint32_t *pages_out, pask_stream_t stream) {
+                                  uint8_t *v_codes, uint16_t *v_scales, uint32_t *pages_out, pask_stream_t stream) try {
     if (!c || !seq_layer_ok(c, layer, seq)) return PASK_ERR_INVALID_ARG;
     uint32_t nh = 0, nl = 0;
     pask_status_t rc = read_lens(c, layer, seq, &nh, &nl, static_cast<cudaStream_t>(stream));
@@ -706,6 +716,8 @@ pask_status_t pask_debug_dump_low(pask_cache_t *c, int32_t layer, int32_t seq, u
         }
     }
     return PASK_OK;
+} catch (...) {   // the staging copy could not be allocated
+    return PASK_ERR_NO_MEMORY;
 }
 
 pask_status_t pask_debug_set_attention_ctas(pask_cache_t *c, int32_t n_ctas) {
@@ -715,7 +727,7 @@ pask_status_t pask_debug_set_attention_ctas(pask_cache_t *c, int32_t n_ctas) {
 }
 
 pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, const uint32_t *pages_low,
-                                   int32_t n_ctas, uint32_t *ranges) {
+                                   int32_t n_ctas, uint32_t *ranges) try {
     if (n_seqs < 1 || n_ctas < 1 || !pages_high || !pages_low || !ranges) return PASK_ERR_INVALID_ARG;
     std::vector<uint64_t> prefix((size_t)n_seqs + 1, 0);
     for (int s = 0; s < n_seqs; s++)
@@ -735,6 +747,8 @@ pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, c
         }
     }
     return PASK_OK;
+} catch (...) {   // the staging copy could not be allocated
+    return PASK_ERR_NO_MEMORY;
 }
 
 pask_status_t pask_debug_page_order(uint32_t pages_high, uint32_t pages_low, uint32_t *order) {

@@ -95,6 +95,7 @@ def test_bad_blobs_and_arguments_are_refused(pask):
         pask.pask_cache_sizes(pask.CacheDesc(0, 8, 2, 128, 16, 4, 1024, 1024, 8, 8))
     assert e.value.status == pask.ERR_INVALID_ARG
     assert pask.pask_status_string(pask.ERR_POOL_EXHAUSTED) == "page pool exhausted"
+    assert pask.pask_status_string(pask.ERR_NO_MEMORY) == "out of host memory"
 
 
 def test_decode_partition_covers_every_page_exactly_once(pask):
