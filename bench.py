@@ -351,7 +351,7 @@ def run_cuda(args, rank, world):
     job = Job(P, w, device, 2 * total_steps + e2e_steps + e2e_warm + 4, dynamic=args.dynamic)
     job.fused = not args.unfused
     # launches per layer: append (+ plan), streaming kernel, combine
-    per_layer_launches = 3 if (job.fused and job.B <= 255 and not args.window) else 4
+    per_layer_launches = 3 if (job.fused and job.B <= 255) else 4
     job.fill()
     job.prepare_steps(total_steps)
     t_setup = time.time() - t_setup

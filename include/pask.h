@@ -272,7 +272,7 @@ pask_status_t pask_decode_attention(pask_cache_t *cache, int32_t layer, int32_t 
 /* pask_append_attend -- one layer of a decode step in one call: pask_append_kv (or, with `actions`
  * != NULL, pask_append_kv_decided) for a ragged batch, then pask_decode_attention with one query
  * per sequence of the same batch.  Results are those of the two calls made one after the other.
- * For small batches (<= 255 sequences and tokens, no recent window) the append's single launch also
+ * For small batches (<= 255 sequences and tokens) the append's single launch also
  * writes the attention's work plan, which saves a launch per layer; otherwise the two calls are
  * simply issued in turn.  If the append is refused (sticky PASK_DEV_* bit) out and lse are
  * undefined.  Arguments as for the two calls. */

@@ -655,7 +655,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
                     uint8_t *__restrict__ actions_out, const SmallLut lut, const int fuse_plan, const Workspace ws) {
     __shared__ int s_seq[kSmallMax], s_cu[kSmallMax + 1];
     __shared__ uint32_t s_cost[kSmallMax + 1], s_page[kSmallMax + 1], s_nh[kSmallMax], s_nl[kSmallMax];   // fused attention plan
-    __shared__ uint32_t s_old_n[kSmallMax];
+    __shared__ uint32_t s_old_n[kSmallMax], s_nw[kSmallMax];
     __shared__ uint32_t s_old_h[kSmallMax], s_old_l[kSmallMax], s_cnt_h[kSmallMax], s_cnt_l[kSmallMax], s_cnt_bad[kSmallMax];
     __shared__ uint32_t s_new_h[kSmallMax], s_new_l[kSmallMax], s_base_h[kSmallMax], s_base_l[kSmallMax];
     __shared__ uint8_t s_act[kSmallMax], s_tok_seq[kSmallMax], s_tok_bad[kSmallMax];
@@ -767,17 +767,62 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     __syncthreads();
     // ---- fused decode-attention plan for the same sequences (what attn_plan_kernel would compute after
     // this append): every CTA knows every sequence's lengths after the call and the ids of the pages the
-    // call allocates, so the plan needs nothing that the commit writes.  Only without a recent window.
+    // call allocates, so the plan needs nothing that the commit writes.
     if (fuse_plan && !s_err) {
-        if (tid < n_seqs) { s_nh[tid] = s_old_h[tid] + s_cnt_h[tid]; s_nl[tid] = s_old_l[tid] + s_cnt_l[tid]; }
+        const uint32_t W = c.window;
+        if (tid < n_seqs) {
+            uint32_t nh = s_old_h[tid] + s_cnt_h[tid], nl = s_old_l[tid] + s_cnt_l[tid], nw = 0;
+            if (W) {
+                // The last min(W, tokens seen) tokens are attended from the bf16 ring whatever their action: the
+                // streams are shortened by the window's HIGH and LOW members.  Here those among this call's tokens
+                // (the last W of the sequence's tokens in the call at most) ...
+                const uint32_t n_i = (uint32_t)(s_cu[tid + 1] - s_cu[tid]), n_new = s_old_n[tid] + n_i;
+                nw = n_new < W ? n_new : W;
+                for (uint32_t r = n_i > W ? n_i - W : 0u; r < n_i; r++) {
+                    const uint32_t a = s_act[s_cu[tid] + r];
+                    nh -= a == PASK_ACTION_RETAIN_HIGH;
+                    nl -= a == PASK_ACTION_RETAIN_LOW;
+                }
+            }
+            s_nh[tid] = nh; s_nl[tid] = nl; s_nw[tid] = nw;
+        }
         if (tid == 0) s_cost[0] = s_page[0] = 0;
         __syncthreads();
+        if (W) {
+            // ... and here those among the older tokens still in the window: token indices [n_new - W, old_n), whose
+            // slots (index mod W) this call does not write.  One thread per 16 slots of a ring.
+            const int per = (int)W / kPageTokens;
+            for (int idx = tid; idx < n_seqs * per; idx += kSmallThreads) {
+                const int sq = idx / per, i = idx - sq * per;
+                const uint32_t old_n = s_old_n[sq], n_new = old_n + (uint32_t)(s_cu[sq + 1] - s_cu[sq]);
+                const uint32_t lo = n_new > W ? n_new - W : 0u;
+                if (lo >= old_n) continue;
+                const uint32_t len = old_n - lo, start = lo % W;
+                const size_t slw = (size_t)s_seq[sq] * c.n_layers + layer;
+                const uint4 a4 = reinterpret_cast<const uint4 *>(c.win_act + slw * W)[i];
+                const uint32_t w4[4] = {a4.x, a4.y, a4.z, a4.w};
+                uint32_t wh = 0, wl = 0;
+#pragma unroll
+                for (int b = 0; b < 16; b++) {
+                    const uint32_t a = (w4[b >> 2] >> (8 * (b & 3))) & 0xffu;
+                    const uint32_t j = 16u * (uint32_t)i + (uint32_t)b;
+                    const uint32_t d = j >= start ? j - start : j + W - start;   // distance from the oldest member's slot
+                    if (d < len) { wh += a == PASK_ACTION_RETAIN_HIGH; wl += a == PASK_ACTION_RETAIN_LOW; }
+                }
+                if (wh) atomicSub(&s_nh[sq], wh);
+                if (wl) atomicSub(&s_nl[sq], wl);
+            }
+            __syncthreads();
+        }
         if (tid < 32) {
             uint32_t carry_c = 0, carry_p = 0;
             for (int base = 0; base < n_seqs; base += 32) {
                 const int idx = base + tid;
                 uint32_t ph = 0, pl = 0;
-                if (idx < n_seqs) { ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens; pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens; }
+                if (idx < n_seqs) {   // the ring's pages have the HIGH format and count as HIGH pages
+                    ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens + (s_nw[idx] + kPageTokens - 1) / kPageTokens;
+                    pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens;
+                }
                 uint32_t ic = ph * kCostHighPage + pl * c.cost_low_page, ip = ph + pl;
 #pragma unroll
                 for (int d = 1; d < 32; d <<= 1) {
@@ -802,20 +847,26 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
                 if (s_page[mid] > gp) e = mid; else a = mid + 1;
             }
             const int s = a - 1;
-            const uint32_t nh = s_nh[s], nl = s_nl[s];
+            const uint32_t nh = s_nh[s], nl = s_nl[s], nw = s_nw[s];
             const uint32_t ph = (nh + kPageTokens - 1) / kPageTokens, pl = (nl + kPageTokens - 1) / kPageTokens;
-            const size_t sl = ((size_t)s_seq[s] * c.n_layers + layer) * c.max_pages;
+            const uint32_t pw = (nw + kPageTokens - 1) / kPageTokens;
+            const size_t slw = (size_t)s_seq[s] * c.n_layers + layer, sl = slw * c.max_pages;
             uint32_t idx, entry;
-            if (page_at(gp - s_page[s], ph, pl, idx)) {
+            if (page_at(gp - s_page[s], ph + pw, pl, idx)) {
                 const uint32_t old_pages = (s_old_h[s] + kPageTokens - 1) / kPageTokens;
-                if (idx < old_pages) {
-                    entry = c.tbl_high[sl + idx];
-                } else {             // a page this call allocates: the commit's formula
-                    const uint32_t kk = s_base_h[s] + (idx - old_pages);
-                    entry = kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]);
+                if (idx >= ph) {     // a page of the recent-window ring
+                    entry = c.cap_high + (uint32_t)slw * (W / kPageTokens) + (idx - ph);
+                    if (idx - ph == pw - 1) entry |= (nw & (kPageTokens - 1)) << kOrderValidShift;
+                } else {
+                    if (idx < old_pages) {
+                        entry = c.tbl_high[sl + idx];
+                    } else {         // a page this call allocates: the commit's formula
+                        const uint32_t kk = s_base_h[s] + (idx - old_pages);
+                        entry = kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]);
+                    }
+                    if (idx == ph - 1) entry |= (nh & (kPageTokens - 1)) << kOrderValidShift;
                 }
                 entry |= kOrderHigh;
-                if (idx == ph - 1) entry |= (nh & (kPageTokens - 1)) << kOrderValidShift;
             } else {
                 const uint32_t old_pages = (s_old_l[s] + kPageTokens - 1) / kPageTokens;
                 if (idx < old_pages) {
@@ -981,7 +1032,7 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
         for (int z = 0; z < 256; z++)
             lut.action[z] = z < c->dev.n_tags ? c->lut[(size_t)z * c->dev.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
         if (total_tokens == 0) return PASK_OK;
-        const int fuse = fuse_ws != nullptr && c->dev.window == 0;
+        const int fuse = fuse_ws != nullptr;
         if (fused) *fused = fuse != 0;
         const cudaError_t e = launch_pdl(append_small_kernel, dim3(total_tokens), dim3(kSmallThreads), 0, stream, c->dev, layer,
                                          group, n_seqs, total_tokens, seq_ids, cu_tokens, static_cast<const uint4 *>(k),

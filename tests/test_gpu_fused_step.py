@@ -56,7 +56,8 @@ def _pair(pask, oracle, batch, prompt, gen, window=0, dynamic=False, **kw):
     return Pair(pask, oracle, w, blob=blob, **kw), w
 
 
-@pytest.mark.parametrize("batch,window,dynamic", [(5, 0, False), (64, 0, False), (7, 0, True), (5, 32, False), (130, 0, False), (255, 0, False), (256, 0, False)])
+@pytest.mark.parametrize("batch,window,dynamic", [(5, 0, False), (64, 0, False), (7, 0, True), (5, 32, False), (130, 0, False), (255, 0, False), (256, 0, False),
+                                                  (64, 64, False), (5, 256, False), (7, 16, True), (200, 48, False)])
 def test_decode_steps(pask, oracle, batch, window, dynamic):
     prompt, gen = (40, 24) if batch > 8 else (150, 70)
     p, w = _pair(pask, oracle, batch, prompt, gen, window=window, dynamic=dynamic)
@@ -87,9 +88,12 @@ def test_decode_steps(pask, oracle, batch, window, dynamic):
     p.compare_state()
 
 
-def test_ragged_small_batches_and_identity_with_separate_calls(pask, oracle):
-    p, w = _pair(pask, oracle, 4, 100, 60)
-    q2, _ = _pair(pask, oracle, 4, 100, 60)                             # second cache: the two separate calls
+@pytest.mark.parametrize("window", [0, 16, 48, 256])
+def test_ragged_small_batches_and_identity_with_separate_calls(pask, oracle, window):
+    # with a recent window the one launch also counts the window's members: a ring that is not yet full,
+    # bursts longer than the window, and sequences that get nothing in a call
+    p, w = _pair(pask, oracle, 4, 100, 60, window=window)
+    q2, _ = _pair(pask, oracle, 4, 100, 60, window=window)              # second cache: the two separate calls
     seqs = [3, 1, 0, 2]
     pos = {s: 0 for s in seqs}
     for counts in ([1, 1, 1, 1], [16, 3, 0, 31], [40, 40, 40, 8], [1, 0, 0, 2], [33, 17, 16, 15]):
