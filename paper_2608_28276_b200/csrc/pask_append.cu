@@ -715,8 +715,11 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         return;
     }
     if (tid < total) {
-        int i = 0;                                   // the sequence this token belongs to
-        while (s_cu[i + 1] <= tid) i++;
+        int i = 0, i_hi = n_seqs - 1;                // the sequence this token belongs to: the first with s_cu[i + 1] > tid
+        while (i < i_hi) {
+            const int mid = (i + i_hi) >> 1;
+            if (s_cu[mid + 1] <= tid) i = mid + 1; else i_hi = mid;
+        }
         int a = lut.action[my_tag];
         if (decided) {   // Algorithm 2 step 7 on the actions pask_decide chose
             a = my_decided;
@@ -765,6 +768,24 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         if (tid == 0 && !fits && !s_err) atomicOr(&s_err, PASK_DEV_POOL_EXHAUSTED);
     }
     __syncthreads();
+    // old page of this CTA's token, if it continues one (page tables are only appended to by the commit)
+    uint32_t my_page = 0, my_at = 0;
+    const uint32_t my_a = s_act[my_tok];
+    const int my_i = s_tok_seq[my_tok];
+    const size_t my_sl = (size_t)s_seq[my_i] * c.n_layers + layer;
+    if (my_a != PASK_ACTION_RELEASE) {
+        const bool high = my_a == PASK_ACTION_RETAIN_HIGH;
+        const uint32_t old = high ? s_old_h[my_i] : s_old_l[my_i];
+        my_at = old + s_pos[my_tok];
+        const uint32_t old_pages = (old + kPageTokens - 1) / kPageTokens, pg = my_at >> 4;
+        if (pg < old_pages) {
+            my_page = (high ? c.tbl_high : c.tbl_low)[my_sl * c.max_pages + pg];
+        } else {   // one of the pages this call allocates: same formula as the commit below
+            const uint32_t kk = (high ? s_base_h[my_i] : s_base_l[my_i]) + (pg - old_pages);
+            const uint32_t fr = high ? s_ctrl[1] : s_ctrl[3], nx = high ? s_ctrl[0] : s_ctrl[2];
+            my_page = kk < fr ? (high ? c.free_high : c.free_low)[fr - 1 - kk] : nx + (kk - fr);
+        }
+    }
     // ---- fused decode-attention plan for the same sequences (what attn_plan_kernel would compute after
     // this append): every CTA knows every sequence's lengths after the call and the ids of the pages the
     // call allocates, so the plan needs nothing that the commit writes.
@@ -879,24 +900,31 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             }
             ws.order[gp] = entry;
         }
-    
     }
-    // old page of this CTA's token, if it continues one (page tables are only appended to by the commit)
-    uint32_t my_page = 0, my_at = 0;
-    const uint32_t my_a = s_act[my_tok];
-    const int my_i = s_tok_seq[my_tok];
-    const size_t my_sl = (size_t)s_seq[my_i] * c.n_layers + layer;
-    if (my_a != PASK_ACTION_RELEASE) {
-        const bool high = my_a == PASK_ACTION_RETAIN_HIGH;
-        const uint32_t old = high ? s_old_h[my_i] : s_old_l[my_i];
-        my_at = old + s_pos[my_tok];
-        const uint32_t old_pages = (old + kPageTokens - 1) / kPageTokens, pg = my_at >> 4;
-        if (pg < old_pages) {
-            my_page = (high ? c.tbl_high : c.tbl_low)[my_sl * c.max_pages + pg];
-        } else {   // one of the pages this call allocates: same formula as the commit below
-            const uint32_t kk = (high ? s_base_h[my_i] : s_base_l[my_i]) + (pg - old_pages);
-            const uint32_t fr = high ? s_ctrl[1] : s_ctrl[3], nx = high ? s_ctrl[0] : s_ctrl[2];
-            my_page = kk < fr ? (high ? c.free_high : c.free_low)[fr - 1 - kk] : nx + (kk - fr);
+    uint32_t pre_h = 0, pre_l = 0;
+    // The token's bytes go out before the arrival ticket: nothing that another CTA still reads is written
+    // (pages are only read by later kernels; the ring slots written are those of this call's tokens), the call
+    // can no longer be refused (s_err is final), and the stores overlap the ticket's round trip.
+    if (!s_err) {
+        // ids of the first page each sequence gets from this call, fetched now for the commit
+        if (tid < n_seqs) {
+            if (s_new_h[tid]) { const uint32_t kk = s_base_h[tid]; pre_h = kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]); }
+            if (s_new_l[tid]) { const uint32_t kk = s_base_l[tid]; pre_l = kk < s_ctrl[3] ? c.free_low[s_ctrl[3] - 1 - kk] : s_ctrl[2] + (kk - s_ctrl[3]); }
+        }
+        // ---- persist this CTA's token: one thread per 16-byte chunk of K and of V
+        if (writer && my_a != PASK_ACTION_RELEASE) persist_chunk(c, my_a, my_at, my_page, my_sl, cg >> 4, cg & 15, which, x);
+
+        // ---- protected recent window: every token, released ones too, also goes to slot (index mod W)
+        // of its (sequence, layer) ring as bf16; of a sequence's tokens in this call only the last W can
+        // still be in the window afterwards (and they have distinct slots)
+        if (c.window) {
+            const int W = (int)c.window, r = my_tok - s_cu[my_i], n_i = s_cu[my_i + 1] - s_cu[my_i];
+            if (r >= n_i - W) {
+                const uint32_t slot = (s_old_n[my_i] + (uint32_t)r) % (uint32_t)W;
+                const uint32_t ring_page = c.cap_high + (uint32_t)my_sl * (uint32_t)(W >> 4) + (slot >> 4);
+                if (writer) persist_chunk(c, PASK_ACTION_RETAIN_HIGH, slot, ring_page, my_sl, cg >> 4, cg & 15, which, x);
+                if (tid == 0) c.win_act[my_sl * (size_t)W + slot] = (uint8_t)my_a;
+            }
         }
     }
     __syncthreads();
@@ -920,11 +948,11 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         const uint32_t ph0 = (oh + kPageTokens - 1) / kPageTokens, pl0 = (ol + kPageTokens - 1) / kPageTokens;
         for (uint32_t x = 0; x < s_new_h[tid]; x++) {
             const uint32_t kk = s_base_h[tid] + x;
-            c.tbl_high[sl * c.max_pages + ph0 + x] = kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]);
+            c.tbl_high[sl * c.max_pages + ph0 + x] = x == 0 ? pre_h : kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]);
         }
         for (uint32_t x = 0; x < s_new_l[tid]; x++) {
             const uint32_t kk = s_base_l[tid] + x;
-            c.tbl_low[sl * c.max_pages + pl0 + x] = kk < s_ctrl[3] ? c.free_low[s_ctrl[3] - 1 - kk] : s_ctrl[2] + (kk - s_ctrl[3]);
+            c.tbl_low[sl * c.max_pages + pl0 + x] = x == 0 ? pre_l : kk < s_ctrl[3] ? c.free_low[s_ctrl[3] - 1 - kk] : s_ctrl[2] + (kk - s_ctrl[3]);
         }
         c.n_high[sl] = oh + ch;
         c.n_low[sl] = ol + cl;
@@ -951,23 +979,6 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             c.ctrl[kCtrlTicket] = 0;
         }
     }
-
-    // ---- persist this CTA's token: one thread per 16-byte chunk of K and of V
-    if (writer && my_a != PASK_ACTION_RELEASE) persist_chunk(c, my_a, my_at, my_page, my_sl, cg >> 4, cg & 15, which, x);
-
-    // ---- protected recent window: every token, released ones too, also goes to slot (index mod W)
-    // of its (sequence, layer) ring as bf16; of a sequence's tokens in this call only the last W can
-    // still be in the window afterwards (and they have distinct slots)
-    if (c.window) {
-        const int W = (int)c.window, r = my_tok - s_cu[my_i], n_i = s_cu[my_i + 1] - s_cu[my_i];
-        if (r >= n_i - W) {
-            const uint32_t slot = (s_old_n[my_i] + (uint32_t)r) % (uint32_t)W;
-            const uint32_t ring_page = c.cap_high + (uint32_t)my_sl * (uint32_t)(W >> 4) + (slot >> 4);
-            if (writer) persist_chunk(c, PASK_ACTION_RETAIN_HIGH, slot, ring_page, my_sl, cg >> 4, cg & 15, which, x);
-            if (tid == 0) c.win_act[my_sl * (size_t)W + slot] = (uint8_t)my_a;
-        }
-    }
-
 }
 
 // General path, recent window: CTA (j, y) copies the y-th newest of sequence j's tokens in this call
