@@ -419,8 +419,8 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     uint8_t *s_ring = smem + off;
     uint8_t *s_scratch = s_ring + (size_t)n_warps * kStages * kStageBytes;
 
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();   // only now: the combine kernel reads the plan's prefix before its own wait
     for (int s = tid; s <= n_seqs; s += blockDim.x) {
         s_cost[s] = __ldg(p.ws.cost_prefix + s);
         s_page[s] = __ldg(p.ws.page_prefix + s);
@@ -869,29 +869,33 @@ combine_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ p
                float *__restrict__ out, float *__restrict__ lse, int n_seqs, int n_q, uint32_t n_ctas) {
     const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
+    // The cost prefix is the plan's, written before the streaming kernel started (that kernel lets
+    // its dependents go only after its own wait for the plan's writer): it can be fetched while the
+    // streaming kernel's last CTAs are still running.
+    const int s = wid / n_q, h = wid % n_q;
+    uint32_t p0 = 0, p1 = 0;
+    uint64_t total = 0;
+    if (wid < n_seqs * n_q) { p0 = __ldg(prefix + s); p1 = __ldg(prefix + s + 1); total = __ldg(prefix + n_seqs); }
     pdl_wait();
     if (wid >= n_seqs * n_q) return;
-    const int s = wid / n_q, h = wid % n_q;
-    const uint32_t p0 = prefix[s], p1 = prefix[s + 1];
-    const uint64_t total = prefix[n_seqs];
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
     float M = -INFINITY, L = 0.f;
     if (p1 > p0) {
         const uint32_t b_first = (uint32_t)((((uint64_t)p0 + 1) * n_ctas - 1) / total);
         const uint32_t b_last = (uint32_t)(((uint64_t)p1 * n_ctas - 1) / total);
-        // online merge, four partials per round trip
-        for (uint32_t b = b_first; b <= b_last; b += 4) {
-            float2 ml[4];
-            float4 v[4];
+        // online merge, eight partials per round trip
+        for (uint32_t b = b_first; b <= b_last; b += 8) {
+            float2 ml[8];
+            float4 v[8];
 #pragma unroll
-            for (int u = 0; u < 4; u++) {
+            for (int u = 0; u < 8; u++) {
                 const bool have = b + u <= b_last;
                 const size_t row = ((size_t)b + u + s) * n_q + h;
                 ml[u] = have ? part_ml[row] : make_float2(-INFINITY, 0.f);
                 v[u] = have ? *reinterpret_cast<const float4 *>(part_o + row * kHeadDim + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
-            for (int u = 0; u < 4; u++) {
+            for (int u = 0; u < 8; u++) {
                 if (ml[u].x == -INFINITY) continue;      // a CTA whose share of this sequence was empty
                 const float Mn = fmaxf(M, ml[u].x);
                 const float fo = exp2f(M - Mn), fn = exp2f(ml[u].x - Mn);   // exp2f(-inf) = 0 on the first one
