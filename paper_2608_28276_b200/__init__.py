@@ -421,4 +421,7 @@ class Cache:
             self.policy = None
 
     def __del__(self):
-        self.close()
+        try:
+            self.close()
+        except Exception:       # interpreter shutdown: the module's globals may already be gone
+            pass
