@@ -338,7 +338,7 @@ __device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uin
         }
         if ((cch & 3) == 0) *reinterpret_cast<__half *>(dst8 + low8_scale_off((int)tau, cch >> 2)) = sh8;
         const uint32_t hb8 = __reduce_max_sync(0xffffffffu, which ? (uint32_t)__half_as_ushort(sh8) : 0u);
-        if ((threadIdx.x & 31) == 0 && hb8 > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb8);
+        if ((threadIdx.x & 31) == 0 && hb8) atomicMax(&c.low_vmax[sl], hb8);
         return;
     }
     if (c.low_bits == 2) {   // two-bit codes: the levels -s, 0, +s with s = fp16(amax), codes offset by 2
@@ -362,7 +362,7 @@ __device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uin
         }
         if ((cch & 3) == 0) *reinterpret_cast<__half *>(dst2 + low2_scale_off((int)tau, cch >> 2)) = sh2;
         const uint32_t hb2 = __reduce_max_sync(0xffffffffu, which ? (uint32_t)__half_as_ushort(sh2) : 0u);
-        if ((threadIdx.x & 31) == 0 && hb2 > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb2);
+        if ((threadIdx.x & 31) == 0 && hb2) atomicMax(&c.low_vmax[sl], hb2);
         return;
     }
     uint8_t *dst = c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLowHeadBytes + (which ? kLowHalfBytes : 0);
@@ -397,9 +397,9 @@ __device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uin
     }
     if (u == 0) *reinterpret_cast<__half *>(dst + low_scale_off((int)tau, w)) = sh;
     // decode attention forms P * (V scale) in fp16 relative to the stream's largest V scale:
-    // keep that maximum per (sequence, layer) -- one atomic per warp, and only when it grows
+    // keep that maximum per (sequence, layer) -- one atomic per warp, nothing comes back (no round trip)
     const uint32_t hb = __reduce_max_sync(0xffffffffu, which ? (uint32_t)__half_as_ushort(sh) : 0u);
-    if ((threadIdx.x & 31) == 0 && hb > c.low_vmax[sl]) atomicMax(&c.low_vmax[sl], hb);
+    if ((threadIdx.x & 31) == 0 && hb) atomicMax(&c.low_vmax[sl], hb);
 }
 
 // General path, second kernel: page-centric.  The plan kernel left, per sequence, its retained
@@ -637,6 +637,21 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
     }
 }
 
+// floor(x / n) for x < 2^48 and 0 < n < 2^24 from inv = 1.0 / n: the product is within 2^-4 / n of x / n, a quotient
+// that is not whole is at least 1 / n away from the next integer, so truncation is never too high and at most one
+// too low (a whole quotient): one correction step makes it exact.
+__device__ __forceinline__ uint32_t div_by(uint64_t x, uint32_t n, double inv) {
+    uint32_t q = (uint32_t)__double2ll_rz((double)x * inv);
+    if ((uint64_t)(q + 1) * n <= x) q++;
+    return q;
+}
+// page_at() of pask_layout.h with the two divisions by n = nh + nl replaced by div_by
+__device__ __forceinline__ bool page_at_rcp(uint32_t v, uint32_t nh, uint32_t n, double inv_n, uint32_t &idx) {
+    const uint32_t h0 = div_by((uint64_t)v * nh, n, inv_n), h1 = div_by((uint64_t)(v + 1) * nh, n, inv_n);
+    idx = h1 > h0 ? h0 : v - h0;
+    return h1 > h0;
+}
+
 // Small calls (decode: a token or a few per sequence): the whole of pask_append_kv in one launch
 // of one CTA per token, built so that the chain of dependent global round trips is as short as it
 // can be.  The table column and the layer's group arrive as kernel arguments; every CTA fetches
@@ -659,7 +674,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     __shared__ uint32_t s_old_h[kSmallMax], s_old_l[kSmallMax], s_cnt_h[kSmallMax], s_cnt_l[kSmallMax], s_cnt_bad[kSmallMax];
     __shared__ uint32_t s_new_h[kSmallMax], s_new_l[kSmallMax], s_base_h[kSmallMax], s_base_l[kSmallMax];
     __shared__ uint8_t s_act[kSmallMax], s_tok_seq[kSmallMax], s_tok_bad[kSmallMax];
-    __shared__ uint32_t s_pos[kSmallMax], s_ctrl[4], s_err;
+    __shared__ uint32_t s_pos[kSmallMax], s_ctrl[4], s_err, s_scan[kSmallThreads / 32];
     __shared__ int s_last;
     const int tid = threadIdx.x;
     pdl_launch_dependents();
@@ -688,10 +703,11 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         s_old_l[tid] = ol;
         s_old_n[tid] = on;
     }
-    int my_tag = 0, my_decided = 0;
+    int my_tag = 0, my_decided = 0, my_lut = 0;
     if (tid < total) {
         my_tag = tags[tid];
         if (decided) my_decided = decided[(size_t)tid * c.n_groups + group];
+        my_lut = lut.action[my_tag];   // (a first touch of the table misses the constant cache: take it while the loads above fly)
     }
     __syncthreads();
 
@@ -700,9 +716,31 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     if (tid < n_seqs) {
         const int seq = s_seq[tid];
         if (seq < 0 || seq >= c.max_seqs) err |= PASK_DEV_BAD_SEQ;
-        for (int j = 0; j < tid; j++) if (s_seq[j] == seq) err |= PASK_DEV_BAD_SEQ;       // named twice
         if (s_cu[tid] < 0 || s_cu[tid + 1] < s_cu[tid] || (tid == 0 && s_cu[0] != 0) ||
             (tid == n_seqs - 1 && s_cu[n_seqs] != total)) err |= PASK_DEV_BAD_RAGGED;
+        // the sequence each token belongs to (offsets are clamped here; a malformed table refuses the call below)
+        const int t_end = s_cu[tid + 1] < total ? s_cu[tid + 1] : total;
+        for (int t = s_cu[tid] > 0 ? s_cu[tid] : 0; t < t_end; t++) s_tok_seq[t] = (uint8_t)tid;
+    }
+    {   // a sequence named twice?  Every thread takes one sequence and a share of the distances to the others
+        // (with one or two warps per scheduler every dependent instruction costs its full latency, so the work
+        // is spread over all 256 threads, by powers of two, four loads at a time).
+        const int lg = 32 - __clz(n_seqs - 1);            // n_seqs <= 2^lg <= 256
+        const int i = tid & ((1 << lg) - 1), part = tid >> lg, per = kSmallThreads >> lg;
+        if (i < n_seqs) {
+            const int mine = s_seq[i];
+            for (int r0 = part; r0 < n_seqs - 1; r0 += 4 * per) {
+                int other[4];
+#pragma unroll
+                for (int u = 0; u < 4; u++) {
+                    int j = i + 1 + r0 + u * per;
+                    j = j >= n_seqs ? j - n_seqs : j;
+                    other[u] = s_seq[j < n_seqs ? j : i];      // (past the last distance: compares with itself, masked below)
+                }
+#pragma unroll
+                for (int u = 0; u < 4; u++) if (r0 + u * per < n_seqs - 1 && other[u] == mine) err |= PASK_DEV_BAD_SEQ;
+            }
+        }
     }
     if (err) atomicOr(&s_err, err);
     __syncthreads();
@@ -715,17 +753,11 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         return;
     }
     if (tid < total) {
-        int i = 0, i_hi = n_seqs - 1;                // the sequence this token belongs to: the first with s_cu[i + 1] > tid
-        while (i < i_hi) {
-            const int mid = (i + i_hi) >> 1;
-            if (s_cu[mid + 1] <= tid) i = mid + 1; else i_hi = mid;
-        }
-        int a = lut.action[my_tag];
+        int a = my_lut;
         if (decided) {   // Algorithm 2 step 7 on the actions pask_decide chose
             a = my_decided;
             if (a > PASK_ACTION_RETAIN_HIGH) { atomicOr(&s_err, PASK_DEV_BAD_ACTION); a = PASK_ACTION_RELEASE; }
         }
-        s_tok_seq[tid] = (uint8_t)i;
         s_act[tid] = (uint8_t)a;
         s_tok_bad[tid] = my_tag != PASK_TAG_PROTECTED && my_tag >= c.n_tags;
         if (actions_out && blockIdx.x == 0) actions_out[tid] = (uint8_t)a;
@@ -756,14 +788,15 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     __syncthreads();
 
     // ---- allocate for the whole call (sequence-major, like the general path) or refuse it
-    uint32_t need_h = 0, need_l = 0;
-    if (tid < n_seqs) {
-        uint32_t bh = 0, bl = 0;
-        for (int j = 0; j < n_seqs; j++) {
-            if (j == tid) { bh = need_h; bl = need_l; }
-            need_h += s_new_h[j]; need_l += s_new_l[j];
-        }
-        s_base_h[tid] = bh; s_base_l[tid] = bl;
+    // exclusive scan over the call's sequences, HIGH pages in the low half-word and LOW pages in the high one
+    // (a call of at most 255 tokens allocates fewer than 2^16 pages)
+    uint32_t need_h, need_l;
+    {
+        uint32_t tot = 0;
+        const uint32_t mine = tid < n_seqs ? (s_new_h[tid] | (s_new_l[tid] << 16)) : 0u;
+        const uint32_t before = block_excl_scan(mine, s_scan, &tot);
+        need_h = tot & 0xffffu; need_l = tot >> 16;
+        if (tid < n_seqs) { s_base_h[tid] = before & 0xffffu; s_base_l[tid] = before >> 16; }
         const bool fits = need_h <= s_ctrl[1] + (c.cap_high - s_ctrl[0]) && need_l <= s_ctrl[3] + (c.cap_low - s_ctrl[2]);
         if (tid == 0 && !fits && !s_err) atomicOr(&s_err, PASK_DEV_POOL_EXHAUSTED);
     }
@@ -860,45 +893,54 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             if (tid <= n_seqs) { ws.cost_prefix[tid] = s_cost[tid]; ws.page_prefix[tid] = s_page[tid]; }
             if (tid < n_seqs) ws.tokens[tid] = make_uint2(s_nh[tid], s_nl[tid]);
         }
-        const uint32_t total_pages = s_page[n_seqs];
-        for (uint32_t gp = blockIdx.x * kSmallThreads + tid; gp < total_pages; gp += gridDim.x * kSmallThreads) {
-            int a = 1, e = n_seqs;   // smallest idx in [1, n_seqs] with s_page[idx] > gp
-            while (a < e) {
-                const int mid = (a + e) >> 1;
-                if (s_page[mid] > gp) e = mid; else a = mid + 1;
-            }
-            const int s = a - 1;
+        // the page-order list, a sequence at a time (CTA b takes sequences b, b + grid, ...): up to four entries per
+        // thread and round, the page-table (or free-stack) reads of a round all in flight together
+        for (int s = blockIdx.x; s < n_seqs; s += gridDim.x) {
             const uint32_t nh = s_nh[s], nl = s_nl[s], nw = s_nw[s];
             const uint32_t ph = (nh + kPageTokens - 1) / kPageTokens, pl = (nl + kPageTokens - 1) / kPageTokens;
             const uint32_t pw = (nw + kPageTokens - 1) / kPageTokens;
+            const uint32_t old_h = (s_old_h[s] + kPageTokens - 1) / kPageTokens, old_l = (s_old_l[s] + kPageTokens - 1) / kPageTokens;
             const size_t slw = (size_t)s_seq[s] * c.n_layers + layer, sl = slw * c.max_pages;
-            uint32_t idx, entry;
-            if (page_at(gp - s_page[s], ph + pw, pl, idx)) {
-                const uint32_t old_pages = (s_old_h[s] + kPageTokens - 1) / kPageTokens;
-                if (idx >= ph) {     // a page of the recent-window ring
-                    entry = c.cap_high + (uint32_t)slw * (W / kPageTokens) + (idx - ph);
-                    if (idx - ph == pw - 1) entry |= (nw & (kPageTokens - 1)) << kOrderValidShift;
-                } else {
-                    if (idx < old_pages) {
-                        entry = c.tbl_high[sl + idx];
-                    } else {         // a page this call allocates: the commit's formula
-                        const uint32_t kk = s_base_h[s] + (idx - old_pages);
-                        entry = kk < s_ctrl[1] ? c.free_high[s_ctrl[1] - 1 - kk] : s_ctrl[0] + (kk - s_ctrl[1]);
+            const uint32_t first = s_page[s], n_pos = ph + pw + pl;
+            const double inv_n = 1.0 / (double)n_pos;   // page_at's two divisions by n_pos, see div_by below
+            for (uint32_t v0 = tid; v0 < n_pos; v0 += 4 * kSmallThreads) {
+                const uint32_t *src[4];    // where the page id is read from, or null when `val` already holds it
+                uint32_t val[4], flags[4];
+#pragma unroll
+                for (int u = 0; u < 4; u++) {
+                    const uint32_t v = v0 + u * kSmallThreads;
+                    src[u] = nullptr; val[u] = 0; flags[u] = 0;
+                    if (v >= n_pos) continue;
+                    uint32_t idx;
+                    if (page_at_rcp(v, ph + pw, n_pos, inv_n, idx)) {
+                        flags[u] = kOrderHigh;
+                        if (idx >= ph) {     // a page of the recent-window ring
+                            val[u] = c.cap_high + (uint32_t)slw * (W / kPageTokens) + (idx - ph);
+                            if (idx - ph == pw - 1) flags[u] |= (nw & (kPageTokens - 1)) << kOrderValidShift;
+                        } else {
+                            if (idx < old_h) {
+                                src[u] = c.tbl_high + sl + idx;
+                            } else {         // a page this call allocates: the commit's formula
+                                const uint32_t kk = s_base_h[s] + (idx - old_h);
+                                if (kk < s_ctrl[1]) src[u] = c.free_high + (s_ctrl[1] - 1 - kk); else val[u] = s_ctrl[0] + (kk - s_ctrl[1]);
+                            }
+                            if (idx == ph - 1) flags[u] |= (nh & (kPageTokens - 1)) << kOrderValidShift;
+                        }
+                    } else {
+                        if (idx < old_l) {
+                            src[u] = c.tbl_low + sl + idx;
+                        } else {
+                            const uint32_t kk = s_base_l[s] + (idx - old_l);
+                            if (kk < s_ctrl[3]) src[u] = c.free_low + (s_ctrl[3] - 1 - kk); else val[u] = s_ctrl[2] + (kk - s_ctrl[3]);
+                        }
+                        if (idx == pl - 1) flags[u] |= (nl & (kPageTokens - 1)) << kOrderValidShift;
                     }
-                    if (idx == ph - 1) entry |= (nh & (kPageTokens - 1)) << kOrderValidShift;
                 }
-                entry |= kOrderHigh;
-            } else {
-                const uint32_t old_pages = (s_old_l[s] + kPageTokens - 1) / kPageTokens;
-                if (idx < old_pages) {
-                    entry = c.tbl_low[sl + idx];
-                } else {
-                    const uint32_t kk = s_base_l[s] + (idx - old_pages);
-                    entry = kk < s_ctrl[3] ? c.free_low[s_ctrl[3] - 1 - kk] : s_ctrl[2] + (kk - s_ctrl[3]);
-                }
-                if (idx == pl - 1) entry |= (nl & (kPageTokens - 1)) << kOrderValidShift;
+#pragma unroll
+                for (int u = 0; u < 4; u++) if (src[u]) val[u] = *src[u];
+#pragma unroll
+                for (int u = 0; u < 4; u++) if (v0 + u * kSmallThreads < n_pos) ws.order[first + v0 + u * kSmallThreads] = val[u] | flags[u];
             }
-            ws.order[gp] = entry;
         }
     }
     uint32_t pre_h = 0, pre_l = 0;
