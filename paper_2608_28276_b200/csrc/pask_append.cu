@@ -56,6 +56,34 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *s_warp
     return before + inc - v;
 }
 
+// the same for three values per thread at once (one barrier; the per-warp slots are used once per kernel)
+__device__ __forceinline__ void block_excl_scan3(uint32_t (&v)[3], uint32_t (*s_warp)[3], uint32_t (&total)[3]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc[3] = {v[0], v[1], v[2]};
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+#pragma unroll
+        for (int k = 0; k < 3; k++) {
+            const uint32_t o = __shfl_up_sync(0xffffffffu, inc[k], d);
+            if (lane >= d) inc[k] += o;
+        }
+    }
+    if (lane == 31) { s_warp[warp][0] = inc[0]; s_warp[warp][1] = inc[1]; s_warp[warp][2] = inc[2]; }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 3; k++) {
+        uint32_t before = 0, tot = 0;
+#pragma unroll
+        for (int w = 0; w < kPlanThreads / 32; w++) {
+            const uint32_t x = s_warp[w][k];
+            if (w < warp) before += x;
+            tot += x;
+        }
+        total[k] = tot;
+        v[k] = before + inc[k] - v[k];
+    }
+}
+
 // One CTA per sequence of the call: decide every token, rank it inside its stream, record the
 // per-sequence plan; the CTA that arrives last allocates pages for the whole call (exclusive scan
 // over sequences in call order, so ids do not depend on scheduling) and commits all counters --
@@ -674,7 +702,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     __shared__ uint32_t s_old_h[kSmallMax], s_old_l[kSmallMax], s_cnt_h[kSmallMax], s_cnt_l[kSmallMax], s_cnt_bad[kSmallMax];
     __shared__ uint32_t s_new_h[kSmallMax], s_new_l[kSmallMax], s_base_h[kSmallMax], s_base_l[kSmallMax];
     __shared__ uint8_t s_act[kSmallMax], s_tok_seq[kSmallMax], s_tok_bad[kSmallMax];
-    __shared__ uint32_t s_pos[kSmallMax], s_ctrl[4], s_err, s_scan[kSmallThreads / 32];
+    __shared__ uint32_t s_pos[kSmallMax], s_ctrl[4], s_err, s_scan3[kSmallThreads / 32][3];
     __shared__ int s_last;
     const int tid = threadIdx.x;
     pdl_launch_dependents();
@@ -703,16 +731,22 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         s_old_l[tid] = ol;
         s_old_n[tid] = on;
     }
-    int my_tag = 0, my_decided = 0, my_lut = 0;
+    // decide every token (Algorithm 2 steps 1-2, or step 7 on the actions pask_decide chose): needs nothing but the tag
+    uint32_t err = 0;
+    int my_act = 0;
     if (tid < total) {
-        my_tag = tags[tid];
-        if (decided) my_decided = decided[(size_t)tid * c.n_groups + group];
-        my_lut = lut.action[my_tag];   // (a first touch of the table misses the constant cache: take it while the loads above fly)
+        const int my_tag = tags[tid];
+        my_act = lut.action[my_tag];
+        if (decided) {
+            my_act = decided[(size_t)tid * c.n_groups + group];
+            if (my_act > PASK_ACTION_RETAIN_HIGH) { err |= PASK_DEV_BAD_ACTION; my_act = PASK_ACTION_RELEASE; }
+        }
+        s_act[tid] = (uint8_t)my_act;
+        s_tok_bad[tid] = my_tag != PASK_TAG_PROTECTED && my_tag >= c.n_tags;
     }
     __syncthreads();
 
-    // ---- validate the call; decide every token
-    uint32_t err = 0;
+    // ---- validate the call
     if (tid < n_seqs) {
         const int seq = s_seq[tid];
         if (seq < 0 || seq >= c.max_seqs) err |= PASK_DEV_BAD_SEQ;
@@ -752,17 +786,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         if (fuse_plan && blockIdx.x == 0 && tid <= n_seqs) ws.cost_prefix[tid] = ws.page_prefix[tid] = 0;   // nothing to attend
         return;
     }
-    if (tid < total) {
-        int a = my_lut;
-        if (decided) {   // Algorithm 2 step 7 on the actions pask_decide chose
-            a = my_decided;
-            if (a > PASK_ACTION_RETAIN_HIGH) { atomicOr(&s_err, PASK_DEV_BAD_ACTION); a = PASK_ACTION_RELEASE; }
-        }
-        s_act[tid] = (uint8_t)a;
-        s_tok_bad[tid] = my_tag != PASK_TAG_PROTECTED && my_tag >= c.n_tags;
-        if (actions_out && blockIdx.x == 0) actions_out[tid] = (uint8_t)a;
-    }
-    __syncthreads();
+    if (actions_out && blockIdx.x == 0 && tid < total) actions_out[tid] = (uint8_t)my_act;
 
     // ---- per token: rank inside its stream; per sequence: counts and new pages
     if (tid < total) {
@@ -787,43 +811,11 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     }
     __syncthreads();
 
-    // ---- allocate for the whole call (sequence-major, like the general path) or refuse it
-    // exclusive scan over the call's sequences, HIGH pages in the low half-word and LOW pages in the high one
-    // (a call of at most 255 tokens allocates fewer than 2^16 pages)
-    uint32_t need_h, need_l;
-    {
-        uint32_t tot = 0;
-        const uint32_t mine = tid < n_seqs ? (s_new_h[tid] | (s_new_l[tid] << 16)) : 0u;
-        const uint32_t before = block_excl_scan(mine, s_scan, &tot);
-        need_h = tot & 0xffffu; need_l = tot >> 16;
-        if (tid < n_seqs) { s_base_h[tid] = before & 0xffffu; s_base_l[tid] = before >> 16; }
-        const bool fits = need_h <= s_ctrl[1] + (c.cap_high - s_ctrl[0]) && need_l <= s_ctrl[3] + (c.cap_low - s_ctrl[2]);
-        if (tid == 0 && !fits && !s_err) atomicOr(&s_err, PASK_DEV_POOL_EXHAUSTED);
-    }
-    __syncthreads();
-    // old page of this CTA's token, if it continues one (page tables are only appended to by the commit)
-    uint32_t my_page = 0, my_at = 0;
-    const uint32_t my_a = s_act[my_tok];
-    const int my_i = s_tok_seq[my_tok];
-    const size_t my_sl = (size_t)s_seq[my_i] * c.n_layers + layer;
-    if (my_a != PASK_ACTION_RELEASE) {
-        const bool high = my_a == PASK_ACTION_RETAIN_HIGH;
-        const uint32_t old = high ? s_old_h[my_i] : s_old_l[my_i];
-        my_at = old + s_pos[my_tok];
-        const uint32_t old_pages = (old + kPageTokens - 1) / kPageTokens, pg = my_at >> 4;
-        if (pg < old_pages) {
-            my_page = (high ? c.tbl_high : c.tbl_low)[my_sl * c.max_pages + pg];
-        } else {   // one of the pages this call allocates: same formula as the commit below
-            const uint32_t kk = (high ? s_base_h[my_i] : s_base_l[my_i]) + (pg - old_pages);
-            const uint32_t fr = high ? s_ctrl[1] : s_ctrl[3], nx = high ? s_ctrl[0] : s_ctrl[2];
-            my_page = kk < fr ? (high ? c.free_high : c.free_low)[fr - 1 - kk] : nx + (kk - fr);
-        }
-    }
-    // ---- fused decode-attention plan for the same sequences (what attn_plan_kernel would compute after
-    // this append): every CTA knows every sequence's lengths after the call and the ids of the pages the
-    // call allocates, so the plan needs nothing that the commit writes.
-    if (fuse_plan && !s_err) {
-        const uint32_t W = c.window;
+    // ---- what the fused decode-attention plan needs per sequence (what attn_plan_kernel would compute after this
+    // append): tokens attended from the two streams and from the recent-window ring after the call
+    const uint32_t W = c.window;
+    uint32_t my_cost = 0, my_pages = 0;
+    if (fuse_plan) {
         if (tid < n_seqs) {
             uint32_t nh = s_old_h[tid] + s_cnt_h[tid], nl = s_old_l[tid] + s_cnt_l[tid], nw = 0;
             if (W) {
@@ -840,9 +832,8 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             }
             s_nh[tid] = nh; s_nl[tid] = nl; s_nw[tid] = nw;
         }
-        if (tid == 0) s_cost[0] = s_page[0] = 0;
-        __syncthreads();
         if (W) {
+            __syncthreads();
             // ... and here those among the older tokens still in the window: token indices [n_new - W, old_n), whose
             // slots (index mod W) this call does not write.  One thread per 16 slots of a ring.
             const int per = (int)W / kPageTokens;
@@ -868,27 +859,52 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             }
             __syncthreads();
         }
-        if (tid < 32) {
-            uint32_t carry_c = 0, carry_p = 0;
-            for (int base = 0; base < n_seqs; base += 32) {
-                const int idx = base + tid;
-                uint32_t ph = 0, pl = 0;
-                if (idx < n_seqs) {   // the ring's pages have the HIGH format and count as HIGH pages
-                    ph = (s_nh[idx] + kPageTokens - 1) / kPageTokens + (s_nw[idx] + kPageTokens - 1) / kPageTokens;
-                    pl = (s_nl[idx] + kPageTokens - 1) / kPageTokens;
-                }
-                uint32_t ic = ph * kCostHighPage + pl * c.cost_low_page, ip = ph + pl;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const uint32_t oc = __shfl_up_sync(0xffffffffu, ic, d), op = __shfl_up_sync(0xffffffffu, ip, d);
-                    if (tid >= d) { ic += oc; ip += op; }
-                }
-                if (idx < n_seqs) { s_cost[idx + 1] = carry_c + ic; s_page[idx + 1] = carry_p + ip; }
-                carry_c += __shfl_sync(0xffffffffu, ic, 31);
-                carry_p += __shfl_sync(0xffffffffu, ip, 31);
-            }
+        if (tid < n_seqs) {   // the ring's pages have the HIGH format and count as HIGH pages
+            const uint32_t ph = (s_nh[tid] + kPageTokens - 1) / kPageTokens + (s_nw[tid] + kPageTokens - 1) / kPageTokens;
+            const uint32_t pl = (s_nl[tid] + kPageTokens - 1) / kPageTokens;
+            my_cost = ph * kCostHighPage + pl * c.cost_low_page;
+            my_pages = ph + pl;
         }
-        __syncthreads();
+    }
+
+    // ---- one exclusive scan over the call's sequences for three things: the pages the call allocates
+    // (sequence-major like the general path; HIGH pages in the low half-word, LOW pages in the high one: a call
+    // of at most 255 tokens allocates fewer than 2^16), and the plan's cost and page prefixes
+    uint32_t need_h, need_l;
+    {
+        uint32_t v3[3] = {tid < n_seqs ? (s_new_h[tid] | (s_new_l[tid] << 16)) : 0u, my_cost, my_pages}, tot3[3];
+        block_excl_scan3(v3, s_scan3, tot3);
+        need_h = tot3[0] & 0xffffu; need_l = tot3[0] >> 16;
+        if (tid < n_seqs) {
+            s_base_h[tid] = v3[0] & 0xffffu; s_base_l[tid] = v3[0] >> 16;
+            s_cost[tid + 1] = v3[1] + my_cost; s_page[tid + 1] = v3[2] + my_pages;
+        }
+        if (tid == 0) s_cost[0] = s_page[0] = 0;
+        const bool fits = need_h <= s_ctrl[1] + (c.cap_high - s_ctrl[0]) && need_l <= s_ctrl[3] + (c.cap_low - s_ctrl[2]);
+        if (tid == 0 && !fits && !s_err) atomicOr(&s_err, PASK_DEV_POOL_EXHAUSTED);
+    }
+    __syncthreads();
+    // old page of this CTA's token, if it continues one (page tables are only appended to by the commit)
+    uint32_t my_page = 0, my_at = 0;
+    const uint32_t my_a = s_act[my_tok];
+    const int my_i = s_tok_seq[my_tok];
+    const size_t my_sl = (size_t)s_seq[my_i] * c.n_layers + layer;
+    if (my_a != PASK_ACTION_RELEASE) {
+        const bool high = my_a == PASK_ACTION_RETAIN_HIGH;
+        const uint32_t old = high ? s_old_h[my_i] : s_old_l[my_i];
+        my_at = old + s_pos[my_tok];
+        const uint32_t old_pages = (old + kPageTokens - 1) / kPageTokens, pg = my_at >> 4;
+        if (pg < old_pages) {
+            my_page = (high ? c.tbl_high : c.tbl_low)[my_sl * c.max_pages + pg];
+        } else {   // one of the pages this call allocates: same formula as the commit below
+            const uint32_t kk = (high ? s_base_h[my_i] : s_base_l[my_i]) + (pg - old_pages);
+            const uint32_t fr = high ? s_ctrl[1] : s_ctrl[3], nx = high ? s_ctrl[0] : s_ctrl[2];
+            my_page = kk < fr ? (high ? c.free_high : c.free_low)[fr - 1 - kk] : nx + (kk - fr);
+        }
+    }
+    // ---- the fused plan itself: every CTA knows every sequence's lengths after the call and the ids of the pages
+    // the call allocates, so the plan needs nothing that the commit writes
+    if (fuse_plan && !s_err) {
         if (blockIdx.x == 0) {
             if (tid <= n_seqs) { ws.cost_prefix[tid] = s_cost[tid]; ws.page_prefix[tid] = s_page[tid]; }
             if (tid < n_seqs) ws.tokens[tid] = make_uint2(s_nh[tid], s_nl[tid]);
@@ -902,7 +918,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
             const uint32_t old_h = (s_old_h[s] + kPageTokens - 1) / kPageTokens, old_l = (s_old_l[s] + kPageTokens - 1) / kPageTokens;
             const size_t slw = (size_t)s_seq[s] * c.n_layers + layer, sl = slw * c.max_pages;
             const uint32_t first = s_page[s], n_pos = ph + pw + pl;
-            const double inv_n = 1.0 / (double)n_pos;   // page_at's two divisions by n_pos, see div_by below
+            const double inv_n = 1.0 / (double)n_pos;   // for page_at_rcp: its two divisions by n_pos
             for (uint32_t v0 = tid; v0 < n_pos; v0 += 4 * kSmallThreads) {
                 const uint32_t *src[4];    // where the page id is read from, or null when `val` already holds it
                 uint32_t val[4], flags[4];
