@@ -432,27 +432,28 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     const uint32_t n_ctas = gridDim.x, b = blockIdx.x;
     const uint32_t lo = (uint32_t)(((uint64_t)total * b) / n_ctas);
     const uint32_t hi = (uint32_t)(((uint64_t)total * (b + 1)) / n_ctas);
-    // first sequence of the span: cost[s0] <= lo < cost[s0 + 1]
-    int s0;
-    {
-        int a = 1, e = n_seqs;  // smallest idx in [1, n_seqs] with cost[idx] > lo
-        while (a < e) {
-            const int mid = (a + e) >> 1;
-            if (s_cost[mid] > lo) e = mid; else a = mid + 1;
-        }
-        s0 = a - 1;
-    }
+    // The sequence holding cost offset x (< total): cost[s] <= x < cost[s + 1].  A warp looks at 32 table entries at
+    // a time -- every 32nd first, then the 32 of the block found -- so the search is two shared-memory reads deep
+    // whatever the batch (dependent steps cost their full latency here: the CTA has nothing else to issue yet).
+    auto seq_of = [&](uint32_t x) -> int {
+        const int i1 = (lane + 1) * 32 < n_seqs ? (lane + 1) * 32 : n_seqs;
+        const int blk = __ffs(__ballot_sync(0xffffffffu, s_cost[i1] > x)) - 1;       // cost[n_seqs] = total > x: never empty
+        const int i2 = 32 * blk + 1 + lane < n_seqs ? 32 * blk + 1 + lane : n_seqs;
+        return 32 * blk + __ffs(__ballot_sync(0xffffffffu, s_cost[i2] > x)) - 1;
+    };
+    // cut_positions() of pask_layout.h, exactly, with the 64-bit division replaced by a double one and a correction step
+    auto cut_at = [&](uint32_t x, uint32_t cs, uint32_t n) -> uint32_t {
+        if (x >= cs) return n;
+        const uint64_t prod = (uint64_t)x * n;                        // < 2^53: exact as a double
+        uint64_t q = (uint64_t)__double2ll_rz((double)prod / (double)cs);
+        if ((q + 1) * cs <= prod) q++; else if (q * cs > prod) q--;
+        return (uint32_t)q;
+    };
+    const int s0 = seq_of(lo);   // first sequence of the span
 
     // the CTA's range of the page-order list, and this warp's pipeline over it
-    auto position_of = [&](uint32_t x) -> uint32_t {   // first position at or after cost offset x
-        if (x >= total) return s_page[n_seqs];
-        int a = 1, e = n_seqs;                          // smallest idx in [1, n_seqs] with cost[idx] > x
-        while (a < e) {
-            const int mid = (a + e) >> 1;
-            if (s_cost[mid] > x) e = mid; else a = mid + 1;
-        }
-        const int s = a - 1;
-        return s_page[s] + cut_positions(x - s_cost[s], s_cost[s + 1] - s_cost[s], s_page[s + 1] - s_page[s]);
+    auto position_of = [&](uint32_t x, int s) -> uint32_t {   // first position at or after cost offset x, which lies in sequence s
+        return s_page[s] + cut_at(x - s_cost[s], s_cost[s + 1] - s_cost[s], s_page[s + 1] - s_page[s]);
     };
     Pipe w;
     w.order = p.ws.order;
@@ -468,8 +469,8 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     w.ring = smem_u32(s_ring + (size_t)warp * kStages * kStageBytes);
     w.bars = smem_u32(s_bar + warp * kStages);
     w.meta = smem_u32(s_bar) + kMaxWarps * kStages * 8 + warp * kStages * 4;   // after the 192 bytes of barriers
-    w.p_pos = position_of(lo);
-    w.p_end = position_of(hi);
+    w.p_pos = position_of(lo, s0);
+    w.p_end = hi >= total ? s_page[n_seqs] : position_of(hi, seq_of(hi));
     w.p_sub = 0; w.pw_base = 0x80000000u; w.pw_entry = 0;
     w.p_stage = 0; w.c_stage = 0; w.c_parity = 0; w.outstanding = 0; w.dead = false;
     const uint32_t scratch = smem_u32(s_scratch + (size_t)warp * kScratchBytes);
@@ -492,8 +493,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         if (s_cost[s + 1] == s_cost[s]) continue;
         const uint32_t c0 = s_cost[s], c1 = s_cost[s + 1], n_pos = s_page[s + 1] - s_page[s];
         // number of this sequence's pages that fall to this CTA (same cuts as position_of)
-        const uint32_t n_pages = cut_positions((hi < c1 ? hi : c1) - c0, c1 - c0, n_pos) -
-                                 cut_positions((lo > c0 ? lo : c0) - c0, c1 - c0, n_pos);
+        const uint32_t n_pages = cut_at((hi < c1 ? hi : c1) - c0, c1 - c0, n_pos) - cut_at((lo > c0 ? lo : c0) - c0, c1 - c0, n_pos);
         const uint2 tk = __ldg(p.ws.tokens + s);
         const uint32_t seq_n_low = tk.y;
 
