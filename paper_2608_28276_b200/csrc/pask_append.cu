@@ -698,7 +698,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
                     uint8_t *__restrict__ actions_out, const SmallLut lut, const int fuse_plan, const Workspace ws) {
     __shared__ int s_seq[kSmallMax], s_cu[kSmallMax + 1];
     __shared__ uint32_t s_cost[kSmallMax + 1], s_page[kSmallMax + 1], s_nh[kSmallMax], s_nl[kSmallMax];   // fused attention plan
-    __shared__ uint32_t s_old_n[kSmallMax], s_nw[kSmallMax];
+    __shared__ uint32_t s_old_n[kSmallMax], s_nw[kSmallMax], s_wstart[kSmallMax], s_wlen[kSmallMax];
     __shared__ uint32_t s_old_h[kSmallMax], s_old_l[kSmallMax], s_cnt_h[kSmallMax], s_cnt_l[kSmallMax], s_cnt_bad[kSmallMax];
     __shared__ uint32_t s_new_h[kSmallMax], s_new_l[kSmallMax], s_base_h[kSmallMax], s_base_l[kSmallMax];
     __shared__ uint8_t s_act[kSmallMax], s_tok_seq[kSmallMax], s_tok_bad[kSmallMax];
@@ -831,28 +831,41 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
                 }
             }
             s_nh[tid] = nh; s_nl[tid] = nl; s_nw[tid] = nw;
+            if (W) {   // ... and where the older members sit in the ring: slots [start, start + len) mod W (token index mod W)
+                const uint32_t old_n = s_old_n[tid], n_new = old_n + (uint32_t)(s_cu[tid + 1] - s_cu[tid]);
+                const uint32_t lo = n_new > W ? n_new - W : 0u;
+                s_wlen[tid] = lo < old_n ? old_n - lo : 0u;
+                s_wstart[tid] = lo % W;
+            }
         }
         if (W) {
             __syncthreads();
             // ... and here those among the older tokens still in the window: token indices [n_new - W, old_n), whose
-            // slots (index mod W) this call does not write.  One thread per 16 slots of a ring.
+            // slots this call does not write.  One thread per 16 slots of a ring; actions are 0, 1, 2, so bit 0 of a byte
+            // says LOW and bit 1 HIGH: four bytes are counted with two population counts under a byte mask.
             const int per = (int)W / kPageTokens;
+            const uint32_t inv_per = (65536u + per - 1) / per;                    // idx / per for idx < 4096, per <= 16
             for (int idx = tid; idx < n_seqs * per; idx += kSmallThreads) {
-                const int sq = idx / per, i = idx - sq * per;
-                const uint32_t old_n = s_old_n[sq], n_new = old_n + (uint32_t)(s_cu[sq + 1] - s_cu[sq]);
-                const uint32_t lo = n_new > W ? n_new - W : 0u;
-                if (lo >= old_n) continue;
-                const uint32_t len = old_n - lo, start = lo % W;
+                const int sq = (int)(((uint32_t)idx * inv_per) >> 16), i = idx - sq * per;
+                const uint32_t len = s_wlen[sq];
+                if (len == 0) continue;
+                // the members' slots inside this piece [p0, p0 + 16), as a 16-bit mask: [a, b) and, wrapped, [0, b - W)
+                const uint32_t a = s_wstart[sq], b = a + len, p0 = 16u * (uint32_t)i;
+                auto piece_bits = [&](uint32_t from, uint32_t to) -> uint32_t {   // slots [from, to) clipped to the piece
+                    const uint32_t f = from > p0 ? from - p0 : 0u, t = to > p0 ? (to - p0 < 16u ? to - p0 : 16u) : 0u;
+                    return f < t ? ((1u << t) - 1u) & ~((1u << f) - 1u) : 0u;
+                };
+                const uint32_t m16 = piece_bits(a, b < W ? b : W) | (b > W ? piece_bits(0u, b - W) : 0u);
+                if (m16 == 0) continue;
                 const size_t slw = (size_t)s_seq[sq] * c.n_layers + layer;
                 const uint4 a4 = reinterpret_cast<const uint4 *>(c.win_act + slw * W)[i];
                 const uint32_t w4[4] = {a4.x, a4.y, a4.z, a4.w};
                 uint32_t wh = 0, wl = 0;
 #pragma unroll
-                for (int b = 0; b < 16; b++) {
-                    const uint32_t a = (w4[b >> 2] >> (8 * (b & 3))) & 0xffu;
-                    const uint32_t j = 16u * (uint32_t)i + (uint32_t)b;
-                    const uint32_t d = j >= start ? j - start : j + W - start;   // distance from the oldest member's slot
-                    if (d < len) { wh += a == PASK_ACTION_RETAIN_HIGH; wl += a == PASK_ACTION_RETAIN_LOW; }
+                for (int k = 0; k < 4; k++) {
+                    const uint32_t sel = (((m16 >> (4 * k)) & 15u) * 0x00204081u) & 0x01010101u;   // bit j -> bit 0 of byte j
+                    wl += __popc(w4[k] & sel);
+                    wh += __popc(w4[k] & (sel << 1));
                 }
                 if (wh) atomicSub(&s_nh[sq], wh);
                 if (wl) atomicSub(&s_nl[sq], wl);

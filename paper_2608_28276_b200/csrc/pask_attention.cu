@@ -265,11 +265,14 @@ attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ 
             const size_t sl = (size_t)seq_ids[s] * c.n_layers + layer;
             const uint4 a4 = reinterpret_cast<const uint4 *>(c.win_act + sl * c.window)[i];
             const uint32_t w4[4] = {a4.x, a4.y, a4.z, a4.w};
+            // actions are 0, 1, 2: bit 0 of a byte says LOW, bit 1 HIGH; the piece's first `in` slots are members
+            const uint32_t in = nw - (uint32_t)i * 16u < 16u ? nw - (uint32_t)i * 16u : 16u, m16 = (1u << in) - 1u;
             uint32_t wh = 0, wl = 0;
 #pragma unroll
-            for (int b = 0; b < 16; b++) {
-                const uint32_t a = (w4[b >> 2] >> (8 * (b & 3))) & 0xffu;
-                if ((uint32_t)i * 16u + b < nw) { wh += a == PASK_ACTION_RETAIN_HIGH; wl += a == PASK_ACTION_RETAIN_LOW; }
+            for (int k = 0; k < 4; k++) {
+                const uint32_t sel = (((m16 >> (4 * k)) & 15u) * 0x00204081u) & 0x01010101u;   // bit j -> bit 0 of byte j
+                wl += __popc(w4[k] & sel);
+                wh += __popc(w4[k] & (sel << 1));
             }
             if (wh) atomicSub(&s_nh[s], wh);
             if (wl && has_low) atomicSub(&s_nl[s], wl);
