@@ -628,27 +628,42 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
                 // to the nearest integer, ties to even, leaving code in the low 4 bits of the sum.
                 // s == 0 means every value is zero: 1/s is replaced by 0 and all codes come out 8.
                 const float inv = sc == 0.0f ? 0.0f : __fdiv_rn(1.0f, sc);
-                uint32_t code[16];
+                // The sums are kept as bit patterns, 0x4B400000 + code, and packed by multiply-adds (a nibble per step,
+                // from the top one down) instead of mask, shift and or per code: the constant upper bits add up to a
+                // known word that is taken off at the end (K words, modulo 2^32) or fall outside the result (V half-words).
+                uint32_t raw[16];
+                // A normal, unsaturated fp16 scale is within 2^-11 of amax / 7, so |x / s| < 7.01 and the clamp cannot
+                // bite: it is only kept for subnormal scales (rounded coarsely) and the saturated one.
+                const uint32_t sbits = __half_as_ushort(sh);
+                if (sbits >= 0x0400u && sbits < 0x7BFFu) {
 #pragma unroll
-                for (int e = 0; e < 16; e++) {
-                    const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
-                    const float cl = fminf(fmaxf(__fmul_rn(f, inv), -7.0f), 7.0f);
-                    code[e] = __float_as_uint(__fadd_rn(cl, 12582920.0f)) & 15u;
+                    for (int e = 0; e < 16; e++) {
+                        const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
+                        raw[e] = __float_as_uint(__fadd_rn(__fmul_rn(f, inv), 12582920.0f));
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; e++) {
+                        const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
+                        const float cl = fminf(fmaxf(__fmul_rn(f, inv), -7.0f), 7.0f);
+                        raw[e] = __float_as_uint(__fadd_rn(cl, 12582920.0f));
+                    }
                 }
                 uint8_t *img = s_low[head & 1] + (which ? kLowHalfBytes : 0);
                 if (!which) {
+                    constexpr uint32_t kRawWord = 0x4B400000u * 0x11111111u;   // what eight constant parts add up to
 #pragma unroll
                     for (int u = 0; u < 2; u++) {  // the words of dims 32w + 8t .. +7, t = 2 half + u
-                        uint32_t word = 0;
+                        uint32_t acc = raw[8 * u + 7];          // nibble n holds dim offset 2 (n & 3) + (n >> 2): low_k_nibble inverted
 #pragma unroll
-                        for (int e = 0; e < 8; e++) word |= code[8 * u + e] << (4 * low_k_nibble(e));
-                        *reinterpret_cast<uint32_t *>(img + low_k_word_off(tau, w, 2 * half + u)) = word;
+                        for (int n = 6; n >= 0; n--) acc = acc * 16u + raw[8 * u + 2 * (n & 3) + (n >> 2)];
+                        *reinterpret_cast<uint32_t *>(img + low_k_word_off(tau, w, 2 * half + u)) = acc - kRawWord;
                     }
                 } else {
 #pragma unroll
                     for (int u = 0; u < 4; u++) {  // the half-words of dims 32w + 4g .. +3, g = 4 half + u
-                        const uint16_t hw = (uint16_t)(code[4 * u] | (code[4 * u + 1] << 4) | (code[4 * u + 2] << 8) | (code[4 * u + 3] << 12));
-                        *reinterpret_cast<uint16_t *>(img + low_v_half_off(tau, w, 4 * half + u)) = hw;
+                        const uint32_t acc = ((raw[4 * u + 3] * 16u + raw[4 * u + 2]) * 16u + raw[4 * u + 1]) * 16u + raw[4 * u];
+                        *reinterpret_cast<uint16_t *>(img + low_v_half_off(tau, w, 4 * half + u)) = (uint16_t)acc;
                     }
                     vmax_bits = max(vmax_bits, (uint32_t)__half_as_ushort(sh));
                 }

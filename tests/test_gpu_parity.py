@@ -194,6 +194,32 @@ def test_low_only_and_extreme_magnitudes(pask, oracle):
         assert_close(go[i:i + 1] / sv, gl[i:i + 1], oo[i:i + 1] / sv, ol[i:i + 1], where=("scaled", i))
 
 
+def test_subnormal_and_saturated_scales_through_both_append_paths(pask, oracle):
+    # groups whose fp16 scale is subnormal (coarsely rounded: the clamp of the codes bites) or saturates at 65504,
+    # next to ordinary ones, through the bulk path (full pages) and the one-launch path; stored bytes bit for bit
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=2, n_layers=1, n_groups=1)
+    w = _workload(cfg, actions=[[1]])
+    p = Pair(pask, oracle, w, pool_high_pages=8, pool_low_pages=128, max_tokens_per_seq=1024, max_append_tokens=4096)
+    n = 200
+    for seq, scales in ((0, (3e-6, 1e-7, 1.0)), (1, (4e5, 3e6, 1.0))):
+        k = normal_bf16(19, 1, 0, seq, 0, n, 8).float()
+        v = normal_bf16(19, 2, 0, seq, 0, n, 8).float()
+        for i, sc in enumerate(scales):                # every third token at each magnitude, heads alternate too
+            k[i::3] *= sc
+            v[i::3, ::2] *= sc
+        k, v = k.to(torch.bfloat16), v.to(torch.bfloat16)
+        tags = np.zeros(n, np.uint8)
+        p.append(0, [seq], [n - 7], None, k=k[:n - 7], v=v[:n - 7], tags=tags[:n - 7])
+        for t in range(n - 7, n):
+            p.append(0, [seq], [1], None, k=k[t:t + 1], v=v[t:t + 1], tags=tags[t:t + 1])
+    p.compare_state()
+    kc, ks, _, _, _ = pask.pask_debug_dump_low(p.gpu.handle, 0, 0, 8)
+    sub = (ks > 0) & (ks < 0x0400)
+    assert sub.any() and (ks == 0).any()                # subnormal scales and scales that underflowed to zero
+    _, ks1, _, _, _ = pask.pask_debug_dump_low(p.gpu.handle, 0, 1, 8)
+    assert (ks1 == 0x7BFF).any()                        # saturated scales
+
+
 def test_device_side_refusals_leave_the_cache_untouched(pask, oracle):
     cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=3, n_layers=1, n_groups=1)
     w = _workload(cfg, actions=[[1], [2]])
