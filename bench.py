@@ -595,6 +595,8 @@ def run_reference(args, rank, world):
     cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, args.warmup + args.steps + 8))
     w = WC.build(cfg)
     smp = OracleSample(w, args.ref_seqs, [0])
+    if world > 1:      # the launcher pins every rank to one OpenMP thread; rank 0 runs alone and takes the host's cores
+        smp.oracle.set_threads(os.cpu_count() or 1)
     for i in range(args.warmup):
         smp.step(i)
     t = sum(smp.step(args.warmup + i) for i in range(args.steps))

@@ -238,3 +238,8 @@ def distortion(o_ref: np.ndarray, o_test: np.ndarray):
 
 def max_threads() -> int:
     return int(lib().orc_max_threads())
+
+
+def set_threads(n: int) -> None:
+    """Threads of the oracle's parallel loops (torchrun pins OMP_NUM_THREADS to 1 per rank)."""
+    lib().orc_set_threads(int(n))

@@ -719,4 +719,14 @@ int orc_max_threads(void) {
 #endif
 }
 
+/* Threads of the parallel loops (a launcher may have pinned OMP_NUM_THREADS to 1 for every rank). */
+void orc_set_threads(int n) {
+#ifdef _OPENMP
+    extern void omp_set_num_threads(int);
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 int orc_sizeof_budget(void) { return (int)sizeof(orc_budget); }
