@@ -492,7 +492,7 @@ def run_cuda(args, rank, world):
         line["config"]["table"] += " + budget-dependent adjustment (pask_decide)"
     if args.full_kv and world == 1:
         line["full_kv"] = run_full_kv(P, args, w, device, total_steps, peak)
-    if args.cpu_seconds > 0:
+    if args.cpu_seconds > 0 and world == 1:          # the oracle beside it: rank 0 at N = 1 only
         line["cpu_baseline"] = cpu_baseline(w, budget_s=args.cpu_seconds, n_seqs=args.ref_seqs)
     print(json.dumps(line))
 
