@@ -67,7 +67,8 @@ typedef int32_t pask_status_t;
 #define PASK_DEV_BAD_SEQ 0x2u         /* sequence id out of range or repeated within one call */
 #define PASK_DEV_SEQ_OVERFLOW 0x4u    /* a stream would exceed max_tokens_per_seq: nothing written */
 #define PASK_DEV_BAD_RAGGED 0x8u      /* cu_tokens not ascending or not ending at total_tokens */
-#define PASK_DEV_TIMEOUT 0x10u        /* a bounded wait inside a kernel ran out; results invalid */
+#define PASK_DEV_TIMEOUT 0x10u        /* a bounded wait inside a kernel ran out: the call's out / lse are void
+                                         (contributions of the pages behind the wait are missing) */
 #define PASK_DEV_RANGE 0x20u          /* a query element had |q| > 65504, outside what the low-precision path
                                          computes in; results for that sequence may be infinite or NaN */
 
@@ -193,7 +194,10 @@ pask_status_t pask_seq_reset(pask_cache_t *cache, int32_t seq, pask_stream_t str
  *   seq_ids        dev int32 [n_seqs]
  *   cu_tokens      dev int32 [n_seqs+1], ascending, cu_tokens[0] = 0, last = total_tokens
  *                  (one token per sequence in decode, many in prefill)
- *   k, v           dev bf16 [total_tokens][n_kv][128], post-RoPE, tokens of a sequence in order
+ *   k, v           dev bf16 [total_tokens][n_kv][128], post-RoPE, tokens of a sequence in order.
+ *                  Values must be finite.  An infinity saturates its group's scale; what a NaN
+ *                  leaves in the low-precision codes of its 32-dim group is undefined and may
+ *                  differ between a small and a large call (the high-precision copy keeps its bits)
  *   tags           dev uint8 [total_tokens]; PASK_TAG_PROTECTED = always high; >= n_tags = high
  *                  and counted in bad_tags
  *   states         dev uint16 [total_tokens] or NULL; not read: this call applies the frozen table
@@ -341,7 +345,13 @@ pask_status_t pask_decode_step_packed(pask_cache_t *cache, int32_t layer, int32_
  * stream and overlaps the call after.  The two streams and six events are created for the cache at
  * the first call (host-side handles; no device memory) and destroyed with it; kernels still run
  * on `stream`, in call order.
- *   staging        dev, >= 2 * pask_step_staging_bytes(cache, n_seqs): two slots used in turn
+ *   staging        dev, 256-byte aligned: its two halves (the second starts at staging_bytes / 2
+ *                  rounded down to 256) are used in turn, whatever n_seqs is, and each must hold
+ *                  pask_step_staging_bytes(cache, n_seqs), else PASK_ERR_WORKSPACE.  n_seqs may
+ *                  change from call to call.  Pass the same buffer and size until the next drain;
+ *                  a call that brings another one first waits for the earlier calls' use of theirs.
+ *                  A call that fails after it was given its slot still uses the slot up: the
+ *                  next call takes the other half.
  *   packed_host    must stay valid, and out_host is not valid, until pask_decode_step_drain returns
  *                  (synchronising `stream` alone is not enough: the output copy is not on it)
  * pask_decode_step_drain blocks the host until every pipelined call issued so far has finished. */
@@ -396,10 +406,7 @@ pask_status_t pask_debug_page_ids(pask_cache_t *cache, int32_t layer, int32_t se
                                   pask_stream_t stream);
 /* out[4] = { high bump counter, high free-stack depth, low bump counter, low free-stack depth }. */
 pask_status_t pask_debug_pool_state(pask_cache_t *cache, uint32_t *out4, pask_stream_t stream);
-/* The cache's first `count` (<= 64) control words: [0] device status, [2..5] pool state, [16..23]
- * wait statistics of decode attention as four 64-bit sums over warps (jobs, jobs that had to wait
- * for their bulk copy, cycles waited, cycles alive) -- filled only by diagnostic builds compiled
- * with PASK_STATS, zero otherwise. */
+/* The cache's first `count` (<= 64) control words: [0] device status, [2..5] pool state. */
 pask_status_t pask_debug_ctrl_words(pask_cache_t *cache, uint32_t *out, int32_t count, pask_stream_t stream);
 /* How the decode-attention kernel splits work.  Each sequence's pages are visited in a fixed order
  * that interleaves its HIGH and LOW pages evenly; pask_debug_page_order writes that order for a
@@ -415,6 +422,16 @@ pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, c
  * SM).  Any value >= 1 gives the same result up to summation order; tests use it to check that.
  * Workspaces must be sized (pask_workspace_bytes) after the change. */
 pask_status_t pask_debug_set_attention_ctas(pask_cache_t *cache, int32_t n_ctas);
+/* The only device-side waits of the library are those of the decode-attention kernel for its bulk
+ * copies into shared memory.  Each is bounded: after `limit_cycles` SM clock cycles (default 2e9,
+ * about a second) the warp gives up, sets PASK_DEV_TIMEOUT, writes empty partials for the rest of
+ * its range, waits (bounded again) until every copy it had issued has landed, and returns; the
+ * context stays usable and pask_cache_reset clears the bit.  pask_debug_set_wait sets the limit
+ * (>= 1000) and, for testing that path without anything going wrong on the GPU, a number of bytes
+ * (multiple of 16, <= 65536; 0 = normal operation) that the first copy of every warp announces to its
+ * barrier on top of what it brings: the copy completes as always, the barrier does not, the wait
+ * runs out.  Host-side settings of the handle, used by the calls issued after it. */
+pask_status_t pask_debug_set_wait(pask_cache_t *cache, int64_t limit_cycles, uint32_t surplus_bytes);
 
 const char *pask_status_string(pask_status_t status);
 

@@ -31,7 +31,7 @@ EXPORTS = [
     "pask_append_kv_decided", "pask_append_attend", "pask_decode_attention",
     "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes", "pask_step_packed_layout", "pask_decode_step_packed", "pask_decode_step_pipelined", "pask_decode_step_drain",
     "pask_budget_state", "pask_distortion", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
-    "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_status_string",
+    "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_debug_set_wait", "pask_status_string",
 ]
 
 
@@ -102,6 +102,7 @@ _lib.pask_debug_ctrl_words.argtypes = [_vp, _vp, _i32, _vp]
 _lib.pask_debug_partition.argtypes = [_i32, _vp, _vp, _i32, _vp]
 _lib.pask_debug_page_order.argtypes = [C.c_uint32, C.c_uint32, _vp]
 _lib.pask_debug_set_attention_ctas.argtypes = [_vp, _i32]
+_lib.pask_debug_set_wait.argtypes = [_vp, C.c_int64, C.c_uint32]
 _lib.pask_status_string.argtypes = [_i32]
 _lib.pask_status_string.restype = C.c_char_p
 
@@ -388,6 +389,11 @@ def pask_debug_page_order(pages_high: int, pages_low: int):
 
 def pask_debug_set_attention_ctas(cache: int, n_ctas: int):
     _check(_lib.pask_debug_set_attention_ctas(cache, n_ctas), "pask_debug_set_attention_ctas")
+
+
+def pask_debug_set_wait(cache: int, limit_cycles: int = 2_000_000_000, surplus_bytes: int = 0):
+    """Bound of the decode-attention kernel's waits for its bulk copies, and the test aid that makes one run out."""
+    _check(_lib.pask_debug_set_wait(cache, limit_cycles, surplus_bytes), "pask_debug_set_wait")
 
 
 class Cache:

@@ -23,8 +23,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     deps = srcs + [os.path.normpath(os.path.join(CSRC, h)) for h in HEADERS]
     if not force and os.path.exists(OUT) and os.path.getmtime(OUT) >= _newest(deps):
         return OUT
-    extra = os.environ.get("PASK_EXTRA_NVCC_FLAGS", "").split()     # e.g. -DPASK_INTERLEAVE=0 for experiments
-    cmd = ["nvcc"] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", OUT] + srcs
+    cmd = ["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", OUT] + srcs + ["-ldl"]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)

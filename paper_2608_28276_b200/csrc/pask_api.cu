@@ -3,6 +3,8 @@
 #include <memory>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "pask_internal.h"
 
 using namespace pask;
@@ -10,6 +12,12 @@ using namespace pask;
 namespace {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// NVTX range around the host side of an entry point (header-only NVTX: a no-op unless a profiler is attached)
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
 
 uint32_t rd32(const uint8_t *p) {
     return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24);
@@ -200,6 +208,8 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     c->meta = meta;
     c->sm_count = sms;
     c->ev_start = c->ev_stop = nullptr;
+    c->wait_cycles = 2000000000LL;   // about one second: give up instead of hanging
+    c->wait_test_surplus = 0;
     c->off = meta_offsets(d, 255, PASK_MAX_GROUPS);
     uint8_t *m = static_cast<uint8_t *>(meta);
     DevCache &v = c->dev;
@@ -335,6 +345,7 @@ static pask_status_t append_common(pask_cache_t *c, int32_t layer, int32_t n_seq
     if (total_tokens > 0 && (!k || !v)) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)k | (uintptr_t)v) & 15) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)seq_ids | (uintptr_t)cu_tokens) & 3) return PASK_ERR_INVALID_ARG;
+    NvtxRange range("pask_append_kv");
     return launch_append(c, layer, n_seqs, total_tokens, seq_ids, cu_tokens, k, v, tags, decided, actions_out,
                          static_cast<cudaStream_t>(stream), fuse_ws, fused);
 }
@@ -361,6 +372,7 @@ pask_status_t pask_decide(pask_cache_t *c, int32_t n_seqs, int32_t total_tokens,
     if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL || n_seqs > c->desc.max_seqs) return PASK_ERR_INVALID_ARG;
     if (total_tokens < 0) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)seq_ids | (uintptr_t)cu_tokens) & 3 || ((uintptr_t)states & 1)) return PASK_ERR_INVALID_ARG;
+    NvtxRange range("pask_decide");
     return launch_decide(c, n_seqs, total_tokens, seq_ids, cu_tokens, tags, states, actions_out,
                          static_cast<cudaStream_t>(stream));
 }
@@ -374,6 +386,7 @@ static pask_status_t attention_common(pask_cache_t *c, bool has_low, int32_t lay
     if (((uintptr_t)q | (uintptr_t)out) & 15 || ((uintptr_t)ws & 255) || ((uintptr_t)lse & 3)) return PASK_ERR_INVALID_ARG;
     if (ws_bytes < attention_workspace_bytes(c, n_seqs)) return PASK_ERR_WORKSPACE;
     if (check_only) return PASK_OK;
+    NvtxRange range(has_low ? "pask_decode_attention" : "pask_decode_attention_full");
     return launch_attention(c, has_low, layer, n_seqs, seq_ids, q, out, lse, ws, ws_bytes,
                             static_cast<cudaStream_t>(stream), plan_done);
 }
@@ -505,7 +518,10 @@ pask_status_t pask_decode_step_pipelined(pask_cache_t *c, int32_t layer, int32_t
     if (!c || !packed_host || !out_host || !staging) return PASK_ERR_INVALID_ARG;
     if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL) return PASK_ERR_INVALID_ARG;
     const size_t slot_bytes = pask_step_staging_bytes(c, n_seqs);
-    if (((uintptr_t)staging & 255) || staging_bytes < 2 * slot_bytes) return PASK_ERR_WORKSPACE;
+    // The two slots are the two halves of the staging buffer, whatever the batch: a call's slot never overlaps the
+    // other slot of an earlier call with a different n_seqs.
+    const size_t slot_stride = (staging_bytes / 2) & ~(size_t)255;
+    if (((uintptr_t)staging & 255) || slot_stride < slot_bytes) return PASK_ERR_WORKSPACE;
     auto &pp = c->pipe;
     if (!pp.ready) {   // host-side handles only; no device memory
         bool ok = cudaStreamCreateWithFlags(&pp.in, cudaStreamNonBlocking) == cudaSuccess &&
@@ -522,26 +538,43 @@ pask_status_t pask_decode_step_pipelined(pask_cache_t *c, int32_t layer, int32_t
     pask_step_packed_layout(c, n_seqs, off, &in_bytes);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const int slot = (int)(pp.calls & 1);
-    uint8_t *p = static_cast<uint8_t *>(staging) + (size_t)slot * slot_bytes;
+    uint8_t *p = static_cast<uint8_t *>(staging) + (size_t)slot * slot_stride;
     float *d_out = reinterpret_cast<float *>(p + in_bytes);
     cudaError_t e = cudaSuccess;
+    // A different staging buffer (or size: the halves move) than the call before: the new slot may overlap either of
+    // the old ones, so the input copy waits for everything the earlier calls still read or write there.
+    const bool moved = pp.calls > 0 && (staging != pp.staging || staging_bytes != pp.staging_bytes);
+    pp.staging = staging;
+    pp.staging_bytes = staging_bytes;
+    // from here on the slot counts as used, whatever happens: the next call takes the other one
+    const uint64_t call = pp.calls++;
+    if (moved) {
+        for (int i = 0; i < 2 && e == cudaSuccess; i++) {
+            if (pp.recorded[i] & 1) e = cudaStreamWaitEvent(pp.in, pp.ev_done[i], 0);
+            if (e == cudaSuccess && (pp.recorded[i] & 2)) e = cudaStreamWaitEvent(pp.in, pp.ev_out[i], 0);
+        }
+    }
     // this slot's inputs were last read by the kernels of two calls ago, its output by that call's copy-out
-    if (pp.calls >= 2) e = cudaStreamWaitEvent(pp.in, pp.ev_done[slot], 0);
+    if (e == cudaSuccess && (pp.recorded[slot] & 1)) e = cudaStreamWaitEvent(pp.in, pp.ev_done[slot], 0);
     if (e == cudaSuccess) e = cudaMemcpyAsync(p, packed_host, in_bytes, cudaMemcpyHostToDevice, pp.in);
     if (e == cudaSuccess) e = cudaEventRecord(pp.ev_in[slot], pp.in);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, pp.ev_in[slot], 0);
-    if (e == cudaSuccess && pp.calls >= 2) e = cudaStreamWaitEvent(stream, pp.ev_out[slot], 0);
+    if (e == cudaSuccess && (pp.recorded[slot] & 2)) e = cudaStreamWaitEvent(stream, pp.ev_out[slot], 0);
+    if (e == cudaSuccess && moved && (pp.recorded[slot ^ 1] & 2)) e = cudaStreamWaitEvent(stream, pp.ev_out[slot ^ 1], 0);
     if (e != cudaSuccess) return PASK_ERR_CUDA;
+    (void)call;
     pask_status_t rc = pask_append_attend(c, layer, n_seqs, n_seqs, reinterpret_cast<const int32_t *>(p + off[0]),
                                           reinterpret_cast<const int32_t *>(p + off[1]), p + off[2], p + off[3], p + off[4],
                                           nullptr, nullptr, p + off[5], d_out, nullptr, ws, ws_bytes, stream_v);
-    if (rc != PASK_OK) return rc;
+    // whatever was enqueued reads this slot: mark its end on the caller's stream even if the step was refused
     e = cudaEventRecord(pp.ev_done[slot], stream);
+    if (e == cudaSuccess) pp.recorded[slot] |= 1;
+    if (rc != PASK_OK) return rc;
     if (e == cudaSuccess) e = cudaStreamWaitEvent(pp.out, pp.ev_done[slot], 0);
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(out_host, d_out, (size_t)n_seqs * c->desc.n_q_heads * kHeadDim * 4, cudaMemcpyDeviceToHost, pp.out);
     if (e == cudaSuccess) e = cudaEventRecord(pp.ev_out[slot], pp.out);
-    pp.calls++;
+    if (e == cudaSuccess) pp.recorded[slot] |= 2;
     return cuda_rc(e);
 }
 
@@ -723,6 +756,13 @@ pask_status_t pask_debug_dump_low(pask_cache_t *c, int32_t layer, int32_t seq, u
 pask_status_t pask_debug_set_attention_ctas(pask_cache_t *c, int32_t n_ctas) {
     if (!c || n_ctas < 1 || n_ctas > 65536) return PASK_ERR_INVALID_ARG;
     c->attn_ctas = n_ctas;
+    return PASK_OK;
+}
+
+pask_status_t pask_debug_set_wait(pask_cache_t *c, int64_t limit_cycles, uint32_t surplus_bytes) {
+    if (!c || limit_cycles < 1000 || surplus_bytes > 65536u || (surplus_bytes & 15u)) return PASK_ERR_INVALID_ARG;
+    c->wait_cycles = limit_cycles;
+    c->wait_test_surplus = surplus_bytes;
     return PASK_OK;
 }
 

@@ -44,7 +44,6 @@ constexpr int kStages = 3;
 constexpr int kStageBytes = 4096;
 constexpr int kMaxWarps = 8;
 constexpr int kScratchBytes = 1152;              // per warp: fp16 query fragments (1024) + accumulator seeds (128)
-constexpr long long kWaitCycles = 2000000000LL;  // about one second: give up instead of hanging
 constexpr int kPlanThreads = 256;
 
 struct AttnParams {
@@ -53,6 +52,8 @@ struct AttnParams {
     const int32_t *seq_ids;
     const uint4 *q;         // bf16 [n_seqs][n_q][128] viewed as 16-byte chunks
     Workspace ws;
+    long long wait_cycles;  // bound of a wait for a bulk copy, in SM clock cycles
+    uint32_t overpost;      // test aid: bytes announced beyond what a warp's first copy brings (0 in normal use)
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -75,42 +76,35 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-// Bounded wait: false if the phase did not complete within kWaitCycles.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
+// Bounded wait: false if the phase did not complete within `limit` clock cycles.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, long long limit) {
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 256; i++)
             if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit) return false;
     }
+}
+// takes `bytes` off the barrier's pending transaction count, as the arrival of that many copied bytes would
+__device__ __forceinline__ void mbar_complete_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 // expect_tx + TMA bulk copy global -> this CTA's shared memory, completion counted on an mbarrier;
 // issued by one elected lane of a converged warp
 // (predicated, no divergent branch); the same lane leaves `word` at shared address `note`
 // The copy carries an L2 evict-first hint: every page is read exactly once per call.
-__device__ __forceinline__ void issue_bulk_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint32_t note,
-                                                   uint32_t word, uint64_t policy) {
-#ifndef PASK_NO_EVICT_FIRST
+// `announced` is the byte count the barrier is told to expect: `bytes`, except in the wait-limit test.
+__device__ __forceinline__ void issue_bulk_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t announced, uint32_t bar,
+                                                   uint32_t note, uint32_t word, uint64_t policy) {
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
         "elect.sync _|P, 0xffffffff;\n\t"
         "@P st.shared.u32 [%4], %5;\n\t"
-        "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %2;\n\t"
+        "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %7;\n\t"
         "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %6;\n\t}"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "r"(note), "r"(word), "l"(policy)
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "r"(note), "r"(word), "l"(policy), "r"(announced)
         : "memory");
-#else
-    (void)policy;
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "elect.sync _|P, 0xffffffff;\n\t"
-        "@P st.shared.u32 [%4], %5;\n\t"
-        "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %2;\n\t"
-        "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "r"(note), "r"(word)
-        : "memory");
-#endif
 }
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {
     uint64_t pol;
@@ -347,6 +341,9 @@ struct Pipe {
     uint32_t stride_high, stride_low;      // page size in bytes
     uint32_t low_two, low_job_bytes;       // 8-bit LOW pages come as two jobs (K half, V half) of low_job_bytes each
     uint32_t *status;         // the cache's device status word
+    long long wait_cycles;    // bound of one wait
+    uint32_t surplus;         // bytes the next copy announces beyond what it brings (wait-limit test; else 0)
+    uint32_t owed;            // such bytes still pending on the barrier of stage 0
     uint64_t policy;          // L2 cache policy of the bulk copies
     int lane;
     uint32_t ring, bars, meta;   // shared-space addresses of this warp's stages, mbarriers and entry words
@@ -373,7 +370,10 @@ struct Pipe {
         const uint8_t *src = is_high ? base_high + (size_t)id * stride_high + p_sub * kHighTileBytes
                                      : base_low + (size_t)id * stride_low + p_sub * low_job_bytes;
         const uint32_t bytes = is_high ? kHighTileBytes : low_job_bytes;
-        issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bars + p_stage * 8, meta + p_stage * 4, entry, policy);
+        issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bytes + surplus, bars + p_stage * 8, meta + p_stage * 4, entry,
+                           policy);
+        owed += surplus;          // (only a warp's first copy, which goes to stage 0, ever announces a surplus)
+        surplus = 0;
         p_stage = p_stage + 1 == kStages ? 0 : p_stage + 1;
         outstanding++;
         const bool two = is_high || low_two;               // a HIGH page is two jobs, an 8-bit LOW page too
@@ -386,7 +386,7 @@ struct Pipe {
     __device__ __forceinline__ uint32_t acquire(uint32_t &entry) {
         const uint32_t bar = bars + c_stage * 8;
         if (!mbar_try_wait(bar, c_parity)) {
-            if (dead || !mbar_wait_slow(bar, c_parity)) {
+            if (dead || !mbar_wait_slow(bar, c_parity, wait_cycles)) {
                 if (!dead && lane == 0) atomicOr(status, PASK_DEV_TIMEOUT);
                 dead = true;
             }
@@ -467,6 +467,9 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     w.low_two = kLow == 8;
     w.low_job_bytes = kLow == 8 ? kLow8HalfBytes : kLow == 2 ? kLow2HeadBytes : kLowHeadBytes;
     w.status = c.ctrl + kCtrlStatus;
+    w.wait_cycles = p.wait_cycles;
+    w.surplus = p.overpost;
+    w.owed = 0;
     w.policy = l2_evict_first_policy();
     w.lane = lane;
     w.ring = smem_u32(s_ring + (size_t)warp * kStages * kStageBytes);
@@ -829,7 +832,9 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 }
             }
         }
-        if (w.dead) break;   // a wait ran out: results are void, the status word says so
+        // A wait ran out: the status word says so and the results of the call are void.  This warp's partials of
+        // this and of the CTA's later sequences are written as empty ones, which the merge skips.
+        if (w.dead) { m_a = m_b = -INFINITY; l_a = l_b = 0.f; }
 
         // ---- this segment's partial: (m, l) per head, unnormalised o
 #pragma unroll
@@ -855,11 +860,16 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     }
 
     // A wait gave up: copies may still be in flight towards this CTA's shared memory.  Give each
-    // outstanding stage one more bounded wait before the CTA retires.
+    // outstanding stage one more bounded wait before the CTA retires; the ring is not read again.
     if (w.dead) {
+        if (w.owed) {   // wait-limit test: bytes were announced that no copy brings; take them off, so that the
+                        // barrier completes exactly when the real copy has landed
+            if (lane == 0) mbar_complete_tx(w.bars, w.owed);
+            __syncwarp();
+        }
         while (w.outstanding > 0) {
             const uint32_t bar = w.bars + w.c_stage * 8;
-            if (!mbar_try_wait(bar, w.c_parity)) mbar_wait_slow(bar, w.c_parity);
+            if (!mbar_try_wait(bar, w.c_parity)) mbar_wait_slow(bar, w.c_parity, w.wait_cycles > 200000000LL ? w.wait_cycles : 200000000LL);
             if (++w.c_stage == kStages) { w.c_stage = 0; w.c_parity ^= 1u; }
             w.outstanding--;
         }
@@ -962,11 +972,23 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
     p.seq_ids = seq_ids;
     p.q = static_cast<const uint4 *>(q);
     carve_workspace(c, n_seqs, static_cast<uint8_t *>(workspace), &p.ws);
+    p.wait_cycles = c->wait_cycles;
+    p.overpost = c->wait_test_surplus;
     const size_t smem = attn_smem_bytes(n_seqs, n_warps);
     auto kern = !has_low ? decode_attn_kernel<0> : c->dev.low_bits == 8 ? decode_attn_kernel<8>
               : c->dev.low_bits == 2 ? decode_attn_kernel<2> : decode_attn_kernel<4>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return PASK_ERR_CUDA;
+    // The shared-memory opt-in is a property of (device, kernel): ask for it once, and again only for a larger size.
+    {
+        static size_t granted[64][4] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return PASK_ERR_CUDA;
+        size_t &have = granted[dev][!has_low ? 0 : c->dev.low_bits == 8 ? 1 : c->dev.low_bits == 2 ? 2 : 3];
+        if (smem > have) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+                return PASK_ERR_CUDA;
+            have = smem;
+        }
+    }
     cudaError_t e = cudaSuccess;
     if (!plan_done)   // (a fused append has already left the plan in the workspace)
         e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(5 * n_seqs + 2) * 4, stream, c->dev,

@@ -89,7 +89,10 @@ decide_kernel(DevCache c, int n_seqs, int total_tokens, const int32_t *__restric
                     const int64_t R = (int64_t)(((uint64_t)c.budget_q16 * full) >> 16) - (int64_t)ret;
                     int64_t B = R - (int64_t)gamma;
                     if (B < 0) B = 0;
-                    if ((int64_t)cost > B) {
+                    // Protected and unknown tags sit at H with floor H in every group and have no row of upgrade
+                    // scores (s_rho holds n_tags rows): neither loop may run for them.
+                    const bool scored = tag < (uint32_t)c.n_tags;
+                    if (scored && (int64_t)cost > B) {
                         // Demote: one adjacent step at a time, smallest upgrade score first, never below a floor
                         while ((int64_t)cost > B) {
                             int pick = -1;
@@ -107,8 +110,10 @@ decide_kernel(DevCache c, int n_seqs, int total_tokens, const int32_t *__restric
                             n_dem++;
                         }
                         if ((int64_t)cost > B) n_conf++;   // floors first
+                    } else if ((int64_t)cost > B) {
+                        n_conf++;                          // a protected / unknown tag over budget: its floors stay
                     }
-                    if (crit) {
+                    if (crit && scored) {
                         // Promote: while an adjacent step up still fits in B, take the one with the largest score
                         for (;;) {
                             int pick = -1;

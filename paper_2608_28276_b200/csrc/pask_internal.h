@@ -22,7 +22,6 @@ enum CtrlWord : int {
     kCtrlItems = 7,     // work items (stream pages touched) of the last committed bulk append
     kCtrlSerial = 8,    // serial of the last launch that marks sequences (duplicate detection); kept on the device so
                         // that a launch recorded in a CUDA graph gets a fresh one at every replay
-    kCtrlStats = 16,    // 8 words of decode-attention wait statistics (diagnostic builds with PASK_STATS only)
     kCtrlWords = 64
 };
 
@@ -126,12 +125,17 @@ struct pask_cache {
     int sm_count;
     int attn_ctas;                // grid of the decode-attention main kernel
     cudaEvent_t ev_start, ev_stop;
+    long long wait_cycles;        // bound of a device-side wait for a bulk copy, in SM clock cycles (about a second)
+    uint32_t wait_test_surplus;   // pask_debug_set_wait: bytes a warp's first copy announces but does not bring
     // pask_decode_step_pipelined: two copy streams and the events that order them against the caller's stream
     struct StepPipe {
         bool ready = false;
         cudaStream_t in = nullptr, out = nullptr;
         cudaEvent_t ev_in[2] = {}, ev_done[2] = {}, ev_out[2] = {};
         uint64_t calls = 0;
+        int recorded[2] = {0, 0};         // per slot: bit 0 = ev_done has been recorded, bit 1 = ev_out
+        const void *staging = nullptr;    // the staging buffer of the call before
+        size_t staging_bytes = 0;
     } pipe;
 };
 

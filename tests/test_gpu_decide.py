@@ -186,3 +186,38 @@ def test_sequence_reset_clears_the_running_budget(pask, oracle):
     p.decide([1], [30], tags, states)                                   # starts again from an empty budget
     p.compare_budget(1)
     p.compare_budget(0)
+
+
+def test_protected_and_unknown_tags_in_critical_states_with_eight_groups(pask, oracle):
+    # tag bytes outside the table (0xFF = protected, 200 and 254 = unknown) have no row of upgrade scores: they stay
+    # at H in all eight groups whatever the budget says, are counted as floor conflicts when over budget, and the
+    # scored tokens around them are adjusted exactly as the oracle adjusts them
+    G, n_tags = 8, 6
+    rng = np.random.default_rng(5)
+    pol = WP.Policy(n_tags, G, np.arange(G, dtype=np.uint8), rng.integers(0, 3, (n_tags, G)).astype(np.uint8),
+                    np.zeros((n_tags, G), np.uint8), rng.random((n_tags, G)).astype(np.float32),
+                    rng.random((n_tags, G)).astype(np.float32), gamma=np.asarray([0, 4096, 0, 1 << 14], np.uint32),
+                    budget_target=0.25, crit=np.asarray([1, 1, 0, 1], np.uint8))
+    blob = WP.write_blob(pol)
+    c = pask.Cache(blob, G, 8, 2, 1, 256, 256, 16, 16)
+    orc = oracle.Cache(oracle.Policy(blob), 8, 2, 1, 16, 16)
+    n = 200
+    tags = rng.integers(0, n_tags, n).astype(np.uint8)
+    tags[rng.random(n) < 0.3] = 0xFF
+    tags[rng.random(n) < 0.1] = 200
+    tags[7] = 254
+    states = rng.integers(0, 4, n).astype(np.uint16)
+    rc, act_o = orc.decide([0], [0, n], tags, states=states, n_groups=G)
+    assert rc == 0
+    d = "cuda"
+    act = torch.full((n, G), 0xEE, dtype=torch.uint8, device=d)
+    pask.pask_decide(c.handle, torch.tensor([0], dtype=torch.int32, device=d), torch.tensor([0, n], dtype=torch.int32, device=d),
+                     torch.from_numpy(tags).to(d), torch.from_numpy(states.astype(np.int16)).to(d), act)
+    got = act.cpu().numpy()
+    assert np.array_equal(got, act_o)
+    assert np.all(got[tags >= n_tags] == 2)
+    g, o = pask.pask_budget_state(c.handle, 0), orc.budget(0)
+    for f in ("decided_full_bytes", "decided_retained_bytes", "n_demoted", "n_promoted", "n_floor_conflicts"):
+        assert getattr(g, f) == getattr(o, f), f
+    assert g.n_floor_conflicts > 0 and g.n_demoted > 0 and g.device_status == 0
+    c.close()

@@ -397,3 +397,49 @@ def test_pipelined_host_steps(pask, oracle):
     for block, out, oo, ol in calls:
         assert_close(out.numpy().astype(np.float64), ol.copy(), oo, ol)
     p.compare_state()
+
+
+def test_pipelined_host_steps_with_a_batch_that_changes_from_call_to_call(pask, oracle):
+    # consecutive pipelined calls with different n_seqs: the two staging slots are the buffer's fixed halves, so a
+    # call's slot never reaches into the slot the call before is still reading; outputs are the oracle's throughout
+    from pask_workloads.tensors import bf16_bits
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=6, n_layers=2, n_groups=2, prompt_len=120, gen_len=60, extra_gen=64)
+    w = WC.build(cfg)
+    p = Pair(pask, oracle, w)
+    everyone = [3, 0, 4, 1, 2, 5]
+    for layer in range(2):
+        p.append(layer, everyone, [180] * 6, [0] * 6)
+    P, h = pask, p.gpu.handle
+    staging = torch.empty(2 * P.pask_step_staging_bytes(h, 6), dtype=torch.uint8, device="cuda")
+    pos = {s: 180 for s in everyone}
+    calls = []
+    for step, seqs in enumerate(([3, 0, 4, 1, 2, 5], [5], [0, 1, 2, 3], [4, 2], [1, 5, 0, 3, 2, 4], [2], [0, 5, 1])):
+        n = len(seqs)
+        off, n_in = P.pask_step_packed_layout(h, n)
+        for layer in range(2):
+            k = torch.stack([w.kv(layer, b, pos[b], 1)[0][0] for b in seqs])
+            v = torch.stack([w.kv(layer, b, pos[b], 1)[1][0] for b in seqs])
+            tags = torch.from_numpy(np.array([w.tags(b, pos[b], 1)[0] for b in seqs], np.uint8))
+            q = torch.stack([w.q(layer, b, pos[b] + 1) for b in seqs])
+            block = torch.zeros(n_in, dtype=torch.uint8).pin_memory()
+            for o, t in zip(off, [torch.tensor(seqs, dtype=torch.int32), torch.arange(n + 1, dtype=torch.int32), k, v, tags, q]):
+                raw = t.contiguous().view(torch.uint8).reshape(-1)
+                block[o:o + raw.numel()] = raw
+            out = torch.full((n, 32, 128), float("nan"), dtype=torch.float32).pin_memory()
+            P.pask_decode_step_pipelined(h, layer, n, block, out, staging, p.gpu.workspace(n))
+            rc, _ = p.orc.append(layer, seqs, list(range(n + 1)), bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags.numpy())
+            assert rc == 0
+            oo, ol = p.orc.attention_batch(layer, seqs, bf16_bits(q).numpy())
+            calls.append((block, out, oo, ol))
+        for b in seqs:
+            pos[b] += 1
+    P.pask_decode_step_drain(h)
+    torch.cuda.synchronize()
+    for block, out, oo, ol in calls:
+        assert_close(out.numpy().astype(np.float64), ol.copy(), oo, ol)
+    p.compare_state()
+    # halves too small for the batch are refused
+    small = torch.empty(2 * P.pask_step_staging_bytes(h, 6) - 512, dtype=torch.uint8, device="cuda")
+    with pytest.raises(P.PaskError) as e:
+        P.pask_decode_step_pipelined(h, 0, 6, calls[0][0], calls[0][1], small, p.gpu.workspace(6))
+    assert e.value.status == P.ERR_WORKSPACE

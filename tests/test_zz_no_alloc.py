@@ -3,7 +3,9 @@
 An engine that has already given all free device memory to its own block pool, or code running
 where a device allocation is not allowed, cannot hand the library a scratch buffer. This entry
 point uses a fixed scratch array built into the library instead. The test calls it through the
-C ABI twice in a row and compares both results with pask_decode_attention on the same cache.
+C ABI twice in a row and compares both results with the CPU oracle's attention over the same
+history (the parity bound of every other attention test) and, as a second check, with
+pask_decode_attention on the same cache.
 (The file name makes pytest collect it after every other test.)"""
 import numpy as np
 import pytest
@@ -11,12 +13,14 @@ import torch
 
 from pask_workloads import configs as WC
 
-from parity import ATOL_MAX, RTOL_L2
+from pask_workloads.tensors import bf16_bits
+
+from parity import ATOL_MAX, RTOL_L2, assert_close
 
 pytestmark = pytest.mark.gpu
 
 
-def test_static_workspace_matches_caller_workspace_twice_in_a_row():
+def test_static_workspace_matches_oracle_and_caller_workspace_twice_in_a_row(oracle):
     import paper_2608_28276_b200 as P
     assert torch.cuda.is_available()
     d = "cuda"
@@ -32,6 +36,10 @@ def test_static_workspace_matches_caller_workspace_twice_in_a_row():
     tags = torch.from_numpy(np.concatenate([w.tags(b, 0, lens[b]) for b in range(cfg.batch)])).to(d)
     P.pask_append_kv(cache.handle, 0, ids, cu, k, v, tags)
     assert P.pask_budget_state(cache.handle, 0).device_status == 0
+    orc = oracle.Cache(oracle.Policy(w.blob), cfg.n_q, cfg.n_kv, cfg.batch, pages, pages)
+    rc, _ = orc.append(0, list(range(cfg.batch)), cu.cpu().numpy(), bf16_bits(k.cpu()).numpy(), bf16_bits(v.cpu()).numpy(),
+                       tags.cpu().numpy())
+    assert rc == 0
 
     def run(fn, q, *extra):
         out = torch.full((cfg.batch, cfg.n_q, 128), float("nan"), dtype=torch.float32, device=d)
@@ -45,7 +53,8 @@ def test_static_workspace_matches_caller_workspace_twice_in_a_row():
         q = torch.stack([w.q(0, b, lens[b] + call) for b in range(cfg.batch)]).to(d)
         ref_out, ref_lse = run(P.pask_decode_attention, q, cache.workspace(cfg.batch))
         got_out, got_lse = run(P.pask_decode_attention_static, q)
-        assert np.all(np.isfinite(got_out))
+        orc_out, orc_lse = orc.attention_batch(0, list(range(cfg.batch)), bf16_bits(q.cpu()).numpy())
+        assert_close(got_out, got_lse, orc_out, orc_lse, where=("static scratch vs oracle, call", call))
         for b in range(cfg.batch):
             assert np.abs(got_out[b] - ref_out[b]).max() <= ATOL_MAX
             assert np.linalg.norm(got_out[b] - ref_out[b]) <= RTOL_L2 * np.linalg.norm(ref_out[b])
