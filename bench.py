@@ -42,6 +42,7 @@ NOMINAL_HBM_GBS = 8000.0
 # summarised in profiles/decode_attn_kernel__qwen3-4b-step-first-4-layers.md (mean of three launches
 # of a 4-layer cut of this workload; traffic grows in proportion to the pages streamed)
 NCU_TRAFFIC_RATIO = 1.009
+NCU_TRAFFIC_PROFILE = "profiles/decode_attn_kernel__qwen3-4b-step-first-4-layers.md"
 STEP_STREAM = 1_000_000          # decode-step inputs of step i come from generator stream (layer, STEP_STREAM + i)
 
 CONFIGS = {c.name: c for c in WC.CONFIGS}
@@ -327,6 +328,141 @@ class Job:
         return per_layer
 
 
+class Runner:
+    """Times decode steps of one Job: blocks of exactly K steps bracketed by a barrier and a device
+    synchronisation on both sides, CUDA events on the launching stream, MAX over ranks."""
+
+    def __init__(self, args, world, device):
+        self.args, self.world, self.device = args, world, device
+
+    def barrier(self):
+        if self.world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def block(self, job, first_step, n_steps, with_events=True, graph=False):
+        """One timed block; returns (ms of the block, [ms of each timed streaming-kernel launch])."""
+        evs = kernel_events(job.cfg.n_layers, n_steps, self.args.event_stride) if (with_events and not graph) else None
+        self.barrier()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for i in range(n_steps):
+            if graph:
+                job.graphs[first_step + i].replay()
+            else:
+                job.run_step(first_step + i, evs[i] if evs else None)
+        t1.record()
+        self.barrier()
+        ms = max_over_ranks(t0.elapsed_time(t1), self.device)
+        kern = [a.elapsed_time(b) for row in (evs or []) for a, b in row.values()]
+        return ms, kern
+
+
+def kernel_figures(job, kern_ms, steps_done, peak):
+    """Roofline figures of the streaming kernel from its live launch times."""
+    alg = job.algorithmic_bytes_per_layer(steps_done)
+    if not kern_ms:
+        return {"algorithmic_bytes_per_launch": alg, "avg_launch_ms": None, "achieved": None, "frac": None}
+    k_ms = sum(kern_ms) / len(kern_ms)
+    achieved = alg / (k_ms * 1e-3) / 1e9
+    return {"algorithmic_bytes_per_launch": alg, "avg_launch_ms": k_ms, "launches_timed": len(kern_ms),
+            "achieved": achieved, "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+
+
+def check_status(P, job, where):
+    st = P.pask_budget_state(job.cache.handle, 0)
+    if st.device_status:
+        raise RuntimeError(f"device status {st.device_status:#x} {where}")
+
+
+def quick_point(P, runner, cfg, device, steps, peak, repeat=0, policy_blob=None, label="pask", clocks_index=None):
+    """One further measurement point: build the workload, fill the cache, 3 warm-up steps, one timed block.
+    Returns a small dict (tokens/s, ms/step, streaming-kernel GB/s and fraction of the peak, clocks)."""
+    warm = 3
+    cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, warm + steps + 8))
+    t_setup = time.time()
+    w = WC.build(cfg, repeat=repeat)
+    if policy_blob == "all_high":                 # the dense comparison cache: every token kept at bf16
+        from pask_workloads.policy import all_high_policy, write_blob
+        policy_blob = write_blob(all_high_policy(w.policy.n_tags, cfg.n_groups, cfg.n_layers))
+    job = Job(P, w, device, warm + steps + 4, policy_blob=policy_blob, label=label)
+    job.fused = policy_blob is None
+    job.fill()
+    job.prepare_steps(warm + steps)
+    t_setup = time.time() - t_setup
+    for i in range(warm):
+        job.run_step(i)
+    sampler = ClockSampler(clocks_index if clocks_index is not None else (device.index or 0))
+    sampler.start()
+    ms, kern = runner.block(job, warm, steps)
+    clocks = sampler.stop()
+    check_status(P, job, f"after {cfg.name}")
+    ret = sum(P.pask_budget_state(job.cache.handle, b).retained_bytes for b in range(job.B))
+    full = sum(P.pask_budget_state(job.cache.handle, b).full_bytes for b in range(job.B))
+    fig = kernel_figures(job, kern, warm + steps // 2, peak)
+    out = {"workload": cfg.name, "kernel": label, "batch": job.B, "layers": cfg.n_layers, "kv_budget_target": cfg.budget,
+           "kv_budget_realised": ret / full, "table": f"{cfg.lut}/{cfg.bias}", "steps": steps, "warmup": warm,
+           "tokens_per_s": job.B * steps / (ms * 1e-3), "ms_per_step": ms / steps,
+           "kernel_GBs": fig["achieved"], "frac": fig["frac"], "frac_of_nominal_8TBs": fig.get("frac_of_nominal_8TBs"),
+           "avg_launch_ms": fig["avg_launch_ms"], "algorithmic_bytes_per_launch": fig["algorithmic_bytes_per_launch"],
+           "clocks": clocks, "setup_s": round(t_setup, 1)}
+    if len(job.fill_ms) > 1:
+        out["bulk_append_ms_per_layer_call"] = sum(job.fill_ms[1:]) / (len(job.fill_ms) - 1)
+        out["tokens_in_cache"] = job.total_tokens
+    job.cache.close()
+    del job
+    torch.cuda.empty_cache()
+    return out
+
+
+def other_configs(P, runner, device, peak, args):
+    """The configurations of the metric's list besides the headline one, each measured in this run:
+    the budget sweep at the batch-64 8K shape against the full-KV kernel, the batch-128 16K case, the
+    concurrency-8 shapes of the paper's latency table, the LOW-heavy and HIGH-heavy tables at the
+    headline shape, and the one-layer batch-8 shape with its layer rotated over replicas."""
+    out, steps = [], max(4, min(args.steps, 10))
+
+    def add(fn, what):
+        try:
+            out.append(fn())
+        except Exception as e:                      # e.g. out of memory on a smaller part: say so, keep going
+            out.append({"workload": what, "unavailable": str(e)[:200]})
+            torch.cuda.empty_cache()
+
+    for b in WC.SWEEP_BUDGETS:
+        cfg = WC.scaled(WC.QWEN3_4B_SWEEP, budget=b, lut="all_high" if b >= 1.0 else "greedy")
+        add(lambda: quick_point(P, runner, cfg, device, steps, peak), f"{cfg.name} @ {b}")
+
+    def full_kv_sweep():
+        r = quick_point(P, runner, WC.QWEN3_4B_SWEEP, device, steps, peak, policy_blob="all_high", label="full-kv bf16 kernel")
+        r["kv_budget_target"] = 1.0
+        return r
+    add(full_kv_sweep, "full-KV at the sweep shape")
+    add(lambda: dict(quick_point(P, runner, WC.QWEN3_8B_LONG, device, max(3, steps // 2), peak),
+                     note="the dense comparison cache of this shape (309 GB) does not fit one GPU: PASK only"),
+        WC.QWEN3_8B_LONG.name)
+    for cfg in (WC.TABLE3_8K, WC.TABLE3_32K):
+        add(lambda: quick_point(P, runner, cfg, device, steps, peak), cfg.name)
+    for bias in ("low", "high"):
+        cfg = WC.scaled(WC.QWEN3_4B_STEP, bias=bias, name=f"{WC.QWEN3_4B_STEP.name}[{bias.upper()}-heavy table]")
+        add(lambda: quick_point(P, runner, cfg, device, steps, peak), cfg.name)
+
+    def one_layer_rotated():
+        # 16 layers = 4 replicas of each layer-group column, every one with its own pages: a step walks
+        # 16 distinct ~45 MB working sets (together far beyond L2), so no launch finds its pages in L2
+        reps = 4
+        base = WC.QWEN3_4B_1LAYER
+        cfg = WC.scaled(base, n_layers=base.n_groups * reps, name=f"{base.name}[x{reps} replicas per column]")
+        r = quick_point(P, runner, cfg, device, 2 * steps, peak)
+        r["layer_tokens_per_s"] = r["tokens_per_s"] * cfg.n_layers
+        r["tokens_per_s_at_36_layers"] = r["layer_tokens_per_s"] / 36.0
+        r["note"] = ("one-layer shape: tokens_per_s counts a pass over all 16 replica layers as one step; "
+                     "layer_tokens_per_s = batch x layer launches / s; L2: rotated over 16 distinct layer caches")
+        return r
+    add(one_layer_rotated, "one-layer shape, rotated")
+    return out
+
+
 def run_cuda(args, rank, world):
     import paper_2608_28276_b200 as P
     device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
@@ -339,7 +475,8 @@ def run_cuda(args, rank, world):
         cfg = WC.scaled(cfg, low_bits=args.low_bits, name=f"{cfg.name}[{args.low_bits}-bit low]")
     if args.layers:
         cfg = WC.scaled(cfg, n_layers=args.layers, name=f"{cfg.name}[first {args.layers} layers]")
-    total_steps = args.warmup + args.steps
+    repeats = max(1, args.repeats)
+    total_steps = args.warmup + repeats * args.steps
     e2e_steps = min(args.steps, 10)
     e2e_warm = 2                       # untimed end-to-end steps (the first call creates the library's copy streams)
     cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, 2 * total_steps + e2e_steps + e2e_warm + 8))
@@ -347,6 +484,8 @@ def run_cuda(args, rank, world):
     if args.window:
         from dataclasses import replace as _replace
         w.policy = _replace(w.policy, recent_window=args.window)
+    runner = Runner(args, world, device)
+    peak, peak_kind = measured_peaks()
     t_setup = time.time()
     job = Job(P, w, device, 2 * total_steps + e2e_steps + e2e_warm + 4, dynamic=args.dynamic)
     job.fused = not args.unfused
@@ -358,93 +497,36 @@ def run_cuda(args, rank, world):
     ret = sum(P.pask_budget_state(job.cache.handle, b).retained_bytes for b in range(job.B))
     full = sum(P.pask_budget_state(job.cache.handle, b).full_bytes for b in range(job.B))
 
-    def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
-
-    def timed(jb, first_step, n_steps, with_events):
-        evs = None
-        if with_events:
-            evs = kernel_events(cfg.n_layers, n_steps, args.event_stride)
-        barrier()
-        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for i in range(n_steps):
-            if args.graph and jb is job:
-                jb.graphs[first_step + i].replay()
-            else:
-                jb.run_step(first_step + i, evs[i] if evs else None)
-        t1.record()
-        barrier()
-        ms = t0.elapsed_time(t1)
-        kern = [a.elapsed_time(b) for row in (evs or []) for a, b in row.values()]
-        return ms, kern
-
     for i in range(args.warmup):
         job.run_step(i)
     if args.graph:
-        job.capture_steps(args.warmup, args.steps)
+        job.capture_steps(args.warmup, repeats * args.steps)
     sampler = ClockSampler(device.index or 0)
     if rank == 0:
         sampler.start()
-    ms, kern_ms = timed(job, args.warmup, args.steps, not args.graph)
+    # the timed region, `repeats` times over: each block is exactly --steps steps between two barriers
+    blocks, kern_ms, kern_by_block = [], [], []
+    for r in range(repeats):
+        ms, kern = runner.block(job, args.warmup + r * args.steps, args.steps, graph=args.graph)
+        blocks.append(ms)
+        kern_ms += kern
+        kern_by_block.append(sum(kern) / len(kern) if kern else None)
     clocks = sampler.stop() if rank == 0 else {}
-    ms = max_over_ranks(ms, device)
-    st = P.pask_budget_state(job.cache.handle, 0)
-    if st.device_status:
-        raise RuntimeError(f"device status {st.device_status:#x} after the timed region")
+    check_status(P, job, "after the timed region")
+    per_block = [whole_job_tokens_per_s(world, job.B, args.steps, ms) for ms in blocks]
+    ms = statistics.median(blocks)
     value = whole_job_tokens_per_s(world, job.B, args.steps, ms)
 
     # ---- end to end: the same step through the host-buffer entry point, copies inside the region
     e2e = None
     if (rank == 0 or world > 1) and not args.dynamic:   # the host-buffer entry point applies the frozen table
-        staging = torch.empty(2 * P.pask_step_staging_bytes(job.cache.handle, job.B), dtype=torch.uint8, device=device)
-        off, in_bytes = P.pask_step_packed_layout(job.cache.handle, job.B)
-        host = []
-        for s in range(e2e_warm + e2e_steps):   # a layer's inputs sit in one pinned block, as an engine would stage them
-            rows = []
-            for layer in range(cfg.n_layers):
-                k, v, q, tags = step_inputs(w, layer, total_steps + s, "cpu")
-                block = torch.zeros(in_bytes, dtype=torch.uint8).pin_memory()
-                parts = [torch.arange(job.B, dtype=torch.int32), torch.arange(job.B + 1, dtype=torch.int32), k, v,
-                         torch.from_numpy(tags), q]
-                for o, t in zip(off, parts):
-                    raw = t.contiguous().view(torch.uint8).reshape(-1)
-                    block[o:o + raw.numel()] = raw
-                rows.append(block)
-            host.append(rows)
-        out_h = torch.empty((job.B, cfg.n_q, 128), dtype=torch.float32).pin_memory()
-        for rows in host[:e2e_warm]:
-            for layer, block in enumerate(rows):
-                P.pask_decode_step_pipelined(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
-        P.pask_decode_step_drain(job.cache.handle)
-        barrier()
-        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for rows in host[e2e_warm:]:
-            for layer, block in enumerate(rows):
-                P.pask_decode_step_pipelined(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
-        P.pask_decode_step_drain(job.cache.handle)      # the host holds every output before the clock stops
-        t1.record()
-        barrier()
-        e_ms = t0.elapsed_time(t1)
-        e_ms = max_over_ranks(e_ms, device)
-        h2d = cfg.n_layers * in_bytes
-        d2h = cfg.n_layers * job.B * cfg.n_q * 128 * 4
-        e2e = {"value": whole_job_tokens_per_s(world, job.B, e2e_steps, e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps,
-               "api": "pask_decode_step_pipelined: one pinned host block in, attention output out, per layer; the "
-                      "copies run on the library's copy streams and overlap the neighbouring layers' kernels"}
+        e2e = end_to_end(P, runner, job, w, cfg, total_steps, e2e_warm, e2e_steps, world, device)
 
     if rank != 0:
         return
-    peak, peak_kind = measured_peaks()
-    alg = job.algorithmic_bytes_per_layer(args.warmup + args.steps // 2)
-    if not kern_ms:      # graph replay carries no per-kernel events: the kernel figures come from a plain run
-        kern_ms = [float("inf")]
-    k_ms = sum(kern_ms) / len(kern_ms)
-    achieved = alg / (k_ms * 1e-3) / 1e9
+    fig = kernel_figures(job, kern_ms, args.warmup + repeats * args.steps // 2, peak)
+    alg = fig["algorithmic_bytes_per_launch"]
+    covered = job.low_bits == 4 and not args.window and cfg.name == DEFAULT_CONFIG and args.bias == "balanced"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -455,21 +537,29 @@ def run_cuda(args, rank, world):
                    "tokens_in_cache_per_gpu": job.total_tokens, "page_tokens": 16,
                    "l2": "inputs larger than L2: each layer streams its own ~%.0f MB of pages" % (alg / 1e6),
                    "setup_s": round(t_setup, 1)},
+        "repeats": {"n": repeats, "statistic": "value = median over the timed blocks, each exactly `steps` steps",
+                    "tokens_per_s": per_block, "min": min(per_block), "max": max(per_block),
+                    "ms_per_block": blocks, "kernel_avg_launch_ms_per_block": kern_by_block},
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": (per_layer_launches * cfg.n_layers + (1 if args.dynamic else 0)) * args.steps,
-        "roofline": {"bound": "hbm", "kernel": f"decode_attn_kernel<{job.low_bits}>", "achieved": achieved, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "algorithmic_bytes_per_launch": alg,
-                     "avg_launch_ms": k_ms, "launches_timed": len(kern_ms), "traffic": alg * NCU_TRAFFIC_RATIO,
-                     "traffic_source": "ncu dram__bytes_read+write of a 4-layer cut, scaled by pages streamed"},
-        "attention_share_of_step": k_ms * cfg.n_layers * args.steps / ms,
-        "attention_only_tokens_per_s": world * job.B / (k_ms * 1e-3 * cfg.n_layers),
+        "roofline": {"bound": "hbm", "kernel": f"decode_attn_kernel<{job.low_bits}>", "achieved": fig["achieved"], "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": fig["frac"],
+                     "frac_of_nominal_8TBs": fig.get("frac_of_nominal_8TBs"), "algorithmic_bytes_per_launch": alg,
+                     "avg_launch_ms": fig["avg_launch_ms"], "launches_timed": fig.get("launches_timed"),
+                     "traffic": alg * NCU_TRAFFIC_RATIO if covered else None,
+                     "traffic_source": (f"estimated: {NCU_TRAFFIC_RATIO} x algorithmic bytes, the ratio of ncu "
+                                        "dram__bytes_read+write to algorithmic bytes in the capture summarised in "
+                                        f"{NCU_TRAFFIC_PROFILE} (a 4-layer cut of this workload)") if covered else
+                                       "no ncu capture covers this configuration"},
     }
+    if fig["avg_launch_ms"]:
+        k_ms = fig["avg_launch_ms"]
+        line["attention_share_of_step"] = k_ms * cfg.n_layers * args.steps / ms
+        line["attention_only_tokens_per_s"] = world * job.B / (k_ms * 1e-3 * cfg.n_layers)
     if args.graph:
         line["config"]["launch"] = "one CUDA graph per step"
         line["roofline"] = None
-        line["attention_share_of_step"] = line["attention_only_tokens_per_s"] = None
     if len(job.fill_ms) > 1:
         f_ms = sum(job.fill_ms[1:]) / (len(job.fill_ms) - 1)
         lg = w.policy.layer_group.astype(np.int64)
@@ -490,43 +580,69 @@ def run_cuda(args, rank, world):
                                   "demoted": sum(s.n_demoted for s in sts), "promoted": sum(s.n_promoted for s in sts),
                                   "floor_conflicts": sum(s.n_floor_conflicts for s in sts)}
         line["config"]["table"] += " + budget-dependent adjustment (pask_decide)"
-    if args.full_kv and world == 1:
-        line["full_kv"] = run_full_kv(P, args, w, device, total_steps, peak)
-    if args.cpu_seconds > 0 and world == 1:          # the oracle beside it: rank 0 at N = 1 only
-        line["cpu_baseline"] = cpu_baseline(w, budget_s=args.cpu_seconds, n_seqs=args.ref_seqs)
+    job.cache.close()
+    del job
+    torch.cuda.empty_cache()
+    if world == 1:
+        if args.seeds > 1:       # the same configuration from the next seeds: spread over inputs, not over time
+            pts = [quick_point(P, runner, cfg, device, args.steps, peak, repeat=r) for r in range(1, args.seeds)]
+            vals = [value] + [p["tokens_per_s"] for p in pts]
+            fr = [fig["frac"]] + [p["frac"] for p in pts]
+            line["seeds"] = {"n": args.seeds, "tokens_per_s": vals, "kernel_frac": fr, "median": statistics.median(vals),
+                             "min": min(vals), "max": max(vals),
+                             "note": "seed + 0 is the headline run (its median block); + 1, + 2: one timed block each"}
+        if args.full_kv:
+            r = quick_point(P, runner, cfg, device, args.steps, peak, policy_blob="all_high", label="full-kv bf16 kernel")
+            line["full_kv"] = {"value": r["tokens_per_s"], "unit": UNIT, "ms_per_step": r["ms_per_step"],
+                               "achieved_GBs": r["kernel_GBs"], "frac": r["frac"],
+                               "algorithmic_bytes_per_launch": r["algorithmic_bytes_per_launch"],
+                               "avg_launch_ms": r["avg_launch_ms"]}
+        if args.other_configs:
+            line["other_configs"] = other_configs(P, runner, device, peak, args)
+        if args.cpu_seconds > 0:          # the oracle beside it: rank 0 at N = 1 only
+            line["cpu_baseline"] = cpu_baseline(w, budget_s=args.cpu_seconds, n_seqs=args.ref_seqs)
     print(json.dumps(line))
 
 
-def run_full_kv(P, args, w, device, total_steps, peak):
-    """The same workload with every token kept at bf16, through the library's full-KV kernel."""
-    from pask_workloads.policy import all_high_policy, write_blob
-    cfg = w.cfg
-    blob = write_blob(all_high_policy(w.policy.n_tags, cfg.n_groups, cfg.n_layers))
-    try:
-        job = Job(P, w, device, total_steps + 4, policy_blob=blob, label="full-kv")
-        job.fill()
-    except Exception as e:      # e.g. not enough memory for the dense cache next to the PASK one
-        return {"unavailable": str(e)[:200]}
-    job.prepare_steps(total_steps)
-    for i in range(args.warmup):
-        job.run_step(i)
-    if args.graph:
-        job.capture_steps(args.warmup, args.steps)
-    evs = kernel_events(cfg.n_layers, args.steps, args.event_stride)
-    torch.cuda.synchronize()
+def end_to_end(P, runner, job, w, cfg, first_step, e2e_warm, e2e_steps, world, device):
+    """The same steps through pask_decode_step_pipelined: inputs start in pinned host memory and the
+    attention output ends there, every layer, inside the timed region."""
+    staging = torch.empty(2 * P.pask_step_staging_bytes(job.cache.handle, job.B), dtype=torch.uint8, device=device)
+    off, in_bytes = P.pask_step_packed_layout(job.cache.handle, job.B)
+    host = []
+    for s in range(e2e_warm + e2e_steps):   # a layer's inputs sit in one pinned block, as an engine would stage them
+        rows = []
+        for layer in range(cfg.n_layers):
+            k, v, q, tags = step_inputs(w, layer, first_step + s, "cpu")
+            block = torch.zeros(in_bytes, dtype=torch.uint8).pin_memory()
+            parts = [torch.arange(job.B, dtype=torch.int32), torch.arange(job.B + 1, dtype=torch.int32), k, v,
+                     torch.from_numpy(tags), q]
+            for o, t in zip(off, parts):
+                raw = t.contiguous().view(torch.uint8).reshape(-1)
+                block[o:o + raw.numel()] = raw
+            rows.append(block)
+        host.append(rows)
+    out_h = torch.empty((job.B, cfg.n_q, 128), dtype=torch.float32).pin_memory()
+    for rows in host[:e2e_warm]:
+        for layer, block in enumerate(rows):
+            P.pask_decode_step_pipelined(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
+    P.pask_decode_step_drain(job.cache.handle)
+    runner.barrier()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
-    for i in range(args.steps):
-        job.run_step(args.warmup + i, evs[i])
+    for rows in host[e2e_warm:]:
+        for layer, block in enumerate(rows):
+            P.pask_decode_step_pipelined(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
+    P.pask_decode_step_drain(job.cache.handle)      # the host holds every output before the clock stops
     t1.record()
-    torch.cuda.synchronize()
-    ms = t0.elapsed_time(t1)
-    kern = [a.elapsed_time(b) for row in evs for a, b in row.values()]
-    alg = job.algorithmic_bytes_per_layer(args.warmup + args.steps // 2)
-    k_ms = sum(kern) / len(kern)
-    return {"value": job.B * args.steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / args.steps,
-            "achieved_GBs": alg / (k_ms * 1e-3) / 1e9, "frac": alg / (k_ms * 1e-3) / 1e9 / peak,
-            "algorithmic_bytes_per_launch": alg, "avg_launch_ms": k_ms}
+    runner.barrier()
+    e_ms = max_over_ranks(t0.elapsed_time(t1), device)
+    h2d = cfg.n_layers * in_bytes
+    d2h = cfg.n_layers * job.B * cfg.n_q * 128 * 4
+    return {"value": whole_job_tokens_per_s(world, job.B, e2e_steps, e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps,
+            "api": "pask_decode_step_pipelined: one pinned host block in, attention output out, per layer; the "
+                   "copies run on the library's copy streams and overlap the neighbouring layers' kernels"}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -556,36 +672,55 @@ class OracleSample:
             del k, v
 
     def step(self, i):
-        B, t = self.B, 0.0
+        """Decode step i on the sampled layers; returns the wall seconds of each sampled layer."""
+        B, ts = self.B, []
         for layer in self.layers:
             k, v, q, tags = step_inputs(self.w, layer, i, "cpu")
             kb, vb, qb = bf16_bits(k[:B]).numpy(), bf16_bits(v[:B]).numpy(), bf16_bits(q[:B]).numpy()
             t0 = time.perf_counter()
             self.cache.append(layer, list(range(B)), np.arange(B + 1, dtype=np.int32), kb, vb, tags[:B])
             self.cache.attention_batch(layer, list(range(B)), qb)
-            t += time.perf_counter() - t0
+            ts.append(time.perf_counter() - t0)
+        return ts
+
+    def full_step_seconds(self, per_layer):
+        """Seconds of a decode step over all layers for the sampled sequences: every sampled layer stands
+        for the layers of its layer group (the groups keep different shares of the tokens)."""
+        lg = self.w.policy.layer_group.astype(np.int64)
+        t = 0.0
+        for layer, sec in zip(self.layers, per_layer):
+            t += sec * int((lg == lg[layer]).sum())
         return t
 
-    def tokens_per_s(self, seconds):
-        """Decode tokens/s of the full model if every layer took as long as the sampled ones."""
-        return self.B / (seconds / len(self.layers) * self.w.cfg.n_layers)
+    def tokens_per_s(self, per_layer):
+        return self.B / self.full_step_seconds(per_layer)
 
     def describe(self, n_steps, seconds):
         cfg = self.w.cfg
-        return (f"layers {self.layers} of {cfg.n_layers} x {self.B} of {cfg.batch} sequences, {n_steps} decode steps "
-                f"(append + fp64 attention), {seconds:.1f} s wall on the host cores, scaled to {cfg.n_layers} layers")
+        return (f"layers {self.layers} (the first of each layer group) of {cfg.n_layers} x {self.B} of {cfg.batch} sequences, "
+                f"{n_steps} decode steps (append + fp64 attention), {seconds:.1f} s wall on the host cores; each sampled "
+                f"layer scaled by the {cfg.n_layers // cfg.n_groups} layers of its group")
 
 
-def cpu_baseline(w, budget_s=15.0, n_seqs=32):
-    smp = OracleSample(w, n_seqs, [0])
+def group_layers(w):
+    """The first layer of every layer group that owns layers."""
+    lg = w.policy.layer_group.astype(np.int64)
+    return [int(np.argmax(lg == g)) for g in range(w.policy.n_groups) if (lg == g).any()]
+
+
+def cpu_baseline(w, budget_s=15.0, n_seqs=64):
+    smp = OracleSample(w, n_seqs, group_layers(w))
     cores = smp.oracle.max_threads()
     smp.step(0)                                    # untimed first touch
-    wall, n = 0.0, 0
-    while n < 16 and wall < budget_s / 4:
-        wall += smp.step(1 + n)
+    acc, wall, n = np.zeros(len(smp.layers)), 0.0, 0
+    while n < 16 and wall < budget_s:
+        ts = smp.step(1 + n)
+        acc += np.asarray(ts)
+        wall += sum(ts)
         n += 1
-    return {"value": smp.tokens_per_s(wall / n), "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": smp.describe(n, wall)}
+    return {"value": smp.tokens_per_s(acc / n), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": smp.describe(n, wall), "measured_s_per_sampled_step": wall / n,
+            "extrapolated_s_per_full_step": smp.full_step_seconds(acc / n)}
 
 
 def run_reference(args, rank, world):
@@ -594,19 +729,27 @@ def run_reference(args, rank, world):
     cfg = CONFIGS[args.config]
     cfg = WC.scaled(cfg, extra_gen=max(cfg.extra_gen, args.warmup + args.steps + 8))
     w = WC.build(cfg)
-    smp = OracleSample(w, args.ref_seqs, [0])
+    smp = OracleSample(w, args.ref_seqs, group_layers(w))
     if world > 1:      # the launcher pins every rank to one OpenMP thread; rank 0 runs alone and takes the host's cores
         smp.oracle.set_threads(os.cpu_count() or 1)
     for i in range(args.warmup):
         smp.step(i)
-    t = sum(smp.step(args.warmup + i) for i in range(args.steps))
-    value = smp.tokens_per_s(t / args.steps)
+    acc = np.zeros(len(smp.layers))
+    for i in range(args.steps):
+        acc += np.asarray(smp.step(args.warmup + i))
+    wall = float(acc.sum())
+    value = smp.tokens_per_s(acc / args.steps)
     base = {"value": value, "unit": UNIT, "cores": smp.oracle.max_threads(), "kind": "oracle",
-            "sample": smp.describe(args.steps, t)}
+            "sample": smp.describe(args.steps, wall), "measured_s_per_sampled_step": wall / args.steps,
+            "extrapolated_s_per_full_step": smp.full_step_seconds(acc / args.steps)}
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": 1e3 * cfg.batch / value, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": 1e3 * smp.full_step_seconds(acc / args.steps) * cfg.batch / smp.B,
+            "measured_ms_per_sampled_step": 1e3 * wall / args.steps,
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "kv_budget_target": cfg.budget},
+            "config": {"workload": cfg.name, "kv_budget_target": cfg.budget,
+                       "note": "ms_per_step is extrapolated from the sampled layers to all layers; "
+                               "measured_ms_per_sampled_step is the wall time actually spent per step"},
             "cpu_baseline": base,
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -632,7 +775,11 @@ def main():
     ap.add_argument("--dynamic", action="store_true",
                     help="decide every token against the running budget (pask_decide) instead of the frozen table alone")
     ap.add_argument("--layers", type=int, default=None, help="profiling aid: keep only the first N layers")
-    ap.add_argument("--ref-seqs", type=int, default=32, help="sequences in the oracle's timed sample")
+    ap.add_argument("--ref-seqs", type=int, default=64, help="sequences in the oracle's timed sample")
+    ap.add_argument("--repeats", type=int, default=5, help="timed blocks of --steps steps each; value = their median")
+    ap.add_argument("--seeds", type=int, default=3, help="N = 1: also run the configuration from the next seeds (1 = only the first)")
+    ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
+                    help="N = 1: skip the further configurations (budget sweep, batch-128 16K, latency-table shapes, ...)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     rank = int(os.environ.get("RANK", 0))

@@ -61,6 +61,7 @@ typedef int32_t pask_status_t;
 #define PASK_ERR_TIMEOUT (-7)
 #define PASK_ERR_WORKSPACE (-8)
 #define PASK_ERR_NO_MEMORY (-9)   /* host memory for a handle or a staging copy could not be had */
+#define PASK_ERR_STALE_PLAN (-10) /* pask_decode_step_ahead without a valid plan for this layer and batch */
 
 /* Sticky bits of the device status word (pask_budget_state_t.device_status). */
 #define PASK_DEV_POOL_EXHAUSTED 0x1u  /* an append needed more pages than a pool had: nothing written */
@@ -74,6 +75,7 @@ typedef int32_t pask_status_t;
 
 #define PASK_DEV_INTERNAL 0x40u       /* an internal bounds check refused an access (a page id out of range) */
 #define PASK_DEV_BAD_ACTION 0x80u     /* pask_append_kv_decided was given an action outside R, L, H; call refused */
+#define PASK_DEV_STALE_PLAN 0x100u    /* pask_decode_step_ahead: the sequences named are not those the plan was made for */
 
 #define PASK_ACTION_RELEASE 0
 #define PASK_ACTION_RETAIN_LOW 1
@@ -285,6 +287,47 @@ pask_status_t pask_append_attend(pask_cache_t *cache, int32_t layer, int32_t n_s
                                  const uint8_t *tags, const uint8_t *actions, uint8_t *actions_out, const void *q,
                                  float *out, float *lse, void *workspace, size_t workspace_bytes,
                                  pask_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Planned-ahead decode steps: the append taken off the layer's critical path.
+ *
+ * In a decode loop the same batch comes back step after step, and what the attention of step t+1
+ * streams at a layer is known as soon as step t has appended there.  pask_decode_step_ahead uses
+ * that: the streaming kernel of a call starts at once from a work plan that describes the cache
+ * BEFORE this call's append (written by the call of the step before, or by pask_plan_ahead); the
+ * append of the new tokens (Algorithm 2 step 7) runs in the shadow of the streaming kernel's tail
+ * and writes the plan of the next step; the merge kernel attends each new token straight from the
+ * call's k / v -- at its stored precision: as given when its action is RETAIN-HIGH, quantised on
+ * the fly exactly as the append quantises it when RETAIN-LOW, not at all when released -- and adds
+ * that one partial to those of the history.  Cache state after the call is bit-identical to
+ * pask_append_attend's; out / lse are the same attention (Section 3.1) summed in another order.
+ *
+ *   plan_area   dev, >= pask_plan_area_bytes(cache, n_seqs), 256-byte aligned, owned by the caller
+ *               and left alone by it from pask_plan_ahead on: it holds, per layer, two plans used in
+ *               turn.  One area serves one batch (a fixed list of sequences in a fixed order).
+ *   pask_plan_ahead(layer)      writes the layer's plan from the cache as it stands.  Call it for
+ *               every layer once the batch is formed (after prefill) and again after anything else
+ *               touched the cache at that layer: pask_append_kv*, pask_append_attend,
+ *               pask_decode_step_*, pask_seq_reset, pask_cache_reset.  The handle remembers which
+ *               layers have a plan; those calls forget it.
+ *   pask_decode_step_ahead(layer)   exactly one new token per sequence: k, v [n_seqs][n_kv][128],
+ *               tags [n_seqs], actions NULL or [n_seqs][n_groups] (from pask_decide), q, out, lse,
+ *               workspace as for pask_append_attend.  seq_ids must be the list the plan was made for.
+ * Errors: PASK_ERR_STALE_PLAN if the handle holds no plan of this layer for n_seqs sequences in
+ * this plan_area (nothing is enqueued); a different list of the same length is only seen on the
+ * device: sticky PASK_DEV_STALE_PLAN, results void.  PASK_ERR_UNSUPPORTED_SHAPE with a protected
+ * recent window (the token that leaves the window changes what the history holds) or more than
+ * 255 sequences: use pask_append_attend there.  A refused append (sticky PASK_DEV_* bit) leaves
+ * out / lse undefined and an empty plan behind.  k, v, tags, actions, q must stay untouched
+ * until the call's kernels have run, as for every call. */
+size_t pask_plan_area_bytes(const pask_cache_t *cache, int32_t n_seqs);
+pask_status_t pask_plan_ahead(pask_cache_t *cache, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                              void *plan_area, size_t plan_area_bytes, pask_stream_t stream);
+pask_status_t pask_decode_step_ahead(pask_cache_t *cache, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                     const void *k, const void *v, const uint8_t *tags, const uint8_t *actions,
+                                     uint8_t *actions_out, const void *q, float *out, float *lse,
+                                     void *workspace, size_t workspace_bytes, void *plan_area,
+                                     size_t plan_area_bytes, pask_stream_t stream);
 
 /* The full high-precision reference (the paper's "Full KV", C_KV = 1): same arguments, for a
  * cache whose policy keeps everything at high precision; the LOW stream is not read at all

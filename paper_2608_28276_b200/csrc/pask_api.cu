@@ -105,6 +105,7 @@ const char *pask_status_string(pask_status_t s) {
         case PASK_ERR_TIMEOUT: return "device wait timed out";
         case PASK_ERR_WORKSPACE: return "workspace too small";
         case PASK_ERR_NO_MEMORY: return "out of host memory";
+        case PASK_ERR_STALE_PLAN: return "no valid plan made ahead for this layer and batch";
         default: return "unknown status";
     }
 }
@@ -208,6 +209,7 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     c->meta = meta;
     c->sm_count = sms;
     c->ev_start = c->ev_stop = nullptr;
+    c->ahead.resize((size_t)d->n_layers);
     c->wait_cycles = 2000000000LL;   // about one second: give up instead of hanging
     c->wait_test_surplus = 0;
     c->off = meta_offsets(d, 255, PASK_MAX_GROUPS);
@@ -323,6 +325,7 @@ pask_status_t pask_cache_reset(pask_cache_t *c, pask_stream_t stream_v) {
     if (!c) return PASK_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     uint8_t *m = static_cast<uint8_t *>(c->meta);
+    for (auto &a : c->ahead) a.valid = false;
     cudaError_t e = cudaMemsetAsync(m + c->off.ctrl, 0, kCtrlWords * 4, stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m + c->off.zero_begin, 0, c->off.zero_end - c->off.zero_begin, stream);
     return cuda_rc(e);
@@ -331,6 +334,7 @@ pask_status_t pask_cache_reset(pask_cache_t *c, pask_stream_t stream_v) {
 pask_status_t pask_seq_reset(pask_cache_t *c, int32_t seq, pask_stream_t stream) {
     if (!c) return PASK_ERR_INVALID_ARG;
     if (seq < 0 || seq >= c->desc.max_seqs) return PASK_ERR_BAD_SEQ;
+    for (auto &a : c->ahead) a.valid = false;
     return launch_seq_reset(c, seq, static_cast<cudaStream_t>(stream));
 }
 
@@ -346,6 +350,7 @@ static pask_status_t append_common(pask_cache_t *c, int32_t layer, int32_t n_seq
     if (((uintptr_t)k | (uintptr_t)v) & 15) return PASK_ERR_INVALID_ARG;
     if (((uintptr_t)seq_ids | (uintptr_t)cu_tokens) & 3) return PASK_ERR_INVALID_ARG;
     NvtxRange range("pask_append_kv");
+    c->ahead[layer].valid = false;       // a plan made ahead for this layer no longer describes it
     return launch_append(c, layer, n_seqs, total_tokens, seq_ids, cu_tokens, k, v, tags, decided, actions_out,
                          static_cast<cudaStream_t>(stream), fuse_ws, fused);
 }
@@ -422,6 +427,57 @@ pask_status_t pask_decode_attention_full(pask_cache_t *c, int32_t layer, int32_t
 size_t pask_workspace_bytes(const pask_cache_t *c, int32_t n_seqs) {
     if (!c || n_seqs < 1) return 0;
     return attention_workspace_bytes(c, n_seqs);
+}
+
+size_t pask_plan_area_bytes(const pask_cache_t *c, int32_t n_seqs) {
+    if (!c || n_seqs < 1 || n_seqs > 255) return 0;
+    return carve_plan_area(c, n_seqs, 0, 0, nullptr, nullptr);
+}
+
+static pask_status_t ahead_args_ok(pask_cache_t *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids, void *area,
+                                   size_t area_bytes) {
+    if (!c || !seq_ids || !area) return PASK_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->desc.n_layers || n_seqs < 1 || n_seqs > c->desc.max_seqs) return PASK_ERR_INVALID_ARG;
+    if (n_seqs > 255 || c->dev.window) return PASK_ERR_UNSUPPORTED_SHAPE;
+    if (((uintptr_t)seq_ids & 3) || ((uintptr_t)area & 255)) return PASK_ERR_INVALID_ARG;
+    if (area_bytes < pask_plan_area_bytes(c, n_seqs)) return PASK_ERR_WORKSPACE;
+    return PASK_OK;
+}
+
+pask_status_t pask_plan_ahead(pask_cache_t *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids, void *area,
+                              size_t area_bytes, pask_stream_t stream) {
+    const pask_status_t ok = ahead_args_ok(c, layer, n_seqs, seq_ids, area, area_bytes);
+    if (ok != PASK_OK) return ok;
+    NvtxRange range("pask_plan_ahead");
+    auto &a = c->ahead[layer];
+    a.valid = false;
+    const pask_status_t rc = launch_plan_ahead(c, layer, n_seqs, seq_ids, area, 0, static_cast<cudaStream_t>(stream));
+    if (rc != PASK_OK) return rc;
+    a.valid = true;
+    a.n_seqs = n_seqs;
+    a.parity = 0;
+    a.area = area;
+    return PASK_OK;
+}
+
+pask_status_t pask_decode_step_ahead(pask_cache_t *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids, const void *k,
+                                     const void *v, const uint8_t *tags, const uint8_t *actions, uint8_t *actions_out,
+                                     const void *q, float *out, float *lse, void *ws, size_t ws_bytes, void *area,
+                                     size_t area_bytes, pask_stream_t stream) {
+    pask_status_t rc = ahead_args_ok(c, layer, n_seqs, seq_ids, area, area_bytes);
+    if (rc != PASK_OK) return rc;
+    if (!k || !v || !tags) return PASK_ERR_INVALID_ARG;
+    if (((uintptr_t)k | (uintptr_t)v) & 15) return PASK_ERR_INVALID_ARG;
+    rc = attention_common(c, true, layer, n_seqs, seq_ids, q, out, lse, ws, ws_bytes, stream, false, true);
+    if (rc != PASK_OK) return rc;
+    auto &a = c->ahead[layer];
+    if (!a.valid || a.n_seqs != n_seqs || a.area != area) return PASK_ERR_STALE_PLAN;
+    NvtxRange range("pask_decode_step_ahead");
+    rc = launch_step_ahead(c, layer, n_seqs, seq_ids, k, v, tags, actions, actions_out, q, out, lse, ws, area, a.parity,
+                           static_cast<cudaStream_t>(stream));
+    if (rc != PASK_OK) { a.valid = false; return rc; }
+    a.parity ^= 1;                      // the append has left the next step's plan in the other block
+    return PASK_OK;
 }
 
 size_t pask_step_staging_bytes(const pask_cache_t *c, int32_t n_seqs) {

@@ -704,13 +704,14 @@ __device__ __forceinline__ bool page_at_rcp(uint32_t v, uint32_t nh, uint32_t n,
 // counter, nobody waits) commits the counters, tables and budget states for everybody.
 constexpr int kSmallMax = 255;       // at most this many sequences and tokens (one thread each, index n_seqs included)
 constexpr int kSmallThreads = 256;
-struct SmallLut { uint8_t action[256]; };
 
-__global__ void __launch_bounds__(kSmallThreads)
-append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, const int32_t *__restrict__ seq_ids,
-                    const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
-                    const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided,
-                    uint8_t *__restrict__ actions_out, const SmallLut lut, const int fuse_plan, const Workspace ws) {
+// (the kernel proper is the wrapper below: it places the dependency wait before or after this body)
+__device__ __forceinline__ void
+append_small_body(const DevCache &c, int layer, int group, int n_seqs, int total, const int32_t *__restrict__ seq_ids,
+                  const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
+                  const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided,
+                  uint8_t *__restrict__ actions_out, const SmallLut &lut, const int fuse_plan, const Workspace &ws,
+                  int32_t *__restrict__ ids_out) {
     __shared__ int s_seq[kSmallMax], s_cu[kSmallMax + 1];
     __shared__ uint32_t s_cost[kSmallMax + 1], s_page[kSmallMax + 1], s_nh[kSmallMax], s_nl[kSmallMax];   // fused attention plan
     __shared__ uint32_t s_old_n[kSmallMax], s_nw[kSmallMax], s_wstart[kSmallMax], s_wlen[kSmallMax];
@@ -720,8 +721,6 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     __shared__ uint32_t s_pos[kSmallMax], s_ctrl[4], s_err, s_scan3[kSmallThreads / 32][3];
     __shared__ int s_last;
     const int tid = threadIdx.x;
-    pdl_launch_dependents();
-    pdl_wait();
     // this CTA's token and this thread's chunk of it: fetch the data first, it depends on nothing
     const int my_tok = blockIdx.x;
     const int chunks = 16 * c.n_kv;
@@ -936,6 +935,7 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
         if (blockIdx.x == 0) {
             if (tid <= n_seqs) { ws.cost_prefix[tid] = s_cost[tid]; ws.page_prefix[tid] = s_page[tid]; }
             if (tid < n_seqs) ws.tokens[tid] = make_uint2(s_nh[tid], s_nl[tid]);
+            if (ids_out && tid < n_seqs) ids_out[tid] = s_seq[tid];     // whom the plan is for
         }
         // the page-order list, a sequence at a time (CTA b takes sequences b, b + grid, ...): up to four entries per
         // thread and round, the page-table (or free-stack) reads of a round all in flight together
@@ -1067,6 +1067,25 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
     }
 }
 
+// Normally the kernel waits for its predecessor in the stream before it reads anything.  With late_wait it does not:
+// it is then launched behind a kernel that needs none of its results and touches nothing it writes (the decode-
+// attention kernel of the same layer, working from a plan of the cache before this append), runs in the shadow of
+// that kernel's tail, and waits for it only before it retires, so that whoever comes next in the stream and waits
+// for this kernel has waited for both.  (Everything before that predecessor is complete: it has done its own wait
+// before it let this kernel start.)
+__global__ void __launch_bounds__(kSmallThreads)
+append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, const int32_t *__restrict__ seq_ids,
+                    const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
+                    const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided,
+                    uint8_t *__restrict__ actions_out, const SmallLut lut, const int fuse_plan, const Workspace ws,
+                    int32_t *__restrict__ ids_out, const int late_wait) {
+    pdl_launch_dependents();
+    if (!late_wait) pdl_wait();
+    append_small_body(c, layer, group, n_seqs, total, seq_ids, cu_tokens, k, v, tags, decided, actions_out, lut, fuse_plan, ws,
+                      ids_out);
+    if (late_wait) pdl_wait();
+}
+
 // General path, recent window: CTA (j, y) copies the y-th newest of sequence j's tokens in this call
 // (released ones too) into the sequence's ring as bf16 and records its action; only the last W
 // tokens of a sequence can still be in the window afterwards, and they have distinct slots.
@@ -1126,15 +1145,14 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
     if (n_seqs <= kSmallMax && total_tokens <= kSmallMax) {
         SmallLut lut;
         const int group = c->layer_group[layer];
-        for (int z = 0; z < 256; z++)
-            lut.action[z] = z < c->dev.n_tags ? c->lut[(size_t)z * c->dev.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
+        fill_small_lut(c, layer, &lut);
         if (total_tokens == 0) return PASK_OK;
         const int fuse = fuse_ws != nullptr;
         if (fused) *fused = fuse != 0;
         const cudaError_t e = launch_pdl(append_small_kernel, dim3(total_tokens), dim3(kSmallThreads), 0, stream, c->dev, layer,
                                          group, n_seqs, total_tokens, seq_ids, cu_tokens, static_cast<const uint4 *>(k),
                                          static_cast<const uint4 *>(v), tags, decided, actions_out, lut, fuse,
-                                         fuse ? *fuse_ws : Workspace{});
+                                         fuse ? *fuse_ws : Workspace{}, (int32_t *)nullptr, 0);
         return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
     }
     append_plan_kernel<<<n_seqs, kPlanThreads, 0, stream>>>(c->dev, layer, n_seqs, total_tokens, seq_ids, cu_tokens, tags,
@@ -1153,6 +1171,24 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
         append_window_kernel<<<dim3(n_seqs, c->dev.window), 256, 0, stream>>>(c->dev, layer, static_cast<const uint4 *>(k),
                                                         static_cast<const uint4 *>(v), tags, decided);
     return cudaGetLastError() == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
+}
+
+void fill_small_lut(const pask_cache *c, int layer, SmallLut *lut) {
+    const int group = c->layer_group[layer];
+    for (int z = 0; z < 256; z++)
+        lut->action[z] = z < c->dev.n_tags ? c->lut[(size_t)z * c->dev.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
+}
+
+pask_status_t launch_append_beside(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,
+                                   const void *k, const void *v, const uint8_t *tags, const uint8_t *decided,
+                                   uint8_t *actions_out, const Workspace &plan_ws, int32_t *ids_out, cudaStream_t stream) {
+    if (n_seqs < 1 || n_seqs > kSmallMax) return PASK_ERR_UNSUPPORTED_SHAPE;
+    SmallLut lut;
+    fill_small_lut(c, layer, &lut);
+    const cudaError_t e = launch_pdl(append_small_kernel, dim3(n_seqs), dim3(kSmallThreads), 0, stream, c->dev, layer,
+                                     (int)c->layer_group[layer], n_seqs, n_seqs, seq_ids, cu_tokens, static_cast<const uint4 *>(k),
+                                     static_cast<const uint4 *>(v), tags, decided, actions_out, lut, 1, plan_ws, ids_out, 1);
+    return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }
 
 pask_status_t launch_seq_reset(pask_cache *c, int seq, cudaStream_t stream) {

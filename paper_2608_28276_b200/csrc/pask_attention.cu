@@ -928,6 +928,131 @@ combine_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ p
     if (lse && lane == 0) lse[orow] = L > 0.f ? (M + log2f(L)) * 0.69314718055994530942f : -INFINITY;
 }
 
+// What the merge kernel of a planned-ahead step needs to attend each sequence's new token from the call's inputs.
+struct NewTokens {
+    const uint2 *k, *v;            // bf16 [n_seqs][n_kv][128] viewed as 8-byte pieces (4 dims)
+    const uint2 *q;                // bf16 [n_seqs][n_q][128]
+    const uint8_t *tags;           // [n_seqs]
+    const uint8_t *decided;        // [n_seqs][n_groups] or null
+    const int32_t *seq_ids, *planned_ids;   // this call's list and the one the plan was made for
+    uint32_t *status;
+    int group, n_groups, n_kv, low_bits;
+};
+
+// Partial (m, l = 1, o = v) of one new token for one query head: the token at the precision it is stored at.
+// lane = 4 consecutive head dims; a 32-dim group is 8 adjacent lanes.
+__device__ __forceinline__ void quantise_like_append(float (&x)[4], int low_bits) {
+    float amax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
+    const float qmax = low_bits == 8 ? 127.0f : low_bits == 2 ? 1.0f : 7.0f;
+    __half sh = __float2half_rn(low_bits == 2 ? amax : __fdiv_rn(amax, qmax));
+    if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);
+    const float s = __half2float(sh);
+    const float inv = s == 0.0f ? 0.0f : __fdiv_rn(1.0f, s);
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        float r = rintf(__fmul_rn(x[i], inv));
+        r = fminf(fmaxf(r, -qmax), qmax);
+        x[i] = __fmul_rn(r, s);          // (code - zero) * scale, exact
+    }
+}
+
+// Merge kernel of a planned-ahead step: the partials of the history (streamed from the plan of the cache before
+// this call's append) and, as one more partial, the sequence's new token taken from the call's k / v.
+__global__ void __launch_bounds__(256)
+combine_new_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ part_ml, const float *__restrict__ part_o,
+                   float *__restrict__ out, float *__restrict__ lse, int n_seqs, int n_q, uint32_t n_ctas, const NewTokens nt,
+                   const SmallLut lut) {
+    const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    const int s = wid / n_q, h = wid % n_q;
+    const bool mine = wid < n_seqs * n_q;
+    // everything that does not come from the kernels before is fetched ahead of the dependency wait
+    uint32_t p0 = 0, p1 = 0;
+    uint64_t total = 0;
+    int act = PASK_ACTION_RELEASE;
+    float kx[4] = {0.f, 0.f, 0.f, 0.f}, vx[4] = {0.f, 0.f, 0.f, 0.f}, qx[4] = {0.f, 0.f, 0.f, 0.f};
+    bool stale = false;
+    if (mine) {
+        p0 = __ldg(prefix + s); p1 = __ldg(prefix + s + 1); total = __ldg(prefix + n_seqs);
+        act = nt.decided ? nt.decided[(size_t)s * nt.n_groups + nt.group] : lut.action[nt.tags[s]];
+        if (act > PASK_ACTION_RETAIN_HIGH) act = PASK_ACTION_RELEASE;      // (the append refuses the call)
+        stale = nt.seq_ids[s] != nt.planned_ids[s];
+        if (act != PASK_ACTION_RELEASE) {
+            const int kv = h / (n_q / nt.n_kv);
+            const uint2 kw = nt.k[((size_t)s * nt.n_kv + kv) * 32 + lane], vw = nt.v[((size_t)s * nt.n_kv + kv) * 32 + lane];
+            const uint2 qw = nt.q[((size_t)s * n_q + h) * 32 + lane];
+            kx[0] = bf_lo(kw.x); kx[1] = bf_hi(kw.x); kx[2] = bf_lo(kw.y); kx[3] = bf_hi(kw.y);
+            vx[0] = bf_lo(vw.x); vx[1] = bf_hi(vw.x); vx[2] = bf_lo(vw.y); vx[3] = bf_hi(vw.y);
+            qx[0] = bf_lo(qw.x); qx[1] = bf_hi(qw.x); qx[2] = bf_lo(qw.y); qx[3] = bf_hi(qw.y);
+        }
+    }
+    float m_new = -INFINITY;
+    if (act == PASK_ACTION_RETAIN_LOW) { quantise_like_append(kx, nt.low_bits); quantise_like_append(vx, nt.low_bits); }
+    if (act != PASK_ACTION_RELEASE) {       // (warp-uniform: one sequence and head per warp)
+        float dot = fmaf(qx[0], kx[0], fmaf(qx[1], kx[1], fmaf(qx[2], kx[2], qx[3] * kx[3])));
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, d);
+        m_new = dot * (0.088388347648318440550f * 1.4426950408889634074f);      // log2 units, as the partials
+    }
+    if (stale && lane == 0 && h == 0) atomicOr(nt.status, PASK_DEV_STALE_PLAN);
+    pdl_wait();
+    if (!mine) return;
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    float M = -INFINITY, L = 0.f;
+    if (p1 > p0) {
+        const uint32_t b_first = (uint32_t)((((uint64_t)p0 + 1) * n_ctas - 1) / total);
+        const uint32_t b_last = (uint32_t)(((uint64_t)p1 * n_ctas - 1) / total);
+        for (uint32_t b = b_first; b <= b_last; b += 8) {
+            float2 ml[8];
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; u++) {
+                const bool have = b + u <= b_last;
+                const size_t row = ((size_t)b + u + s) * n_q + h;
+                ml[u] = have ? part_ml[row] : make_float2(-INFINITY, 0.f);
+                v[u] = have ? *reinterpret_cast<const float4 *>(part_o + row * kHeadDim + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; u++) {
+                if (ml[u].x == -INFINITY) continue;
+                const float Mn = fmaxf(M, ml[u].x);
+                const float fo = exp2f(M - Mn), fn = exp2f(ml[u].x - Mn);
+                o.x = fmaf(fn, v[u].x, o.x * fo); o.y = fmaf(fn, v[u].y, o.y * fo);
+                o.z = fmaf(fn, v[u].z, o.z * fo); o.w = fmaf(fn, v[u].w, o.w * fo);
+                L = fmaf(fn, ml[u].y, L * fo);
+                M = Mn;
+            }
+        }
+    }
+    if (m_new != -INFINITY) {                // the new token: weight 1 at its own score
+        const float Mn = fmaxf(M, m_new);
+        const float fo = exp2f(M - Mn), fn = exp2f(m_new - Mn);
+        o.x = fmaf(fn, vx[0], o.x * fo); o.y = fmaf(fn, vx[1], o.y * fo);
+        o.z = fmaf(fn, vx[2], o.z * fo); o.w = fmaf(fn, vx[3], o.w * fo);
+        L = fmaf(fn, 1.0f, L * fo);
+        M = Mn;
+    }
+    const size_t orow = (size_t)s * n_q + h;
+    if (L > 0.f) {
+        const float inv = 1.0f / L;
+        o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
+    }
+    *reinterpret_cast<float4 *>(out + orow * kHeadDim + lane * 4) = o;
+    if (lse && lane == 0) lse[orow] = L > 0.f ? (M + log2f(L)) * 0.69314718055994530942f : -INFINITY;
+}
+
+// cu_tokens of a call with one token per sequence, and the list of sequences a stand-alone plan is for
+__global__ void ahead_setup_kernel(int32_t *iota, int n_iota, int32_t *ids_out, const int32_t *__restrict__ seq_ids, int n_seqs) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n_iota) iota[i] = i;
+    if (i < n_seqs) ids_out[i] = seq_ids[i];
+}
+
 size_t attn_smem_bytes(int n_seqs, int n_warps) {
     size_t off = align_up((size_t)(2 * n_seqs + 2) * 4, 128) + 384;
     off = align_up(off, 1024);
@@ -962,41 +1087,47 @@ int attention_grid(const pask_cache *c) { return 2 * c->sm_count; }
 
 size_t attention_workspace_bytes(const pask_cache *c, int n_seqs) { return carve_workspace(c, n_seqs, nullptr, nullptr); }
 
-pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seqs, const int32_t *seq_ids, const void *q,
-                               float *out, float *lse, void *workspace, size_t, cudaStream_t stream, bool plan_done) {
+// The streaming kernel of one call: grid, shared memory, optional timing events around it.
+static cudaError_t launch_stream_kernel(pask_cache *c, bool has_low, AttnParams &p, cudaStream_t stream) {
     const int n_warps = c->desc.n_kv_heads;
-    AttnParams p;
     p.c = c->dev;
-    p.layer = layer;
-    p.n_seqs = n_seqs;
-    p.seq_ids = seq_ids;
-    p.q = static_cast<const uint4 *>(q);
-    carve_workspace(c, n_seqs, static_cast<uint8_t *>(workspace), &p.ws);
     p.wait_cycles = c->wait_cycles;
     p.overpost = c->wait_test_surplus;
-    const size_t smem = attn_smem_bytes(n_seqs, n_warps);
+    const size_t smem = attn_smem_bytes(p.n_seqs, n_warps);
     auto kern = !has_low ? decode_attn_kernel<0> : c->dev.low_bits == 8 ? decode_attn_kernel<8>
               : c->dev.low_bits == 2 ? decode_attn_kernel<2> : decode_attn_kernel<4>;
     // The shared-memory opt-in is a property of (device, kernel): ask for it once, and again only for a larger size.
     {
         static size_t granted[64][4] = {};
         int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return PASK_ERR_CUDA;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
         size_t &have = granted[dev][!has_low ? 0 : c->dev.low_bits == 8 ? 1 : c->dev.low_bits == 2 ? 2 : 3];
         if (smem > have) {
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-                return PASK_ERR_CUDA;
+            const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
             have = smem;
         }
     }
+    if (c->ev_start) cudaEventRecord(c->ev_start, stream);
+    const cudaError_t e = launch_pdl(kern, dim3(c->attn_ctas), dim3(32 * n_warps), smem, stream, p);
+    if (c->ev_stop) cudaEventRecord(c->ev_stop, stream);
+    c->ev_start = c->ev_stop = nullptr;
+    return e;
+}
+
+pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seqs, const int32_t *seq_ids, const void *q,
+                               float *out, float *lse, void *workspace, size_t, cudaStream_t stream, bool plan_done) {
+    AttnParams p;
+    p.layer = layer;
+    p.n_seqs = n_seqs;
+    p.seq_ids = seq_ids;
+    p.q = static_cast<const uint4 *>(q);
+    carve_workspace(c, n_seqs, static_cast<uint8_t *>(workspace), &p.ws);
     cudaError_t e = cudaSuccess;
     if (!plan_done)   // (a fused append has already left the plan in the workspace)
         e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(5 * n_seqs + 2) * 4, stream, c->dev,
                        layer, n_seqs, seq_ids, p.ws, has_low ? 1 : 0);
-    if (c->ev_start) cudaEventRecord(c->ev_start, stream);
-    if (e == cudaSuccess) e = launch_pdl(kern, dim3(c->attn_ctas), dim3(32 * n_warps), smem, stream, p);
-    if (c->ev_stop) cudaEventRecord(c->ev_stop, stream);
-    c->ev_start = c->ev_stop = nullptr;
+    if (e == cudaSuccess) e = launch_stream_kernel(c, has_low, p, stream);
     const int warps = n_seqs * c->desc.n_q_heads;
     if (e == cudaSuccess)
         e = launch_pdl(combine_kernel, dim3((warps + 7) / 8), dim3(256), 0, stream, (const uint32_t *)p.ws.cost_prefix,
@@ -1005,7 +1136,98 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
     return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------- planned-ahead decode steps
+
+// Plan area of a batch of n_seqs sequences: cu_tokens = 0, 1, ..., 255 for the one-token-per-sequence append, then per
+// layer two plan blocks (ids, cost prefix, page prefix, token counts, page-order list), used in turn.
+size_t carve_plan_area(const pask_cache *c, int n_seqs, int layer, int parity, uint8_t *base, PlanBlock *pb) {
+    const size_t max_pages = (size_t)n_seqs * (2 * c->dev.max_pages + c->dev.window / kPageTokens);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
+    take(257 * 4);                                         // cu_tokens
+    const size_t head = off;
+    const size_t o_ids = take((size_t)n_seqs * 4), o_cost = take((size_t)(n_seqs + 1) * 4), o_page = take((size_t)(n_seqs + 1) * 4);
+    const size_t o_tok = take((size_t)n_seqs * sizeof(uint2)), o_order = take(max_pages * 4);
+    const size_t block = off - head;
+    if (pb) {
+        uint8_t *b = base + (size_t)(2 * layer + parity) * block;
+        pb->ids = reinterpret_cast<int32_t *>(b + o_ids);
+        pb->cost_prefix = reinterpret_cast<uint32_t *>(b + o_cost);
+        pb->page_prefix = reinterpret_cast<uint32_t *>(b + o_page);
+        pb->tokens = reinterpret_cast<uint2 *>(b + o_tok);
+        pb->order = reinterpret_cast<uint32_t *>(b + o_order);
+    }
+    return head + (size_t)2 * c->desc.n_layers * block;
+}
+
+static Workspace plan_view(const PlanBlock &pb, const Workspace &parts) {
+    Workspace w = parts;
+    w.cost_prefix = pb.cost_prefix;
+    w.page_prefix = pb.page_prefix;
+    w.tokens = pb.tokens;
+    w.order = pb.order;
+    return w;
+}
+
+pask_status_t launch_plan_ahead(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, void *area, int parity,
+                                cudaStream_t stream) {
+    PlanBlock pb;
+    carve_plan_area(c, n_seqs, layer, parity, static_cast<uint8_t *>(area), &pb);
+    cudaError_t e = launch_pdl(ahead_setup_kernel, dim3(2), dim3(256), 0, stream, static_cast<int32_t *>(area), 257, pb.ids,
+                               seq_ids, n_seqs);
+    if (e == cudaSuccess)
+        e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(5 * n_seqs + 2) * 4, stream, c->dev,
+                       layer, n_seqs, seq_ids, plan_view(pb, Workspace{}), 1);
+    return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
+}
+
+// One layer of a planned-ahead decode step.  In stream order: the streaming kernel over the plan of the cache as
+// it was before this call; the one-launch append, which does not wait for that kernel (it needs nothing from it
+// and writes nothing it reads: slots past the planned token counts, table entries and counters the plan has
+// replaced, the other plan block) and so runs as its CTAs retire; the merge kernel, which waits for both.
+pask_status_t launch_step_ahead(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const void *k, const void *v,
+                                const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out, const void *q, float *out,
+                                float *lse, void *workspace, void *area, int cur, cudaStream_t stream) {
+    PlanBlock pc, pn;
+    carve_plan_area(c, n_seqs, layer, cur, static_cast<uint8_t *>(area), &pc);
+    carve_plan_area(c, n_seqs, layer, cur ^ 1, static_cast<uint8_t *>(area), &pn);
+    AttnParams p;
+    p.layer = layer;
+    p.n_seqs = n_seqs;
+    p.seq_ids = seq_ids;
+    p.q = static_cast<const uint4 *>(q);
+    Workspace parts;
+    carve_workspace(c, n_seqs, static_cast<uint8_t *>(workspace), &parts);
+    p.ws = plan_view(pc, parts);
+    cudaError_t e = launch_stream_kernel(c, true, p, stream);
+    if (e != cudaSuccess) return PASK_ERR_CUDA;
+    const pask_status_t rc = launch_append_beside(c, layer, n_seqs, seq_ids, static_cast<const int32_t *>(area), k, v, tags, decided,
+                                                  actions_out, plan_view(pn, Workspace{}), pn.ids, stream);
+    if (rc != PASK_OK) return rc;
+    NewTokens nt;
+    nt.k = static_cast<const uint2 *>(k);
+    nt.v = static_cast<const uint2 *>(v);
+    nt.q = static_cast<const uint2 *>(q);
+    nt.tags = tags;
+    nt.decided = decided;
+    nt.seq_ids = seq_ids;
+    nt.planned_ids = pc.ids;
+    nt.status = c->dev.ctrl + kCtrlStatus;
+    nt.group = c->layer_group[layer];
+    nt.n_groups = c->dev.n_groups;
+    nt.n_kv = c->desc.n_kv_heads;
+    nt.low_bits = (int)c->dev.low_bits;
+    SmallLut lut;
+    fill_small_lut(c, layer, &lut);
+    const int warps = n_seqs * c->desc.n_q_heads;
+    e = launch_pdl(combine_new_kernel, dim3((warps + 7) / 8), dim3(256), 0, stream, (const uint32_t *)pc.cost_prefix,
+                   (const float2 *)parts.part_ml, (const float *)parts.part_o, out, lse, n_seqs, (int)c->desc.n_q_heads,
+                   (uint32_t)c->attn_ctas, nt, lut);
+    return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
+}
+
 }  // namespace pask
+
 
 // ---------------------------------------------------------------- decode attention without a caller workspace
 //

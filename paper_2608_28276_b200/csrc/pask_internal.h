@@ -99,6 +99,15 @@ struct Workspace {
     float *part_o;          // [slots][n_q][128] unnormalised outputs
 };
 
+// One layer's work plan of a planned-ahead decode step, inside the caller's plan area: what Workspace holds of a
+// plan, plus the list of sequences it was made for.
+struct PlanBlock {
+    int32_t *ids;           // [n_seqs] the sequences the plan describes, in call order
+    uint32_t *cost_prefix, *page_prefix;
+    uint2 *tokens;
+    uint32_t *order;
+};
+
 struct MetaOffsets {
     size_t ctrl, free_high, free_low, n_high, n_low, tbl_high, tbl_low, budget, seq_mark, low_vmax, n_tok, win_act, plan, tok_list, item_base, lut,
         layer_group, dec_row, dec_rho, gamma, crit, total;
@@ -125,6 +134,14 @@ struct pask_cache {
     int sm_count;
     int attn_ctas;                // grid of the decode-attention main kernel
     cudaEvent_t ev_start, ev_stop;
+    // planned-ahead decode steps: which layers hold a plan, for how many sequences, in which area, and which of the
+    // layer's two plan blocks is the current one
+    struct Ahead {
+        bool valid = false;
+        int n_seqs = 0, parity = 0;
+        const void *area = nullptr;
+    };
+    std::vector<Ahead> ahead;     // [n_layers]
     long long wait_cycles;        // bound of a device-side wait for a bulk copy, in SM clock cycles (about a second)
     uint32_t wait_test_surplus;   // pask_debug_set_wait: bytes a warp's first copy announces but does not bring
     // pask_decode_step_pipelined: two copy streams and the events that order them against the caller's stream
@@ -180,6 +197,21 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
                                const void *q, float *out, float *lse, void *workspace, size_t workspace_bytes,
                                cudaStream_t stream, bool plan_done = false);
 size_t carve_workspace(const pask_cache *c, int n_seqs, uint8_t *base, Workspace *ws);
+// the plan block of (layer, parity) inside a plan area for n_seqs sequences; returns the size of the whole area
+size_t carve_plan_area(const pask_cache *c, int n_seqs, int layer, int parity, uint8_t *base, PlanBlock *pb);
+pask_status_t launch_plan_ahead(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, void *area, int parity,
+                                cudaStream_t stream);
+// streaming kernel over the plan block `cur`, then the append that writes the other block, then the merge with the new tokens
+pask_status_t launch_step_ahead(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const void *k, const void *v,
+                                const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out, const void *q, float *out,
+                                float *lse, void *workspace, void *area, int cur, cudaStream_t stream);
+// the one-launch append with its dependency wait moved to its end (it runs beside the kernel before it) and the
+// call's sequence list recorded next to the plan it writes
+pask_status_t launch_append_beside(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,
+                                   const void *k, const void *v, const uint8_t *tags, const uint8_t *decided,
+                                   uint8_t *actions_out, const Workspace &plan_ws, int32_t *ids_out, cudaStream_t stream);
+struct SmallLut { uint8_t action[256]; };
+void fill_small_lut(const pask_cache *c, int layer, SmallLut *lut);
 size_t attention_workspace_bytes(const pask_cache *c, int n_seqs);
 int attention_grid(const pask_cache *c);
 }  // namespace pask
