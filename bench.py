@@ -212,6 +212,15 @@ class Job:
         self.lse = torch.empty((self.B, cfg.n_q), dtype=torch.float32, device=device)
         self.attn = P.pask_decode_attention_full if policy_blob is not None else P.pask_decode_attention
         self.fused = False
+        self.ahead = False          # planned-ahead steps (pask_decode_step_ahead): set by plan_ahead()
+        self.area = None
+
+    def plan_ahead(self):
+        """Plan every layer's next decode step from the cache as it stands; run_step then uses pask_decode_step_ahead."""
+        self.area = torch.empty(self.P.pask_plan_area_bytes(self.cache.handle, self.B), dtype=torch.uint8, device=self.device)
+        for layer in range(self.cfg.n_layers):
+            self.P.pask_plan_ahead(self.cache.handle, layer, self.ids, self.area)
+        self.ahead = True
 
     def fill(self):
         """Append the whole history, one ragged bulk call per layer (generated on the device)."""
@@ -292,6 +301,10 @@ class Job:
         for layer, (k, v, q, tags) in enumerate(self.steps[s]):
             if events is not None and layer in events:
                 P.pask_cache_set_timing_events(h, *events[layer])
+            if self.ahead:     # streaming from the plan made a step ahead, the append beside it
+                P.pask_decode_step_ahead(h, layer, self.ids, k, v, tags, q, self.out, self.lse, self.ws, self.area,
+                                         actions=self.decided if self.dynamic else None)
+                continue
             if self.fused:     # the library's one-call form of append + attention for a layer
                 P.pask_append_attend(h, layer, self.ids, self.cu1, k, v, tags, q, self.out, self.lse, self.ws,
                                      actions=self.decided if self.dynamic else None)
@@ -389,6 +402,8 @@ def quick_point(P, runner, cfg, device, steps, peak, repeat=0, policy_blob=None,
     job.fused = policy_blob is None
     job.fill()
     job.prepare_steps(warm + steps)
+    if job.fused and job.B <= 255 and runner.args.ahead:
+        job.plan_ahead()
     t_setup = time.time() - t_setup
     for i in range(warm):
         job.run_step(i)
@@ -493,6 +508,9 @@ def run_cuda(args, rank, world):
     per_layer_launches = 3 if (job.fused and job.B <= 255) else 4
     job.fill()
     job.prepare_steps(total_steps)
+    use_ahead = args.ahead and job.fused and job.B <= 255 and not args.window
+    if use_ahead:
+        job.plan_ahead()
     t_setup = time.time() - t_setup
     ret = sum(P.pask_budget_state(job.cache.handle, b).retained_bytes for b in range(job.B))
     full = sum(P.pask_budget_state(job.cache.handle, b).full_bytes for b in range(job.B))
@@ -534,6 +552,8 @@ def run_cuda(args, rank, world):
         "config": {"workload": cfg.name, "batch_per_gpu": job.B, "layers": cfg.n_layers, "layer_groups": cfg.n_groups,
                    "kv_budget_target": cfg.budget, "kv_budget_realised": ret / full, "table": f"greedy/{cfg.bias}",
                    "recent_window": args.window,
+                   "step_call": "pask_decode_step_ahead (plan made a step ahead, append beside the streaming kernel)" if use_ahead
+                                else "pask_append_attend" if job.fused else "pask_append_kv + pask_decode_attention",
                    "tokens_in_cache_per_gpu": job.total_tokens, "page_tokens": 16,
                    "l2": "inputs larger than L2: each layer streams its own ~%.0f MB of pages" % (alg / 1e6),
                    "setup_s": round(t_setup, 1)},
@@ -770,6 +790,8 @@ def main():
     ap.add_argument("--low-bits", type=int, default=4, choices=[2, 4, 8], help="width of the RETAIN-LOW codes")
     ap.add_argument("--unfused", action="store_true",
                     help="issue pask_append_kv and pask_decode_attention separately instead of pask_append_attend")
+    ap.add_argument("--no-ahead", dest="ahead", action="store_false",
+                    help="use pask_append_attend per layer instead of the planned-ahead step (pask_decode_step_ahead)")
     ap.add_argument("--window", type=int, default=0, help="protected recent window in tokens (multiple of 16, <= 256)")
     ap.add_argument("--graph", action="store_true", help="replay each timed step as one CUDA graph (launch-bound shapes)")
     ap.add_argument("--dynamic", action="store_true",

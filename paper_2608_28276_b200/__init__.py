@@ -17,9 +17,9 @@ LIB_PATH = os.path.join(_HERE, "libpask.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_POLICY, ERR_UNSUPPORTED_SHAPE, ERR_POOL_EXHAUSTED = -1, -2, -3, -4
-ERR_BAD_SEQ, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE, ERR_NO_MEMORY = -5, -6, -7, -8, -9
+ERR_BAD_SEQ, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE, ERR_NO_MEMORY, ERR_STALE_PLAN = -5, -6, -7, -8, -9, -10
 DEV_POOL_EXHAUSTED, DEV_BAD_SEQ, DEV_SEQ_OVERFLOW, DEV_BAD_RAGGED, DEV_TIMEOUT, DEV_RANGE, DEV_INTERNAL = 1, 2, 4, 8, 16, 32, 64
-DEV_BAD_ACTION = 128
+DEV_BAD_ACTION, DEV_STALE_PLAN = 128, 256
 ACTION_RELEASE, ACTION_RETAIN_LOW, ACTION_RETAIN_HIGH = 0, 1, 2
 TAG_PROTECTED = 0xFF
 MAX_GROUPS = 8
@@ -28,7 +28,7 @@ MAX_WINDOW = 256
 EXPORTS = [
     "pask_load_policy", "pask_free_policy", "pask_policy_action", "pask_cache_sizes", "pask_cache_create",
     "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decide",
-    "pask_append_kv_decided", "pask_append_attend", "pask_decode_attention",
+    "pask_append_kv_decided", "pask_append_attend", "pask_plan_area_bytes", "pask_plan_ahead", "pask_decode_step_ahead", "pask_decode_attention",
     "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes", "pask_step_packed_layout", "pask_decode_step_packed", "pask_decode_step_pipelined", "pask_decode_step_drain",
     "pask_budget_state", "pask_distortion", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
     "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_debug_set_wait", "pask_status_string",
@@ -79,6 +79,10 @@ _lib.pask_decide.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_append_kv_decided.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_append_attend.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.pask_decode_attention.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.pask_plan_area_bytes.argtypes = [_vp, _i32]
+_lib.pask_plan_area_bytes.restype = _sz
+_lib.pask_plan_ahead.argtypes = [_vp, _i32, _i32, _vp, _vp, _sz, _vp]
+_lib.pask_decode_step_ahead.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
 _lib.pask_decode_attention_full.argtypes = _lib.pask_decode_attention.argtypes
 _lib.pask_decode_attention_static.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.pask_workspace_bytes.argtypes = [_vp, _i32]
@@ -214,6 +218,28 @@ def pask_append_attend(cache: int, layer: int, seq_ids, cu_tokens, k, v, tags, q
                                    _dptr(q, torch.bfloat16), _dptr(out, torch.float32), _dptr(lse, torch.float32),
                                    _dptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "pask_append_attend")
+
+
+def pask_plan_area_bytes(cache: int, n_seqs: int) -> int:
+    return int(_lib.pask_plan_area_bytes(cache, n_seqs))
+
+
+def pask_plan_ahead(cache: int, layer: int, seq_ids, plan_area, stream=None):
+    """Write the layer's decode-attention plan for this batch from the cache as it stands (see pask.h)."""
+    _check(_lib.pask_plan_ahead(cache, layer, seq_ids.numel(), _dptr(seq_ids, torch.int32), _dptr(plan_area),
+                                plan_area.numel() * plan_area.element_size(), _stream(stream)), "pask_plan_ahead")
+
+
+def pask_decode_step_ahead(cache: int, layer: int, seq_ids, k, v, tags, q, out, lse, workspace, plan_area, actions=None,
+                           actions_out=None, stream=None):
+    """One layer of a decode step, one new token per sequence, from the plan made ahead: the streaming kernel starts at
+    once, the append runs beside it and leaves the next step's plan, the merge attends the new token from k / v."""
+    _check(_lib.pask_decode_step_ahead(cache, layer, seq_ids.numel(), _dptr(seq_ids, torch.int32), _dptr(k, torch.bfloat16),
+                                       _dptr(v, torch.bfloat16), _dptr(tags, torch.uint8), _dptr(actions, torch.uint8),
+                                       _dptr(actions_out, torch.uint8), _dptr(q, torch.bfloat16), _dptr(out, torch.float32),
+                                       _dptr(lse, torch.float32), _dptr(workspace), workspace.numel() * workspace.element_size(),
+                                       _dptr(plan_area), plan_area.numel() * plan_area.element_size(), _stream(stream)),
+           "pask_decode_step_ahead")
 
 
 def pask_workspace_bytes(cache: int, n_seqs: int) -> int:

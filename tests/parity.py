@@ -103,7 +103,7 @@ class Pair:
         return rc
 
     # ------------------------------------------------------------------ state
-    def compare_state(self, layers=None, seqs=None):
+    def compare_state(self, layers=None, seqs=None, expect_status=0):
         P, h = self.pask, self.gpu.handle
         layers = range(self.cfg.n_layers) if layers is None else layers
         seqs = range(self.max_seqs) if seqs is None else seqs
@@ -122,7 +122,7 @@ class Pair:
                 assert np.array_equal(gvs, ovs), ("low V scales", l, s)
                 assert np.array_equal(gkc, okc), ("low K codes", l, s)
                 assert np.array_equal(gvc, ovc), ("low V codes", l, s)
-            self.compare_budget(s)
+            self.compare_budget(s, expect_status=expect_status)
         assert P.pask_debug_pool_state(h) == self.orc.pool_state()
 
     def compare_budget(self, s, expect_status=0):

@@ -1,0 +1,205 @@
+"""Planned-ahead decode steps (pask_plan_ahead + pask_decode_step_ahead) against the oracle and against
+pask_append_attend.
+
+The streaming kernel of such a step works from a plan of the cache before the step's append, the
+append runs beside it and the merge attends the new token from the call's inputs.  The cache state
+it leaves (pages, codes, scales, page ids, counters) must be bit-identical to the oracle's and to
+what pask_append_attend leaves; out / lse must agree with the fp64 oracle within the usual bound."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from pask_workloads import configs as WC
+from pask_workloads import policy as WP
+from pask_workloads.tensors import bf16_bits
+
+from parity import Pair, assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pask():
+    import paper_2608_28276_b200 as P
+    assert torch.cuda.is_available()
+    return P
+
+
+def _pair(pask, oracle, batch, prompt, gen, low_bits=4, dynamic=False, **kw):
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=batch, prompt_len=prompt, gen_len=gen, extra_gen=80, low_bits=low_bits)
+    w = WC.build(cfg)
+    blob = w.dynamic_blob(reserve_tokens=4, budget=0.3) if dynamic else w.blob
+    return Pair(pask, oracle, w, blob=blob, **kw), w
+
+
+def _ahead_step(p, area, layer, seqs, pos, acts=None):
+    """One planned-ahead call on the GPU, append + attention on the oracle; compares actions and outputs."""
+    d = "cuda"
+    n = len(seqs)
+    ones = [1] * n
+    tags, states, k, v = p.gather(seqs, ones, pos, layer)
+    act_o, act_g = acts if acts else (None, None)
+    rc, used_o = p.orc.append(layer, seqs, list(range(n + 1)), bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags, decided=act_o)
+    assert rc == 0
+    q = torch.stack([p.w.q(layer, int(s), int(t) + 1) for s, t in zip(seqs, pos)])
+    out = torch.full((n, p.cfg.n_q, 128), float("nan"), dtype=torch.float32, device=d)
+    lse = torch.full((n, p.cfg.n_q), float("nan"), dtype=torch.float32, device=d)
+    used_g = torch.full((n,), 0xEE, dtype=torch.uint8, device=d)
+    ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+    p.pask.pask_decode_step_ahead(p.gpu.handle, layer, ids, k.to(d), v.to(d), torch.from_numpy(tags).to(d), q.to(d), out, lse,
+                                  p.gpu.workspace(n), area, actions=act_g, actions_out=used_g)
+    torch.cuda.synchronize()
+    assert np.array_equal(used_g.cpu().numpy(), used_o)
+    oo, ol = p.orc.attention_batch(layer, seqs, bf16_bits(q).numpy())
+    assert_close(out.cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64), oo, ol, where=(layer, seqs))
+    return out, lse, (ids, k.to(d), v.to(d), torch.from_numpy(tags).to(d), q.to(d))
+
+
+@pytest.mark.parametrize("batch,low_bits,dynamic", [(5, 4, False), (64, 4, False), (7, 4, True), (3, 8, False), (3, 2, False),
+                                                    (255, 4, False)])
+def test_steps_ahead_against_the_oracle(pask, oracle, batch, low_bits, dynamic):
+    prompt, gen = (40, 24) if batch > 8 else (150, 70)
+    p, w = _pair(pask, oracle, batch, prompt, gen, low_bits=low_bits, dynamic=dynamic)
+    seqs = list(range(batch))[::-1]
+    lens = [w.total_len(s) - (3 * s) % 17 for s in seqs]
+    if dynamic:
+        tags, states = p.gather(seqs, lens, [0] * batch)
+        _, act_o, act_g = p.decide(seqs, lens, tags, states)
+        for layer in range(w.cfg.n_layers):
+            _, _, k, v = p.gather(seqs, lens, [0] * batch, layer)
+            p.append_decided(layer, seqs, lens, k, v, tags, act_o, act_g)
+    else:
+        for layer in range(w.cfg.n_layers):
+            p.append(layer, seqs, lens, [0] * batch)
+    area = torch.empty(pask.pask_plan_area_bytes(p.gpu.handle, batch), dtype=torch.uint8, device="cuda")
+    ids = torch.tensor(seqs, dtype=torch.int32, device="cuda")
+    for layer in range(w.cfg.n_layers):
+        pask.pask_plan_ahead(p.gpu.handle, layer, ids, area)
+    pos = list(lens)
+    for step in range(36):                  # long enough for pages of both streams to fill up and new ones to be taken
+        acts = None
+        if dynamic:
+            tags, states = p.gather(seqs, [1] * batch, pos)
+            _, act_o, act_g = p.decide(seqs, [1] * batch, tags, states)
+            acts = (act_o, act_g)
+        for layer in range(w.cfg.n_layers):
+            _ahead_step(p, area, layer, seqs, pos, acts)
+        pos = [x + 1 for x in pos]
+    p.compare_state()
+    assert pask.pask_budget_state(p.gpu.handle, 0).device_status == 0
+
+
+def test_same_state_and_close_outputs_as_the_fused_call(pask, oracle):
+    p, w = _pair(pask, oracle, 4, 100, 60)
+    p2, _ = _pair(pask, oracle, 4, 100, 60)
+    seqs = [3, 1, 0, 2]
+    lens = [150, 97, 160, 33]
+    for layer in range(w.cfg.n_layers):
+        p.append(layer, seqs, lens, [0] * 4)
+        p2.append(layer, seqs, lens, [0] * 4)
+    area = torch.empty(pask.pask_plan_area_bytes(p.gpu.handle, 4), dtype=torch.uint8, device="cuda")
+    cu = torch.arange(5, dtype=torch.int32, device="cuda")
+    for layer in range(w.cfg.n_layers):
+        pask.pask_plan_ahead(p.gpu.handle, layer, torch.tensor(seqs, dtype=torch.int32, device="cuda"), area)
+    pos = list(lens)
+    for step in range(20):
+        for layer in range(w.cfg.n_layers):
+            out, lse, (ids, k, v, tags, q) = _ahead_step(p, area, layer, seqs, pos)
+            out2, lse2 = torch.empty_like(out), torch.empty_like(lse)
+            pask.pask_append_attend(p2.gpu.handle, layer, ids, cu, k, v, tags, q, out2, lse2, p2.gpu.workspace(4))
+            torch.cuda.synchronize()
+            assert float((out - out2).abs().max()) < 2e-4 and float((lse - lse2).abs().max()) < 2e-4     # (a new RETAIN-LOW token: exact here, P * scale in fp16 there)
+        pos = [x + 1 for x in pos]
+    # the two caches hold the same bytes
+    for s in seqs:
+        for layer in range(w.cfg.n_layers):
+            a, b = pask.pask_debug_dump_high(p.gpu.handle, layer, s, 8), pask.pask_debug_dump_high(p2.gpu.handle, layer, s, 8)
+            assert all(np.array_equal(x, y) for x, y in zip(a, b))
+            a, b = pask.pask_debug_dump_low(p.gpu.handle, layer, s, 8), pask.pask_debug_dump_low(p2.gpu.handle, layer, s, 8)
+            assert all(np.array_equal(x, y) for x, y in zip(a, b))
+    p.compare_state()
+
+
+def test_stale_plans_are_refused_or_flagged(pask, oracle):
+    p, w = _pair(pask, oracle, 3, 60, 40)
+    seqs = [0, 1, 2]
+    for layer in range(w.cfg.n_layers):
+        p.append(layer, seqs, [100] * 3, [0] * 3)
+    P, h, d = pask, p.gpu.handle, "cuda"
+    area = torch.empty(P.pask_plan_area_bytes(h, 3), dtype=torch.uint8, device=d)
+    ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+    tags, states, k, v = p.gather(seqs, [1] * 3, [100] * 3, 0)
+    q = torch.stack([w.q(0, s, 101) for s in seqs]).to(d)
+    out = torch.zeros((3, 32, 128), dtype=torch.float32, device=d)
+    lse = torch.zeros((3, 32), dtype=torch.float32, device=d)
+    args = (k.to(d), v.to(d), torch.from_numpy(tags).to(d), q, out, lse, p.gpu.workspace(3), area)
+
+    def refused(layer=0, ids_=ids, a=args):
+        with pytest.raises(P.PaskError) as e:
+            P.pask_decode_step_ahead(h, layer, ids_, *a)
+        return e.value.status
+
+    assert refused() == P.ERR_STALE_PLAN                                  # no plan yet
+    P.pask_plan_ahead(h, 0, ids, area)
+    assert refused(layer=1) == P.ERR_STALE_PLAN                           # another layer
+    assert refused(ids_=ids[:2].contiguous(), a=(k[:2].to(d), v[:2].to(d), torch.from_numpy(tags[:2]).to(d), q[:2].contiguous(),
+                                                 out[:2], lse[:2], p.gpu.workspace(3), area)) == P.ERR_STALE_PLAN   # another batch size
+    other = torch.empty_like(area)
+    assert refused(a=args[:-1] + (other,)) == P.ERR_STALE_PLAN            # another plan area
+    small = torch.empty(area.numel() - 256, dtype=torch.uint8, device=d)
+    assert refused(a=args[:-1] + (small,)) == P.ERR_WORKSPACE
+    # an append through another call forgets the plan
+    p.append(0, seqs, [1] * 3, [100] * 3)
+    assert refused() == P.ERR_STALE_PLAN
+    # a different list of the same length is only seen on the device
+    P.pask_plan_ahead(h, 0, ids, area)
+    swapped = torch.tensor([1, 0, 2], dtype=torch.int32, device=d)
+    P.pask_decode_step_ahead(h, 0, swapped, *args)
+    torch.cuda.synchronize()
+    assert P.pask_budget_state(h, 0).device_status & P.DEV_STALE_PLAN
+    # a protected recent window is not served by this path
+    pw = Pair(pask, oracle, w, blob=WP.write_blob(replace(w.policy, recent_window=16)))
+    with pytest.raises(P.PaskError) as e:
+        P.pask_plan_ahead(pw.gpu.handle, 0, ids, area)
+    assert e.value.status == P.ERR_UNSUPPORTED_SHAPE
+
+
+def test_refused_append_inside_a_step_ahead(pask, oracle):
+    # the pools hold one page more than the history needs: within a few steps a call wants a page that is not there.
+    # Nothing is written by that call, the sticky bit says why, and both sides still hold the same state.
+    seqs, n0 = [0, 1], 64
+    probe, w = _pair(pask, oracle, 2, 40, 20)
+    for layer in range(w.cfg.n_layers):
+        probe.append(layer, seqs, [n0] * 2, [0] * 2)
+    used_h, _, used_l, _ = probe.orc.pool_state()
+    p, w = _pair(pask, oracle, 2, 40, 20, pool_high_pages=used_h + 1, pool_low_pages=used_l + 1)
+    P, h, d = pask, p.gpu.handle, "cuda"
+    for layer in range(w.cfg.n_layers):
+        p.append(layer, seqs, [n0] * 2, [0] * 2)
+    area = torch.empty(P.pask_plan_area_bytes(h, 2), dtype=torch.uint8, device=d)
+    ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+    for layer in range(w.cfg.n_layers):
+        P.pask_plan_ahead(h, layer, ids, area)
+    pos, failed = n0, False
+    for step in range(40):
+        for layer in range(w.cfg.n_layers):
+            tags, states, k, v = p.gather(seqs, [1] * 2, [pos] * 2, layer)
+            rc, _ = p.orc.append(layer, seqs, [0, 1, 2], bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags)
+            q = torch.stack([w.q(layer, s, pos + 1) for s in seqs]).to(d)
+            out = torch.zeros((2, 32, 128), dtype=torch.float32, device=d)
+            lse = torch.zeros((2, 32), dtype=torch.float32, device=d)
+            P.pask_decode_step_ahead(h, layer, ids, k.to(d), v.to(d), torch.from_numpy(tags).to(d), q, out, lse, p.gpu.workspace(2), area)
+            torch.cuda.synchronize()
+            st = P.pask_budget_state(h, 0).device_status
+            if rc != 0:
+                assert st & P.DEV_POOL_EXHAUSTED
+                failed = True
+                break
+            assert st == 0
+        if failed:
+            break
+        pos += 1
+    assert failed
+    p.compare_state(expect_status=P.DEV_POOL_EXHAUSTED)       # the refused call changed nothing on either side
