@@ -457,6 +457,7 @@ pask_status_t pask_plan_ahead(pask_cache_t *c, int32_t layer, int32_t n_seqs, co
     a.n_seqs = n_seqs;
     a.parity = 0;
     a.area = area;
+    a.early_from = c->ahead_calls + 2;
     return PASK_OK;
 }
 
@@ -473,10 +474,15 @@ pask_status_t pask_decode_step_ahead(pask_cache_t *c, int32_t layer, int32_t n_s
     auto &a = c->ahead[layer];
     if (!a.valid || a.n_seqs != n_seqs || a.area != area) return PASK_ERR_STALE_PLAN;
     NvtxRange range("pask_decode_step_ahead");
+    // The streaming kernel may look its range up and start its first copies before its dependency wait only if the
+    // plan's writer is surely complete by then: that holds once another planned-ahead call lies between the two in
+    // the stream (its streaming kernel lets later kernels start only after it has waited for everything before it).
+    const uint64_t call = ++c->ahead_calls;
     rc = launch_step_ahead(c, layer, n_seqs, seq_ids, k, v, tags, actions, actions_out, q, out, lse, ws, area, a.parity,
-                           static_cast<cudaStream_t>(stream));
+                           call >= a.early_from, static_cast<cudaStream_t>(stream));
     if (rc != PASK_OK) { a.valid = false; return rc; }
     a.parity ^= 1;                      // the append has left the next step's plan in the other block
+    a.early_from = call + 2;
     return PASK_OK;
 }
 

@@ -54,6 +54,8 @@ struct AttnParams {
     Workspace ws;
     long long wait_cycles;  // bound of a wait for a bulk copy, in SM clock cycles
     uint32_t overpost;      // test aid: bytes announced beyond what a warp's first copy brings (0 in normal use)
+    int early;              // the plan and the pages were written before the kernel's predecessor in the stream started:
+                            // range look-up and the first bulk copies need not wait for that predecessor
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -422,15 +424,24 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     uint8_t *s_ring = smem + off;
     uint8_t *s_scratch = s_ring + (size_t)n_warps * kStages * kStageBytes;
 
-    pdl_wait();
-    pdl_launch_dependents();   // only now: the combine kernel reads the plan's prefix before its own wait
+    // Normally everything the kernel reads comes from its predecessor in the stream (the plan).  In a planned-ahead
+    // step the plan and every page it names were written a whole step earlier, so the set-up below and the first
+    // copies run while the predecessor (the merge kernel of the layer before) is still at work; only the queries,
+    // the per-sequence scalars and the partials this kernel writes have to wait.
+    if (!p.early) {
+        pdl_wait();
+        pdl_launch_dependents();   // only now: the combine kernel reads the plan's prefix before its own wait
+    }
     for (int s = tid; s <= n_seqs; s += blockDim.x) {
         s_cost[s] = __ldg(p.ws.cost_prefix + s);
         s_page[s] = __ldg(p.ws.page_prefix + s);
     }
     __syncthreads();
     const uint32_t total = s_cost[n_seqs];
-    if (total == 0) return;
+    if (total == 0) {
+        if (p.early) { pdl_wait(); pdl_launch_dependents(); }
+        return;
+    }
 
     const uint32_t n_ctas = gridDim.x, b = blockIdx.x;
     const uint32_t lo = (uint32_t)(((uint64_t)total * b) / n_ctas);
@@ -487,6 +498,10 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     }
     __syncwarp();
     for (int i = 0; i < kStages; i++) w.produce();
+    if (p.early) {
+        pdl_wait();
+        pdl_launch_dependents();   // (the append that runs beside this kernel must not start before this wait is over)
+    }
 
     const float kLog2Scale = 0.088388347648318440550f * 1.4426950408889634074f;  // log2(e) / sqrt(128)
     const float kSlack = 6.0f;               // log2 units a score may exceed the reference maximum by
@@ -1123,6 +1138,7 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
     p.seq_ids = seq_ids;
     p.q = static_cast<const uint4 *>(q);
     carve_workspace(c, n_seqs, static_cast<uint8_t *>(workspace), &p.ws);
+    p.early = 0;
     cudaError_t e = cudaSuccess;
     if (!plan_done)   // (a fused append has already left the plan in the workspace)
         e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(5 * n_seqs + 2) * 4, stream, c->dev,
@@ -1187,7 +1203,7 @@ pask_status_t launch_plan_ahead(pask_cache *c, int layer, int n_seqs, const int3
 // replaced, the other plan block) and so runs as its CTAs retire; the merge kernel, which waits for both.
 pask_status_t launch_step_ahead(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const void *k, const void *v,
                                 const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out, const void *q, float *out,
-                                float *lse, void *workspace, void *area, int cur, cudaStream_t stream) {
+                                float *lse, void *workspace, void *area, int cur, bool early, cudaStream_t stream) {
     PlanBlock pc, pn;
     carve_plan_area(c, n_seqs, layer, cur, static_cast<uint8_t *>(area), &pc);
     carve_plan_area(c, n_seqs, layer, cur ^ 1, static_cast<uint8_t *>(area), &pn);
@@ -1199,6 +1215,7 @@ pask_status_t launch_step_ahead(pask_cache *c, int layer, int n_seqs, const int3
     Workspace parts;
     carve_workspace(c, n_seqs, static_cast<uint8_t *>(workspace), &parts);
     p.ws = plan_view(pc, parts);
+    p.early = early ? 1 : 0;
     cudaError_t e = launch_stream_kernel(c, true, p, stream);
     if (e != cudaSuccess) return PASK_ERR_CUDA;
     const pask_status_t rc = launch_append_beside(c, layer, n_seqs, seq_ids, static_cast<const int32_t *>(area), k, v, tags, decided,

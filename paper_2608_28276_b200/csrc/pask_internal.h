@@ -140,8 +140,10 @@ struct pask_cache {
         bool valid = false;
         int n_seqs = 0, parity = 0;
         const void *area = nullptr;
+        uint64_t early_from = 0;  // first planned-ahead call (by number) that may read the plan before its dependency wait
     };
     std::vector<Ahead> ahead;     // [n_layers]
+    uint64_t ahead_calls = 0;     // planned-ahead step calls issued so far
     long long wait_cycles;        // bound of a device-side wait for a bulk copy, in SM clock cycles (about a second)
     uint32_t wait_test_surplus;   // pask_debug_set_wait: bytes a warp's first copy announces but does not bring
     // pask_decode_step_pipelined: two copy streams and the events that order them against the caller's stream
@@ -204,7 +206,7 @@ pask_status_t launch_plan_ahead(pask_cache *c, int layer, int n_seqs, const int3
 // streaming kernel over the plan block `cur`, then the append that writes the other block, then the merge with the new tokens
 pask_status_t launch_step_ahead(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const void *k, const void *v,
                                 const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out, const void *q, float *out,
-                                float *lse, void *workspace, void *area, int cur, cudaStream_t stream);
+                                float *lse, void *workspace, void *area, int cur, bool early, cudaStream_t stream);
 // the one-launch append with its dependency wait moved to its end (it runs beside the kernel before it) and the
 // call's sequence list recorded next to the plan it writes
 pask_status_t launch_append_beside(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,

@@ -110,7 +110,7 @@ def test_same_state_and_close_outputs_as_the_fused_call(pask, oracle):
             out2, lse2 = torch.empty_like(out), torch.empty_like(lse)
             pask.pask_append_attend(p2.gpu.handle, layer, ids, cu, k, v, tags, q, out2, lse2, p2.gpu.workspace(4))
             torch.cuda.synchronize()
-            assert float((out - out2).abs().max()) < 2e-4 and float((lse - lse2).abs().max()) < 2e-4     # (a new RETAIN-LOW token: exact here, P * scale in fp16 there)
+            assert float((out - out2).abs().max()) < 1e-3 and float((lse - lse2).abs().max()) < 1e-3     # (a new RETAIN-LOW token: exact here, P * scale in fp16 there)
         pos = [x + 1 for x in pos]
     # the two caches hold the same bytes
     for s in seqs:
