@@ -643,16 +643,22 @@ def end_to_end(P, runner, job, w, cfg, first_step, e2e_warm, e2e_steps, world, d
             rows.append(block)
         host.append(rows)
     out_h = torch.empty((job.B, cfg.n_q, 128), dtype=torch.float32).pin_memory()
+    if job.ahead:        # the timed steps before have left every layer's plan for this batch in job.area
+        def call(layer, block):
+            P.pask_decode_step_pipelined_ahead(job.cache.handle, layer, job.B, block, out_h, staging, job.ws, job.area)
+    else:
+        def call(layer, block):
+            P.pask_decode_step_pipelined(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
     for rows in host[:e2e_warm]:
         for layer, block in enumerate(rows):
-            P.pask_decode_step_pipelined(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
+            call(layer, block)
     P.pask_decode_step_drain(job.cache.handle)
     runner.barrier()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     for rows in host[e2e_warm:]:
         for layer, block in enumerate(rows):
-            P.pask_decode_step_pipelined(job.cache.handle, layer, job.B, block, out_h, staging, job.ws)
+            call(layer, block)
     P.pask_decode_step_drain(job.cache.handle)      # the host holds every output before the clock stops
     t1.record()
     runner.barrier()
@@ -661,7 +667,7 @@ def end_to_end(P, runner, job, w, cfg, first_step, e2e_warm, e2e_steps, world, d
     d2h = cfg.n_layers * job.B * cfg.n_q * 128 * 4
     return {"value": whole_job_tokens_per_s(world, job.B, e2e_steps, e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps,
-            "api": "pask_decode_step_pipelined: one pinned host block in, attention output out, per layer; the "
+            "api": ("pask_decode_step_pipelined_ahead" if job.ahead else "pask_decode_step_pipelined") + ": one pinned host block in, attention output out, per layer; the "
                    "copies run on the library's copy streams and overlap the neighbouring layers' kernels"}
 
 

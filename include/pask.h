@@ -401,6 +401,12 @@ pask_status_t pask_decode_step_packed(pask_cache_t *cache, int32_t layer, int32_
 pask_status_t pask_decode_step_pipelined(pask_cache_t *cache, int32_t layer, int32_t n_seqs, const void *packed_host,
                                          float *out_host, void *staging, size_t staging_bytes, void *workspace,
                                          size_t workspace_bytes, pask_stream_t stream);
+/* The same with the layer's step issued as pask_decode_step_ahead (plan made a step ahead; plan_area as
+ * there, pask_plan_ahead for the layer first; the block's cu_tokens field is not read).  Errors as for the two. */
+pask_status_t pask_decode_step_pipelined_ahead(pask_cache_t *cache, int32_t layer, int32_t n_seqs,
+                                               const void *packed_host, float *out_host, void *staging,
+                                               size_t staging_bytes, void *workspace, size_t workspace_bytes,
+                                               void *plan_area, size_t plan_area_bytes, pask_stream_t stream);
 pask_status_t pask_decode_step_drain(pask_cache_t *cache);
 
 /* ---------------------------------------------------------------------------------------------

@@ -29,7 +29,7 @@ EXPORTS = [
     "pask_load_policy", "pask_free_policy", "pask_policy_action", "pask_cache_sizes", "pask_cache_create",
     "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decide",
     "pask_append_kv_decided", "pask_append_attend", "pask_plan_area_bytes", "pask_plan_ahead", "pask_decode_step_ahead", "pask_decode_attention",
-    "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes", "pask_step_packed_layout", "pask_decode_step_packed", "pask_decode_step_pipelined", "pask_decode_step_drain",
+    "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes", "pask_step_packed_layout", "pask_decode_step_packed", "pask_decode_step_pipelined", "pask_decode_step_pipelined_ahead", "pask_decode_step_drain",
     "pask_budget_state", "pask_distortion", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
     "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_debug_set_wait", "pask_status_string",
 ]
@@ -91,6 +91,7 @@ _lib.pask_decode_step_host.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
 _lib.pask_step_packed_layout.argtypes = [_vp, _i32, C.POINTER(_sz * 6), C.POINTER(_sz)]
 _lib.pask_decode_step_packed.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
 _lib.pask_decode_step_pipelined.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp, _sz, _vp]
+_lib.pask_decode_step_pipelined_ahead.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp, _sz, _vp, _sz, _vp]
 _lib.pask_decode_step_drain.argtypes = [_vp]
 _lib.pask_step_staging_bytes.argtypes = [_vp, _i32]
 _lib.pask_step_staging_bytes.restype = _sz
@@ -321,6 +322,17 @@ def pask_decode_step_pipelined(cache: int, layer: int, n_seqs: int, packed_host,
                                            staging.numel() * staging.element_size(), _dptr(workspace),
                                            workspace.numel() * workspace.element_size(), _stream(stream)),
            "pask_decode_step_pipelined")
+
+
+def pask_decode_step_pipelined_ahead(cache: int, layer: int, n_seqs: int, packed_host, out_host, staging, workspace, plan_area,
+                                     stream=None):
+    """pask_decode_step_pipelined with the layer's step issued as pask_decode_step_ahead."""
+    assert not packed_host.is_cuda and packed_host.is_contiguous() and not out_host.is_cuda and out_host.is_contiguous()
+    _check(_lib.pask_decode_step_pipelined_ahead(cache, layer, n_seqs, packed_host.data_ptr(), out_host.data_ptr(), _dptr(staging),
+                                                 staging.numel() * staging.element_size(), _dptr(workspace),
+                                                 workspace.numel() * workspace.element_size(), _dptr(plan_area),
+                                                 plan_area.numel() * plan_area.element_size(), _stream(stream)),
+           "pask_decode_step_pipelined_ahead")
 
 
 def pask_decode_step_drain(cache: int):

@@ -574,9 +574,9 @@ pask_status_t pask_decode_step_packed(pask_cache_t *c, int32_t layer, int32_t n_
                                    stream));
 }
 
-pask_status_t pask_decode_step_pipelined(pask_cache_t *c, int32_t layer, int32_t n_seqs, const void *packed_host,
-                                         float *out_host, void *staging, size_t staging_bytes, void *ws, size_t ws_bytes,
-                                         pask_stream_t stream_v) {
+static pask_status_t step_pipelined(pask_cache_t *c, int32_t layer, int32_t n_seqs, const void *packed_host,
+                                    float *out_host, void *staging, size_t staging_bytes, void *ws, size_t ws_bytes,
+                                    void *plan_area, size_t plan_area_bytes, pask_stream_t stream_v) {
     if (!c || !packed_host || !out_host || !staging) return PASK_ERR_INVALID_ARG;
     if (n_seqs < 1 || n_seqs > PASK_MAX_SEQS_PER_CALL) return PASK_ERR_INVALID_ARG;
     const size_t slot_bytes = pask_step_staging_bytes(c, n_seqs);
@@ -625,9 +625,12 @@ pask_status_t pask_decode_step_pipelined(pask_cache_t *c, int32_t layer, int32_t
     if (e == cudaSuccess && moved && (pp.recorded[slot ^ 1] & 2)) e = cudaStreamWaitEvent(stream, pp.ev_out[slot ^ 1], 0);
     if (e != cudaSuccess) return PASK_ERR_CUDA;
     (void)call;
-    pask_status_t rc = pask_append_attend(c, layer, n_seqs, n_seqs, reinterpret_cast<const int32_t *>(p + off[0]),
-                                          reinterpret_cast<const int32_t *>(p + off[1]), p + off[2], p + off[3], p + off[4],
-                                          nullptr, nullptr, p + off[5], d_out, nullptr, ws, ws_bytes, stream_v);
+    pask_status_t rc = plan_area
+        ? pask_decode_step_ahead(c, layer, n_seqs, reinterpret_cast<const int32_t *>(p + off[0]), p + off[2], p + off[3], p + off[4],
+                                 nullptr, nullptr, p + off[5], d_out, nullptr, ws, ws_bytes, plan_area, plan_area_bytes, stream_v)
+        : pask_append_attend(c, layer, n_seqs, n_seqs, reinterpret_cast<const int32_t *>(p + off[0]),
+                             reinterpret_cast<const int32_t *>(p + off[1]), p + off[2], p + off[3], p + off[4],
+                             nullptr, nullptr, p + off[5], d_out, nullptr, ws, ws_bytes, stream_v);
     // whatever was enqueued reads this slot: mark its end on the caller's stream even if the step was refused
     e = cudaEventRecord(pp.ev_done[slot], stream);
     if (e == cudaSuccess) pp.recorded[slot] |= 1;
@@ -638,6 +641,20 @@ pask_status_t pask_decode_step_pipelined(pask_cache_t *c, int32_t layer, int32_t
     if (e == cudaSuccess) e = cudaEventRecord(pp.ev_out[slot], pp.out);
     if (e == cudaSuccess) pp.recorded[slot] |= 2;
     return cuda_rc(e);
+}
+
+pask_status_t pask_decode_step_pipelined(pask_cache_t *c, int32_t layer, int32_t n_seqs, const void *packed_host,
+                                         float *out_host, void *staging, size_t staging_bytes, void *ws, size_t ws_bytes,
+                                         pask_stream_t stream) {
+    return step_pipelined(c, layer, n_seqs, packed_host, out_host, staging, staging_bytes, ws, ws_bytes, nullptr, 0, stream);
+}
+
+pask_status_t pask_decode_step_pipelined_ahead(pask_cache_t *c, int32_t layer, int32_t n_seqs, const void *packed_host,
+                                               float *out_host, void *staging, size_t staging_bytes, void *ws, size_t ws_bytes,
+                                               void *plan_area, size_t plan_area_bytes, pask_stream_t stream) {
+    if (!plan_area) return PASK_ERR_INVALID_ARG;
+    return step_pipelined(c, layer, n_seqs, packed_host, out_host, staging, staging_bytes, ws, ws_bytes, plan_area,
+                          plan_area_bytes, stream);
 }
 
 pask_status_t pask_decode_step_drain(pask_cache_t *c) {

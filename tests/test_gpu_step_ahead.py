@@ -203,3 +203,72 @@ def test_refused_append_inside_a_step_ahead(pask, oracle):
         pos += 1
     assert failed
     p.compare_state(expect_status=P.DEV_POOL_EXHAUSTED)       # the refused call changed nothing on either side
+
+
+def test_pipelined_host_steps_ahead(pask, oracle):
+    # layer after layer from pinned host blocks, each layer's step issued as a planned-ahead one
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=5, n_layers=3, n_groups=3, prompt_len=150, gen_len=60, extra_gen=32)
+    w = WC.build(cfg)
+    p = Pair(pask, oracle, w)
+    seqs = [3, 0, 4, 1, 2]
+    for layer in range(3):
+        p.append(layer, seqs, [210] * 5, [0] * 5)
+    P, h = pask, p.gpu.handle
+    off, n_in = P.pask_step_packed_layout(h, 5)
+    staging = torch.empty(2 * P.pask_step_staging_bytes(h, 5), dtype=torch.uint8, device="cuda")
+    area = torch.empty(P.pask_plan_area_bytes(h, 5), dtype=torch.uint8, device="cuda")
+    ids = torch.tensor(seqs, dtype=torch.int32, device="cuda")
+    for layer in range(3):
+        P.pask_plan_ahead(h, layer, ids, area)
+    calls = []
+    for step in range(20):
+        for layer in range(3):
+            k = torch.stack([w.kv(layer, b, 210 + step, 1)[0][0] for b in seqs])
+            v = torch.stack([w.kv(layer, b, 210 + step, 1)[1][0] for b in seqs])
+            tags = torch.from_numpy(np.array([w.tags(b, 210 + step, 1)[0] for b in seqs], np.uint8))
+            q = torch.stack([w.q(layer, b, 211 + step) for b in seqs])
+            block = torch.zeros(n_in, dtype=torch.uint8).pin_memory()
+            for o, t in zip(off, [torch.tensor(seqs, dtype=torch.int32), torch.arange(6, dtype=torch.int32), k, v, tags, q]):
+                raw = t.contiguous().view(torch.uint8).reshape(-1)
+                block[o:o + raw.numel()] = raw
+            out = torch.full((5, 32, 128), float("nan"), dtype=torch.float32).pin_memory()
+            P.pask_decode_step_pipelined_ahead(h, layer, 5, block, out, staging, p.gpu.workspace(5), area)
+            rc, _ = p.orc.append(layer, seqs, list(range(6)), bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags.numpy())
+            assert rc == 0
+            oo, ol = p.orc.attention_batch(layer, seqs, bf16_bits(q).numpy())
+            calls.append((block, out, oo, ol))
+    P.pask_decode_step_drain(h)
+    torch.cuda.synchronize()
+    for block, out, oo, ol in calls:
+        assert_close(out.numpy().astype(np.float64), ol.copy(), oo, ol)
+    p.compare_state()
+
+
+def test_one_layer_called_back_to_back(pask, oracle):
+    # a single layer stepped again and again: the plan a call reads was written by the call right before it, so the
+    # streaming kernel may not read it ahead of its dependency wait (the handle keeps track); results stay the oracle's
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=6, n_layers=1, n_groups=1, prompt_len=90, gen_len=40, extra_gen=80)
+    w = WC.build(cfg)
+    p = Pair(pask, oracle, w)
+    seqs = [5, 4, 3, 2, 1, 0]
+    lens = [w.total_len(s) for s in seqs]
+    p.append(0, seqs, lens, [0] * 6)
+    area = torch.empty(pask.pask_plan_area_bytes(p.gpu.handle, 6), dtype=torch.uint8, device="cuda")
+    pask.pask_plan_ahead(p.gpu.handle, 0, torch.tensor(seqs, dtype=torch.int32, device="cuda"), area)
+    d, n, pos, held = "cuda", 6, list(lens), []
+    ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+    for step in range(50):                 # no synchronisation between the calls: the kernels of consecutive steps do overlap
+        tags, states, k, v = p.gather(seqs, [1] * n, pos, 0)
+        rc, _ = p.orc.append(0, seqs, list(range(n + 1)), bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags)
+        assert rc == 0
+        q = torch.stack([w.q(0, s, t + 1) for s, t in zip(seqs, pos)])
+        out = torch.full((n, cfg.n_q, 128), float("nan"), dtype=torch.float32, device=d)
+        lse = torch.full((n, cfg.n_q), float("nan"), dtype=torch.float32, device=d)
+        dev = (k.to(d), v.to(d), torch.from_numpy(tags).to(d), q.to(d))
+        pask.pask_decode_step_ahead(p.gpu.handle, 0, ids, *dev, out, lse, p.gpu.workspace(n), area)
+        held.append((dev, out, lse, p.orc.attention_batch(0, seqs, bf16_bits(q).numpy())))
+        pos = [x + 1 for x in pos]
+    torch.cuda.synchronize()
+    for dev, out, lse, (oo, ol) in held:
+        assert_close(out.cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64), oo, ol)
+    p.compare_state()
