@@ -438,19 +438,43 @@ __device__ __forceinline__ void persist_chunk(const DevCache &c, uint32_t a, uin
 // one run of 128-bit stores in the packed layout; a partly filled page (the first and last page of
 // a stream's range at most) is written token by token with persist_chunk.
 constexpr int kWriteThreads = 256;
-constexpr int kRowBytes = 2 * kHeadDim + 16;      // one token's K (or V) row of a head in shared memory, padded
+constexpr int kRowPad = 16;                       // bytes between two staged rows (bank spread: rows are 2^k bytes)
+constexpr long long kWriteWaitCycles = 2000000000LL;   // bound of the wait for a page's staged rows (about a second)
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// waits for a phase of an mbarrier, at most `limit` clock cycles; false if it gave up
+__device__ __noinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, long long limit) {
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; i++) {
+            uint32_t done;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+            if (done) return true;
+        }
+        if (clock64() - t0 > limit) return false;
+    }
+}
 
 __global__ void __launch_bounds__(kWriteThreads, 3)
 append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__ k, const uint4 *__restrict__ v) {
     extern __shared__ __align__(16) uint8_t s_dyn[];                    // the page's source rows, see in_row()
-    __shared__ __align__(16) uint8_t s_low[2][kLowHeadBytes];           // one head of a LOW page, packed (two in turn)
+    __shared__ __align__(16) uint8_t s_low[4][kLowHeadBytes];           // packed heads of a LOW page (two pairs in turn)
     __shared__ uint32_t s_tok[kPageTokens];
-    // source rows of the page being written: [head][K|V][token][kRowBytes]
+    __shared__ __align__(8) uint64_t s_bar;                             // completion of a page's row copies
+    // source rows of the page being written: [K|V][token] whole rows (all heads, as they lie in memory), kRowPad apart
+    const int row_bytes = c.n_kv * 2 * kHeadDim, row_stride = row_bytes + kRowPad;
     auto in_row = [&](int head, int which, int tau) -> uint8_t * {
-        return s_dyn + (size_t)((head * 2 + which) * kPageTokens + tau) * kRowBytes;
+        return s_dyn + (size_t)(which * kPageTokens + tau) * row_stride + head * (2 * kHeadDim);
     };
     if (c.ctrl[kCtrlPlanOk] == 0) return;
     const int tid = threadIdx.x;
+    uint32_t bar_parity = 0;
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&s_bar)) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     const uint32_t n_items = c.ctrl[kCtrlItems];
     const uint32_t item0 = (uint32_t)(((uint64_t)n_items * blockIdx.x) / gridDim.x);
     const uint32_t item1 = (uint32_t)(((uint64_t)n_items * (blockIdx.x + 1)) / gridDim.x);
@@ -472,6 +496,7 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
         base_j = s_base[j];
         base_next = s_base[j + 1];
         __syncthreads();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the buffer is next written by bulk copies
     }
     const int chunks = 16 * c.n_kv;                // 16-byte chunks per token per tensor (a power of two)
     const int chunks_shift = 31 - __clz(chunks);
@@ -507,19 +532,29 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
             }
             continue;
         }
-        // ---- a full page: all 16 tokens' rows (every head, K and V) go to shared memory with
-        // asynchronous 16-byte copies, all in flight at once; then each head leaves as one packed block
-        {
-            const int per_tensor = kPageTokens * chunks;        // 16-byte chunks of K (or of V) in the page
-            for (int idx = tid; idx < 2 * per_tensor; idx += kWriteThreads) {
-                const int which = idx >= per_tensor, rem = which ? idx - per_tensor : idx;
-                const int tau = rem >> chunks_shift, cc = rem & (chunks - 1);      // consecutive threads: consecutive bytes of a row
-                cp_async16(in_row(cc >> 4, which, tau) + (cc & 15) * 16, (which ? v : k) + (size_t)s_tok[tau] * chunks + cc);
-            }
-            asm volatile("cp.async.commit_group;" ::: "memory");
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        // ---- a full page: the 16 tokens' K rows and V rows (all heads of a token lie together) go to shared memory
+        // as 32 bulk copies issued by one warp, completion counted on an mbarrier; then each head leaves as one
+        // packed block
+        if (tid < 2 * kPageTokens) {
+            const int which = tid >> 4, tau = tid & 15;
+            const uint32_t bar = smem_addr(&s_bar);
+            if (tid == 0)
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2u * kPageTokens * (uint32_t)row_bytes) : "memory");
+            __syncwarp();
+            const void *src = (which ? v : k) + (size_t)s_tok[tau] * chunks;
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr(in_row(0, which, tau))), "l"(src), "r"((uint32_t)row_bytes), "r"(bar) : "memory");
         }
-        __syncthreads();
+        {   // bounded wait: rows that never arrive set the sticky time-out bit and end this CTA's work (after one more
+            // bounded wait, so that no copy is still on its way into shared memory when the CTA retires)
+            const bool ok = mbar_wait_bounded(smem_addr(&s_bar), bar_parity, kWriteWaitCycles);
+            if (!__syncthreads_and(ok)) {
+                mbar_wait_bounded(smem_addr(&s_bar), bar_parity, kWriteWaitCycles);
+                if (tid == 0) atomicOr(&c.ctrl[kCtrlStatus], PASK_DEV_TIMEOUT);
+                return;
+            }
+            bar_parity ^= 1u;
+        }
         uint32_t vmax_bits = 0;
         for (int head = 0; head < c.n_kv; head++) {
             if (high) {
@@ -541,6 +576,7 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
                     dst[256 + tid] = make_uint4(a.x, a.y, b.x, b.y);
                 }
             } else {
+                if (c.low_bits == 4) break;     // four-bit codes: two heads at a time, below
                 // thread = (K|V, token, 32-dim group, half of it): 16 values
                 const int half = tid & 1, w = (tid >> 1) & 3, tau = (tid >> 3) & 15, which = tid >> 7;
                 const uint4 x0 = *reinterpret_cast<const uint4 *>(in_row(head, which, tau) + 64 * w + 32 * half);
@@ -619,58 +655,87 @@ append_write_kernel(DevCache c, int layer, int n_seqs, const uint4 *__restrict__
                     if (tid < kLow2HeadBytes / 16) dst2[tid] = reinterpret_cast<const uint4 *>(s_low[head & 1])[tid];
                     continue;
                 }
-                const float s32 = __fdiv_rn(amax, 7.0f);
-                __half sh = __float2half_rn(s32);
-                if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);   // saturate, never infinite
-                const float sc = __half2float(sh);
-                // code = clamp(rint(x * (1/s)), -7, 7) + 8.  Clamping first gives the same integer
-                // (the bounds are integers), and adding 1.5 * 2^23 + 8 to a value in [-7, 7] rounds it
-                // to the nearest integer, ties to even, leaving code in the low 4 bits of the sum.
-                // s == 0 means every value is zero: 1/s is replaced by 0 and all codes come out 8.
-                const float inv = sc == 0.0f ? 0.0f : __fdiv_rn(1.0f, sc);
-                // The sums are kept as bit patterns, 0x4B400000 + code, and packed by multiply-adds (a nibble per step,
-                // from the top one down) instead of mask, shift and or per code: the constant upper bits add up to a
-                // known word that is taken off at the end (K words, modulo 2^32) or fall outside the result (V half-words).
-                uint32_t raw[16];
-                // A normal, unsaturated fp16 scale is within 2^-11 of amax / 7, so |x / s| < 7.01 and the clamp cannot
-                // bite: it is only kept for subnormal scales (rounded coarsely) and the saturated one.
-                const uint32_t sbits = __half_as_ushort(sh);
-                if (sbits >= 0x0400u && sbits < 0x7BFFu) {
+            }
+        }
+        if (!high && c.low_bits == 4) {
+            // Four-bit codes.  thread = (head of a pair, K|V, 32-dim group, token): one whole group, 32 values -- the
+            // group's amax, scale and reciprocal are worked out once, by one thread.  A quarter warp reads eight
+            // different rows (kRowPad apart: no bank conflicts).
+            const int hsel = tid >> 7, which = (tid >> 6) & 1, w = (tid >> 4) & 3, tau = tid & 15;
+            for (int hp = 0; hp < c.n_kv; hp += 2) {
+                const int head = hp + hsel;
+                uint8_t *img = s_low[(hp & 2) + hsel] + (which ? kLowHalfBytes : 0);
+                if (head < c.n_kv) {
+                    uint32_t xs[16];
 #pragma unroll
-                    for (int e = 0; e < 16; e++) {
-                        const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
-                        raw[e] = __float_as_uint(__fadd_rn(__fmul_rn(f, inv), 12582920.0f));
+                    for (int q4 = 0; q4 < 4; q4++) {
+                        const uint4 x = *reinterpret_cast<const uint4 *>(in_row(head, which, tau) + 64 * w + 16 * q4);
+                        xs[4 * q4] = x.x; xs[4 * q4 + 1] = x.y; xs[4 * q4 + 2] = x.z; xs[4 * q4 + 3] = x.w;
                     }
-                } else {
+                    // amax on the packed bf16 pairs (abs and max are exact in any format)
+                    __nv_bfloat162 m2 = __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&xs[0]));
 #pragma unroll
-                    for (int e = 0; e < 16; e++) {
-                        const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
-                        const float cl = fminf(fmaxf(__fmul_rn(f, inv), -7.0f), 7.0f);
-                        raw[e] = __float_as_uint(__fadd_rn(cl, 12582920.0f));
+                    for (int e = 1; e < 16; e++) m2 = __hmax2(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&xs[e])));
+                    const uint32_t m2b = *reinterpret_cast<const uint32_t *>(&m2);
+                    const float amax = fmaxf(bf16_lo(m2b), bf16_hi(m2b));
+                    const float s32 = __fdiv_rn(amax, 7.0f);
+                    __half sh = __float2half_rn(s32);
+                    if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);   // saturate, never infinite
+                    const float sc = __half2float(sh);
+                    // code = clamp(rint(x * (1/s)), -7, 7) + 8.  Clamping first gives the same integer (the bounds are
+                    // integers), and adding 1.5 * 2^23 + 8 to a value in [-7, 7] rounds it to the nearest integer, ties
+                    // to even, leaving code in the low 4 bits of the sum.  s == 0 means every value is zero: 1/s is
+                    // replaced by 0 and all codes come out 8.
+                    const float inv = sc == 0.0f ? 0.0f : __fdiv_rn(1.0f, sc);
+                    // The sums are kept as bit patterns, 0x4B400000 + code, and packed by multiply-adds (a nibble per
+                    // step, from the top one down) instead of mask, shift and or per code: the constant upper bits add
+                    // up to a known word that is taken off at the end (K words, modulo 2^32) or fall outside the result
+                    // (V half-words).  A normal, unsaturated fp16 scale is within 2^-11 of amax / 7, so |x / s| < 7.01
+                    // and the clamp cannot bite: it is only kept for subnormal scales (rounded coarsely) and the
+                    // saturated one.
+                    uint32_t raw[32];
+                    const uint32_t sbits = __half_as_ushort(sh);
+                    if (sbits >= 0x0400u && sbits < 0x7BFFu) {
+#pragma unroll
+                        for (int e = 0; e < 32; e++) {
+                            const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
+                            raw[e] = __float_as_uint(__fadd_rn(__fmul_rn(f, inv), 12582920.0f));
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; e++) {
+                            const float f = (e & 1) ? bf16_hi(xs[e >> 1]) : bf16_lo(xs[e >> 1]);
+                            const float cl = fminf(fmaxf(__fmul_rn(f, inv), -7.0f), 7.0f);
+                            raw[e] = __float_as_uint(__fadd_rn(cl, 12582920.0f));
+                        }
                     }
+                    if (!which) {
+                        constexpr uint32_t kRawWord = 0x4B400000u * 0x11111111u;   // what eight constant parts add up to
+#pragma unroll
+                        for (int t = 0; t < 4; t++) {  // the word of dims 32w + 8t .. +7
+                            uint32_t acc = raw[8 * t + 7];          // nibble n holds dim offset 2 (n & 3) + (n >> 2): low_k_nibble inverted
+#pragma unroll
+                            for (int n = 6; n >= 0; n--) acc = acc * 16u + raw[8 * t + 2 * (n & 3) + (n >> 2)];
+                            *reinterpret_cast<uint32_t *>(img + low_k_word_off(tau, w, t)) = acc - kRawWord;
+                        }
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < 8; g++) {  // the half-word of dims 32w + 4g .. +3
+                            const uint32_t acc = ((raw[4 * g + 3] * 16u + raw[4 * g + 2]) * 16u + raw[4 * g + 1]) * 16u + raw[4 * g];
+                            *reinterpret_cast<uint16_t *>(img + low_v_half_off(tau, w, g)) = (uint16_t)acc;
+                        }
+                        vmax_bits = max(vmax_bits, (uint32_t)__half_as_ushort(sh));
+                    }
+                    *reinterpret_cast<__half *>(img + low_scale_off(tau, w)) = sh;
                 }
-                uint8_t *img = s_low[head & 1] + (which ? kLowHalfBytes : 0);
-                if (!which) {
-                    constexpr uint32_t kRawWord = 0x4B400000u * 0x11111111u;   // what eight constant parts add up to
-#pragma unroll
-                    for (int u = 0; u < 2; u++) {  // the words of dims 32w + 8t .. +7, t = 2 half + u
-                        uint32_t acc = raw[8 * u + 7];          // nibble n holds dim offset 2 (n & 3) + (n >> 2): low_k_nibble inverted
-#pragma unroll
-                        for (int n = 6; n >= 0; n--) acc = acc * 16u + raw[8 * u + 2 * (n & 3) + (n >> 2)];
-                        *reinterpret_cast<uint32_t *>(img + low_k_word_off(tau, w, 2 * half + u)) = acc - kRawWord;
-                    }
-                } else {
-#pragma unroll
-                    for (int u = 0; u < 4; u++) {  // the half-words of dims 32w + 4g .. +3, g = 4 half + u
-                        const uint32_t acc = ((raw[4 * u + 3] * 16u + raw[4 * u + 2]) * 16u + raw[4 * u + 1]) * 16u + raw[4 * u];
-                        *reinterpret_cast<uint16_t *>(img + low_v_half_off(tau, w, 4 * half + u)) = (uint16_t)acc;
-                    }
-                    vmax_bits = max(vmax_bits, (uint32_t)__half_as_ushort(sh));
-                }
-                if (half == 0) *reinterpret_cast<__half *>(img + low_scale_off(tau, w)) = sh;
                 __syncthreads();
-                uint4 *dst = reinterpret_cast<uint4 *>(c.pool_low + (size_t)page * c.low_page_bytes + (size_t)head * kLowHeadBytes);
-                if (tid < kLowHeadBytes / 16) dst[tid] = reinterpret_cast<const uint4 *>(s_low[head & 1])[tid];
+                // the two packed heads leave; the next pair is assembled in the other two buffers meanwhile
+                for (int x = tid; x < 2 * (kLowHeadBytes / 16); x += kWriteThreads) {
+                    const int hh = x >= kLowHeadBytes / 16, r = hh ? x - kLowHeadBytes / 16 : x;
+                    if (hp + hh < c.n_kv)
+                        reinterpret_cast<uint4 *>(c.pool_low + (size_t)page * c.low_page_bytes + (size_t)(hp + hh) * kLowHeadBytes)[r] =
+                            reinterpret_cast<const uint4 *>(s_low[(hp & 2) + hh])[r];
+                }
             }
         }
         if (!high) {   // largest V scale of the stream (decode attention forms P * scale relative to it)
@@ -1161,7 +1226,7 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
         // at most one item per 16 tokens plus two partly filled pages per stream
         const long long bound = (long long)total_tokens / 16 + 4LL * n_seqs;
         const int ctas = bound < (long long)c->sm_count * 3 ? (int)bound : c->sm_count * 3;
-        const size_t smem = (size_t)c->desc.n_kv_heads * 2 * kPageTokens * kRowBytes;
+        const size_t smem = (size_t)2 * kPageTokens * (c->desc.n_kv_heads * 2 * kHeadDim + kRowPad);
         if (cudaFuncSetAttribute(append_write_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return PASK_ERR_CUDA;
         append_write_kernel<<<ctas, kWriteThreads, smem, stream>>>(c->dev, layer, n_seqs, static_cast<const uint4 *>(k),
