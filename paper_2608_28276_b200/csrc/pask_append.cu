@@ -12,7 +12,8 @@ namespace pask {
 
 namespace {
 
-constexpr int kPlanThreads = 256;
+constexpr int kPlanThreads = 256;      // threads of the one-launch append (and of its three-value scan)
+constexpr int kBulkThreads = 1024;     // threads of the bulk append's plan kernel: 4096 tokens of a sequence per round
 
 // Plan records are written by other CTAs of the same launch: read them through L2.
 __device__ __forceinline__ AppendPlan load_plan_cg(const AppendPlan *p) {
@@ -33,7 +34,7 @@ __device__ __forceinline__ uint32_t pages_touched(uint32_t old, uint32_t cnt) {
     return cnt ? ((old + cnt - 1) >> 4) - (old >> 4) + 1 : 0u;
 }
 
-// exclusive scan of one value per thread over a 256-thread block; returns the block total too
+// exclusive scan of one value per thread over a block of kBulkThreads; returns the block total too
 __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *s_warp, uint32_t *total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t inc = v;
@@ -46,7 +47,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *s_warp
     __syncthreads();
     uint32_t before = 0, tot = 0;
 #pragma unroll
-    for (int w = 0; w < kPlanThreads / 32; w++) {
+    for (int w = 0; w < kBulkThreads / 32; w++) {
         const uint32_t x = s_warp[w];
         if (w < warp) before += x;
         tot += x;
@@ -88,18 +89,18 @@ __device__ __forceinline__ void block_excl_scan3(uint32_t (&v)[3], uint32_t (*s_
 // per-sequence plan; the CTA that arrives last allocates pages for the whole call (exclusive scan
 // over sequences in call order, so ids do not depend on scheduling) and commits all counters --
 // or refuses the whole call.
-__global__ void __launch_bounds__(kPlanThreads)
+__global__ void __launch_bounds__(kBulkThreads)
 append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const int32_t *__restrict__ seq_ids,
                    const int32_t *__restrict__ cu_tokens, const uint8_t *__restrict__ tags,
                    const uint8_t *__restrict__ decided, uint8_t *__restrict__ actions_out) {
     __shared__ uint8_t s_lut[256];
-    __shared__ uint32_t s_wh[2 * (kPlanThreads / 32)], s_wb[2 * (kPlanThreads / 32)];
-    __shared__ uint32_t s_scan[kPlanThreads / 32];
+    __shared__ uint32_t s_wh[2 * (kBulkThreads / 32)], s_wb[2 * (kBulkThreads / 32)];
+    __shared__ uint32_t s_scan[kBulkThreads / 32];
     __shared__ uint32_t s_first_h[PASK_MAX_SEQS_PER_CALL], s_first_l[PASK_MAX_SEQS_PER_CALL];
     __shared__ int s_flag;
     const int i = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int group = c.layer_group[layer];
-    s_lut[tid] = tid < c.n_tags ? c.lut[tid * c.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
+    if (tid < 256) s_lut[tid] = tid < c.n_tags ? c.lut[tid * c.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
     // this launch's serial: every CTA reads it before its arrival ticket, the CTA arriving last stores it back
     uint32_t serial = c.ctrl[kCtrlSerial] + 1u;
     if (serial == 0) serial = 1;
@@ -124,7 +125,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
     uint32_t run_h = 0, run_l = 0, run_b = 0;
     if (!err) {
         int buf = 0;
-        for (int base = t0; base < t1; base += 4 * kPlanThreads, buf ^= 1) {
+        for (int base = t0; base < t1; base += 4 * kBulkThreads, buf ^= 1) {
             const int tb = base + 4 * tid;
             int a[4];
             uint32_t cnt = 0, nbad = 0;
@@ -150,15 +151,15 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
                 if (lane >= d) inc += o;
             }
             nbad = __reduce_add_sync(0xffffffffu, nbad);
-            if (lane == 31) { s_wh[buf * (kPlanThreads / 32) + warp] = inc; s_wb[buf * (kPlanThreads / 32) + warp] = nbad; }
+            if (lane == 31) { s_wh[buf * (kBulkThreads / 32) + warp] = inc; s_wb[buf * (kBulkThreads / 32) + warp] = nbad; }
             __syncthreads();
             uint32_t before = 0, tot = 0, tot_b = 0;
 #pragma unroll
-            for (int w = 0; w < kPlanThreads / 32; w++) {
-                const uint32_t x = s_wh[buf * (kPlanThreads / 32) + w];
+            for (int w = 0; w < kBulkThreads / 32; w++) {
+                const uint32_t x = s_wh[buf * (kBulkThreads / 32) + w];
                 if (w < warp) before += x;
                 tot += x;
-                tot_b += s_wb[buf * (kPlanThreads / 32) + w];
+                tot_b += s_wb[buf * (kBulkThreads / 32) + w];
             }
             const uint32_t excl = before + inc - cnt;
             uint32_t pos_h = run_h + (excl & 0xffffu), pos_l = run_l + (excl >> 16);
@@ -209,7 +210,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
 
     // ---- last CTA: allocate for the whole call and commit, or refuse
     __threadfence();
-    constexpr int kPer = PASK_MAX_SEQS_PER_CALL / kPlanThreads;  // sequences per thread, blocked
+    constexpr int kPer = PASK_MAX_SEQS_PER_CALL / kBulkThreads;  // sequences per thread, blocked
     uint32_t nh[kPer], nl[kPer], ni[kPer];
     uint32_t sum_h = 0, sum_l = 0, sum_i = 0;
     int any_bad = 0;
@@ -277,7 +278,7 @@ append_plan_kernel(DevCache c, int layer, int n_seqs, int total_tokens, const in
     // page tables: a warp per sequence, its lanes over the sequence's new pages (a prefill hands
     // out hundreds of pages per sequence)
     __syncthreads();
-    for (int j = warp; j < n_seqs; j += kPlanThreads / 32) {
+    for (int j = warp; j < n_seqs; j += kBulkThreads / 32) {
         const AppendPlan p = load_plan_cg(&c.plan[j]);
         const size_t sl = (size_t)p.seq * c.n_layers + layer;
         const uint32_t ph0 = (p.old_high + kPageTokens - 1) / kPageTokens, pl0 = (p.old_low + kPageTokens - 1) / kPageTokens;
@@ -1220,7 +1221,7 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
                                          fuse ? *fuse_ws : Workspace{}, (int32_t *)nullptr, 0);
         return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
     }
-    append_plan_kernel<<<n_seqs, kPlanThreads, 0, stream>>>(c->dev, layer, n_seqs, total_tokens, seq_ids, cu_tokens, tags,
+    append_plan_kernel<<<n_seqs, kBulkThreads, 0, stream>>>(c->dev, layer, n_seqs, total_tokens, seq_ids, cu_tokens, tags,
                                                            decided, actions_out);
     if (total_tokens > 0) {
         // at most one item per 16 tokens plus two partly filled pages per stream
