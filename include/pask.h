@@ -471,8 +471,9 @@ pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, c
  * SM).  Any value >= 1 gives the same result up to summation order; tests use it to check that.
  * Workspaces must be sized (pask_workspace_bytes) after the change. */
 pask_status_t pask_debug_set_attention_ctas(pask_cache_t *cache, int32_t n_ctas);
-/* The only device-side waits of the library are those of the decode-attention kernel for its bulk
- * copies into shared memory.  Each is bounded: after `limit_cycles` SM clock cycles (default 2e9,
+/* The device-side waits of the library are those of the decode-attention kernel for its bulk copies
+ * into shared memory (and one of the same kind, with a fixed bound of about a second, in the bulk
+ * append's write kernel for a page's source rows).  Each is bounded: after `limit_cycles` SM clock cycles (default 2e9,
  * about a second) the warp gives up, sets PASK_DEV_TIMEOUT, writes empty partials for the rest of
  * its range, waits (bounded again) until every copy it had issued has landed, and returns; the
  * context stays usable and pask_cache_reset clears the bit.  pask_debug_set_wait sets the limit

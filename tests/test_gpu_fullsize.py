@@ -26,22 +26,32 @@ LAYERS = (0, 9, 18, 35)
 SEQS = (0, 17, 42, 63)
 
 
-def test_full_size_decode_step_sampled_against_oracle(oracle):
+@pytest.mark.parametrize("mode", ["ahead", "fused"])
+def test_full_size_decode_step_sampled_against_oracle(oracle, mode):
     import bench
     import paper_2608_28276_b200 as P
     dev = torch.device("cuda", 0)
     cfg = WC.scaled(WC.QWEN3_4B_STEP, extra_gen=16)
     w = WC.build(cfg)
-    job = bench.Job(P, w, dev, 4)
+    job = bench.Job(P, w, dev, 6)
     job.fill()
-    job.prepare_steps(1)
+    # "ahead": the call bench.py times by default -- planned-ahead steps; three of them, so that the last one streams from
+    # a plan written by the step before and sets its pipeline up ahead of its dependency wait.  "fused": one
+    # pask_append_attend per layer (the append launch carries the plan), bench.py --no-ahead.
+    n_steps = 3 if mode == "ahead" else 1
+    job.prepare_steps(n_steps)
+    if mode == "ahead":
+        job.plan_ahead()
     outs = {}
     h = job.cache.handle
-    for layer, (k, v, q, tags) in enumerate(job.steps[0]):          # one decode step, keeping sampled outputs
-        # the call bench.py times: a layer's append + attention in one (the append launch carries the plan)
-        P.pask_append_attend(h, layer, job.ids, job.cu1, k, v, tags, q, job.out, job.lse, job.ws)
-        if layer in LAYERS:
-            outs[layer] = (job.out.cpu().numpy().astype(np.float64), job.lse.cpu().numpy().astype(np.float64))
+    for step in range(n_steps):
+        for layer, (k, v, q, tags) in enumerate(job.steps[step]):      # whole decode steps, keeping the last one's sampled outputs
+            if mode == "ahead":
+                P.pask_decode_step_ahead(h, layer, job.ids, k, v, tags, q, job.out, job.lse, job.ws, job.area)
+            else:
+                P.pask_append_attend(h, layer, job.ids, job.cu1, k, v, tags, q, job.out, job.lse, job.ws)
+            if layer in LAYERS and step == n_steps - 1:
+                outs[layer] = (job.out.cpu().numpy().astype(np.float64), job.lse.cpu().numpy().astype(np.float64))
     torch.cuda.synchronize()
     assert P.pask_budget_state(h, 0).device_status == 0
 
@@ -54,20 +64,22 @@ def test_full_size_decode_step_sampled_against_oracle(oracle):
     tags_hist = np.concatenate([w.tags(b, 0, n) for b, n in zip(SEQS, lens)])
     zeros = np.zeros((int(cu[-1]), cfg.n_kv, 128), np.uint16)
     zeros1 = np.zeros((len(SEQS), cfg.n_kv, 128), np.uint16)
+    one = np.arange(len(SEQS) + 1, dtype=np.int32)
     for layer in range(cfg.n_layers):
-        ks, vs, qs, st = bench.step_inputs(w, layer, 0, "cpu")
         if layer in LAYERS:
             k = torch.cat([normal_bf16(w.seed, TENSOR_K, layer, b, 0, n, cfg.n_kv, dev) for b, n in zip(SEQS, lens)]).cpu()
             v = torch.cat([normal_bf16(w.seed, TENSOR_V, layer, b, 0, n, cfg.n_kv, dev) for b, n in zip(SEQS, lens)]).cpu()
             rc, _ = orc.append(layer, ids, cu, bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags_hist)
-            assert rc == 0
-            rc, _ = orc.append(layer, ids, np.arange(len(SEQS) + 1, dtype=np.int32), bf16_bits(ks[list(SEQS)]).numpy(),
-                               bf16_bits(vs[list(SEQS)]).numpy(), st[list(SEQS)])
         else:
             rc, _ = orc.append(layer, ids, cu, zeros, zeros, tags_hist)
-            assert rc == 0
-            rc, _ = orc.append(layer, ids, np.arange(len(SEQS) + 1, dtype=np.int32), zeros1, zeros1, st[list(SEQS)])
         assert rc == 0
+        for step in range(n_steps):
+            ks, vs, qs, st = bench.step_inputs(w, layer, step, "cpu")
+            if layer in LAYERS:
+                rc, _ = orc.append(layer, ids, one, bf16_bits(ks[list(SEQS)]).numpy(), bf16_bits(vs[list(SEQS)]).numpy(), st[list(SEQS)])
+            else:
+                rc, _ = orc.append(layer, ids, one, zeros1, zeros1, st[list(SEQS)])
+            assert rc == 0
 
     # ---- budget states (all 36 layers of accounting), bit exact
     for i, b in enumerate(SEQS):
@@ -79,7 +91,7 @@ def test_full_size_decode_step_sampled_against_oracle(oracle):
 
     # ---- stored streams and attention on the sampled (layer, sequence) pairs
     for layer in LAYERS:
-        q = bench.step_inputs(w, layer, 0, "cpu")[2]
+        q = bench.step_inputs(w, layer, n_steps - 1, "cpu")[2]
         oo, ol = orc.attention_batch(layer, ids, bf16_bits(q[list(SEQS)]).numpy())
         go, gl = outs[layer]
         assert_close(go[list(SEQS)], gl[list(SEQS)], oo, ol, where=("full size", layer))
