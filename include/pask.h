@@ -319,7 +319,9 @@ pask_status_t pask_append_attend(pask_cache_t *cache, int32_t layer, int32_t n_s
  * recent window (the token that leaves the window changes what the history holds) or more than
  * 255 sequences: use pask_append_attend there.  A refused append (sticky PASK_DEV_* bit) leaves
  * out / lse undefined and an empty plan behind.  k, v, tags, actions, q must stay untouched
- * until the call's kernels have run, as for every call. */
+ * until the call's kernels have run, as for every call.  The calls only enqueue work and may be
+ * recorded by a stream capture; which of a layer's two plan blocks a call reads is fixed when it is
+ * recorded, so a graph that is replayed repeatedly must hold an even number of calls per layer. */
 size_t pask_plan_area_bytes(const pask_cache_t *cache, int32_t n_seqs);
 pask_status_t pask_plan_ahead(pask_cache_t *cache, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                               void *plan_area, size_t plan_area_bytes, pask_stream_t stream);

@@ -272,3 +272,64 @@ def test_one_layer_called_back_to_back(pask, oracle):
     for dev, out, lse, (oo, ol) in held:
         assert_close(out.cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64), oo, ol)
     p.compare_state()
+
+
+def test_two_steps_ahead_replayed_as_a_cuda_graph(pask, oracle):
+    # Planned-ahead calls only enqueue work, so a stream capture can record them.  Which of a layer's two plan blocks a
+    # call reads is fixed when it is recorded, so a graph that is replayed over and over must hold an even number of
+    # steps: here two steps of every layer, replayed four times on new inputs.
+    p, w = _pair(pask, oracle, 6, 120, 60)
+    seqs = [2, 5, 0, 3, 1, 4]
+    lens = [w.total_len(s) - 5 * i for i, s in enumerate(seqs)]
+    L, d = w.cfg.n_layers, "cuda"
+    for layer in range(L):
+        p.append(layer, seqs, lens, [0] * 6)
+    h = p.gpu.handle
+    ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+    area = torch.empty(pask.pask_plan_area_bytes(h, 6), dtype=torch.uint8, device=d)
+    ws = p.gpu.workspace(6)
+    mk = lambda shape, dt: [[torch.zeros(shape, dtype=dt, device=d) for _ in range(L)] for _ in range(2)]
+    ks, vs = mk((6, w.cfg.n_kv, 128), torch.bfloat16), mk((6, w.cfg.n_kv, 128), torch.bfloat16)
+    qs, outs = mk((6, w.cfg.n_q, 128), torch.bfloat16), mk((6, w.cfg.n_q, 128), torch.float32)
+    lses, tgs = mk((6, w.cfg.n_q), torch.float32), mk((6,), torch.uint8)
+    # first use of every kernel outside the capture, on a throw-away cache
+    warm, _ = _pair(pask, oracle, 6, 120, 60)
+    warm_area = torch.empty_like(area)
+    pask.pask_plan_ahead(warm.gpu.handle, 0, ids, warm_area)
+    pask.pask_decode_step_ahead(warm.gpu.handle, 0, ids, ks[0][0], vs[0][0], tgs[0][0], qs[0][0], outs[0][0], lses[0][0],
+                                warm.gpu.workspace(6), warm_area)
+    for layer in range(L):
+        pask.pask_plan_ahead(h, layer, ids, area)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for half in range(2):
+                for layer in range(L):
+                    pask.pask_decode_step_ahead(h, layer, ids, ks[half][layer], vs[half][layer], tgs[half][layer], qs[half][layer],
+                                                outs[half][layer], lses[half][layer], ws, area)
+    torch.cuda.current_stream().wait_stream(side)
+    pos = list(lens)
+    for rep in range(4):
+        want = [[None] * L for _ in range(2)]
+        for half in range(2):
+            for layer in range(L):
+                tags, _, k, v = p.gather(seqs, [1] * 6, pos, layer)
+                q = torch.stack([w.q(layer, s, t + 1) for s, t in zip(seqs, pos)])
+                ks[half][layer].copy_(k); vs[half][layer].copy_(v); qs[half][layer].copy_(q)
+                tgs[half][layer].copy_(torch.from_numpy(tags))
+                rc, _ = p.orc.append(layer, seqs, list(range(7)), bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags)
+                assert rc == 0
+                want[half][layer] = p.orc.attention_batch(layer, seqs, bf16_bits(q).numpy())
+            pos = [x + 1 for x in pos]
+        graph.replay()
+        torch.cuda.synchronize()
+        for half in range(2):
+            for layer in range(L):
+                oo, ol = want[half][layer]
+                assert_close(outs[half][layer].cpu().numpy().astype(np.float64), lses[half][layer].cpu().numpy().astype(np.float64),
+                             oo, ol, where=(rep, half, layer))
+    p.compare_state()
+    assert pask.pask_budget_state(h, 0).device_status == 0
