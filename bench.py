@@ -122,6 +122,16 @@ def kernel_events(n_layers, n_steps, stride):
     return evs
 
 
+def kernel_spans(n_layers, n_steps, stride, device):
+    """Device words for the in-kernel timing of launches that carry NO events (so that they overlap their launch
+    with their neighbours as in the un-timed step): per step {layer: int64[2] preset to (all ones, 0)}."""
+    out = []
+    for s in range(n_steps):
+        out.append({l: torch.tensor([-1, 0], dtype=torch.int64, device=device)
+                    for l in range(n_layers) if (l + s) % stride == stride // 2 and stride > 1})
+    return out
+
+
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons sampled every 20 ms while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -293,14 +303,17 @@ class Job:
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
 
-    def run_step(self, s, events=None):
-        """events: {layer: (start, stop)} for the launches of this step whose streaming kernel is timed."""
+    def run_step(self, s, events=None, spans=None):
+        """events: {layer: (start, stop)} for the launches of this step whose streaming kernel is timed;
+        spans: {layer: int64[2]} for those that time themselves from inside (pask_cache_set_timing_span)."""
         P, h = self.P, self.cache.handle
         if self.dynamic:       # Algorithm 2 steps 1-6 once per token, then step 7 layer by layer
             P.pask_decide(h, self.ids, self.cu1, self.steps[s][0][3], self.step_states[s], self.decided)
         for layer, (k, v, q, tags) in enumerate(self.steps[s]):
             if events is not None and layer in events:
                 P.pask_cache_set_timing_events(h, *events[layer])
+            if spans is not None and layer in spans:
+                P.pask_cache_set_timing_span(h, spans[layer])
             if self.ahead:     # streaming from the plan made a step ahead, the append beside it
                 P.pask_decode_step_ahead(h, layer, self.ids, k, v, tags, q, self.out, self.lse, self.ws, self.area,
                                          actions=self.decided if self.dynamic else None)
@@ -356,6 +369,7 @@ class Runner:
     def block(self, job, first_step, n_steps, with_events=True, graph=False):
         """One timed block; returns (ms of the block, [ms of each timed streaming-kernel launch])."""
         evs = kernel_events(job.cfg.n_layers, n_steps, self.args.event_stride) if (with_events and not graph) else None
+        sps = kernel_spans(job.cfg.n_layers, n_steps, self.args.event_stride, self.device) if evs else None
         self.barrier()
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0.record()
@@ -363,11 +377,14 @@ class Runner:
             if graph:
                 job.graphs[first_step + i].replay()
             else:
-                job.run_step(first_step + i, evs[i] if evs else None)
+                job.run_step(first_step + i, evs[i] if evs else None, sps[i] if sps else None)
         t1.record()
         self.barrier()
         ms = max_over_ranks(t0.elapsed_time(t1), self.device)
         kern = [a.elapsed_time(b) for row in (evs or []) for a, b in row.values()]
+        # in-kernel spans (ns of the GPU's global timer) of launches that carried no events
+        self.last_spans_ms = [float(v[1] - v[0]) * 1e-6 for row in (sps or []) for v in (t.tolist() for t in row.values())
+                              if v[1] > 0 and v[0] > 0]
         return ms, kern
 
 
@@ -415,12 +432,17 @@ def quick_point(P, runner, cfg, device, steps, peak, repeat=0, policy_blob=None,
     ret = sum(P.pask_budget_state(job.cache.handle, b).retained_bytes for b in range(job.B))
     full = sum(P.pask_budget_state(job.cache.handle, b).full_bytes for b in range(job.B))
     fig = kernel_figures(job, kern, warm + steps // 2, peak)
+    spans = runner.last_spans_ms
     out = {"workload": cfg.name, "kernel": label, "batch": job.B, "layers": cfg.n_layers, "kv_budget_target": cfg.budget,
            "kv_budget_realised": ret / full, "table": f"{cfg.lut}/{cfg.bias}", "steps": steps, "warmup": warm,
            "tokens_per_s": job.B * steps / (ms * 1e-3), "ms_per_step": ms / steps,
            "kernel_GBs": fig["achieved"], "frac": fig["frac"], "frac_of_nominal_8TBs": fig.get("frac_of_nominal_8TBs"),
            "avg_launch_ms": fig["avg_launch_ms"], "algorithmic_bytes_per_launch": fig["algorithmic_bytes_per_launch"],
            "clocks": clocks, "setup_s": round(t_setup, 1)}
+    if spans:      # the kernel timed from inside on launches without events (see roofline.in_kernel of the headline)
+        sp = sum(spans) / len(spans)
+        out["in_kernel_span_ms"] = sp
+        out["in_kernel_frac"] = fig["algorithmic_bytes_per_launch"] / (sp * 1e-3) / 1e9 / peak
     if len(job.fill_ms) > 1:
         out["bulk_append_ms_per_layer_call"] = sum(job.fill_ms[1:]) / (len(job.fill_ms) - 1)
         out["tokens_in_cache"] = job.total_tokens
@@ -523,11 +545,12 @@ def run_cuda(args, rank, world):
     if rank == 0:
         sampler.start()
     # the timed region, `repeats` times over: each block is exactly --steps steps between two barriers
-    blocks, kern_ms, kern_by_block = [], [], []
+    blocks, kern_ms, kern_by_block, span_ms = [], [], [], []
     for r in range(repeats):
         ms, kern = runner.block(job, args.warmup + r * args.steps, args.steps, graph=args.graph)
         blocks.append(ms)
         kern_ms += kern
+        span_ms += runner.last_spans_ms
         kern_by_block.append(sum(kern) / len(kern) if kern else None)
     clocks = sampler.stop() if rank == 0 else {}
     check_status(P, job, "after the timed region")
@@ -573,6 +596,13 @@ def run_cuda(args, rank, world):
                                         f"{NCU_TRAFFIC_PROFILE} (a 4-layer cut of this workload)") if covered else
                                        "no ncu capture covers this configuration"},
     }
+    if span_ms and line["roofline"]:
+        sp = sum(span_ms) / len(span_ms)
+        line["roofline"]["in_kernel"] = {
+            "avg_span_ms": sp, "launches": len(span_ms), "achieved": alg / (sp * 1e-3) / 1e9, "frac": alg / (sp * 1e-3) / 1e9 / peak,
+            "what": "the same kernel timed from inside (pask_cache_set_timing_span: first CTA released -> last CTA done, GPU "
+                    "global timer) on launches of the timed region that carry no events and so keep their launch overlap; "
+                    "the event figure above adds the launch and completion latency around a kernel that stands alone"}
     if fig["avg_launch_ms"]:
         k_ms = fig["avg_launch_ms"]
         line["attention_share_of_step"] = k_ms * cfg.n_layers * args.steps / ms

@@ -437,6 +437,15 @@ pask_status_t pask_budget_state(pask_cache_t *cache, int32_t seq, pask_budget_st
  * and `stop` just after its main (page-streaming) kernel on the call's stream, then forgets
  * them.  Pass NULLs to clear. */
 pask_status_t pask_cache_set_timing_events(pask_cache_t *cache, pask_event_t start, pask_event_t stop);
+/* The same from inside the kernel: the streaming kernel of the next decode-attention call on this
+ * cache (any flavour) leaves in span_dev[0] the earliest time at which one of its CTAs was free to
+ * start its work (its dependency wait over) and in span_dev[1] the latest time at which one had
+ * finished, both in nanoseconds of the GPU's global timer (atomicMin / atomicMax: the caller sets
+ * the two 64-bit words to all ones and to zero beforehand; dev memory, 8-byte aligned).  Unlike the
+ * pair of events this does not keep the kernel from overlapping its launch with its neighbours,
+ * and it leaves out the launch and completion latency that a pair of events includes.  NULL
+ * cancels.  One launch only, like the events. */
+pask_status_t pask_cache_set_timing_span(pask_cache_t *cache, void *span_dev);
 
 /* ---------------------------------------------------------------------------------------------
  * Debug / test access to the cache in canonical form (the physical packing inside pages is

@@ -30,7 +30,7 @@ EXPORTS = [
     "pask_cache_destroy", "pask_cache_reset", "pask_seq_reset", "pask_append_kv", "pask_decide",
     "pask_append_kv_decided", "pask_append_attend", "pask_plan_area_bytes", "pask_plan_ahead", "pask_decode_step_ahead", "pask_decode_attention",
     "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes", "pask_step_packed_layout", "pask_decode_step_packed", "pask_decode_step_pipelined", "pask_decode_step_pipelined_ahead", "pask_decode_step_drain",
-    "pask_budget_state", "pask_distortion", "pask_cache_set_timing_events", "pask_debug_stream_len", "pask_debug_dump_high",
+    "pask_budget_state", "pask_distortion", "pask_cache_set_timing_events", "pask_cache_set_timing_span", "pask_debug_stream_len", "pask_debug_dump_high",
     "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_debug_set_wait", "pask_status_string",
 ]
 
@@ -107,6 +107,7 @@ _lib.pask_debug_ctrl_words.argtypes = [_vp, _vp, _i32, _vp]
 _lib.pask_debug_partition.argtypes = [_i32, _vp, _vp, _i32, _vp]
 _lib.pask_debug_page_order.argtypes = [C.c_uint32, C.c_uint32, _vp]
 _lib.pask_debug_set_attention_ctas.argtypes = [_vp, _i32]
+_lib.pask_cache_set_timing_span.argtypes = [_vp, _vp]
 _lib.pask_debug_set_wait.argtypes = [_vp, C.c_int64, C.c_uint32]
 _lib.pask_status_string.argtypes = [_i32]
 _lib.pask_status_string.restype = C.c_char_p
@@ -423,6 +424,12 @@ def pask_debug_page_order(pages_high: int, pages_low: int):
     out = np.zeros(pages_high + pages_low, np.uint32)
     _check(_lib.pask_debug_page_order(pages_high, pages_low, out.ctypes.data), "pask_debug_page_order")
     return (out >> 31).astype(bool), (out & 0x7FFFFFFF).astype(np.int64)
+
+
+def pask_cache_set_timing_span(cache: int, span):
+    """span: int64 device tensor [2] preset to (-1, 0) (all ones, zero), or None: the next streaming kernel leaves its
+    earliest CTA start and latest CTA end there (GPU global timer, ns)."""
+    _check(_lib.pask_cache_set_timing_span(cache, None if span is None else span.data_ptr()), "pask_cache_set_timing_span")
 
 
 def pask_debug_set_attention_ctas(cache: int, n_ctas: int):

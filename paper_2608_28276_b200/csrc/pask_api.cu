@@ -209,6 +209,7 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     c->meta = meta;
     c->sm_count = sms;
     c->ev_start = c->ev_stop = nullptr;
+    c->span = nullptr;
     c->ahead.resize((size_t)d->n_layers);
     c->wait_cycles = 2000000000LL;   // about one second: give up instead of hanging
     c->wait_test_surplus = 0;
@@ -685,6 +686,12 @@ pask_status_t pask_cache_set_timing_events(pask_cache_t *c, pask_event_t start, 
     if (!c) return PASK_ERR_INVALID_ARG;
     c->ev_start = static_cast<cudaEvent_t>(start);
     c->ev_stop = static_cast<cudaEvent_t>(stop);
+    return PASK_OK;
+}
+
+pask_status_t pask_cache_set_timing_span(pask_cache_t *c, void *span_dev) {
+    if (!c || ((uintptr_t)span_dev & 7)) return PASK_ERR_INVALID_ARG;
+    c->span = static_cast<unsigned long long *>(span_dev);
     return PASK_OK;
 }
 

@@ -54,6 +54,7 @@ struct AttnParams {
     Workspace ws;
     long long wait_cycles;  // bound of a wait for a bulk copy, in SM clock cycles
     uint32_t overpost;      // test aid: bytes announced beyond what a warp's first copy brings (0 in normal use)
+    unsigned long long *span;   // optional: {earliest CTA start, latest CTA end} of this launch in %globaltimer ns, else null
     int early;              // the plan and the pages were written before the kernel's predecessor in the stream started:
                             // range look-up and the first bulk copies need not wait for that predecessor
 };
@@ -62,6 +63,11 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---------------------------------------------------------------- PTX helpers
 
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -431,6 +437,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     if (!p.early) {
         pdl_wait();
         pdl_launch_dependents();   // only now: the combine kernel reads the plan's prefix before its own wait
+        if (p.span && tid == 0) atomicMin(p.span, globaltimer_ns());
     }
     for (int s = tid; s <= n_seqs; s += blockDim.x) {
         s_cost[s] = __ldg(p.ws.cost_prefix + s);
@@ -501,6 +508,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     if (p.early) {
         pdl_wait();
         pdl_launch_dependents();   // (the append that runs beside this kernel must not start before this wait is over)
+        if (p.span && tid == 0) atomicMin(p.span, globaltimer_ns());
     }
 
     const float kLog2Scale = 0.088388347648318440550f * 1.4426950408889634074f;  // log2(e) / sqrt(128)
@@ -874,6 +882,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         }
     }
 
+    if (p.span && lane == 0) atomicMax(p.span + 1, globaltimer_ns());
     // A wait gave up: copies may still be in flight towards this CTA's shared memory.  Give each
     // outstanding stage one more bounded wait before the CTA retires; the ring is not read again.
     if (w.dead) {
@@ -1123,10 +1132,12 @@ static cudaError_t launch_stream_kernel(pask_cache *c, bool has_low, AttnParams 
             have = smem;
         }
     }
+    p.span = c->span;
     if (c->ev_start) cudaEventRecord(c->ev_start, stream);
     const cudaError_t e = launch_pdl(kern, dim3(c->attn_ctas), dim3(32 * n_warps), smem, stream, p);
     if (c->ev_stop) cudaEventRecord(c->ev_stop, stream);
     c->ev_start = c->ev_stop = nullptr;
+    c->span = nullptr;
     return e;
 }
 

@@ -134,6 +134,7 @@ struct pask_cache {
     int sm_count;
     int attn_ctas;                // grid of the decode-attention main kernel
     cudaEvent_t ev_start, ev_stop;
+    unsigned long long *span;     // pask_cache_set_timing_span: where the next streaming kernel leaves its start and end
     // planned-ahead decode steps: which layers hold a plan, for how many sequences, in which area, and which of the
     // layer's two plan blocks is the current one
     struct Ahead {

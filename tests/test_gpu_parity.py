@@ -443,3 +443,20 @@ def test_pipelined_host_steps_with_a_batch_that_changes_from_call_to_call(pask, 
     with pytest.raises(P.PaskError) as e:
         P.pask_decode_step_pipelined(h, 0, 6, calls[0][0], calls[0][1], small, p.gpu.workspace(6))
     assert e.value.status == P.ERR_WORKSPACE
+
+
+def test_the_streaming_kernel_times_itself_on_request(pask, oracle):
+    # pask_cache_set_timing_span: the next streaming kernel leaves its earliest start and latest end (GPU global timer);
+    # one launch only, results unaffected
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=3, n_layers=1, n_groups=1, prompt_len=300, gen_len=100)
+    w = WC.build(cfg)
+    p = Pair(pask, oracle, w)
+    seqs = [0, 1, 2]
+    p.append(0, seqs, [400] * 3, [0] * 3)
+    span = torch.tensor([-1, 0], dtype=torch.int64, device="cuda")
+    pask.pask_cache_set_timing_span(p.gpu.handle, span)
+    p.check_attention(0, seqs)
+    a, b = span.tolist()
+    assert 0 < a < b and b - a < 10_000_000            # a few microseconds, in nanoseconds
+    p.check_attention(0, seqs)                          # the request was for one launch
+    assert span.tolist() == [a, b]
