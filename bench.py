@@ -539,13 +539,14 @@ def run_cuda(args, rank, world):
     t_setup = time.time()
     job = Job(P, w, device, 2 * total_steps + e2e_steps + e2e_warm + 4, dynamic=args.dynamic)
     job.fused = not args.unfused
-    # launches per layer: append (+ plan), streaming kernel, combine
-    per_layer_launches = 3 if (job.fused and job.B <= 255) else 4
     job.fill()
     job.prepare_steps(total_steps)
     use_ahead = args.ahead and job.fused and job.B <= 255 and not args.window
     if use_ahead:
         job.plan_ahead()
+    # launches per layer: planned-ahead step = streaming kernel + the kernel that ends the step (append and merge);
+    # pask_append_attend = append (+ plan), streaming kernel, combine; the two separate calls = four
+    per_layer_launches = 2 if use_ahead else 3 if (job.fused and job.B <= 255) else 4
     t_setup = time.time() - t_setup
     ret = sum(P.pask_budget_state(job.cache.handle, b).retained_bytes for b in range(job.B))
     full = sum(P.pask_budget_state(job.cache.handle, b).full_bytes for b in range(job.B))

@@ -7,6 +7,7 @@
 #include <cuda_fp16.h>
 
 #include "pask_internal.h"
+#include "pask_merge.h"
 
 namespace pask {
 
@@ -777,7 +778,7 @@ append_small_body(const DevCache &c, int layer, int group, int n_seqs, int total
                   const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
                   const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided,
                   uint8_t *__restrict__ actions_out, const SmallLut &lut, const int fuse_plan, const Workspace &ws,
-                  int32_t *__restrict__ ids_out) {
+                  int32_t *__restrict__ ids_out, const uint32_t n_role) {   // n_role: the CTAs that run this body (one per token)
     __shared__ int s_seq[kSmallMax], s_cu[kSmallMax + 1];
     __shared__ uint32_t s_cost[kSmallMax + 1], s_page[kSmallMax + 1], s_nh[kSmallMax], s_nl[kSmallMax];   // fused attention plan
     __shared__ uint32_t s_old_n[kSmallMax], s_nw[kSmallMax], s_wstart[kSmallMax], s_wlen[kSmallMax];
@@ -861,7 +862,7 @@ append_small_body(const DevCache &c, int layer, int group, int n_seqs, int total
     if (s_err) {   // every CTA sees the same; the last one to get here resets the arrival counter
         if (tid == 0) {
             atomicOr(&c.ctrl[kCtrlStatus], s_err);
-            if (atomicAdd(&c.ctrl[kCtrlTicket], 1u) == gridDim.x - 1) { c.ctrl[kCtrlPlanOk] = 0; c.ctrl[kCtrlTicket] = 0; }
+            if (atomicAdd(&c.ctrl[kCtrlTicket], 1u) == n_role - 1) { c.ctrl[kCtrlPlanOk] = 0; c.ctrl[kCtrlTicket] = 0; }
         }
         if (fuse_plan && blockIdx.x == 0 && tid <= n_seqs) ws.cost_prefix[tid] = ws.page_prefix[tid] = 0;   // nothing to attend
         return;
@@ -1005,7 +1006,7 @@ append_small_body(const DevCache &c, int layer, int group, int n_seqs, int total
         }
         // the page-order list, a sequence at a time (CTA b takes sequences b, b + grid, ...): up to four entries per
         // thread and round, the page-table (or free-stack) reads of a round all in flight together
-        for (int s = blockIdx.x; s < n_seqs; s += gridDim.x) {
+        for (int s = blockIdx.x; s < n_seqs; s += (int)n_role) {
             const uint32_t nh = s_nh[s], nl = s_nl[s], nw = s_nw[s];
             const uint32_t ph = (nh + kPageTokens - 1) / kPageTokens, pl = (nl + kPageTokens - 1) / kPageTokens;
             const uint32_t pw = (nw + kPageTokens - 1) / kPageTokens;
@@ -1080,7 +1081,7 @@ append_small_body(const DevCache &c, int layer, int group, int n_seqs, int total
         }
     }
     __syncthreads();
-    if (tid == 0) s_last = atomicAdd(&c.ctrl[kCtrlTicket], 1u) == gridDim.x - 1;   // every read of the old state is done
+    if (tid == 0) s_last = atomicAdd(&c.ctrl[kCtrlTicket], 1u) == n_role - 1;   // every read of the old state is done
     __syncthreads();
     if (s_err) {
         if (tid == 0) {
@@ -1133,23 +1134,36 @@ append_small_body(const DevCache &c, int layer, int group, int n_seqs, int total
     }
 }
 
-// Normally the kernel waits for its predecessor in the stream before it reads anything.  With late_wait it does not:
-// it is then launched behind a kernel that needs none of its results and touches nothing it writes (the decode-
-// attention kernel of the same layer, working from a plan of the cache before this append), runs in the shadow of
-// that kernel's tail, and waits for it only before it retires, so that whoever comes next in the stream and waits
-// for this kernel has waited for both.  (Everything before that predecessor is complete: it has done its own wait
-// before it let this kernel start.)
 __global__ void __launch_bounds__(kSmallThreads)
 append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, const int32_t *__restrict__ seq_ids,
                     const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
                     const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided,
-                    uint8_t *__restrict__ actions_out, const SmallLut lut, const int fuse_plan, const Workspace ws,
-                    int32_t *__restrict__ ids_out, const int late_wait) {
+                    uint8_t *__restrict__ actions_out, const SmallLut lut, const int fuse_plan, const Workspace ws) {
     pdl_launch_dependents();
-    if (!late_wait) pdl_wait();
+    pdl_wait();
     append_small_body(c, layer, group, n_seqs, total, seq_ids, cu_tokens, k, v, tags, decided, actions_out, lut, fuse_plan, ws,
-                      ids_out);
-    if (late_wait) pdl_wait();
+                      nullptr, gridDim.x);
+}
+
+// The kernel that ends a planned-ahead decode step.  Its first n_seqs CTAs run the one-launch append (one token per
+// sequence) WITHOUT waiting for the kernel before them in the stream: that is the decode-attention kernel of the same
+// layer, which works from a plan of the cache before this append, needs none of its results and touches nothing it
+// writes, so the append runs in the shadow of that kernel's tail.  (Everything before that predecessor is complete:
+// it has done its own wait before it let this kernel start.)  Every CTA then waits for the predecessor and merges
+// its partials, the new tokens included -- so whoever comes next in the stream and waits for this kernel has waited
+// for both.
+__global__ void __launch_bounds__(kSmallThreads)
+step_tail_kernel(DevCache c, int layer, int group, int n_seqs, const int32_t *__restrict__ seq_ids,
+                 const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
+                 const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided, uint8_t *__restrict__ actions_out,
+                 const SmallLut lut, const Workspace plan_ws, int32_t *__restrict__ ids_out, const uint32_t *__restrict__ prefix,
+                 const float2 *__restrict__ part_ml, const float *__restrict__ part_o, float *__restrict__ out,
+                 float *__restrict__ lse, int n_q, uint32_t n_ctas, const NewTokens nt) {
+    pdl_launch_dependents();
+    if ((int)blockIdx.x < n_seqs)
+        append_small_body(c, layer, group, n_seqs, n_seqs, seq_ids, cu_tokens, k, v, tags, decided, actions_out, lut, 1, plan_ws,
+                          ids_out, (uint32_t)n_seqs);
+    merge_rows_with_new_token(prefix, part_ml, part_o, out, lse, n_seqs, n_q, n_ctas, nt, lut);
 }
 
 // General path, recent window: CTA (j, y) copies the y-th newest of sequence j's tokens in this call
@@ -1218,7 +1232,7 @@ pask_status_t launch_append(pask_cache *c, int layer, int n_seqs, int total_toke
         const cudaError_t e = launch_pdl(append_small_kernel, dim3(total_tokens), dim3(kSmallThreads), 0, stream, c->dev, layer,
                                          group, n_seqs, total_tokens, seq_ids, cu_tokens, static_cast<const uint4 *>(k),
                                          static_cast<const uint4 *>(v), tags, decided, actions_out, lut, fuse,
-                                         fuse ? *fuse_ws : Workspace{}, (int32_t *)nullptr, 0);
+                                         fuse ? *fuse_ws : Workspace{});
         return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
     }
     append_plan_kernel<<<n_seqs, kBulkThreads, 0, stream>>>(c->dev, layer, n_seqs, total_tokens, seq_ids, cu_tokens, tags,
@@ -1245,15 +1259,18 @@ void fill_small_lut(const pask_cache *c, int layer, SmallLut *lut) {
         lut->action[z] = z < c->dev.n_tags ? c->lut[(size_t)z * c->dev.n_groups + group] : (uint8_t)PASK_ACTION_RETAIN_HIGH;
 }
 
-pask_status_t launch_append_beside(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,
-                                   const void *k, const void *v, const uint8_t *tags, const uint8_t *decided,
-                                   uint8_t *actions_out, const Workspace &plan_ws, int32_t *ids_out, cudaStream_t stream) {
+pask_status_t launch_step_tail(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,
+                               const void *k, const void *v, const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out,
+                               const Workspace &plan_ws, int32_t *ids_out, const uint32_t *prefix, const float2 *part_ml,
+                               const float *part_o, float *out, float *lse, const NewTokens &nt, cudaStream_t stream) {
     if (n_seqs < 1 || n_seqs > kSmallMax) return PASK_ERR_UNSUPPORTED_SHAPE;
     SmallLut lut;
     fill_small_lut(c, layer, &lut);
-    const cudaError_t e = launch_pdl(append_small_kernel, dim3(n_seqs), dim3(kSmallThreads), 0, stream, c->dev, layer,
-                                     (int)c->layer_group[layer], n_seqs, n_seqs, seq_ids, cu_tokens, static_cast<const uint4 *>(k),
-                                     static_cast<const uint4 *>(v), tags, decided, actions_out, lut, 1, plan_ws, ids_out, 1);
+    const int n_q = c->desc.n_q_heads, merge_ctas = (n_seqs * n_q + 7) / 8;      // one warp per (sequence, query head)
+    const cudaError_t e = launch_pdl(step_tail_kernel, dim3(merge_ctas > n_seqs ? merge_ctas : n_seqs), dim3(kSmallThreads), 0,
+                                     stream, c->dev, layer, (int)c->layer_group[layer], n_seqs, seq_ids, cu_tokens,
+                                     static_cast<const uint4 *>(k), static_cast<const uint4 *>(v), tags, decided, actions_out, lut,
+                                     plan_ws, ids_out, prefix, part_ml, part_o, out, lse, n_q, (uint32_t)c->attn_ctas, nt);
     return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }
 

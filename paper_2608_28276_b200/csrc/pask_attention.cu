@@ -35,6 +35,7 @@
 #include <cuda_fp16.h>
 
 #include "pask_internal.h"
+#include "pask_merge.h"
 
 namespace pask {
 
@@ -913,13 +914,16 @@ combine_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ p
     uint32_t p0 = 0, p1 = 0;
     uint64_t total = 0;
     if (wid < n_seqs * n_q) { p0 = __ldg(prefix + s); p1 = __ldg(prefix + s + 1); total = __ldg(prefix + n_seqs); }
+    uint32_t b_first = 1, b_last = 0;       // the CTAs that hold partials of this sequence (two 64-bit divisions, ahead of the wait)
+    if (p1 > p0) {
+        b_first = (uint32_t)((((uint64_t)p0 + 1) * n_ctas - 1) / total);
+        b_last = (uint32_t)(((uint64_t)p1 * n_ctas - 1) / total);
+    }
     pdl_wait();
     if (wid >= n_seqs * n_q) return;
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
     float M = -INFINITY, L = 0.f;
     if (p1 > p0) {
-        const uint32_t b_first = (uint32_t)((((uint64_t)p0 + 1) * n_ctas - 1) / total);
-        const uint32_t b_last = (uint32_t)(((uint64_t)p1 * n_ctas - 1) / total);
         // online merge, eight partials per round trip
         for (uint32_t b = b_first; b <= b_last; b += 8) {
             float2 ml[8];
@@ -942,122 +946,6 @@ combine_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ p
                 M = Mn;
             }
         }
-    }
-    const size_t orow = (size_t)s * n_q + h;
-    if (L > 0.f) {
-        const float inv = 1.0f / L;
-        o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
-    }
-    *reinterpret_cast<float4 *>(out + orow * kHeadDim + lane * 4) = o;
-    if (lse && lane == 0) lse[orow] = L > 0.f ? (M + log2f(L)) * 0.69314718055994530942f : -INFINITY;
-}
-
-// What the merge kernel of a planned-ahead step needs to attend each sequence's new token from the call's inputs.
-struct NewTokens {
-    const uint2 *k, *v;            // bf16 [n_seqs][n_kv][128] viewed as 8-byte pieces (4 dims)
-    const uint2 *q;                // bf16 [n_seqs][n_q][128]
-    const uint8_t *tags;           // [n_seqs]
-    const uint8_t *decided;        // [n_seqs][n_groups] or null
-    const int32_t *seq_ids, *planned_ids;   // this call's list and the one the plan was made for
-    uint32_t *status;
-    int group, n_groups, n_kv, low_bits;
-};
-
-// Partial (m, l = 1, o = v) of one new token for one query head: the token at the precision it is stored at.
-// lane = 4 consecutive head dims; a 32-dim group is 8 adjacent lanes.
-__device__ __forceinline__ void quantise_like_append(float (&x)[4], int low_bits) {
-    float amax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
-    const float qmax = low_bits == 8 ? 127.0f : low_bits == 2 ? 1.0f : 7.0f;
-    __half sh = __float2half_rn(low_bits == 2 ? amax : __fdiv_rn(amax, qmax));
-    if (__hisinf(sh)) sh = __ushort_as_half((unsigned short)0x7BFF);
-    const float s = __half2float(sh);
-    const float inv = s == 0.0f ? 0.0f : __fdiv_rn(1.0f, s);
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-        float r = rintf(__fmul_rn(x[i], inv));
-        r = fminf(fmaxf(r, -qmax), qmax);
-        x[i] = __fmul_rn(r, s);          // (code - zero) * scale, exact
-    }
-}
-
-// Merge kernel of a planned-ahead step: the partials of the history (streamed from the plan of the cache before
-// this call's append) and, as one more partial, the sequence's new token taken from the call's k / v.
-__global__ void __launch_bounds__(256)
-combine_new_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ part_ml, const float *__restrict__ part_o,
-                   float *__restrict__ out, float *__restrict__ lse, int n_seqs, int n_q, uint32_t n_ctas, const NewTokens nt,
-                   const SmallLut lut) {
-    const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    pdl_launch_dependents();
-    const int s = wid / n_q, h = wid % n_q;
-    const bool mine = wid < n_seqs * n_q;
-    // everything that does not come from the kernels before is fetched ahead of the dependency wait
-    uint32_t p0 = 0, p1 = 0;
-    uint64_t total = 0;
-    int act = PASK_ACTION_RELEASE;
-    float kx[4] = {0.f, 0.f, 0.f, 0.f}, vx[4] = {0.f, 0.f, 0.f, 0.f}, qx[4] = {0.f, 0.f, 0.f, 0.f};
-    bool stale = false;
-    if (mine) {
-        p0 = __ldg(prefix + s); p1 = __ldg(prefix + s + 1); total = __ldg(prefix + n_seqs);
-        act = nt.decided ? nt.decided[(size_t)s * nt.n_groups + nt.group] : lut.action[nt.tags[s]];
-        if (act > PASK_ACTION_RETAIN_HIGH) act = PASK_ACTION_RELEASE;      // (the append refuses the call)
-        stale = nt.seq_ids[s] != nt.planned_ids[s];
-        if (act != PASK_ACTION_RELEASE) {
-            const int kv = h / (n_q / nt.n_kv);
-            const uint2 kw = nt.k[((size_t)s * nt.n_kv + kv) * 32 + lane], vw = nt.v[((size_t)s * nt.n_kv + kv) * 32 + lane];
-            const uint2 qw = nt.q[((size_t)s * n_q + h) * 32 + lane];
-            kx[0] = bf_lo(kw.x); kx[1] = bf_hi(kw.x); kx[2] = bf_lo(kw.y); kx[3] = bf_hi(kw.y);
-            vx[0] = bf_lo(vw.x); vx[1] = bf_hi(vw.x); vx[2] = bf_lo(vw.y); vx[3] = bf_hi(vw.y);
-            qx[0] = bf_lo(qw.x); qx[1] = bf_hi(qw.x); qx[2] = bf_lo(qw.y); qx[3] = bf_hi(qw.y);
-        }
-    }
-    float m_new = -INFINITY;
-    if (act == PASK_ACTION_RETAIN_LOW) { quantise_like_append(kx, nt.low_bits); quantise_like_append(vx, nt.low_bits); }
-    if (act != PASK_ACTION_RELEASE) {       // (warp-uniform: one sequence and head per warp)
-        float dot = fmaf(qx[0], kx[0], fmaf(qx[1], kx[1], fmaf(qx[2], kx[2], qx[3] * kx[3])));
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, d);
-        m_new = dot * (0.088388347648318440550f * 1.4426950408889634074f);      // log2 units, as the partials
-    }
-    if (stale && lane == 0 && h == 0) atomicOr(nt.status, PASK_DEV_STALE_PLAN);
-    pdl_wait();
-    if (!mine) return;
-    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-    float M = -INFINITY, L = 0.f;
-    if (p1 > p0) {
-        const uint32_t b_first = (uint32_t)((((uint64_t)p0 + 1) * n_ctas - 1) / total);
-        const uint32_t b_last = (uint32_t)(((uint64_t)p1 * n_ctas - 1) / total);
-        for (uint32_t b = b_first; b <= b_last; b += 8) {
-            float2 ml[8];
-            float4 v[8];
-#pragma unroll
-            for (int u = 0; u < 8; u++) {
-                const bool have = b + u <= b_last;
-                const size_t row = ((size_t)b + u + s) * n_q + h;
-                ml[u] = have ? part_ml[row] : make_float2(-INFINITY, 0.f);
-                v[u] = have ? *reinterpret_cast<const float4 *>(part_o + row * kHeadDim + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int u = 0; u < 8; u++) {
-                if (ml[u].x == -INFINITY) continue;
-                const float Mn = fmaxf(M, ml[u].x);
-                const float fo = exp2f(M - Mn), fn = exp2f(ml[u].x - Mn);
-                o.x = fmaf(fn, v[u].x, o.x * fo); o.y = fmaf(fn, v[u].y, o.y * fo);
-                o.z = fmaf(fn, v[u].z, o.z * fo); o.w = fmaf(fn, v[u].w, o.w * fo);
-                L = fmaf(fn, ml[u].y, L * fo);
-                M = Mn;
-            }
-        }
-    }
-    if (m_new != -INFINITY) {                // the new token: weight 1 at its own score
-        const float Mn = fmaxf(M, m_new);
-        const float fo = exp2f(M - Mn), fn = exp2f(m_new - Mn);
-        o.x = fmaf(fn, vx[0], o.x * fo); o.y = fmaf(fn, vx[1], o.y * fo);
-        o.z = fmaf(fn, vx[2], o.z * fo); o.w = fmaf(fn, vx[3], o.w * fo);
-        L = fmaf(fn, 1.0f, L * fo);
-        M = Mn;
     }
     const size_t orow = (size_t)s * n_q + h;
     if (L > 0.f) {
@@ -1209,9 +1097,10 @@ pask_status_t launch_plan_ahead(pask_cache *c, int layer, int n_seqs, const int3
 }
 
 // One layer of a planned-ahead decode step.  In stream order: the streaming kernel over the plan of the cache as
-// it was before this call; the one-launch append, which does not wait for that kernel (it needs nothing from it
-// and writes nothing it reads: slots past the planned token counts, table entries and counters the plan has
-// replaced, the other plan block) and so runs as its CTAs retire; the merge kernel, which waits for both.
+// it was before this call; then one kernel that ends the step: its first CTAs do the one-launch append, which does
+// not wait for the streaming kernel (it needs nothing from it and writes nothing it reads: slots past the planned
+// token counts, table entries and counters the plan has replaced, the other plan block) and so runs as that kernel's
+// CTAs retire; all of its CTAs then wait for the streaming kernel and merge its partials with the new tokens.
 pask_status_t launch_step_ahead(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const void *k, const void *v,
                                 const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out, const void *q, float *out,
                                 float *lse, void *workspace, void *area, int cur, bool early, cudaStream_t stream) {
@@ -1229,9 +1118,6 @@ pask_status_t launch_step_ahead(pask_cache *c, int layer, int n_seqs, const int3
     p.early = early ? 1 : 0;
     cudaError_t e = launch_stream_kernel(c, true, p, stream);
     if (e != cudaSuccess) return PASK_ERR_CUDA;
-    const pask_status_t rc = launch_append_beside(c, layer, n_seqs, seq_ids, static_cast<const int32_t *>(area), k, v, tags, decided,
-                                                  actions_out, plan_view(pn, Workspace{}), pn.ids, stream);
-    if (rc != PASK_OK) return rc;
     NewTokens nt;
     nt.k = static_cast<const uint2 *>(k);
     nt.v = static_cast<const uint2 *>(v);
@@ -1245,13 +1131,8 @@ pask_status_t launch_step_ahead(pask_cache *c, int layer, int n_seqs, const int3
     nt.n_groups = c->dev.n_groups;
     nt.n_kv = c->desc.n_kv_heads;
     nt.low_bits = (int)c->dev.low_bits;
-    SmallLut lut;
-    fill_small_lut(c, layer, &lut);
-    const int warps = n_seqs * c->desc.n_q_heads;
-    e = launch_pdl(combine_new_kernel, dim3((warps + 7) / 8), dim3(256), 0, stream, (const uint32_t *)pc.cost_prefix,
-                   (const float2 *)parts.part_ml, (const float *)parts.part_o, out, lse, n_seqs, (int)c->desc.n_q_heads,
-                   (uint32_t)c->attn_ctas, nt, lut);
-    return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
+    return launch_step_tail(c, layer, n_seqs, seq_ids, static_cast<const int32_t *>(area), k, v, tags, decided, actions_out,
+                            plan_view(pn, Workspace{}), pn.ids, pc.cost_prefix, parts.part_ml, parts.part_o, out, lse, nt, stream);
 }
 
 }  // namespace pask

@@ -208,11 +208,14 @@ pask_status_t launch_plan_ahead(pask_cache *c, int layer, int n_seqs, const int3
 pask_status_t launch_step_ahead(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const void *k, const void *v,
                                 const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out, const void *q, float *out,
                                 float *lse, void *workspace, void *area, int cur, bool early, cudaStream_t stream);
-// the one-launch append with its dependency wait moved to its end (it runs beside the kernel before it) and the
-// call's sequence list recorded next to the plan it writes
-pask_status_t launch_append_beside(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,
-                                   const void *k, const void *v, const uint8_t *tags, const uint8_t *decided,
-                                   uint8_t *actions_out, const Workspace &plan_ws, int32_t *ids_out, cudaStream_t stream);
+// the kernel that ends a planned-ahead step: the one-launch append (its first n_seqs CTAs; it writes the plan `plan_ws`
+// and the sequence list `ids_out`), then, behind the dependency wait, the merge of the streaming kernel's partials
+// with the new tokens
+struct NewTokens;
+pask_status_t launch_step_tail(pask_cache *c, int layer, int n_seqs, const int32_t *seq_ids, const int32_t *cu_tokens,
+                               const void *k, const void *v, const uint8_t *tags, const uint8_t *decided, uint8_t *actions_out,
+                               const Workspace &plan_ws, int32_t *ids_out, const uint32_t *prefix, const float2 *part_ml,
+                               const float *part_o, float *out, float *lse, const NewTokens &nt, cudaStream_t stream);
 struct SmallLut { uint8_t action[256]; };
 void fill_small_lut(const pask_cache *c, int layer, SmallLut *lut);
 size_t attention_workspace_bytes(const pask_cache *c, int n_seqs);
