@@ -122,19 +122,6 @@ def kernel_events(n_layers, n_steps, stride):
     return evs
 
 
-def event_pair_floor_ms(device, n=30):
-    """What a pair of CUDA events reports around a kernel that does nothing (one-element fill): the launch and
-    completion latency that the event figure of any stand-alone launch contains."""
-    x = torch.zeros(1, device=device)
-    out = []
-    for _ in range(n):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(); x.fill_(1.0); b.record()
-        b.synchronize()
-        out.append(a.elapsed_time(b))
-    return statistics.median(out[5:])
-
-
 def kernel_spans(n_layers, n_steps, stride, device):
     """Device words for the in-kernel timing of launches that carry NO events (so that they overlap their launch
     with their neighbours as in the un-timed step): per step {layer: int64[2] preset to (all ones, 0)}."""
@@ -614,7 +601,6 @@ def run_cuda(args, rank, world):
         sp = sum(span_ms) / len(span_ms)
         line["roofline"]["in_kernel"] = {
             "avg_span_ms": sp, "launches": len(span_ms), "achieved": alg / (sp * 1e-3) / 1e9, "frac": alg / (sp * 1e-3) / 1e9 / peak,
-            "event_pair_around_an_empty_kernel_ms": event_pair_floor_ms(device),
             "what": "the same kernel timed from inside (pask_cache_set_timing_span: first CTA released -> last CTA done, GPU "
                     "global timer) on launches of the timed region that carry no events and so keep their launch overlap; "
                     "the event figure above adds the launch and completion latency around a kernel that stands alone"}
