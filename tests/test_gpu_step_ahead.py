@@ -333,3 +333,86 @@ def test_two_steps_ahead_replayed_as_a_cuda_graph(pask, oracle):
                              oo, ol, where=(rep, half, layer))
     p.compare_state()
     assert pask.pask_budget_state(h, 0).device_status == 0
+
+
+@pytest.mark.parametrize("seed,n_kv,low_bits", [(1, 8, 4), (2, 2, 4), (3, 1, 4), (4, 4, 8), (5, 8, 2), (6, 2, 4)])
+def test_random_sequences_of_planned_ahead_steps(pask, oracle, seed, n_kv, low_bits):
+    # Seeded differential fuzz: batches that change (and are then planned again), arbitrary per-token actions, bulk
+    # appends and sequence resets in between (each makes the handle forget its plans), several layers in any order --
+    # outputs of every planned-ahead call and the state after every call against the oracle.
+    from pask_workloads.rng import CounterRng
+    from pask_workloads.tensors import normal_bf16
+    rng = CounterRng(seed, 777)
+    n_layers, G, B = 3, 2, 5
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, n_kv=n_kv, n_q=4 * n_kv, n_layers=n_layers, n_groups=G, batch=B, prompt_len=8, gen_len=8,
+                    extra_gen=8, low_bits=low_bits)
+    w = WC.build(cfg)
+    p = Pair(pask, oracle, w, pool_high_pages=600, pool_low_pages=600, max_tokens_per_seq=2048, max_append_tokens=1024)
+    P, h, d = pask, p.gpu.handle, "cuda"
+    serial, planned = 0, None                    # planned: (tuple of sequences, set of layers that hold a plan)
+    area = torch.empty(P.pask_plan_area_bytes(h, B), dtype=torch.uint8, device=d)
+
+    def data(total):
+        nonlocal serial
+        serial += 1
+        k = normal_bf16(seed, 1, serial, 0, 0, total, n_kv)
+        v = normal_bf16(seed, 2, serial, 0, 0, total, n_kv)
+        tags = np.asarray([rng.below(14) if rng.unit() < 0.9 else 0xFF for _ in range(total)], np.uint8)
+        acts = np.asarray([[rng.weighted([3, 3, 3]) for _ in range(G)] for _ in range(total)], np.uint8).reshape(total, G)
+        return k, v, tags, acts
+
+    for call in range(60):
+        u = rng.unit()
+        if u < 0.08:                                                    # forget a sequence
+            s = rng.below(B)
+            P.pask_seq_reset(h, s)
+            p.orc.seq_reset(s)
+            planned = None
+        elif u < 0.25:                                                  # a ragged append through the ordinary call
+            n_seqs = 1 + rng.below(B)
+            seqs = [int(x) for x in np.random.default_rng(seed * 1000 + call).permutation(B)[:n_seqs]]
+            counts = [[1, rng.below(40), rng.below(300)][rng.below(3)] for _ in seqs]
+            total = int(sum(counts))
+            if total == 0:
+                continue
+            cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+            k, v, tags, acts = data(total)
+            layer = rng.below(n_layers)
+            rc, _ = p.orc.append(layer, seqs, cu, bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags, decided=acts)
+            assert rc == 0
+            P.pask_append_kv_decided(h, layer, torch.tensor(seqs, dtype=torch.int32, device=d), torch.from_numpy(cu).to(d),
+                                     k.to(d), v.to(d), torch.from_numpy(tags).to(d), torch.from_numpy(acts).to(d), total_tokens=total)
+            if planned:
+                planned[1].discard(layer)
+        else:                                                           # a planned-ahead step of one layer
+            if planned is None or rng.unit() < 0.1:                     # a new batch (or the first one)
+                n_seqs = 1 + rng.below(B)
+                seqs = tuple(int(x) for x in np.random.default_rng(seed * 2000 + call).permutation(B)[:n_seqs])
+                planned = (seqs, set())
+            seqs = list(planned[0])
+            n = len(seqs)
+            ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+            layer = rng.below(n_layers)
+            if layer not in planned[1]:
+                P.pask_plan_ahead(h, layer, ids, area)
+                planned[1].add(layer)
+            k, v, tags, acts = data(n)
+            q = normal_bf16(seed, 0, serial, 0, 0, n, 4 * n_kv)
+            rc, used_o = p.orc.append(layer, seqs, list(range(n + 1)), bf16_bits(k).numpy(), bf16_bits(v).numpy(), tags, decided=acts)
+            assert rc == 0
+            out = torch.full((n, 4 * n_kv, 128), float("nan"), dtype=torch.float32, device=d)
+            lse = torch.full((n, 4 * n_kv), float("nan"), dtype=torch.float32, device=d)
+            used_g = torch.full((n,), 0xEE, dtype=torch.uint8, device=d)
+            P.pask_decode_step_ahead(h, layer, ids, k.to(d), v.to(d), torch.from_numpy(tags).to(d), q.to(d), out, lse, p.gpu.workspace(n),
+                                     area, actions=torch.from_numpy(acts).to(d), actions_out=used_g)
+            torch.cuda.synchronize()
+            assert np.array_equal(used_g.cpu().numpy(), used_o)
+            oo, ol = p.orc.attention_batch(layer, seqs, bf16_bits(q).numpy())
+            assert_close(out.cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64), oo, ol, where=(call, layer, seqs))
+        torch.cuda.synchronize()
+        assert P.pask_budget_state(h, 0).device_status == 0
+        for s in range(B):
+            for l in range(n_layers):
+                assert P.pask_debug_stream_len(h, l, s) == p.orc.stream_len(l, s)
+        assert P.pask_debug_pool_state(h) == p.orc.pool_state()
+    p.compare_state()
