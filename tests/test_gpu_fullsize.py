@@ -23,15 +23,17 @@ from parity import assert_close
 pytestmark = pytest.mark.gpu
 
 LAYERS = (0, 9, 18, 35)
-SEQS = (0, 17, 42, 63)
 
 
-@pytest.mark.parametrize("mode", ["ahead", "fused"])
-def test_full_size_decode_step_sampled_against_oracle(oracle, mode):
+# the headline configuration in both of its call forms, and the longest sequences any configuration has (the
+# concurrency-8, 32K-input shape of the paper's latency table: 33 792 tokens, 2112-entry page tables, deep splits)
+@pytest.mark.parametrize("mode,base,SEQS", [("ahead", WC.QWEN3_4B_STEP, (0, 17, 42, 63)), ("fused", WC.QWEN3_4B_STEP, (0, 17, 42, 63)),
+                                            ("ahead", WC.TABLE3_32K, (0, 3, 7))])
+def test_full_size_decode_step_sampled_against_oracle(oracle, mode, base, SEQS):
     import bench
     import paper_2608_28276_b200 as P
     dev = torch.device("cuda", 0)
-    cfg = WC.scaled(WC.QWEN3_4B_STEP, extra_gen=16)
+    cfg = WC.scaled(base, extra_gen=16)
     w = WC.build(cfg)
     job = bench.Job(P, w, dev, 6)
     job.fill()
