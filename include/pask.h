@@ -493,6 +493,12 @@ pask_status_t pask_debug_set_attention_ctas(pask_cache_t *cache, int32_t n_ctas)
  * barrier on top of what it brings: the copy completes as always, the barrier does not, the wait
  * runs out.  Host-side settings of the handle, used by the calls issued after it. */
 pask_status_t pask_debug_set_wait(pask_cache_t *cache, int64_t limit_cycles, uint32_t surplus_bytes);
+/* Where, inside a plan area for n_seqs sequences, the page-order list of (layer, parity) lies: byte
+ * offset and length.  For tests of the streaming kernel's own bounds check: a page id beyond what
+ * the pools hold (a plan somebody overwrote) is never dereferenced -- the kernel reads page 0
+ * instead and sets PASK_DEV_INTERNAL.  Host only. */
+pask_status_t pask_debug_plan_order_span(const pask_cache_t *cache, int32_t n_seqs, int32_t layer, int32_t parity,
+                                         size_t *offset, size_t *bytes);
 
 const char *pask_status_string(pask_status_t status);
 

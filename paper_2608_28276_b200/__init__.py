@@ -31,7 +31,7 @@ EXPORTS = [
     "pask_append_kv_decided", "pask_append_attend", "pask_plan_area_bytes", "pask_plan_ahead", "pask_decode_step_ahead", "pask_decode_attention",
     "pask_decode_attention_full", "pask_decode_attention_static", "pask_workspace_bytes", "pask_decode_step_host", "pask_step_staging_bytes", "pask_step_packed_layout", "pask_decode_step_packed", "pask_decode_step_pipelined", "pask_decode_step_pipelined_ahead", "pask_decode_step_drain",
     "pask_budget_state", "pask_distortion", "pask_cache_set_timing_events", "pask_cache_set_timing_span", "pask_debug_stream_len", "pask_debug_dump_high",
-    "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_debug_set_wait", "pask_status_string",
+    "pask_debug_dump_low", "pask_debug_pool_state", "pask_debug_ctrl_words", "pask_debug_page_order", "pask_debug_page_ids", "pask_debug_partition", "pask_debug_set_attention_ctas", "pask_debug_set_wait", "pask_debug_plan_order_span", "pask_status_string",
 ]
 
 
@@ -109,6 +109,7 @@ _lib.pask_debug_page_order.argtypes = [C.c_uint32, C.c_uint32, _vp]
 _lib.pask_debug_set_attention_ctas.argtypes = [_vp, _i32]
 _lib.pask_cache_set_timing_span.argtypes = [_vp, _vp]
 _lib.pask_debug_set_wait.argtypes = [_vp, C.c_int64, C.c_uint32]
+_lib.pask_debug_plan_order_span.argtypes = [_vp, _i32, _i32, _i32, C.POINTER(_sz), C.POINTER(_sz)]
 _lib.pask_status_string.argtypes = [_i32]
 _lib.pask_status_string.restype = C.c_char_p
 
@@ -434,6 +435,13 @@ def pask_cache_set_timing_span(cache: int, span):
 
 def pask_debug_set_attention_ctas(cache: int, n_ctas: int):
     _check(_lib.pask_debug_set_attention_ctas(cache, n_ctas), "pask_debug_set_attention_ctas")
+
+
+def pask_debug_plan_order_span(cache: int, n_seqs: int, layer: int, parity: int):
+    """(byte offset, byte length) of the page-order list of (layer, parity) inside a plan area for n_seqs sequences."""
+    off, n = _sz(0), _sz(0)
+    _check(_lib.pask_debug_plan_order_span(cache, n_seqs, layer, parity, C.byref(off), C.byref(n)), "pask_debug_plan_order_span")
+    return int(off.value), int(n.value)
 
 
 def pask_debug_set_wait(cache: int, limit_cycles: int = 2_000_000_000, surplus_bytes: int = 0):

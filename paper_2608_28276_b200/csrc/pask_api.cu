@@ -845,6 +845,18 @@ pask_status_t pask_debug_set_attention_ctas(pask_cache_t *c, int32_t n_ctas) {
     return PASK_OK;
 }
 
+pask_status_t pask_debug_plan_order_span(const pask_cache_t *c, int32_t n_seqs, int32_t layer, int32_t parity, size_t *offset,
+                                         size_t *bytes) {
+    if (!c || !offset || !bytes || n_seqs < 1 || n_seqs > 255 || layer < 0 || layer >= c->desc.n_layers || (parity & ~1))
+        return PASK_ERR_INVALID_ARG;
+    PlanBlock pb;
+    uint8_t origin = 0;                                             // any base will do: only the distance from it is used
+    carve_plan_area(c, n_seqs, layer, parity, &origin, &pb);
+    *offset = (size_t)(reinterpret_cast<const uint8_t *>(pb.order) - &origin);
+    *bytes = (size_t)n_seqs * (2 * (size_t)c->dev.max_pages + c->dev.window / kPageTokens) * 4;
+    return PASK_OK;
+}
+
 pask_status_t pask_debug_set_wait(pask_cache_t *c, int64_t limit_cycles, uint32_t surplus_bytes) {
     if (!c || limit_cycles < 1000 || surplus_bytes > 65536u || (surplus_bytes & 15u)) return PASK_ERR_INVALID_ARG;
     c->wait_cycles = limit_cycles;

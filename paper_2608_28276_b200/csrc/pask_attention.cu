@@ -349,6 +349,7 @@ struct Pipe {
     const uint8_t *base_high, *base_low;   // pool + this warp's head offset
     uint32_t stride_high, stride_low;      // page size in bytes
     uint32_t low_two, low_job_bytes;       // 8-bit LOW pages come as two jobs (K half, V half) of low_job_bytes each
+    uint32_t lim_high, lim_low;            // pages the two pools hold: an id beyond them is refused, not dereferenced
     uint32_t *status;         // the cache's device status word
     long long wait_cycles;    // bound of one wait
     uint32_t surplus;         // bytes the next copy announces beyond what it brings (wait-limit test; else 0)
@@ -374,8 +375,12 @@ struct Pipe {
             pw_entry = p_pos + lane < p_end ? __ldg(order + p_pos + lane) : 0u;
         }
         const uint32_t entry = __shfl_sync(0xffffffffu, pw_entry, (int)(p_pos - pw_base));
-        const uint32_t id = entry & kOrderIdMask;
+        uint32_t id = entry & kOrderIdMask;
         const bool is_high = entry & kOrderHigh;
+        if (id >= (is_high ? lim_high : lim_low)) {     // never expected (a plan somebody overwrote): flag it, read page 0
+            if (lane == 0) atomicOr(status, PASK_DEV_INTERNAL);
+            id = 0;
+        }
         const uint8_t *src = is_high ? base_high + (size_t)id * stride_high + p_sub * kHighTileBytes
                                      : base_low + (size_t)id * stride_low + p_sub * low_job_bytes;
         const uint32_t bytes = is_high ? kHighTileBytes : low_job_bytes;
@@ -485,6 +490,8 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     w.stride_low = c.low_page_bytes;
     w.low_two = kLow == 8;
     w.low_job_bytes = kLow == 8 ? kLow8HalfBytes : kLow == 2 ? kLow2HeadBytes : kLowHeadBytes;
+    w.lim_high = c.high_limit;
+    w.lim_low = c.cap_low;
     w.status = c.ctrl + kCtrlStatus;
     w.wait_cycles = p.wait_cycles;
     w.surplus = p.overpost;

@@ -145,3 +145,38 @@ def test_everything_on_a_side_stream_and_after_a_cache_reset(oracle):
                 assert pask.pask_debug_pool_state(p.gpu.handle) == (0, 0, 0, 0)
                 assert pask.pask_budget_state(p.gpu.handle, 1).full_bytes == 0
     torch.cuda.synchronize()
+
+
+def test_page_ids_beyond_the_pools_are_refused_not_dereferenced(oracle):
+    # The streaming kernel checks every page id of its plan against what the pools hold.  A plan whose page-order
+    # list somebody has overwritten with ids far beyond the pools must not make the kernel read there: it reads
+    # page 0 instead and sets PASK_DEV_INTERNAL (the results of that call are void).
+    import paper_2608_28276_b200 as pask
+    from parity import Pair
+    cfg = WC.scaled(WC.QWEN3_4B_1LAYER, batch=3, n_layers=1, n_groups=1, prompt_len=200, gen_len=100, extra_gen=16)
+    w = WC.build(cfg)
+    p = Pair(pask, oracle, w)
+    seqs = [0, 1, 2]
+    p.append(0, seqs, [300] * 3, [0] * 3)
+    h, d = p.gpu.handle, "cuda"
+    ids = torch.tensor(seqs, dtype=torch.int32, device=d)
+    area = torch.zeros(pask.pask_plan_area_bytes(h, 3), dtype=torch.uint8, device=d)
+    pask.pask_plan_ahead(h, 0, ids, area)
+    torch.cuda.synchronize()
+    off, nbytes = pask.pask_debug_plan_order_span(h, 3, 0, 0)
+    order = area[off:off + nbytes].view(torch.int32)
+    pages = sum((x + 15) // 16 for s in seqs for x in pask.pask_debug_stream_len(h, 0, s))
+    assert int((order != 0).sum()) >= pages - 1                       # this is where the plan's page list lies
+    order[:pages] |= 0x07FFFFFF                                          # every id becomes the largest one an entry can hold
+    k, v = w.kv(0, 0, 300, 1)
+    kk = torch.cat([w.kv(0, s, 300, 1)[0] for s in seqs]).to(d)
+    vv = torch.cat([w.kv(0, s, 300, 1)[1] for s in seqs]).to(d)
+    tags = torch.from_numpy(np.array([w.tags(s, 300, 1)[0] for s in seqs], np.uint8)).to(d)
+    q = torch.stack([w.q(0, s, 301) for s in seqs]).to(d)
+    out = torch.zeros((3, cfg.n_q, 128), dtype=torch.float32, device=d)
+    lse = torch.zeros((3, cfg.n_q), dtype=torch.float32, device=d)
+    pask.pask_decode_step_ahead(h, 0, ids, kk, vv, tags, q, out, lse, p.gpu.workspace(3), area)
+    torch.cuda.synchronize()                                             # the call returns, nothing faulted
+    assert pask.pask_budget_state(h, 0).device_status & pask.DEV_INTERNAL
+    # the append of that call went through as usual (it does not depend on the plan it was given)
+    assert pask.pask_debug_stream_len(h, 0, 0)[0] + pask.pask_debug_stream_len(h, 0, 0)[1] >= 1
