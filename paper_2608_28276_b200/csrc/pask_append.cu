@@ -1158,12 +1158,12 @@ step_tail_kernel(DevCache c, int layer, int group, int n_seqs, const int32_t *__
                  const uint8_t *__restrict__ tags, const uint8_t *__restrict__ decided, uint8_t *__restrict__ actions_out,
                  const SmallLut lut, const Workspace plan_ws, int32_t *__restrict__ ids_out, const uint32_t *__restrict__ prefix,
                  const float2 *__restrict__ part_ml, const float *__restrict__ part_o, float *__restrict__ out,
-                 float *__restrict__ lse, int n_q, uint32_t n_ctas, const NewTokens nt) {
+                 float *__restrict__ lse, int n_q, uint32_t n_ctas, uint32_t split, const NewTokens nt) {
     pdl_launch_dependents();
     if ((int)blockIdx.x < n_seqs)
         append_small_body(c, layer, group, n_seqs, n_seqs, seq_ids, cu_tokens, k, v, tags, decided, actions_out, lut, 1, plan_ws,
                           ids_out, (uint32_t)n_seqs);
-    merge_rows_with_new_token(prefix, part_ml, part_o, out, lse, n_seqs, n_q, n_ctas, nt, lut);
+    merge_rows_with_new_token(prefix, part_ml, part_o, out, lse, n_seqs, n_q, n_ctas, split, nt, lut);
 }
 
 // General path, recent window: CTA (j, y) copies the y-th newest of sequence j's tokens in this call
@@ -1266,11 +1266,14 @@ pask_status_t launch_step_tail(pask_cache *c, int layer, int n_seqs, const int32
     if (n_seqs < 1 || n_seqs > kSmallMax) return PASK_ERR_UNSUPPORTED_SHAPE;
     SmallLut lut;
     fill_small_lut(c, layer, &lut);
-    const int n_q = c->desc.n_q_heads, merge_ctas = (n_seqs * n_q + 7) / 8;      // one warp per (sequence, query head)
+    static_assert(kSmallThreads == kMergeThreads, "the append role and the merge share one CTA shape");
+    const int n_q = c->desc.n_q_heads, split = merge_split(n_seqs, c->attn_ctas);
+    const int merge_ctas = (n_seqs * n_q * split + 7) / 8;      // `split` warps per (sequence, query head)
     const cudaError_t e = launch_pdl(step_tail_kernel, dim3(merge_ctas > n_seqs ? merge_ctas : n_seqs), dim3(kSmallThreads), 0,
                                      stream, c->dev, layer, (int)c->layer_group[layer], n_seqs, seq_ids, cu_tokens,
                                      static_cast<const uint4 *>(k), static_cast<const uint4 *>(v), tags, decided, actions_out, lut,
-                                     plan_ws, ids_out, prefix, part_ml, part_o, out, lse, n_q, (uint32_t)c->attn_ctas, nt);
+                                     plan_ws, ids_out, prefix, part_ml, part_o, out, lse, n_q, (uint32_t)c->attn_ctas,
+                                     (uint32_t)split, nt);
     return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }
 

@@ -908,52 +908,33 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     }
 }
 
-// Merge the partials of each (sequence, query head): one warp each, lane = 4 output dims.
-__global__ void __launch_bounds__(256)
+// Merge the partials of each (sequence, query head): `split` adjacent warps a row, lane = 4 output dims.
+__global__ void __launch_bounds__(kMergeThreads)
 combine_kernel(const uint32_t *__restrict__ prefix, const float2 *__restrict__ part_ml, const float *__restrict__ part_o,
-               float *__restrict__ out, float *__restrict__ lse, int n_seqs, int n_q, uint32_t n_ctas) {
+               float *__restrict__ out, float *__restrict__ lse, int n_seqs, int n_q, uint32_t n_ctas, uint32_t split) {
     const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     // The cost prefix is the plan's, written before the streaming kernel started (that kernel lets
     // its dependents go only after its own wait for the plan's writer): it can be fetched while the
     // streaming kernel's last CTAs are still running.
-    const int s = wid / n_q, h = wid % n_q;
+    const int row_id = wid / (int)split;
+    const uint32_t sub = (uint32_t)wid % split;
+    const int s = row_id / n_q, h = row_id % n_q;
+    const bool mine = row_id < n_seqs * n_q;
     uint32_t p0 = 0, p1 = 0;
     uint64_t total = 0;
-    if (wid < n_seqs * n_q) { p0 = __ldg(prefix + s); p1 = __ldg(prefix + s + 1); total = __ldg(prefix + n_seqs); }
+    if (mine) { p0 = __ldg(prefix + s); p1 = __ldg(prefix + s + 1); total = __ldg(prefix + n_seqs); }
     uint32_t b_first = 1, b_last = 0;       // the CTAs that hold partials of this sequence (two 64-bit divisions, ahead of the wait)
     if (p1 > p0) {
         b_first = (uint32_t)((((uint64_t)p0 + 1) * n_ctas - 1) / total);
         b_last = (uint32_t)(((uint64_t)p1 * n_ctas - 1) / total);
     }
     pdl_wait();
-    if (wid >= n_seqs * n_q) return;
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
     float M = -INFINITY, L = 0.f;
-    if (p1 > p0) {
-        // online merge, eight partials per round trip
-        for (uint32_t b = b_first; b <= b_last; b += 8) {
-            float2 ml[8];
-            float4 v[8];
-#pragma unroll
-            for (int u = 0; u < 8; u++) {
-                const bool have = b + u <= b_last;
-                const size_t row = ((size_t)b + u + s) * n_q + h;
-                ml[u] = have ? part_ml[row] : make_float2(-INFINITY, 0.f);
-                v[u] = have ? *reinterpret_cast<const float4 *>(part_o + row * kHeadDim + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int u = 0; u < 8; u++) {
-                if (ml[u].x == -INFINITY) continue;      // a CTA whose share of this sequence was empty
-                const float Mn = fmaxf(M, ml[u].x);
-                const float fo = exp2f(M - Mn), fn = exp2f(ml[u].x - Mn);   // exp2f(-inf) = 0 on the first one
-                o.x = fmaf(fn, v[u].x, o.x * fo); o.y = fmaf(fn, v[u].y, o.y * fo);
-                o.z = fmaf(fn, v[u].z, o.z * fo); o.w = fmaf(fn, v[u].w, o.w * fo);
-                L = fmaf(fn, ml[u].y, L * fo);
-                M = Mn;
-            }
-        }
-    }
+    if (p1 > p0) merge_share(part_ml, part_o, s, h, n_q, b_first, b_last, sub, split, lane, o, M, L);
+    merge_across_warps(sub, split, lane, o, M, L);
+    if (!mine || sub != 0) return;
     const size_t orow = (size_t)s * n_q + h;
     if (L > 0.f) {
         const float inv = 1.0f / L;
@@ -1050,11 +1031,11 @@ pask_status_t launch_attention(pask_cache *c, bool has_low, int layer, int n_seq
         e = launch_pdl(attn_plan_kernel, dim3(c->sm_count), dim3(kPlanThreads), (size_t)(5 * n_seqs + 2) * 4, stream, c->dev,
                        layer, n_seqs, seq_ids, p.ws, has_low ? 1 : 0);
     if (e == cudaSuccess) e = launch_stream_kernel(c, has_low, p, stream);
-    const int warps = n_seqs * c->desc.n_q_heads;
+    const int split = merge_split(n_seqs, c->attn_ctas), warps = n_seqs * c->desc.n_q_heads * split;
     if (e == cudaSuccess)
-        e = launch_pdl(combine_kernel, dim3((warps + 7) / 8), dim3(256), 0, stream, (const uint32_t *)p.ws.cost_prefix,
+        e = launch_pdl(combine_kernel, dim3((warps + 7) / 8), dim3(kMergeThreads), 0, stream, (const uint32_t *)p.ws.cost_prefix,
                        (const float2 *)p.ws.part_ml, (const float *)p.ws.part_o, out, lse, n_seqs, (int)c->desc.n_q_heads,
-                       (uint32_t)c->attn_ctas);
+                       (uint32_t)c->attn_ctas, (uint32_t)split);
     return e == cudaSuccess ? PASK_OK : PASK_ERR_CUDA;
 }
 

@@ -40,25 +40,92 @@ __device__ __forceinline__ void quantise_like_append(float (&x)[4], int low_bits
     }
 }
 
-// The merge of a planned-ahead step for the (sequence, query head) rows of this CTA's warps (one warp each, lane = 4
-// output dims): the partials of the history (streamed from the plan of the cache before this call's append) and, as
-// one more partial, the sequence's new token taken from the call's k / v.  Everything that does not come from the
-// kernels before is fetched first; the function then executes the kernel's dependency wait itself.
+// How many warps share the partials of one (sequence, query head) row.  A row has about n_ctas / n_seqs partials, and a
+// warp takes eight per round trip to L2: small batches, whose rows have dozens, are split so that one round trip does.
+inline int merge_split(int n_seqs, int n_ctas) {
+    int split = 1;
+    while (split < 8 && n_ctas / n_seqs + 2 > 8 * split) split *= 2;
+    return split;
+}
+
+constexpr int kMergeThreads = 256;     // CTA of the kernels that merge: 8 warps = 8 / split rows
+
+// Online merge of the partials b_first + sub, b_first + sub + split, ... <= b_last of row (s, h) into (o, M, L); lane = 4
+// output dims.  Eight partials per round trip.
+__device__ __forceinline__ void merge_share(const float2 *__restrict__ part_ml, const float *__restrict__ part_o, int s, int h,
+                                            int n_q, uint32_t b_first, uint32_t b_last, uint32_t sub, uint32_t split, int lane,
+                                            float4 &o, float &M, float &L) {
+    for (uint32_t b = b_first + sub; b <= b_last; b += 8 * split) {
+        float2 ml[8];
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; u++) {
+            const bool have = b + u * split <= b_last;
+            const size_t row = ((size_t)b + u * split + s) * n_q + h;
+            ml[u] = have ? part_ml[row] : make_float2(-INFINITY, 0.f);
+            v[u] = have ? *reinterpret_cast<const float4 *>(part_o + row * kHeadDim + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; u++) {
+            if (ml[u].x == -INFINITY) continue;      // a CTA whose share of this sequence was empty
+            const float Mn = fmaxf(M, ml[u].x);
+            const float fo = exp2f(M - Mn), fn = exp2f(ml[u].x - Mn);   // exp2f(-inf) = 0 on the first one
+            o.x = fmaf(fn, v[u].x, o.x * fo); o.y = fmaf(fn, v[u].y, o.y * fo);
+            o.z = fmaf(fn, v[u].z, o.z * fo); o.w = fmaf(fn, v[u].w, o.w * fo);
+            L = fmaf(fn, ml[u].y, L * fo);
+            M = Mn;
+        }
+    }
+}
+
+// The `split` warps of a row (adjacent warps of one CTA; every thread of the CTA calls this) hand their shares to the
+// row's first warp, which merges them in warp order: the result is the same whatever the timing.
+__device__ __forceinline__ void merge_across_warps(uint32_t sub, uint32_t split, int lane, float4 &o, float &M, float &L) {
+    __shared__ float4 s_o[kMergeThreads / 32][32];
+    __shared__ float2 s_ml[kMergeThreads / 32];
+    if (split == 1) return;
+    const int warp = threadIdx.x >> 5;
+    if (sub != 0) {
+        s_o[warp][lane] = o;
+        if (lane == 0) s_ml[warp] = make_float2(M, L);
+    }
+    __syncthreads();
+    if (sub != 0) return;
+    for (uint32_t w = 1; w < split; w++) {
+        const float2 ml = s_ml[warp + w];
+        if (ml.x == -INFINITY) continue;
+        const float4 v = s_o[warp + w][lane];
+        const float Mn = fmaxf(M, ml.x);
+        const float fo = exp2f(M - Mn), fn = exp2f(ml.x - Mn);
+        o.x = fmaf(fn, v.x, o.x * fo); o.y = fmaf(fn, v.y, o.y * fo);
+        o.z = fmaf(fn, v.z, o.z * fo); o.w = fmaf(fn, v.w, o.w * fo);
+        L = fmaf(fn, ml.y, L * fo);
+        M = Mn;
+    }
+}
+
+// The merge of a planned-ahead step for the (sequence, query head) rows of this CTA's warps (`split` adjacent warps a
+// row, lane = 4 output dims): the partials of the history (streamed from the plan of the cache before this call's
+// append) and, as one more partial, the sequence's new token taken from the call's k / v.  Everything that does not
+// come from the kernels before is fetched first; the function then executes the kernel's dependency wait itself.
+// Every thread of the CTA must call it (it holds a block-wide barrier when split > 1).
 __device__ __forceinline__ void merge_rows_with_new_token(const uint32_t *__restrict__ prefix, const float2 *__restrict__ part_ml,
                                                           const float *__restrict__ part_o, float *__restrict__ out,
                                                           float *__restrict__ lse, int n_seqs, int n_q, uint32_t n_ctas,
-                                                          const NewTokens &nt, const SmallLut &lut) {
+                                                          uint32_t split, const NewTokens &nt, const SmallLut &lut) {
     const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    const int s = wid / n_q, h = wid % n_q;
-    const bool mine = wid < n_seqs * n_q;
+    const int row_id = wid / (int)split;
+    const uint32_t sub = (uint32_t)wid % split;
+    const int s = row_id / n_q, h = row_id % n_q;
+    const bool mine = row_id < n_seqs * n_q;
     // everything that does not come from the kernels before is fetched ahead of the dependency wait
     uint32_t p0 = 0, p1 = 0;
     uint64_t total = 0;
     int act = PASK_ACTION_RELEASE;
     float kx[4] = {0.f, 0.f, 0.f, 0.f}, vx[4] = {0.f, 0.f, 0.f, 0.f}, qx[4] = {0.f, 0.f, 0.f, 0.f};
     bool stale = false;
-    if (mine) {
-        p0 = __ldg(prefix + s); p1 = __ldg(prefix + s + 1); total = __ldg(prefix + n_seqs);
+    if (mine) { p0 = __ldg(prefix + s); p1 = __ldg(prefix + s + 1); total = __ldg(prefix + n_seqs); }
+    if (mine && sub == 0) {       // the new token is the business of the row's first warp
         act = nt.decided ? nt.decided[(size_t)s * nt.n_groups + nt.group] : lut.action[nt.tags[s]];
         if (act > PASK_ACTION_RETAIN_HIGH) act = PASK_ACTION_RELEASE;      // (the append refuses the call)
         stale = nt.seq_ids[s] != nt.planned_ids[s];
@@ -87,32 +154,11 @@ __device__ __forceinline__ void merge_rows_with_new_token(const uint32_t *__rest
         b_last = (uint32_t)(((uint64_t)p1 * n_ctas - 1) / total);
     }
     pdl_wait();
-    if (!mine) return;
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
     float M = -INFINITY, L = 0.f;
-    if (p1 > p0) {
-        for (uint32_t b = b_first; b <= b_last; b += 8) {
-            float2 ml[8];
-            float4 v[8];
-#pragma unroll
-            for (int u = 0; u < 8; u++) {
-                const bool have = b + u <= b_last;
-                const size_t row = ((size_t)b + u + s) * n_q + h;
-                ml[u] = have ? part_ml[row] : make_float2(-INFINITY, 0.f);
-                v[u] = have ? *reinterpret_cast<const float4 *>(part_o + row * kHeadDim + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int u = 0; u < 8; u++) {
-                if (ml[u].x == -INFINITY) continue;
-                const float Mn = fmaxf(M, ml[u].x);
-                const float fo = exp2f(M - Mn), fn = exp2f(ml[u].x - Mn);
-                o.x = fmaf(fn, v[u].x, o.x * fo); o.y = fmaf(fn, v[u].y, o.y * fo);
-                o.z = fmaf(fn, v[u].z, o.z * fo); o.w = fmaf(fn, v[u].w, o.w * fo);
-                L = fmaf(fn, ml[u].y, L * fo);
-                M = Mn;
-            }
-        }
-    }
+    if (p1 > p0) merge_share(part_ml, part_o, s, h, n_q, b_first, b_last, sub, split, lane, o, M, L);
+    merge_across_warps(sub, split, lane, o, M, L);
+    if (!mine || sub != 0) return;
     if (m_new != -INFINITY) {                // the new token: weight 1 at its own score
         const float Mn = fmaxf(M, m_new);
         const float fo = exp2f(M - Mn), fn = exp2f(m_new - Mn);
