@@ -1149,9 +1149,11 @@ append_small_kernel(DevCache c, int layer, int group, int n_seqs, int total, con
 // sequence) WITHOUT waiting for the kernel before them in the stream: that is the decode-attention kernel of the same
 // layer, which works from a plan of the cache before this append, needs none of its results and touches nothing it
 // writes, so the append runs in the shadow of that kernel's tail.  (Everything before that predecessor is complete:
-// it has done its own wait before it let this kernel start.)  Every CTA then waits for the predecessor and merges
-// its partials, the new tokens included -- so whoever comes next in the stream and waits for this kernel has waited
-// for both.
+// it has done its own wait before it let this kernel start.)  The other CTAs wait for the predecessor and merge its
+// partials, the new tokens included; the kernel is complete when they are -- so whoever comes next in the stream and
+// waits for this kernel has waited for both.  (The two roles have CTAs of their own: with a short streaming kernel the
+// append, which also writes the next step's plan, ends after the partials are ready, and the merge does not queue
+// behind it.)
 __global__ void __launch_bounds__(kSmallThreads)
 step_tail_kernel(DevCache c, int layer, int group, int n_seqs, const int32_t *__restrict__ seq_ids,
                  const int32_t *__restrict__ cu_tokens, const uint4 *__restrict__ k, const uint4 *__restrict__ v,
@@ -1160,10 +1162,13 @@ step_tail_kernel(DevCache c, int layer, int group, int n_seqs, const int32_t *__
                  const float2 *__restrict__ part_ml, const float *__restrict__ part_o, float *__restrict__ out,
                  float *__restrict__ lse, int n_q, uint32_t n_ctas, uint32_t split, const NewTokens nt) {
     pdl_launch_dependents();
-    if ((int)blockIdx.x < n_seqs)
+    if ((int)blockIdx.x < n_seqs) {
+        // (no wait of its own: the kernel is complete only when its merging CTAs are, and those have waited)
         append_small_body(c, layer, group, n_seqs, n_seqs, seq_ids, cu_tokens, k, v, tags, decided, actions_out, lut, 1, plan_ws,
                           ids_out, (uint32_t)n_seqs);
-    merge_rows_with_new_token(prefix, part_ml, part_o, out, lse, n_seqs, n_q, n_ctas, split, nt, lut);
+        return;
+    }
+    merge_rows_with_new_token(prefix, part_ml, part_o, out, lse, n_seqs, n_q, n_ctas, split, nt, lut, (uint32_t)n_seqs);
 }
 
 // General path, recent window: CTA (j, y) copies the y-th newest of sequence j's tokens in this call
@@ -1269,7 +1274,7 @@ pask_status_t launch_step_tail(pask_cache *c, int layer, int n_seqs, const int32
     static_assert(kSmallThreads == kMergeThreads, "the append role and the merge share one CTA shape");
     const int n_q = c->desc.n_q_heads, split = merge_split(n_seqs, c->attn_ctas);
     const int merge_ctas = (n_seqs * n_q * split + 7) / 8;      // `split` warps per (sequence, query head)
-    const cudaError_t e = launch_pdl(step_tail_kernel, dim3(merge_ctas > n_seqs ? merge_ctas : n_seqs), dim3(kSmallThreads), 0,
+    const cudaError_t e = launch_pdl(step_tail_kernel, dim3(n_seqs + merge_ctas), dim3(kSmallThreads), 0,
                                      stream, c->dev, layer, (int)c->layer_group[layer], n_seqs, seq_ids, cu_tokens,
                                      static_cast<const uint4 *>(k), static_cast<const uint4 *>(v), tags, decided, actions_out, lut,
                                      plan_ws, ids_out, prefix, part_ml, part_o, out, lse, n_q, (uint32_t)c->attn_ctas,

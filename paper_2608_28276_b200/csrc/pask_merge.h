@@ -108,12 +108,14 @@ __device__ __forceinline__ void merge_across_warps(uint32_t sub, uint32_t split,
 // row, lane = 4 output dims): the partials of the history (streamed from the plan of the cache before this call's
 // append) and, as one more partial, the sequence's new token taken from the call's k / v.  Everything that does not
 // come from the kernels before is fetched first; the function then executes the kernel's dependency wait itself.
-// Every thread of the CTA must call it (it holds a block-wide barrier when split > 1).
+// Every thread of the CTA must call it (it holds a block-wide barrier when split > 1).  The CTAs that merge are those
+// from first_cta on.
 __device__ __forceinline__ void merge_rows_with_new_token(const uint32_t *__restrict__ prefix, const float2 *__restrict__ part_ml,
                                                           const float *__restrict__ part_o, float *__restrict__ out,
                                                           float *__restrict__ lse, int n_seqs, int n_q, uint32_t n_ctas,
-                                                          uint32_t split, const NewTokens &nt, const SmallLut &lut) {
-    const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+                                                          uint32_t split, const NewTokens &nt, const SmallLut &lut,
+                                                          uint32_t first_cta) {
+    const int wid = ((blockIdx.x - first_cta) * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     const int row_id = wid / (int)split;
     const uint32_t sub = (uint32_t)wid % split;
     const int s = row_id / n_q, h = row_id % n_q;
