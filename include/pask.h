@@ -474,7 +474,9 @@ pask_status_t pask_debug_ctrl_words(pask_cache_t *cache, uint32_t *out, int32_t 
  * for a HIGH page.  For a batch whose sequences hold the given page counts and a grid of `n_ctas`,
  * pask_debug_partition writes for each CTA b and sequence index s the half-open range of positions
  * of that order which b processes, as ranges[(b * n_seqs + s) * 2 + {0,1}] (empty: begin == end).
- * Host only, no GPU. */
+ * A batch of at most n_ctas / 16 sequences is cut so that every non-empty sequence has whole CTAs
+ * of its own (its share of the cost, rounded, at least one; inside it equal numbers of positions):
+ * no CTA then works on two sequences.  Host only, no GPU. */
 pask_status_t pask_debug_page_order(uint32_t pages_high, uint32_t pages_low, uint32_t *order);
 pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, const uint32_t *pages_low,
                                    int32_t n_ctas, uint32_t *ranges);

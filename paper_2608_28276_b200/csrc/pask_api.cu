@@ -264,6 +264,7 @@ pask_status_t pask_cache_create(const pask_cache_desc_t *d, const pask_policy_t 
     v.bytes_h = 2u * d->n_kv_heads * kHeadDim * 2u;
     v.bytes_l = 2u * d->n_kv_heads * (kHeadDim * pol->low_bits / 8 + kGroupsPerHead * 2);
     c->attn_ctas = attention_grid(c);
+    c->dev.attn_ctas = (uint32_t)c->attn_ctas;
     c->lut = pol->eff;
     c->layer_group = pol->layer_group;
     // per tag byte: the table's actions and floors packed two bits per group, and what the actions cost
@@ -842,6 +843,7 @@ pask_status_t pask_debug_dump_low(pask_cache_t *c, int32_t layer, int32_t seq, u
 pask_status_t pask_debug_set_attention_ctas(pask_cache_t *c, int32_t n_ctas) {
     if (!c || n_ctas < 1 || n_ctas > 65536) return PASK_ERR_INVALID_ARG;
     c->attn_ctas = n_ctas;
+    c->dev.attn_ctas = (uint32_t)n_ctas;
     return PASK_OK;
 }
 
@@ -870,6 +872,11 @@ pask_status_t pask_debug_partition(int32_t n_seqs, const uint32_t *pages_high, c
     std::vector<uint64_t> prefix((size_t)n_seqs + 1, 0);
     for (int s = 0; s < n_seqs; s++)
         prefix[s + 1] = prefix[s] + (uint64_t)pages_high[s] * kCostHighPage + (uint64_t)pages_low[s] * kCostLowPage;
+    if (prefix[n_seqs] <= 0xffffffffull) {      // a small batch: whole CTAs per sequence, as the plan kernels cut it
+        std::vector<uint32_t> snapped(prefix.begin(), prefix.end());
+        snap_cost_prefix(snapped.data(), n_seqs, (uint32_t)n_ctas);
+        for (int s = 0; s <= n_seqs; s++) prefix[s] = snapped[s];
+    }
     const uint64_t total = prefix[n_seqs];
     for (int b = 0; b < n_ctas; b++) {
         const uint64_t lo = total * b / n_ctas, hi = total * (b + 1) / n_ctas;

@@ -978,6 +978,10 @@ append_small_body(const DevCache &c, int layer, int group, int n_seqs, int total
         if (tid == 0 && !fits && !s_err) atomicOr(&s_err, PASK_DEV_POOL_EXHAUSTED);
     }
     __syncthreads();
+    if (fuse_plan && blockIdx.x == 0) {          // (block 0 writes the prefix)
+        if (tid == 0) snap_cost_prefix(s_cost, n_seqs, c.attn_ctas);
+        __syncthreads();
+    }
     // old page of this CTA's token, if it continues one (page tables are only appended to by the commit)
     uint32_t my_page = 0, my_at = 0;
     const uint32_t my_a = s_act[my_tok];

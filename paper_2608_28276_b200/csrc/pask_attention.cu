@@ -304,6 +304,8 @@ attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ 
         }
     }
     __syncthreads();
+    if (tid == 0) snap_cost_prefix(s_cost, n_seqs, c.attn_ctas);
+    __syncthreads();
     if (blockIdx.x == 0) {
         for (int s = tid; s <= n_seqs; s += kPlanThreads) { ws.cost_prefix[s] = s_cost[s]; ws.page_prefix[s] = s_page[s]; }
         for (int s = tid; s < n_seqs; s += kPlanThreads) ws.tokens[s] = make_uint2(s_nh[s], s_nl[s]);

@@ -87,6 +87,7 @@ struct DevCache {
     uint32_t low_bits;               // 2, 4 or 8: width of the RETAIN-LOW codes
     uint32_t low_head_bytes;         // one KV head of a LOW page (2304 or 4352)
     uint32_t cost_low_page;          // cost of a LOW page in units of n_kv * 256 bytes (9 or 17)
+    uint32_t attn_ctas;              // grid of the decode-attention main kernel (the plans are cut for it)
 };
 
 // workspace of one decode-attention call

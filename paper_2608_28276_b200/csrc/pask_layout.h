@@ -162,6 +162,34 @@ PASK_HD uint32_t cut_positions(uint32_t x, uint32_t cs, uint32_t n) {
     return x >= cs ? n : (uint32_t)(((uint64_t)x * n) / cs);
 }
 
+// A small batch (at least kSnapCtasPerSeq CTAs per sequence): the cost line is replaced by one on which every
+// non-empty sequence covers a whole number of CTA shares -- cost[s] becomes the first CTA of sequence s and
+// cost[n_seqs] the grid -- so that no CTA's range crosses from one sequence into the next (a second segment costs a
+// CTA a fresh set-up of about two microseconds, which a short kernel feels as a straggler).  Every non-empty
+// sequence gets one CTA, and the others are shared out by cost (rounded cumulatively, so the error does not add up):
+// no CTA then carries more than grid / (grid - sequences) <= 16/15 of an even share.  Inside a sequence the cuts fall
+// at equal numbers of positions of its order list as before.  Everything that reads the prefix (the streaming
+// kernel's ranges, the merge's list of CTAs per sequence) works from it unchanged.
+constexpr uint32_t kSnapCtasPerSeq = 16;
+PASK_HD void snap_cost_prefix(uint32_t *cost, int n_seqs, uint32_t n_ctas) {
+    const uint32_t total = cost[n_seqs];
+    if (total == 0 || (uint64_t)n_seqs * kSnapCtasPerSeq > n_ctas) return;
+    uint32_t n_ne = 0;                       // non-empty sequences
+    for (int s = 0; s < n_seqs; s++) n_ne += cost[s + 1] > cost[s];
+    const uint32_t rest = n_ctas - n_ne;     // CTAs shared out by cost
+    uint32_t old_lo = cost[0], at = 0, given = 0;      // old cost[s]; new cost[s]; of `rest`, given to the sequences before
+    for (int s = 0; s < n_seqs; s++) {
+        const uint32_t old_hi = cost[s + 1];
+        if (old_hi > old_lo) {
+            const uint32_t upto = (uint32_t)(((uint64_t)old_hi * rest + total / 2) / total);
+            at += 1 + (upto - given);
+            given = upto;
+        }
+        cost[s + 1] = at;
+        old_lo = old_hi;
+    }
+}
+
 // entries of the per-call page order list built by the plan kernel
 constexpr uint32_t kOrderHigh = 0x80000000u;   // the page has the HIGH (bf16) format (else LOW)
 constexpr int kOrderValidShift = 27;           // bits 27..30: tokens of the page to attend, 0 meaning all 16

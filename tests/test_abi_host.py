@@ -100,7 +100,8 @@ def test_bad_blobs_and_arguments_are_refused(pask):
 
 def test_decode_partition_covers_every_page_exactly_once(pask):
     rng = np.random.default_rng(3)
-    cases = [([5], [0], 4), ([0], [7], 3), ([0, 0, 3], [0, 2, 0], 8), ([1], [1], 296)]
+    cases = [([5], [0], 4), ([0], [7], 3), ([0, 0, 3], [0, 2, 0], 8), ([1], [1], 296),
+             ([513] * 8, [0] * 8, 296), ([100, 0, 3000, 1, 0, 40], [900, 0, 100, 0, 2, 7], 296), ([2000, 1], [0, 0], 32)]
     for _ in range(30):
         n = int(rng.integers(1, 40))
         cases.append((rng.integers(0, 60, n), rng.integers(0, 90, n), int(rng.choice([1, 2, 7, 64, 296]))))
@@ -128,7 +129,19 @@ def test_decode_partition_covers_every_page_exactly_once(pask):
                 seen[a:e] += 1
                 cost[b] += 32 * is_high[a:e].sum() + 9 * (~is_high[a:e]).sum()
             assert np.all(seen == 1)
-        # balance: no CTA streams more than its share plus about one page of each kind per cut
         total = float(32 * ph.sum() + 9 * pl.sum())
         assert cost.sum() == total
-        assert cost.max() <= total / g + 2 * (32 + 9) + 1e-9
+        if 16 * len(ph) <= g:
+            # a small batch: every non-empty sequence has whole CTAs of its own, one plus its share of the others, so a
+            # CTA streams at most g / (g - sequences) of an even share plus about a page of each kind
+            owners = [set(np.nonzero(r[:, s, 1] > r[:, s, 0])[0]) for s in range(len(ph))]
+            for s in range(len(ph)):
+                assert (len(owners[s]) > 0) == (ph[s] + pl[s] > 0)
+                assert all(owners[s].isdisjoint(owners[t]) for t in range(s))
+                if ph[s] + pl[s] >= g:      # enough pages to give every CTA some: the count is one plus the rounded share
+                    n_ne = int(np.count_nonzero(ph + pl))
+                    assert abs(len(owners[s]) - 1 - (g - n_ne) * (32.0 * ph[s] + 9.0 * pl[s]) / total) <= 1.0
+            assert cost.max() <= total / (g - len(ph)) + 2 * (32 + 9) + 1e-9
+        else:
+            # balance: no CTA streams more than its share plus about one page of each kind per cut
+            assert cost.max() <= total / g + 2 * (32 + 9) + 1e-9
