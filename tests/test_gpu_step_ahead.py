@@ -416,3 +416,31 @@ def test_random_sequences_of_planned_ahead_steps(pask, oracle, seed, n_kv, low_b
                 assert P.pask_debug_stream_len(h, l, s) == p.orc.stream_len(l, s)
         assert P.pask_debug_pool_state(h) == p.orc.pool_state()
     p.compare_state()
+
+
+@pytest.mark.parametrize("batch", [2, 12, 18, 19, 30, 37, 50])
+def test_unequal_small_batches_through_both_attention_paths(pask, oracle, batch):
+    # How the partials of a row are merged and how the cost line is cut depend on the batch: up to 18 sequences
+    # every non-empty one gets whole CTAs of the streaming kernel; below 43 a row's partials are shared by 2, 4 or
+    # 8 warps.  One long sequence, short ones of every page-boundary case and one that holds nothing, through
+    # pask_decode_attention and through planned-ahead steps.
+    p, w = _pair(pask, oracle, batch, 1500, 100)
+    seqs = list(range(batch))
+    lens = [w.total_len(0)] + [(7 * s * s + 1) % 97 for s in range(1, batch)]
+    lens[-1] = 0                                     # named in every call, holds nothing until the first step
+    some = [s for s in seqs if lens[s] > 0]
+    for layer in range(w.cfg.n_layers):
+        p.append(layer, some, [lens[s] for s in some], [0] * len(some))
+        p.check_attention(layer, seqs, pos=1600)
+        p.check_attention(layer, seqs[::-1][: max(1, batch // 2)], pos=1601)      # another batch size, another cut
+    area = torch.empty(pask.pask_plan_area_bytes(p.gpu.handle, batch), dtype=torch.uint8, device="cuda")
+    ids = torch.tensor(seqs, dtype=torch.int32, device="cuda")
+    for layer in range(w.cfg.n_layers):
+        pask.pask_plan_ahead(p.gpu.handle, layer, ids, area)
+    pos = list(lens)
+    for step in range(20):
+        for layer in range(w.cfg.n_layers):
+            _ahead_step(p, area, layer, seqs, pos)
+        pos = [x + 1 for x in pos]
+    p.compare_state()
+    assert pask.pask_budget_state(p.gpu.handle, 0).device_status == 0
