@@ -410,6 +410,20 @@ struct Pipe {
         entry = lds32(meta + c_stage * 4);
         return ring + c_stage * kStageBytes;
     }
+    // The same for the job after the oldest one, which stays the oldest (two stages are then held at once).
+    __device__ __forceinline__ uint32_t acquire_next(uint32_t &entry) {
+        uint32_t stage = c_stage + 1, parity = c_parity;
+        if (stage == kStages) { stage = 0; parity ^= 1u; }
+        const uint32_t bar = bars + stage * 8;
+        if (!mbar_try_wait(bar, parity)) {
+            if (dead || !mbar_wait_slow(bar, parity, wait_cycles)) {
+                if (!dead && lane == 0) atomicOr(status, PASK_DEV_TIMEOUT);
+                dead = true;
+            }
+        }
+        entry = lds32(meta + stage * 4);
+        return ring + stage * kStageBytes;
+    }
     // All lanes are done reading the oldest stage: hand it back to the producer.
     __device__ __forceinline__ void release() {
         __syncwarp();
@@ -610,12 +624,118 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         for (int m = 0; m < 8; m++) acc[m][0] = acc[m][1] = acc[m][2] = acc[m][3] = 0.f;
         float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
 
+        // P.V over the four-bit V codes of the page in stage `stage`, weights p0..p3 (heads a, a+1 x tokens g, g+8); the
+        // stage is handed back as soon as its V half is in registers
+        auto pv_low4 = [&](uint32_t stage, uint32_t n_valid, float p0, float p1, float p2, float p3) {
+            const uint32_t vb = stage + kLowHalfBytes;
+            const uint4 v0 = lds128(vb + lane * 16);        // tokens 2t, 2t+1
+            const uint4 v1 = lds128(vb + 512 + lane * 16);  // tokens 2t+8, 2t+9
+            uint2 vs0 = lds64(vb + kLowCodesBytes + g * 8);
+            uint2 vs1 = lds64(vb + kLowCodesBytes + (g + 8) * 8);
+            w.release();   // everything of this stage is in registers now
+            if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
+                if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
+                if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
+            }
+            const uint32_t c0[4] = {v0.x, v0.y, v0.z, v0.w}, c1[4] = {v1.x, v1.y, v1.z, v1.w};
+            const uint32_t p01 = pack_f16(p0, p1), p23 = pack_f16(p2, p3);
+#pragma unroll
+            for (int v = 0; v < 2; v++) {
+                // B columns 0-3: heads x group 2v, columns 4-7: heads x group 2v + 1
+                const uint32_t s0b = hmul2(prmt(v ? vs0.y : vs0.x, 0u, bsel), down);
+                const uint32_t s1b = hmul2(prmt(v ? vs1.y : vs1.x, 0u, bsel), down);
+                const uint32_t b0 = movmatrix_trans(hmul2(p01, s0b)), b1 = movmatrix_trans(hmul2(p23, s1b));
+#pragma unroll
+                for (int qq = 0; qq < 2; qq++) {
+                    const int q = 2 * v + qq;
+                    const uint32_t e0 = c0[q] >> 8, e1 = c1[q] >> 8;
+                    uint32_t a[2][4];
+                    a[0][0] = hsub2(nib_even(c0[q]), 0x64086408u);               // (1024 + code) - 1032
+                    a[0][1] = hfma2(nib_odd(c0[q]), 0x2C002C00u, 0xD480D480u);   // (1024 + 16 code) / 16 - 72
+                    a[0][2] = hsub2(nib_even(e0), 0x64086408u);
+                    a[0][3] = hfma2(nib_odd(e0), 0x2C002C00u, 0xD480D480u);
+                    a[1][0] = hsub2(nib_even(c1[q]), 0x64086408u);
+                    a[1][1] = hfma2(nib_odd(c1[q]), 0x2C002C00u, 0xD480D480u);
+                    a[1][2] = hsub2(nib_even(e1), 0x64086408u);
+                    a[1][3] = hfma2(nib_odd(e1), 0x2C002C00u, 0xD480D480u);
+#pragma unroll
+                    for (int r = 0; r < 2; r++)
+                        mma_f16(acc[2 * q + r], a[0][2 * r], a[0][2 * r + 1], a[1][2 * r], a[1][2 * r + 1], b0, b1);
+                }
+            }
+        };
+
         for (uint32_t page = 0; page < n_pages; ++page) {
             uint32_t entry;
             uint32_t st = w.acquire(entry);
             if (w.dead) break;
             const bool is_high = entry & kOrderHigh;
             const uint32_t n_valid = (((entry >> kOrderValidShift) - 1u) & 15u) + 1u;   // 0 in the entry means all 16
+
+            // ---- two full four-bit pages in a row are taken together: two independent chains of loads, logic, MMAs
+            // and exponentials for the four resident warps of a scheduler to interleave instead of one (the warp-level
+            // MMA and the half-rate logic pipe leave an in-order warp waiting most of the time), one look at the running
+            // maxima, and the query operands fetched once for both
+            if (kLow == 4 && !is_high && n_valid == 16u && page + 1 < n_pages) {
+                uint32_t entry_b;
+                const uint32_t st_b = w.acquire_next(entry_b);
+                if (w.dead) break;
+                if (!(entry_b & kOrderHigh) && ((entry_b >> kOrderValidShift) & 15u) == 0u) {
+                    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+                    {
+                        const uint4 ka0 = lds128(st + lane * 16), ka1 = lds128(st + 512 + lane * 16);
+                        const uint4 kb0 = lds128(st_b + lane * 16), kb1 = lds128(st_b + 512 + lane * 16);
+                        const uint2 sa0 = lds64(st + kLowCodesBytes + g * 8), sa1 = lds64(st + kLowCodesBytes + (g + 8) * 8);
+                        const uint2 sb0 = lds64(st_b + kLowCodesBytes + g * 8), sb1 = lds64(st_b + kLowCodesBytes + (g + 8) * 8);
+                        const uint32_t wa0[4] = {ka0.x, ka0.y, ka0.z, ka0.w}, wa1[4] = {ka1.x, ka1.y, ka1.z, ka1.w};
+                        const uint32_t wb0[4] = {kb0.x, kb0.y, kb0.z, kb0.w}, wb1[4] = {kb1.x, kb1.y, kb1.z, kb1.w};
+                        const float2 fa0[2] = {unpack_f16(sa0.x), unpack_f16(sa0.y)}, fa1[2] = {unpack_f16(sa1.x), unpack_f16(sa1.y)};
+                        const float2 fb0[2] = {unpack_f16(sb0.x), unpack_f16(sb0.y)}, fb1[2] = {unpack_f16(sb1.x), unpack_f16(sb1.y)};
+#pragma unroll
+                        for (int j = 0; j < 4; j++) {
+                            const uint4 qa = lds128(scratch + j * 256 + (g & 3) * 64 + t * 16);
+                            const uint4 seed = lds128(scratch + 1024 + ((t & 1) * 4 + j) * 16);
+                            float ca[4], cb[4];
+                            const uint32_t ua0 = wa0[j] >> 8, ua1 = wa1[j] >> 8, ub0 = wb0[j] >> 8, ub1 = wb1[j] >> 8;
+                            mma_f16_seed(ca, nib_even(wa0[j]), nib_even(wa1[j]), nib_odd(wa0[j]), nib_odd(wa1[j]), qa.x, qa.y, seed);
+                            mma_f16_seed(cb, nib_even(wb0[j]), nib_even(wb1[j]), nib_odd(wb0[j]), nib_odd(wb1[j]), qa.x, qa.y, seed);
+                            mma_f16(ca, nib_even(ua0), nib_even(ua1), nib_odd(ua0), nib_odd(ua1), qa.z, qa.w);
+                            mma_f16(cb, nib_even(ub0), nib_even(ub1), nib_odd(ub0), nib_odd(ub1), qa.z, qa.w);
+                            const float a0f = (j & 1) ? fa0[j >> 1].y : fa0[j >> 1].x, a1f = (j & 1) ? fa1[j >> 1].y : fa1[j >> 1].x;
+                            const float b0f = (j & 1) ? fb0[j >> 1].y : fb0[j >> 1].x, b1f = (j & 1) ? fb1[j >> 1].y : fb1[j >> 1].x;
+                            sa[0] = fmaf(a0f, ca[0], sa[0]); sa[1] = fmaf(a0f, ca[1], sa[1]);
+                            sa[2] = fmaf(a1f, ca[2], sa[2]); sa[3] = fmaf(a1f, ca[3], sa[3]);
+                            sb[0] = fmaf(b0f, cb[0], sb[0]); sb[1] = fmaf(b0f, cb[1], sb[1]);
+                            sb[2] = fmaf(b1f, cb[2], sb[2]); sb[3] = fmaf(b1f, cb[3], sb[3]);
+                        }
+                    }
+                    // online softmax over the 32 tokens of the two pages, as below for one
+                    const float za0 = sa[0] * kLog2Scale, za1 = sa[1] * kLog2Scale, za2 = sa[2] * kLog2Scale, za3 = sa[3] * kLog2Scale;
+                    const float zb0 = sb[0] * kLog2Scale, zb1 = sb[1] * kLog2Scale, zb2 = sb[2] * kLog2Scale, zb3 = sb[3] * kLog2Scale;
+                    float ta = fmaxf(fmaxf(za0, za2), fmaxf(zb0, zb2)), tb = fmaxf(fmaxf(za1, za3), fmaxf(zb1, zb3));
+                    if (__any_sync(0xffffffffu, ta > m_a + kSlack || tb > m_b + kSlack)) {
+#pragma unroll
+                        for (int d = 4; d < 32; d <<= 1) {
+                            ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, d));
+                            tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, d));
+                        }
+                        const float mna = fmaxf(m_a, ta), mnb = fmaxf(m_b, tb);
+                        const float fa = mna == -INFINITY ? 1.f : ex2(m_a - mna), fb = mnb == -INFINITY ? 1.f : ex2(m_b - mnb);
+#pragma unroll
+                        for (int m = 0; m < 8; m++) { acc[m][0] *= fa; acc[m][2] *= fa; acc[m][1] *= fb; acc[m][3] *= fb; }
+                        l_a *= fa; l_b *= fb;
+                        m_a = mna; m_b = mnb;
+                    }
+                    const float pa0 = ex2(za0 - m_a), pa1 = ex2(za1 - m_b), pa2 = ex2(za2 - m_a), pa3 = ex2(za3 - m_b);
+                    const float pb0 = ex2(zb0 - m_a), pb1 = ex2(zb1 - m_b), pb2 = ex2(zb2 - m_a), pb3 = ex2(zb3 - m_b);
+                    l_a += (pa0 + pa2) + (pb0 + pb2);
+                    l_b += (pa1 + pa3) + (pb1 + pb3);
+                    pv_low4(st, 16u, pa0, pa1, pa2, pa3);
+                    pv_low4(st_b, 16u, pb0, pb1, pb2, pb3);
+                    ++page;          // (the loop's own increment counts the second page)
+                    continue;
+                }
+            }
 
             float sc[4] = {0.f, 0.f, 0.f, 0.f};
             if (is_high) {
@@ -827,42 +947,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                     }
                 }
             } else if (kHasLow) {
-                const uint32_t vb = st + kLowHalfBytes;
-                const uint4 v0 = lds128(vb + lane * 16);        // tokens 2t, 2t+1
-                const uint4 v1 = lds128(vb + 512 + lane * 16);  // tokens 2t+8, 2t+9
-                uint2 vs0 = lds64(vb + kLowCodesBytes + g * 8);
-                uint2 vs1 = lds64(vb + kLowCodesBytes + (g + 8) * 8);
-                w.release();   // everything of this stage is in registers now
-                if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
-                    if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
-                    if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
-                }
-                const uint32_t c0[4] = {v0.x, v0.y, v0.z, v0.w}, c1[4] = {v1.x, v1.y, v1.z, v1.w};
-                const uint32_t p01 = pack_f16(p0, p1), p23 = pack_f16(p2, p3);
-#pragma unroll
-                for (int v = 0; v < 2; v++) {
-                    // B columns 0-3: heads x group 2v, columns 4-7: heads x group 2v + 1
-                    const uint32_t s0b = hmul2(prmt(v ? vs0.y : vs0.x, 0u, bsel), down);
-                    const uint32_t s1b = hmul2(prmt(v ? vs1.y : vs1.x, 0u, bsel), down);
-                    const uint32_t b0 = movmatrix_trans(hmul2(p01, s0b)), b1 = movmatrix_trans(hmul2(p23, s1b));
-#pragma unroll
-                    for (int qq = 0; qq < 2; qq++) {
-                        const int q = 2 * v + qq;
-                        const uint32_t e0 = c0[q] >> 8, e1 = c1[q] >> 8;
-                        uint32_t a[2][4];
-                        a[0][0] = hsub2(nib_even(c0[q]), 0x64086408u);               // (1024 + code) - 1032
-                        a[0][1] = hfma2(nib_odd(c0[q]), 0x2C002C00u, 0xD480D480u);   // (1024 + 16 code) / 16 - 72
-                        a[0][2] = hsub2(nib_even(e0), 0x64086408u);
-                        a[0][3] = hfma2(nib_odd(e0), 0x2C002C00u, 0xD480D480u);
-                        a[1][0] = hsub2(nib_even(c1[q]), 0x64086408u);
-                        a[1][1] = hfma2(nib_odd(c1[q]), 0x2C002C00u, 0xD480D480u);
-                        a[1][2] = hsub2(nib_even(e1), 0x64086408u);
-                        a[1][3] = hfma2(nib_odd(e1), 0x2C002C00u, 0xD480D480u);
-#pragma unroll
-                        for (int r = 0; r < 2; r++)
-                            mma_f16(acc[2 * q + r], a[0][2 * r], a[0][2 * r + 1], a[1][2 * r], a[1][2 * r + 1], b0, b1);
-                    }
-                }
+                pv_low4(st, n_valid, p0, p1, p2, p3);
             }
         }
         // A wait ran out: the status word says so and the results of the call are void.  This warp's partials of
