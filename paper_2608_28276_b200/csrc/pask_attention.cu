@@ -351,7 +351,6 @@ struct Pipe {
     const uint8_t *base_high, *base_low;   // pool + this warp's head offset
     uint32_t stride_high, stride_low;      // page size in bytes
     uint32_t low_two, low_job_bytes;       // 8-bit LOW pages come as two jobs (K half, V half) of low_job_bytes each
-    uint32_t lim_high, lim_low;            // pages the two pools hold: an id beyond them is refused, not dereferenced
     uint32_t *status;         // the cache's device status word
     long long wait_cycles;    // bound of one wait
     uint32_t surplus;         // bytes the next copy announces beyond what it brings (wait-limit test; else 0)
@@ -370,19 +369,23 @@ struct Pipe {
     bool dead;
 
     // Issue the next job into stage p_stage.  Warp-uniform.
-    __device__ __forceinline__ void produce() {
+    // (`c`: the kernel's own parameter block -- what the check below reads from it costs no registers.)
+    __device__ __forceinline__ void produce(const DevCache &c) {
         if (p_pos == p_end) return;
         if (p_pos - pw_base >= 32u) {
             pw_base = p_pos;
-            pw_entry = p_pos + lane < p_end ? __ldg(order + p_pos + lane) : 0u;
+            uint32_t e = p_pos + lane < p_end ? __ldg(order + p_pos + lane) : 0u;
+            // A page id beyond its pool is never expected (a plan somebody overwrote): flag it and read page 0
+            // instead.  Checked here, by the lane that fetches the entry, once per 32 pages -- not per job.
+            if ((e & kOrderIdMask) >= ((e & kOrderHigh) ? c.high_limit : c.cap_low)) {
+                atomicOr(status, PASK_DEV_INTERNAL);
+                e &= ~kOrderIdMask;
+            }
+            pw_entry = e;
         }
         const uint32_t entry = __shfl_sync(0xffffffffu, pw_entry, (int)(p_pos - pw_base));
-        uint32_t id = entry & kOrderIdMask;
+        const uint32_t id = entry & kOrderIdMask;
         const bool is_high = entry & kOrderHigh;
-        if (id >= (is_high ? lim_high : lim_low)) {     // never expected (a plan somebody overwrote): flag it, read page 0
-            if (lane == 0) atomicOr(status, PASK_DEV_INTERNAL);
-            id = 0;
-        }
         const uint8_t *src = is_high ? base_high + (size_t)id * stride_high + p_sub * kHighTileBytes
                                      : base_low + (size_t)id * stride_low + p_sub * low_job_bytes;
         const uint32_t bytes = is_high ? kHighTileBytes : low_job_bytes;
@@ -425,11 +428,11 @@ struct Pipe {
         return ring + stage * kStageBytes;
     }
     // All lanes are done reading the oldest stage: hand it back to the producer.
-    __device__ __forceinline__ void release() {
+    __device__ __forceinline__ void release(const DevCache &c) {
         __syncwarp();
         outstanding--;
         if (++c_stage == kStages) { c_stage = 0; c_parity ^= 1u; }
-        if (!dead) produce();
+        if (!dead) produce(c);
     }
 };
 
@@ -506,8 +509,6 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     w.stride_low = c.low_page_bytes;
     w.low_two = kLow == 8;
     w.low_job_bytes = kLow == 8 ? kLow8HalfBytes : kLow == 2 ? kLow2HeadBytes : kLowHeadBytes;
-    w.lim_high = c.high_limit;
-    w.lim_low = c.cap_low;
     w.status = c.ctrl + kCtrlStatus;
     w.wait_cycles = p.wait_cycles;
     w.surplus = p.overpost;
@@ -528,7 +529,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncwarp();
-    for (int i = 0; i < kStages; i++) w.produce();
+    for (int i = 0; i < kStages; i++) w.produce(c);
     if (p.early) {
         pdl_wait();
         pdl_launch_dependents();   // (the append that runs beside this kernel must not start before this wait is over)
@@ -632,7 +633,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
             const uint4 v1 = lds128(vb + 512 + lane * 16);  // tokens 2t+8, 2t+9
             uint2 vs0 = lds64(vb + kLowCodesBytes + g * 8);
             uint2 vs1 = lds64(vb + kLowCodesBytes + (g + 8) * 8);
-            w.release();   // everything of this stage is in registers now
+            w.release(c);   // everything of this stage is in registers now
             if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
                 if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
                 if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
@@ -750,7 +751,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 }
 #pragma unroll
                 for (int i = 0; i < 4; i++) sc[i] += sc2[i];
-                w.release();
+                w.release(c);
             } else if (kLow == 8) {
                 // ---- QK^T over 8-bit K codes: per 32-dim group two k-chunks, A = 1024 + code by byte permutes
                 const uint2 ks0 = lds64(st + kLow8CodesBytes + g * 8);
@@ -760,7 +761,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 uint4 kw[4];
 #pragma unroll
                 for (int j = 0; j < 4; j++) kw[j] = lds128(st + j * 512 + lane * 16);
-                w.release();
+                w.release(c);
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
                     const uint2 qa = lds64(scratch + (2 * j) * 128 + (g & 3) * 32 + t * 8);
@@ -882,7 +883,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                         mma_bf16(acc[4 * e + r], a0, a1, a2, a3, bl0, bl1);
                     }
                 }
-                w.release();
+                w.release(c);
             } else if (kLow == 8) {
                 // ---- P.V over 8-bit V codes: the V half is a job of its own
                 const uint32_t p01 = pack_f16(p0, p1), p23 = pack_f16(p2, p3);
@@ -893,7 +894,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 for (int q = 0; q < 4; q++) vw[q] = lds128(st + q * 512 + lane * 16);   // group q: tiles r = 0 (x, y) and 1 (z, w)
                 uint2 vs0 = lds64(st + kLow8CodesBytes + g * 8);
                 uint2 vs1 = lds64(st + kLow8CodesBytes + (g + 8) * 8);
-                w.release();
+                w.release(c);
                 if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
                     if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
                     if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
@@ -923,7 +924,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 const uint4 vq = lds128(vb2 + lane * 16);        // byte 0: tokens 2t, 2t+1; byte 1: tokens 2t+8, 2t+9
                 uint2 vs0 = lds64(vb2 + kLow2CodesBytes + g * 8);
                 uint2 vs1 = lds64(vb2 + kLow2CodesBytes + (g + 8) * 8);
-                w.release();   // everything of this stage is in registers now
+                w.release(c);   // everything of this stage is in registers now
                 if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
                     if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
                     if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
