@@ -43,6 +43,7 @@ namespace {
 
 constexpr int kStages = 3;
 constexpr int kStageBytes = 4096;
+constexpr int kBarBytesPerWarp = 40;          // kStages mbarriers (8 bytes each), then kStages entry words (4 bytes each)
 constexpr int kMaxWarps = 8;
 constexpr int kScratchBytes = 1152;              // per warp: fp16 query fragments (1024) + accumulator seeds (128)
 constexpr int kPlanThreads = 256;
@@ -95,6 +96,10 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, long 
         if (clock64() - t0 > limit) return false;
     }
 }
+// adds `bytes` to the barrier's pending transaction count without arriving
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
 // takes `bytes` off the barrier's pending transaction count, as the arrival of that many copied bytes would
 __device__ __forceinline__ void mbar_complete_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -103,16 +108,15 @@ __device__ __forceinline__ void mbar_complete_tx(uint32_t bar, uint32_t bytes) {
 // issued by one elected lane of a converged warp
 // (predicated, no divergent branch); the same lane leaves `word` at shared address `note`
 // The copy carries an L2 evict-first hint: every page is read exactly once per call.
-// `announced` is the byte count the barrier is told to expect: `bytes`, except in the wait-limit test.
-__device__ __forceinline__ void issue_bulk_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t announced, uint32_t bar,
-                                                   uint32_t note, uint32_t word, uint64_t policy) {
+__device__ __forceinline__ void issue_bulk_elected(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint32_t note,
+                                                   uint32_t word, uint64_t policy) {
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
         "elect.sync _|P, 0xffffffff;\n\t"
         "@P st.shared.u32 [%4], %5;\n\t"
-        "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %7;\n\t"
+        "@P mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %2;\n\t"
         "@P cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %6;\n\t}"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "r"(note), "r"(word), "l"(policy), "r"(announced)
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "r"(note), "r"(word), "l"(policy)
         : "memory");
 }
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {
@@ -346,18 +350,17 @@ attn_plan_kernel(DevCache c, int layer, int n_seqs, const int32_t *__restrict__ 
 // copy per job (HIGH page: K tile, then V tile; LOW page: K and V halves together), leaving the
 // page's list entry next to the stage's mbarrier; the consumer side waits for the jobs in the same
 // order and reads the entry back, so it needs no bookkeeping of its own.
+// Whatever the kernel was given as a parameter (pools, strides, the order list, the wait limit) is read from the
+// parameter block where it is used, not copied into the warp's state: every register the pipeline holds for the
+// whole loop is one the MMA operands do not get.
+template <int kLow>
 struct Pipe {
-    const uint32_t *order;    // the page-order list
-    const uint8_t *base_high, *base_low;   // pool + this warp's head offset
-    uint32_t stride_high, stride_low;      // page size in bytes
-    uint32_t low_two, low_job_bytes;       // 8-bit LOW pages come as two jobs (K half, V half) of low_job_bytes each
-    uint32_t *status;         // the cache's device status word
-    long long wait_cycles;    // bound of one wait
-    uint32_t surplus;         // bytes the next copy announces beyond what it brings (wait-limit test; else 0)
-    uint32_t owed;            // such bytes still pending on the barrier of stage 0
+    static constexpr bool kLowTwo = kLow == 8;     // 8-bit LOW pages come as two jobs (K half, V half)
+    static constexpr uint32_t kLowJobBytes = kLow == 8 ? kLow8HalfBytes : kLow == 2 ? kLow2HeadBytes : kLowHeadBytes;
+    static constexpr uint32_t kLowHeadStride = kLow == 8 ? kLow8HeadBytes : kLow == 2 ? kLow2HeadBytes : kLowHeadBytes;
     uint64_t policy;          // L2 cache policy of the bulk copies
-    int lane;
-    uint32_t ring, bars, meta;   // shared-space addresses of this warp's stages, mbarriers and entry words
+    int lane, warp;
+    uint32_t ring, bars;      // shared-space addresses of this warp's stages and of its mbarriers (the entry words follow those)
     // producer
     uint32_t p_pos, p_end;    // next position and end of the CTA's range
     uint32_t p_sub;           // 0: K tile next, 1: V tile next (HIGH pages)
@@ -369,16 +372,16 @@ struct Pipe {
     bool dead;
 
     // Issue the next job into stage p_stage.  Warp-uniform.
-    // (`c`: the kernel's own parameter block -- what the check below reads from it costs no registers.)
-    __device__ __forceinline__ void produce(const DevCache &c) {
+    __device__ __forceinline__ void produce(const AttnParams &p) {
+        const DevCache &c = p.c;
         if (p_pos == p_end) return;
         if (p_pos - pw_base >= 32u) {
             pw_base = p_pos;
-            uint32_t e = p_pos + lane < p_end ? __ldg(order + p_pos + lane) : 0u;
+            uint32_t e = p_pos + lane < p_end ? __ldg(p.ws.order + p_pos + lane) : 0u;
             // A page id beyond its pool is never expected (a plan somebody overwrote): flag it and read page 0
             // instead.  Checked here, by the lane that fetches the entry, once per 32 pages -- not per job.
             if ((e & kOrderIdMask) >= ((e & kOrderHigh) ? c.high_limit : c.cap_low)) {
-                atomicOr(status, PASK_DEV_INTERNAL);
+                atomicOr(c.ctrl + kCtrlStatus, PASK_DEV_INTERNAL);
                 e &= ~kOrderIdMask;
             }
             pw_entry = e;
@@ -386,53 +389,46 @@ struct Pipe {
         const uint32_t entry = __shfl_sync(0xffffffffu, pw_entry, (int)(p_pos - pw_base));
         const uint32_t id = entry & kOrderIdMask;
         const bool is_high = entry & kOrderHigh;
-        const uint8_t *src = is_high ? base_high + (size_t)id * stride_high + p_sub * kHighTileBytes
-                                     : base_low + (size_t)id * stride_low + p_sub * low_job_bytes;
-        const uint32_t bytes = is_high ? kHighTileBytes : low_job_bytes;
-        issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bytes + surplus, bars + p_stage * 8, meta + p_stage * 4, entry,
-                           policy);
-        owed += surplus;          // (only a warp's first copy, which goes to stage 0, ever announces a surplus)
-        surplus = 0;
+        const uint8_t *src = is_high ? c.pool_high + ((size_t)id * c.high_page_bytes + (uint32_t)warp * kHighHeadBytes + p_sub * kHighTileBytes)
+                                     : c.pool_low + ((size_t)id * c.low_page_bytes + (uint32_t)warp * kLowHeadStride + p_sub * kLowJobBytes);
+        const uint32_t bytes = is_high ? (uint32_t)kHighTileBytes : kLowJobBytes;
+        issue_bulk_elected(ring + p_stage * kStageBytes, src, bytes, bars + p_stage * 8, bars + kStages * 8 + p_stage * 4, entry, policy);
         p_stage = p_stage + 1 == kStages ? 0 : p_stage + 1;
         outstanding++;
-        const bool two = is_high || low_two;               // a HIGH page is two jobs, an 8-bit LOW page too
+        const bool two = is_high || kLowTwo;               // a HIGH page is two jobs, an 8-bit LOW page too
         const uint32_t page_done = two ? p_sub : 1u;
         p_sub = two ? p_sub ^ 1u : 0u;
         p_pos += page_done;
     }
 
-    // Wait for the oldest outstanding job; returns the shared address of its stage and the page's entry.
-    __device__ __forceinline__ uint32_t acquire(uint32_t &entry) {
-        const uint32_t bar = bars + c_stage * 8;
-        if (!mbar_try_wait(bar, c_parity)) {
-            if (dead || !mbar_wait_slow(bar, c_parity, wait_cycles)) {
-                if (!dead && lane == 0) atomicOr(status, PASK_DEV_TIMEOUT);
+    __device__ __forceinline__ void wait_for(const AttnParams &p, uint32_t bar, uint32_t parity) {
+        if (!mbar_try_wait(bar, parity)) {
+            if (dead || !mbar_wait_slow(bar, parity, p.wait_cycles)) {
+                if (!dead && lane == 0) atomicOr(p.c.ctrl + kCtrlStatus, PASK_DEV_TIMEOUT);
                 dead = true;
             }
         }
-        entry = lds32(meta + c_stage * 4);
+    }
+    // Wait for the oldest outstanding job; returns the shared address of its stage and the page's entry.
+    __device__ __forceinline__ uint32_t acquire(const AttnParams &p, uint32_t &entry) {
+        wait_for(p, bars + c_stage * 8, c_parity);
+        entry = lds32(bars + kStages * 8 + c_stage * 4);
         return ring + c_stage * kStageBytes;
     }
     // The same for the job after the oldest one, which stays the oldest (two stages are then held at once).
-    __device__ __forceinline__ uint32_t acquire_next(uint32_t &entry) {
+    __device__ __forceinline__ uint32_t acquire_next(const AttnParams &p, uint32_t &entry) {
         uint32_t stage = c_stage + 1, parity = c_parity;
         if (stage == kStages) { stage = 0; parity ^= 1u; }
-        const uint32_t bar = bars + stage * 8;
-        if (!mbar_try_wait(bar, parity)) {
-            if (dead || !mbar_wait_slow(bar, parity, wait_cycles)) {
-                if (!dead && lane == 0) atomicOr(status, PASK_DEV_TIMEOUT);
-                dead = true;
-            }
-        }
-        entry = lds32(meta + stage * 4);
+        wait_for(p, bars + stage * 8, parity);
+        entry = lds32(bars + kStages * 8 + stage * 4);
         return ring + stage * kStageBytes;
     }
     // All lanes are done reading the oldest stage: hand it back to the producer.
-    __device__ __forceinline__ void release(const DevCache &c) {
+    __device__ __forceinline__ void release(const AttnParams &p) {
         __syncwarp();
         outstanding--;
         if (++c_stage == kStages) { c_stage = 0; c_parity ^= 1u; }
-        if (!dead) produce(c);
+        if (!dead) produce(p);
     }
 };
 
@@ -501,23 +497,12 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     auto position_of = [&](uint32_t x, int s) -> uint32_t {   // first position at or after cost offset x, which lies in sequence s
         return s_page[s] + cut_at(x - s_cost[s], s_cost[s + 1] - s_cost[s], s_page[s + 1] - s_page[s]);
     };
-    Pipe w;
-    w.order = p.ws.order;
-    w.base_high = c.pool_high + (size_t)warp * kHighHeadBytes;
-    w.base_low = c.pool_low + (size_t)warp * (kLow == 8 ? kLow8HeadBytes : kLow == 2 ? kLow2HeadBytes : kLowHeadBytes);
-    w.stride_high = c.high_page_bytes;
-    w.stride_low = c.low_page_bytes;
-    w.low_two = kLow == 8;
-    w.low_job_bytes = kLow == 8 ? kLow8HalfBytes : kLow == 2 ? kLow2HeadBytes : kLowHeadBytes;
-    w.status = c.ctrl + kCtrlStatus;
-    w.wait_cycles = p.wait_cycles;
-    w.surplus = p.overpost;
-    w.owed = 0;
+    Pipe<kLow> w;
     w.policy = l2_evict_first_policy();
     w.lane = lane;
+    w.warp = warp;
     w.ring = smem_u32(s_ring + (size_t)warp * kStages * kStageBytes);
-    w.bars = smem_u32(s_bar + warp * kStages);
-    w.meta = smem_u32(s_bar) + kMaxWarps * kStages * 8 + warp * kStages * 4;   // after the 192 bytes of barriers
+    w.bars = smem_u32(s_bar) + warp * kBarBytesPerWarp;      // three mbarriers, then the three entry words
     w.p_pos = position_of(lo, s0);
     w.p_end = hi >= total ? s_page[n_seqs] : position_of(hi, seq_of(hi));
     w.p_sub = 0; w.pw_base = 0x80000000u; w.pw_entry = 0;
@@ -529,7 +514,13 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncwarp();
-    for (int i = 0; i < kStages; i++) w.produce(c);
+    // Wait-limit test only: the barrier of the warp's first job is told to expect more bytes than the copy brings.
+    const bool had_job = w.p_pos != w.p_end;
+    if (p.overpost && had_job) {
+        if (lane == 0) mbar_expect_tx(w.bars, p.overpost);
+        __syncwarp();
+    }
+    for (int i = 0; i < kStages; i++) w.produce(p);
     if (p.early) {
         pdl_wait();
         pdl_launch_dependents();   // (the append that runs beside this kernel must not start before this wait is over)
@@ -633,7 +624,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
             const uint4 v1 = lds128(vb + 512 + lane * 16);  // tokens 2t+8, 2t+9
             uint2 vs0 = lds64(vb + kLowCodesBytes + g * 8);
             uint2 vs1 = lds64(vb + kLowCodesBytes + (g + 8) * 8);
-            w.release(c);   // everything of this stage is in registers now
+            w.release(p);   // everything of this stage is in registers now
             if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
                 if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
                 if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
@@ -668,7 +659,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
 
         for (uint32_t page = 0; page < n_pages; ++page) {
             uint32_t entry;
-            uint32_t st = w.acquire(entry);
+            uint32_t st = w.acquire(p, entry);
             if (w.dead) break;
             const bool is_high = entry & kOrderHigh;
             const uint32_t n_valid = (((entry >> kOrderValidShift) - 1u) & 15u) + 1u;   // 0 in the entry means all 16
@@ -679,7 +670,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
             // maxima, and the query operands fetched once for both
             if (kLow == 4 && !is_high && n_valid == 16u && page + 1 < n_pages) {
                 uint32_t entry_b;
-                const uint32_t st_b = w.acquire_next(entry_b);
+                const uint32_t st_b = w.acquire_next(p, entry_b);
                 if (w.dead) break;
                 if (!(entry_b & kOrderHigh) && ((entry_b >> kOrderValidShift) & 15u) == 0u) {
                     float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
@@ -751,7 +742,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 }
 #pragma unroll
                 for (int i = 0; i < 4; i++) sc[i] += sc2[i];
-                w.release(c);
+                w.release(p);
             } else if (kLow == 8) {
                 // ---- QK^T over 8-bit K codes: per 32-dim group two k-chunks, A = 1024 + code by byte permutes
                 const uint2 ks0 = lds64(st + kLow8CodesBytes + g * 8);
@@ -761,7 +752,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 uint4 kw[4];
 #pragma unroll
                 for (int j = 0; j < 4; j++) kw[j] = lds128(st + j * 512 + lane * 16);
-                w.release(c);
+                w.release(p);
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
                     const uint2 qa = lds64(scratch + (2 * j) * 128 + (g & 3) * 32 + t * 8);
@@ -861,7 +852,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 split_pair(p2 * down_f, p3 * down_f, h23, l23);
                 const uint32_t bh0 = movmatrix_trans(h01), bh1 = movmatrix_trans(h23);
                 const uint32_t bl0 = movmatrix_trans(l01), bl1 = movmatrix_trans(l23);
-                st = w.acquire(entry);
+                st = w.acquire(p, entry);
                 if (w.dead) break;
 #pragma unroll
                 for (int e = 0; e < 2; e++) {
@@ -883,18 +874,18 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                         mma_bf16(acc[4 * e + r], a0, a1, a2, a3, bl0, bl1);
                     }
                 }
-                w.release(c);
+                w.release(p);
             } else if (kLow == 8) {
                 // ---- P.V over 8-bit V codes: the V half is a job of its own
                 const uint32_t p01 = pack_f16(p0, p1), p23 = pack_f16(p2, p3);
-                st = w.acquire(entry);
+                st = w.acquire(p, entry);
                 if (w.dead) break;
                 uint4 vw[4];
 #pragma unroll
                 for (int q = 0; q < 4; q++) vw[q] = lds128(st + q * 512 + lane * 16);   // group q: tiles r = 0 (x, y) and 1 (z, w)
                 uint2 vs0 = lds64(st + kLow8CodesBytes + g * 8);
                 uint2 vs1 = lds64(st + kLow8CodesBytes + (g + 8) * 8);
-                w.release(c);
+                w.release(p);
                 if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
                     if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
                     if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
@@ -924,7 +915,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                 const uint4 vq = lds128(vb2 + lane * 16);        // byte 0: tokens 2t, 2t+1; byte 1: tokens 2t+8, 2t+9
                 uint2 vs0 = lds64(vb2 + kLow2CodesBytes + g * 8);
                 uint2 vs1 = lds64(vb2 + kLow2CodesBytes + (g + 8) * 8);
-                w.release(c);   // everything of this stage is in registers now
+                w.release(p);   // everything of this stage is in registers now
                 if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
                     if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
                     if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
@@ -982,14 +973,14 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
     // A wait gave up: copies may still be in flight towards this CTA's shared memory.  Give each
     // outstanding stage one more bounded wait before the CTA retires; the ring is not read again.
     if (w.dead) {
-        if (w.owed) {   // wait-limit test: bytes were announced that no copy brings; take them off, so that the
+        if (p.overpost && had_job) {   // wait-limit test: bytes were announced that no copy brings; take them off, so that the
                         // barrier completes exactly when the real copy has landed
-            if (lane == 0) mbar_complete_tx(w.bars, w.owed);
+            if (lane == 0) mbar_complete_tx(w.bars, p.overpost);
             __syncwarp();
         }
         while (w.outstanding > 0) {
             const uint32_t bar = w.bars + w.c_stage * 8;
-            if (!mbar_try_wait(bar, w.c_parity)) mbar_wait_slow(bar, w.c_parity, w.wait_cycles > 200000000LL ? w.wait_cycles : 200000000LL);
+            if (!mbar_try_wait(bar, w.c_parity)) mbar_wait_slow(bar, w.c_parity, p.wait_cycles > 200000000LL ? p.wait_cycles : 200000000LL);
             if (++w.c_stage == kStages) { w.c_stage = 0; w.c_parity ^= 1u; }
             w.outstanding--;
         }
