@@ -657,6 +657,62 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
             }
         };
 
+        // the same for a page of two-bit codes, and its scores (QK^T: one word per 32-dim group holds both token rows of
+        // this lane; byte 0: token g, byte 1: token g + 8)
+        auto qk_low2 = [&](uint32_t stage, float (&sc)[4]) {
+            const uint4 kq = lds128(stage + lane * 16);
+            const uint2 ks0 = lds64(stage + kLow2CodesBytes + g * 8);
+            const uint2 ks1 = lds64(stage + kLow2CodesBytes + (g + 8) * 8);
+            const uint32_t kwd[4] = {kq.x, kq.y, kq.z, kq.w};
+            const float2 f0[2] = {unpack_f16(ks0.x), unpack_f16(ks0.y)};
+            const float2 f1[2] = {unpack_f16(ks1.x), unpack_f16(ks1.y)};
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                const uint4 qa = lds128(scratch + j * 256 + (g & 3) * 64 + t * 16);
+                const uint4 seed = lds128(scratch + 1024 + ((t & 1) * 4 + j) * 16);
+                float cj[4];
+                const uint32_t x = kwd[j], y = x >> 8;
+                mma_f16_seed(cj, two_bit(x, 0), two_bit(y, 0), two_bit(x, 1), two_bit(y, 1), qa.x, qa.y, seed);
+                mma_f16(cj, two_bit(x, 2), two_bit(y, 2), two_bit(x, 3), two_bit(y, 3), qa.z, qa.w);
+                const float s0f = (j & 1) ? f0[j >> 1].y : f0[j >> 1].x;
+                const float s1f = (j & 1) ? f1[j >> 1].y : f1[j >> 1].x;
+                sc[0] = fmaf(s0f, cj[0], sc[0]);
+                sc[1] = fmaf(s0f, cj[1], sc[1]);
+                sc[2] = fmaf(s1f, cj[2], sc[2]);
+                sc[3] = fmaf(s1f, cj[3], sc[3]);
+            }
+        };
+        // P.V over 2-bit V codes: fields 0, 1 of a byte are rows g, g+8 of tile 2q, fields 2, 3 of tile 2q+1
+        auto pv_low2 = [&](uint32_t stage, uint32_t n_valid, float p0, float p1, float p2, float p3) {
+            const uint32_t vb2 = stage + kLow2HalfBytes;
+            const uint4 vq = lds128(vb2 + lane * 16);        // byte 0: tokens 2t, 2t+1; byte 1: tokens 2t+8, 2t+9
+            uint2 vs0 = lds64(vb2 + kLow2CodesBytes + g * 8);
+            uint2 vs1 = lds64(vb2 + kLow2CodesBytes + (g + 8) * 8);
+            w.release(p);   // everything of this stage is in registers now
+            if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
+                if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
+                if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
+            }
+            const uint32_t cw[4] = {vq.x, vq.y, vq.z, vq.w};
+            const uint32_t p01 = pack_f16(p0, p1), p23 = pack_f16(p2, p3);
+#pragma unroll
+            for (int v = 0; v < 2; v++) {
+                const uint32_t s0b = hmul2(prmt(v ? vs0.y : vs0.x, 0u, bsel), down);
+                const uint32_t s1b = hmul2(prmt(v ? vs1.y : vs1.x, 0u, bsel), down);
+                const uint32_t b0 = movmatrix_trans(hmul2(p01, s0b)), b1 = movmatrix_trans(hmul2(p23, s1b));
+#pragma unroll
+                for (int qq = 0; qq < 2; qq++) {
+                    const int q = 2 * v + qq;
+                    const uint32_t x = cw[q], y = x >> 8;
+                    // (1024 + 4^i code) / 4^i - (1024 / 4^i + 2) = code - 2, exact in fp16
+                    mma_f16(acc[2 * q], hsub2(two_bit(x, 0), 0x64026402u), hfma2(two_bit(x, 1), 0x34003400u, 0xDC08DC08u),
+                            hsub2(two_bit(y, 0), 0x64026402u), hfma2(two_bit(y, 1), 0x34003400u, 0xDC08DC08u), b0, b1);
+                    mma_f16(acc[2 * q + 1], hfma2(two_bit(x, 2), 0x2C002C00u, 0xD420D420u), hfma2(two_bit(x, 3), 0x24002400u, 0xCC80CC80u),
+                            hfma2(two_bit(y, 2), 0x2C002C00u, 0xD420D420u), hfma2(two_bit(y, 3), 0x24002400u, 0xCC80CC80u), b0, b1);
+                }
+            }
+        };
+
         for (uint32_t page = 0; page < n_pages; ++page) {
             uint32_t entry;
             uint32_t st = w.acquire(p, entry);
@@ -664,17 +720,20 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
             const bool is_high = entry & kOrderHigh;
             const uint32_t n_valid = (((entry >> kOrderValidShift) - 1u) & 15u) + 1u;   // 0 in the entry means all 16
 
-            // ---- two full four-bit pages in a row are taken together: two independent chains of loads, logic, MMAs
+            // ---- two full four-bit (or two-bit) pages in a row are taken together: two independent chains of loads, logic, MMAs
             // and exponentials for the four resident warps of a scheduler to interleave instead of one (the warp-level
             // MMA and the half-rate logic pipe leave an in-order warp waiting most of the time), one look at the running
             // maxima, and the query operands fetched once for both
-            if (kLow == 4 && !is_high && n_valid == 16u && page + 1 < n_pages) {
+            if ((kLow == 4 || kLow == 2) && !is_high && n_valid == 16u && page + 1 < n_pages) {
                 uint32_t entry_b;
                 const uint32_t st_b = w.acquire_next(p, entry_b);
                 if (w.dead) break;
                 if (!(entry_b & kOrderHigh) && ((entry_b >> kOrderValidShift) & 15u) == 0u) {
                     float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
-                    {
+                    if (kLow == 2) {
+                        qk_low2(st, sa);
+                        qk_low2(st_b, sb);
+                    } else {
                         const uint4 ka0 = lds128(st + lane * 16), ka1 = lds128(st + 512 + lane * 16);
                         const uint4 kb0 = lds128(st_b + lane * 16), kb1 = lds128(st_b + 512 + lane * 16);
                         const uint2 sa0 = lds64(st + kLowCodesBytes + g * 8), sa1 = lds64(st + kLowCodesBytes + (g + 8) * 8);
@@ -722,8 +781,13 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                     const float pb0 = ex2(zb0 - m_a), pb1 = ex2(zb1 - m_b), pb2 = ex2(zb2 - m_a), pb3 = ex2(zb3 - m_b);
                     l_a += (pa0 + pa2) + (pb0 + pb2);
                     l_b += (pa1 + pa3) + (pb1 + pb3);
-                    pv_low4(st, 16u, pa0, pa1, pa2, pa3);
-                    pv_low4(st_b, 16u, pb0, pb1, pb2, pb3);
+                    if (kLow == 2) {
+                        pv_low2(st, 16u, pa0, pa1, pa2, pa3);
+                        pv_low2(st_b, 16u, pb0, pb1, pb2, pb3);
+                    } else {
+                        pv_low4(st, 16u, pa0, pa1, pa2, pa3);
+                        pv_low4(st_b, 16u, pb0, pb1, pb2, pb3);
+                    }
                     ++page;          // (the loop's own increment counts the second page)
                     continue;
                 }
@@ -771,28 +835,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                     sc[3] = fmaf(s1f, cj[3], sc[3]);
                 }
             } else if (kLow == 2) {
-                // ---- QK^T over 2-bit K codes: one word per 32-dim group holds both token rows of this lane
-                const uint4 kq = lds128(st + lane * 16);
-                const uint2 ks0 = lds64(st + kLow2CodesBytes + g * 8);
-                const uint2 ks1 = lds64(st + kLow2CodesBytes + (g + 8) * 8);
-                const uint32_t kwd[4] = {kq.x, kq.y, kq.z, kq.w};
-                const float2 f0[2] = {unpack_f16(ks0.x), unpack_f16(ks0.y)};
-                const float2 f1[2] = {unpack_f16(ks1.x), unpack_f16(ks1.y)};
-#pragma unroll
-                for (int j = 0; j < 4; j++) {
-                    const uint4 qa = lds128(scratch + j * 256 + (g & 3) * 64 + t * 16);
-                    const uint4 seed = lds128(scratch + 1024 + ((t & 1) * 4 + j) * 16);
-                    float cj[4];
-                    const uint32_t x = kwd[j], y = x >> 8;      // byte 0: token g, byte 1: token g + 8
-                    mma_f16_seed(cj, two_bit(x, 0), two_bit(y, 0), two_bit(x, 1), two_bit(y, 1), qa.x, qa.y, seed);
-                    mma_f16(cj, two_bit(x, 2), two_bit(y, 2), two_bit(x, 3), two_bit(y, 3), qa.z, qa.w);
-                    const float s0f = (j & 1) ? f0[j >> 1].y : f0[j >> 1].x;
-                    const float s1f = (j & 1) ? f1[j >> 1].y : f1[j >> 1].x;
-                    sc[0] = fmaf(s0f, cj[0], sc[0]);
-                    sc[1] = fmaf(s0f, cj[1], sc[1]);
-                    sc[2] = fmaf(s1f, cj[2], sc[2]);
-                    sc[3] = fmaf(s1f, cj[3], sc[3]);
-                }
+                qk_low2(st, sc);
             } else if (kHasLow) {
                 const uint4 k0 = lds128(st + lane * 16);
                 const uint4 k1 = lds128(st + 512 + lane * 16);
@@ -910,34 +953,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) decode_attn_kernel(const __
                     }
                 }
             } else if (kLow == 2) {
-                // ---- P.V over 2-bit V codes: fields 0, 1 of a byte are rows g, g+8 of tile 2q, fields 2, 3 of tile 2q+1
-                const uint32_t vb2 = st + kLow2HalfBytes;
-                const uint4 vq = lds128(vb2 + lane * 16);        // byte 0: tokens 2t, 2t+1; byte 1: tokens 2t+8, 2t+9
-                uint2 vs0 = lds64(vb2 + kLow2CodesBytes + g * 8);
-                uint2 vs1 = lds64(vb2 + kLow2CodesBytes + (g + 8) * 8);
-                w.release(p);   // everything of this stage is in registers now
-                if (n_valid < 16u) {   // partial tail page: stale scales must not reach the MMA
-                    if ((uint32_t)g >= n_valid) vs0 = make_uint2(0, 0);
-                    if ((uint32_t)g + 8u >= n_valid) vs1 = make_uint2(0, 0);
-                }
-                const uint32_t cw[4] = {vq.x, vq.y, vq.z, vq.w};
-                const uint32_t p01 = pack_f16(p0, p1), p23 = pack_f16(p2, p3);
-#pragma unroll
-                for (int v = 0; v < 2; v++) {
-                    const uint32_t s0b = hmul2(prmt(v ? vs0.y : vs0.x, 0u, bsel), down);
-                    const uint32_t s1b = hmul2(prmt(v ? vs1.y : vs1.x, 0u, bsel), down);
-                    const uint32_t b0 = movmatrix_trans(hmul2(p01, s0b)), b1 = movmatrix_trans(hmul2(p23, s1b));
-#pragma unroll
-                    for (int qq = 0; qq < 2; qq++) {
-                        const int q = 2 * v + qq;
-                        const uint32_t x = cw[q], y = x >> 8;
-                        // (1024 + 4^i code) / 4^i - (1024 / 4^i + 2) = code - 2, exact in fp16
-                        mma_f16(acc[2 * q], hsub2(two_bit(x, 0), 0x64026402u), hfma2(two_bit(x, 1), 0x34003400u, 0xDC08DC08u),
-                                hsub2(two_bit(y, 0), 0x64026402u), hfma2(two_bit(y, 1), 0x34003400u, 0xDC08DC08u), b0, b1);
-                        mma_f16(acc[2 * q + 1], hfma2(two_bit(x, 2), 0x2C002C00u, 0xD420D420u), hfma2(two_bit(x, 3), 0x24002400u, 0xCC80CC80u),
-                                hfma2(two_bit(y, 2), 0x2C002C00u, 0xD420D420u), hfma2(two_bit(y, 3), 0x24002400u, 0xCC80CC80u), b0, b1);
-                    }
-                }
+                pv_low2(st, n_valid, p0, p1, p2, p3);
             } else if (kHasLow) {
                 pv_low4(st, n_valid, p0, p1, p2, p3);
             }
